@@ -1,0 +1,142 @@
+"""Seeded synthetic inputs shaped like the paper's workloads.
+
+This module holds input generators only: random weights, token ids, heavy-tailed gradient
+scores, index samples and activations.  It contains none of the method's arithmetic (no
+quantizer, no mask selection, no Philox/Gaussian perturbation, no forward pass), so the same
+arrays can be handed to the CUDA library and to an independent checker.
+
+Every generator draws from numpy.random.default_rng([seed, purpose, i]) so that streams with
+different purposes never overlap.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+PURPOSE_WEIGHTS = 0
+PURPOSE_MASK_BATCH = 1
+PURPOSE_TRAIN_BATCH = 2
+PURPOSE_SCORES = 3
+PURPOSE_INDICES = 4
+PURPOSE_ACTIVATION = 5
+PURPOSE_LABELS = 6
+PURPOSE_CODES = 7
+
+
+def rng(seed: int, purpose: int, i: int = 0) -> np.random.Generator:
+    return np.random.default_rng([int(seed), int(purpose), int(i)])
+
+
+def bf16_round(a) -> np.ndarray:
+    """fp32 array rounded to the nearest bf16-representable value (ties to even), still fp32."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    b = a.view(np.uint32).astype(np.uint64)
+    b = ((b + 0x7FFF + ((b >> 16) & 1)) >> 16) << 16
+    return b.astype(np.uint32).view(np.float32).reshape(a.shape)
+
+
+# name -> architecture dictionary (the decoder shapes of the paper's Section 4 models)
+MODEL_SHAPES = {
+    "tiny": dict(arch="llama", n_layers=2, d_model=256, n_heads=4, n_kv_heads=4, d_ff=1024,
+                 vocab=1024, max_pos=0, group=64, sz_fmt="f16", rho=1e-3),
+    "tiny_gqa": dict(arch="llama", n_layers=2, d_model=256, n_heads=4, n_kv_heads=2, d_ff=512,
+                     vocab=512, max_pos=0, group=0, sz_fmt="bf16", rho=1e-2),
+    "tiny_opt": dict(arch="opt", n_layers=2, d_model=256, n_heads=4, n_kv_heads=4, d_ff=1024,
+                     vocab=1024, max_pos=128, group=128, sz_fmt="bf16", rho=1e-3),
+    "llama2_7b": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, n_kv_heads=32,
+                      d_ff=11008, vocab=32000, max_pos=0, group=128, sz_fmt="bf16", rho=1e-3),
+    "mistral_7b": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, n_kv_heads=8,
+                       d_ff=14336, vocab=32000, max_pos=0, group=0, sz_fmt="bf16", rho=1e-2),
+    "opt_13b": dict(arch="opt", n_layers=40, d_model=5120, n_heads=40, n_kv_heads=40,
+                    d_ff=20480, vocab=50272, max_pos=2048, group=128, sz_fmt="bf16", rho=1e-3),
+}
+
+LLAMA_LINEARS = ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down")
+OPT_LINEARS = ("wq", "wk", "wv", "wo", "fc1", "fc2")
+
+
+def linear_names(shape: dict):
+    return LLAMA_LINEARS if shape["arch"] == "llama" else OPT_LINEARS
+
+
+def linear_shape(shape: dict, name: str):
+    d = shape["d_model"]
+    kv = shape["n_kv_heads"] * (d // shape["n_heads"])
+    ff = shape["d_ff"]
+    return {"wq": (d, d), "wk": (kv, d), "wv": (kv, d), "wo": (d, d), "w_gate": (ff, d),
+            "w_up": (ff, d), "w_down": (d, ff), "fc1": (ff, d), "fc2": (d, ff)}[name]
+
+
+def init_params(shape: dict, seed: int = 0, std: float = 0.02):
+    """Random-init weights N(0, std).  Returns (params, lin_W): params holds embeddings, LM
+    head, position table (bf16-representable fp32), norm gains (1) and biases; lin_W is
+    [layer][name] -> fp32 [N, K]."""
+    g = rng(seed, PURPOSE_WEIGHTS)
+    d, V = shape["d_model"], shape["vocab"]
+    opt = shape["arch"] == "opt"
+    params = {"embed": bf16_round(g.normal(0, std, (V, d))),
+              "lm_head": bf16_round(g.normal(0, std, (V, d))),
+              "final_norm": np.ones(d, np.float32)}
+    if opt:
+        params["pos"] = bf16_round(g.normal(0, std, (shape["max_pos"], d)))
+        params["final_norm_b"] = np.zeros(d, np.float32)
+    lin_W = []
+    for l in range(shape["n_layers"]):
+        params[f"l{l}.attn_norm"] = np.ones(d, np.float32)
+        params[f"l{l}.mlp_norm"] = np.ones(d, np.float32)
+        if opt:
+            params[f"l{l}.attn_norm_b"] = np.zeros(d, np.float32)
+            params[f"l{l}.mlp_norm_b"] = np.zeros(d, np.float32)
+        layer = {}
+        for nm in linear_names(shape):
+            N, K = linear_shape(shape, nm)
+            layer[nm] = g.normal(0, std, (N, K)).astype(np.float32)
+            if opt:
+                params[f"l{l}.{nm}_b"] = g.normal(0, std, N).astype(np.float32)
+        lin_W.append(layer)
+    return params, lin_W
+
+
+def token_batch(vocab: int, B: int, S: int, seed: int, purpose: int, i: int) -> np.ndarray:
+    """Uniform token ids, int32 [B, S]."""
+    return rng(seed, purpose, i).integers(0, vocab, (B, S), dtype=np.int32)
+
+
+def binary_labels(B: int, seed: int, i: int) -> np.ndarray:
+    return rng(seed, PURPOSE_LABELS, i).integers(0, 2, (B,), dtype=np.int32)
+
+
+def student_t_gradient(n: int, nu: float = 3.0, seed: int = 0, i: int = 0) -> np.ndarray:
+    """Heavy-tailed stand-in for a first-order gradient: g = N(0,1) / sqrt(chi2_nu / nu), fp32.
+    (A few coordinates carry most of the squared norm, as the paper observes for LLM linears.)"""
+    g = rng(seed, PURPOSE_SCORES, i)
+    t = g.standard_normal(n) / np.sqrt(g.chisquare(nu, n) / nu)
+    return t.astype(np.float32)
+
+
+def sorted_random_indices(n: int, k: int, seed: int = 0, i: int = 0) -> np.ndarray:
+    """k distinct indices in [0, n), ascending, int64 (without materialising a permutation)."""
+    g = rng(seed, PURPOSE_INDICES, i)
+    if k > n:
+        raise ValueError("k > n")
+    if k * 4 > n:
+        return np.sort(g.choice(n, size=k, replace=False)).astype(np.int64)
+    got = np.unique(g.integers(0, n, int(k * 1.1) + 16, dtype=np.int64))
+    while got.size < k:
+        got = np.unique(np.concatenate([got, g.integers(0, n, k, dtype=np.int64)]))
+    if got.size > k:
+        got = np.sort(g.choice(got, size=k, replace=False))
+    return got.astype(np.int64)
+
+
+def activation(M: int, K: int, seed: int = 0, i: int = 0) -> np.ndarray:
+    """x ~ N(0,1), bf16-representable fp32 [M, K]."""
+    return bf16_round(rng(seed, PURPOSE_ACTIVATION, i).standard_normal((M, K)).astype(np.float32))
+
+
+def gaussian_matrix(N: int, K: int, std: float, seed: int = 0, i: int = 0) -> np.ndarray:
+    return rng(seed, PURPOSE_WEIGHTS, 1000 + i).normal(0, std, (N, K)).astype(np.float32)
+
+
+def random_codes(N: int, K: int, seed: int = 0, i: int = 0) -> np.ndarray:
+    """Uniform random packed nibbles uint8 [N, K/2] (timing stand-in for a quantized tensor)."""
+    return rng(seed, PURPOSE_CODES, i).integers(0, 256, (N, K // 2), dtype=np.uint8)
