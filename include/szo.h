@@ -1,0 +1,204 @@
+/* szo.h - C ABI of the sensitive-sparse zeroth-order (ZO) fine-tuning step for sm_100a.
+ *
+ * The library implements the hot path of "Zeroth-Order Fine-Tuning of LLMs with Extreme
+ * Sparsity": the SPSA / ZO-SGD step restricted to k "sensitive" parameters, on linear layers
+ * whose weight is a frozen 4-bit quantized dense part plus k fp32 sparse values.
+ *
+ * Conventions (all entry points)
+ *   pointers   Device pointers unless the name ends in _host.  The caller owns every buffer it
+ *              passes; the library allocates only inside *_create (freed by *_destroy).
+ *              Buffers must be 16-byte aligned (SZO_ERR_ALIGNMENT otherwise).
+ *   stream     `void* stream` is a cudaStream_t (NULL = default stream).  Calls enqueue work and
+ *              return; none synchronises unless its comment says so.
+ *   errors     Arguments are validated on the host before any launch.  Return value 0 = SZO_OK,
+ *              negative = error; szo_last_error() gives a thread-local detail string.  Kernels
+ *              never trap: a bounded wait that expires inside a kernel is recorded in a device
+ *              status word readable with szo_device_status().
+ *   layouts    Matrices are row-major.  A linear has weight W[N,K] (out, in), input x[M,K],
+ *              output y[M,N].  int4 codes: uint8 [N,K/2], two codes per byte, even column in the
+ *              low nibble.  scales/zeros: 16-bit floats [N,K/G], G = group size along K.
+ *   determinism Same inputs give bitwise-same outputs (no floating-point atomics).
+ */
+#ifndef SZO_H_
+#define SZO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t szo_status;
+enum {
+  SZO_OK = 0,
+  SZO_ERR_INVALID_ARG = -1,
+  SZO_ERR_SHAPE = -2,
+  SZO_ERR_ALIGNMENT = -3,
+  SZO_ERR_UNSUPPORTED = -4,
+  SZO_ERR_WORKSPACE = -5,
+  SZO_ERR_CUDA = -6,
+  SZO_ERR_NONFINITE = -7,
+  SZO_ERR_TIMEOUT = -8
+};
+
+typedef enum { SZO_F32 = 0, SZO_BF16 = 1, SZO_F16 = 2 } szo_dtype;
+
+/* How szo_linear_fwd evaluates y = x Dequantize(Q)^T + x S^T (the paper's appendix
+ * "Implementation of Sparse Operations in Linear Layers" gives the two orders). */
+typedef enum {
+  SZO_MODE_AUTO = 0,          /* SPARSE_ADD */
+  SZO_MODE_SPARSE_ADD = 1,    /* DenseMM(SparseAdd(S, Dequantize(Q)), x): S is added to the
+                                 dequantised bf16 tile in shared memory before the tensor-core MMA */
+  SZO_MODE_SPMM = 2,          /* SparseAddMM(Dequantize(Q) x, S, x): tensor-core GEMM on the dense
+                                 part, then a row-bucketed CSR SpMM with fp32 values */
+  SZO_MODE_FP32_VALIDATE = 3  /* fp32 CUDA-core evaluation of the same expression (exact fp32
+                                 sparse term); slow, for checking losses and projected gradients */
+} szo_linear_mode;
+
+const char* szo_status_string(szo_status s);   /* static storage */
+const char* szo_last_error(void);              /* thread-local; valid until the next call */
+int szo_version(void);
+
+/* Reads and clears the device status word (0 = no kernel reported a problem, else a negative
+ * szo_status).  Synchronises the device. */
+szo_status szo_device_status(int32_t* status_host);
+
+/* ---- Quantizer Q for w_dense (Section 3.5, "Integration with quantization": the dense part is
+ * stored in 4 bits; the paper leaves the choice of quantizer open).  Uniform asymmetric,
+ * group-wise: for each row and each group of G consecutive columns, scale =
+ * round16((max-min)/15), zero = round16(min), code = clamp(rint((w-zero)/scale), 0, 15) (0 when
+ * scale == 0), IEEE fp32, ties to even.
+ *   W        w_dtype [N,K] (SZO_F32 or SZO_BF16)      codes   uint8 [N,K/2]
+ *   scales, zeros  sz_dtype [N,K/G] (SZO_BF16 or SZO_F16)
+ * Requires K % G == 0, G % 2 == 0.  Non-finite weights are not detected. */
+szo_status szo_quantize(const void* W, szo_dtype w_dtype, int64_t N, int64_t K, int32_t G,
+                        szo_dtype sz_dtype, uint8_t* codes, void* scales, void* zeros, void* stream);
+
+/* ---- Sensitive parameter mask (Definition 3: the mask with k nonzeros that maximises
+ * ||m (.) grad f||^2, i.e. the k largest squared-gradient scores).  Ties go to the lowest index;
+ * idx_out[k] is ascending.  Two-phase: call with workspace == NULL to obtain *workspace_bytes,
+ * then again with a workspace of at least that size.  Cold path: the second call synchronises the
+ * stream and returns SZO_ERR_NONFINITE if any score is NaN (idx_out is then unspecified).
+ *   scores  fp32 [n]      idx_out  int64 [k]      0 <= k <= n */
+szo_status szo_select_mask(const float* scores, int64_t n, int64_t k, int64_t* idx_out,
+                           void* workspace, size_t* workspace_bytes, void* stream);
+
+/* ---- Sparse perturbation (Definition 4, zbar = z (.) m_k; Section 3.4 update rule on w_sparse;
+ * Section 2.1 seed trick: z is regenerated, never stored).
+ *   S_out[j] = fma(scale, z_j, S_in[j]),  z_j = Gaussian(Philox4x32-10(key = seed,
+ *   counter = (idx_base + idx[j], step))): Box-Muller on the top 24 bits of words 0 and 1.
+ * idx[k] int64, tensor-local flat indices; idx_base makes them global over all linear
+ * parameters.  S_out may alias S_in.  Entries outside idx are never touched. */
+szo_status szo_perturb(const float* S_in, float* S_out, const int64_t* idx, int64_t k,
+                       int64_t idx_base, uint64_t seed, uint64_t step, float scale, void* stream);
+
+/* ---- Projected gradient (Definition 1, SPSA): *g_dev = (*f_plus_dev - *f_minus_dev) / (2 eps),
+ * fp64, all on the device. */
+szo_status szo_projected_gradient(const double* f_plus_dev, const double* f_minus_dev, float eps,
+                                  double* g_dev, void* stream);
+
+/* ---- ZO-SGD update (Definition 2 with Definition 4): S[j] = fma(-(float)(lr*g), z_j, S[j]) with
+ * g as above and the same z as szo_perturb for (seed, step).  The losses are read on the device. */
+szo_status szo_update(float* S, const int64_t* idx, int64_t k, int64_t idx_base, uint64_t seed,
+                      uint64_t step, float lr, const double* f_plus_dev, const double* f_minus_dev,
+                      float eps, void* stream);
+
+/* ---- Decomposed linear layer (Section 3.4: w = w_sparse + w_dense; appendix on sparse
+ * operations: y = x Dequantize(Q(w_dense))^T + x w_sparse^T).
+ * A plan owns only derived, immutable data (kernel-layout scale/zero table, tile buckets and
+ * row pointers of idx, tensor maps); the caller's codes, scales, zeros, idx and bias must
+ * outlive it.  G == 0 means a dense bf16 weight [N,K] instead of codes (scales/zeros NULL).
+ * Requires K % 64 == 0 and, for G > 0, G % 32 == 0.  idx[nnz] ascending flat indices n*K + c.
+ * bias fp32 [N] or NULL.  szo_linear_create synchronises the stream. */
+typedef struct szo_linear szo_linear_t;
+szo_status szo_linear_create(szo_linear_t** out, int64_t N, int64_t K, int32_t G,
+                             const void* codes_or_bf16_W, const void* scales, const void* zeros,
+                             szo_dtype sz_dtype, const int64_t* idx, int64_t nnz, const float* bias,
+                             void* stream);
+/* x: x_dtype [M,K] (SZO_BF16; SZO_F32 also accepted in SZO_MODE_FP32_VALIDATE);
+ * S_pert: fp32 [nnz] current (already perturbed) sparse values; y: y_dtype [M,N] (SZO_BF16 or
+ * SZO_F32).  workspace: at least szo_linear_workspace_bytes(plan, M, mode) bytes (may be NULL
+ * when that is 0). */
+szo_status szo_linear_fwd(const szo_linear_t* plan, const void* x, szo_dtype x_dtype, int64_t M,
+                          const float* S_pert, void* y, szo_dtype y_dtype, int32_t mode,
+                          void* workspace, size_t workspace_bytes, void* stream);
+size_t szo_linear_workspace_bytes(const szo_linear_t* plan, int64_t M, int32_t mode);
+void szo_linear_destroy(szo_linear_t* plan);
+
+/* ---- Whole loss path and ZO step on one GPU (Definition 1 evaluates the loss twice per step;
+ * Section 4 names the decoder families).  arch 0: RMSNorm, rotary positions, SiLU-gated MLP
+ * (Llama/Mistral; grouped-query attention when n_kv_heads < n_heads); arch 1: LayerNorm, learned
+ * positions, biases, ReLU MLP (OPT).  Linear order within a layer: arch 0: q,k,v,o,gate,up,down;
+ * arch 1: q,k,v,o,fc1,fc2.  The flat parameter index that keys z runs over the linears in model
+ * order, row-major inside each. */
+typedef struct {
+  int32_t arch;
+  int32_t n_layers, d_model, n_heads, n_kv_heads, d_ff, vocab, max_pos;
+  float norm_eps, rope_base;
+  int32_t group;       /* int4 group size; 0 = dense bf16 linears */
+  int32_t sz_dtype;    /* szo_dtype of scales/zeros */
+  int32_t act_dtype;   /* SZO_BF16 (tensor-core path) or SZO_F32 (validation path) */
+  int32_t linear_mode; /* szo_linear_mode used by every linear */
+  int32_t loss_kind;   /* 0: mean next-token cross-entropy over B*(S-1) positions;
+                          1: 2-way cross-entropy over two candidate ids at the last position */
+  int32_t max_batch, max_seq;
+} szo_model_config;
+
+typedef struct {
+  const void* codes;     /* uint8 [N,K/2], or bf16 [N,K] when group == 0 */
+  const void* scales;    /* sz_dtype [N,K/G] or NULL */
+  const void* zeros;
+  const int64_t* idx;    /* [nnz] ascending tensor-local flat indices */
+  int64_t nnz;
+  const float* bias;     /* fp32 [N] or NULL */
+} szo_linear_weights;
+
+typedef struct {
+  const float* attn_norm_g; const float* attn_norm_b;   /* fp32 [d]; *_b NULL for arch 0 */
+  const float* mlp_norm_g;  const float* mlp_norm_b;
+  szo_linear_weights lin[7];
+} szo_layer_weights;
+
+typedef struct {
+  const void* embed;     /* bf16 [vocab, d] */
+  const void* pos;       /* bf16 [max_pos, d] (arch 1) or NULL */
+  const void* lm_head;   /* bf16 [vocab, d] */
+  const float* final_norm_g; const float* final_norm_b;
+} szo_model_weights;
+
+typedef struct szo_model szo_model_t;
+/* layers_host: host array of n_layers entries holding device pointers.  S_all: fp32 [k_total],
+ * the trainable sparse values of all linears concatenated in model order (the only mutable
+ * state; caller-owned, updated in place by szo_model_zo_step).  Synchronises the stream. */
+szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg,
+                            const szo_model_weights* top, const szo_layer_weights* layers_host,
+                            float* S_all, void* stream);
+int64_t szo_model_k_total(const szo_model_t* m);
+/* Global flat indices int64 [k_total] of the sparse entries (device pointer owned by the model). */
+const int64_t* szo_model_gidx(const szo_model_t* m);
+/* tokens int32 [B,S]; labels int32 [B] in {0,1} and cand int32 [2] for loss_kind 1 (else NULL);
+ * S_vals fp32 [k_total] values to evaluate at (NULL = the model's S_all); *loss_dev fp64. */
+szo_status szo_model_loss(szo_model_t* m, const int32_t* tokens, const int32_t* labels,
+                          const int32_t* cand, int32_t B, int32_t S, const float* S_vals,
+                          double* loss_dev, void* stream);
+/* One step in the seed trick's in-place order: S += eps z; f+; S -= 2 eps z; f-; S += eps z;
+ * g = (f+ - f-)/(2 eps); S -= lr g z.  Outputs are device scalars (fp64); no host read-back. */
+szo_status szo_model_zo_step(szo_model_t* m, const int32_t* tokens, const int32_t* labels,
+                             const int32_t* cand, int32_t B, int32_t S, uint64_t seed,
+                             uint64_t step, float eps, float lr, double* f_plus_dev,
+                             double* f_minus_dev, double* g_dev, void* stream);
+/* Same step through HOST buffers: copies tokens (and labels, cand) to the device, runs the step
+ * and copies (f+, f-, g) back into out3_host[3]; synchronises the stream. */
+szo_status szo_model_zo_step_host(szo_model_t* m, const int32_t* tokens_host,
+                                  const int32_t* labels_host, const int32_t* cand_host, int32_t B,
+                                  int32_t S, uint64_t seed, uint64_t step, float eps, float lr,
+                                  double* out3_host, void* stream);
+/* Number of kernel launches the last szo_model_zo_step on this model enqueued. */
+int64_t szo_model_last_launches(const szo_model_t* m);
+void szo_model_destroy(szo_model_t* m);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SZO_H_ */

@@ -1,0 +1,70 @@
+// Shared host-side helpers of the szo library: error reporting, argument checks, and the
+// declarations of the internal launchers that the model driver calls directly.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <cstdarg>
+#include <cstdint>
+#include <cstdio>
+
+#include "../../include/szo.h"
+
+namespace szo {
+
+// Thread-local detail string behind szo_last_error().
+char* last_error_buffer();
+szo_status fail(szo_status code, const char* fmt, ...);
+
+// Device status word (one per device, allocated on first use on the current device).
+int32_t* device_status_word();
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t dtype_size(int dt) { return dt == SZO_F32 ? 4 : 2; }
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline size_t round_up(size_t a, size_t b) { return (a + b - 1) / b * b; }
+
+#define SZO_CHECK_CUDA(expr)                                                              \
+  do {                                                                                    \
+    cudaError_t e__ = (expr);                                                             \
+    if (e__ != cudaSuccess)                                                               \
+      return ::szo::fail(SZO_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e__));  \
+  } while (0)
+
+#define SZO_CHECK_LAUNCH(name)                                                            \
+  do {                                                                                    \
+    cudaError_t e__ = cudaGetLastError();                                                 \
+    if (e__ != cudaSuccess)                                                               \
+      return ::szo::fail(SZO_ERR_CUDA, "launch of %s failed: %s", name,                   \
+                         cudaGetErrorString(e__));                                        \
+  } while (0)
+
+#define SZO_REQUIRE(cond, code, ...)                    \
+  do {                                                  \
+    if (!(cond)) return ::szo::fail(code, __VA_ARGS__); \
+  } while (0)
+
+#define SZO_TRY(expr)                    \
+  do {                                   \
+    szo_status s__ = (expr);             \
+    if (s__ != SZO_OK) return s__;       \
+  } while (0)
+
+// Launch counter used by the model to report how many kernels one step enqueued.
+extern thread_local int64_t g_launch_count;
+inline void count_launch(int n = 1) { g_launch_count += n; }
+
+// Scale of a sparse axpy pass: a host value, or -(float)(lr * (f+ - f-) / (2 eps)) formed on
+// the device from the two losses (when f_plus != nullptr).
+struct ScaleArg {
+  float scale;
+  float lr, eps;
+  const double* f_plus;
+  const double* f_minus;
+};
+szo_status launch_sparse_axpy(const float* S_in, float* S_out, const int64_t* idx, int64_t k,
+                              int64_t idx_base, uint64_t seed, uint64_t step, ScaleArg sa,
+                              cudaStream_t st);
+
+}  // namespace szo

@@ -1,0 +1,146 @@
+// Sparse perturb / restore / update passes of the ZO step and the projected gradient.
+//
+// Definition 4 (sensitive sparse ZO-SGD) perturbs and updates only the k masked coordinates; the
+// Section 3.4 decomposition makes them a contiguous fp32 vector S.  z is regenerated from a
+// counter-based generator (Section 2.1 seed trick) keyed by (seed, step, global parameter index):
+// Philox4x32-10 (Salmon et al., SC'11) followed by the Box-Muller cosine branch.
+#include "common.cuh"
+
+namespace szo {
+
+constexpr uint32_t kPhiloxM0 = 0xD2511F53u;
+constexpr uint32_t kPhiloxM1 = 0xCD9E8D57u;
+constexpr uint32_t kPhiloxW0 = 0x9E3779B9u;
+constexpr uint32_t kPhiloxW1 = 0xBB67AE85u;
+
+// Ten Philox rounds; only output words 0 and 1 are consumed by the Gaussian draw.
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                              uint32_t k0, uint32_t k1, uint32_t& r0, uint32_t& r1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(kPhiloxM0, c0), lo0 = kPhiloxM0 * c0;
+    const uint32_t hi1 = __umulhi(kPhiloxM1, c2), lo1 = kPhiloxM1 * c2;
+    c0 = hi1 ^ c1 ^ k0;
+    c1 = lo1;
+    c2 = hi0 ^ c3 ^ k1;
+    c3 = lo0;
+    k0 += kPhiloxW0;
+    k1 += kPhiloxW1;
+  }
+  r0 = c0;
+  r1 = c1;
+}
+
+// z = sqrt(-2 ln u1) cos(2 pi u2), u1 = ((r0 >> 8) + 1) 2^-24 in (0,1], u2 = (r1 >> 8) 2^-24 in [0,1).
+__device__ __forceinline__ float gaussian_from_words(uint32_t r0, uint32_t r1) {
+  const float u1 = static_cast<float>((r0 >> 8) + 1u) * 5.9604644775390625e-8f;
+  const float two_u2 = static_cast<float>(r1 >> 8) * 1.1920928955078125e-7f;   // 2*u2, exact
+  const float rad = sqrtf(-2.0f * logf(u1));
+  return rad * cospif(two_u2);
+}
+
+__device__ __forceinline__ float z_of(uint64_t gidx, uint32_t step_lo, uint32_t step_hi,
+                                      uint32_t seed_lo, uint32_t seed_hi) {
+  uint32_t r0, r1;
+  philox4x32_10(static_cast<uint32_t>(gidx), static_cast<uint32_t>(gidx >> 32), step_lo, step_hi,
+                seed_lo, seed_hi, r0, r1);
+  return gaussian_from_words(r0, r1);
+}
+
+__device__ __forceinline__ float resolve_scale(const ScaleArg& a) {
+  if (a.f_plus == nullptr) return a.scale;
+  const double g = (*a.f_plus - *a.f_minus) / (2.0 * static_cast<double>(a.eps));
+  return -static_cast<float>(static_cast<double>(a.lr) * g);
+}
+
+// Two entries per thread: one 16-byte index load, one 8-byte value load and store.
+__global__ void __launch_bounds__(256)
+sparse_axpy_kernel(const float* __restrict__ S_in, float* __restrict__ S_out,
+                   const int64_t* __restrict__ idx, int64_t k, int64_t idx_base, uint32_t seed_lo,
+                   uint32_t seed_hi, uint32_t step_lo, uint32_t step_hi, ScaleArg sa) {
+  const float scale = resolve_scale(sa);
+  const int64_t pairs = k >> 1;
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  for (int64_t p = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; p < pairs; p += stride) {
+    const longlong2 id = reinterpret_cast<const longlong2*>(idx)[p];
+    const float2 s = reinterpret_cast<const float2*>(S_in)[p];
+    const float z0 = z_of(static_cast<uint64_t>(idx_base + id.x), step_lo, step_hi, seed_lo, seed_hi);
+    const float z1 = z_of(static_cast<uint64_t>(idx_base + id.y), step_lo, step_hi, seed_lo, seed_hi);
+    float2 o;
+    o.x = fmaf(scale, z0, s.x);
+    o.y = fmaf(scale, z1, s.y);
+    reinterpret_cast<float2*>(S_out)[p] = o;
+  }
+  if ((k & 1) && blockIdx.x == 0 && threadIdx.x == 0) {
+    const int64_t j = k - 1;
+    const float z = z_of(static_cast<uint64_t>(idx_base + idx[j]), step_lo, step_hi, seed_lo, seed_hi);
+    S_out[j] = fmaf(scale, z, S_in[j]);
+  }
+}
+
+__global__ void projected_gradient_kernel(const double* f_plus, const double* f_minus, float eps,
+                                          double* g) {
+  *g = (*f_plus - *f_minus) / (2.0 * static_cast<double>(eps));
+}
+
+szo_status launch_sparse_axpy(const float* S_in, float* S_out, const int64_t* idx, int64_t k,
+                              int64_t idx_base, uint64_t seed, uint64_t step, ScaleArg sa,
+                              cudaStream_t st) {
+  if (k == 0) return SZO_OK;
+  const int64_t pairs = (k + 1) / 2;
+  int64_t blocks = ceil_div(pairs, 256);
+  const int64_t cap = 148 * 8;
+  if (blocks > cap) blocks = cap;
+  sparse_axpy_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(
+      S_in, S_out, idx, k, idx_base, static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32),
+      static_cast<uint32_t>(step), static_cast<uint32_t>(step >> 32), sa);
+  count_launch();
+  SZO_CHECK_LAUNCH("sparse_axpy_kernel");
+  return SZO_OK;
+}
+
+}  // namespace szo
+
+extern "C" {
+
+szo_status szo_perturb(const float* S_in, float* S_out, const int64_t* idx, int64_t k,
+                       int64_t idx_base, uint64_t seed, uint64_t step, float scale, void* stream) {
+  SZO_REQUIRE(k >= 0, SZO_ERR_INVALID_ARG, "k < 0");
+  if (k == 0) return SZO_OK;
+  SZO_REQUIRE(S_in && S_out && idx, SZO_ERR_INVALID_ARG, "NULL pointer");
+  SZO_REQUIRE(idx_base >= 0, SZO_ERR_INVALID_ARG, "idx_base < 0");
+  SZO_REQUIRE(szo::aligned16(S_in) && szo::aligned16(S_out) && szo::aligned16(idx), SZO_ERR_ALIGNMENT,
+              "S_in, S_out and idx must be 16-byte aligned");
+  szo::ScaleArg sa{scale, 0.f, 0.f, nullptr, nullptr};
+  return szo::launch_sparse_axpy(S_in, S_out, idx, k, idx_base, seed, step, sa,
+                                 static_cast<cudaStream_t>(stream));
+}
+
+szo_status szo_update(float* S, const int64_t* idx, int64_t k, int64_t idx_base, uint64_t seed,
+                      uint64_t step, float lr, const double* f_plus_dev, const double* f_minus_dev,
+                      float eps, void* stream) {
+  SZO_REQUIRE(k >= 0, SZO_ERR_INVALID_ARG, "k < 0");
+  SZO_REQUIRE(f_plus_dev && f_minus_dev, SZO_ERR_INVALID_ARG, "NULL loss pointer");
+  SZO_REQUIRE(eps != 0.f, SZO_ERR_INVALID_ARG, "eps == 0");
+  if (k == 0) return SZO_OK;
+  SZO_REQUIRE(S && idx, SZO_ERR_INVALID_ARG, "NULL pointer");
+  SZO_REQUIRE(idx_base >= 0, SZO_ERR_INVALID_ARG, "idx_base < 0");
+  SZO_REQUIRE(szo::aligned16(S) && szo::aligned16(idx), SZO_ERR_ALIGNMENT,
+              "S and idx must be 16-byte aligned");
+  szo::ScaleArg sa{0.f, lr, eps, f_plus_dev, f_minus_dev};
+  return szo::launch_sparse_axpy(S, S, idx, k, idx_base, seed, step, sa,
+                                 static_cast<cudaStream_t>(stream));
+}
+
+szo_status szo_projected_gradient(const double* f_plus_dev, const double* f_minus_dev, float eps,
+                                  double* g_dev, void* stream) {
+  SZO_REQUIRE(f_plus_dev && f_minus_dev && g_dev, SZO_ERR_INVALID_ARG, "NULL pointer");
+  SZO_REQUIRE(eps != 0.f, SZO_ERR_INVALID_ARG, "eps == 0");
+  szo::projected_gradient_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(f_plus_dev, f_minus_dev,
+                                                                              eps, g_dev);
+  szo::count_launch();
+  SZO_CHECK_LAUNCH("projected_gradient_kernel");
+  return SZO_OK;
+}
+
+}  // extern "C"
