@@ -1,0 +1,153 @@
+"""GPU parity: szo_perturb / szo_update / szo_projected_gradient / szo_quantize / szo_select_mask
+through the C ABI against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import szo_oracle as so
+from paper_2406_02913_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2406_02913_b200 import binding
+    binding.lib()
+    return binding
+
+
+def _z_tol(z_ref):
+    return 1e-6 * np.maximum(1.0, np.abs(z_ref.astype(np.float64)))
+
+
+@pytest.mark.parametrize("k", [1, 2, 7, 4096, 100_003])
+def test_perturb_matches_oracle(B, k):
+    n = 12_582_912_000                                      # OPT-13B linear parameter count (> 2^32)
+    idx = wl.sorted_random_indices(n, k, seed=1, i=k)
+    S = wl.rng(2, wl.PURPOSE_WEIGHTS, k).normal(0, 0.02, k).astype(np.float32)
+    seed, step, base = 0x1234_5678_9ABC_DEF0, 3 + (1 << 33), 17
+    d_idx = torch.from_numpy(idx).cuda()
+    d_S = torch.from_numpy(S).cuda()
+    # z itself: S_in = 0, scale = 1  ->  S_out = z exactly
+    zero = torch.zeros_like(d_S)
+    out = torch.empty_like(d_S)
+    B.szo_perturb(zero, out, d_idx, base, seed, step, 1.0)
+    z = out.cpu().numpy()
+    z_ref = so.gaussian(seed, step, idx + base)
+    assert np.all(np.abs(z.astype(np.float64) - z_ref) <= _z_tol(z_ref))
+    # the axpy with the GPU's own z is a single fp32 fma (bit-exact), out of place
+    eps = np.float32(1e-3)
+    B.szo_perturb(d_S, out, d_idx, base, seed, step, float(eps))
+    assert np.array_equal(out.cpu().numpy().view(np.uint32), so.fmaf32(eps, z, S).view(np.uint32))
+    assert np.array_equal(d_S.cpu().numpy(), S)                          # input untouched
+    ref = so.perturb(S, idx + base, seed, step, eps)
+    assert np.all(np.abs(out.cpu().numpy().astype(np.float64) - ref) <= 3e-8)
+
+
+def test_perturb_in_place_sequence_and_canaries(B):
+    k = 33_333
+    idx = wl.sorted_random_indices(16_777_216, k, seed=3)
+    S = wl.rng(4, wl.PURPOSE_WEIGHTS).normal(0, 0.02, k).astype(np.float32)
+    buf = torch.full((k + 64,), 7.25, dtype=torch.float32, device="cuda")    # canaries on both sides
+    view = buf[32:32 + k]
+    view.copy_(torch.from_numpy(S))
+    d_idx = torch.from_numpy(idx).cuda()
+    eps = np.float32(1e-3)
+    ref = S.copy()
+    z0 = torch.zeros(k, device="cuda")
+    zbuf = torch.empty(k, device="cuda")
+    B.szo_perturb(z0, zbuf, d_idx, 0, 1234, 5, 1.0)
+    z = zbuf.cpu().numpy()
+    for sc in (eps, np.float32(-2.0) * eps, eps):                 # +eps, -2eps, +eps (seed trick order)
+        B.szo_perturb(view, view, d_idx, 0, 1234, 5, float(sc))
+        ref = so.fmaf32(sc, z, ref)
+        assert np.array_equal(view.cpu().numpy().view(np.uint32), ref.view(np.uint32))
+    full = buf.cpu().numpy()
+    assert (full[:32] == 7.25).all() and (full[32 + k:] == 7.25).all()
+    assert np.max(np.abs(ref - S)) <= 2 * np.spacing(np.float32(0.25))
+
+
+def test_update_and_projected_gradient(B):
+    k = 5001
+    idx = wl.sorted_random_indices(1 << 24, k, seed=5)
+    S = wl.rng(6, wl.PURPOSE_WEIGHTS).normal(0, 0.02, k).astype(np.float32)
+    f = torch.tensor([6.931471805599453, 6.931099123], dtype=torch.float64, device="cuda")
+    g = torch.zeros(1, dtype=torch.float64, device="cuda")
+    eps, lr = np.float32(1e-3), np.float32(1e-5)
+    B.szo_projected_gradient(f[0:1], f[1:2], float(eps), g)
+    g_ref = so.projected_gradient(6.931471805599453, 6.931099123, eps)
+    assert g.item() == g_ref
+    d_S = torch.from_numpy(S).cuda()
+    d_idx = torch.from_numpy(idx).cuda()
+    zbuf = torch.empty(k, device="cuda")
+    B.szo_perturb(torch.zeros(k, device="cuda"), zbuf, d_idx, 99, 42, 7, 1.0)
+    B.szo_update(d_S, d_idx, 99, 42, 7, float(lr), f[0:1], f[1:2], float(eps))
+    sc = so.zo_update_scale(6.931471805599453, 6.931099123, eps, lr)
+    ref = so.fmaf32(sc, zbuf.cpu().numpy(), S)
+    assert np.array_equal(d_S.cpu().numpy().view(np.uint32), ref.view(np.uint32))
+    full = so.perturb(S, idx + 99, 42, 7, sc)
+    assert np.allclose(d_S.cpu().numpy(), full, rtol=0, atol=1e-12 + abs(float(sc)) * 1e-5)
+
+
+def test_perturb_empty_and_bad_arguments(B):
+    e = torch.empty(0, device="cuda")
+    B.szo_perturb(e, e, torch.empty(0, dtype=torch.int64, device="cuda"), 0, 1, 1, 1.0)
+    S = torch.zeros(16, device="cuda")
+    idx = torch.arange(16, dtype=torch.int64, device="cuda")
+    with pytest.raises(B.SzoError) as ei:
+        B.szo_perturb(S[1:], S[1:], idx[:15], 0, 1, 1, 1.0)            # misaligned
+    assert ei.value.name == "SZO_ERR_ALIGNMENT"
+    with pytest.raises(B.SzoError):
+        B.szo_perturb(S, S, idx, -5, 1, 1, 1.0)
+
+
+@pytest.mark.parametrize("N,K,G,fmt,wdt", [(64, 256, 64, "f16", torch.float32), (96, 4096, 128, "bf16", torch.float32),
+                                           (33, 320, 32, "bf16", torch.float32), (16, 512, 128, "bf16", torch.bfloat16)])
+def test_quantize_bit_exact(B, N, K, G, fmt, wdt):
+    W = wl.gaussian_matrix(N, K, 0.02, seed=7, i=N)
+    if wdt == torch.bfloat16:
+        W = wl.bf16_round(W)
+    idx = wl.sorted_random_indices(N * K, max(1, N * K // 1000), seed=8)
+    _, Wd = so.decompose(W, idx)
+    Wd[1, :G] = 0.03125                                       # constant group -> scale 0
+    codes, sb, zb = so.quantize_int4(Wd, G, fmt)
+    dW = torch.from_numpy(Wd).cuda().to(wdt)
+    g_codes, g_s, g_z = B.szo_quantize(dW, G, fmt)
+    assert np.array_equal(g_codes.cpu().numpy(), codes)
+    assert np.array_equal(g_s.cpu().view(torch.int16).numpy().view(np.uint16), sb)
+    assert np.array_equal(g_z.cpu().view(torch.int16).numpy().view(np.uint16), zb)
+
+
+def test_quantize_rejects_bad_shapes(B):
+    W = torch.zeros((4, 100), device="cuda")
+    with pytest.raises(B.SzoError) as ei:
+        B.szo_quantize(W, 64, "bf16")
+    assert ei.value.name == "SZO_ERR_SHAPE"
+
+
+@pytest.mark.parametrize("n,k", [(1, 1), (37, 5), (8192, 8), (8193, 8193), (1_000_003, 1000), (16_777_216, 16_777)])
+def test_select_mask_matches_oracle(B, n, k):
+    g = wl.student_t_gradient(n, 3.0, seed=9, i=n % 1000)
+    scores = (g * g).astype(np.float32)
+    got = B.szo_select_mask(torch.from_numpy(scores).cuda(), k).cpu().numpy()
+    assert np.array_equal(got, so.select_mask(scores, k))
+
+
+def test_select_mask_ties_zero_k_and_nan(B):
+    n = 50_000
+    scores = wl.rng(10, wl.PURPOSE_SCORES).integers(0, 6, n).astype(np.float32)      # heavy ties
+    for k in (0, 1, 777, 25_000, n):
+        got = B.szo_select_mask(torch.from_numpy(scores).cuda(), k).cpu().numpy()
+        assert np.array_equal(got, so.select_mask(scores, k))
+    same = np.ones(10_000, np.float32)
+    assert np.array_equal(B.szo_select_mask(torch.from_numpy(same).cuda(), 100).cpu().numpy(), np.arange(100))
+    z = np.array([0.0, -0.0, 0.0, 1.0] * 4, np.float32)
+    assert np.array_equal(B.szo_select_mask(torch.from_numpy(z).cuda(), 6).cpu().numpy(), so.select_mask(z, 6))
+    bad = scores.copy()
+    bad[123] = np.nan
+    with pytest.raises(B.SzoError) as ei:
+        B.szo_select_mask(torch.from_numpy(bad).cuda(), 5)
+    assert ei.value.name == "SZO_ERR_NONFINITE"
+    with pytest.raises(B.SzoError):
+        B.szo_select_mask(torch.from_numpy(same).cuda(), same.size + 1)
