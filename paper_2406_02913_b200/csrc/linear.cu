@@ -397,8 +397,9 @@ szo_status szo_linear_fwd(const szo_linear_t* p, const void* x, szo_dtype x_dtyp
   if (M == 0) return SZO_OK;
   SZO_REQUIRE(x && y, SZO_ERR_INVALID_ARG, "x or y is NULL");
   SZO_REQUIRE(p->nnz == 0 || S_pert, SZO_ERR_INVALID_ARG, "S_pert is NULL");
-  SZO_REQUIRE(aligned16(x) && aligned16(y) && aligned16(S_pert) && aligned16(workspace), SZO_ERR_ALIGNMENT,
-              "buffers must be 16-byte aligned");
+  SZO_REQUIRE(aligned16(x) && aligned16(y) && aligned16(workspace), SZO_ERR_ALIGNMENT,
+              "x, y and workspace must be 16-byte aligned");
+  SZO_REQUIRE((reinterpret_cast<uintptr_t>(S_pert) & 3u) == 0, SZO_ERR_ALIGNMENT, "S_pert must be 4-byte aligned");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (mode == SZO_MODE_FP32_VALIDATE)
     return linear_fwd_fp32(p, x, x_dtype, M, S_pert, y, y_dtype, workspace, workspace_bytes, st);

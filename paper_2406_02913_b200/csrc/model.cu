@@ -1,0 +1,565 @@
+// Loss path of a decoder-only language model and the whole ZO-SGD step on one GPU.
+//
+// Definition 1 (SPSA) evaluates the loss at w + eps z and w - eps z; Definitions 2 and 4 update the
+// k sensitive values.  Everything between the linear layers (embedding, RMSNorm/LayerNorm, rotary
+// positions, causal attention, SiLU-gated or ReLU MLP, residuals, cross-entropy) is plain CUDA
+// here.  The residual stream is fp32; activations fed to the linears are T = bf16 (tensor-core
+// path) or fp32 (validation path); per-token losses are summed in fp64 in a fixed order so that
+// f+ and f- are produced by the identical, deterministic kernel sequence.
+#include <vector>
+
+#include "linear.cuh"
+
+namespace szo {
+
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// Block-wide sum with a fixed reduction tree (blockDim.x a multiple of 32, <= 1024).
+__device__ __forceinline__ float block_sum(float v, float* scratch) {
+#pragma unroll
+  for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  const int w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) scratch[w] = v;
+  __syncthreads();
+  float t = 0.f;
+  for (int i = 0; i < nw; ++i) t += scratch[i];
+  return t;
+}
+
+// h[m, :] = embed[tok[m], :] (+ pos[m % S, :])
+__global__ void embed_kernel(const int32_t* __restrict__ tok, const __nv_bfloat16* __restrict__ embed,
+                             const __nv_bfloat16* __restrict__ pos, int S, int d, int vocab,
+                             float* __restrict__ h) {
+  const int64_t m = blockIdx.x;
+  int32_t t = tok[m];
+  t = t < 0 ? 0 : (t >= vocab ? vocab - 1 : t);
+  const __nv_bfloat16* e = embed + static_cast<int64_t>(t) * d;
+  const __nv_bfloat16* p = pos ? pos + static_cast<int64_t>(m % S) * d : nullptr;
+  for (int c = threadIdx.x; c < d; c += blockDim.x)
+    h[m * d + c] = __bfloat162float(e[c]) + (p ? __bfloat162float(p[c]) : 0.f);
+}
+
+// RMSNorm (beta == nullptr): x / sqrt(mean x^2 + eps) * gamma; LayerNorm otherwise.
+// row_stride/row_offset select which rows are normalised (all rows, or the last token of each
+// sequence when only that one feeds the loss).
+template <typename T>
+__global__ void __launch_bounds__(256)
+norm_kernel(const float* __restrict__ h, const float* __restrict__ gamma, const float* __restrict__ beta,
+            int d, float eps, bool layer_norm, int64_t row_stride, int64_t row_offset, T* __restrict__ out) {
+  __shared__ float scratch[32];
+  const int64_t m = static_cast<int64_t>(blockIdx.x) * row_stride + row_offset;
+  const float* x = h + m * d;
+  T* o = out + static_cast<int64_t>(blockIdx.x) * d;
+  float s = 0.f;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) s += x[c];
+  const float mu = layer_norm ? block_sum(s, scratch) / d : 0.f;
+  float q = 0.f;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    const float t = x[c] - mu;
+    q = fmaf(t, t, q);
+  }
+  const float var = block_sum(q, scratch) / d;
+  const float r = 1.0f / sqrtf(var + eps);
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    const float v = (x[c] - mu) * r * gamma[c] + (beta ? beta[c] : 0.f);
+    o[c] = from_f32<T>(v);
+  }
+}
+
+// cos/sin table [max_seq, hd/2] from fp64 math: angle = p * base^(-2i/hd).
+__global__ void rope_table_kernel(int max_seq, int half, double base, float2* __restrict__ tab) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= max_seq * half) return;
+  const int p = i / half, j = i % half;
+  const double ang = static_cast<double>(p) * pow(base, -2.0 * j / (2.0 * half));
+  tab[i] = make_float2(static_cast<float>(cos(ang)), static_cast<float>(sin(ang)));
+}
+
+// In-place rotation of the pairs (i, i + hd/2) of every head of x [M, n_heads*hd].
+template <typename T>
+__global__ void rope_kernel(T* __restrict__ x, const float2* __restrict__ tab, int64_t M, int S, int n_heads,
+                            int hd) {
+  const int half = hd >> 1;
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= M * n_heads * half) return;
+  const int j = static_cast<int>(i % half);
+  const int64_t mh = i / half;
+  const int64_t m = mh / n_heads;
+  const float2 cs = tab[static_cast<int64_t>(m % S) * half + j];
+  T* p = x + mh * hd;
+  const float a = to_f32<T>(p[j]), b = to_f32<T>(p[j + half]);
+  p[j] = from_f32<T>(a * cs.x - b * cs.y);
+  p[j + half] = from_f32<T>(b * cs.x + a * cs.y);
+}
+
+// Causal softmax attention, one warp per query; lanes split the head dimension.
+template <typename T, int HD>
+__global__ void __launch_bounds__(128)
+attn_warp_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v, T* __restrict__ o,
+                 int S, int H, int Hkv, float scale) {
+  constexpr int E = HD / 32;
+  const int lane = threadIdx.x & 31;
+  const int s = blockIdx.x * 4 + (threadIdx.x >> 5);
+  const int hq = blockIdx.y, b = blockIdx.z;
+  if (s >= S) return;
+  const int hk = hq / (H / Hkv);
+  const int64_t dq = static_cast<int64_t>(H) * HD, dk = static_cast<int64_t>(Hkv) * HD;
+  const T* qp = q + (static_cast<int64_t>(b) * S + s) * dq + hq * HD;
+  float qr[E], acc[E];
+#pragma unroll
+  for (int j = 0; j < E; ++j) {
+    qr[j] = to_f32<T>(qp[lane + 32 * j]) * scale;
+    acc[j] = 0.f;
+  }
+  float mx = -INFINITY, l = 0.f;
+  for (int t = 0; t <= s; ++t) {
+    const T* kp = k + (static_cast<int64_t>(b) * S + t) * dk + hk * HD;
+    const T* vp = v + (static_cast<int64_t>(b) * S + t) * dk + hk * HD;
+    float dot = 0.f;
+#pragma unroll
+    for (int j = 0; j < E; ++j) dot = fmaf(qr[j], to_f32<T>(kp[lane + 32 * j]), dot);
+#pragma unroll
+    for (int off = 16; off; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+    const float mn = fmaxf(mx, dot);
+    const float corr = expf(mx - mn), p = expf(dot - mn);
+    l = l * corr + p;
+#pragma unroll
+    for (int j = 0; j < E; ++j) acc[j] = fmaf(p, to_f32<T>(vp[lane + 32 * j]), acc[j] * corr);
+    mx = mn;
+  }
+  T* op = o + (static_cast<int64_t>(b) * S + s) * dq + hq * HD;
+  const float inv = 1.0f / l;
+#pragma unroll
+  for (int j = 0; j < E; ++j) op[lane + 32 * j] = from_f32<T>(acc[j] * inv);
+}
+
+template <typename T>
+__global__ void silu_mul_kernel(const T* __restrict__ gate, const T* __restrict__ up, int64_t n, T* __restrict__ out) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const float g = to_f32<T>(gate[i]);
+  out[i] = from_f32<T>(g / (1.0f + expf(-g)) * to_f32<T>(up[i]));
+}
+
+template <typename T>
+__global__ void relu_kernel(T* __restrict__ x, int64_t n) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i < n) x[i] = from_f32<T>(fmaxf(to_f32<T>(x[i]), 0.f));
+}
+
+template <typename T>
+__global__ void residual_add_kernel(float* __restrict__ h, const T* __restrict__ y, int64_t n) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i < n) h[i] += to_f32<T>(y[i]);
+}
+
+// Next-token cross-entropy of row m (position s < S-1 predicts tok[m+1]); 0 for the last position.
+__global__ void __launch_bounds__(256)
+ce_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__ tok, int S, int V,
+               double* __restrict__ tok_loss) {
+  __shared__ float scratch[32];
+  const int64_t m = blockIdx.x;
+  if ((m % S) == S - 1) {
+    if (threadIdx.x == 0) tok_loss[m] = 0.0;
+    return;
+  }
+  const float* row = logits + m * V;
+  float mx = -INFINITY;
+  for (int c = threadIdx.x; c < V; c += blockDim.x) mx = fmaxf(mx, row[c]);
+#pragma unroll
+  for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = mx;
+  __syncthreads();
+  for (int i = 0; i < (blockDim.x >> 5); ++i) mx = fmaxf(mx, scratch[i]);
+  float s = 0.f;
+  for (int c = threadIdx.x; c < V; c += blockDim.x) s += expf(row[c] - mx);
+  s = block_sum(s, scratch);
+  if (threadIdx.x == 0) {
+    int32_t t = tok[m + 1];
+    t = t < 0 ? 0 : (t >= V ? V - 1 : t);
+    tok_loss[m] = (static_cast<double>(mx) + log(static_cast<double>(s))) - static_cast<double>(row[t]);
+  }
+}
+
+// 2-way cross-entropy over the logits of two candidate ids for the normalised last-token state.
+template <typename T>
+__global__ void __launch_bounds__(256)
+cls2_kernel(const T* __restrict__ a_last, const __nv_bfloat16* __restrict__ lm_head, const int32_t* __restrict__ cand,
+            const int32_t* __restrict__ labels, int d, int V, double* __restrict__ seq_loss) {
+  __shared__ float scratch[32];
+  const int b = blockIdx.x;
+  const T* a = a_last + static_cast<int64_t>(b) * d;
+  int32_t c0 = cand[0], c1 = cand[1];
+  c0 = c0 < 0 ? 0 : (c0 >= V ? V - 1 : c0);
+  c1 = c1 < 0 ? 0 : (c1 >= V ? V - 1 : c1);
+  const __nv_bfloat16* e0 = lm_head + static_cast<int64_t>(c0) * d;
+  const __nv_bfloat16* e1 = lm_head + static_cast<int64_t>(c1) * d;
+  float s0 = 0.f, s1 = 0.f;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    const float x = to_f32<T>(a[c]);
+    s0 = fmaf(x, __bfloat162float(e0[c]), s0);
+    s1 = fmaf(x, __bfloat162float(e1[c]), s1);
+  }
+  s0 = block_sum(s0, scratch);
+  s1 = block_sum(s1, scratch);
+  if (threadIdx.x == 0) {
+    const double l0 = s0, l1 = s1, mx = l0 > l1 ? l0 : l1;
+    const double lse = mx + log(exp(l0 - mx) + exp(l1 - mx));
+    seq_loss[b] = lse - (labels[b] ? l1 : l0);
+  }
+}
+
+// *out = (sum of v[0..n)) / denom, fixed order, fp64.
+__global__ void __launch_bounds__(1024) mean_f64_kernel(const double* __restrict__ v, int64_t n, double denom,
+                                                        double* __restrict__ out) {
+  __shared__ double s[1024];
+  double t = 0.0;
+  for (int64_t i = threadIdx.x; i < n; i += 1024) t += v[i];
+  s[threadIdx.x] = t;
+  __syncthreads();
+  for (int o = 512; o; o >>= 1) {
+    if (threadIdx.x < o) s[threadIdx.x] += s[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *out = s[0] / denom;
+}
+
+__global__ void gidx_kernel(const int64_t* __restrict__ idx, int64_t nnz, int64_t base, int64_t* __restrict__ out) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i < nnz) out[i] = base + idx[i];
+}
+
+}  // namespace szo
+
+using namespace szo;
+
+struct szo_model {
+  szo_model_config cfg;
+  szo_model_weights top;
+  std::vector<szo_layer_weights> layers;
+  std::vector<szo_linear_t*> plans;      // n_layers * n_lin
+  std::vector<int64_t> offsets;          // start of each linear's entries in S_all (+ total)
+  szo_linear_t* lm_head_plan = nullptr;
+  int n_lin = 0;
+  float* S_all = nullptr;
+  int64_t k_total = 0;
+  int64_t* gidx = nullptr;
+  int64_t Mmax = 0;
+  // activations
+  float* h = nullptr;
+  void *a = nullptr, *q = nullptr, *k = nullptr, *v = nullptr, *o = nullptr, *y = nullptr, *gate = nullptr,
+       *up = nullptr;
+  float* logits = nullptr;
+  double* tok_loss = nullptr;
+  float2* rope_tab = nullptr;
+  void* ws = nullptr;
+  size_t ws_bytes = 0;
+  int32_t *d_tokens = nullptr, *d_labels = nullptr, *d_cand = nullptr;
+  double* d_scalars = nullptr;
+  int64_t last_launches = 0;
+  std::vector<void*> owned;
+};
+
+namespace {
+
+template <typename P> szo_status dev_alloc(szo_model* m, P** p, size_t bytes) {
+  void* q = nullptr;
+  SZO_CHECK_CUDA(cudaMalloc(&q, bytes ? bytes : 16));
+  m->owned.push_back(q);
+  *p = static_cast<P*>(q);
+  return SZO_OK;
+}
+
+void linear_shape(const szo_model_config& c, int j, int64_t* N, int64_t* K) {
+  const int64_t d = c.d_model, kv = static_cast<int64_t>(c.n_kv_heads) * (c.d_model / c.n_heads), ff = c.d_ff;
+  if (c.arch == 0) {
+    const int64_t n[7] = {d, kv, kv, d, ff, ff, d}, k[7] = {d, d, d, d, d, d, ff};
+    *N = n[j]; *K = k[j];
+  } else {
+    const int64_t n[6] = {d, kv, kv, d, ff, d}, k[6] = {d, d, d, d, d, ff};
+    *N = n[j]; *K = k[j];
+  }
+}
+
+unsigned blocks_for(int64_t n, int t) { return static_cast<unsigned>(ceil_div(n, t)); }
+
+template <typename T>
+szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand, int B,
+                      int S, const float* Sv, double* loss_dev, cudaStream_t st) {
+  const szo_model_config& c = m->cfg;
+  const int64_t M = static_cast<int64_t>(B) * S;
+  const int d = c.d_model, H = c.n_heads, Hkv = c.n_kv_heads, hd = d / H, ff = c.d_ff;
+  const int64_t dkv = static_cast<int64_t>(Hkv) * hd;
+  const int act = c.act_dtype;
+  const bool opt = c.arch == 1;
+  T *a = static_cast<T*>(m->a), *q = static_cast<T*>(m->q), *k = static_cast<T*>(m->k), *v = static_cast<T*>(m->v),
+    *o = static_cast<T*>(m->o), *y = static_cast<T*>(m->y), *gate = static_cast<T*>(m->gate),
+    *up = static_cast<T*>(m->up);
+  auto lin = [&](int layer, int j, const void* x, void* out) -> szo_status {
+    const int t = layer * m->n_lin + j;
+    return szo_linear_fwd(m->plans[t], x, static_cast<szo_dtype>(act), M, Sv + m->offsets[t], out,
+                          static_cast<szo_dtype>(act), c.linear_mode, m->ws, m->ws_bytes, st);
+  };
+  embed_kernel<<<static_cast<unsigned>(M), 128, 0, st>>>(tokens, static_cast<const __nv_bfloat16*>(m->top.embed),
+                                                        static_cast<const __nv_bfloat16*>(m->top.pos), S, d,
+                                                        c.vocab, m->h);
+  count_launch();
+  for (int l = 0; l < c.n_layers; ++l) {
+    const szo_layer_weights& L = m->layers[l];
+    norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, L.attn_norm_g, L.attn_norm_b, d, c.norm_eps, opt,
+                                                            1, 0, a);
+    count_launch();
+    SZO_TRY(lin(l, 0, a, q));
+    SZO_TRY(lin(l, 1, a, k));
+    SZO_TRY(lin(l, 2, a, v));
+    if (!opt) {
+      rope_kernel<T><<<blocks_for(M * H * (hd / 2), 256), 256, 0, st>>>(q, m->rope_tab, M, S, H, hd);
+      rope_kernel<T><<<blocks_for(M * Hkv * (hd / 2), 256), 256, 0, st>>>(k, m->rope_tab, M, S, Hkv, hd);
+      count_launch(2);
+    }
+    {
+      dim3 grid(static_cast<unsigned>(ceil_div(S, 4)), H, B);
+      const float scale = 1.0f / sqrtf(static_cast<float>(hd));
+      if (hd == 64) attn_warp_kernel<T, 64><<<grid, 128, 0, st>>>(q, k, v, o, S, H, Hkv, scale);
+      else attn_warp_kernel<T, 128><<<grid, 128, 0, st>>>(q, k, v, o, S, H, Hkv, scale);
+      count_launch();
+    }
+    SZO_TRY(lin(l, 3, o, y));
+    residual_add_kernel<T><<<blocks_for(M * d, 256), 256, 0, st>>>(m->h, y, M * d);
+    norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, L.mlp_norm_g, L.mlp_norm_b, d, c.norm_eps, opt, 1,
+                                                            0, a);
+    count_launch(2);
+    if (!opt) {
+      SZO_TRY(lin(l, 4, a, gate));
+      SZO_TRY(lin(l, 5, a, up));
+      silu_mul_kernel<T><<<blocks_for(M * ff, 256), 256, 0, st>>>(gate, up, M * ff, gate);
+      count_launch();
+      SZO_TRY(lin(l, 6, gate, y));
+    } else {
+      SZO_TRY(lin(l, 4, a, gate));
+      relu_kernel<T><<<blocks_for(M * ff, 256), 256, 0, st>>>(gate, M * ff);
+      count_launch();
+      SZO_TRY(lin(l, 5, gate, y));
+    }
+    residual_add_kernel<T><<<blocks_for(M * d, 256), 256, 0, st>>>(m->h, y, M * d);
+    count_launch();
+  }
+  if (c.loss_kind == 0) {
+    norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, m->top.final_norm_g, m->top.final_norm_b, d,
+                                                            c.norm_eps, opt, 1, 0, a);
+    count_launch();
+    const int mode = c.linear_mode == SZO_MODE_FP32_VALIDATE ? SZO_MODE_FP32_VALIDATE : SZO_MODE_SPARSE_ADD;
+    SZO_TRY(szo_linear_fwd(m->lm_head_plan, a, static_cast<szo_dtype>(act), M, nullptr, m->logits, SZO_F32, mode,
+                           m->ws, m->ws_bytes, st));
+    ce_rows_kernel<<<static_cast<unsigned>(M), 256, 0, st>>>(m->logits, tokens, S, c.vocab, m->tok_loss);
+    mean_f64_kernel<<<1, 1024, 0, st>>>(m->tok_loss, M, static_cast<double>(B) * (S - 1), loss_dev);
+    count_launch(2);
+  } else {
+    norm_kernel<T><<<static_cast<unsigned>(B), 256, 0, st>>>(m->h, m->top.final_norm_g, m->top.final_norm_b, d,
+                                                            c.norm_eps, opt, S, S - 1, a);
+    cls2_kernel<T><<<static_cast<unsigned>(B), 256, 0, st>>>(a, static_cast<const __nv_bfloat16*>(m->top.lm_head), cand,
+                                                            labels, d, c.vocab, m->tok_loss);
+    mean_f64_kernel<<<1, 1024, 0, st>>>(m->tok_loss, B, static_cast<double>(B), loss_dev);
+    count_launch(3);
+  }
+  SZO_CHECK_LAUNCH("model kernels");
+  return SZO_OK;
+}
+
+szo_status run_loss(szo_model* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand, int B, int S,
+                    const float* Sv, double* loss_dev, cudaStream_t st) {
+  if (m->cfg.act_dtype == SZO_F32) return run_loss_t<float>(m, tokens, labels, cand, B, S, Sv, loss_dev, st);
+  return run_loss_t<__nv_bfloat16>(m, tokens, labels, cand, B, S, Sv, loss_dev, st);
+}
+
+szo_status check_batch(const szo_model* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand, int B,
+                       int S) {
+  SZO_REQUIRE(m != nullptr, SZO_ERR_INVALID_ARG, "model is NULL");
+  SZO_REQUIRE(tokens != nullptr, SZO_ERR_INVALID_ARG, "tokens is NULL");
+  SZO_REQUIRE(B >= 1 && B <= m->cfg.max_batch && S >= 2 && S <= m->cfg.max_seq, SZO_ERR_SHAPE,
+              "need 1 <= B <= %d and 2 <= S <= %d (got B=%d, S=%d)", m->cfg.max_batch, m->cfg.max_seq, B, S);
+  SZO_REQUIRE(m->cfg.loss_kind == 0 || (labels && cand), SZO_ERR_INVALID_ARG,
+              "labels and cand are required for the 2-candidate loss");
+  SZO_REQUIRE(m->cfg.arch == 0 || S <= m->cfg.max_pos, SZO_ERR_SHAPE, "S exceeds the position table");
+  return SZO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, const szo_model_weights* top,
+                            const szo_layer_weights* layers_host, float* S_all, void* stream) {
+  SZO_REQUIRE(out && cfg && top && layers_host, SZO_ERR_INVALID_ARG, "NULL argument");
+  *out = nullptr;
+  const szo_model_config& c = *cfg;
+  SZO_REQUIRE(c.arch == 0 || c.arch == 1, SZO_ERR_INVALID_ARG, "arch must be 0 or 1");
+  SZO_REQUIRE(c.n_layers > 0 && c.d_model > 0 && c.n_heads > 0 && c.n_kv_heads > 0 && c.d_ff > 0 && c.vocab > 1,
+              SZO_ERR_SHAPE, "non-positive model dimension");
+  SZO_REQUIRE(c.d_model % c.n_heads == 0 && c.n_heads % c.n_kv_heads == 0, SZO_ERR_SHAPE,
+              "d_model %% n_heads and n_heads %% n_kv_heads must be 0");
+  const int hd = c.d_model / c.n_heads;
+  SZO_REQUIRE(hd == 64 || hd == 128, SZO_ERR_UNSUPPORTED, "head dimension must be 64 or 128 (got %d)", hd);
+  SZO_REQUIRE(c.act_dtype == SZO_BF16 || c.act_dtype == SZO_F32, SZO_ERR_UNSUPPORTED, "act_dtype must be bf16 or f32");
+  SZO_REQUIRE(c.act_dtype == SZO_BF16 || c.linear_mode == SZO_MODE_FP32_VALIDATE, SZO_ERR_UNSUPPORTED,
+              "fp32 activations need the fp32 validation mode");
+  SZO_REQUIRE(c.loss_kind == 0 || c.loss_kind == 1, SZO_ERR_INVALID_ARG, "loss_kind must be 0 or 1");
+  SZO_REQUIRE(c.max_batch > 0 && c.max_seq > 1, SZO_ERR_SHAPE, "max_batch/max_seq");
+  SZO_REQUIRE(c.arch == 0 || (top->pos && c.max_pos >= c.max_seq), SZO_ERR_INVALID_ARG, "position table missing/short");
+  SZO_REQUIRE(top->embed && top->lm_head && top->final_norm_g, SZO_ERR_INVALID_ARG, "missing top-level weights");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  szo_model* m = new szo_model();
+  m->cfg = c;
+  m->top = *top;
+  m->n_lin = c.arch == 0 ? 7 : 6;
+  m->layers.assign(layers_host, layers_host + c.n_layers);
+  m->S_all = S_all;
+  m->Mmax = static_cast<int64_t>(c.max_batch) * c.max_seq;
+  auto bail = [&](szo_status s) {
+    szo_model_destroy(m);
+    return s;
+  };
+#define SZO_M_TRY(expr)                    \
+  do {                                     \
+    szo_status s__ = (expr);               \
+    if (s__ != SZO_OK) return bail(s__);   \
+  } while (0)
+  // plans and offsets
+  size_t ws_need = 0;
+  m->offsets.push_back(0);
+  for (int l = 0; l < c.n_layers; ++l) {
+    for (int j = 0; j < m->n_lin; ++j) {
+      int64_t N, K;
+      linear_shape(c, j, &N, &K);
+      const szo_linear_weights& w = m->layers[l].lin[j];
+      szo_linear_t* p = nullptr;
+      SZO_M_TRY(szo_linear_create(&p, N, K, c.group, w.codes, w.scales, w.zeros, static_cast<szo_dtype>(c.sz_dtype),
+                                  w.idx, w.nnz, w.bias, st));
+      m->plans.push_back(p);
+      m->offsets.push_back(m->offsets.back() + w.nnz);
+      const size_t need = szo_linear_workspace_bytes(p, m->Mmax, c.linear_mode);
+      if (need > ws_need) ws_need = need;
+    }
+  }
+  m->k_total = m->offsets.back();
+  if (m->k_total > 0 && S_all == nullptr) return bail(fail(SZO_ERR_INVALID_ARG, "S_all is NULL"));
+  if (c.loss_kind == 0) {
+    SZO_M_TRY(szo_linear_create(&m->lm_head_plan, c.vocab, c.d_model, 0, top->lm_head, nullptr, nullptr, SZO_BF16,
+                                nullptr, 0, nullptr, st));
+    const size_t need = szo_linear_workspace_bytes(m->lm_head_plan, m->Mmax, c.linear_mode);
+    if (need > ws_need) ws_need = need;
+  }
+  // buffers
+  const size_t e = c.act_dtype == SZO_F32 ? 4 : 2;
+  const int64_t Mx = m->Mmax, d = c.d_model, dkv = static_cast<int64_t>(c.n_kv_heads) * hd, ff = c.d_ff;
+  SZO_M_TRY(dev_alloc(m, &m->gidx, m->k_total * sizeof(int64_t)));
+  SZO_M_TRY(dev_alloc(m, &m->h, Mx * d * sizeof(float)));
+  SZO_M_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->a), Mx * d * e));
+  SZO_M_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->q), Mx * d * e));
+  SZO_M_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->k), Mx * dkv * e));
+  SZO_M_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->v), Mx * dkv * e));
+  SZO_M_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->o), Mx * d * e));
+  SZO_M_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->y), Mx * d * e));
+  SZO_M_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->gate), Mx * ff * e));
+  SZO_M_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->up), Mx * ff * e));
+  if (c.loss_kind == 0) SZO_M_TRY(dev_alloc(m, &m->logits, Mx * c.vocab * sizeof(float)));
+  SZO_M_TRY(dev_alloc(m, &m->tok_loss, Mx * sizeof(double)));
+  SZO_M_TRY(dev_alloc(m, &m->rope_tab, static_cast<size_t>(c.max_seq) * (hd / 2) * sizeof(float2)));
+  if (ws_need) SZO_M_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->ws), ws_need));
+  m->ws_bytes = ws_need;
+  SZO_M_TRY(dev_alloc(m, &m->d_tokens, Mx * sizeof(int32_t)));
+  SZO_M_TRY(dev_alloc(m, &m->d_labels, c.max_batch * sizeof(int32_t)));
+  SZO_M_TRY(dev_alloc(m, &m->d_cand, 16));
+  SZO_M_TRY(dev_alloc(m, &m->d_scalars, 4 * sizeof(double)));
+  // global indices and the rotary table
+  int64_t base = 0;
+  for (int l = 0, t = 0; l < c.n_layers; ++l) {
+    for (int j = 0; j < m->n_lin; ++j, ++t) {
+      int64_t N, K;
+      linear_shape(c, j, &N, &K);
+      const szo_linear_weights& w = m->layers[l].lin[j];
+      if (w.nnz)
+        gidx_kernel<<<blocks_for(w.nnz, 256), 256, 0, st>>>(w.idx, w.nnz, base, m->gidx + m->offsets[t]);
+      base += N * K;
+    }
+  }
+  rope_table_kernel<<<blocks_for(static_cast<int64_t>(c.max_seq) * (hd / 2), 256), 256, 0, st>>>(
+      c.max_seq, hd / 2, static_cast<double>(c.rope_base), m->rope_tab);
+  if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
+    return bail(fail(SZO_ERR_CUDA, "model set-up kernels failed"));
+#undef SZO_M_TRY
+  *out = m;
+  return SZO_OK;
+}
+
+int64_t szo_model_k_total(const szo_model_t* m) { return m ? m->k_total : 0; }
+const int64_t* szo_model_gidx(const szo_model_t* m) { return m ? m->gidx : nullptr; }
+int64_t szo_model_last_launches(const szo_model_t* m) { return m ? m->last_launches : 0; }
+
+szo_status szo_model_loss(szo_model_t* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand,
+                          int32_t B, int32_t S, const float* S_vals, double* loss_dev, void* stream) {
+  SZO_TRY(check_batch(m, tokens, labels, cand, B, S));
+  SZO_REQUIRE(loss_dev != nullptr, SZO_ERR_INVALID_ARG, "loss_dev is NULL");
+  return run_loss(m, tokens, labels, cand, B, S, S_vals ? S_vals : m->S_all, loss_dev, static_cast<cudaStream_t>(stream));
+}
+
+szo_status szo_model_zo_step(szo_model_t* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand,
+                             int32_t B, int32_t S, uint64_t seed, uint64_t step, float eps, float lr,
+                             double* f_plus_dev, double* f_minus_dev, double* g_dev, void* stream) {
+  SZO_TRY(check_batch(m, tokens, labels, cand, B, S));
+  SZO_REQUIRE(f_plus_dev && f_minus_dev && g_dev, SZO_ERR_INVALID_ARG, "NULL output scalar");
+  SZO_REQUIRE(eps != 0.f, SZO_ERR_INVALID_ARG, "eps == 0");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t before = g_launch_count;
+  const int64_t k = m->k_total;
+  float* Sv = m->S_all;
+  ScaleArg sa{eps, 0.f, 0.f, nullptr, nullptr};
+  SZO_TRY(launch_sparse_axpy(Sv, Sv, m->gidx, k, 0, seed, step, sa, st));                 // S += eps z
+  SZO_TRY(run_loss(m, tokens, labels, cand, B, S, Sv, f_plus_dev, st));                   // f+
+  sa.scale = -2.0f * eps;
+  SZO_TRY(launch_sparse_axpy(Sv, Sv, m->gidx, k, 0, seed, step, sa, st));                 // S -= 2 eps z
+  SZO_TRY(run_loss(m, tokens, labels, cand, B, S, Sv, f_minus_dev, st));                  // f-
+  sa.scale = eps;
+  SZO_TRY(launch_sparse_axpy(Sv, Sv, m->gidx, k, 0, seed, step, sa, st));                 // S += eps z
+  SZO_TRY(szo_projected_gradient(f_plus_dev, f_minus_dev, eps, g_dev, stream));           // g
+  ScaleArg su{0.f, lr, eps, f_plus_dev, f_minus_dev};
+  SZO_TRY(launch_sparse_axpy(Sv, Sv, m->gidx, k, 0, seed, step, su, st));                 // S -= lr g z
+  m->last_launches = g_launch_count - before;
+  return SZO_OK;
+}
+
+szo_status szo_model_zo_step_host(szo_model_t* m, const int32_t* tokens_host, const int32_t* labels_host,
+                                  const int32_t* cand_host, int32_t B, int32_t S, uint64_t seed, uint64_t step,
+                                  float eps, float lr, double* out3_host, void* stream) {
+  SZO_TRY(check_batch(m, tokens_host, labels_host, cand_host, B, S));
+  SZO_REQUIRE(out3_host != nullptr, SZO_ERR_INVALID_ARG, "out3_host is NULL");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  SZO_CHECK_CUDA(cudaMemcpyAsync(m->d_tokens, tokens_host, static_cast<size_t>(B) * S * sizeof(int32_t),
+                                 cudaMemcpyHostToDevice, st));
+  if (m->cfg.loss_kind == 1) {
+    SZO_CHECK_CUDA(cudaMemcpyAsync(m->d_labels, labels_host, B * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    SZO_CHECK_CUDA(cudaMemcpyAsync(m->d_cand, cand_host, 2 * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+  }
+  SZO_TRY(szo_model_zo_step(m, m->d_tokens, m->d_labels, m->d_cand, B, S, seed, step, eps, lr, m->d_scalars,
+                            m->d_scalars + 1, m->d_scalars + 2, stream));
+  SZO_CHECK_CUDA(cudaMemcpyAsync(out3_host, m->d_scalars, 3 * sizeof(double), cudaMemcpyDeviceToHost, st));
+  SZO_CHECK_CUDA(cudaStreamSynchronize(st));
+  return SZO_OK;
+}
+
+void szo_model_destroy(szo_model_t* m) {
+  if (!m) return;
+  for (szo_linear_t* p : m->plans) szo_linear_destroy(p);
+  szo_linear_destroy(m->lm_head_plan);
+  for (void* p : m->owned) cudaFree(p);
+  delete m;
+}
+
+}  // extern "C"
