@@ -1,0 +1,141 @@
+"""GPU parity of szo_linear_fwd (every mode) against the fp64 oracle on seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import szo_oracle as so
+from paper_2406_02913_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+LINEAR_TOL = 2e-2      # max |y - y_ref| / max |y_ref|, bf16 inputs with fp32 accumulation
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2406_02913_b200 import binding
+    binding.lib()
+    return binding
+
+
+def make_case(N, K, G, fmt, M, rho, seed, bias=False):
+    W = wl.gaussian_matrix(N, K, 0.02, seed=seed, i=1)
+    nnz = int(rho * N * K)
+    g = wl.student_t_gradient(N * K, 3.0, seed=seed, i=2)
+    idx = so.select_mask(g * g, nnz)
+    S, Wd = so.decompose(W, idx)
+    if G > 0:
+        codes, sb, zb = so.quantize_int4(Wd, G, fmt)
+        deq = so.dequantize(codes, sb, zb, G, fmt)
+    else:
+        Wd = wl.bf16_round(Wd)
+        codes, sb, zb, deq = Wd, None, None, Wd.astype(np.float64)
+    x = wl.activation(M, K, seed=seed, i=3)
+    b = wl.rng(seed, wl.PURPOSE_WEIGHTS, 77).normal(0, 0.02, N).astype(np.float32) if bias else None
+    # a perturbed S, as the forward sees it inside a ZO step
+    S_pert = so.perturb(S, idx, 1234, 0, np.float32(1e-3))
+    return dict(N=N, K=K, G=G, fmt=fmt, M=M, idx=idx, S=S_pert, codes=codes, sb=sb, zb=zb, deq=deq, x=x, bias=b)
+
+
+def upload(B, c):
+    dt = torch.bfloat16 if c["fmt"] == "bf16" else torch.float16
+    if c["G"] > 0:
+        codes = torch.from_numpy(c["codes"]).cuda()
+        sc = torch.from_numpy(c["sb"].view(np.int16)).cuda().view(dt)
+        ze = torch.from_numpy(c["zb"].view(np.int16)).cuda().view(dt)
+    else:
+        codes, sc, ze = torch.from_numpy(c["codes"]).cuda().to(torch.bfloat16), None, None
+    idx = torch.from_numpy(c["idx"]).cuda()
+    bias = None if c["bias"] is None else torch.from_numpy(c["bias"]).cuda()
+    plan = B.Linear(c["N"], c["K"], c["G"], codes, sc, ze, c["fmt"], idx, bias)
+    return plan, torch.from_numpy(c["x"]).cuda(), torch.from_numpy(c["S"]).cuda()
+
+
+def max_rel(y, ref):
+    return float(np.max(np.abs(y.astype(np.float64) - ref)) / np.max(np.abs(ref)))
+
+
+CASES = [
+    # N, K, G, fmt, M, rho, bias
+    (256, 256, 64, "f16", 256, 1e-3, False),        # tiny-config q/k/v/o
+    (1024, 256, 64, "f16", 100, 1e-3, False),       # ragged M
+    (256, 1024, 64, "f16", 37, 1e-3, True),
+    (384, 512, 128, "bf16", 300, 1e-2, True),       # several tiles and a ragged tail in M and N
+    (200, 320, 32, "bf16", 65, 5e-3, False),        # N not a multiple of the tile
+    (256, 512, 0, "bf16", 130, 1e-2, False),        # dense bf16 weight (no quantization)
+]
+
+
+@pytest.mark.parametrize("N,K,G,fmt,M,rho,bias", CASES)
+def test_fp32_validation_mode(B, N, K, G, fmt, M, rho, bias):
+    c = make_case(N, K, G, fmt, M, rho, seed=N + K + M, bias=bias)
+    plan, x, S = upload(B, c)
+    ref = so.linear_fwd(c["x"], c["deq"], c["idx"], c["S"], c["bias"])
+    y = plan.fwd(x, S, B.MODE_FP32_VALIDATE, torch.float32).cpu().numpy()
+    assert max_rel(y, ref) < 2e-6
+    y16 = plan.fwd(x.to(torch.bfloat16), S, B.MODE_FP32_VALIDATE, torch.bfloat16).float().cpu().numpy()
+    assert max_rel(y16, ref) < 4e-3                                    # only the output rounding
+    plan.close()
+
+
+@pytest.mark.parametrize("N,K,G,fmt,M,rho,bias", CASES)
+@pytest.mark.parametrize("mode", ["sparse_add", "spmm"])
+def test_tensor_core_modes(B, N, K, G, fmt, M, rho, bias, mode):
+    c = make_case(N, K, G, fmt, M, rho, seed=N + K + M, bias=bias)
+    plan, x, S = upload(B, c)
+    ref = so.linear_fwd(c["x"], c["deq"], c["idx"], c["S"], c["bias"])
+    md = B.MODE_SPARSE_ADD if mode == "sparse_add" else B.MODE_SPMM
+    xb = x.to(torch.bfloat16)
+    y = plan.fwd(xb, S, md, torch.float32).cpu().numpy()
+    assert max_rel(y, ref) < LINEAR_TOL
+    assert max_rel(y, ref) < 5e-3          # in practice: bf16 weight rounding only
+    yb = plan.fwd(xb, S, md, torch.bfloat16).float().cpu().numpy()
+    assert max_rel(yb, ref) < LINEAR_TOL
+    # determinism: bitwise-same output on a second launch
+    y2 = plan.fwd(xb, S, md, torch.float32).cpu().numpy()
+    assert np.array_equal(y, y2)
+    assert B.device_status() == 0
+    plan.close()
+
+
+def test_special_cases_identity_input_and_sparse_only(B):
+    # x = I returns W_eff^T tile by tile (exposes layout mistakes); zero codes leave the sparse term
+    N, K, G = 256, 256, 64
+    c = make_case(N, K, G, "bf16", K, 2e-3, seed=5)
+    c["x"] = np.eye(K, dtype=np.float32)
+    plan, x, S = upload(B, c)
+    Weff = so.effective_weight(c["deq"], c["idx"], c["S"])
+    for md in (B.MODE_FP32_VALIDATE, B.MODE_SPARSE_ADD, B.MODE_SPMM):
+        y = plan.fwd(x.to(torch.bfloat16), S, md, torch.float32).cpu().numpy()
+        tol = 1e-6 if md == B.MODE_FP32_VALIDATE else 2.0 ** -8
+        assert np.max(np.abs(y - Weff.T)) <= tol * np.max(np.abs(Weff))
+    plan.close()
+    zc = dict(c)
+    zc["codes"] = np.zeros_like(c["codes"])
+    zc["sb"] = np.zeros_like(c["sb"])
+    zc["zb"] = np.zeros_like(c["zb"])
+    zc["x"] = wl.activation(64, K, seed=6)
+    plan, x, S = upload(B, zc)
+    ref = so.linear_fwd(zc["x"], np.zeros((N, K)), c["idx"], c["S"])
+    for md in (B.MODE_FP32_VALIDATE, B.MODE_SPARSE_ADD, B.MODE_SPMM):
+        y = plan.fwd(x.to(torch.bfloat16), S, md, torch.float32).cpu().numpy()
+        assert max_rel(y, ref) < (1e-5 if md != B.MODE_SPARSE_ADD else 5e-3)
+    plan.close()
+
+
+def test_linear_argument_errors(B):
+    c = make_case(64, 128, 64, "bf16", 8, 1e-2, seed=9)
+    plan, x, S = upload(B, c)
+    with pytest.raises(B.SzoError) as ei:
+        plan.fwd(x, S, B.MODE_SPARSE_ADD, torch.float32)               # fp32 x outside validation
+    assert ei.value.name == "SZO_ERR_UNSUPPORTED"
+    bad = torch.from_numpy(c["idx"][::-1].copy()).cuda()
+    with pytest.raises(B.SzoError) as ei:
+        B.Linear(64, 128, 64, plan._keep[0], plan._keep[1], plan._keep[2], "bf16", bad)
+    assert ei.value.name == "SZO_ERR_INVALID_ARG"
+    with pytest.raises(B.SzoError) as ei:
+        B.Linear(64, 100, 0, plan._keep[0], None, None, "bf16", None)
+    assert ei.value.name == "SZO_ERR_SHAPE"
+    y = plan.fwd(x[:0].to(torch.bfloat16), S, B.MODE_SPARSE_ADD, torch.float32)     # M = 0
+    assert y.shape == (0, 64)
+    plan.close()

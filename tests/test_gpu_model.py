@@ -1,0 +1,153 @@
+"""GPU parity of the whole loss path and ZO step (szo_model_*) against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import model_oracle as mo
+from oracle import szo_oracle as so
+from paper_2406_02913_b200 import workloads as wl
+from tests.fixtures import DecoderFixture
+
+pytestmark = pytest.mark.gpu
+
+LOSS_TOL = 1e-3        # relative, bf16 tensor-core path
+G_TOL = 1e-3           # relative, projected gradient in the fp32 validation mode
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2406_02913_b200 import binding
+    binding.lib()
+    return binding
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    return DecoderFixture("tiny", seed=0, mask="gradient", B=4, S=64)
+
+
+def build_gpu(B, fx, act, mode, loss_kind=0, quantize_on_gpu=True):
+    qfun = (lambda W, G, fmt: B.szo_quantize(W, G, fmt)) if quantize_on_gpu else None
+    t = fx.gpu_tensors(torch, qfun)
+    S = torch.from_numpy(fx.S_init.copy()).cuda()
+    m = B.Model(fx.shape, fx.names, t, S, act_dtype=act, linear_mode=mode, loss_kind=loss_kind,
+                max_batch=fx.B, max_seq=fx.S)
+    return m, S, t
+
+
+def test_fixture_mask_and_codes_reproduced_by_the_library(B, tiny):
+    """The library's own select_mask and quantize give the oracle's mask and codes bit for bit
+    on the tiny decoder (k = floor(1e-3 n) per tensor from 4 accumulated squared gradients)."""
+    fx = tiny
+    assert len(fx.S_init) == 2092
+    for l in range(fx.shape["n_layers"]):
+        for nm in fx.names:
+            sc = torch.from_numpy(fx.scores[l][nm].ravel()).cuda()
+            k = len(fx.idx[l][nm])
+            assert np.array_equal(B.szo_select_mask(sc, k).cpu().numpy(), fx.idx[l][nm])
+            codes, sb, zb = fx.q[l][nm]
+            gc, gs, gz = B.szo_quantize(torch.from_numpy(fx.W_dense[l][nm]).cuda(), fx.shape["group"], fx.shape["sz_fmt"])
+            assert np.array_equal(gc.cpu().numpy(), codes)
+            assert np.array_equal(gs.cpu().view(torch.int16).numpy().view(np.uint16), sb)
+            assert np.array_equal(gz.cpu().view(torch.int16).numpy().view(np.uint16), zb)
+
+
+def test_model_gidx_matches_model_order(B, tiny):
+    m, S, _ = build_gpu(B, tiny, B.SZO_F32, B.MODE_FP32_VALIDATE)
+    assert m.k_total == len(tiny.gidx)
+    assert np.array_equal(m.gidx().cpu().numpy(), tiny.gidx)
+    m.close()
+
+
+def test_loss_fp32_validation_matches_oracle(B, tiny):
+    fx = tiny
+    m, S, _ = build_gpu(B, fx, B.SZO_F32, B.MODE_FP32_VALIDATE)
+    om = fx.oracle_model()
+    for i in range(2):
+        toks = fx.batch(i)
+        ref = om.loss(om.S, toks)
+        got = m.loss(torch.from_numpy(toks).cuda()).item()
+        assert abs(got - ref) <= 2e-6 * abs(ref)
+    m.close()
+
+
+def test_ten_zo_steps_fp32_validation(B, tiny):
+    """Config 1: 10 ZO-SGD steps, eps 1e-3, lr 1e-5, Philox seed 1234; per-step f+, f-, g and the
+    final S against the oracle."""
+    fx = tiny
+    m, S, _ = build_gpu(B, fx, B.SZO_F32, B.MODE_FP32_VALIDATE)
+    om = fx.oracle_model()
+    frozen = {k: v.clone() for k, v in m.tensors.items()}
+    eps, lr = 1e-3, 1e-5
+    for step in range(10):
+        toks = fx.batch(step)
+        fp, fm, g = mo.zo_step(om, toks, 1234, step, eps, lr)
+        out = m.zo_step(torch.from_numpy(toks).cuda(), 1234, step, eps, lr).cpu().numpy()
+        assert abs(out[0] - fp) <= 2e-6 * abs(fp) and abs(out[1] - fm) <= 2e-6 * abs(fm)
+        # g amplifies the loss error by f / (f+ - f-); the bound is relative to the gradient scale
+        assert abs(out[2] - g) <= G_TOL * max(abs(g), 1e-2), (step, out[2], g)
+    assert np.allclose(S.cpu().numpy(), om.S, rtol=0, atol=2e-7)
+    assert m.last_launches() > 0
+    for k, v in frozen.items():                      # frozen parts are bit-identical after the steps
+        assert torch.equal(v, m.tensors[k]), k
+    assert B.device_status() == 0
+    m.close()
+
+
+@pytest.mark.parametrize("name,loss_kind", [("tiny_opt", 0), ("tiny_gqa", 1)])
+def test_other_architectures_fp32_validation(B, name, loss_kind):
+    fx = DecoderFixture(name, seed=1, mask="random", B=3, S=32)
+    m, S, _ = build_gpu(B, fx, B.SZO_F32, B.MODE_FP32_VALIDATE, loss_kind, quantize_on_gpu=fx.shape["group"] > 0)
+    om = fx.oracle_model()
+    toks = fx.batch(0)
+    kind = "lm" if loss_kind == 0 else "cls2"
+    labels = wl.binary_labels(fx.B, 1, 0)
+    cand = np.array([11, 301], np.int32)
+    ref = om.loss(om.S, toks, kind, labels, cand)
+    d = lambda a: torch.from_numpy(a).cuda()
+    got = m.loss(d(toks), d(labels), d(cand)).item()
+    assert abs(got - ref) <= 3e-6 * abs(ref)
+    fp, fm, g = mo.zo_step(om, toks, 7, 3, 1e-3, 1e-4, kind, labels, cand)
+    out = m.zo_step(d(toks), 7, 3, 1e-3, 1e-4, d(labels), d(cand)).cpu().numpy()
+    assert abs(out[0] - fp) <= 3e-6 * abs(fp) and abs(out[1] - fm) <= 3e-6 * abs(fm)
+    assert abs(out[2] - g) <= G_TOL * max(abs(g), 1e-2)
+    assert np.allclose(S.cpu().numpy(), om.S, rtol=0, atol=2e-7)
+    m.close()
+
+
+@pytest.mark.parametrize("mode", ["sparse_add", "spmm"])
+def test_bf16_tensor_core_path_losses(B, tiny, mode):
+    fx = tiny
+    md = B.MODE_SPARSE_ADD if mode == "sparse_add" else B.MODE_SPMM
+    m, S, _ = build_gpu(B, fx, B.SZO_BF16, md)
+    om = fx.oracle_model()
+    for step in range(3):
+        toks = fx.batch(step)
+        fp, fm, g = mo.zo_step(om, toks, 1234, step, 1e-3, 1e-5)
+        out = m.zo_step(torch.from_numpy(toks).cuda(), 1234, step, 1e-3, 1e-5).cpu().numpy()
+        assert abs(out[0] - fp) <= LOSS_TOL * abs(fp) and abs(out[1] - fm) <= LOSS_TOL * abs(fm)
+        assert np.isfinite(out[2])
+        om.S = S.cpu().numpy().copy()      # follow the GPU's own trajectory (g differs at bf16)
+    assert B.device_status() == 0
+    m.close()
+
+
+def test_host_buffer_step_equals_device_step(B, tiny):
+    fx = tiny
+    m1, S1, _ = build_gpu(B, fx, B.SZO_F32, B.MODE_FP32_VALIDATE)
+    m2, S2, _ = build_gpu(B, fx, B.SZO_F32, B.MODE_FP32_VALIDATE)
+    toks = fx.batch(0)
+    a = m1.zo_step(torch.from_numpy(toks).cuda(), 1, 0, 1e-3, 1e-5).cpu().numpy()
+    b = m2.zo_step_host(torch.from_numpy(toks).pin_memory(), 1, 0, 1e-3, 1e-5)
+    assert tuple(a) == tuple(b) and torch.equal(S1, S2)
+    m1.close()
+    m2.close()
+
+
+def test_model_argument_errors(B, tiny):
+    m, S, _ = build_gpu(B, tiny, B.SZO_F32, B.MODE_FP32_VALIDATE)
+    toks = torch.zeros((tiny.B + 1, tiny.S), dtype=torch.int32, device="cuda")
+    with pytest.raises(B.SzoError) as ei:
+        m.loss(toks)
+    assert ei.value.name == "SZO_ERR_SHAPE"
+    m.close()
