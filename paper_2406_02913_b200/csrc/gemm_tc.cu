@@ -1,17 +1,532 @@
-// Tensor-core path of the decomposed linear layer (placeholder until the tcgen05 kernel lands).
+// Tensor-core path of the decomposed linear layer for sm_100a:
+//   y[m, n] = sum_k x[m,k] * (Dequantize(Q)[n,k] + S[n,k]) + bias[n]
+// as one persistent, warp-specialised tcgen05 kernel (appendix "Implementation of Sparse Operations
+// in Linear Layers": DenseMM(SparseAdd(w_sparse, Dequantize(Q(w_dense))), x)).
+//
+// Orientation: the WEIGHT is the MMA's A operand (128 rows of W per tile = UMMA M), the tokens are
+// the N dimension (BT <= 256 per tile).  A weight element is therefore dequantised once per
+// 2*BT flops, and the accumulator D[n, m] sits in TMEM with one output feature per lane.
+//
+// Per CTA (one per SM, static round-robin over tiles):
+//   warp 0       TMA producer: x tile [BT x 64] bf16 (and the bf16 weight tile in dense mode) with
+//                the 128-byte swizzle, completion on full[s]
+//   warp 1       allocates TMEM, issues tcgen05.mma (one thread), commits to empty[s] / acc_full
+//   warps 4-11   weight producers: int4 codes -> bf16 (q*scale+zero) written in the swizzled K-major
+//                layout the MMA descriptor expects, then the tile's sparse values are added in shared
+//                memory (SparseAdd), fence.proxy.async, arrive on a_ready[s]
+//   warps 12-15  epilogue: tcgen05.ld of the fp32 accumulator, + bias, store y; double-buffered
+//                accumulator so the next tile's main loop overlaps
+// Every mbarrier wait is bounded; on expiry the kernel records SZO_ERR_TIMEOUT in the device status
+// word, lets in-flight copies land, frees its TMEM and returns.
+#include <cuda.h>
+
 #include "linear.cuh"
 
 namespace szo {
 
-szo_status tc_plan_create(szo_linear* p, cudaStream_t) {
-  p->tc = nullptr;
+namespace {
+
+constexpr int kBM = 128;           // weight rows per tile (UMMA M)
+constexpr int kBK = 64;            // K per stage: 64 bf16 = one 128-byte swizzle row
+constexpr int kUmmaK = 16;
+constexpr int kNumWarps = 16;
+constexpr int kDeqWarp0 = 4, kNumDeqWarps = 8;
+constexpr int kEpiWarp0 = 12;
+constexpr int kATileBytes = kBM * kBK * 2;   // 16 KiB
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
+
+struct TcParams {
+  int64_t M, N, K;
+  int G;
+  int nkb;                 // K / 64
+  int64_t m_tiles, n_tiles;
+  const uint8_t* codes;    // [N, K/2]
+  const float2* sz;        // [N, K/G]
+  const int32_t* bucket_ptr;
+  const int32_t* bucket_eid;
+  const uint16_t* bucket_pos;
+  int64_t n_kblocks;       // buckets per row group
+  int64_t n_rowgroups;
+  const float* S;          // sparse values (nullptr: no SparseAdd)
+  const float* bias;
+  void* y;
+  int y_f32;
+  int32_t* status;
+};
+
+// ------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: false when the limit expired or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  while (true) {
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > kWaitLimitNs) {
+      *abort_flag = 1;
+      atomicExch(status, static_cast<int32_t>(SZO_ERR_TIMEOUT));
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t result_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(result_smem), "r"(ncols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor: K-major tile whose rows are 128 bytes, 128-byte swizzle,
+// 8-row groups 1024 bytes apart (SBO), descriptor version 1, layout type 2 (SWIZZLE_128B).
+__device__ __forceinline__ uint64_t make_desc_sw128(uint32_t smem_addr) {
+  return static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | (static_cast<uint64_t>(1024 >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor, kind::f16: fp32 accumulate, bf16 x bf16, both operands K-major.
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// Eight codes of one 32-bit word -> eight bf16 values q*scale+zero (one rounding each).
+template <bool kFast>
+__device__ __forceinline__ uint4 dequant_word(uint32_t w, float2 p) {
+  uint32_t o[4];
+  if constexpr (kFast) {
+    // scale and zero are bf16 values: exact packed arithmetic.  (128+q) as bf16 is 0x4300|q.
+    const __nv_bfloat162 s2 = __floats2bfloat162_rn(p.x, p.x), z2 = __floats2bfloat162_rn(p.y, p.y);
+    const uint32_t magic = 0x43004300u;
+    const __nv_bfloat162 m2 = *reinterpret_cast<const __nv_bfloat162*>(&magic);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t x = w >> (8 * i);
+      const uint32_t t = (x & 0xFu) | ((x << 12) & 0xF0000u) | magic;
+      const __nv_bfloat162 q2 = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&t), m2);
+      const __nv_bfloat162 r = __hfma2(q2, s2, z2);
+      o[i] = *reinterpret_cast<const uint32_t*>(&r);
+    }
+  } else {
+    float f[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const float q = __uint_as_float(0x4B000000u | ((w >> (4 * e)) & 0xFu)) - 8388608.0f;
+      f[e] = fmaf(q, p.x, p.y);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) o[i] = pack_bf16x2(f[2 * i], f[2 * i + 1]);
+  }
+  return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// ------------------------------------------------------------------------------ the kernel
+// kDequant: A tile produced from int4 codes (else loaded as bf16 by TMA).  kFast: bf16 scales/zeros.
+template <int BT, int kStages, bool kDequant, bool kFast>
+__global__ void __launch_bounds__(kNumWarps * 32, 1)
+szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                     const TcParams P) {
+  constexpr int kBTileBytes = BT * kBK * 2;
+  constexpr int kStageBytes = kATileBytes + kBTileBytes;
+  constexpr int kAccStride = BT < 32 ? 32 : BT;             // TMEM columns per accumulator buffer
+  constexpr uint32_t kTmemCols = static_cast<uint32_t>(2 * kAccStride);
+  constexpr uint32_t kIdesc = make_idesc(kBM, BT);
+
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) unsigned long long bars[3 * kStages + 4];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag_s;
+
+  const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  unsigned char* tiles_ptr = smem_raw + (tiles_base - smem_u32(smem_raw));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile int* abort_flag = &abort_flag_s;
+
+  auto full_bar = [&](int s) { return smem_u32(&bars[s]); };
+  auto aready_bar = [&](int s) { return smem_u32(&bars[kStages + s]); };
+  auto empty_bar = [&](int s) { return smem_u32(&bars[2 * kStages + s]); };
+  auto accfull_bar = [&](int a) { return smem_u32(&bars[3 * kStages + a]); };
+  auto accempty_bar = [&](int a) { return smem_u32(&bars[3 * kStages + 2 + a]); };
+  auto a_tile = [&](int s) { return tiles_base + static_cast<uint32_t>(s) * kStageBytes; };
+  auto b_tile = [&](int s) { return tiles_base + static_cast<uint32_t>(s) * kStageBytes + kATileBytes; };
+
+  const bool a_proc = kDequant || (P.S != nullptr);   // weight-producer warps take part
+  if (threadIdx.x == 0) {
+    abort_flag_s = 0;
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(aready_bar(s), kNumDeqWarps);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(accfull_bar(a), 1);
+      mbar_init(accempty_bar(a), 4);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  const int64_t total_tiles = P.m_tiles * P.n_tiles;
+  const int64_t my_tiles = (total_tiles > blockIdx.x) ? (total_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+  const int64_t my_iters = my_tiles * P.nkb;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      for (int64_t it = 0; it < my_iters; ++it) {
+        const int64_t tile = blockIdx.x + (it / P.nkb) * gridDim.x;
+        const int kb = static_cast<int>(it % P.nkb);
+        const int64_t n_tile = tile / P.m_tiles, m_tile = tile % P.m_tiles;
+        const int s = static_cast<int>(it % kStages);
+        const uint32_t ph = static_cast<uint32_t>((it / kStages) & 1);
+        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, P.status)) break;
+        mbar_expect_tx(full_bar(s), kDequant ? kBTileBytes : kStageBytes);
+        tma_load_2d(b_tile(s), &tmap_x, kb * kBK, static_cast<int>(m_tile * BT), full_bar(s));
+        if constexpr (!kDequant) tma_load_2d(a_tile(s), &tmap_w, kb * kBK, static_cast<int>(n_tile * kBM), full_bar(s));
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      bool ok = true;
+      for (int64_t lt = 0; lt < my_tiles && ok; ++lt) {
+        const int as = static_cast<int>(lt & 1);
+        const uint32_t aph = static_cast<uint32_t>((lt >> 1) & 1);
+        if (!mbar_wait(accempty_bar(as), aph ^ 1u, abort_flag, P.status)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kAccStride);
+        for (int kb = 0; kb < P.nkb; ++kb) {
+          const int64_t it = lt * P.nkb + kb;
+          const int s = static_cast<int>(it % kStages);
+          const uint32_t ph = static_cast<uint32_t>((it / kStages) & 1);
+          if (!mbar_wait(full_bar(s), ph, abort_flag, P.status)) { ok = false; break; }
+          if (a_proc && !mbar_wait(aready_bar(s), ph, abort_flag, P.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t adesc = make_desc_sw128(a_tile(s)), bdesc = make_desc_sw128(b_tile(s));
+#pragma unroll
+          for (int k = 0; k < kBK / kUmmaK; ++k) {
+            // advance both descriptors by 16 elements = 32 bytes (>> 4 = 2) inside the swizzle row
+            umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc, (kb | k) ? 1u : 0u);
+          }
+          umma_commit(empty_bar(s));
+        }
+        if (ok) umma_commit(accfull_bar(as));
+      }
+    }
+  } else if (warp >= kDeqWarp0 && warp < kDeqWarp0 + kNumDeqWarps) {
+    // ---------------------------------------------------------------- weight producers
+    if (a_proc) {
+      const int dw = warp - kDeqWarp0;             // rows [16 dw, 16 dw + 16) of the tile
+      const int sub = lane >> 3, chunk = lane & 7; // 4 rows x 8 sixteen-byte chunks per pass
+      const int64_t words_per_row = P.K / 8;
+      const int groups_per_row = kDequant ? static_cast<int>(P.K / P.G) : 1;
+      uint32_t cw[4] = {0u, 0u, 0u, 0u};
+      auto load_codes = [&](int64_t it, uint32_t (&dst)[4]) {
+        const int64_t tile = blockIdx.x + (it / P.nkb) * gridDim.x;
+        const int kb = static_cast<int>(it % P.nkb);
+        const int64_t n0 = (tile / P.m_tiles) * kBM;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int64_t n = n0 + dw * 16 + i * 4 + sub;
+          dst[i] = (n < P.N) ? __ldg(reinterpret_cast<const uint32_t*>(P.codes) + n * words_per_row + kb * 8 + chunk) : 0u;
+        }
+      };
+      if constexpr (kDequant) {
+        if (my_iters > 0) load_codes(0, cw);
+      }
+      for (int64_t it = 0; it < my_iters; ++it) {
+        const int64_t tile = blockIdx.x + (it / P.nkb) * gridDim.x;
+        const int kb = static_cast<int>(it % P.nkb);
+        const int64_t n0 = (tile / P.m_tiles) * kBM;
+        const int s = static_cast<int>(it % kStages);
+        const uint32_t ph = static_cast<uint32_t>((it / kStages) & 1);
+        unsigned char* A = tiles_ptr + static_cast<size_t>(s) * kStageBytes;
+        if constexpr (kDequant) {
+          uint32_t cn[4] = {0u, 0u, 0u, 0u};
+          if (it + 1 < my_iters) load_codes(it + 1, cn);
+          float2 sz[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int64_t n = n0 + dw * 16 + i * 4 + sub;
+            sz[i] = (n < P.N) ? __ldg(P.sz + n * groups_per_row + (kb * kBK + chunk * 8) / P.G) : make_float2(0.f, 0.f);
+          }
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, P.status)) break;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int r = dw * 16 + i * 4 + sub;
+            const uint4 v = dequant_word<kFast>(cw[i], sz[i]);
+            *reinterpret_cast<uint4*>(A + r * 128 + ((chunk ^ (r & 7)) << 4)) = v;
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) cw[i] = cn[i];
+        } else {
+          if (!mbar_wait(full_bar(s), ph, abort_flag, P.status)) break;   // TMA wrote the bf16 tile
+        }
+        if (P.S != nullptr) {
+          __syncwarp();
+          // SparseAdd: entries of bucket (row group, k-block) that fall in this warp's 16 rows
+          const int64_t rg = (n0 >> 5) + (dw >> 1);
+          const int64_t b = rg * P.n_kblocks + kb;
+          int32_t e0 = 0, e1 = 0;
+          if (rg < P.n_rowgroups) {
+            e0 = __ldg(P.bucket_ptr + b);
+            e1 = __ldg(P.bucket_ptr + b + 1);
+          }
+          for (int32_t e = e0 + lane; e < e1; e += 32) {
+            const uint32_t pos = __ldg(P.bucket_pos + e);
+            const int lr = static_cast<int>(pos >> 6), lc = static_cast<int>(pos & 63);
+            if ((lr >> 4) == (dw & 1)) {
+              const int r = (dw >> 1) * 32 + lr;
+              __nv_bfloat16* el = reinterpret_cast<__nv_bfloat16*>(A + r * 128 + (((lc >> 3) ^ (r & 7)) << 4) + (lc & 7) * 2);
+              *el = __float2bfloat16_rn(__bfloat162float(*el) + __ldg(P.S + __ldg(P.bucket_eid + e)));
+            }
+          }
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(aready_bar(s));
+      }
+    }
+  } else if (warp >= kEpiWarp0) {
+    // ---------------------------------------------------------------- epilogue
+    const int qd = warp & 3;                        // TMEM lane quarter this warp may read
+    for (int64_t lt = 0; lt < my_tiles; ++lt) {
+      const int64_t tile = blockIdx.x + lt * gridDim.x;
+      const int64_t n_tile = tile / P.m_tiles, m_tile = tile % P.m_tiles;
+      const int as = static_cast<int>(lt & 1);
+      const uint32_t aph = static_cast<uint32_t>((lt >> 1) & 1);
+      if (!mbar_wait(accfull_bar(as), aph, abort_flag, P.status)) break;
+      tc_fence_after();
+      const int64_t n = n_tile * kBM + qd * 32 + lane;
+      const float bias = (P.bias != nullptr && n < P.N) ? P.bias[n] : 0.f;
+      const int64_t m0 = m_tile * BT;
+      for (int c0 = 0; c0 < BT; c0 += 32) {
+        uint32_t v[32];
+        tmem_ld32(tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + static_cast<uint32_t>(as * kAccStride + c0), v);
+        if (n < P.N) {
+          if (P.y_f32) {
+            float* y = static_cast<float*>(P.y);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int64_t m = m0 + c0 + j;
+              if (c0 + j < BT && m < P.M) y[m * P.N + n] = __uint_as_float(v[j]) + bias;
+            }
+          } else {
+            __nv_bfloat16* y = static_cast<__nv_bfloat16*>(P.y);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int64_t m = m0 + c0 + j;
+              if (c0 + j < BT && m < P.M) y[m * P.N + n] = __float2bfloat16_rn(__uint_as_float(v[j]) + bias);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(accempty_bar(as));
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  if (*abort_flag) {
+    // a wait expired somewhere: give copies and MMAs in flight time to land before the CTA exits
+    for (int i = 0; i < 200; ++i) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// ------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 matrix [rows, cols] row-major, box [box_rows x 64 cols], 128-byte swizzle, zero fill.
+szo_status make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  SZO_REQUIRE(fn != nullptr, SZO_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols) * 2};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBK), static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  SZO_REQUIRE(r == CUDA_SUCCESS, SZO_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", static_cast<int>(r));
   return SZO_OK;
 }
 
-void tc_plan_destroy(szo_linear* p) { p->tc = nullptr; }
+struct TcPlan {
+  CUtensorMap w_map;    // dense bf16 weight (G == 0)
+  bool has_w_map;
+  int sms;
+};
 
-szo_status linear_fwd_tc(const szo_linear*, const void*, int64_t, const float*, void*, int, bool, cudaStream_t) {
-  return fail(SZO_ERR_UNSUPPORTED, "tensor-core path not built");
+template <int BT, int kStages, bool kDequant, bool kFast>
+szo_status launch_tc(const CUtensorMap& mx, const CUtensorMap& mw, const TcParams& P, int sms, cudaStream_t st) {
+  constexpr size_t smem = static_cast<size_t>(kStages) * (kATileBytes + BT * kBK * 2) + 1024;
+  auto kern = szo_linear_tc_kernel<BT, kStages, kDequant, kFast>;
+  static bool configured = false;
+  if (!configured) {
+    SZO_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    configured = true;
+  }
+  const int64_t tiles = P.m_tiles * P.n_tiles;
+  const unsigned grid = static_cast<unsigned>(tiles < sms ? tiles : sms);
+  kern<<<grid, kNumWarps * 32, smem, st>>>(mx, mw, P);
+  count_launch();
+  SZO_CHECK_LAUNCH("szo_linear_tc_kernel");
+  return SZO_OK;
+}
+
+template <int BT, int kStages>
+szo_status dispatch_kind(const szo_linear* p, const CUtensorMap& mx, const CUtensorMap& mw, const TcParams& P, int sms,
+                         cudaStream_t st) {
+  if (p->G == 0) return launch_tc<BT, kStages, false, false>(mx, mw, P, sms, st);
+  if (p->sz_dtype == SZO_BF16) return launch_tc<BT, kStages, true, true>(mx, mw, P, sms, st);
+  return launch_tc<BT, kStages, true, false>(mx, mw, P, sms, st);
+}
+
+}  // namespace
+
+szo_status tc_plan_create(szo_linear* p, cudaStream_t) {
+  TcPlan* t = new TcPlan();
+  t->has_w_map = false;
+  int dev = 0;
+  t->sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&t->sms, cudaDevAttrMultiProcessorCount, dev);
+  if (p->G == 0) {
+    const szo_status s = make_map(&t->w_map, p->codes, p->N, p->K, kBM);
+    if (s != SZO_OK) {
+      delete t;
+      return s;
+    }
+    t->has_w_map = true;
+  }
+  p->tc = t;
+  return SZO_OK;
+}
+
+void tc_plan_destroy(szo_linear* p) {
+  delete static_cast<TcPlan*>(p->tc);
+  p->tc = nullptr;
+}
+
+szo_status linear_fwd_tc(const szo_linear* p, const void* x, int64_t M, const float* S, void* y, int y_dtype,
+                         bool sparse_add, cudaStream_t st) {
+  const TcPlan* t = static_cast<const TcPlan*>(p->tc);
+  SZO_REQUIRE(t != nullptr, SZO_ERR_INVALID_ARG, "plan has no tensor-core data");
+  SZO_REQUIRE(M < (int64_t(1) << 31) && p->N < (int64_t(1) << 31), SZO_ERR_SHAPE, "M or N too large");
+  int BT = 256;
+  if (M <= 16) BT = 16; else if (M <= 32) BT = 32; else if (M <= 64) BT = 64; else if (M <= 128) BT = 128;
+  CUtensorMap mx;
+  SZO_TRY(make_map(&mx, x, M, p->K, BT));
+  TcParams P{};
+  P.M = M; P.N = p->N; P.K = p->K; P.G = p->G; P.nkb = static_cast<int>(p->K / kBK);
+  P.m_tiles = ceil_div(M, BT); P.n_tiles = ceil_div(p->N, kBM);
+  P.codes = static_cast<const uint8_t*>(p->codes);
+  P.sz = p->sz;
+  P.bucket_ptr = p->bucket_ptr; P.bucket_eid = p->bucket_eid; P.bucket_pos = p->bucket_pos;
+  P.n_kblocks = p->n_kblocks;
+  P.n_rowgroups = p->n_rowgroups;
+  P.S = (sparse_add && p->nnz > 0) ? S : nullptr;
+  P.bias = p->bias;
+  P.y = y; P.y_f32 = (y_dtype == SZO_F32) ? 1 : 0;
+  P.status = device_status_word();
+  SZO_REQUIRE(P.status != nullptr, SZO_ERR_CUDA, "no device status word");
+  const CUtensorMap& mw = t->has_w_map ? t->w_map : mx;   // unused by the kernel when dequantising
+  switch (BT) {
+    case 16: return dispatch_kind<16, 6>(p, mx, mw, P, t->sms, st);
+    case 32: return dispatch_kind<32, 6>(p, mx, mw, P, t->sms, st);
+    case 64: return dispatch_kind<64, 6>(p, mx, mw, P, t->sms, st);
+    case 128: return dispatch_kind<128, 6>(p, mx, mw, P, t->sms, st);
+    default: return dispatch_kind<256, 4>(p, mx, mw, P, t->sms, st);
+  }
 }
 
 }  // namespace szo
