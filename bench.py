@@ -1,0 +1,289 @@
+#!/usr/bin/env python
+"""Benchmark: sensitive-sparse ZO-SGD steps per second on a Llama-2-7B-shaped 4-bit decoder.
+
+One step = +eps perturb, forward, -2eps perturb, forward, restore, projected gradient, update, all
+through the C ABI (szo_model_zo_step).  Prints ONE JSON line (rank 0).
+
+    python bench.py --gpus 1 --steps 5 --warmup 3
+    python bench.py --impl reference          # the CPU oracle on a bounded sample of the same work
+
+Multi-GPU: the step does not shard (one GPU holds the whole model and nothing is exchanged), so
+--gpus N runs N independent replicas, one process per GPU, and reports their aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+WORKLOAD = "llama2_7b"
+BATCH, SEQ = 16, 256
+EPS, LR, SEED = 1e-3, 1e-6, 1234
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self._stop = index, [], threading.Event()
+        self._t = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
+                parts = [p.strip() for p in out.strip().split(",")]
+                if len(parts) >= 6:
+                    self.rows.append(parts)
+            except Exception:
+                pass
+            self._stop.wait(0.2)
+
+    def __enter__(self):
+        self._t.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._t.join(timeout=6)
+
+    def summary(self):
+        if not self.rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
+        sm = [float(r[0]) for r in self.rows if r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[2 + i].lower().startswith("active") for r in self.rows)]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(self.rows)}
+
+
+def linear_flops_per_forward(shape, M):
+    from paper_2406_02913_b200 import workloads as wl
+    per_layer = sum(2 * M * n * k for n, k in (wl.linear_shape(shape, nm) for nm in wl.linear_names(shape)))
+    return per_layer * shape["n_layers"]
+
+
+# ------------------------------------------------------------------------------------ oracle leg
+def oracle_sample(shape, tokens_sample=32, k_sample=500_000):
+    """Times the CPU oracle, as it stands, on a bounded sample of the step: the seven linears of one
+    decoder layer (dequantize, add the sparse values, fp64 product) for `tokens_sample` tokens, and
+    one sparse perturb pass over `k_sample` entries.  Extrapolated to a whole step by the layer
+    count, the token count and the total k."""
+    import numpy as np
+    from oracle import szo_oracle as so
+    from paper_2406_02913_b200 import workloads as wl
+
+    G, fmt = shape["group"], shape["sz_fmt"]
+    t_lin, t_prep = 0.0, 0.0
+    for j, nm in enumerate(wl.linear_names(shape)):
+        N, K = wl.linear_shape(shape, nm)
+        codes = wl.random_codes(N, K, seed=1, i=j)
+        sc = (0.004 + 0.002 * wl.rng(1, wl.PURPOSE_WEIGHTS, 50 + j).random((N, K // G))).astype(np.float32)
+        sb, scv = so.round_to_16(sc, fmt)
+        zb, _ = so.round_to_16(-7.5 * scv, fmt)
+        idx = wl.sorted_random_indices(N * K, int(shape["rho"] * N * K), seed=1, i=j)
+        S = wl.rng(1, wl.PURPOSE_WEIGHTS, 80 + j).normal(0, 0.02, idx.size).astype(np.float32)
+        x = wl.activation(tokens_sample, K, seed=1, i=j)
+        t0 = time.perf_counter()
+        deq = so.dequantize(codes, sb, zb, G, fmt)
+        t1 = time.perf_counter()
+        so.effective_weight(deq, idx, S)
+        t2 = time.perf_counter()
+        so.linear_fwd(x, deq, idx, S)
+        t3 = time.perf_counter()
+        t_prep += (t1 - t0) + (t2 - t1)
+        t_lin += max((t3 - t2) - (t2 - t1), 0.0)
+    gidx = wl.sorted_random_indices(6_476_005_376, k_sample, seed=2)
+    Sv = np.zeros(k_sample, np.float32)
+    t0 = time.perf_counter()
+    so.perturb(Sv, gidx, SEED, 0, np.float32(EPS))
+    t_pert = time.perf_counter() - t0
+    M = BATCH * SEQ
+    d_lin = sum(n * k for n, k in (wl.linear_shape(shape, nm) for nm in wl.linear_names(shape))) * shape["n_layers"]
+    k_total = int(shape["rho"] * d_lin)
+    # the weight preparation (dequantize, add the sparse values) does not depend on the token count;
+    # the fp64 product does
+    step_s = 2 * shape["n_layers"] * (t_prep + t_lin * (M / tokens_sample)) + 4 * t_pert * (k_total / k_sample)
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
+    sample = (f"one decoder layer's 7 linears: weight preparation {t_prep:.2f} s + fp64 product at {tokens_sample} "
+              f"tokens {t_lin:.2f} s; one perturb pass over "
+              f"{k_sample} entries ({t_pert:.2f} s); extrapolated x{shape['n_layers']} layers x2 forwards, product "
+              f"x{M // tokens_sample} token blocks, + 4 passes over k={k_total}; attention and norms not included")
+    return dict(value=1.0 / step_s, unit="steps/s", cores=cores, kind="oracle", sample=sample), step_s
+
+
+def run_reference(args):
+    from paper_2406_02913_b200 import workloads as wl
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    shape = wl.MODEL_SHAPES[WORKLOAD]
+    vals = []
+    for i in range(args.warmup + args.steps):
+        cb, step_s = oracle_sample(shape, tokens_sample=16, k_sample=200_000)
+        if i >= args.warmup:
+            vals.append(step_s)
+    ms = 1e3 * sum(vals) / len(vals)
+    value = 1e3 / ms
+    cb["value"] = value
+    line = {"impl": "reference", "metric": "zo_steps_per_s", "value": value, "unit": "steps/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(shape), "cpu_baseline": cb,
+            "e2e": {"value": value, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+    return 0
+
+
+def workload_config(shape):
+    return {"workload": "llama2_7b-shaped decoder, int4 group-128 + 0.1% fp32 sparse, full ZO step",
+            "batch": BATCH, "seq_len": SEQ, "tokens_per_step": BATCH * SEQ, "n_layers": shape["n_layers"],
+            "d_model": shape["d_model"], "d_ff": shape["d_ff"], "loss": "last-token 2-candidate CE",
+            "eps": EPS, "lr": LR, "l2": "inputs larger than L2 (3.4 GB of weights streamed per forward)",
+            "parallelism": "replicas"}
+
+
+# ------------------------------------------------------------------------------------ GPU leg
+def run_ours(args):
+    import numpy as np
+    import torch
+    from paper_2406_02913_b200 import binding as B
+    from paper_2406_02913_b200 import build as build_mod
+    from paper_2406_02913_b200 import workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl")
+    if rank == 0:
+        build_mod.build()
+    if dist is not None:
+        dist.barrier()
+    B.lib()
+
+    shape = wl.MODEL_SHAPES[WORKLOAD]
+    tensors, S_all = wl.device_decoder_tensors(shape, seed=rank)
+    model = B.Model(shape, wl.linear_names(shape), tensors, S_all, act_dtype=B.SZO_BF16,
+                    linear_mode=B.MODE_SPARSE_ADD, loss_kind=B.LOSS_CLS2, max_batch=BATCH, max_seq=SEQ)
+    n_steps = args.warmup + args.steps
+    toks_host = [torch.from_numpy(wl.token_batch(shape["vocab"], BATCH, SEQ, rank, wl.PURPOSE_TRAIN_BATCH, i)).pin_memory()
+                 for i in range(n_steps)]
+    labs_host = [torch.from_numpy(wl.binary_labels(BATCH, rank, i)).pin_memory() for i in range(n_steps)]
+    cand_host = torch.tensor([9906, 13], dtype=torch.int32).pin_memory()
+    toks_dev = [t.cuda() for t in toks_host]
+    labs_dev = [t.cuda() for t in labs_host]
+    cand_dev = cand_host.cuda()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if dist is None:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- device-resident inputs (the headline value)
+    for i in range(args.warmup):
+        model.zo_step(toks_dev[i], SEED, i, EPS, LR, labs_dev[i], cand_dev)
+    barrier()
+    model.enable_timing(True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clk:
+        ev0.record()
+        for i in range(args.warmup, n_steps):
+            model.zo_step(toks_dev[i], SEED, i, EPS, LR, labs_dev[i], cand_dev)
+        ev1.record()
+        barrier()
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1))
+    lin_ms, lin_launches = model.linear_time()
+    model.enable_timing(False)
+    launches = model.last_launches() * args.steps
+    last = model._scalars[:3].cpu().numpy()
+
+    # ---- host-resident inputs through the same API (end to end)
+    for i in range(min(args.warmup, 1)):
+        model.zo_step_host(toks_host[i], SEED, n_steps + i, EPS, LR, labs_host[i], cand_host)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(args.warmup, n_steps):
+        model.zo_step_host(toks_host[i], SEED, n_steps + i, EPS, LR, labs_host[i], cand_host)
+    torch.cuda.synchronize()
+    e2e_ms = max_over_ranks(1e3 * (time.perf_counter() - t0))
+
+    if rank != 0:
+        return 0
+    peaks = measured_peaks()
+    M = BATCH * SEQ
+    ms_per_step = ms_total / args.steps
+    steps_per_s = world * 1e3 / ms_per_step
+    flops_fwd = linear_flops_per_forward(shape, M)
+    lin_flops_total = 2 * flops_fwd * args.steps
+    achieved = lin_flops_total / (lin_ms * 1e-3) / 1e12 if lin_ms > 0 else 0.0
+    peak = peaks["bf16_tflops_sustained"]
+    cb, _ = oracle_sample(shape)
+    line = {
+        "metric": "zo_steps_per_s", "value": steps_per_s, "unit": "steps/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(shape),
+        "tokens_per_s": steps_per_s * M,
+        "e2e": {"value": world * 1e3 * args.steps / e2e_ms, "unit": "steps/s",
+                "h2d_bytes_per_step": BATCH * SEQ * 4 + BATCH * 4 + 8, "d2h_bytes_per_step": 24},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "kernel": "szo_linear_tc_kernel", "achieved": achieved, "peak": peak,
+                     "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                     "peak_source": f"{peaks['source']} (sustained cuBLAS bf16)",
+                     "launches": int(lin_launches), "avg_launch_ms": lin_ms / max(lin_launches, 1),
+                     "linear_ms_per_step": lin_ms / args.steps},
+        "cpu_baseline": cb,
+        "clocks": clk.summary(),
+        "last_step": {"f_plus": float(last[0]), "f_minus": float(last[1]), "g": float(last[2])},
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    return run_reference(args) if args.impl == "reference" else run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -196,6 +196,12 @@ szo_status szo_model_zo_step_host(szo_model_t* m, const int32_t* tokens_host,
                                   double* out3_host, void* stream);
 /* Number of kernel launches the last szo_model_zo_step on this model enqueued. */
 int64_t szo_model_last_launches(const szo_model_t* m);
+/* Measurement aid (no counterpart in the paper): when enabled, the model brackets every
+ * decoder-block linear launch with CUDA events on the launching stream.  szo_model_linear_time
+ * synchronises the device, returns the summed elapsed milliseconds and the number of launches
+ * since the last call (or since enabling), and resets the counters. */
+szo_status szo_model_enable_timing(szo_model_t* m, int32_t on);
+szo_status szo_model_linear_time(szo_model_t* m, double* ms_total_host, int64_t* launches_host);
 void szo_model_destroy(szo_model_t* m);
 
 #ifdef __cplusplus

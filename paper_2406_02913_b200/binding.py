@@ -92,6 +92,8 @@ _SIGS = {
                                            C.c_int32, C.c_uint64, C.c_uint64, C.c_float, C.c_float,
                                            C.c_void_p, C.c_void_p]),
     "szo_model_last_launches": (C.c_int64, [C.c_void_p]),
+    "szo_model_enable_timing": (C.c_int32, [C.c_void_p, C.c_int32]),
+    "szo_model_linear_time": (C.c_int32, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "szo_model_destroy": (None, [C.c_void_p]),
 }
 
@@ -298,6 +300,15 @@ class Model:
         _check(lib().szo_model_zo_step_host(self.h, hp(tokens_host), hp(labels_host), hp(cand_host), B, S,
                                             seed, step, eps, lr, C.cast(out, C.c_void_p), _stream()))
         return out[0], out[1], out[2]
+
+    def enable_timing(self, on: bool = True):
+        _check(lib().szo_model_enable_timing(self.h, 1 if on else 0))
+
+    def linear_time(self):
+        """(total ms, launches) of the decoder-block linears since the last call."""
+        ms, n = C.c_double(0), C.c_int64(0)
+        _check(lib().szo_model_linear_time(self.h, C.byref(ms), C.byref(n)))
+        return ms.value, n.value
 
     def last_launches(self) -> int:
         return lib().szo_model_last_launches(self.h)

@@ -265,6 +265,10 @@ struct szo_model {
   double* d_scalars = nullptr;
   int64_t last_launches = 0;
   std::vector<void*> owned;
+  // measurement aid: CUDA events around every decoder-block linear launch
+  bool timing = false;
+  std::vector<cudaEvent_t> events;
+  size_t events_used = 0;
 };
 
 namespace {
@@ -304,8 +308,21 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
     *up = static_cast<T*>(m->up);
   auto lin = [&](int layer, int j, const void* x, void* out) -> szo_status {
     const int t = layer * m->n_lin + j;
-    return szo_linear_fwd(m->plans[t], x, static_cast<szo_dtype>(act), M, Sv + m->offsets[t], out,
-                          static_cast<szo_dtype>(act), c.linear_mode, m->ws, m->ws_bytes, st);
+    if (m->timing) {
+      while (m->events.size() < m->events_used + 2) {
+        cudaEvent_t e;
+        SZO_CHECK_CUDA(cudaEventCreate(&e));
+        m->events.push_back(e);
+      }
+      SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used], st));
+    }
+    const szo_status rc = szo_linear_fwd(m->plans[t], x, static_cast<szo_dtype>(act), M, Sv + m->offsets[t], out,
+                                         static_cast<szo_dtype>(act), c.linear_mode, m->ws, m->ws_bytes, st);
+    if (m->timing) {
+      SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used + 1], st));
+      m->events_used += 2;
+    }
+    return rc;
   };
   embed_kernel<<<static_cast<unsigned>(M), 128, 0, st>>>(tokens, static_cast<const __nv_bfloat16*>(m->top.embed),
                                                         static_cast<const __nv_bfloat16*>(m->top.pos), S, d,
@@ -554,8 +571,31 @@ szo_status szo_model_zo_step_host(szo_model_t* m, const int32_t* tokens_host, co
   return SZO_OK;
 }
 
+szo_status szo_model_enable_timing(szo_model_t* m, int32_t on) {
+  SZO_REQUIRE(m != nullptr, SZO_ERR_INVALID_ARG, "model is NULL");
+  m->timing = on != 0;
+  m->events_used = 0;
+  return SZO_OK;
+}
+
+szo_status szo_model_linear_time(szo_model_t* m, double* ms_total_host, int64_t* launches_host) {
+  SZO_REQUIRE(m && ms_total_host && launches_host, SZO_ERR_INVALID_ARG, "NULL argument");
+  SZO_CHECK_CUDA(cudaDeviceSynchronize());
+  double total = 0.0;
+  for (size_t i = 0; i + 1 < m->events_used; i += 2) {
+    float ms = 0.f;
+    SZO_CHECK_CUDA(cudaEventElapsedTime(&ms, m->events[i], m->events[i + 1]));
+    total += ms;
+  }
+  *ms_total_host = total;
+  *launches_host = static_cast<int64_t>(m->events_used / 2);
+  m->events_used = 0;
+  return SZO_OK;
+}
+
 void szo_model_destroy(szo_model_t* m) {
   if (!m) return;
+  for (cudaEvent_t e : m->events) cudaEventDestroy(e);
   for (szo_linear_t* p : m->plans) szo_linear_destroy(p);
   szo_linear_destroy(m->lm_head_plan);
   for (void* p : m->owned) cudaFree(p);

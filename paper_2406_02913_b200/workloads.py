@@ -140,3 +140,57 @@ def gaussian_matrix(N: int, K: int, std: float, seed: int = 0, i: int = 0) -> np
 def random_codes(N: int, K: int, seed: int = 0, i: int = 0) -> np.ndarray:
     """Uniform random packed nibbles uint8 [N, K/2] (timing stand-in for a quantized tensor)."""
     return rng(seed, PURPOSE_CODES, i).integers(0, 256, (N, K // 2), dtype=np.uint8)
+
+
+# ------------------------------------------------------------------------------ large workloads
+# Full-size decoders (billions of parameters) are generated directly in device memory with a seeded
+# torch generator: quantizing 6.5 G fp32 weights on the host only to time a step would take
+# minutes.  These are input generators too: random codes, scales, zeros, indices and values.
+def device_decoder_tensors(shape: dict, seed: int = 0, device: str = "cuda"):
+    """Random-init quantized decoder in device memory, named as binding.Model expects.
+    Codes are uniform nibbles; scale ~ U(0.004, 0.006) and zero = -7.5 scale so that the
+    dequantised weights are centred with a spread close to N(0, 0.02); the sensitive set of each
+    tensor is a sorted random sample of floor(rho n) indices with values N(0, 0.02).
+    Returns (tensors, S_all)."""
+    import torch
+
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed))
+    d, V, G = shape["d_model"], shape["vocab"], shape["group"]
+    sz_dt = torch.bfloat16 if shape["sz_fmt"] == "bf16" else torch.float16
+    opt = shape["arch"] == "opt"
+    randn = lambda *s: torch.randn(*s, generator=g, device=device, dtype=torch.float32)
+    t = {"embed": (randn(V, d) * 0.02).to(torch.bfloat16), "lm_head": (randn(V, d) * 0.02).to(torch.bfloat16),
+         "final_norm": torch.ones(d, device=device)}
+    if opt:
+        t["pos"] = (randn(shape["max_pos"], d) * 0.02).to(torch.bfloat16)
+        t["final_norm_b"] = torch.zeros(d, device=device)
+    S_parts = []
+    for l in range(shape["n_layers"]):
+        for nm in ("attn_norm", "mlp_norm"):
+            t[f"l{l}.{nm}"] = torch.ones(d, device=device)
+            if opt:
+                t[f"l{l}.{nm}_b"] = torch.zeros(d, device=device)
+        for nm in linear_names(shape):
+            N, K = linear_shape(shape, nm)
+            p = f"l{l}.{nm}."
+            if G > 0:
+                t[p + "codes"] = torch.randint(0, 256, (N, K // 2), generator=g, device=device, dtype=torch.uint8)
+                sc = (0.004 + 0.002 * torch.rand(N, K // G, generator=g, device=device)).to(sz_dt)
+                t[p + "scales"] = sc
+                t[p + "zeros"] = (-7.5 * sc.float()).to(sz_dt)
+            else:
+                t[p + "codes"] = (randn(N, K) * 0.02).to(torch.bfloat16)
+            k = int(shape["rho"] * N * K)
+            draw = torch.randint(0, N * K, (int(k * 1.05) + 64,), generator=g, device=device, dtype=torch.int64)
+            u = torch.unique(draw)
+            while u.numel() < k:
+                more = torch.randint(0, N * K, (k,), generator=g, device=device, dtype=torch.int64)
+                u = torch.unique(torch.cat([u, more]))
+            keep = torch.randperm(u.numel(), generator=g, device=device)[:k]
+            t[p + "idx"] = torch.sort(u[keep]).values.contiguous()
+            S_parts.append(randn(k) * 0.02)
+            if opt:
+                t[p + "bias"] = randn(N) * 0.02
+    S_all = torch.cat(S_parts).contiguous() if S_parts else torch.zeros(0, device=device)
+    return t, S_all
