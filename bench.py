@@ -221,11 +221,15 @@ def run_ours(args):
     model.enable_timing(True)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(local) as clk:
+        if args.profile_range:
+            torch.cuda.profiler.start()
         ev0.record()
         for i in range(args.warmup, n_steps):
             model.zo_step(toks_dev[i], SEED, i, EPS, LR, labs_dev[i], cand_dev)
         ev1.record()
         barrier()
+        if args.profile_range:
+            torch.cuda.profiler.stop()
     ms_total = max_over_ranks(ev0.elapsed_time(ev1))
     lin_ms, lin_launches = model.linear_time()
     model.enable_timing(False)
@@ -280,6 +284,8 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--profile-range", action="store_true",
+                    help="bracket the timed region with cudaProfilerStart/Stop (for ncu --profile-from-start off)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     return run_reference(args) if args.impl == "reference" else run_ours(args)

@@ -1,0 +1,145 @@
+"""Kernel microbenchmarks through the C ABI: one JSON line per case.
+
+    python -m paper_2406_02913_b200.microbench linear --M 8192 [--N 4096 --K 4096 --mode sparse_add]
+    python -m paper_2406_02913_b200.microbench sparse --k 6476005
+    python -m paper_2406_02913_b200.microbench sweep            # the single-linear and k-sweep cases
+
+linear: x bf16 [M,K] ~ N(0,1); W [N,K] int4 group-128 with bf16 scales/zeros quantized (by the
+library) from N(0,0.02); 0.1 % sparse entries chosen as the top-k of squared Student-t(3) scores
+(by the library); the perturbed forward is timed.  sparse: one perturb pass over k sorted random
+indices.  Timing: CUDA events on the launching stream, L2 flushed by writing a 512 MB buffer before
+every timed launch, median of the repetitions.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2406_02913_b200 import binding as B  # noqa: E402
+from paper_2406_02913_b200 import workloads as wl  # noqa: E402
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return p["hbm_gbs"], p["bf16_tflops"], "measured"
+    return 6650.0, 1590.0, "fallback"
+
+
+_flush = None
+
+
+def flush_l2():
+    global _flush
+    if _flush is None:
+        _flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    _flush.fill_(1)
+
+
+def time_call(fn, reps, warmup=3, flush=True):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(reps):
+        if flush:
+            flush_l2()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    return statistics.median(ts), min(ts)
+
+
+def linear_case(M, N, K, G, mode, rho, reps, out_dtype=torch.bfloat16):
+    W = torch.from_numpy(wl.gaussian_matrix(N, K, 0.02, seed=0, i=1)).cuda()
+    g = torch.from_numpy(wl.student_t_gradient(N * K, 3.0, seed=0, i=2)).cuda()
+    nnz = int(rho * N * K)
+    idx = B.szo_select_mask(g * g, nnz)
+    S = W.view(-1)[idx].contiguous()
+    W.view(-1)[idx] = 0.0
+    plan_args = None
+    if G > 0:
+        codes, sc, ze = B.szo_quantize(W, G, "bf16")
+        plan_args = (codes, sc, ze)
+    else:
+        plan_args = (W.to(torch.bfloat16), None, None)
+    plan = B.Linear(N, K, G, plan_args[0], plan_args[1], plan_args[2], "bf16", idx)
+    x = torch.from_numpy(wl.activation(M, K, seed=0, i=3)).cuda().to(torch.bfloat16)
+    S_pert = torch.empty_like(S)
+    B.szo_perturb(S, S_pert, idx, 0, 1234, 0, 1e-3)
+    y = torch.empty((M, N), dtype=out_dtype, device="cuda")
+    md = {"sparse_add": B.MODE_SPARSE_ADD, "spmm": B.MODE_SPMM, "fp32": B.MODE_FP32_VALIDATE}[mode]
+    med, best = time_call(lambda: plan.fwd(x, S_pert, md, out_dtype, y=y), reps)
+    hbm, tf, src = peaks()
+    flops = 2.0 * M * N * K
+    byts = (N * K / 2 + 4 * N * K / max(G, 1) if G > 0 else 2 * N * K) + 2 * M * K + y.element_size() * M * N + 8 * nnz
+    t_roof = max(flops / (tf * 1e12), byts / (hbm * 1e9))
+    line = {"case": "linear", "M": M, "N": N, "K": K, "G": G, "mode": mode, "nnz": nnz, "ms_median": med,
+            "ms_min": best, "tflops": flops / (med * 1e-3) / 1e12, "gbs": byts / (med * 1e-3) / 1e9,
+            "bound": "tensor" if flops / (tf * 1e12) >= byts / (hbm * 1e9) else "hbm",
+            "roofline_ms": t_roof * 1e3, "frac_of_roofline": t_roof * 1e3 / med, "peaks": src,
+            "status": B.device_status()}
+    print(json.dumps(line), flush=True)
+    plan.close()
+    return line
+
+
+def sparse_case(k, reps, n_total=12_582_912_000):
+    g = torch.Generator(device="cuda")
+    g.manual_seed(k % 1000003)
+    idx = torch.sort(torch.randint(0, n_total, (k,), generator=g, device="cuda", dtype=torch.int64)).values
+    S = torch.randn(k, generator=g, device="cuda") * 0.02
+    out = torch.empty_like(S)
+    hbm, _, src = peaks()
+    res = {}
+    for name, dst, fl in (("out_of_place_cold", out, True), ("in_place_cold", S, True), ("in_place_warm", S, False)):
+        med, best = time_call(lambda: B.szo_perturb(S, dst, idx, 0, 1234, 1, 1e-3), reps, flush=fl)
+        res[name] = {"ms_median": med, "gbs": 16.0 * k / (med * 1e-3) / 1e9, "frac_hbm": 16.0 * k / (med * 1e-3) / 1e9 / hbm}
+    line = {"case": "sparse_perturb", "k": k, "bytes_per_entry": 16, "peaks": src, **res}
+    print(json.dumps(line), flush=True)
+    return line
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("what", choices=["linear", "sparse", "sweep"])
+    ap.add_argument("--M", type=int, default=8192)
+    ap.add_argument("--N", type=int, default=4096)
+    ap.add_argument("--K", type=int, default=4096)
+    ap.add_argument("--G", type=int, default=128)
+    ap.add_argument("--rho", type=float, default=1e-3)
+    ap.add_argument("--mode", default="sparse_add")
+    ap.add_argument("--k", type=int, default=6_476_005)
+    ap.add_argument("--reps", type=int, default=20)
+    a = ap.parse_args()
+    B.lib()
+    if a.what == "linear":
+        linear_case(a.M, a.N, a.K, a.G, a.mode, a.rho, a.reps)
+    elif a.what == "sparse":
+        sparse_case(a.k, a.reps)
+    else:
+        for M in (16, 256, 8192):
+            for mode in ("sparse_add", "spmm"):
+                linear_case(M, 4096, 4096, 128, mode, 1e-3, a.reps)
+        for N, K in ((4096, 4096), (11008, 4096), (4096, 11008)):
+            linear_case(4096, N, K, 128, "sparse_add", 1e-3, a.reps)
+        for k in (100_000, 1_000_000, 6_476_005, 12_582_912, 100_000_000):
+            sparse_case(k, a.reps)
+
+
+if __name__ == "__main__":
+    main()
