@@ -33,6 +33,11 @@ constexpr int kNumWarps = 16;
 constexpr int kDeqWarp0 = 4, kNumDeqWarps = 8;
 constexpr int kEpiWarp0 = 12;
 constexpr int kATileBytes = kBM * kBK * 2;   // 16 KiB
+constexpr int kCodesBytes = kBM * kBK / 2;   // 4 KiB of packed codes per stage
+constexpr int kSzBytes = 2048;               // (scale, zero) fp32 pairs: 128 rows x up to 2 groups
+constexpr int kLook = 4;                     // SparseAdd look-ahead in k-blocks
+constexpr int kRecSlots = 8, kRecCap = 64;   // ring of per-k-block sparse records in shared memory
+constexpr int kBoundSlots = 16;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 
 struct TcParams {
@@ -41,13 +46,11 @@ struct TcParams {
   int nkb;                 // K / 64
   int64_t m_tiles, n_tiles;
   const uint8_t* codes;    // [N, K/2]
-  const float2* sz;        // [N, K/G]
+  const float2* sz;        // [K/G][Npad]
+  int64_t Npad;
   const int32_t* bucket_ptr;
-  const int32_t* bucket_eid;
-  const uint16_t* bucket_pos;
-  int64_t n_kblocks;       // buckets per row group
-  int64_t n_rowgroups;
-  const float* S;          // sparse values (nullptr: no SparseAdd)
+  int64_t n_kblocks;       // buckets per 128-row tile
+  const uint2* Sb;         // sparse records (position in tile, value bits) in bucket order; nullptr: none
   const float* bias;
   void* y;
   int y_f32;
@@ -103,6 +106,22 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
       : "memory");
+}
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_4(uint32_t dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_8(uint32_t dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait_group() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 __device__ __forceinline__ void tmem_alloc(uint32_t result_smem, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(result_smem), "r"(ncols)
@@ -194,13 +213,15 @@ __global__ void __launch_bounds__(kNumWarps * 32, 1)
 szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                      const TcParams P) {
   constexpr int kBTileBytes = BT * kBK * 2;
-  constexpr int kStageBytes = kATileBytes + kBTileBytes;
+  constexpr int kStageBytes = kATileBytes + kBTileBytes + (kDequant ? kCodesBytes + kSzBytes : 0);
   constexpr int kAccStride = BT < 32 ? 32 : BT;             // TMEM columns per accumulator buffer
   constexpr uint32_t kTmemCols = static_cast<uint32_t>(2 * kAccStride);
   constexpr uint32_t kIdesc = make_idesc(kBM, BT);
 
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[3 * kStages + 4];
+  __shared__ __align__(8) unsigned long long bars[4 * kStages + 4];
+  __shared__ __align__(16) uint2 rec_ring[kRecSlots][kRecCap];      // sparse records, per k-block
+  __shared__ __align__(8) int32_t bound_ring[kBoundSlots][2];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
 
@@ -209,20 +230,23 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &abort_flag_s;
 
-  auto full_bar = [&](int s) { return smem_u32(&bars[s]); };
-  auto aready_bar = [&](int s) { return smem_u32(&bars[kStages + s]); };
-  auto empty_bar = [&](int s) { return smem_u32(&bars[2 * kStages + s]); };
-  auto accfull_bar = [&](int a) { return smem_u32(&bars[3 * kStages + a]); };
-  auto accempty_bar = [&](int a) { return smem_u32(&bars[3 * kStages + 2 + a]); };
+  auto full_bar = [&](int s) { return smem_u32(&bars[s]); };              // TMA bytes landed
+  auto deq_bar = [&](int s) { return smem_u32(&bars[kStages + s]); };     // dequantised tile written
+  auto aready_bar = [&](int s) { return smem_u32(&bars[2 * kStages + s]); };  // sparse values added
+  auto empty_bar = [&](int s) { return smem_u32(&bars[3 * kStages + s]); };   // MMAs of the stage done
+  auto accfull_bar = [&](int a) { return smem_u32(&bars[4 * kStages + a]); };
+  auto accempty_bar = [&](int a) { return smem_u32(&bars[4 * kStages + 2 + a]); };
   auto a_tile = [&](int s) { return tiles_base + static_cast<uint32_t>(s) * kStageBytes; };
   auto b_tile = [&](int s) { return tiles_base + static_cast<uint32_t>(s) * kStageBytes + kATileBytes; };
+  auto c_tile = [&](int s) { return tiles_base + static_cast<uint32_t>(s) * kStageBytes + kATileBytes + kBTileBytes; };
 
-  const bool a_proc = kDequant || (P.S != nullptr);   // weight-producer warps take part
+  const bool sparse = P.Sb != nullptr;
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
     for (int s = 0; s < kStages; ++s) {
       mbar_init(full_bar(s), 1);
-      mbar_init(aready_bar(s), kNumDeqWarps);
+      mbar_init(deq_bar(s), kNumDeqWarps);
+      mbar_init(aready_bar(s), 1);
       mbar_init(empty_bar(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
@@ -240,20 +264,30 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
   const int64_t total_tiles = P.m_tiles * P.n_tiles;
   const int64_t my_tiles = (total_tiles > blockIdx.x) ? (total_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
   const int64_t my_iters = my_tiles * P.nkb;
+  auto tile_of = [&](int64_t it) { return blockIdx.x + (it / P.nkb) * gridDim.x; };
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
+      const int groups_kb = (kDequant && P.G < kBK) ? kBK / P.G : 1;   // scale groups per k-block
       for (int64_t it = 0; it < my_iters; ++it) {
-        const int64_t tile = blockIdx.x + (it / P.nkb) * gridDim.x;
+        const int64_t tile = tile_of(it);
         const int kb = static_cast<int>(it % P.nkb);
         const int64_t n_tile = tile / P.m_tiles, m_tile = tile % P.m_tiles;
         const int s = static_cast<int>(it % kStages);
         const uint32_t ph = static_cast<uint32_t>((it / kStages) & 1);
         if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, P.status)) break;
-        mbar_expect_tx(full_bar(s), kDequant ? kBTileBytes : kStageBytes);
+        if constexpr (kDequant) {
+          mbar_expect_tx(full_bar(s), kBTileBytes + kCodesBytes + groups_kb * 1024);
+          tma_load_2d(c_tile(s), &tmap_w, kb * (kBK / 2), static_cast<int>(n_tile * kBM), full_bar(s));
+          const int64_t g0 = (static_cast<int64_t>(kb) * kBK) / P.G;
+          for (int g = 0; g < groups_kb; ++g)
+            bulk_load_1d(c_tile(s) + kCodesBytes + g * 1024, P.sz + (g0 + g) * P.Npad + n_tile * kBM, 1024, full_bar(s));
+        } else {
+          mbar_expect_tx(full_bar(s), kBTileBytes + kATileBytes);
+          tma_load_2d(a_tile(s), &tmap_w, kb * kBK, static_cast<int>(n_tile * kBM), full_bar(s));
+        }
         tma_load_2d(b_tile(s), &tmap_x, kb * kBK, static_cast<int>(m_tile * BT), full_bar(s));
-        if constexpr (!kDequant) tma_load_2d(a_tile(s), &tmap_w, kb * kBK, static_cast<int>(n_tile * kBM), full_bar(s));
       }
     }
   } else if (warp == 1) {
@@ -271,7 +305,11 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
           const int s = static_cast<int>(it % kStages);
           const uint32_t ph = static_cast<uint32_t>((it / kStages) & 1);
           if (!mbar_wait(full_bar(s), ph, abort_flag, P.status)) { ok = false; break; }
-          if (a_proc && !mbar_wait(aready_bar(s), ph, abort_flag, P.status)) { ok = false; break; }
+          if (sparse) {
+            if (!mbar_wait(aready_bar(s), ph, abort_flag, P.status)) { ok = false; break; }
+          } else if (kDequant) {
+            if (!mbar_wait(deq_bar(s), ph, abort_flag, P.status)) { ok = false; break; }
+          }
           tc_fence_after();
           const uint64_t adesc = make_desc_sw128(a_tile(s)), bdesc = make_desc_sw128(b_tile(s));
 #pragma unroll
@@ -284,78 +322,83 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
         if (ok) umma_commit(accfull_bar(as));
       }
     }
-  } else if (warp >= kDeqWarp0 && warp < kDeqWarp0 + kNumDeqWarps) {
-    // ---------------------------------------------------------------- weight producers
-    if (a_proc) {
-      const int dw = warp - kDeqWarp0;             // rows [16 dw, 16 dw + 16) of the tile
-      const int sub = lane >> 3, chunk = lane & 7; // 4 rows x 8 sixteen-byte chunks per pass
-      const int64_t words_per_row = P.K / 8;
-      const int groups_per_row = kDequant ? static_cast<int>(P.K / P.G) : 1;
-      uint32_t cw[4] = {0u, 0u, 0u, 0u};
-      auto load_codes = [&](int64_t it, uint32_t (&dst)[4]) {
-        const int64_t tile = blockIdx.x + (it / P.nkb) * gridDim.x;
-        const int kb = static_cast<int>(it % P.nkb);
-        const int64_t n0 = (tile / P.m_tiles) * kBM;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int64_t n = n0 + dw * 16 + i * 4 + sub;
-          dst[i] = (n < P.N) ? __ldg(reinterpret_cast<const uint32_t*>(P.codes) + n * words_per_row + kb * 8 + chunk) : 0u;
+  } else if (warp == 2) {
+    // ---------------------------------------------------------------- SparseAdd warp
+    // Adds the sparse values of bucket (tile, k-block) to the bf16 weight tile in shared memory.
+    // Bucket bounds and records are brought in with cp.async kLook / 2*kLook iterations ahead.
+    if (sparse && my_iters > 0) {
+      auto bucket_of = [&](int64_t it) { return (tile_of(it) / P.m_tiles) * P.n_kblocks + (it % P.nkb); };
+      auto issue_bounds = [&](int64_t it) {           // lanes 0,1 copy bucket_ptr[b], bucket_ptr[b+1]
+        if (it < my_iters && lane < 2)
+          cp_async_4(smem_u32(&bound_ring[it % kBoundSlots][lane]), P.bucket_ptr + bucket_of(it) + lane);
+      };
+      auto issue_records = [&](int64_t it) {          // needs bounds(it) in shared memory
+        if (it < my_iters) {
+          const int32_t e0 = bound_ring[it % kBoundSlots][0], e1 = bound_ring[it % kBoundSlots][1];
+          const int32_t n = (e1 - e0 < kRecCap) ? e1 - e0 : kRecCap;
+          for (int32_t j = lane; j < n; j += 32) cp_async_8(smem_u32(&rec_ring[it % kRecSlots][j]), P.Sb + e0 + j);
         }
       };
-      if constexpr (kDequant) {
-        if (my_iters > 0) load_codes(0, cw);
+      // prologue: bounds of 0..2*kLook-1, then records of 0..kLook-1
+      for (int64_t j = 0; j < 2 * kLook; ++j) issue_bounds(j);
+      cp_async_commit();
+      cp_async_wait_all();
+      __syncwarp();
+      for (int64_t j = 0; j < kLook; ++j) {
+        issue_records(j);
+        cp_async_commit();
       }
       for (int64_t it = 0; it < my_iters; ++it) {
-        const int64_t tile = blockIdx.x + (it / P.nkb) * gridDim.x;
-        const int kb = static_cast<int>(it % P.nkb);
-        const int64_t n0 = (tile / P.m_tiles) * kBM;
         const int s = static_cast<int>(it % kStages);
         const uint32_t ph = static_cast<uint32_t>((it / kStages) & 1);
+        // group(j) = { bounds(j + 2 kLook), records(j + kLook) }, committed in iteration j.  Groups
+        // retire in order: with at most kLook - 1 still pending, group(it - kLook) has landed, i.e.
+        // records(it) and bounds(it + kLook), which the next record copies are addressed from.
+        cp_async_wait_group<kLook - 1>();
+        __syncwarp();
+        issue_bounds(it + 2 * kLook);
+        issue_records(it + kLook);
+        cp_async_commit();
+        const int32_t e0 = bound_ring[it % kBoundSlots][0], e1 = bound_ring[it % kBoundSlots][1];
+        if (!mbar_wait(kDequant ? deq_bar(s) : full_bar(s), ph, abort_flag, P.status)) break;
         unsigned char* A = tiles_ptr + static_cast<size_t>(s) * kStageBytes;
-        if constexpr (kDequant) {
-          uint32_t cn[4] = {0u, 0u, 0u, 0u};
-          if (it + 1 < my_iters) load_codes(it + 1, cn);
-          float2 sz[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const int64_t n = n0 + dw * 16 + i * 4 + sub;
-            sz[i] = (n < P.N) ? __ldg(P.sz + n * groups_per_row + (kb * kBK + chunk * 8) / P.G) : make_float2(0.f, 0.f);
-          }
-          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, P.status)) break;
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const int r = dw * 16 + i * 4 + sub;
-            const uint4 v = dequant_word<kFast>(cw[i], sz[i]);
-            *reinterpret_cast<uint4*>(A + r * 128 + ((chunk ^ (r & 7)) << 4)) = v;
-          }
-#pragma unroll
-          for (int i = 0; i < 4; ++i) cw[i] = cn[i];
-        } else {
-          if (!mbar_wait(full_bar(s), ph, abort_flag, P.status)) break;   // TMA wrote the bf16 tile
-        }
-        if (P.S != nullptr) {
-          __syncwarp();
-          // SparseAdd: entries of bucket (row group, k-block) that fall in this warp's 16 rows
-          const int64_t rg = (n0 >> 5) + (dw >> 1);
-          const int64_t b = rg * P.n_kblocks + kb;
-          int32_t e0 = 0, e1 = 0;
-          if (rg < P.n_rowgroups) {
-            e0 = __ldg(P.bucket_ptr + b);
-            e1 = __ldg(P.bucket_ptr + b + 1);
-          }
-          for (int32_t e = e0 + lane; e < e1; e += 32) {
-            const uint32_t pos = __ldg(P.bucket_pos + e);
-            const int lr = static_cast<int>(pos >> 6), lc = static_cast<int>(pos & 63);
-            if ((lr >> 4) == (dw & 1)) {
-              const int r = (dw >> 1) * 32 + lr;
-              __nv_bfloat16* el = reinterpret_cast<__nv_bfloat16*>(A + r * 128 + (((lc >> 3) ^ (r & 7)) << 4) + (lc & 7) * 2);
-              *el = __float2bfloat16_rn(__bfloat162float(*el) + __ldg(P.S + __ldg(P.bucket_eid + e)));
-            }
-          }
+        for (int32_t j = lane; j < e1 - e0; j += 32) {
+          const uint2 rec = (j < kRecCap) ? rec_ring[it % kRecSlots][j] : __ldg(P.Sb + e0 + j);
+          const int r = static_cast<int>(rec.x >> 6), c = static_cast<int>(rec.x & 63);
+          __nv_bfloat16* el = reinterpret_cast<__nv_bfloat16*>(A + r * 128 + (((c >> 3) ^ (r & 7)) << 4) + (c & 7) * 2);
+          *el = __float2bfloat16_rn(__bfloat162float(*el) + __uint_as_float(rec.y));
         }
         fence_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(aready_bar(s));
+      }
+      cp_async_wait_all();
+    }
+  } else if (warp >= kDeqWarp0 && warp < kDeqWarp0 + kNumDeqWarps) {
+    // ---------------------------------------------------------------- dequantisation warps
+    // codes and (scale, zero) of the stage are already in shared memory (TMA); each warp converts
+    // rows [16 dw, 16 dw + 16): per pass 4 rows x 8 sixteen-byte chunks, conflict-free both ways.
+    if constexpr (kDequant) {
+      const int dw = warp - kDeqWarp0;
+      const int sub = lane >> 3, chunk = lane & 7;
+      const int gsel = (P.G < kBK) ? (chunk * 8) / P.G : 0;
+      for (int64_t it = 0; it < my_iters; ++it) {
+        const int s = static_cast<int>(it % kStages);
+        const uint32_t ph = static_cast<uint32_t>((it / kStages) & 1);
+        unsigned char* A = tiles_ptr + static_cast<size_t>(s) * kStageBytes;
+        const unsigned char* C = A + kATileBytes + kBTileBytes;
+        const float2* SZ = reinterpret_cast<const float2*>(C + kCodesBytes) + gsel * kBM;
+        if (!mbar_wait(full_bar(s), ph, abort_flag, P.status)) break;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int r = dw * 16 + i * 4 + sub;
+          const uint32_t w = *reinterpret_cast<const uint32_t*>(C + r * 32 + chunk * 4);
+          const uint4 v = dequant_word<kFast>(w, SZ[r]);
+          *reinterpret_cast<uint4*>(A + r * 128 + ((chunk ^ (r & 7)) << 4)) = v;
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(deq_bar(s));
       }
     }
   } else if (warp >= kEpiWarp0) {
@@ -371,23 +414,25 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
       const int64_t n = n_tile * kBM + qd * 32 + lane;
       const float bias = (P.bias != nullptr && n < P.N) ? P.bias[n] : 0.f;
       const int64_t m0 = m_tile * BT;
+      const int mlimit = static_cast<int>((P.M - m0 < BT) ? P.M - m0 : BT);   // valid tokens in this tile
       for (int c0 = 0; c0 < BT; c0 += 32) {
         uint32_t v[32];
         tmem_ld32(tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + static_cast<uint32_t>(as * kAccStride + c0), v);
-        if (n < P.N) {
+        if (n < P.N && c0 < mlimit) {
+          const int cnt = mlimit - c0;                 // tokens c0 .. c0+cnt-1 are valid (cnt may exceed 32)
           if (P.y_f32) {
-            float* y = static_cast<float*>(P.y);
+            float* yp = static_cast<float*>(P.y) + (m0 + c0) * P.N + n;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-              const int64_t m = m0 + c0 + j;
-              if (c0 + j < BT && m < P.M) y[m * P.N + n] = __uint_as_float(v[j]) + bias;
+              if (j < cnt) *yp = __uint_as_float(v[j]) + bias;
+              yp += P.N;
             }
           } else {
-            __nv_bfloat16* y = static_cast<__nv_bfloat16*>(P.y);
+            __nv_bfloat16* yp = static_cast<__nv_bfloat16*>(P.y) + (m0 + c0) * P.N + n;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-              const int64_t m = m0 + c0 + j;
-              if (c0 + j < BT && m < P.M) y[m * P.N + n] = __float2bfloat16_rn(__uint_as_float(v[j]) + bias);
+              if (j < cnt) *yp = __float2bfloat16_rn(__uint_as_float(v[j]) + bias);
+              yp += P.N;
             }
           }
         }
@@ -442,14 +487,29 @@ szo_status make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t co
 }
 
 struct TcPlan {
-  CUtensorMap w_map;    // dense bf16 weight (G == 0)
-  bool has_w_map;
+  CUtensorMap w_map;    // dense bf16 weight (G == 0) or the packed codes as bytes (G > 0)
   int sms;
 };
 
+// uint8 matrix [rows, cols_bytes] row-major, box [128 rows x 32 bytes], no swizzle.
+szo_status make_codes_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols_bytes) {
+  EncodeTiledFn fn = encode_fn();
+  SZO_REQUIRE(fn != nullptr, SZO_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols_bytes), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols_bytes)};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBK / 2), static_cast<cuuint32_t>(kBM)};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  SZO_REQUIRE(r == CUDA_SUCCESS, SZO_ERR_CUDA, "cuTensorMapEncodeTiled (codes) failed (%d)", static_cast<int>(r));
+  return SZO_OK;
+}
+
 template <int BT, int kStages, bool kDequant, bool kFast>
 szo_status launch_tc(const CUtensorMap& mx, const CUtensorMap& mw, const TcParams& P, int sms, cudaStream_t st) {
-  constexpr size_t smem = static_cast<size_t>(kStages) * (kATileBytes + BT * kBK * 2) + 1024;
+  constexpr size_t smem =
+      static_cast<size_t>(kStages) * (kATileBytes + BT * kBK * 2 + (kDequant ? kCodesBytes + kSzBytes : 0)) + 1024;
   auto kern = szo_linear_tc_kernel<BT, kStages, kDequant, kFast>;
   static bool configured = false;
   if (!configured) {
@@ -476,17 +536,14 @@ szo_status dispatch_kind(const szo_linear* p, const CUtensorMap& mx, const CUten
 
 szo_status tc_plan_create(szo_linear* p, cudaStream_t) {
   TcPlan* t = new TcPlan();
-  t->has_w_map = false;
   int dev = 0;
   t->sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&t->sms, cudaDevAttrMultiProcessorCount, dev);
-  if (p->G == 0) {
-    const szo_status s = make_map(&t->w_map, p->codes, p->N, p->K, kBM);
-    if (s != SZO_OK) {
-      delete t;
-      return s;
-    }
-    t->has_w_map = true;
+  const szo_status s = (p->G == 0) ? make_map(&t->w_map, p->codes, p->N, p->K, kBM)
+                                   : make_codes_map(&t->w_map, p->codes, p->N, p->K / 2);
+  if (s != SZO_OK) {
+    delete t;
+    return s;
   }
   p->tc = t;
   return SZO_OK;
@@ -497,8 +554,8 @@ void tc_plan_destroy(szo_linear* p) {
   p->tc = nullptr;
 }
 
-szo_status linear_fwd_tc(const szo_linear* p, const void* x, int64_t M, const float* S, void* y, int y_dtype,
-                         bool sparse_add, cudaStream_t st) {
+szo_status linear_fwd_tc(const szo_linear* p, const void* x, int64_t M, const uint2* S_bucket, void* y,
+                         int y_dtype, cudaStream_t st) {
   const TcPlan* t = static_cast<const TcPlan*>(p->tc);
   SZO_REQUIRE(t != nullptr, SZO_ERR_INVALID_ARG, "plan has no tensor-core data");
   SZO_REQUIRE(M < (int64_t(1) << 31) && p->N < (int64_t(1) << 31), SZO_ERR_SHAPE, "M or N too large");
@@ -511,20 +568,20 @@ szo_status linear_fwd_tc(const szo_linear* p, const void* x, int64_t M, const fl
   P.m_tiles = ceil_div(M, BT); P.n_tiles = ceil_div(p->N, kBM);
   P.codes = static_cast<const uint8_t*>(p->codes);
   P.sz = p->sz;
-  P.bucket_ptr = p->bucket_ptr; P.bucket_eid = p->bucket_eid; P.bucket_pos = p->bucket_pos;
+  P.bucket_ptr = p->bucket_ptr;
   P.n_kblocks = p->n_kblocks;
-  P.n_rowgroups = p->n_rowgroups;
-  P.S = (sparse_add && p->nnz > 0) ? S : nullptr;
+  P.Npad = p->Npad;
+  P.Sb = (p->nnz > 0) ? S_bucket : nullptr;
   P.bias = p->bias;
   P.y = y; P.y_f32 = (y_dtype == SZO_F32) ? 1 : 0;
   P.status = device_status_word();
   SZO_REQUIRE(P.status != nullptr, SZO_ERR_CUDA, "no device status word");
-  const CUtensorMap& mw = t->has_w_map ? t->w_map : mx;   // unused by the kernel when dequantising
+  const CUtensorMap& mw = t->w_map;
   switch (BT) {
     case 16: return dispatch_kind<16, 6>(p, mx, mw, P, t->sms, st);
     case 32: return dispatch_kind<32, 6>(p, mx, mw, P, t->sms, st);
     case 64: return dispatch_kind<64, 6>(p, mx, mw, P, t->sms, st);
-    case 128: return dispatch_kind<128, 6>(p, mx, mw, P, t->sms, st);
+    case 128: return dispatch_kind<128, 5>(p, mx, mw, P, t->sms, st);
     default: return dispatch_kind<256, 4>(p, mx, mw, P, t->sms, st);
   }
 }

@@ -7,14 +7,18 @@
 namespace szo {
 
 // ------------------------------------------------------------------------------ plan kernels
+// (scale, zero) widened to fp32 and transposed to [K/G][Npad] so that the 128 rows of a tile are
+// contiguous for one group (one bulk copy per tile and k-block).
 template <typename SZ>
-__global__ void widen_sz_kernel(const SZ* __restrict__ scales, const SZ* __restrict__ zeros, int64_t n,
-                                float2* __restrict__ out) {
+__global__ void widen_sz_kernel(const SZ* __restrict__ scales, const SZ* __restrict__ zeros, int64_t N,
+                                int64_t groups, int64_t Npad, float2* __restrict__ out) {
   const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (i < n) out[i] = make_float2(static_cast<float>(scales[i]), static_cast<float>(zeros[i]));
+  if (i >= N * groups) return;
+  const int64_t n = i / groups, g = i % groups;
+  out[g * Npad + n] = make_float2(static_cast<float>(scales[i]), static_cast<float>(zeros[i]));
 }
 
-// Per entry: column, validity (strictly ascending, in range) and the size of its (32-row, 64-col)
+// Per entry: column, validity (strictly ascending, in range) and the size of its (128-row, 64-col)
 // bucket, counted into bucket_ptr[b + 1].
 __global__ void entry_kernel(const int64_t* __restrict__ idx, int64_t nnz, int64_t N, int64_t K,
                              int64_t nkb, int32_t* __restrict__ ent_col, int32_t* __restrict__ bucket_ptr,
@@ -29,7 +33,7 @@ __global__ void entry_kernel(const int64_t* __restrict__ idx, int64_t nnz, int64
   }
   const int64_t row = v / K, col = v % K;
   ent_col[e] = static_cast<int32_t>(col);
-  atomicAdd(&bucket_ptr[(row >> 5) * nkb + (col >> 6) + 1], 1);
+  atomicAdd(&bucket_ptr[(row >> 7) * nkb + (col >> 6) + 1], 1);
 }
 
 // In-place inclusive scan of a[0..n) by one block (chunks of 1024, carried sequentially).
@@ -68,7 +72,7 @@ __global__ void row_ptr_kernel(const int64_t* __restrict__ idx, int64_t nnz, int
   row_ptr[r] = static_cast<int32_t>(lo);
 }
 
-// One thread per 32-row group walks its entries in index order and appends them to their buckets.
+// One thread per 128-row tile walks its entries in index order and appends them to their buckets.
 __global__ void bucket_fill_kernel(const int64_t* __restrict__ idx, const int32_t* __restrict__ row_ptr,
                                    const int32_t* __restrict__ ent_col, int64_t N, int64_t K, int64_t nkb,
                                    int64_t n_rowgroups, const int32_t* __restrict__ bucket_ptr,
@@ -76,7 +80,7 @@ __global__ void bucket_fill_kernel(const int64_t* __restrict__ idx, const int32_
                                    uint16_t* __restrict__ bucket_pos) {
   const int64_t g = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (g >= n_rowgroups) return;
-  const int64_t r0 = g * 32, r1 = (r0 + 32 < N) ? r0 + 32 : N;
+  const int64_t r0 = g * 128, r1 = (r0 + 128 < N) ? r0 + 128 : N;
   for (int32_t e = row_ptr[r0]; e < row_ptr[r1]; ++e) {
     const int32_t col = ent_col[e];
     const int64_t row = idx[e] / K;
@@ -90,11 +94,11 @@ __global__ void bucket_fill_kernel(const int64_t* __restrict__ idx, const int32_
 // ------------------------------------------------------------------------------ fp32 path
 // W_eff[n, c] = fma(q, scale, zero) in fp32 (two elements per thread), or the widened bf16 weight.
 __global__ void dequant_f32_kernel(const uint8_t* __restrict__ codes, const float2* __restrict__ sz,
-                                   int64_t N, int64_t K, int G, float* __restrict__ W) {
+                                   int64_t N, int64_t K, int G, int64_t Npad, float* __restrict__ W) {
   const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (t >= N * K / 2) return;
   const int64_t n = (2 * t) / K, c = (2 * t) % K;
-  const float2 p = sz[n * (K / G) + c / G];
+  const float2 p = sz[(c / G) * Npad + n];
   const uint8_t b = codes[t];
   W[2 * t] = fmaf(static_cast<float>(b & 15), p.x, p.y);
   W[2 * t + 1] = fmaf(static_cast<float>(b >> 4), p.x, p.y);
@@ -182,7 +186,7 @@ szo_status linear_fwd_fp32(const szo_linear* p, const void* x, int x_dtype, int6
   const int64_t NK = p->N * p->K;
   if (p->G > 0) {
     dequant_f32_kernel<<<static_cast<unsigned>(ceil_div(NK / 2, 256)), 256, 0, st>>>(
-        static_cast<const uint8_t*>(p->codes), p->sz, p->N, p->K, p->G, W);
+        static_cast<const uint8_t*>(p->codes), p->sz, p->N, p->K, p->G, p->Npad, W);
   } else {
     widen_bf16_kernel<<<static_cast<unsigned>(ceil_div(NK, 256)), 256, 0, st>>>(
         static_cast<const __nv_bfloat16*>(p->codes), NK, W);
@@ -275,6 +279,41 @@ szo_status linear_spmm(const szo_linear* p, const void* x, int64_t M, const floa
   return SZO_OK;
 }
 
+// rec[p] = (position of bucket entry p inside its tile, bits of S[eid[p]])
+__global__ void gather_values_kernel(const float* __restrict__ S, const int32_t* __restrict__ eid,
+                                     const uint16_t* __restrict__ pos, int64_t n, uint2* __restrict__ out) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = make_uint2(pos[i], __float_as_uint(S[eid[i]]));
+}
+
+szo_status gather_values(const float* S, const int32_t* eid, const uint16_t* pos, int64_t n, uint2* out,
+                         cudaStream_t st) {
+  if (n == 0) return SZO_OK;
+  gather_values_kernel<<<static_cast<unsigned>(ceil_div(n, 256)), 256, 0, st>>>(S, eid, pos, n, out);
+  count_launch();
+  SZO_CHECK_LAUNCH("gather_values_kernel");
+  return SZO_OK;
+}
+
+szo_status linear_fwd_impl(const szo_linear* p, const void* x, int x_dtype, int64_t M, const float* S_pert,
+                           const uint2* S_bucket, void* y, int y_dtype, int32_t mode, void* workspace,
+                           size_t workspace_bytes, cudaStream_t st) {
+  if (mode == SZO_MODE_FP32_VALIDATE)
+    return linear_fwd_fp32(p, x, x_dtype, M, S_pert, y, y_dtype, workspace, workspace_bytes, st);
+  if (mode == SZO_MODE_SPMM) {
+    SZO_TRY(linear_fwd_tc(p, x, M, nullptr, y, y_dtype, st));
+    return linear_spmm(p, x, M, S_pert, y, y_dtype, st);
+  }
+  if (p->nnz > 0 && S_bucket == nullptr) {
+    const size_t need = round_up(static_cast<size_t>(p->nnz) * sizeof(uint2), 256);
+    SZO_REQUIRE(workspace && workspace_bytes >= need, SZO_ERR_WORKSPACE,
+                "SparseAdd needs a workspace of %zu bytes for the bucket-ordered values", need);
+    SZO_TRY(gather_values(S_pert, p->bucket_eid, p->bucket_pos, p->nnz, static_cast<uint2*>(workspace), st));
+    S_bucket = static_cast<const uint2*>(workspace);
+  }
+  return linear_fwd_tc(p, x, M, S_bucket, y, y_dtype, st);
+}
+
 static void free_plan(szo_linear* p) {
   if (!p) return;
   tc_plan_destroy(p);
@@ -318,7 +357,8 @@ szo_status szo_linear_create(szo_linear_t** out, int64_t N, int64_t K, int32_t G
   *p = szo_linear{};
   p->N = N; p->K = K; p->G = G; p->sz_dtype = sz_dtype; p->nnz = nnz;
   p->codes = codes_or_bf16_W; p->scales = scales; p->zeros = zeros; p->idx = idx; p->bias = bias;
-  p->n_rowgroups = ceil_div(N, 32);
+  p->n_rowgroups = ceil_div(N, 128);
+  p->Npad = p->n_rowgroups * 128;
   p->n_kblocks = K / 64;
   const int64_t nb = p->n_rowgroups * p->n_kblocks;
   int32_t* cursor = nullptr;
@@ -338,13 +378,14 @@ szo_status szo_linear_create(szo_linear_t** out, int64_t N, int64_t K, int32_t G
   } while (0)
   if (G > 0) {
     const int64_t ng = N * (K / G);
-    SZO_PLAN_CUDA(cudaMalloc(&p->sz, ng * sizeof(float2)));
+    SZO_PLAN_CUDA(cudaMalloc(&p->sz, p->Npad * (K / G) * sizeof(float2)));
+    SZO_PLAN_CUDA(cudaMemsetAsync(p->sz, 0, p->Npad * (K / G) * sizeof(float2), st));
     if (sz_dtype == SZO_BF16)
       widen_sz_kernel<__nv_bfloat16><<<static_cast<unsigned>(ceil_div(ng, 256)), 256, 0, st>>>(
-          static_cast<const __nv_bfloat16*>(scales), static_cast<const __nv_bfloat16*>(zeros), ng, p->sz);
+          static_cast<const __nv_bfloat16*>(scales), static_cast<const __nv_bfloat16*>(zeros), N, K / G, p->Npad, p->sz);
     else
       widen_sz_kernel<__half><<<static_cast<unsigned>(ceil_div(ng, 256)), 256, 0, st>>>(
-          static_cast<const __half*>(scales), static_cast<const __half*>(zeros), ng, p->sz);
+          static_cast<const __half*>(scales), static_cast<const __half*>(zeros), N, K / G, p->Npad, p->sz);
   }
   SZO_PLAN_CUDA(cudaMalloc(&p->row_ptr, (N + 1) * sizeof(int32_t)));
   SZO_PLAN_CUDA(cudaMalloc(&p->bucket_ptr, (nb + 1) * sizeof(int32_t)));
@@ -382,7 +423,9 @@ szo_status szo_linear_create(szo_linear_t** out, int64_t N, int64_t K, int32_t G
 
 size_t szo_linear_workspace_bytes(const szo_linear_t* p, int64_t M, int32_t mode) {
   if (!p) return 0;
-  return mode == SZO_MODE_FP32_VALIDATE ? linear_ws_fp32(p, M) : 0;
+  if (mode == SZO_MODE_FP32_VALIDATE) return linear_ws_fp32(p, M);
+  if (mode == SZO_MODE_SPMM) return 0;
+  return round_up(static_cast<size_t>(p->nnz) * sizeof(uint2), 256);   // bucket-ordered sparse records
 }
 
 szo_status szo_linear_fwd(const szo_linear_t* p, const void* x, szo_dtype x_dtype, int64_t M,
@@ -401,13 +444,7 @@ szo_status szo_linear_fwd(const szo_linear_t* p, const void* x, szo_dtype x_dtyp
               "x, y and workspace must be 16-byte aligned");
   SZO_REQUIRE((reinterpret_cast<uintptr_t>(S_pert) & 3u) == 0, SZO_ERR_ALIGNMENT, "S_pert must be 4-byte aligned");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (mode == SZO_MODE_FP32_VALIDATE)
-    return linear_fwd_fp32(p, x, x_dtype, M, S_pert, y, y_dtype, workspace, workspace_bytes, st);
-  if (mode == SZO_MODE_SPMM) {
-    SZO_TRY(linear_fwd_tc(p, x, M, S_pert, y, y_dtype, /*sparse_add=*/false, st));
-    return linear_spmm(p, x, M, S_pert, y, y_dtype, st);
-  }
-  return linear_fwd_tc(p, x, M, S_pert, y, y_dtype, /*sparse_add=*/true, st);
+  return linear_fwd_impl(p, x, x_dtype, M, S_pert, nullptr, y, y_dtype, mode, workspace, workspace_bytes, st);
 }
 
 void szo_linear_destroy(szo_linear_t* p) { free_plan(p); }

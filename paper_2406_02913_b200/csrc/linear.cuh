@@ -14,10 +14,11 @@ struct szo_linear {
   const int64_t* idx;
   const float* bias;
   // derived, owned by the plan (device memory)
-  float2* sz;            // [N, K/G] (scale, zero) widened to fp32 (G > 0)
+  float2* sz;            // [K/G][Npad] (scale, zero) widened to fp32, group-major (G > 0)
+  int64_t Npad;          // N rounded up to a multiple of 128
   int32_t* ent_col;      // [nnz] column of entry e
   int32_t* row_ptr;      // [N+1] entries of row r are [row_ptr[r], row_ptr[r+1])
-  int32_t* bucket_ptr;   // [n_rowgroups * n_kblocks + 1]; bucket = (row/32, col/64)
+  int32_t* bucket_ptr;   // [n_rowgroups * n_kblocks + 1]; bucket = (row/128, col/64)
   int32_t* bucket_eid;   // [nnz] entry id (index into S) in bucket order
   uint16_t* bucket_pos;  // [nnz] (local_row << 6) | local_col in bucket order
   int64_t n_rowgroups, n_kblocks;
@@ -38,7 +39,18 @@ szo_status linear_spmm(const szo_linear* p, const void* x, int64_t M, const floa
 // tensor-core path (gemm_tc.cu)
 szo_status tc_plan_create(szo_linear* p, cudaStream_t st);
 void tc_plan_destroy(szo_linear* p);
-szo_status linear_fwd_tc(const szo_linear* p, const void* x, int64_t M, const float* S, void* y,
-                         int y_dtype, bool sparse_add, cudaStream_t st);
+// S_bucket: the sparse entries gathered into bucket order as records
+// (bucket_pos[p], bits of S[bucket_eid[p]]), or nullptr to leave the sparse term out (it is then
+// applied by linear_spmm).
+szo_status linear_fwd_tc(const szo_linear* p, const void* x, int64_t M, const uint2* S_bucket, void* y,
+                         int y_dtype, cudaStream_t st);
+// out[p] = (pos[p], bits of S[eid[p]]) for p in [0, n)
+szo_status gather_values(const float* S, const int32_t* eid, const uint16_t* pos, int64_t n, uint2* out,
+                         cudaStream_t st);
+// Forward with every option: S_bucket may be given (pre-gathered, SparseAdd mode) to skip the
+// per-call gather into the workspace.
+szo_status linear_fwd_impl(const szo_linear* p, const void* x, int x_dtype, int64_t M, const float* S_pert,
+                           const uint2* S_bucket, void* y, int y_dtype, int32_t mode, void* workspace,
+                           size_t workspace_bytes, cudaStream_t st);
 
 }  // namespace szo
