@@ -84,6 +84,24 @@ szo_status szo_quantize(const void* W, szo_dtype w_dtype, int64_t N, int64_t K, 
 szo_status szo_select_mask(const float* scores, int64_t n, int64_t k, int64_t* idx_out,
                            void* workspace, size_t* workspace_bytes, void* stream);
 
+/* ---- Sensitive parameter mask without any allocation.  The paper has no counterpart: this is a
+ * packaging variant of szo_select_mask for callers that cannot obtain device memory themselves,
+ * for example a plug-in running inside a host application that owns the allocator and hands out only
+ * the input and output buffers, or a process whose memory budget is fixed before it starts.  The
+ * scratch that szo_select_mask takes as a workspace lives here in a fixed array inside the library
+ * (about 194 KiB of device memory on every GPU that loads the library, until the process exits), so
+ * the call performs no cudaMalloc/cudaFree and needs no workspace query.
+ *   limit     n <= 67 108 864 (2^26) scores; larger n returns SZO_ERR_WORKSPACE and touches nothing.
+ *   set-up    the first call on each device looks up the array's device address (the device must be
+ *             current, as for every call); make that first call before starting any stream capture.
+ *   sharing   every call on a device uses the same array and finds the previous call's contents in
+ *             it; the function clears what it needs.  Two calls that overlap on the GPU (different
+ *             streams or threads) race on it: serialise them.
+ * Results, tie rule, NaN handling and the final stream synchronisation are those of
+ * szo_select_mask. */
+szo_status szo_select_mask_static(const float* scores, int64_t n, int64_t k, int64_t* idx_out,
+                                  void* stream);
+
 /* ---- Sparse perturbation (Definition 4, zbar = z (.) m_k; Section 3.4 update rule on w_sparse;
  * Section 2.1 seed trick: z is regenerated, never stored).
  *   S_out[j] = fma(scale, z_j, S_in[j]),  z_j = Gaussian(Philox4x32-10(key = seed,

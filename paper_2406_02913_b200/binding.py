@@ -66,6 +66,7 @@ _SIGS = {
                                  C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "szo_select_mask": (C.c_int32, [C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
                                     C.POINTER(C.c_size_t), C.c_void_p]),
+    "szo_select_mask_static": (C.c_int32, [C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]),
     "szo_perturb": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
                                 C.c_uint64, C.c_uint64, C.c_float, C.c_void_p]),
     "szo_projected_gradient": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p]),
@@ -165,6 +166,13 @@ def szo_select_mask(scores: torch.Tensor, k: int) -> torch.Tensor:
     ws = torch.empty((max(nbytes.value, 16),), dtype=torch.uint8, device=scores.device)
     _check(lib().szo_select_mask(_ptr(scores), n, k, _ptr(idx), _ptr(ws), C.byref(nbytes), _stream()))
     return idx[:k]
+
+
+def szo_select_mask_static(scores: torch.Tensor, k: int, out: torch.Tensor) -> torch.Tensor:
+    """Top-k mask into the caller's `out` (int64, at least k long) using the library's built-in
+    scratch: for callers that must not allocate device memory.  At most 2**26 scores."""
+    _check(lib().szo_select_mask_static(_ptr(scores), scores.numel(), k, _ptr(out), _stream()))
+    return out[:k]
 
 
 def szo_perturb(S_in, S_out, idx, idx_base: int, seed: int, step: int, scale: float):

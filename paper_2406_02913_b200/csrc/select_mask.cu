@@ -268,3 +268,79 @@ extern "C" szo_status szo_select_mask(const float* scores, int64_t n, int64_t k,
   SZO_REQUIRE(nan_flag == 0, SZO_ERR_NONFINITE, "scores contain NaN");
   return SZO_OK;
 }
+
+
+// ------------------------------------------------------------------------------ no-allocation variant
+// Same selection with the scratch memory held inside the library image instead of a caller
+// workspace.  kStaticSelectMaxN bounds the size: 2^26 scores need 8192 blocks of per-block counts
+// and offsets next to the selection state.
+namespace szo {
+constexpr int64_t kStaticSelectMaxN = int64_t(1) << 26;
+constexpr size_t kStaticStateBytes = (sizeof(SelectState) + 255) / 256 * 256;
+constexpr size_t kStaticBlocks = static_cast<size_t>(kStaticSelectMaxN / kSelTile);
+constexpr size_t kStaticScratchBytes =
+    kStaticStateBytes + 2 * kStaticBlocks * sizeof(uint32_t) + 2 * kStaticBlocks * sizeof(unsigned long long);
+static __device__ __align__(256) unsigned char g_select_scratch[kStaticScratchBytes];
+
+// Device address of g_select_scratch on the current device, looked up once per device.  In host
+// code the symbol name is only a handle; the address a kernel can use comes from
+// cudaGetSymbolAddress, with the device that will run the kernels current.
+static szo_status static_scratch_address(unsigned char** out) {
+  static unsigned char* cached[64] = {nullptr};
+  int dev = 0;
+  SZO_CHECK_CUDA(cudaGetDevice(&dev));
+  SZO_REQUIRE(dev >= 0 && dev < 64, SZO_ERR_UNSUPPORTED, "device ordinal %d not supported", dev);
+  if (cached[dev] == nullptr) {
+    unsigned char* ptr = nullptr;
+    SZO_CHECK_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_select_scratch));
+    SZO_REQUIRE(ptr != nullptr, SZO_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
+    cached[dev] = ptr;
+  }
+  *out = cached[dev];
+  return SZO_OK;
+}
+}  // namespace szo
+
+extern "C" szo_status szo_select_mask_static(const float* scores, int64_t n, int64_t k, int64_t* idx_out,
+                                             void* stream) {
+  using namespace szo;
+  SZO_REQUIRE(n >= 0 && k >= 0 && k <= n, SZO_ERR_INVALID_ARG, "need 0 <= k <= n (k=%lld, n=%lld)",
+              (long long)k, (long long)n);
+  SZO_REQUIRE(n <= kStaticSelectMaxN, SZO_ERR_WORKSPACE,
+              "n = %lld exceeds the built-in scratch of szo_select_mask_static (at most %lld scores); "
+              "use szo_select_mask with a caller workspace",
+              (long long)n, (long long)kStaticSelectMaxN);
+  if (k == 0) return SZO_OK;
+  SZO_REQUIRE(scores && idx_out, SZO_ERR_INVALID_ARG, "NULL pointer");
+  SZO_REQUIRE(aligned16(scores) && aligned16(idx_out), SZO_ERR_ALIGNMENT, "buffers must be 16-byte aligned");
+  unsigned char* ws = nullptr;
+  SZO_TRY(static_scratch_address(&ws));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t nblocks = ceil_div(n, kSelTile);
+  // fixed carve-up of the array (sized for the maximum), independent of n
+  SelectState* state = reinterpret_cast<SelectState*>(ws);
+  uint32_t* blk_gt = reinterpret_cast<uint32_t*>(ws + kStaticStateBytes);
+  uint32_t* blk_eq = blk_gt + kStaticBlocks;
+  unsigned long long* off_gt = reinterpret_cast<unsigned long long*>(blk_eq + kStaticBlocks);
+  unsigned long long* off_eq = off_gt + kStaticBlocks;
+  // The array keeps whatever the previous call left: the state and histogram are cleared here, the
+  // per-block counts and offsets of the nblocks in use are fully overwritten before they are read.
+  select_init_kernel<<<1, 256, 0, st>>>(state, static_cast<unsigned long long>(k));
+  int64_t hist_blocks = ceil_div(n, kSelBlock * 8);
+  if (hist_blocks > 148 * 8) hist_blocks = 148 * 8;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    select_hist_kernel<<<static_cast<unsigned>(hist_blocks), kSelBlock, 0, st>>>(scores, n, shift, state);
+    select_pick_kernel<<<1, 32, 0, st>>>(state, shift);
+  }
+  select_count_kernel<<<static_cast<unsigned>(nblocks), kSelBlock, 0, st>>>(scores, n, state, blk_gt, blk_eq);
+  select_scan_kernel<<<1, 1024, 0, st>>>(blk_gt, blk_eq, nblocks, off_gt, off_eq);
+  select_write_kernel<<<static_cast<unsigned>(nblocks), kSelBlock, 0, st>>>(scores, n, state, off_gt, off_eq,
+                                                                          idx_out, k);
+  count_launch(12);
+  SZO_CHECK_LAUNCH("select_mask kernels (static scratch)");
+  int32_t nan_flag = 0;
+  SZO_CHECK_CUDA(cudaMemcpyAsync(&nan_flag, &state->nan_flag, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  SZO_CHECK_CUDA(cudaStreamSynchronize(st));
+  SZO_REQUIRE(nan_flag == 0, SZO_ERR_NONFINITE, "scores contain NaN");
+  return SZO_OK;
+}
