@@ -185,6 +185,13 @@ typedef struct {
   const float* final_norm_g; const float* final_norm_b;
 } szo_model_weights;
 
+/* Causal softmax attention, one block of the loss f that Definition 1 evaluates (scale 1/sqrt(head_dim),
+ * grouped-query attention when n_kv_heads < n_heads).  q, o: dtype [B*S, n_heads*head_dim]; k, v: dtype
+ * [B*S, n_kv_heads*head_dim]; token b*S+s is position s of sequence b.  dtype SZO_BF16 (tensor-core
+ * flash kernel) or SZO_F32; head_dim 64 or 128. */
+szo_status szo_attention(const void* q, const void* k, const void* v, void* o, szo_dtype dtype, int32_t B, int32_t S,
+                         int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, void* stream);
+
 typedef struct szo_model szo_model_t;
 /* layers_host: host array of n_layers entries holding device pointers.  S_all: fp32 [k_total],
  * the trainable sparse values of all linears concatenated in model order (the only mutable

@@ -79,6 +79,8 @@ _SIGS = {
                                    C.c_int, C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p]),
     "szo_linear_workspace_bytes": (C.c_size_t, [C.c_void_p, C.c_int64, C.c_int32]),
     "szo_linear_destroy": (None, [C.c_void_p]),
+    "szo_attention": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int32, C.c_int32,
+                                  C.c_int32, C.c_int32, C.c_int32, C.c_void_p]),
     "szo_model_create": (C.c_int32, [C.POINTER(C.c_void_p), C.POINTER(ModelConfig),
                                      C.POINTER(ModelWeights), C.POINTER(LayerWeights), C.c_void_p,
                                      C.c_void_p]),
@@ -229,6 +231,14 @@ class Linear:
             self.close()
         except Exception:
             pass
+
+
+def szo_attention(q, k, v, B: int, S: int, n_heads: int, n_kv_heads: int, head_dim: int):
+    """Causal attention; q [B*S, H*hd], k/v [B*S, Hkv*hd] (bf16 or fp32).  Returns o like q."""
+    o = torch.empty_like(q)
+    _check(lib().szo_attention(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _DT[q.dtype], B, S, n_heads, n_kv_heads,
+                               head_dim, _stream()))
+    return o
 
 
 # ------------------------------------------------------------------------------ model

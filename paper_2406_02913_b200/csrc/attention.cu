@@ -1,0 +1,220 @@
+// Causal softmax attention for the bf16 activation path: a flash-style kernel on warp-level tensor
+// core MMAs (mma.sync m16n8k16, bf16 inputs, fp32 accumulation and softmax statistics).
+//
+// The loss path needs attention only as one block of the black-box loss f (Definition 1); it is a
+// few percent of a step's flops, so the legacy warp-level MMA is enough here and the tcgen05
+// machinery is kept for the linears.  One CTA = 64 queries of one (batch, head); 4 warps x 16 rows;
+// K/V tiles of 64 keys staged in padded shared memory; online softmax; grouped-query attention by
+// mapping query head h to KV head h / (H / Hkv).  q, k, v, o are [B*S, heads*HD] bf16 row-major.
+#include "common.cuh"
+
+namespace szo {
+
+namespace {
+
+constexpr int kQT = 64, kKT = 64;
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// Copies a [rows x HD] bf16 tile (row stride `ld` elements in global memory) into padded shared
+// memory (row stride HD + 8), zero-filling rows at or beyond `valid`.
+template <int HD>
+__device__ __forceinline__ void load_tile(__nv_bfloat16* dst, const __nv_bfloat16* src, int64_t ld, int valid) {
+  constexpr int kChunks = HD / 8;                 // 16-byte chunks per row
+  for (int i = threadIdx.x; i < 64 * kChunks; i += 128) {
+    const int r = i / kChunks, c = i % kChunks;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (r < valid) v = *reinterpret_cast<const uint4*>(src + r * ld + c * 8);
+    *reinterpret_cast<uint4*>(dst + r * (HD + 8) + c * 8) = v;
+  }
+}
+
+template <int HD>
+__global__ void __launch_bounds__(128)
+flash_attn_bf16_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                       const __nv_bfloat16* __restrict__ v, __nv_bfloat16* __restrict__ o, int S, int H, int Hkv,
+                       float scale_log2e) {
+  constexpr int LDS = HD + 8;
+  extern __shared__ __align__(16) unsigned char smem_attn[];
+  __nv_bfloat16* sQ = reinterpret_cast<__nv_bfloat16*>(smem_attn);
+  __nv_bfloat16* sK = sQ + kQT * LDS;
+  __nv_bfloat16* sV = sK + kKT * LDS;
+
+  const int qt = blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
+  const int hk = hq / (H / Hkv);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int64_t ldq = static_cast<int64_t>(H) * HD, ldk = static_cast<int64_t>(Hkv) * HD;
+  const int q0 = qt * kQT;
+  const __nv_bfloat16* qbase = q + (static_cast<int64_t>(b) * S + q0) * ldq + hq * HD;
+  load_tile<HD>(sQ, qbase, ldq, S - q0 < kQT ? S - q0 : kQT);
+  __syncthreads();
+
+  // this warp's 16 query rows as A fragments, kept in registers
+  uint32_t qa[HD / 16][4];
+#pragma unroll
+  for (int ks = 0; ks < HD / 16; ++ks) {
+    const uint32_t addr = static_cast<uint32_t>(__cvta_generic_to_shared(
+        sQ + (warp * 16 + (lane & 15)) * LDS + ks * 16 + (lane >> 4) * 8));
+    ldsm_x4(addr, qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3]);
+  }
+
+  float oacc[HD / 8][4];
+#pragma unroll
+  for (int i = 0; i < HD / 8; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
+  float mrow[2] = {-INFINITY, -INFINITY}, lrow[2] = {0.f, 0.f};
+  const int row_a = q0 + warp * 16 + g, row_b = row_a + 8;     // the two query rows of this thread
+
+  for (int kt = 0; kt <= qt; ++kt) {
+    const int k0 = kt * kKT;
+    const int valid = S - k0 < kKT ? S - k0 : kKT;
+    __syncthreads();                                            // previous tile fully consumed
+    load_tile<HD>(sK, k + (static_cast<int64_t>(b) * S + k0) * ldk + hk * HD, ldk, valid);
+    load_tile<HD>(sV, v + (static_cast<int64_t>(b) * S + k0) * ldk + hk * HD, ldk, valid);
+    __syncthreads();
+
+    // scores: 16 rows x 64 keys per warp
+    float sacc[kKT / 8][4];
+#pragma unroll
+    for (int i = 0; i < kKT / 8; ++i) sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < HD / 16; ++ks) {
+#pragma unroll
+      for (int np = 0; np < kKT / 16; ++np) {                   // two key tiles of 8 per ldmatrix.x4
+        uint32_t b0, b1, b2, b3;
+        const uint32_t addr = static_cast<uint32_t>(__cvta_generic_to_shared(
+            sK + (np * 16 + (lane & 7) + (lane >> 4) * 8) * LDS + ks * 16 + ((lane >> 3) & 1) * 8));
+        ldsm_x4(addr, b0, b1, b2, b3);
+        mma_bf16(sacc[2 * np], qa[ks], b0, b1);
+        mma_bf16(sacc[2 * np + 1], qa[ks], b2, b3);
+      }
+    }
+    // causal mask (diagonal tile) and keys beyond the sequence
+    if (kt == qt || valid < kKT) {
+#pragma unroll
+      for (int i = 0; i < kKT / 8; ++i) {
+        const int c = k0 + i * 8 + 2 * t;
+        if (c > row_a || c >= S) sacc[i][0] = -INFINITY;
+        if (c + 1 > row_a || c + 1 >= S) sacc[i][1] = -INFINITY;
+        if (c > row_b || c >= S) sacc[i][2] = -INFINITY;
+        if (c + 1 > row_b || c + 1 >= S) sacc[i][3] = -INFINITY;
+      }
+    }
+    // online softmax, rows g and g+8
+    float mx[2] = {mrow[0], mrow[1]};
+#pragma unroll
+    for (int i = 0; i < kKT / 8; ++i) {
+      mx[0] = fmaxf(mx[0], fmaxf(sacc[i][0], sacc[i][1]));
+      mx[1] = fmaxf(mx[1], fmaxf(sacc[i][2], sacc[i][3]));
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+    }
+    float corr[2], msc[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      // a row always has at least its own key in the first tile, so mx is finite from then on
+      msc[r] = (mx[r] == -INFINITY) ? 0.f : mx[r] * scale_log2e;
+      corr[r] = (mrow[r] == -INFINITY) ? 0.f : exp2f(mrow[r] * scale_log2e - msc[r]);
+      mrow[r] = mx[r];
+      lrow[r] *= corr[r];
+    }
+    uint32_t pa[kKT / 16][4];
+    float psum[2] = {0.f, 0.f};
+#pragma unroll
+    for (int i = 0; i < kKT / 8; ++i) {
+      const float p0 = exp2f(sacc[i][0] * scale_log2e - msc[0]), p1 = exp2f(sacc[i][1] * scale_log2e - msc[0]);
+      const float p2 = exp2f(sacc[i][2] * scale_log2e - msc[1]), p3 = exp2f(sacc[i][3] * scale_log2e - msc[1]);
+      psum[0] += p0 + p1;
+      psum[1] += p2 + p3;
+      // accumulator layout of two adjacent 8-key tiles = A fragment of one 16-key step
+      pa[i >> 1][(i & 1) * 2 + 0] = pack2(p0, p1);
+      pa[i >> 1][(i & 1) * 2 + 1] = pack2(p2, p3);
+    }
+    lrow[0] += psum[0];
+    lrow[1] += psum[1];
+#pragma unroll
+    for (int i = 0; i < HD / 8; ++i) {
+      oacc[i][0] *= corr[0];
+      oacc[i][1] *= corr[0];
+      oacc[i][2] *= corr[1];
+      oacc[i][3] *= corr[1];
+    }
+    // O += P V
+#pragma unroll
+    for (int ks = 0; ks < kKT / 16; ++ks) {
+#pragma unroll
+      for (int dp = 0; dp < HD / 16; ++dp) {                    // two 8-wide d tiles per ldmatrix.x4.trans
+        uint32_t b0, b1, b2, b3;
+        const uint32_t addr = static_cast<uint32_t>(__cvta_generic_to_shared(
+            sV + (ks * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * LDS + dp * 16 + (lane >> 4) * 8));
+        ldsm_x4_trans(addr, b0, b1, b2, b3);
+        mma_bf16(oacc[2 * dp], pa[ks], b0, b1);
+        mma_bf16(oacc[2 * dp + 1], pa[ks], b2, b3);
+      }
+    }
+  }
+  // row sums across the quad, normalise, store
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 1);
+    lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 2);
+  }
+  const float inv_a = 1.0f / lrow[0], inv_b = 1.0f / lrow[1];
+  __nv_bfloat16* obase = o + static_cast<int64_t>(b) * S * ldq + hq * HD;
+#pragma unroll
+  for (int i = 0; i < HD / 8; ++i) {
+    const int c = i * 8 + 2 * t;
+    if (row_a < S) *reinterpret_cast<uint32_t*>(obase + row_a * ldq + c) = pack2(oacc[i][0] * inv_a, oacc[i][1] * inv_a);
+    if (row_b < S) *reinterpret_cast<uint32_t*>(obase + row_b * ldq + c) = pack2(oacc[i][2] * inv_b, oacc[i][3] * inv_b);
+  }
+}
+
+}  // namespace
+
+szo_status launch_flash_attention_bf16(const void* q, const void* k, const void* v, void* o, int B, int S, int H,
+                                       int Hkv, int hd, cudaStream_t st) {
+  SZO_REQUIRE(hd == 64 || hd == 128, SZO_ERR_UNSUPPORTED, "head dimension must be 64 or 128");
+  const float scale_log2e = 1.4426950408889634f / sqrtf(static_cast<float>(hd));
+  dim3 grid(static_cast<unsigned>(ceil_div(S, kQT)), H, B);
+  const size_t smem = static_cast<size_t>(3) * 64 * (hd + 8) * 2;
+  auto* qb = static_cast<const __nv_bfloat16*>(q);
+  auto* kb = static_cast<const __nv_bfloat16*>(k);
+  auto* vb = static_cast<const __nv_bfloat16*>(v);
+  auto* ob = static_cast<__nv_bfloat16*>(o);
+  if (hd == 64) {
+    flash_attn_bf16_kernel<64><<<grid, 128, smem, st>>>(qb, kb, vb, ob, S, H, Hkv, scale_log2e);
+  } else {
+    static bool configured = false;
+    if (!configured) {
+      SZO_CHECK_CUDA(cudaFuncSetAttribute(flash_attn_bf16_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(smem)));
+      configured = true;
+    }
+    flash_attn_bf16_kernel<128><<<grid, 128, smem, st>>>(qb, kb, vb, ob, S, H, Hkv, scale_log2e);
+  }
+  count_launch();
+  SZO_CHECK_LAUNCH("flash_attn_bf16_kernel");
+  return SZO_OK;
+}
+
+}  // namespace szo

@@ -67,4 +67,8 @@ szo_status launch_sparse_axpy(const float* S_in, float* S_out, const int64_t* id
                               int64_t idx_base, uint64_t seed, uint64_t step, ScaleArg sa,
                               cudaStream_t st);
 
+// Causal attention for bf16 activations (attention.cu); q, k, v, o are [B*S, heads*hd] row-major.
+szo_status launch_flash_attention_bf16(const void* q, const void* k, const void* v, void* o, int B, int S, int H,
+                                       int Hkv, int hd, cudaStream_t st);
+
 }  // namespace szo

@@ -139,24 +139,62 @@ attn_warp_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __re
   for (int j = 0; j < E; ++j) op[lane + 32 * j] = from_f32<T>(acc[j] * inv);
 }
 
+// Elementwise kernels work on 16-byte vectors (8 bf16 or 4 fp32 per thread); every tensor they
+// touch has a multiple of 8 elements per row and 16-byte aligned rows.
+template <typename T> struct Vec16 {
+  static constexpr int kN = 16 / sizeof(T);
+  T v[16 / sizeof(T)];
+};
+template <typename T> __device__ __forceinline__ Vec16<T> load16(const T* p) {
+  Vec16<T> r;
+  *reinterpret_cast<uint4*>(r.v) = *reinterpret_cast<const uint4*>(p);
+  return r;
+}
+template <typename T> __device__ __forceinline__ void store16(T* p, const Vec16<T>& r) {
+  *reinterpret_cast<uint4*>(p) = *reinterpret_cast<const uint4*>(r.v);
+}
+
 template <typename T>
 __global__ void silu_mul_kernel(const T* __restrict__ gate, const T* __restrict__ up, int64_t n, T* __restrict__ out) {
-  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  constexpr int kN = Vec16<T>::kN;
+  const int64_t i = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) * kN;
   if (i >= n) return;
-  const float g = to_f32<T>(gate[i]);
-  out[i] = from_f32<T>(g / (1.0f + expf(-g)) * to_f32<T>(up[i]));
+  const Vec16<T> g = load16(gate + i), u = load16(up + i);
+  Vec16<T> r;
+#pragma unroll
+  for (int j = 0; j < kN; ++j) {
+    const float x = to_f32<T>(g.v[j]);
+    r.v[j] = from_f32<T>(x / (1.0f + expf(-x)) * to_f32<T>(u.v[j]));
+  }
+  store16(out + i, r);
 }
 
 template <typename T>
 __global__ void relu_kernel(T* __restrict__ x, int64_t n) {
-  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (i < n) x[i] = from_f32<T>(fmaxf(to_f32<T>(x[i]), 0.f));
+  constexpr int kN = Vec16<T>::kN;
+  const int64_t i = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) * kN;
+  if (i >= n) return;
+  Vec16<T> r = load16(x + i);
+#pragma unroll
+  for (int j = 0; j < kN; ++j) r.v[j] = from_f32<T>(fmaxf(to_f32<T>(r.v[j]), 0.f));
+  store16(x + i, r);
 }
 
 template <typename T>
 __global__ void residual_add_kernel(float* __restrict__ h, const T* __restrict__ y, int64_t n) {
-  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (i < n) h[i] += to_f32<T>(y[i]);
+  constexpr int kN = Vec16<T>::kN;
+  const int64_t i = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) * kN;
+  if (i >= n) return;
+  const Vec16<T> r = load16(y + i);
+#pragma unroll
+  for (int j = 0; j < kN; j += 4) {
+    float4 a = *reinterpret_cast<float4*>(h + i + j);
+    a.x += to_f32<T>(r.v[j]);
+    a.y += to_f32<T>(r.v[j + 1]);
+    a.z += to_f32<T>(r.v[j + 2]);
+    a.w += to_f32<T>(r.v[j + 3]);
+    *reinterpret_cast<float4*>(h + i + j) = a;
+  }
 }
 
 // Next-token cross-entropy of row m (position s < S-1 predicts tok[m+1]); 0 for the last position.
@@ -341,7 +379,9 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
       rope_kernel<T><<<blocks_for(M * Hkv * (hd / 2), 256), 256, 0, st>>>(k, m->rope_tab, M, S, Hkv, hd);
       count_launch(2);
     }
-    {
+    if constexpr (sizeof(T) == 2) {
+      SZO_TRY(launch_flash_attention_bf16(q, k, v, o, B, S, H, Hkv, hd, st));
+    } else {
       dim3 grid(static_cast<unsigned>(ceil_div(S, 4)), H, B);
       const float scale = 1.0f / sqrtf(static_cast<float>(hd));
       if (hd == 64) attn_warp_kernel<T, 64><<<grid, 128, 0, st>>>(q, k, v, o, S, H, Hkv, scale);
@@ -349,23 +389,23 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
       count_launch();
     }
     SZO_TRY(lin(l, 3, o, y));
-    residual_add_kernel<T><<<blocks_for(M * d, 256), 256, 0, st>>>(m->h, y, M * d);
+    residual_add_kernel<T><<<blocks_for(M * d / Vec16<T>::kN, 256), 256, 0, st>>>(m->h, y, M * d);
     norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, L.mlp_norm_g, L.mlp_norm_b, d, c.norm_eps, opt, 1,
                                                             0, a);
     count_launch(2);
     if (!opt) {
       SZO_TRY(lin(l, 4, a, gate));
       SZO_TRY(lin(l, 5, a, up));
-      silu_mul_kernel<T><<<blocks_for(M * ff, 256), 256, 0, st>>>(gate, up, M * ff, gate);
+      silu_mul_kernel<T><<<blocks_for(M * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, up, M * ff, gate);
       count_launch();
       SZO_TRY(lin(l, 6, gate, y));
     } else {
       SZO_TRY(lin(l, 4, a, gate));
-      relu_kernel<T><<<blocks_for(M * ff, 256), 256, 0, st>>>(gate, M * ff);
+      relu_kernel<T><<<blocks_for(M * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, M * ff);
       count_launch();
       SZO_TRY(lin(l, 5, gate, y));
     }
-    residual_add_kernel<T><<<blocks_for(M * d, 256), 256, 0, st>>>(m->h, y, M * d);
+    residual_add_kernel<T><<<blocks_for(M * d / Vec16<T>::kN, 256), 256, 0, st>>>(m->h, y, M * d);
     count_launch();
   }
   if (c.loss_kind == 0) {
@@ -424,6 +464,7 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
               "d_model %% n_heads and n_heads %% n_kv_heads must be 0");
   const int hd = c.d_model / c.n_heads;
   SZO_REQUIRE(hd == 64 || hd == 128, SZO_ERR_UNSUPPORTED, "head dimension must be 64 or 128 (got %d)", hd);
+  SZO_REQUIRE(c.d_model % 8 == 0 && c.d_ff % 8 == 0, SZO_ERR_SHAPE, "d_model and d_ff must be multiples of 8");
   SZO_REQUIRE(c.act_dtype == SZO_BF16 || c.act_dtype == SZO_F32, SZO_ERR_UNSUPPORTED, "act_dtype must be bf16 or f32");
   SZO_REQUIRE(c.act_dtype == SZO_BF16 || c.linear_mode == SZO_MODE_FP32_VALIDATE, SZO_ERR_UNSUPPORTED,
               "fp32 activations need the fp32 validation mode");
@@ -513,6 +554,25 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
     return bail(fail(SZO_ERR_CUDA, "model set-up kernels failed"));
 #undef SZO_M_TRY
   *out = m;
+  return SZO_OK;
+}
+
+szo_status szo_attention(const void* q, const void* k, const void* v, void* o, szo_dtype dtype, int32_t B, int32_t S,
+                         int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, void* stream) {
+  SZO_REQUIRE(q && k && v && o, SZO_ERR_INVALID_ARG, "NULL pointer");
+  SZO_REQUIRE(B > 0 && S > 0 && n_heads > 0 && n_kv_heads > 0 && n_heads % n_kv_heads == 0, SZO_ERR_SHAPE, "bad shape");
+  SZO_REQUIRE(head_dim == 64 || head_dim == 128, SZO_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
+  SZO_REQUIRE(dtype == SZO_BF16 || dtype == SZO_F32, SZO_ERR_UNSUPPORTED, "dtype must be bf16 or f32");
+  SZO_REQUIRE(aligned16(q) && aligned16(k) && aligned16(v) && aligned16(o), SZO_ERR_ALIGNMENT, "buffers must be 16-byte aligned");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (dtype == SZO_BF16) return launch_flash_attention_bf16(q, k, v, o, B, S, n_heads, n_kv_heads, head_dim, st);
+  dim3 grid(static_cast<unsigned>(ceil_div(S, 4)), n_heads, B);
+  const float scale = 1.0f / sqrtf(static_cast<float>(head_dim));
+  auto *qf = static_cast<const float*>(q), *kf = static_cast<const float*>(k), *vf = static_cast<const float*>(v);
+  if (head_dim == 64) attn_warp_kernel<float, 64><<<grid, 128, 0, st>>>(qf, kf, vf, static_cast<float*>(o), S, n_heads, n_kv_heads, scale);
+  else attn_warp_kernel<float, 128><<<grid, 128, 0, st>>>(qf, kf, vf, static_cast<float*>(o), S, n_heads, n_kv_heads, scale);
+  count_launch();
+  SZO_CHECK_LAUNCH("attn_warp_kernel");
   return SZO_OK;
 }
 

@@ -158,3 +158,19 @@ def test_model_argument_errors(B, tiny):
         m.loss(toks)
     assert ei.value.name == "SZO_ERR_SHAPE"
     m.close()
+
+
+@pytest.mark.parametrize("B_,S,H,Hkv,hd", [(2, 64, 4, 4, 64), (1, 256, 4, 2, 128), (3, 100, 2, 1, 128), (2, 37, 4, 2, 64),
+                                           (1, 200, 8, 8, 64)])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_attention_matches_oracle(B, B_, S, H, Hkv, hd, dtype):
+    g = wl.rng(3, wl.PURPOSE_ACTIVATION, S + hd)
+    mk = lambda heads: wl.bf16_round(g.standard_normal((B_ * S, heads * hd)).astype(np.float32))
+    q, k, v = mk(H), mk(Hkv), mk(Hkv)
+    t64 = lambda a, heads: torch.from_numpy(a.astype(np.float64)).view(B_, S, heads, hd)
+    ref = mo.causal_attention(t64(q, H), t64(k, Hkv), t64(v, Hkv)).reshape(B_ * S, H * hd).numpy()
+    dt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    d = lambda a: torch.from_numpy(a).cuda().to(dt)
+    got = B.szo_attention(d(q), d(k), d(v), B_, S, H, Hkv, hd).float().cpu().numpy()
+    tol = 1.5e-2 if dtype == "bf16" else 2e-6          # bf16: probabilities and outputs are rounded to bf16
+    assert np.max(np.abs(got - ref)) <= tol * np.max(np.abs(ref))
