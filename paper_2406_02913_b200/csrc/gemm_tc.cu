@@ -390,6 +390,7 @@ szo_status linear_fwd_tc(const szo_linear* p, const void* x, int64_t M, const ui
   P.sz = p->sz;
   P.bucket_ptr = p->bucket_ptr;
   P.n_kblocks = p->n_kblocks;
+  P.n_rowtiles = p->n_rowgroups;
   P.Npad = p->Npad;
   P.Sb = (p->nnz > 0) ? S_bucket : nullptr;
   P.bias = p->bias;
@@ -397,6 +398,13 @@ szo_status linear_fwd_tc(const szo_linear* p, const void* x, int64_t M, const ui
   P.status = device_status_word();
   SZO_REQUIRE(P.status != nullptr, SZO_ERR_CUDA, "no device status word");
   const CUtensorMap& mw = t->w_map;
+  if (M > 128) {
+    // pair tiles of 256 weight rows x 256 tokens on two-CTA clusters
+    SZO_TRY(make_map(&mx, x, M, p->K, 128));
+    P.m_tiles = ceil_div(M, 256);
+    P.n_tiles = ceil_div(p->N, 256);
+    return linear_fwd_tc2(p, mx, mw, P, t->sms, st);
+  }
   switch (BT) {
     case 16: return dispatch_kind<16, 6>(p, mx, mw, P, t->sms, st);
     case 32: return dispatch_kind<32, 6>(p, mx, mw, P, t->sms, st);

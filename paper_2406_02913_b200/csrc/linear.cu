@@ -358,7 +358,7 @@ szo_status szo_linear_create(szo_linear_t** out, int64_t N, int64_t K, int32_t G
   p->N = N; p->K = K; p->G = G; p->sz_dtype = sz_dtype; p->nnz = nnz;
   p->codes = codes_or_bf16_W; p->scales = scales; p->zeros = zeros; p->idx = idx; p->bias = bias;
   p->n_rowgroups = ceil_div(N, 128);
-  p->Npad = p->n_rowgroups * 128;
+  p->Npad = ceil_div(N, 256) * 256;   // the pair-tile kernel copies 128-row strips up to this bound
   p->n_kblocks = K / 64;
   const int64_t nb = p->n_rowgroups * p->n_kblocks;
   int32_t* cursor = nullptr;

@@ -15,7 +15,7 @@ struct szo_linear {
   const float* bias;
   // derived, owned by the plan (device memory)
   float2* sz;            // [K/G][Npad] (scale, zero) widened to fp32, group-major (G > 0)
-  int64_t Npad;          // N rounded up to a multiple of 128
+  int64_t Npad;          // N rounded up to a multiple of 256
   int32_t* ent_col;      // [nnz] column of entry e
   int32_t* row_ptr;      // [N+1] entries of row r are [row_ptr[r], row_ptr[r+1])
   int32_t* bucket_ptr;   // [n_rowgroups * n_kblocks + 1]; bucket = (row/128, col/64)

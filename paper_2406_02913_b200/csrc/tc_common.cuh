@@ -33,6 +33,7 @@ struct TcParams {
   int64_t Npad;
   const int32_t* bucket_ptr;
   int64_t n_kblocks;       // buckets per 128-row tile
+  int64_t n_rowtiles;      // number of 128-row tiles that have buckets
   const uint2* Sb;         // sparse records (position in tile, value bits) in bucket order; nullptr: none
   const float* bias;
   void* y;
@@ -191,4 +192,10 @@ __device__ __forceinline__ uint4 dequant_word(uint32_t w, float2 p) {
 
 
 }  // namespace tc
+
+// Two-CTA pair-tile kernel (gemm_tc2.cu): tmap_x has a [128 x 64] box; P.m_tiles / P.n_tiles count
+// 256-wide tiles.
+szo_status linear_fwd_tc2(const szo_linear* p, const CUtensorMap& mx, const CUtensorMap& mw, const tc::TcParams& P,
+                          int sms, cudaStream_t st);
+
 }  // namespace szo
