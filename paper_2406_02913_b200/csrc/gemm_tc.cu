@@ -18,6 +18,8 @@
 //                accumulator so the next tile's main loop overlaps
 // Every mbarrier wait is bounded; on expiry the kernel records SZO_ERR_TIMEOUT in the device status
 // word, lets in-flight copies land, frees its TMEM and returns.
+#include <cstdlib>
+
 #include "tc_common.cuh"
 
 namespace szo {
@@ -398,7 +400,12 @@ szo_status linear_fwd_tc(const szo_linear* p, const void* x, int64_t M, const ui
   P.status = device_status_word();
   SZO_REQUIRE(P.status != nullptr, SZO_ERR_CUDA, "no device status word");
   const CUtensorMap& mw = t->w_map;
-  if (M > 128) {
+  // SZO_LINEAR_KERNEL=1cta|2cta selects the kernel for M > 128 (A/B measurement); default below.
+  static const int forced = [] {
+    const char* e = getenv("SZO_LINEAR_KERNEL");
+    return (e && e[0] == '1') ? 1 : (e && e[0] == '2') ? 2 : 0;
+  }();
+  if (M > 128 && forced != 1) {
     // pair tiles of 256 weight rows x 256 tokens on two-CTA clusters
     SZO_TRY(make_map(&mx, x, M, p->K, 128));
     P.m_tiles = ceil_div(M, 256);
