@@ -29,19 +29,31 @@ namespace {
 using namespace tc;
 
 // ------------------------------------------------------------------------------ the kernel
+// Three rings in shared memory, each with its own life time:
+//   X ring  token tile [BT x 64] bf16 (+ the bf16 weight tile in dense mode): TMA -> MMA
+//   C ring  packed codes [128 x 32 B] + (scale, zero) strip of the k-block:      TMA -> conversion
+//   A ring  dequantised weight tile [128 x 64] bf16, swizzled K-major:           conversion -> MMA
+// so that the small code tiles can be fetched far ahead while the large token tiles are held only
+// for the TMA latency.  The eight conversion warps form kGroups groups that take alternate
+// k-blocks, which keeps several stages in conversion at once.
 // kDequant: A tile produced from int4 codes (else loaded as bf16 by TMA).  kFast: bf16 scales/zeros.
-template <int BT, int kStages, bool kDequant, bool kFast>
+template <int BT, int kXS, bool kDequant, bool kFast>
 __global__ void __launch_bounds__(kNumWarps * 32, 1)
 szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                      const TcParams P) {
   constexpr int kBTileBytes = BT * kBK * 2;
-  constexpr int kStageBytes = kATileBytes + kBTileBytes + (kDequant ? kCodesBytes + kSzBytes : 0);
+  constexpr int kXStageBytes = kBTileBytes + (kDequant ? 0 : kATileBytes);
+  constexpr int kCStageBytes = kCodesBytes + kSzBytes;
+  constexpr int kCS = kDequant ? 6 : 1;                      // C ring stages
+  constexpr int kAS = kDequant ? 3 : kXS;                    // A ring slots (dense: the X stage itself)
+  constexpr int kGroups = 2, kWarpsPerGroup = kNumDeqWarps / kGroups;
   constexpr int kAccStride = BT < 32 ? 32 : BT;             // TMEM columns per accumulator buffer
   constexpr uint32_t kTmemCols = static_cast<uint32_t>(2 * kAccStride);
   constexpr uint32_t kIdesc = make_idesc(kBM, BT);
+  constexpr uint32_t kXBase = 0, kCBase = kXS * kXStageBytes, kABase = kCBase + (kDequant ? kCS * kCStageBytes : 0);
 
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[4 * kStages + 4];
+  __shared__ __align__(8) unsigned long long bars[2 * kXS + 2 * kCS + 3 * kAS + 4];
   __shared__ __align__(16) uint2 rec_ring[kRecSlots][kRecCap];      // sparse records, per k-block
   __shared__ __align__(8) int32_t bound_ring[kBoundSlots][2];
   __shared__ uint32_t tmem_base_slot;
@@ -52,24 +64,36 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &abort_flag_s;
 
-  auto full_bar = [&](int s) { return smem_u32(&bars[s]); };              // TMA bytes landed
-  auto deq_bar = [&](int s) { return smem_u32(&bars[kStages + s]); };     // dequantised tile written
-  auto aready_bar = [&](int s) { return smem_u32(&bars[2 * kStages + s]); };  // sparse values added
-  auto empty_bar = [&](int s) { return smem_u32(&bars[3 * kStages + s]); };   // MMAs of the stage done
-  auto accfull_bar = [&](int a) { return smem_u32(&bars[4 * kStages + a]); };
-  auto accempty_bar = [&](int a) { return smem_u32(&bars[4 * kStages + 2 + a]); };
-  auto a_tile = [&](int s) { return tiles_base + static_cast<uint32_t>(s) * kStageBytes; };
-  auto b_tile = [&](int s) { return tiles_base + static_cast<uint32_t>(s) * kStageBytes + kATileBytes; };
-  auto c_tile = [&](int s) { return tiles_base + static_cast<uint32_t>(s) * kStageBytes + kATileBytes + kBTileBytes; };
+  auto xfull_bar = [&](int s) { return smem_u32(&bars[s]); };                  // X stage landed (TMA)
+  auto xempty_bar = [&](int s) { return smem_u32(&bars[kXS + s]); };           // its MMAs retired
+  auto cfull_bar = [&](int c) { return smem_u32(&bars[2 * kXS + c]); };        // C stage landed (TMA)
+  auto cempty_bar = [&](int c) { return smem_u32(&bars[2 * kXS + kCS + c]); }; // converted by its group
+  auto adone_bar = [&](int t) { return smem_u32(&bars[2 * kXS + 2 * kCS + t]); };            // A slot written
+  auto aready_bar = [&](int t) { return smem_u32(&bars[2 * kXS + 2 * kCS + kAS + t]); };     // sparse values added
+  auto aempty_bar = [&](int t) { return smem_u32(&bars[2 * kXS + 2 * kCS + 2 * kAS + t]); }; // its MMAs retired
+  auto accfull_bar = [&](int a) { return smem_u32(&bars[2 * kXS + 2 * kCS + 3 * kAS + a]); };
+  auto accempty_bar = [&](int a) { return smem_u32(&bars[2 * kXS + 2 * kCS + 3 * kAS + 2 + a]); };
+  auto b_off = [&](int s) { return kXBase + static_cast<uint32_t>(s) * kXStageBytes; };
+  auto c_off = [&](int c) { return kCBase + static_cast<uint32_t>(c) * kCStageBytes; };
+  auto a_off = [&](int s, int t) {     // weight tile of iteration (X stage s, A slot t)
+    return kDequant ? kABase + static_cast<uint32_t>(t) * kATileBytes : b_off(s) + kBTileBytes;
+  };
 
   const bool sparse = P.Sb != nullptr;
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(full_bar(s), 1);
-      mbar_init(deq_bar(s), kNumDeqWarps);
-      mbar_init(aready_bar(s), 1);
-      mbar_init(empty_bar(s), 1);
+    for (int s = 0; s < kXS; ++s) {
+      mbar_init(xfull_bar(s), 1);
+      mbar_init(xempty_bar(s), 1);
+    }
+    for (int c = 0; c < kCS; ++c) {
+      mbar_init(cfull_bar(c), 1);
+      mbar_init(cempty_bar(c), kWarpsPerGroup);
+    }
+    for (int t = 0; t < kAS; ++t) {
+      mbar_init(adone_bar(t), kWarpsPerGroup);
+      mbar_init(aready_bar(t), 1);
+      mbar_init(aempty_bar(t), 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(accfull_bar(a), 1);
@@ -89,27 +113,37 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
   auto tile_of = [&](int64_t it) { return blockIdx.x + (it / P.nkb) * gridDim.x; };
 
   if (warp == 0) {
-    // ---------------------------------------------------------------- TMA producer
+    // ---------------------------------------------------------------- X producer (token tiles)
     if (lane == 0) {
-      const int groups_kb = (kDequant && P.G < kBK) ? kBK / P.G : 1;   // scale groups per k-block
       for (int64_t it = 0; it < my_iters; ++it) {
         const int64_t tile = tile_of(it);
         const int kb = static_cast<int>(it % P.nkb);
-        const int64_t n_tile = tile / P.m_tiles, m_tile = tile % P.m_tiles;
-        const int s = static_cast<int>(it % kStages);
-        const uint32_t ph = static_cast<uint32_t>((it / kStages) & 1);
-        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, P.status)) break;
-        if constexpr (kDequant) {
-          mbar_expect_tx(full_bar(s), kBTileBytes + kCodesBytes + groups_kb * 1024);
-          tma_load_2d(c_tile(s), &tmap_w, kb * (kBK / 2), static_cast<int>(n_tile * kBM), full_bar(s));
+        const int s = static_cast<int>(it % kXS);
+        const uint32_t ph = static_cast<uint32_t>((it / kXS) & 1);
+        if (!mbar_wait(xempty_bar(s), ph ^ 1u, abort_flag, P.status)) break;
+        mbar_expect_tx(xfull_bar(s), kXStageBytes);
+        tma_load_2d(tiles_base + b_off(s), &tmap_x, kb * kBK, static_cast<int>((tile % P.m_tiles) * BT), xfull_bar(s));
+        if constexpr (!kDequant)
+          tma_load_2d(tiles_base + a_off(s, 0), &tmap_w, kb * kBK, static_cast<int>((tile / P.m_tiles) * kBM), xfull_bar(s));
+      }
+    }
+  } else if (warp == 3) {
+    // ---------------------------------------------------------------- C producer (codes, scale/zero)
+    if constexpr (kDequant) {
+      if (lane == 0) {
+        const int groups_kb = (P.G < kBK) ? kBK / P.G : 1;     // scale groups per k-block
+        for (int64_t it = 0; it < my_iters; ++it) {
+          const int kb = static_cast<int>(it % P.nkb);
+          const int64_t n0 = (tile_of(it) / P.m_tiles) * kBM;
+          const int c = static_cast<int>(it % kCS);
+          const uint32_t ph = static_cast<uint32_t>((it / kCS) & 1);
+          if (!mbar_wait(cempty_bar(c), ph ^ 1u, abort_flag, P.status)) break;
+          mbar_expect_tx(cfull_bar(c), kCodesBytes + groups_kb * 1024);
+          tma_load_2d(tiles_base + c_off(c), &tmap_w, kb * (kBK / 2), static_cast<int>(n0), cfull_bar(c));
           const int64_t g0 = (static_cast<int64_t>(kb) * kBK) / P.G;
           for (int g = 0; g < groups_kb; ++g)
-            bulk_load_1d(c_tile(s) + kCodesBytes + g * 1024, P.sz + (g0 + g) * P.Npad + n_tile * kBM, 1024, full_bar(s));
-        } else {
-          mbar_expect_tx(full_bar(s), kBTileBytes + kATileBytes);
-          tma_load_2d(a_tile(s), &tmap_w, kb * kBK, static_cast<int>(n_tile * kBM), full_bar(s));
+            bulk_load_1d(tiles_base + c_off(c) + kCodesBytes + g * 1024, P.sz + (g0 + g) * P.Npad + n0, 1024, cfull_bar(c));
         }
-        tma_load_2d(b_tile(s), &tmap_x, kb * kBK, static_cast<int>(m_tile * BT), full_bar(s));
       }
     }
   } else if (warp == 1) {
@@ -124,22 +158,23 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kAccStride);
         for (int kb = 0; kb < P.nkb; ++kb) {
           const int64_t it = lt * P.nkb + kb;
-          const int s = static_cast<int>(it % kStages);
-          const uint32_t ph = static_cast<uint32_t>((it / kStages) & 1);
-          if (!mbar_wait(full_bar(s), ph, abort_flag, P.status)) { ok = false; break; }
+          const int s = static_cast<int>(it % kXS), t = static_cast<int>(it % kAS);
+          const uint32_t ph = static_cast<uint32_t>((it / kXS) & 1), pht = static_cast<uint32_t>((it / kAS) & 1);
+          if (!mbar_wait(xfull_bar(s), ph, abort_flag, P.status)) { ok = false; break; }
           if (sparse) {
-            if (!mbar_wait(aready_bar(s), ph, abort_flag, P.status)) { ok = false; break; }
+            if (!mbar_wait(aready_bar(t), pht, abort_flag, P.status)) { ok = false; break; }
           } else if (kDequant) {
-            if (!mbar_wait(deq_bar(s), ph, abort_flag, P.status)) { ok = false; break; }
+            if (!mbar_wait(adone_bar(t), pht, abort_flag, P.status)) { ok = false; break; }
           }
           tc_fence_after();
-          const uint64_t adesc = make_desc_sw128(a_tile(s)), bdesc = make_desc_sw128(b_tile(s));
+          const uint64_t adesc = make_desc_sw128(tiles_base + a_off(s, t)), bdesc = make_desc_sw128(tiles_base + b_off(s));
 #pragma unroll
           for (int k = 0; k < kBK / kUmmaK; ++k) {
             // advance both descriptors by 16 elements = 32 bytes (>> 4 = 2) inside the swizzle row
             umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc, (kb | k) ? 1u : 0u);
           }
-          umma_commit(empty_bar(s));
+          umma_commit(xempty_bar(s));
+          if constexpr (kDequant) umma_commit(aempty_bar(t));
         }
         if (ok) umma_commit(accfull_bar(as));
       }
@@ -171,8 +206,8 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
         cp_async_commit();
       }
       for (int64_t it = 0; it < my_iters; ++it) {
-        const int s = static_cast<int>(it % kStages);
-        const uint32_t ph = static_cast<uint32_t>((it / kStages) & 1);
+        const int s = static_cast<int>(it % kXS), t = static_cast<int>(it % kAS);
+        const uint32_t ph = static_cast<uint32_t>((it / kXS) & 1), pht = static_cast<uint32_t>((it / kAS) & 1);
         // group(j) = { bounds(j + 2 kLook), records(j + kLook) }, committed in iteration j.  Groups
         // retire in order: with at most kLook - 1 still pending, group(it - kLook) has landed, i.e.
         // records(it) and bounds(it + kLook), which the next record copies are addressed from.
@@ -182,8 +217,8 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
         issue_records(it + kLook);
         cp_async_commit();
         const int32_t e0 = bound_ring[it % kBoundSlots][0], e1 = bound_ring[it % kBoundSlots][1];
-        if (!mbar_wait(kDequant ? deq_bar(s) : full_bar(s), ph, abort_flag, P.status)) break;
-        unsigned char* A = tiles_ptr + static_cast<size_t>(s) * kStageBytes;
+        if (!mbar_wait(kDequant ? adone_bar(t) : xfull_bar(s), kDequant ? pht : ph, abort_flag, P.status)) break;
+        unsigned char* A = tiles_ptr + a_off(s, t);
         for (int32_t j = lane; j < e1 - e0; j += 32) {
           const uint2 rec = (j < kRecCap) ? rec_ring[it % kRecSlots][j] : __ldg(P.Sb + e0 + j);
           const int r = static_cast<int>(rec.x >> 6), c = static_cast<int>(rec.x & 63);
@@ -192,35 +227,48 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
         }
         fence_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(aready_bar(s));
+        if (lane == 0) mbar_arrive(aready_bar(t));
       }
       cp_async_wait_all();
     }
   } else if (warp >= kDeqWarp0 && warp < kDeqWarp0 + kNumDeqWarps) {
-    // ---------------------------------------------------------------- dequantisation warps
-    // codes and (scale, zero) of the stage are already in shared memory (TMA); each warp converts
-    // rows [16 dw, 16 dw + 16): per pass 4 rows x 8 sixteen-byte chunks, conflict-free both ways.
+    // ---------------------------------------------------------------- conversion warps
+    // Group gq converts the k-blocks it = gq (mod kGroups); inside a group each warp converts 32 rows
+    // in eight passes of 4 rows x 8 sixteen-byte chunks (conflict-free loads and stores).
     if constexpr (kDequant) {
       const int dw = warp - kDeqWarp0;
+      const int gq = dw / kWarpsPerGroup, wq = dw % kWarpsPerGroup;
+      constexpr int kRowsPerWarp = kBM / kWarpsPerGroup, kPasses = kRowsPerWarp / 4;
       const int sub = lane >> 3, chunk = lane & 7;
       const int gsel = (P.G < kBK) ? (chunk * 8) / P.G : 0;
-      for (int64_t it = 0; it < my_iters; ++it) {
-        const int s = static_cast<int>(it % kStages);
-        const uint32_t ph = static_cast<uint32_t>((it / kStages) & 1);
-        unsigned char* A = tiles_ptr + static_cast<size_t>(s) * kStageBytes;
-        const unsigned char* C = A + kATileBytes + kBTileBytes;
+      for (int64_t it = gq; it < my_iters; it += kGroups) {
+        const int c = static_cast<int>(it % kCS), t = static_cast<int>(it % kAS);
+        const uint32_t phc = static_cast<uint32_t>((it / kCS) & 1), pht = static_cast<uint32_t>((it / kAS) & 1);
+        unsigned char* A = tiles_ptr + a_off(0, t);
+        const unsigned char* C = tiles_ptr + c_off(c);
         const float2* SZ = reinterpret_cast<const float2*>(C + kCodesBytes) + gsel * kBM;
-        if (!mbar_wait(full_bar(s), ph, abort_flag, P.status)) break;
+        if (!mbar_wait(cfull_bar(c), phc, abort_flag, P.status)) break;
+        uint32_t w[kPasses];
+        float2 zs[kPasses];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int r = dw * 16 + i * 4 + sub;
-          const uint32_t w = *reinterpret_cast<const uint32_t*>(C + r * 32 + chunk * 4);
-          const uint4 v = dequant_word<kFast>(w, SZ[r]);
+        for (int i = 0; i < kPasses; ++i) {
+          const int r = wq * kRowsPerWarp + i * 4 + sub;
+          w[i] = *reinterpret_cast<const uint32_t*>(C + r * 32 + chunk * 4);
+          zs[i] = SZ[r];
+        }
+        if (!mbar_wait(aempty_bar(t), pht ^ 1u, abort_flag, P.status)) break;
+#pragma unroll
+        for (int i = 0; i < kPasses; ++i) {
+          const int r = wq * kRowsPerWarp + i * 4 + sub;
+          const uint4 v = dequant_word<kFast>(w[i], zs[i]);
           *reinterpret_cast<uint4*>(A + r * 128 + ((chunk ^ (r & 7)) << 4)) = v;
         }
         fence_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(deq_bar(s));
+        if (lane == 0) {
+          mbar_arrive(adone_bar(t));
+          mbar_arrive(cempty_bar(c));
+        }
       }
     }
   } else if (warp >= kEpiWarp0) {
@@ -328,11 +376,11 @@ szo_status make_codes_map(CUtensorMap* map, const void* base, int64_t rows, int6
   return SZO_OK;
 }
 
-template <int BT, int kStages, bool kDequant, bool kFast>
+template <int BT, int kXS, bool kDequant, bool kFast>
 szo_status launch_tc(const CUtensorMap& mx, const CUtensorMap& mw, const TcParams& P, int sms, cudaStream_t st) {
-  constexpr size_t smem =
-      static_cast<size_t>(kStages) * (kATileBytes + BT * kBK * 2 + (kDequant ? kCodesBytes + kSzBytes : 0)) + 1024;
-  auto kern = szo_linear_tc_kernel<BT, kStages, kDequant, kFast>;
+  constexpr size_t smem = static_cast<size_t>(kXS) * (BT * kBK * 2 + (kDequant ? 0 : kATileBytes)) +
+                          (kDequant ? 6 * (kCodesBytes + kSzBytes) + 3 * kATileBytes : 0) + 1024;
+  auto kern = szo_linear_tc_kernel<BT, kXS, kDequant, kFast>;
   static bool configured = false;
   if (!configured) {
     SZO_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
@@ -346,12 +394,13 @@ szo_status launch_tc(const CUtensorMap& mx, const CUtensorMap& mw, const TcParam
   return SZO_OK;
 }
 
-template <int BT, int kStages>
+// kXD / kXQ: token-tile stages in dense and in dequantising mode (the latter also holds the C and A rings)
+template <int BT, int kXD, int kXQ>
 szo_status dispatch_kind(const szo_linear* p, const CUtensorMap& mx, const CUtensorMap& mw, const TcParams& P, int sms,
                          cudaStream_t st) {
-  if (p->G == 0) return launch_tc<BT, kStages, false, false>(mx, mw, P, sms, st);
-  if (p->sz_dtype == SZO_BF16) return launch_tc<BT, kStages, true, true>(mx, mw, P, sms, st);
-  return launch_tc<BT, kStages, true, false>(mx, mw, P, sms, st);
+  if (p->G == 0) return launch_tc<BT, kXD, false, false>(mx, mw, P, sms, st);
+  if (p->sz_dtype == SZO_BF16) return launch_tc<BT, kXQ, true, true>(mx, mw, P, sms, st);
+  return launch_tc<BT, kXQ, true, false>(mx, mw, P, sms, st);
 }
 
 }  // namespace
@@ -400,12 +449,13 @@ szo_status linear_fwd_tc(const szo_linear* p, const void* x, int64_t M, const ui
   P.status = device_status_word();
   SZO_REQUIRE(P.status != nullptr, SZO_ERR_CUDA, "no device status word");
   const CUtensorMap& mw = t->w_map;
-  // SZO_LINEAR_KERNEL=1cta|2cta selects the kernel for M > 128 (A/B measurement); default below.
+  // SZO_LINEAR_KERNEL=2cta selects the pair-tile kernel for M > 128 (A/B measurement); the one-CTA
+  // kernel measured faster and is the default.
   static const int forced = [] {
     const char* e = getenv("SZO_LINEAR_KERNEL");
     return (e && e[0] == '1') ? 1 : (e && e[0] == '2') ? 2 : 0;
   }();
-  if (M > 128 && forced != 1) {
+  if (M > 128 && forced == 2) {
     // pair tiles of 256 weight rows x 256 tokens on two-CTA clusters
     SZO_TRY(make_map(&mx, x, M, p->K, 128));
     P.m_tiles = ceil_div(M, 256);
@@ -413,11 +463,11 @@ szo_status linear_fwd_tc(const szo_linear* p, const void* x, int64_t M, const ui
     return linear_fwd_tc2(p, mx, mw, P, t->sms, st);
   }
   switch (BT) {
-    case 16: return dispatch_kind<16, 6>(p, mx, mw, P, t->sms, st);
-    case 32: return dispatch_kind<32, 6>(p, mx, mw, P, t->sms, st);
-    case 64: return dispatch_kind<64, 6>(p, mx, mw, P, t->sms, st);
-    case 128: return dispatch_kind<128, 5>(p, mx, mw, P, t->sms, st);
-    default: return dispatch_kind<256, 4>(p, mx, mw, P, t->sms, st);
+    case 16: return dispatch_kind<16, 8, 8>(p, mx, mw, P, t->sms, st);
+    case 32: return dispatch_kind<32, 8, 8>(p, mx, mw, P, t->sms, st);
+    case 64: return dispatch_kind<64, 8, 8>(p, mx, mw, P, t->sms, st);
+    case 128: return dispatch_kind<128, 6, 6>(p, mx, mw, P, t->sms, st);
+    default: return dispatch_kind<256, 4, 4>(p, mx, mw, P, t->sms, st);
   }
 }
 

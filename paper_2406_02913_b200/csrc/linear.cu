@@ -7,15 +7,22 @@
 namespace szo {
 
 // ------------------------------------------------------------------------------ plan kernels
-// (scale, zero) widened to fp32 and transposed to [K/G][Npad] so that the 128 rows of a tile are
-// contiguous for one group (one bulk copy per tile and k-block).
+// Kernel-ready (scale, zero) table, transposed to [K/G][Npad] so that the 128 rows of a tile are
+// contiguous for one group (one bulk copy per tile and k-block).  fp16 inputs are widened to fp32
+// pairs; bf16 inputs are stored as the bit patterns of the packed pairs (scale,scale), (zero,zero)
+// that the packed-bf16 conversion consumes directly.
+__device__ __forceinline__ float2 sz_entry(__half s, __half z) { return make_float2(__half2float(s), __half2float(z)); }
+__device__ __forceinline__ float2 sz_entry(__nv_bfloat16 s, __nv_bfloat16 z) {
+  const uint32_t sb = *reinterpret_cast<const uint16_t*>(&s), zb = *reinterpret_cast<const uint16_t*>(&z);
+  return make_float2(__uint_as_float(sb | (sb << 16)), __uint_as_float(zb | (zb << 16)));
+}
 template <typename SZ>
 __global__ void widen_sz_kernel(const SZ* __restrict__ scales, const SZ* __restrict__ zeros, int64_t N,
                                 int64_t groups, int64_t Npad, float2* __restrict__ out) {
   const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i >= N * groups) return;
   const int64_t n = i / groups, g = i % groups;
-  out[g * Npad + n] = make_float2(static_cast<float>(scales[i]), static_cast<float>(zeros[i]));
+  out[g * Npad + n] = sz_entry(scales[i], zeros[i]);
 }
 
 // Per entry: column, validity (strictly ascending, in range) and the size of its (128-row, 64-col)
@@ -92,16 +99,18 @@ __global__ void bucket_fill_kernel(const int64_t* __restrict__ idx, const int32_
 }
 
 // ------------------------------------------------------------------------------ fp32 path
-// W_eff[n, c] = fma(q, scale, zero) in fp32 (two elements per thread), or the widened bf16 weight.
-__global__ void dequant_f32_kernel(const uint8_t* __restrict__ codes, const float2* __restrict__ sz,
-                                   int64_t N, int64_t K, int G, int64_t Npad, float* __restrict__ W) {
+// W_eff[n, c] = fma(q, scale, zero) in fp32 (two elements per thread), from the caller's tables.
+template <typename SZ>
+__global__ void dequant_f32_kernel(const uint8_t* __restrict__ codes, const SZ* __restrict__ scales,
+                                   const SZ* __restrict__ zeros, int64_t N, int64_t K, int G, float* __restrict__ W) {
   const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (t >= N * K / 2) return;
   const int64_t n = (2 * t) / K, c = (2 * t) % K;
-  const float2 p = sz[(c / G) * Npad + n];
+  const int64_t gi = n * (K / G) + c / G;
+  const float s = static_cast<float>(scales[gi]), z = static_cast<float>(zeros[gi]);
   const uint8_t b = codes[t];
-  W[2 * t] = fmaf(static_cast<float>(b & 15), p.x, p.y);
-  W[2 * t + 1] = fmaf(static_cast<float>(b >> 4), p.x, p.y);
+  W[2 * t] = fmaf(static_cast<float>(b & 15), s, z);
+  W[2 * t + 1] = fmaf(static_cast<float>(b >> 4), s, z);
 }
 
 __global__ void widen_bf16_kernel(const __nv_bfloat16* __restrict__ in, int64_t n, float* __restrict__ out) {
@@ -185,8 +194,14 @@ szo_status linear_fwd_fp32(const szo_linear* p, const void* x, int x_dtype, int6
   float* W = static_cast<float*>(ws);
   const int64_t NK = p->N * p->K;
   if (p->G > 0) {
-    dequant_f32_kernel<<<static_cast<unsigned>(ceil_div(NK / 2, 256)), 256, 0, st>>>(
-        static_cast<const uint8_t*>(p->codes), p->sz, p->N, p->K, p->G, p->Npad, W);
+    if (p->sz_dtype == SZO_BF16)
+      dequant_f32_kernel<__nv_bfloat16><<<static_cast<unsigned>(ceil_div(NK / 2, 256)), 256, 0, st>>>(
+          static_cast<const uint8_t*>(p->codes), static_cast<const __nv_bfloat16*>(p->scales),
+          static_cast<const __nv_bfloat16*>(p->zeros), p->N, p->K, p->G, W);
+    else
+      dequant_f32_kernel<__half><<<static_cast<unsigned>(ceil_div(NK / 2, 256)), 256, 0, st>>>(
+          static_cast<const uint8_t*>(p->codes), static_cast<const __half*>(p->scales),
+          static_cast<const __half*>(p->zeros), p->N, p->K, p->G, W);
   } else {
     widen_bf16_kernel<<<static_cast<unsigned>(ceil_div(NK, 256)), 256, 0, st>>>(
         static_cast<const __nv_bfloat16*>(p->codes), NK, W);

@@ -29,7 +29,7 @@ struct TcParams {
   int nkb;                 // K / 64
   int64_t m_tiles, n_tiles;
   const uint8_t* codes;    // [N, K/2]
-  const float2* sz;        // [K/G][Npad]
+  const float2* sz;        // [K/G][Npad]; fp32 (scale, zero), or packed bf16 pairs when kFast
   int64_t Npad;
   const int32_t* bucket_ptr;
   int64_t n_kblocks;       // buckets per 128-row tile
@@ -163,19 +163,32 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&v);
 }
 
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+  return d;
+}
+
 // Eight codes of one 32-bit word -> eight bf16 values q*scale+zero (one rounding each).
+// kFast (bf16 scales/zeros): p carries the bit patterns of the packed pairs (scale,scale) and
+// (zero,zero); the arithmetic is exact packed bf16: (128+q) as bf16 is 0x4300|q, minus 128, then
+// one fused multiply-add.  Otherwise p = (scale, zero) in fp32: fp32 fma, then one conversion.
 template <bool kFast>
 __device__ __forceinline__ uint4 dequant_word(uint32_t w, float2 p) {
   uint32_t o[4];
   if constexpr (kFast) {
-    // scale and zero are bf16 values: exact packed arithmetic.  (128+q) as bf16 is 0x4300|q.
-    const __nv_bfloat162 s2 = __floats2bfloat162_rn(p.x, p.x), z2 = __floats2bfloat162_rn(p.y, p.y);
+    const uint32_t sb = __float_as_uint(p.x), zb = __float_as_uint(p.y);
+    const __nv_bfloat162 s2 = *reinterpret_cast<const __nv_bfloat162*>(&sb);
+    const __nv_bfloat162 z2 = *reinterpret_cast<const __nv_bfloat162*>(&zb);
     const uint32_t magic = 0x43004300u;
     const __nv_bfloat162 m2 = *reinterpret_cast<const __nv_bfloat162*>(&magic);
+    const uint32_t lo = w & 0x0F0F0F0Fu;          // codes of the even columns, one per byte
+    const uint32_t hi = (w >> 4) & 0x0F0F0F0Fu;   // codes of the odd columns
+    // byte permute: [lo.byte[i], 0, hi.byte[i], 0]; selector bit 3 replicates the (zero) sign bit
+    const uint32_t sel[4] = {0x8480u, 0x9591u, 0xA6A2u, 0xB7B3u};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const uint32_t x = w >> (8 * i);
-      const uint32_t t = (x & 0xFu) | ((x << 12) & 0xF0000u) | magic;
+      const uint32_t t = prmt(lo, hi, sel[i]) | magic;
       const __nv_bfloat162 q2 = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&t), m2);
       const __nv_bfloat162 r = __hfma2(q2, s2, z2);
       o[i] = *reinterpret_cast<const uint32_t*>(&r);
@@ -192,7 +205,6 @@ __device__ __forceinline__ uint4 dequant_word(uint32_t w, float2 p) {
   }
   return make_uint4(o[0], o[1], o[2], o[3]);
 }
-
 
 }  // namespace tc
 
