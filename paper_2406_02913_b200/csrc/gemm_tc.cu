@@ -139,7 +139,8 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
           const uint32_t ph = static_cast<uint32_t>((it / kCS) & 1);
           if (!mbar_wait(cempty_bar(c), ph ^ 1u, abort_flag, P.status)) break;
           mbar_expect_tx(cfull_bar(c), kCodesBytes + groups_kb * 1024);
-          tma_load_2d(tiles_base + c_off(c), &tmap_w, kb * (kBK / 2), static_cast<int>(n0), cfull_bar(c));
+          bulk_load_1d(tiles_base + c_off(c), P.codes + ((n0 / kBM) * P.nkb + kb) * static_cast<int64_t>(kCodesBytes),
+                       kCodesBytes, cfull_bar(c));
           const int64_t g0 = (static_cast<int64_t>(kb) * kBK) / P.G;
           for (int g = 0; g < groups_kb; ++g)
             bulk_load_1d(tiles_base + c_off(c) + kCodesBytes + g * 1024, P.sz + (g0 + g) * P.Npad + n0, 1024, cfull_bar(c));
@@ -410,6 +411,8 @@ szo_status tc_plan_create(szo_linear* p, cudaStream_t) {
   int dev = 0;
   t->sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&t->sms, cudaDevAttrMultiProcessorCount, dev);
+  // the dense bf16 weight is fetched by TMA; packed codes are fetched with plain bulk copies from the
+  // plan's tile-ordered copy, so that map only has to be valid (it is never used)
   const szo_status s = (p->G == 0) ? make_map(&t->w_map, p->codes, p->N, p->K, kBM)
                                    : make_codes_map(&t->w_map, p->codes, p->N, p->K / 2);
   if (s != SZO_OK) {
@@ -437,7 +440,7 @@ szo_status linear_fwd_tc(const szo_linear* p, const void* x, int64_t M, const ui
   TcParams P{};
   P.M = M; P.N = p->N; P.K = p->K; P.G = p->G; P.nkb = static_cast<int>(p->K / kBK);
   P.m_tiles = ceil_div(M, BT); P.n_tiles = ceil_div(p->N, kBM);
-  P.codes = static_cast<const uint8_t*>(p->codes);
+  P.codes = p->codes_tiled;
   P.sz = p->sz;
   P.bucket_ptr = p->bucket_ptr;
   P.n_kblocks = p->n_kblocks;

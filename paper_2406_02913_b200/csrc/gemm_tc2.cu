@@ -180,7 +180,8 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, P.status)) break;
         if constexpr (kDequant) {
           mbar_expect_tx(full_bar(s), kBHalfBytes + kCodesBytes + groups_kb * 1024);
-          tma_load_2d(c_tile(s), &tmap_w, kb * (kBK / 2), static_cast<int>(row0), full_bar(s));
+          bulk_load_1d(c_tile(s), P.codes + ((row0 / kBM) * P.nkb + kb) * static_cast<int64_t>(kCodesBytes), kCodesBytes,
+                       full_bar(s));
           const int64_t g0 = (static_cast<int64_t>(kb) * kBK) / P.G;
           for (int g = 0; g < groups_kb; ++g)
             bulk_load_1d(c_tile(s) + kCodesBytes + g * 1024, P.sz + (g0 + g) * P.Npad + row0, 1024, full_bar(s));

@@ -25,6 +25,22 @@ __global__ void widen_sz_kernel(const SZ* __restrict__ scales, const SZ* __restr
   out[g * Npad + n] = sz_entry(scales[i], zeros[i]);
 }
 
+// Copy of the packed codes in tile order: block (t, kb) holds rows [128 t, 128 t + 128) x bytes
+// [32 kb, 32 kb + 32) of the caller's [N, K/2] array, 4 KiB contiguous, rows beyond N zero.  One thread
+// moves 16 bytes.
+__global__ void tile_codes_kernel(const uint8_t* __restrict__ codes, int64_t N, int64_t K, int64_t n_tiles,
+                                  uint8_t* __restrict__ out) {
+  const int64_t nkb = K / 64;
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;     // 16-byte unit
+  if (i >= n_tiles * nkb * 256) return;
+  const int64_t half = i & 1, r = (i >> 1) & 127, blk = i >> 8;
+  const int64_t t = blk / nkb, kb = blk % nkb;
+  const int64_t row = t * 128 + r;
+  uint4 v = make_uint4(0u, 0u, 0u, 0u);
+  if (row < N) v = *reinterpret_cast<const uint4*>(codes + row * (K / 2) + kb * 32 + half * 16);
+  *reinterpret_cast<uint4*>(out + i * 16) = v;
+}
+
 // Per entry: column, validity (strictly ascending, in range) and the size of its (128-row, 64-col)
 // bucket, counted into bucket_ptr[b + 1].
 __global__ void entry_kernel(const int64_t* __restrict__ idx, int64_t nnz, int64_t N, int64_t K,
@@ -333,6 +349,7 @@ static void free_plan(szo_linear* p) {
   if (!p) return;
   tc_plan_destroy(p);
   cudaFree(p->sz);
+  cudaFree(p->codes_tiled);
   cudaFree(p->ent_col);
   cudaFree(p->row_ptr);
   cudaFree(p->bucket_ptr);
@@ -401,6 +418,13 @@ szo_status szo_linear_create(szo_linear_t** out, int64_t N, int64_t K, int32_t G
     else
       widen_sz_kernel<__half><<<static_cast<unsigned>(ceil_div(ng, 256)), 256, 0, st>>>(
           static_cast<const __half*>(scales), static_cast<const __half*>(zeros), N, K / G, p->Npad, p->sz);
+  }
+  if (G > 0) {
+    const int64_t n_code_tiles = p->Npad / 128;      // padded to an even count for the pair-tile kernel
+    const int64_t units = n_code_tiles * (K / 64) * 256;
+    SZO_PLAN_CUDA(cudaMalloc(&p->codes_tiled, units * 16));
+    tile_codes_kernel<<<static_cast<unsigned>(ceil_div(units, 256)), 256, 0, st>>>(
+        static_cast<const uint8_t*>(codes_or_bf16_W), N, K, n_code_tiles, p->codes_tiled);
   }
   SZO_PLAN_CUDA(cudaMalloc(&p->row_ptr, (N + 1) * sizeof(int32_t)));
   SZO_PLAN_CUDA(cudaMalloc(&p->bucket_ptr, (nb + 1) * sizeof(int32_t)));

@@ -28,7 +28,7 @@ struct TcParams {
   int G;
   int nkb;                 // K / 64
   int64_t m_tiles, n_tiles;
-  const uint8_t* codes;    // [N, K/2]
+  const uint8_t* codes;    // tile order: block (128-row tile t, k-block kb) = 4 KiB at (t * nkb + kb) * 4096
   const float2* sz;        // [K/G][Npad]; fp32 (scale, zero), or packed bf16 pairs when kFast
   int64_t Npad;
   const int32_t* bucket_ptr;
