@@ -161,11 +161,11 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
           const int64_t it = lt * P.nkb + kb;
           const int s = static_cast<int>(it % kXS), t = static_cast<int>(it % kAS);
           const uint32_t ph = static_cast<uint32_t>((it / kXS) & 1), pht = static_cast<uint32_t>((it / kAS) & 1);
-          if (!mbar_wait(xfull_bar(s), ph, abort_flag, P.status)) { ok = false; break; }
+          if (!mbar_wait(xfull_bar(s), ph, abort_flag, P.status, 0)) { ok = false; break; }
           if (sparse) {
-            if (!mbar_wait(aready_bar(t), pht, abort_flag, P.status)) { ok = false; break; }
+            if (!mbar_wait(aready_bar(t), pht, abort_flag, P.status, 0)) { ok = false; break; }
           } else if (kDequant) {
-            if (!mbar_wait(adone_bar(t), pht, abort_flag, P.status)) { ok = false; break; }
+            if (!mbar_wait(adone_bar(t), pht, abort_flag, P.status, 0)) { ok = false; break; }
           }
           tc_fence_after();
           const uint64_t adesc = make_desc_sw128(tiles_base + a_off(s, t)), bdesc = make_desc_sw128(tiles_base + b_off(s));
@@ -280,7 +280,7 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
       const int64_t n_tile = tile / P.m_tiles, m_tile = tile % P.m_tiles;
       const int as = static_cast<int>(lt & 1);
       const uint32_t aph = static_cast<uint32_t>((lt >> 1) & 1);
-      if (!mbar_wait(accfull_bar(as), aph, abort_flag, P.status)) break;
+      if (!mbar_wait(accfull_bar(as), aph, abort_flag, P.status, 256)) break;
       tc_fence_after();
       const int64_t n = n_tile * kBM + qd * 32 + lane;
       const float bias = (P.bias != nullptr && n < P.N) ? P.bias[n] : 0.f;

@@ -70,21 +70,25 @@ __device__ __forceinline__ unsigned long long global_ns() {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait: false when the limit expired or another role already gave up.  The common case
-// (the phase completes within a few polls) touches no timer; after that the SM cycle counter
-// bounds the wait (kWaitLimitCycles is about two seconds at 2 GHz).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-  for (int i = 0; i < 256; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
+// Bounded wait: false when the limit expired or another role already gave up.  Between polls the
+// warp sleeps for `backoff_ns` so that waiting roles do not take issue slots from the few threads
+// that feed the tensor core; the SM cycle counter bounds the wait (kWaitLimitCycles is about two
+// seconds at 2 GHz).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                          unsigned backoff_ns = 32) {
+  if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
+  int polls = 0;
   while (true) {
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitCycles) {
-      *abort_flag = 1;
-      atomicExch(status, static_cast<int32_t>(SZO_ERR_TIMEOUT));
-      return false;
+    if (backoff_ns) __nanosleep(backoff_ns);
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((++polls & 1023) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitLimitCycles) {
+        *abort_flag = 1;
+        atomicExch(status, static_cast<int32_t>(SZO_ERR_TIMEOUT));
+        return false;
+      }
     }
   }
 }
