@@ -127,7 +127,7 @@ szo_status szo_update(float* S, const int64_t* idx, int64_t k, int64_t idx_base,
  * A plan owns only derived, immutable data (kernel-layout scale/zero table, tile buckets and
  * row pointers of idx, tensor maps); the caller's codes, scales, zeros, idx and bias must
  * outlive it.  G == 0 means a dense bf16 weight [N,K] instead of codes (scales/zeros NULL).
- * Requires K % 64 == 0 and, for G > 0, G % 32 == 0.  idx[nnz] ascending flat indices n*K + c.
+ * Requires K % 64 == 0 and, for G > 0, G == 32 or G % 64 == 0.  idx[nnz] ascending flat indices n*K + c.
  * bias fp32 [N] or NULL.  szo_linear_create synchronises the stream. */
 typedef struct szo_linear szo_linear_t;
 szo_status szo_linear_create(szo_linear_t** out, int64_t N, int64_t K, int32_t G,

@@ -107,24 +107,28 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
 
-  const int64_t total_tiles = P.m_tiles * P.n_tiles;
-  const int64_t my_tiles = (total_tiles > blockIdx.x) ? (total_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
-  const int64_t my_iters = my_tiles * P.nkb;
-  auto tile_of = [&](int64_t it) { return blockIdx.x + (it / P.nkb) * gridDim.x; };
+  // tiles of this CTA: tile(lt) = blockIdx.x + lt * gridDim.x, tile = n_tile * m_tiles + m_tile
+  const int total_tiles = static_cast<int>(P.m_tiles * P.n_tiles), m_tiles = static_cast<int>(P.m_tiles);
+  const int my_tiles = (total_tiles > static_cast<int>(blockIdx.x))
+                           ? (total_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x)
+                           : 0;
+  const int nkb = P.nkb;
 
   if (warp == 0) {
     // ---------------------------------------------------------------- X producer (token tiles)
     if (lane == 0) {
-      for (int64_t it = 0; it < my_iters; ++it) {
-        const int64_t tile = tile_of(it);
-        const int kb = static_cast<int>(it % P.nkb);
-        const int s = static_cast<int>(it % kXS);
-        const uint32_t ph = static_cast<uint32_t>((it / kXS) & 1);
-        if (!mbar_wait(xempty_bar(s), ph ^ 1u, abort_flag, P.status)) break;
-        mbar_expect_tx(xfull_bar(s), kXStageBytes);
-        tma_load_2d(tiles_base + b_off(s), &tmap_x, kb * kBK, static_cast<int>((tile % P.m_tiles) * BT), xfull_bar(s));
-        if constexpr (!kDequant)
-          tma_load_2d(tiles_base + a_off(s, 0), &tmap_w, kb * kBK, static_cast<int>((tile / P.m_tiles) * kBM), xfull_bar(s));
+      RingPos x{0, 0};
+      bool ok = true;
+      for (int lt = 0; lt < my_tiles && ok; ++lt) {
+        const int tile = blockIdx.x + lt * gridDim.x;
+        const int m0 = (tile % m_tiles) * BT, n0 = (tile / m_tiles) * kBM;
+        for (int kb = 0; kb < nkb; ++kb) {
+          if (!mbar_wait(xempty_bar(x.idx), x.phase ^ 1u, abort_flag, P.status)) { ok = false; break; }
+          mbar_expect_tx(xfull_bar(x.idx), kXStageBytes);
+          tma_load_2d(tiles_base + b_off(x.idx), &tmap_x, kb * kBK, m0, xfull_bar(x.idx));
+          if constexpr (!kDequant) tma_load_2d(tiles_base + a_off(x.idx, 0), &tmap_w, kb * kBK, n0, xfull_bar(x.idx));
+          x.advance(kXS);
+        }
       }
     }
   } else if (warp == 3) {
@@ -132,50 +136,56 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
     if constexpr (kDequant) {
       if (lane == 0) {
         const int groups_kb = (P.G < kBK) ? kBK / P.G : 1;     // scale groups per k-block
-        for (int64_t it = 0; it < my_iters; ++it) {
-          const int kb = static_cast<int>(it % P.nkb);
-          const int64_t n0 = (tile_of(it) / P.m_tiles) * kBM;
-          const int c = static_cast<int>(it % kCS);
-          const uint32_t ph = static_cast<uint32_t>((it / kCS) & 1);
-          if (!mbar_wait(cempty_bar(c), ph ^ 1u, abort_flag, P.status)) break;
-          mbar_expect_tx(cfull_bar(c), kCodesBytes + groups_kb * 1024);
-          bulk_load_1d(tiles_base + c_off(c), P.codes + ((n0 / kBM) * P.nkb + kb) * static_cast<int64_t>(kCodesBytes),
-                       kCodesBytes, cfull_bar(c));
-          const int64_t g0 = (static_cast<int64_t>(kb) * kBK) / P.G;
-          for (int g = 0; g < groups_kb; ++g)
-            bulk_load_1d(tiles_base + c_off(c) + kCodesBytes + g * 1024, P.sz + (g0 + g) * P.Npad + n0, 1024, cfull_bar(c));
+        RingPos c{0, 0};
+        bool ok = true;
+        for (int lt = 0; lt < my_tiles && ok; ++lt) {
+          const int n_tile = (blockIdx.x + lt * gridDim.x) / m_tiles;
+          const uint8_t* codes = P.codes + static_cast<int64_t>(n_tile) * nkb * kCodesBytes;
+          const float2* sz = P.sz + static_cast<int64_t>(n_tile) * kBM;
+          for (int kb = 0; kb < nkb; ++kb) {
+            if (!mbar_wait(cempty_bar(c.idx), c.phase ^ 1u, abort_flag, P.status)) { ok = false; break; }
+            mbar_expect_tx(cfull_bar(c.idx), kCodesBytes + groups_kb * 1024);
+            bulk_load_1d(tiles_base + c_off(c.idx), codes + static_cast<int64_t>(kb) * kCodesBytes, kCodesBytes,
+                         cfull_bar(c.idx));
+            const int g0 = (kb * kBK) / P.G;
+            for (int g = 0; g < groups_kb; ++g)
+              bulk_load_1d(tiles_base + c_off(c.idx) + kCodesBytes + g * 1024, sz + static_cast<int64_t>(g0 + g) * P.Npad,
+                           1024, cfull_bar(c.idx));
+            c.advance(kCS);
+          }
         }
       }
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
+      RingPos x{0, 0}, a{0, 0};
       bool ok = true;
-      for (int64_t lt = 0; lt < my_tiles && ok; ++lt) {
-        const int as = static_cast<int>(lt & 1);
+      for (int lt = 0; lt < my_tiles && ok; ++lt) {
+        const int as = lt & 1;
         const uint32_t aph = static_cast<uint32_t>((lt >> 1) & 1);
-        if (!mbar_wait(accempty_bar(as), aph ^ 1u, abort_flag, P.status)) break;
+        if (!mbar_wait(accempty_bar(as), aph ^ 1u, abort_flag, P.status, 0)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kAccStride);
-        for (int kb = 0; kb < P.nkb; ++kb) {
-          const int64_t it = lt * P.nkb + kb;
-          const int s = static_cast<int>(it % kXS), t = static_cast<int>(it % kAS);
-          const uint32_t ph = static_cast<uint32_t>((it / kXS) & 1), pht = static_cast<uint32_t>((it / kAS) & 1);
-          if (!mbar_wait(xfull_bar(s), ph, abort_flag, P.status, 0)) { ok = false; break; }
+        for (int kb = 0; kb < nkb; ++kb) {
+          if (!mbar_wait(xfull_bar(x.idx), x.phase, abort_flag, P.status, 0)) { ok = false; break; }
           if (sparse) {
-            if (!mbar_wait(aready_bar(t), pht, abort_flag, P.status, 0)) { ok = false; break; }
+            if (!mbar_wait(aready_bar(a.idx), a.phase, abort_flag, P.status, 0)) { ok = false; break; }
           } else if (kDequant) {
-            if (!mbar_wait(adone_bar(t), pht, abort_flag, P.status, 0)) { ok = false; break; }
+            if (!mbar_wait(adone_bar(a.idx), a.phase, abort_flag, P.status, 0)) { ok = false; break; }
           }
           tc_fence_after();
-          const uint64_t adesc = make_desc_sw128(tiles_base + a_off(s, t)), bdesc = make_desc_sw128(tiles_base + b_off(s));
+          const uint64_t adesc = make_desc_sw128(tiles_base + a_off(x.idx, a.idx));
+          const uint64_t bdesc = make_desc_sw128(tiles_base + b_off(x.idx));
 #pragma unroll
           for (int k = 0; k < kBK / kUmmaK; ++k) {
             // advance both descriptors by 16 elements = 32 bytes (>> 4 = 2) inside the swizzle row
             umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc, (kb | k) ? 1u : 0u);
           }
-          umma_commit(xempty_bar(s));
-          if constexpr (kDequant) umma_commit(aempty_bar(t));
+          umma_commit(xempty_bar(x.idx));
+          if constexpr (kDequant) umma_commit(aempty_bar(a.idx));
+          x.advance(kXS);
+          a.advance(kAS);
         }
         if (ok) umma_commit(accfull_bar(as));
       }
@@ -183,52 +193,75 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
   } else if (warp == 2) {
     // ---------------------------------------------------------------- SparseAdd warp
     // Adds the sparse values of bucket (tile, k-block) to the bf16 weight tile in shared memory.
-    // Bucket bounds and records are brought in with cp.async kLook / 2*kLook iterations ahead.
-    if (sparse && my_iters > 0) {
-      auto bucket_of = [&](int64_t it) { return (tile_of(it) / P.m_tiles) * P.n_kblocks + (it % P.nkb); };
-      auto issue_bounds = [&](int64_t it) {           // lanes 0,1 copy bucket_ptr[b], bucket_ptr[b+1]
-        if (it < my_iters && lane < 2)
-          cp_async_4(smem_u32(&bound_ring[it % kBoundSlots][lane]), P.bucket_ptr + bucket_of(it) + lane);
+    // Bucket bounds and records are brought in with cp.async kLook / 2*kLook iterations ahead; each of
+    // the three streams (bounds, records, apply) walks the (tile, k-block) sequence with its own cursor.
+    if (sparse && my_tiles > 0) {
+      struct Cursor {
+        int lt, kb, bucket0;     // bucket0 = n_tile * n_kblocks for the cursor's tile
       };
-      auto issue_records = [&](int64_t it) {          // needs bounds(it) in shared memory
-        if (it < my_iters) {
-          const int32_t e0 = bound_ring[it % kBoundSlots][0], e1 = bound_ring[it % kBoundSlots][1];
-          const int32_t n = (e1 - e0 < kRecCap) ? e1 - e0 : kRecCap;
-          for (int32_t j = lane; j < n; j += 32) cp_async_8(smem_u32(&rec_ring[it % kRecSlots][j]), P.Sb + e0 + j);
+      const int n_kblocks = static_cast<int>(P.n_kblocks);
+      auto start = [&]() {
+        return Cursor{0, 0, static_cast<int>((blockIdx.x / m_tiles)) * n_kblocks};
+      };
+      auto step = [&](Cursor& c) {
+        if (++c.kb == nkb) {
+          c.kb = 0;
+          ++c.lt;
+          c.bucket0 = ((blockIdx.x + c.lt * gridDim.x) / m_tiles) * n_kblocks;
         }
       };
-      // prologue: bounds of 0..2*kLook-1, then records of 0..kLook-1
-      for (int64_t j = 0; j < 2 * kLook; ++j) issue_bounds(j);
+      Cursor cb = start(), cr = start();            // bounds stream, records stream
+      int ib = 0, ir = 0;                           // their iteration numbers (ring slots)
+      auto issue_bounds = [&]() {                   // lanes 0,1 copy bucket_ptr[b], bucket_ptr[b+1]
+        if (cb.lt < my_tiles) {
+          if (lane < 2) cp_async_4(smem_u32(&bound_ring[ib & (kBoundSlots - 1)][lane]), P.bucket_ptr + cb.bucket0 + cb.kb + lane);
+          step(cb);
+          ++ib;
+        }
+      };
+      auto issue_records = [&]() {                  // needs the bounds of that iteration in shared memory
+        if (cr.lt < my_tiles) {
+          const int32_t e0 = bound_ring[ir & (kBoundSlots - 1)][0], e1 = bound_ring[ir & (kBoundSlots - 1)][1];
+          const int32_t n = (e1 - e0 < kRecCap) ? e1 - e0 : kRecCap;
+          for (int32_t j = lane; j < n; j += 32) cp_async_8(smem_u32(&rec_ring[ir & (kRecSlots - 1)][j]), P.Sb + e0 + j);
+          step(cr);
+          ++ir;
+        }
+      };
+      // prologue: bounds of iterations 0..2*kLook-1, then records of 0..kLook-1
+      for (int j = 0; j < 2 * kLook; ++j) issue_bounds();
       cp_async_commit();
       cp_async_wait_all();
       __syncwarp();
-      for (int64_t j = 0; j < kLook; ++j) {
-        issue_records(j);
+      for (int j = 0; j < kLook; ++j) {
+        issue_records();
         cp_async_commit();
       }
-      for (int64_t it = 0; it < my_iters; ++it) {
-        const int s = static_cast<int>(it % kXS), t = static_cast<int>(it % kAS);
-        const uint32_t ph = static_cast<uint32_t>((it / kXS) & 1), pht = static_cast<uint32_t>((it / kAS) & 1);
+      RingPos x{0, 0}, a{0, 0};
+      const int my_iters = my_tiles * nkb;
+      for (int it = 0; it < my_iters; ++it) {
         // group(j) = { bounds(j + 2 kLook), records(j + kLook) }, committed in iteration j.  Groups
         // retire in order: with at most kLook - 1 still pending, group(it - kLook) has landed, i.e.
         // records(it) and bounds(it + kLook), which the next record copies are addressed from.
         cp_async_wait_group<kLook - 1>();
         __syncwarp();
-        issue_bounds(it + 2 * kLook);
-        issue_records(it + kLook);
+        issue_bounds();
+        issue_records();
         cp_async_commit();
-        const int32_t e0 = bound_ring[it % kBoundSlots][0], e1 = bound_ring[it % kBoundSlots][1];
-        if (!mbar_wait(kDequant ? adone_bar(t) : xfull_bar(s), kDequant ? pht : ph, abort_flag, P.status)) break;
-        unsigned char* A = tiles_ptr + a_off(s, t);
+        const int32_t e0 = bound_ring[it & (kBoundSlots - 1)][0], e1 = bound_ring[it & (kBoundSlots - 1)][1];
+        if (!mbar_wait(kDequant ? adone_bar(a.idx) : xfull_bar(x.idx), kDequant ? a.phase : x.phase, abort_flag, P.status, 0)) break;
+        unsigned char* A = tiles_ptr + a_off(x.idx, a.idx);
         for (int32_t j = lane; j < e1 - e0; j += 32) {
-          const uint2 rec = (j < kRecCap) ? rec_ring[it % kRecSlots][j] : __ldg(P.Sb + e0 + j);
+          const uint2 rec = (j < kRecCap) ? rec_ring[it & (kRecSlots - 1)][j] : __ldg(P.Sb + e0 + j);
           const int r = static_cast<int>(rec.x >> 6), c = static_cast<int>(rec.x & 63);
           __nv_bfloat16* el = reinterpret_cast<__nv_bfloat16*>(A + r * 128 + (((c >> 3) ^ (r & 7)) << 4) + (c & 7) * 2);
           *el = __float2bfloat16_rn(__bfloat162float(*el) + __uint_as_float(rec.y));
         }
         fence_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(aready_bar(t));
+        if (lane == 0) mbar_arrive(aready_bar(a.idx));
+        x.advance(kXS);
+        a.advance(kAS);
       }
       cp_async_wait_all();
     }
@@ -242,13 +275,17 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
       constexpr int kRowsPerWarp = kBM / kWarpsPerGroup, kPasses = kRowsPerWarp / 4;
       const int sub = lane >> 3, chunk = lane & 7;
       const int gsel = (P.G < kBK) ? (chunk * 8) / P.G : 0;
-      for (int64_t it = gq; it < my_iters; it += kGroups) {
-        const int c = static_cast<int>(it % kCS), t = static_cast<int>(it % kAS);
-        const uint32_t phc = static_cast<uint32_t>((it / kCS) & 1), pht = static_cast<uint32_t>((it / kAS) & 1);
-        unsigned char* A = tiles_ptr + a_off(0, t);
-        const unsigned char* C = tiles_ptr + c_off(c);
+      RingPos c{0, 0}, a{0, 0};
+      for (int j = 0; j < gq; ++j) {
+        c.advance(kCS);
+        a.advance(kAS);
+      }
+      const int my_iters = my_tiles * nkb;
+      for (int it = gq; it < my_iters; it += kGroups) {
+        unsigned char* A = tiles_ptr + a_off(0, a.idx);
+        const unsigned char* C = tiles_ptr + c_off(c.idx);
         const float2* SZ = reinterpret_cast<const float2*>(C + kCodesBytes) + gsel * kBM;
-        if (!mbar_wait(cfull_bar(c), phc, abort_flag, P.status)) break;
+        if (!mbar_wait(cfull_bar(c.idx), c.phase, abort_flag, P.status)) break;
         uint32_t w[kPasses];
         float2 zs[kPasses];
 #pragma unroll
@@ -257,7 +294,7 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
           w[i] = *reinterpret_cast<const uint32_t*>(C + r * 32 + chunk * 4);
           zs[i] = SZ[r];
         }
-        if (!mbar_wait(aempty_bar(t), pht ^ 1u, abort_flag, P.status)) break;
+        if (!mbar_wait(aempty_bar(a.idx), a.phase ^ 1u, abort_flag, P.status)) break;
 #pragma unroll
         for (int i = 0; i < kPasses; ++i) {
           const int r = wq * kRowsPerWarp + i * 4 + sub;
@@ -267,18 +304,23 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
         fence_async_smem();
         __syncwarp();
         if (lane == 0) {
-          mbar_arrive(adone_bar(t));
-          mbar_arrive(cempty_bar(c));
+          mbar_arrive(adone_bar(a.idx));
+          mbar_arrive(cempty_bar(c.idx));
+        }
+#pragma unroll
+        for (int j = 0; j < kGroups; ++j) {
+          c.advance(kCS);
+          a.advance(kAS);
         }
       }
     }
   } else if (warp >= kEpiWarp0) {
     // ---------------------------------------------------------------- epilogue
     const int qd = warp & 3;                        // TMEM lane quarter this warp may read
-    for (int64_t lt = 0; lt < my_tiles; ++lt) {
-      const int64_t tile = blockIdx.x + lt * gridDim.x;
-      const int64_t n_tile = tile / P.m_tiles, m_tile = tile % P.m_tiles;
-      const int as = static_cast<int>(lt & 1);
+    for (int lt = 0; lt < my_tiles; ++lt) {
+      const int tile = blockIdx.x + lt * gridDim.x;
+      const int64_t n_tile = tile / m_tiles, m_tile = tile % m_tiles;
+      const int as = lt & 1;
       const uint32_t aph = static_cast<uint32_t>((lt >> 1) & 1);
       if (!mbar_wait(accfull_bar(as), aph, abort_flag, P.status, 256)) break;
       tc_fence_after();

@@ -372,8 +372,8 @@ szo_status szo_linear_create(szo_linear_t** out, int64_t N, int64_t K, int32_t G
   *out = nullptr;
   SZO_REQUIRE(N > 0 && K > 0, SZO_ERR_SHAPE, "N and K must be positive");
   SZO_REQUIRE(K % 64 == 0, SZO_ERR_SHAPE, "K (%lld) must be a multiple of 64", (long long)K);
-  SZO_REQUIRE(G >= 0 && (G == 0 || (G % 32 == 0 && K % G == 0)), SZO_ERR_SHAPE,
-              "G (%d) must be 0 or a multiple of 32 dividing K", G);
+  SZO_REQUIRE(G >= 0 && (G == 0 || ((G == 32 || G % 64 == 0) && K % G == 0)), SZO_ERR_SHAPE,
+              "G (%d) must be 0, 32 or a multiple of 64, and divide K", G);
   SZO_REQUIRE(N * K < (int64_t(1) << 40), SZO_ERR_SHAPE, "tensor too large");
   SZO_REQUIRE(nnz >= 0 && nnz <= N * K && nnz < (int64_t(1) << 31), SZO_ERR_INVALID_ARG, "bad nnz");
   SZO_REQUIRE(codes_or_bf16_W != nullptr, SZO_ERR_INVALID_ARG, "weight pointer is NULL");

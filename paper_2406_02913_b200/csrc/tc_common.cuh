@@ -41,6 +41,21 @@ struct TcParams {
   int32_t* status;
 };
 
+// Position in a ring of n slots: slot index and the parity of the current pass over the ring.
+// Every role keeps running cursors instead of deriving them from the iteration number: the
+// producer and MMA roles are single threads, where an integer division per k-block would be a
+// large part of the loop.
+struct RingPos {
+  int idx;
+  uint32_t phase;
+  __device__ __forceinline__ void advance(int n) {
+    if (++idx == n) {
+      idx = 0;
+      phase ^= 1u;
+    }
+  }
+};
+
 // ------------------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
