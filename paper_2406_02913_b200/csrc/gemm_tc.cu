@@ -28,6 +28,9 @@ namespace {
 
 using namespace tc;
 
+constexpr int kCStages = 4;   // code-tile stages (cover the TMA latency)
+constexpr int kASlots = 4;    // dequantised weight slots (cover conversion + SparseAdd)
+
 // ------------------------------------------------------------------------------ the kernel
 // Three rings in shared memory, each with its own life time:
 //   X ring  token tile [BT x 64] bf16 (+ the bf16 weight tile in dense mode): TMA -> MMA
@@ -44,8 +47,8 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
   constexpr int kBTileBytes = BT * kBK * 2;
   constexpr int kXStageBytes = kBTileBytes + (kDequant ? 0 : kATileBytes);
   constexpr int kCStageBytes = kCodesBytes + kSzBytes;
-  constexpr int kCS = kDequant ? 6 : 1;                      // C ring stages
-  constexpr int kAS = kDequant ? 3 : kXS;                    // A ring slots (dense: the X stage itself)
+  constexpr int kCS = kDequant ? kCStages : 1;               // C ring stages
+  constexpr int kAS = kDequant ? kASlots : kXS;                    // A ring slots (dense: the X stage itself)
   constexpr int kGroups = 2, kWarpsPerGroup = kNumDeqWarps / kGroups;
   constexpr int kAccStride = BT < 32 ? 32 : BT;             // TMEM columns per accumulator buffer
   constexpr uint32_t kTmemCols = static_cast<uint32_t>(2 * kAccStride);
@@ -53,7 +56,7 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
   constexpr uint32_t kXBase = 0, kCBase = kXS * kXStageBytes, kABase = kCBase + (kDequant ? kCS * kCStageBytes : 0);
 
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[2 * kXS + 2 * kCS + 3 * kAS + 4];
+  __shared__ __align__(8) unsigned long long bars[2 * kXS + 2 * kCS + 3 * kAS + 4 + kRecSlots];
   __shared__ __align__(16) uint2 rec_ring[kRecSlots][kRecCap];      // sparse records, per k-block
   __shared__ __align__(8) int32_t bound_ring[kBoundSlots][2];
   __shared__ uint32_t tmem_base_slot;
@@ -73,6 +76,7 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
   auto aempty_bar = [&](int t) { return smem_u32(&bars[2 * kXS + 2 * kCS + 2 * kAS + t]); }; // its MMAs retired
   auto accfull_bar = [&](int a) { return smem_u32(&bars[2 * kXS + 2 * kCS + 3 * kAS + a]); };
   auto accempty_bar = [&](int a) { return smem_u32(&bars[2 * kXS + 2 * kCS + 3 * kAS + 2 + a]); };
+  auto recready_bar = [&](int r) { return smem_u32(&bars[2 * kXS + 2 * kCS + 3 * kAS + 4 + r]); };  // records of a k-block landed
   auto b_off = [&](int s) { return kXBase + static_cast<uint32_t>(s) * kXStageBytes; };
   auto c_off = [&](int c) { return kCBase + static_cast<uint32_t>(c) * kCStageBytes; };
   auto a_off = [&](int s, int t) {     // weight tile of iteration (X stage s, A slot t)
@@ -99,6 +103,7 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
       mbar_init(accfull_bar(a), 1);
       mbar_init(accempty_bar(a), 4);
     }
+    for (int r = 0; r < kRecSlots; ++r) mbar_init(recready_bar(r), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), kTmemCols);
@@ -169,10 +174,10 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kAccStride);
         for (int kb = 0; kb < nkb; ++kb) {
           if (!mbar_wait(xfull_bar(x.idx), x.phase, abort_flag, P.status, 0)) { ok = false; break; }
-          if (sparse) {
-            if (!mbar_wait(aready_bar(a.idx), a.phase, abort_flag, P.status, 0)) { ok = false; break; }
-          } else if (kDequant) {
+          if constexpr (kDequant) {     // converted (and, with sparse entries, already SparseAdd-ed) by the conversion warps
             if (!mbar_wait(adone_bar(a.idx), a.phase, abort_flag, P.status, 0)) { ok = false; break; }
+          } else if (sparse) {          // dense weight tile: SparseAdd-ed by warp 2
+            if (!mbar_wait(aready_bar(a.idx), a.phase, abort_flag, P.status, 0)) { ok = false; break; }
           }
           tc_fence_after();
           const uint64_t adesc = make_desc_sw128(tiles_base + a_off(x.idx, a.idx));
@@ -245,23 +250,36 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
         // records(it) and bounds(it + kLook), which the next record copies are addressed from.
         cp_async_wait_group<kLook - 1>();
         __syncwarp();
-        issue_bounds();
-        issue_records();
-        cp_async_commit();
-        const int32_t e0 = bound_ring[it & (kBoundSlots - 1)][0], e1 = bound_ring[it & (kBoundSlots - 1)][1];
-        if (!mbar_wait(kDequant ? adone_bar(a.idx) : xfull_bar(x.idx), kDequant ? a.phase : x.phase, abort_flag, P.status, 0)) break;
-        unsigned char* A = tiles_ptr + a_off(x.idx, a.idx);
-        for (int32_t j = lane; j < e1 - e0; j += 32) {
-          const uint2 rec = (j < kRecCap) ? rec_ring[it & (kRecSlots - 1)][j] : __ldg(P.Sb + e0 + j);
-          const int r = static_cast<int>(rec.x >> 6), c = static_cast<int>(rec.x & 63);
-          __nv_bfloat16* el = reinterpret_cast<__nv_bfloat16*>(A + r * 128 + (((c >> 3) ^ (r & 7)) << 4) + (c & 7) * 2);
-          *el = __float2bfloat16_rn(__bfloat162float(*el) + __uint_as_float(rec.y));
+        if constexpr (kDequant) {
+          // The conversion warps apply the records themselves.  Tell them records(it) are in shared
+          // memory, then keep at most kRecSlots - kLook iterations ahead of them so that a ring slot
+          // is not refilled while its previous k-block is still being converted.
+          if (lane == 0) mbar_arrive(recready_bar(it & (kRecSlots - 1)));
+          if (it >= kRecSlots - kLook) {
+            if (!mbar_wait(adone_bar(a.idx), a.phase, abort_flag, P.status)) break;
+            a.advance(kAS);
+          }
+          issue_bounds();
+          issue_records();
+          cp_async_commit();
+        } else {
+          issue_bounds();
+          issue_records();
+          cp_async_commit();
+          const int32_t e0 = bound_ring[it & (kBoundSlots - 1)][0], e1 = bound_ring[it & (kBoundSlots - 1)][1];
+          if (!mbar_wait(xfull_bar(x.idx), x.phase, abort_flag, P.status, 0)) break;
+          unsigned char* A = tiles_ptr + a_off(x.idx, x.idx);
+          for (int32_t j = lane; j < e1 - e0; j += 32) {
+            const uint2 rec = (j < kRecCap) ? rec_ring[it & (kRecSlots - 1)][j] : __ldg(P.Sb + e0 + j);
+            const int r = static_cast<int>(rec.x >> 6), c = static_cast<int>(rec.x & 63);
+            __nv_bfloat16* el = reinterpret_cast<__nv_bfloat16*>(A + r * 128 + (((c >> 3) ^ (r & 7)) << 4) + (c & 7) * 2);
+            *el = __float2bfloat16_rn(__bfloat162float(*el) + __uint_as_float(rec.y));
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(aready_bar(x.idx));
+          x.advance(kXS);
         }
-        fence_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(aready_bar(a.idx));
-        x.advance(kXS);
-        a.advance(kAS);
       }
       cp_async_wait_all();
     }
@@ -300,6 +318,20 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
           const int r = wq * kRowsPerWarp + i * 4 + sub;
           const uint4 v = dequant_word<kFast>(w[i], zs[i]);
           *reinterpret_cast<uint4*>(A + r * 128 + ((chunk ^ (r & 7)) << 4)) = v;
+        }
+        if (sparse) {
+          // SparseAdd: add the bucket's fp32 values to this warp's rows of the bf16 tile
+          if (!mbar_wait(recready_bar(it & (kRecSlots - 1)), static_cast<uint32_t>((it / kRecSlots) & 1), abort_flag, P.status)) break;
+          __syncwarp();
+          const int32_t e0 = bound_ring[it & (kBoundSlots - 1)][0], e1 = bound_ring[it & (kBoundSlots - 1)][1];
+          for (int32_t j = lane; j < e1 - e0; j += 32) {
+            const uint2 rec = (j < kRecCap) ? rec_ring[it & (kRecSlots - 1)][j] : __ldg(P.Sb + e0 + j);
+            const int r = static_cast<int>(rec.x >> 6), col = static_cast<int>(rec.x & 63);
+            if (r / kRowsPerWarp == wq) {
+              __nv_bfloat16* el = reinterpret_cast<__nv_bfloat16*>(A + r * 128 + (((col >> 3) ^ (r & 7)) << 4) + (col & 7) * 2);
+              *el = __float2bfloat16_rn(__bfloat162float(*el) + __uint_as_float(rec.y));
+            }
+          }
         }
         fence_async_smem();
         __syncwarp();
@@ -422,7 +454,7 @@ szo_status make_codes_map(CUtensorMap* map, const void* base, int64_t rows, int6
 template <int BT, int kXS, bool kDequant, bool kFast>
 szo_status launch_tc(const CUtensorMap& mx, const CUtensorMap& mw, const TcParams& P, int sms, cudaStream_t st) {
   constexpr size_t smem = static_cast<size_t>(kXS) * (BT * kBK * 2 + (kDequant ? 0 : kATileBytes)) +
-                          (kDequant ? 6 * (kCodesBytes + kSzBytes) + 3 * kATileBytes : 0) + 1024;
+                          (kDequant ? kCStages * (kCodesBytes + kSzBytes) + kASlots * kATileBytes : 0) + 1024;
   auto kern = szo_linear_tc_kernel<BT, kXS, kDequant, kFast>;
   static bool configured = false;
   if (!configured) {
