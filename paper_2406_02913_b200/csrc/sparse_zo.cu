@@ -13,19 +13,26 @@ constexpr uint32_t kPhiloxM1 = 0xCD9E8D57u;
 constexpr uint32_t kPhiloxW0 = 0x9E3779B9u;
 constexpr uint32_t kPhiloxW1 = 0xBB67AE85u;
 
+// The ten round keys (key + r * Weyl constant) are the same for every entry of a pass: the host
+// computes them once and passes them by value, so that each round is two wide multiplies and two
+// three-input XORs.
+struct PhiloxKeys {
+  uint32_t k0[10], k1[10];
+};
+
 // Ten Philox rounds; only output words 0 and 1 are consumed by the Gaussian draw.
 __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                              uint32_t k0, uint32_t k1, uint32_t& r0, uint32_t& r1) {
+                                              const PhiloxKeys& K, uint32_t& r0, uint32_t& r1) {
 #pragma unroll
   for (int r = 0; r < 10; ++r) {
-    const uint32_t hi0 = __umulhi(kPhiloxM0, c0), lo0 = kPhiloxM0 * c0;
-    const uint32_t hi1 = __umulhi(kPhiloxM1, c2), lo1 = kPhiloxM1 * c2;
-    c0 = hi1 ^ c1 ^ k0;
-    c1 = lo1;
-    c2 = hi0 ^ c3 ^ k1;
-    c3 = lo0;
-    k0 += kPhiloxW0;
-    k1 += kPhiloxW1;
+    const unsigned long long p0 = static_cast<unsigned long long>(kPhiloxM0) * c0;   // (hi0, lo0)
+    const unsigned long long p1 = static_cast<unsigned long long>(kPhiloxM1) * c2;   // (hi1, lo1)
+    const uint32_t n0 = static_cast<uint32_t>(p1 >> 32) ^ c1 ^ K.k0[r];
+    const uint32_t n2 = static_cast<uint32_t>(p0 >> 32) ^ c3 ^ K.k1[r];
+    c1 = static_cast<uint32_t>(p1);
+    c3 = static_cast<uint32_t>(p0);
+    c0 = n0;
+    c2 = n2;
   }
   r0 = c0;
   r1 = c1;
@@ -39,11 +46,9 @@ __device__ __forceinline__ float gaussian_from_words(uint32_t r0, uint32_t r1) {
   return rad * cospif(two_u2);
 }
 
-__device__ __forceinline__ float z_of(uint64_t gidx, uint32_t step_lo, uint32_t step_hi,
-                                      uint32_t seed_lo, uint32_t seed_hi) {
+__device__ __forceinline__ float z_of(uint64_t gidx, uint32_t step_lo, uint32_t step_hi, const PhiloxKeys& K) {
   uint32_t r0, r1;
-  philox4x32_10(static_cast<uint32_t>(gidx), static_cast<uint32_t>(gidx >> 32), step_lo, step_hi,
-                seed_lo, seed_hi, r0, r1);
+  philox4x32_10(static_cast<uint32_t>(gidx), static_cast<uint32_t>(gidx >> 32), step_lo, step_hi, K, r0, r1);
   return gaussian_from_words(r0, r1);
 }
 
@@ -53,27 +58,34 @@ __device__ __forceinline__ float resolve_scale(const ScaleArg& a) {
   return -static_cast<float>(static_cast<double>(a.lr) * g);
 }
 
-// Two entries per thread: one 16-byte index load, one 8-byte value load and store.
+// Four entries per thread and iteration: two 16-byte index loads, one 16-byte value load and store,
+// four independent Philox/Box-Muller chains in flight.
 __global__ void __launch_bounds__(256)
 sparse_axpy_kernel(const float* __restrict__ S_in, float* __restrict__ S_out,
-                   const int64_t* __restrict__ idx, int64_t k, int64_t idx_base, uint32_t seed_lo,
-                   uint32_t seed_hi, uint32_t step_lo, uint32_t step_hi, ScaleArg sa) {
+                   const int64_t* __restrict__ idx, int64_t k, int64_t idx_base, const PhiloxKeys K,
+                   uint32_t step_lo, uint32_t step_hi, ScaleArg sa) {
   const float scale = resolve_scale(sa);
-  const int64_t pairs = k >> 1;
+  const int64_t quads = k >> 2;
   const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
-  for (int64_t p = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; p < pairs; p += stride) {
-    const longlong2 id = reinterpret_cast<const longlong2*>(idx)[p];
-    const float2 s = reinterpret_cast<const float2*>(S_in)[p];
-    const float z0 = z_of(static_cast<uint64_t>(idx_base + id.x), step_lo, step_hi, seed_lo, seed_hi);
-    const float z1 = z_of(static_cast<uint64_t>(idx_base + id.y), step_lo, step_hi, seed_lo, seed_hi);
-    float2 o;
+  for (int64_t p = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; p < quads; p += stride) {
+    const longlong2 ia = reinterpret_cast<const longlong2*>(idx)[2 * p];
+    const longlong2 ib = reinterpret_cast<const longlong2*>(idx)[2 * p + 1];
+    const float4 s = reinterpret_cast<const float4*>(S_in)[p];
+    const float z0 = z_of(static_cast<uint64_t>(idx_base + ia.x), step_lo, step_hi, K);
+    const float z1 = z_of(static_cast<uint64_t>(idx_base + ia.y), step_lo, step_hi, K);
+    const float z2 = z_of(static_cast<uint64_t>(idx_base + ib.x), step_lo, step_hi, K);
+    const float z3 = z_of(static_cast<uint64_t>(idx_base + ib.y), step_lo, step_hi, K);
+    float4 o;
     o.x = fmaf(scale, z0, s.x);
     o.y = fmaf(scale, z1, s.y);
-    reinterpret_cast<float2*>(S_out)[p] = o;
+    o.z = fmaf(scale, z2, s.z);
+    o.w = fmaf(scale, z3, s.w);
+    reinterpret_cast<float4*>(S_out)[p] = o;
   }
-  if ((k & 1) && blockIdx.x == 0 && threadIdx.x == 0) {
-    const int64_t j = k - 1;
-    const float z = z_of(static_cast<uint64_t>(idx_base + idx[j]), step_lo, step_hi, seed_lo, seed_hi);
+  // up to three trailing entries
+  const int64_t j = (quads << 2) + static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (j < k && blockIdx.x == 0 && threadIdx.x < 3) {
+    const float z = z_of(static_cast<uint64_t>(idx_base + idx[j]), step_lo, step_hi, K);
     S_out[j] = fmaf(scale, z, S_in[j]);
   }
 }
@@ -87,13 +99,20 @@ szo_status launch_sparse_axpy(const float* S_in, float* S_out, const int64_t* id
                               int64_t idx_base, uint64_t seed, uint64_t step, ScaleArg sa,
                               cudaStream_t st) {
   if (k == 0) return SZO_OK;
-  const int64_t pairs = (k + 1) / 2;
-  int64_t blocks = ceil_div(pairs, 256);
+  PhiloxKeys K;
+  uint32_t k0 = static_cast<uint32_t>(seed), k1 = static_cast<uint32_t>(seed >> 32);
+  for (int r = 0; r < 10; ++r) {
+    K.k0[r] = k0;
+    K.k1[r] = k1;
+    k0 += kPhiloxW0;
+    k1 += kPhiloxW1;
+  }
+  const int64_t quads = (k + 3) / 4;
+  int64_t blocks = ceil_div(quads, 256);
   const int64_t cap = 148 * 8;
   if (blocks > cap) blocks = cap;
   sparse_axpy_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(
-      S_in, S_out, idx, k, idx_base, static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32),
-      static_cast<uint32_t>(step), static_cast<uint32_t>(step >> 32), sa);
+      S_in, S_out, idx, k, idx_base, K, static_cast<uint32_t>(step), static_cast<uint32_t>(step >> 32), sa);
   count_launch();
   SZO_CHECK_LAUNCH("sparse_axpy_kernel");
   return SZO_OK;
