@@ -39,11 +39,45 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
 }
 
 // z = sqrt(-2 ln u1) cos(2 pi u2), u1 = ((r0 >> 8) + 1) 2^-24 in (0,1], u2 = (r1 >> 8) 2^-24 in [0,1).
+// The pass is bound by instruction issue as much as by memory, so ln and cos are evaluated by short
+// polynomials without the special-case handling of the library routines (u1 is a normal number in
+// (0,1], the cosine argument is exactly reduced):
+//   ln u1:  u1 = f 2^e with f in [sqrt(1/2), sqrt(2)), s = f - 1, ln(1+s) = s - s^2/2 + s^3 P(s)
+//   cos(2 pi u2) = -cos(pi y), y = 2 u2 - 1; with a = |y| and b = min(a, 1 - a) in [0, 1/2]:
+//                  cos(pi a) = +-cos(pi b) = +-C(b^2)
+// P (degree 7) and C (degree 6) are least-squares fits on Chebyshev nodes (fit_gauss_polys.py, which
+// also checks |z - z_fp64| <= 5e-7 max(1,|z|) for this arithmetic).
 __device__ __forceinline__ float gaussian_from_words(uint32_t r0, uint32_t r1) {
   const float u1 = static_cast<float>((r0 >> 8) + 1u) * 5.9604644775390625e-8f;
-  const float two_u2 = static_cast<float>(r1 >> 8) * 1.1920928955078125e-7f;   // 2*u2, exact
-  const float rad = sqrtf(-2.0f * logf(u1));
-  return rad * cospif(two_u2);
+  const int bits = __float_as_int(u1);
+  const int e = (bits - 0x3F3504F3) >> 23;
+  const float s = __int_as_float(bits - (e << 23)) - 1.0f;
+  float p = -8.102270427e-02f;
+  p = fmaf(p, s, 1.271267889e-01f);
+  p = fmaf(p, s, -1.297214522e-01f);
+  p = fmaf(p, s, 1.420211430e-01f);
+  p = fmaf(p, s, -1.664225085e-01f);
+  p = fmaf(p, s, 2.000147135e-01f);
+  p = fmaf(p, s, -2.500029652e-01f);
+  p = fmaf(p, s, 3.333332856e-01f);
+  const float s2 = s * s;
+  const float lg = fmaf(s2 * s, p, fmaf(-0.5f, s2, s));
+  const float L = fmaf(static_cast<float>(e), 0.6931471805599453f, lg);
+  float rad;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rad) : "f"(-2.0f * L));
+
+  const float x = static_cast<float>(r1 >> 8) * 1.1920928955078125e-7f;   // 2 u2 in [0, 2), exact
+  const float a = fabsf(x - 1.0f);
+  const float b = fminf(a, 1.0f - a);
+  const float t = b * b;
+  float c = 1.840005517e-03f;
+  c = fmaf(c, t, -2.577632849e-02f);
+  c = fmaf(c, t, 2.353254400e-01f);
+  c = fmaf(c, t, -1.335262316e+00f);
+  c = fmaf(c, t, 4.058712108e+00f);
+  c = fmaf(c, t, -4.934802200e+00f);
+  c = fmaf(c, t, 1.0f);
+  return (a > 0.5f) ? rad * c : -(rad * c);
 }
 
 __device__ __forceinline__ float z_of(uint64_t gidx, uint32_t step_lo, uint32_t step_hi, const PhiloxKeys& K) {
@@ -107,10 +141,15 @@ szo_status launch_sparse_axpy(const float* S_in, float* S_out, const int64_t* id
     k0 += kPhiloxW0;
     k1 += kPhiloxW1;
   }
+  // grid: whole waves of 148 x 8 blocks when there is enough work, so that every SM gets the same share
   const int64_t quads = (k + 3) / 4;
   int64_t blocks = ceil_div(quads, 256);
-  const int64_t cap = 148 * 8;
-  if (blocks > cap) blocks = cap;
+  const int64_t wave = 148 * 8;
+  if (blocks > wave) {
+    const int64_t sweeps = ceil_div(blocks, wave);          // iterations of the grid-stride loop
+    blocks = ceil_div(ceil_div(quads, sweeps), 256);        // just enough threads for that many sweeps
+    if (blocks > wave) blocks = wave;
+  }
   sparse_axpy_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(
       S_in, S_out, idx, k, idx_base, K, static_cast<uint32_t>(step), static_cast<uint32_t>(step >> 32), sa);
   count_launch();
