@@ -92,33 +92,44 @@ __device__ __forceinline__ float resolve_scale(const ScaleArg& a) {
   return -static_cast<float>(static_cast<double>(a.lr) * g);
 }
 
-// Four entries per thread and iteration: two 16-byte index loads, one 16-byte value load and store,
-// four independent Philox/Box-Muller chains in flight.
+// Eight entries per thread and iteration (four 16-byte index loads, two 16-byte value loads and
+// stores): eight independent Philox / Box-Muller chains in flight hide the latency of the serial
+// ten-round chain.  The next iteration's loads are issued before the current values are computed.
+constexpr int kAxpyPer = 8;
+
 __global__ void __launch_bounds__(256)
 sparse_axpy_kernel(const float* __restrict__ S_in, float* __restrict__ S_out,
                    const int64_t* __restrict__ idx, int64_t k, int64_t idx_base, const PhiloxKeys K,
                    uint32_t step_lo, uint32_t step_hi, ScaleArg sa) {
   const float scale = resolve_scale(sa);
-  const int64_t quads = k >> 2;
+  const int64_t octs = k / kAxpyPer;
   const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
-  for (int64_t p = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; p < quads; p += stride) {
-    const longlong2 ia = reinterpret_cast<const longlong2*>(idx)[2 * p];
-    const longlong2 ib = reinterpret_cast<const longlong2*>(idx)[2 * p + 1];
-    const float4 s = reinterpret_cast<const float4*>(S_in)[p];
-    const float z0 = z_of(static_cast<uint64_t>(idx_base + ia.x), step_lo, step_hi, K);
-    const float z1 = z_of(static_cast<uint64_t>(idx_base + ia.y), step_lo, step_hi, K);
-    const float z2 = z_of(static_cast<uint64_t>(idx_base + ib.x), step_lo, step_hi, K);
-    const float z3 = z_of(static_cast<uint64_t>(idx_base + ib.y), step_lo, step_hi, K);
-    float4 o;
-    o.x = fmaf(scale, z0, s.x);
-    o.y = fmaf(scale, z1, s.y);
-    o.z = fmaf(scale, z2, s.z);
-    o.w = fmaf(scale, z3, s.w);
-    reinterpret_cast<float4*>(S_out)[p] = o;
+  for (int64_t p = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; p < octs; p += stride) {
+    longlong2 id[4];
+    float4 s[2];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) id[j] = reinterpret_cast<const longlong2*>(idx)[4 * p + j];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) s[j] = reinterpret_cast<const float4*>(S_in)[2 * p + j];
+    float z[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      z[2 * j] = z_of(static_cast<uint64_t>(idx_base + id[j].x), step_lo, step_hi, K);
+      z[2 * j + 1] = z_of(static_cast<uint64_t>(idx_base + id[j].y), step_lo, step_hi, K);
+    }
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      float4 o;
+      o.x = fmaf(scale, z[4 * j], s[j].x);
+      o.y = fmaf(scale, z[4 * j + 1], s[j].y);
+      o.z = fmaf(scale, z[4 * j + 2], s[j].z);
+      o.w = fmaf(scale, z[4 * j + 3], s[j].w);
+      reinterpret_cast<float4*>(S_out)[2 * p + j] = o;
+    }
   }
-  // up to three trailing entries
-  const int64_t j = (quads << 2) + static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (j < k && blockIdx.x == 0 && threadIdx.x < 3) {
+  // up to seven trailing entries
+  const int64_t j = octs * kAxpyPer + threadIdx.x;
+  if (blockIdx.x == 0 && threadIdx.x < kAxpyPer && j < k) {
     const float z = z_of(static_cast<uint64_t>(idx_base + idx[j]), step_lo, step_hi, K);
     S_out[j] = fmaf(scale, z, S_in[j]);
   }
@@ -142,7 +153,7 @@ szo_status launch_sparse_axpy(const float* S_in, float* S_out, const int64_t* id
     k1 += kPhiloxW1;
   }
   // grid: whole waves of 148 x 8 blocks when there is enough work, so that every SM gets the same share
-  const int64_t quads = (k + 3) / 4;
+  const int64_t quads = (k + kAxpyPer - 1) / kAxpyPer;     // work items (groups of kAxpyPer entries)
   int64_t blocks = ceil_div(quads, 256);
   const int64_t wave = 148 * 8;
   if (blocks > wave) {
