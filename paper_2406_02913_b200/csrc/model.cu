@@ -45,30 +45,65 @@ __global__ void embed_kernel(const int32_t* __restrict__ tok, const __nv_bfloat1
     h[m * d + c] = __bfloat162float(e[c]) + (p ? __bfloat162float(p[c]) : 0.f);
 }
 
-// RMSNorm (beta == nullptr): x / sqrt(mean x^2 + eps) * gamma; LayerNorm otherwise.
-// row_stride/row_offset select which rows are normalised (all rows, or the last token of each
-// sequence when only that one feeds the loss).
+// Residual add fused with the norm that follows it: h[m] += y[m] (when y != nullptr; written back
+// unless the rows are a strided selection), then RMSNorm (x / sqrt(mean x^2 + eps) * gamma) or
+// LayerNorm of the row.  One block per row; the row (d <= 8192 floats) lives in registers, so global
+// memory is read once.  row_stride/row_offset select which rows are normalised (all rows, or the
+// last token of each sequence when only that one feeds the loss).
 template <typename T>
 __global__ void __launch_bounds__(256)
-norm_kernel(const float* __restrict__ h, const float* __restrict__ gamma, const float* __restrict__ beta,
-            int d, float eps, bool layer_norm, int64_t row_stride, int64_t row_offset, T* __restrict__ out) {
+add_norm_kernel(float* __restrict__ h, const T* __restrict__ y, const float* __restrict__ gamma,
+                const float* __restrict__ beta, int d, float eps, bool layer_norm, int64_t row_stride,
+                int64_t row_offset, T* __restrict__ out) {
+  constexpr int kMaxV = 8;                       // float4 per thread: d <= 256 * 4 * 8
   __shared__ float scratch[32];
   const int64_t m = static_cast<int64_t>(blockIdx.x) * row_stride + row_offset;
-  const float* x = h + m * d;
+  float* x = h + m * d;
   T* o = out + static_cast<int64_t>(blockIdx.x) * d;
+  const int nv = d >> 2;                         // float4 units in a row
+  float4 v[kMaxV];
   float s = 0.f;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) s += x[c];
+#pragma unroll
+  for (int i = 0; i < kMaxV; ++i) {
+    const int c = threadIdx.x + i * 256;
+    v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (c < nv) {
+      v[i] = reinterpret_cast<const float4*>(x)[c];
+      if (y != nullptr) {
+        const T* yp = y + m * d + c * 4;
+        v[i].x += to_f32<T>(yp[0]);
+        v[i].y += to_f32<T>(yp[1]);
+        v[i].z += to_f32<T>(yp[2]);
+        v[i].w += to_f32<T>(yp[3]);
+        if (row_stride == 1) reinterpret_cast<float4*>(x)[c] = v[i];
+      }
+      s += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+    }
+  }
   const float mu = layer_norm ? block_sum(s, scratch) / d : 0.f;
   float q = 0.f;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) {
-    const float t = x[c] - mu;
-    q = fmaf(t, t, q);
+#pragma unroll
+  for (int i = 0; i < kMaxV; ++i) {
+    if (threadIdx.x + i * 256 < nv) {
+      const float a0 = v[i].x - mu, a1 = v[i].y - mu, a2 = v[i].z - mu, a3 = v[i].w - mu;
+      q += (a0 * a0 + a1 * a1) + (a2 * a2 + a3 * a3);
+    }
   }
   const float var = block_sum(q, scratch) / d;
   const float r = 1.0f / sqrtf(var + eps);
-  for (int c = threadIdx.x; c < d; c += blockDim.x) {
-    const float v = (x[c] - mu) * r * gamma[c] + (beta ? beta[c] : 0.f);
-    o[c] = from_f32<T>(v);
+#pragma unroll
+  for (int i = 0; i < kMaxV; ++i) {
+    const int c = threadIdx.x + i * 256;
+    if (c < nv) {
+      const float4 g = reinterpret_cast<const float4*>(gamma)[c];
+      float4 bt = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (beta) bt = reinterpret_cast<const float4*>(beta)[c];
+      T* op = o + c * 4;
+      op[0] = from_f32<T>((v[i].x - mu) * r * g.x + bt.x);
+      op[1] = from_f32<T>((v[i].y - mu) * r * g.y + bt.y);
+      op[2] = from_f32<T>((v[i].z - mu) * r * g.z + bt.z);
+      op[3] = from_f32<T>((v[i].w - mu) * r * g.w + bt.w);
+    }
   }
 }
 
@@ -81,21 +116,33 @@ __global__ void rope_table_kernel(int max_seq, int half, double base, float2* __
   tab[i] = make_float2(static_cast<float>(cos(ang)), static_cast<float>(sin(ang)));
 }
 
-// In-place rotation of the pairs (i, i + hd/2) of every head of x [M, n_heads*hd].
+// In-place rotation of the pairs (i, i + hd/2) of every head of q [M, H*hd] and k [M, Hkv*hd] in one
+// launch.  A thread rotates kN consecutive pairs (one 16-byte vector from each half of a head).
 template <typename T>
-__global__ void rope_kernel(T* __restrict__ x, const float2* __restrict__ tab, int64_t M, int S, int n_heads,
-                            int hd) {
-  const int half = hd >> 1;
+__global__ void rope_kernel(T* __restrict__ q, T* __restrict__ k, const float2* __restrict__ tab, int64_t M, int S,
+                            int H, int Hkv, int hd) {
+  constexpr int kN = 16 / sizeof(T);
+  const int half = hd >> 1, vec_per_head = half / kN;
+  const int64_t per_token = static_cast<int64_t>(H + Hkv) * vec_per_head;
   const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (i >= M * n_heads * half) return;
-  const int j = static_cast<int>(i % half);
-  const int64_t mh = i / half;
-  const int64_t m = mh / n_heads;
-  const float2 cs = tab[static_cast<int64_t>(m % S) * half + j];
-  T* p = x + mh * hd;
-  const float a = to_f32<T>(p[j]), b = to_f32<T>(p[j + half]);
-  p[j] = from_f32<T>(a * cs.x - b * cs.y);
-  p[j + half] = from_f32<T>(b * cs.x + a * cs.y);
+  if (i >= M * per_token) return;
+  const int64_t m = i / per_token;
+  int r = static_cast<int>(i % per_token);
+  const int head = r / vec_per_head, j0 = (r % vec_per_head) * kN;
+  T* p = (head < H) ? q + (m * H + head) * hd : k + (m * Hkv + (head - H)) * hd;
+  const float2* cs = tab + static_cast<int64_t>(m % S) * half + j0;
+  T lo[kN], hi[kN];
+  *reinterpret_cast<uint4*>(lo) = *reinterpret_cast<const uint4*>(p + j0);
+  *reinterpret_cast<uint4*>(hi) = *reinterpret_cast<const uint4*>(p + half + j0);
+#pragma unroll
+  for (int j = 0; j < kN; ++j) {
+    const float a = to_f32<T>(lo[j]), b = to_f32<T>(hi[j]);
+    const float2 t = cs[j];
+    lo[j] = from_f32<T>(a * t.x - b * t.y);
+    hi[j] = from_f32<T>(b * t.x + a * t.y);
+  }
+  *reinterpret_cast<uint4*>(p + j0) = *reinterpret_cast<const uint4*>(lo);
+  *reinterpret_cast<uint4*>(p + half + j0) = *reinterpret_cast<const uint4*>(hi);
 }
 
 // Causal softmax attention, one warp per query; lanes split the head dimension.
@@ -269,6 +316,11 @@ __global__ void __launch_bounds__(1024) mean_f64_kernel(const double* __restrict
   if (threadIdx.x == 0) *out = s[0] / denom;
 }
 
+__global__ void offset_eid_kernel(const int32_t* __restrict__ eid, int64_t n, int32_t off, int32_t* __restrict__ out) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = eid[i] + off;
+}
+
 __global__ void gidx_kernel(const int64_t* __restrict__ idx, int64_t nnz, int64_t base, int64_t* __restrict__ out) {
   const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i < nnz) out[i] = base + idx[i];
@@ -289,6 +341,9 @@ struct szo_model {
   float* S_all = nullptr;
   int64_t k_total = 0;
   int64_t* gidx = nullptr;
+  int32_t* geid = nullptr;      // [k_total] entry id in S_all of each bucket-ordered record
+  uint16_t* gpos = nullptr;     // [k_total] in-tile position of each bucket-ordered record
+  uint2* recs = nullptr;        // [k_total] (position, value) records of the current forward
   int64_t Mmax = 0;
   // activations
   float* h = nullptr;
@@ -344,6 +399,7 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
   T *a = static_cast<T*>(m->a), *q = static_cast<T*>(m->q), *k = static_cast<T*>(m->k), *v = static_cast<T*>(m->v),
     *o = static_cast<T*>(m->o), *y = static_cast<T*>(m->y), *gate = static_cast<T*>(m->gate),
     *up = static_cast<T*>(m->up);
+  const bool pregather = c.linear_mode != SZO_MODE_FP32_VALIDATE && c.linear_mode != SZO_MODE_SPMM && m->k_total > 0;
   auto lin = [&](int layer, int j, const void* x, void* out) -> szo_status {
     const int t = layer * m->n_lin + j;
     if (m->timing) {
@@ -354,8 +410,9 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
       }
       SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used], st));
     }
-    const szo_status rc = szo_linear_fwd(m->plans[t], x, static_cast<szo_dtype>(act), M, Sv + m->offsets[t], out,
-                                         static_cast<szo_dtype>(act), c.linear_mode, m->ws, m->ws_bytes, st);
+    const szo_status rc = linear_fwd_impl(m->plans[t], x, act, M, Sv + m->offsets[t],
+                                          pregather ? m->recs + m->offsets[t] : nullptr, out, act, c.linear_mode,
+                                          m->ws, m->ws_bytes, st);
     if (m->timing) {
       SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used + 1], st));
       m->events_used += 2;
@@ -366,18 +423,21 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
                                                         static_cast<const __nv_bfloat16*>(m->top.pos), S, d,
                                                         c.vocab, m->h);
   count_launch();
+  // One gather of all sparse values into the bucket order of every linear (SparseAdd mode)
+  if (pregather) SZO_TRY(gather_values(Sv, m->geid, m->gpos, m->k_total, m->recs, st));
+  const T* pending = nullptr;     // projection output still to be added to the residual stream
   for (int l = 0; l < c.n_layers; ++l) {
     const szo_layer_weights& L = m->layers[l];
-    norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, L.attn_norm_g, L.attn_norm_b, d, c.norm_eps, opt,
-                                                            1, 0, a);
+    add_norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, pending, L.attn_norm_g, L.attn_norm_b, d,
+                                                                c.norm_eps, opt, 1, 0, a);
     count_launch();
     SZO_TRY(lin(l, 0, a, q));
     SZO_TRY(lin(l, 1, a, k));
     SZO_TRY(lin(l, 2, a, v));
     if (!opt) {
-      rope_kernel<T><<<blocks_for(M * H * (hd / 2), 256), 256, 0, st>>>(q, m->rope_tab, M, S, H, hd);
-      rope_kernel<T><<<blocks_for(M * Hkv * (hd / 2), 256), 256, 0, st>>>(k, m->rope_tab, M, S, Hkv, hd);
-      count_launch(2);
+      const int64_t n_vec = M * (H + Hkv) * ((hd / 2) / Vec16<T>::kN);
+      rope_kernel<T><<<blocks_for(n_vec, 256), 256, 0, st>>>(q, k, m->rope_tab, M, S, H, Hkv, hd);
+      count_launch();
     }
     if constexpr (sizeof(T) == 2) {
       SZO_TRY(launch_flash_attention_bf16(q, k, v, o, B, S, H, Hkv, hd, st));
@@ -389,10 +449,9 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
       count_launch();
     }
     SZO_TRY(lin(l, 3, o, y));
-    residual_add_kernel<T><<<blocks_for(M * d / Vec16<T>::kN, 256), 256, 0, st>>>(m->h, y, M * d);
-    norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, L.mlp_norm_g, L.mlp_norm_b, d, c.norm_eps, opt, 1,
-                                                            0, a);
-    count_launch(2);
+    add_norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, y, L.mlp_norm_g, L.mlp_norm_b, d, c.norm_eps,
+                                                                opt, 1, 0, a);
+    count_launch();
     if (!opt) {
       SZO_TRY(lin(l, 4, a, gate));
       SZO_TRY(lin(l, 5, a, up));
@@ -405,12 +464,11 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
       count_launch();
       SZO_TRY(lin(l, 5, gate, y));
     }
-    residual_add_kernel<T><<<blocks_for(M * d / Vec16<T>::kN, 256), 256, 0, st>>>(m->h, y, M * d);
-    count_launch();
+    pending = y;                  // added by the next norm (next layer's, or the final one)
   }
   if (c.loss_kind == 0) {
-    norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, m->top.final_norm_g, m->top.final_norm_b, d,
-                                                            c.norm_eps, opt, 1, 0, a);
+    add_norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, pending, m->top.final_norm_g,
+                                                                m->top.final_norm_b, d, c.norm_eps, opt, 1, 0, a);
     count_launch();
     const int mode = c.linear_mode == SZO_MODE_FP32_VALIDATE ? SZO_MODE_FP32_VALIDATE : SZO_MODE_SPARSE_ADD;
     SZO_TRY(szo_linear_fwd(m->lm_head_plan, a, static_cast<szo_dtype>(act), M, nullptr, m->logits, SZO_F32, mode,
@@ -419,8 +477,8 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
     mean_f64_kernel<<<1, 1024, 0, st>>>(m->tok_loss, M, static_cast<double>(B) * (S - 1), loss_dev);
     count_launch(2);
   } else {
-    norm_kernel<T><<<static_cast<unsigned>(B), 256, 0, st>>>(m->h, m->top.final_norm_g, m->top.final_norm_b, d,
-                                                            c.norm_eps, opt, S, S - 1, a);
+    add_norm_kernel<T><<<static_cast<unsigned>(B), 256, 0, st>>>(m->h, pending, m->top.final_norm_g,
+                                                                m->top.final_norm_b, d, c.norm_eps, opt, S, S - 1, a);
     cls2_kernel<T><<<static_cast<unsigned>(B), 256, 0, st>>>(a, static_cast<const __nv_bfloat16*>(m->top.lm_head), cand,
                                                             labels, d, c.vocab, m->tok_loss);
     mean_f64_kernel<<<1, 1024, 0, st>>>(m->tok_loss, B, static_cast<double>(B), loss_dev);
@@ -465,6 +523,7 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
   const int hd = c.d_model / c.n_heads;
   SZO_REQUIRE(hd == 64 || hd == 128, SZO_ERR_UNSUPPORTED, "head dimension must be 64 or 128 (got %d)", hd);
   SZO_REQUIRE(c.d_model % 8 == 0 && c.d_ff % 8 == 0, SZO_ERR_SHAPE, "d_model and d_ff must be multiples of 8");
+  SZO_REQUIRE(c.d_model <= 8192, SZO_ERR_UNSUPPORTED, "d_model above 8192 is not supported by the norm kernel");
   SZO_REQUIRE(c.act_dtype == SZO_BF16 || c.act_dtype == SZO_F32, SZO_ERR_UNSUPPORTED, "act_dtype must be bf16 or f32");
   SZO_REQUIRE(c.act_dtype == SZO_BF16 || c.linear_mode == SZO_MODE_FP32_VALIDATE, SZO_ERR_UNSUPPORTED,
               "fp32 activations need the fp32 validation mode");
@@ -546,6 +605,19 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
       if (w.nnz)
         gidx_kernel<<<blocks_for(w.nnz, 256), 256, 0, st>>>(w.idx, w.nnz, base, m->gidx + m->offsets[t]);
       base += N * K;
+    }
+  }
+  // model-wide bucket order: linear t's records occupy [offsets[t], offsets[t+1]) and refer to S_all
+  SZO_M_TRY(dev_alloc(m, &m->geid, m->k_total * sizeof(int32_t)));
+  SZO_M_TRY(dev_alloc(m, &m->gpos, m->k_total * sizeof(uint16_t)));
+  SZO_M_TRY(dev_alloc(m, &m->recs, m->k_total * sizeof(uint2)));
+  if (m->k_total >= (int64_t(1) << 31)) return bail(fail(SZO_ERR_SHAPE, "more than 2^31 sparse entries"));
+  for (size_t t = 0; t < m->plans.size(); ++t) {
+    const szo_linear* p = m->plans[t];
+    if (p->nnz) {
+      offset_eid_kernel<<<blocks_for(p->nnz, 256), 256, 0, st>>>(p->bucket_eid, p->nnz, static_cast<int32_t>(m->offsets[t]),
+                                                               m->geid + m->offsets[t]);
+      cudaMemcpyAsync(m->gpos + m->offsets[t], p->bucket_pos, p->nnz * sizeof(uint16_t), cudaMemcpyDeviceToDevice, st);
     }
   }
   rope_table_kernel<<<blocks_for(static_cast<int64_t>(c.max_seq) * (hd / 2), 256), 256, 0, st>>>(
