@@ -1,0 +1,93 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times: the fused
+linear at the Llama-2-7B shapes (M = 4096 tokens) and the sparse passes at k = 6.48 M, checked on
+sampled outputs that the oracle computes one by one (a full fp64 product would take minutes)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import szo_oracle as so
+from paper_2406_02913_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2406_02913_b200 import binding
+    binding.lib()
+    return binding
+
+
+def _bf16_bits(t):
+    return t.cpu().view(torch.int16).numpy().view(np.uint16)
+
+
+@pytest.mark.parametrize("N,K,mode", [(4096, 4096, "sparse_add"), (11008, 4096, "sparse_add"), (4096, 11008, "sparse_add"),
+                                      (4096, 4096, "spmm")])
+def test_llama7b_linear_sampled_outputs(B, N, K, mode):
+    M, G, rho = 4096, 128, 1e-3
+    g = torch.Generator(device="cuda")
+    g.manual_seed(N * 7 + K)
+    codes = torch.randint(0, 256, (N, K // 2), generator=g, device="cuda", dtype=torch.uint8)
+    sc = (0.004 + 0.002 * torch.rand(N, K // G, generator=g, device="cuda")).to(torch.bfloat16)
+    ze = (-7.5 * sc.float()).to(torch.bfloat16)
+    nnz = int(rho * N * K)
+    idx_np = wl.sorted_random_indices(N * K, nnz, seed=N + K)
+    idx = torch.from_numpy(idx_np).cuda()
+    S = (torch.randn(nnz, generator=g, device="cuda") * 0.02).contiguous()
+    x = torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16)
+    plan = B.Linear(N, K, G, codes, sc, ze, "bf16", idx)
+    md = B.MODE_SPARSE_ADD if mode == "sparse_add" else B.MODE_SPMM
+    y = plan.fwd(x, S, md, torch.float32)
+    torch.cuda.synchronize()
+    assert B.device_status() == 0
+
+    # oracle on sampled rows of W (all their columns) x sampled tokens, plus the tile corners
+    r = wl.rng(5, wl.PURPOSE_INDICES, N + K)
+    rows = np.unique(np.concatenate([r.integers(0, N, 24), [0, 127, 128, N - 129, N - 1]]))
+    toks = np.unique(np.concatenate([r.integers(0, M, 24), [0, 255, 256, M - 257, M - 1]]))
+    codes_h = codes[rows].cpu().numpy()
+    deq = so.dequantize(codes_h, _bf16_bits(sc[rows]), _bf16_bits(ze[rows]), G, "bf16")       # [rows, K] fp64
+    S_h = S.cpu().numpy().astype(np.float64)
+    for i, n in enumerate(rows):
+        lo, hi = np.searchsorted(idx_np, [n * K, (n + 1) * K])
+        np.add.at(deq[i], idx_np[lo:hi] - n * K, S_h[lo:hi])
+    xs = x[toks].float().cpu().numpy().astype(np.float64)
+    ref = xs @ deq.T                                                                          # [toks, rows]
+    got = y[toks][:, rows].cpu().numpy().astype(np.float64)
+    scale = np.max(np.abs(ref))
+    assert np.max(np.abs(got - ref)) <= 2e-2 * scale
+    assert np.max(np.abs(got - ref)) <= 4e-3 * scale           # observed: bf16 weight rounding only
+    # everything finite, and bitwise repeatable
+    assert torch.isfinite(y).all()
+    y2 = plan.fwd(x, S, md, torch.float32)
+    assert torch.equal(y, y2)
+    plan.close()
+
+
+def test_sparse_passes_at_7b_scale(B):
+    """k = 0.1 % of the Llama-2-7B linear parameters: the +eps, -2eps, +eps sequence and an update,
+    checked on a sample of entries (z and the fp32 fma), with the unsampled rest checked for the
+    restore property."""
+    n_total, k = 6_476_005_376, 6_476_005
+    idx_np = wl.sorted_random_indices(n_total, k, seed=77)
+    idx = torch.from_numpy(idx_np).cuda()
+    S0 = torch.from_numpy(wl.rng(78, wl.PURPOSE_WEIGHTS).normal(0, 0.02, k).astype(np.float32)).cuda()
+    S = S0.clone()
+    seed, step, eps = 1234, 41, np.float32(1e-3)
+    samp = np.unique(np.concatenate([wl.rng(79, wl.PURPOSE_INDICES).integers(0, k, 20000), np.arange(16), k - 1 - np.arange(16)]))
+    z_ref = so.gaussian(seed, step, idx_np[samp])
+    B.szo_perturb(S, S, idx, 0, seed, step, float(eps))
+    s1 = S.cpu().numpy()
+    ref1 = so.fmaf32(eps, z_ref, S0.cpu().numpy()[samp])
+    assert np.all(np.abs(s1[samp].astype(np.float64) - ref1) <= 1e-6 * 1e-3 * np.maximum(1, np.abs(z_ref)) + 4e-9)
+    B.szo_perturb(S, S, idx, 0, seed, step, float(np.float32(-2.0) * eps))
+    B.szo_perturb(S, S, idx, 0, seed, step, float(eps))
+    s3 = S.cpu().numpy()
+    assert np.max(np.abs(s3 - S0.cpu().numpy())) <= 2 * np.spacing(np.float32(0.25))        # restored up to rounding
+    f = torch.tensor([0.69, 0.71], dtype=torch.float64, device="cuda")
+    B.szo_update(S, idx, 0, seed, step, 1e-3, f[0:1], f[1:2], float(eps))
+    sc = so.zo_update_scale(0.69, 0.71, eps, 1e-3)
+    got = S.cpu().numpy()[samp].astype(np.float64)
+    ref = s3[samp].astype(np.float64) + float(sc) * z_ref.astype(np.float64)
+    assert np.all(np.abs(got - ref) <= abs(float(sc)) * 1e-6 * np.maximum(1, np.abs(z_ref)) + 4e-9)

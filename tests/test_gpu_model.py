@@ -174,3 +174,24 @@ def test_attention_matches_oracle(B, B_, S, H, Hkv, hd, dtype):
     got = B.szo_attention(d(q), d(k), d(v), B_, S, H, Hkv, hd).float().cpu().numpy()
     tol = 1.5e-2 if dtype == "bf16" else 2e-6          # bf16: probabilities and outputs are rounded to bf16
     assert np.max(np.abs(got - ref)) <= tol * np.max(np.abs(ref))
+
+
+@pytest.mark.parametrize("name,loss_kind,mode", [("tiny_opt", 0, "sparse_add"), ("tiny_gqa", 1, "sparse_add"),
+                                                 ("tiny_gqa", 0, "spmm")])
+def test_other_architectures_bf16_tensor_core_path(B, name, loss_kind, mode):
+    """OPT-shaped (LayerNorm, biases, ReLU, learned positions, int4) and Mistral-shaped (GQA, dense bf16
+    weights, 1 % mask) decoders on the tensor-core path: losses within 1e-3 of the oracle."""
+    fx = DecoderFixture(name, seed=2, mask="random", B=3, S=48)
+    md = B.MODE_SPARSE_ADD if mode == "sparse_add" else B.MODE_SPMM
+    m, S, _ = build_gpu(B, fx, B.SZO_BF16, md, loss_kind, quantize_on_gpu=fx.shape["group"] > 0)
+    om = fx.oracle_model()
+    toks = fx.batch(0)
+    kind = "lm" if loss_kind == 0 else "cls2"
+    labels = wl.binary_labels(fx.B, 2, 0)
+    cand = np.array([5, 77], np.int32)
+    d = lambda a: torch.from_numpy(a).cuda()
+    fp, fm, g = mo.zo_step(om, toks, 9, 1, 1e-3, 1e-4, kind, labels, cand)
+    out = m.zo_step(d(toks), 9, 1, 1e-3, 1e-4, d(labels), d(cand)).cpu().numpy()
+    assert abs(out[0] - fp) <= LOSS_TOL * abs(fp) and abs(out[1] - fm) <= LOSS_TOL * abs(fm)
+    assert np.isfinite(out[2]) and B.device_status() == 0
+    m.close()
