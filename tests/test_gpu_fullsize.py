@@ -80,7 +80,7 @@ def test_sparse_passes_at_7b_scale(B):
     B.szo_perturb(S, S, idx, 0, seed, step, float(eps))
     s1 = S.cpu().numpy()
     ref1 = so.fmaf32(eps, z_ref, S0.cpu().numpy()[samp])
-    assert np.all(np.abs(s1[samp].astype(np.float64) - ref1) <= 1e-6 * 1e-3 * np.maximum(1, np.abs(z_ref)) + 4e-9)
+    assert np.all(np.abs(s1[samp].astype(np.float64) - ref1) <= 1e-6 * 1e-3 * np.maximum(1, np.abs(z_ref)) + 1.5e-8)   # + one fp32 ulp of the sum
     B.szo_perturb(S, S, idx, 0, seed, step, float(np.float32(-2.0) * eps))
     B.szo_perturb(S, S, idx, 0, seed, step, float(eps))
     s3 = S.cpu().numpy()
@@ -90,4 +90,4 @@ def test_sparse_passes_at_7b_scale(B):
     sc = so.zo_update_scale(0.69, 0.71, eps, 1e-3)
     got = S.cpu().numpy()[samp].astype(np.float64)
     ref = s3[samp].astype(np.float64) + float(sc) * z_ref.astype(np.float64)
-    assert np.all(np.abs(got - ref) <= abs(float(sc)) * 1e-6 * np.maximum(1, np.abs(z_ref)) + 4e-9)
+    assert np.all(np.abs(got - ref) <= abs(float(sc)) * 1e-6 * np.maximum(1, np.abs(z_ref)) + 1.5e-8)   # + one fp32 ulp of the sum
