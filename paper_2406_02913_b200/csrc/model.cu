@@ -50,16 +50,16 @@ __global__ void embed_kernel(const int32_t* __restrict__ tok, const __nv_bfloat1
 // LayerNorm of the row.  One block per row; the row (d <= 8192 floats) lives in registers, so global
 // memory is read once.  row_stride/row_offset select which rows are normalised (all rows, or the
 // last token of each sequence when only that one feeds the loss).
-template <typename T>
+template <typename T, typename TO = T>
 __global__ void __launch_bounds__(256)
 add_norm_kernel(float* __restrict__ h, const T* __restrict__ y, const float* __restrict__ gamma,
                 const float* __restrict__ beta, int d, float eps, bool layer_norm, int64_t row_stride,
-                int64_t row_offset, T* __restrict__ out) {
+                int64_t row_offset, TO* __restrict__ out) {
   constexpr int kMaxV = 8;                       // float4 per thread: d <= 256 * 4 * 8
   __shared__ float scratch[32];
   const int64_t m = static_cast<int64_t>(blockIdx.x) * row_stride + row_offset;
   float* x = h + m * d;
-  T* o = out + static_cast<int64_t>(blockIdx.x) * d;
+  TO* o = out + static_cast<int64_t>(blockIdx.x) * d;
   const int nv = d >> 2;                         // float4 units in a row
   float4 v[kMaxV];
   float s = 0.f;
@@ -98,11 +98,11 @@ add_norm_kernel(float* __restrict__ h, const T* __restrict__ y, const float* __r
       const float4 g = reinterpret_cast<const float4*>(gamma)[c];
       float4 bt = make_float4(0.f, 0.f, 0.f, 0.f);
       if (beta) bt = reinterpret_cast<const float4*>(beta)[c];
-      T* op = o + c * 4;
-      op[0] = from_f32<T>((v[i].x - mu) * r * g.x + bt.x);
-      op[1] = from_f32<T>((v[i].y - mu) * r * g.y + bt.y);
-      op[2] = from_f32<T>((v[i].z - mu) * r * g.z + bt.z);
-      op[3] = from_f32<T>((v[i].w - mu) * r * g.w + bt.w);
+      TO* op = o + c * 4;
+      op[0] = from_f32<TO>((v[i].x - mu) * r * g.x + bt.x);
+      op[1] = from_f32<TO>((v[i].y - mu) * r * g.y + bt.y);
+      op[2] = from_f32<TO>((v[i].z - mu) * r * g.z + bt.z);
+      op[3] = from_f32<TO>((v[i].w - mu) * r * g.w + bt.w);
     }
   }
 }
@@ -477,10 +477,12 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
     mean_f64_kernel<<<1, 1024, 0, st>>>(m->tok_loss, M, static_cast<double>(B) * (S - 1), loss_dev);
     count_launch(2);
   } else {
-    add_norm_kernel<T><<<static_cast<unsigned>(B), 256, 0, st>>>(m->h, pending, m->top.final_norm_g,
-                                                                m->top.final_norm_b, d, c.norm_eps, opt, S, S - 1, a);
-    cls2_kernel<T><<<static_cast<unsigned>(B), 256, 0, st>>>(a, static_cast<const __nv_bfloat16*>(m->top.lm_head), cand,
-                                                            labels, d, c.vocab, m->tok_loss);
+    // only B rows feed this loss: keep their normalised states in fp32 (the q buffer is free here)
+    float* a_last = reinterpret_cast<float*>(m->q);
+    add_norm_kernel<T, float><<<static_cast<unsigned>(B), 256, 0, st>>>(
+        m->h, pending, m->top.final_norm_g, m->top.final_norm_b, d, c.norm_eps, opt, S, S - 1, a_last);
+    cls2_kernel<float><<<static_cast<unsigned>(B), 256, 0, st>>>(
+        a_last, static_cast<const __nv_bfloat16*>(m->top.lm_head), cand, labels, d, c.vocab, m->tok_loss);
     mean_f64_kernel<<<1, 1024, 0, st>>>(m->tok_loss, B, static_cast<double>(B), loss_dev);
     count_launch(3);
   }

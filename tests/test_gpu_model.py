@@ -192,6 +192,11 @@ def test_other_architectures_bf16_tensor_core_path(B, name, loss_kind, mode):
     d = lambda a: torch.from_numpy(a).cuda()
     fp, fm, g = mo.zo_step(om, toks, 9, 1, 1e-3, 1e-4, kind, labels, cand)
     out = m.zo_step(d(toks), 9, 1, 1e-3, 1e-4, d(labels), d(cand)).cpu().numpy()
-    assert abs(out[0] - fp) <= LOSS_TOL * abs(fp) and abs(out[1] - fm) <= LOSS_TOL * abs(fm)
+    # The LM loss averages B*(S-1) positions.  The 2-candidate loss of three sequences does not: it is
+    # softplus(+-(l1 - l0)) of two logits of size ~0.3 whose bf16-path error is ~1.5e-3 absolute
+    # (activations carry 2^-9 relative rounding), and |d loss / d (l1 - l0)| <= 1/2, i.e. about
+    # 1.2e-3 of a loss near ln 2: the bound for that case is 3e-3.
+    tol = LOSS_TOL if loss_kind == 0 else 3e-3
+    assert abs(out[0] - fp) <= tol * abs(fp) and abs(out[1] - fm) <= tol * abs(fm)
     assert np.isfinite(out[2]) and B.device_status() == 0
     m.close()
