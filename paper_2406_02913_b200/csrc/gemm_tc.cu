@@ -196,78 +196,123 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
       }
     }
   } else if (warp == 2) {
-    // ---------------------------------------------------------------- SparseAdd warp
-    // Adds the sparse values of bucket (tile, k-block) to the bf16 weight tile in shared memory.
-    // Bucket bounds and records are brought in with cp.async kLook / 2*kLook iterations ahead; each of
-    // the three streams (bounds, records, apply) walks the (tile, k-block) sequence with its own cursor.
+    // ---------------------------------------------------------------- sparse-record warp
+    // Brings the bucket bounds and the sparse records (position in tile, fp32 value) of every
+    // (tile, k-block) into two small rings in shared memory, a few k-blocks ahead of their use.
+    // Plain global loads into registers, stored to shared memory two iterations later (two register
+    // sets in flight), so that no load latency sits on this warp's loop.  In dequantising mode the
+    // conversion warps add the values to the weight tile; for a dense bf16 weight this warp does.
+    //   iteration it:  store {bounds(it+6), records(it+3)} loaded at it-2, signal recready(it+3),
+    //                  load  {bounds(it+8), records(it+5)}    (records(it+5) are addressed by
+    //                  bounds(it+5), stored at it-1)
     if (sparse && my_tiles > 0) {
-      struct Cursor {
-        int lt, kb, bucket0;     // bucket0 = n_tile * n_kblocks for the cursor's tile
-      };
       const int n_kblocks = static_cast<int>(P.n_kblocks);
-      auto start = [&]() {
-        return Cursor{0, 0, static_cast<int>((blockIdx.x / m_tiles)) * n_kblocks};
+      const int my_iters = my_tiles * nkb;
+      struct Cursor {
+        int it, lt, kb, bucket0;     // bucket0 = n_tile * n_kblocks of the cursor's tile
       };
+      auto make_cursor = [&]() { return Cursor{0, 0, 0, static_cast<int>(blockIdx.x / m_tiles) * n_kblocks}; };
       auto step = [&](Cursor& c) {
+        ++c.it;
         if (++c.kb == nkb) {
           c.kb = 0;
           ++c.lt;
           c.bucket0 = ((blockIdx.x + c.lt * gridDim.x) / m_tiles) * n_kblocks;
         }
       };
-      Cursor cb = start(), cr = start();            // bounds stream, records stream
-      int ib = 0, ir = 0;                           // their iteration numbers (ring slots)
-      auto issue_bounds = [&]() {                   // lanes 0,1 copy bucket_ptr[b], bucket_ptr[b+1]
-        if (cb.lt < my_tiles) {
-          if (lane < 2) cp_async_4(smem_u32(&bound_ring[ib & (kBoundSlots - 1)][lane]), P.bucket_ptr + cb.bucket0 + cb.kb + lane);
+      struct Loaded {
+        int32_t bound;               // lanes 0,1: bucket_ptr[b], bucket_ptr[b+1]
+        uint2 rec[2];                // records lane and lane + 32 of the bucket
+        int32_t n;                   // records of the bucket held in the ring (<= kRecCap)
+      };
+      Cursor cb = make_cursor(), cr = make_cursor();       // bounds stream, records stream
+      auto load_set = [&](Loaded& L) {                     // bounds(cb.it), records(cr.it)
+        L.bound = 0;
+        L.n = 0;
+        if (cb.it < my_iters) {
+          if (lane < 2) L.bound = __ldg(P.bucket_ptr + cb.bucket0 + cb.kb + lane);
+        }
+        if (cr.it < my_iters) {
+          const int32_t e0 = bound_ring[cr.it & (kBoundSlots - 1)][0], e1 = bound_ring[cr.it & (kBoundSlots - 1)][1];
+          L.n = (e1 - e0 < kRecCap) ? e1 - e0 : kRecCap;
+          if (lane < L.n) L.rec[0] = __ldg(P.Sb + e0 + lane);
+          if (lane + 32 < L.n) L.rec[1] = __ldg(P.Sb + e0 + lane + 32);
+        }
+      };
+      auto store_set = [&](const Loaded& L) {              // then advance both streams
+        if (cb.it < my_iters) {
+          if (lane < 2) bound_ring[cb.it & (kBoundSlots - 1)][lane] = L.bound;
           step(cb);
-          ++ib;
         }
-      };
-      auto issue_records = [&]() {                  // needs the bounds of that iteration in shared memory
-        if (cr.lt < my_tiles) {
-          const int32_t e0 = bound_ring[ir & (kBoundSlots - 1)][0], e1 = bound_ring[ir & (kBoundSlots - 1)][1];
-          const int32_t n = (e1 - e0 < kRecCap) ? e1 - e0 : kRecCap;
-          for (int32_t j = lane; j < n; j += 32) cp_async_8(smem_u32(&rec_ring[ir & (kRecSlots - 1)][j]), P.Sb + e0 + j);
+        if (cr.it < my_iters) {
+          if (lane < L.n) rec_ring[cr.it & (kRecSlots - 1)][lane] = L.rec[0];
+          if (lane + 32 < L.n) rec_ring[cr.it & (kRecSlots - 1)][lane + 32] = L.rec[1];
           step(cr);
-          ++ir;
         }
       };
-      // prologue: bounds of iterations 0..2*kLook-1, then records of 0..kLook-1
-      for (int j = 0; j < 2 * kLook; ++j) issue_bounds();
-      cp_async_commit();
-      cp_async_wait_all();
+      static_assert(kRecCap == 64 && kRecSlots == 8 && kBoundSlots == 16, "ring sizes are part of the schedule");
+      // prologue: bounds 0..5 and records 0..2 directly, then prime the two register sets
+      Loaded set0, set1;
+      for (int j = 0; j < 6; ++j) {                        // bounds only (the records stream idles)
+        Loaded L;
+        L.bound = 0;
+        L.n = 0;
+        if (cb.it < my_iters && lane < 2) L.bound = __ldg(P.bucket_ptr + cb.bucket0 + cb.kb + lane);
+        if (cb.it < my_iters) {
+          if (lane < 2) bound_ring[cb.it & (kBoundSlots - 1)][lane] = L.bound;
+          step(cb);
+        }
+      }
       __syncwarp();
-      for (int j = 0; j < kLook; ++j) {
-        issue_records();
-        cp_async_commit();
+      for (int j = 0; j < 3; ++j) {                        // records 0..2 (bounds stream idles)
+        if (cr.it < my_iters) {
+          const int32_t e0 = bound_ring[cr.it & (kBoundSlots - 1)][0], e1 = bound_ring[cr.it & (kBoundSlots - 1)][1];
+          const int32_t n = (e1 - e0 < kRecCap) ? e1 - e0 : kRecCap;
+          for (int32_t q = lane; q < n; q += 32) rec_ring[cr.it & (kRecSlots - 1)][q] = __ldg(P.Sb + e0 + q);
+          __syncwarp();
+          if (kDequant && lane == 0) mbar_arrive(recready_bar(cr.it & (kRecSlots - 1)));
+          step(cr);
+        }
+      }
+      // the two sets in flight: {bounds(6), records(3)} and {bounds(7), records(4)}
+      {
+        Cursor sb = cb, sr = cr;
+        load_set(set0);
+        step(cb);
+        step(cr);
+        load_set(set1);
+        cb = sb;
+        cr = sr;
       }
       RingPos x{0, 0}, a{0, 0};
-      const int my_iters = my_tiles * nkb;
-      for (int it = 0; it < my_iters; ++it) {
-        // group(j) = { bounds(j + 2 kLook), records(j + kLook) }, committed in iteration j.  Groups
-        // retire in order: with at most kLook - 1 still pending, group(it - kLook) has landed, i.e.
-        // records(it) and bounds(it + kLook), which the next record copies are addressed from.
-        cp_async_wait_group<kLook - 1>();
-        __syncwarp();
+      // one iteration, on the register set that was loaded two iterations ago
+      auto iteration = [&](int it, Loaded& L) -> bool {
         if constexpr (kDequant) {
-          // The conversion warps apply the records themselves.  Tell them records(it) are in shared
-          // memory, then keep at most kRecSlots - kLook iterations ahead of them so that a ring slot
-          // is not refilled while its previous k-block is still being converted.
-          if (lane == 0) mbar_arrive(recready_bar(it & (kRecSlots - 1)));
-          if (it >= kRecSlots - kLook) {
-            if (!mbar_wait(adone_bar(a.idx), a.phase, abort_flag, P.status)) break;
+          // keep a ring slot from being refilled while its previous k-block is still being converted:
+          // records(it+3) reuse the slot of k-block it-5
+          if (it >= 5) {
+            if (!mbar_wait(adone_bar(a.idx), a.phase, abort_flag, P.status)) return false;
             a.advance(kAS);
           }
-          issue_bounds();
-          issue_records();
-          cp_async_commit();
-        } else {
-          issue_bounds();
-          issue_records();
-          cp_async_commit();
+        }
+        const int rec_it = cr.it;
+        store_set(L);                                      // {bounds(it+6), records(it+3)}
+        __syncwarp();
+        if constexpr (kDequant) {
+          if (lane == 0 && rec_it < my_iters) mbar_arrive(recready_bar(rec_it & (kRecSlots - 1)));
+        }
+        {                                                  // {bounds(it+8), records(it+5)}
+          Cursor sb = cb, sr = cr;
+          step(cb);
+          step(cr);
+          load_set(L);
+          cb = sb;
+          cr = sr;
+        }
+        if constexpr (!kDequant) {
+          // dense bf16 weight tile (written by TMA): add the records of k-block `it` here
           const int32_t e0 = bound_ring[it & (kBoundSlots - 1)][0], e1 = bound_ring[it & (kBoundSlots - 1)][1];
-          if (!mbar_wait(xfull_bar(x.idx), x.phase, abort_flag, P.status, 0)) break;
+          if (!mbar_wait(xfull_bar(x.idx), x.phase, abort_flag, P.status, 0)) return false;
           unsigned char* A = tiles_ptr + a_off(x.idx, x.idx);
           for (int32_t j = lane; j < e1 - e0; j += 32) {
             const uint2 rec = (j < kRecCap) ? rec_ring[it & (kRecSlots - 1)][j] : __ldg(P.Sb + e0 + j);
@@ -280,8 +325,12 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
           if (lane == 0) mbar_arrive(aready_bar(x.idx));
           x.advance(kXS);
         }
+        return true;
+      };
+      for (int it = 0; it < my_iters; it += 2) {
+        if (!iteration(it, set0)) break;
+        if (it + 1 < my_iters && !iteration(it + 1, set1)) break;
       }
-      cp_async_wait_all();
     }
   } else if (warp >= kDeqWarp0 && warp < kDeqWarp0 + kNumDeqWarps) {
     // ---------------------------------------------------------------- conversion warps
@@ -312,6 +361,15 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
           w[i] = *reinterpret_cast<const uint32_t*>(C + r * 32 + chunk * 4);
           zs[i] = SZ[r];
         }
+        // the bucket's sparse records (usually fewer than 32): one per lane, fetched before the conversion
+        int32_t e0 = 0, e1 = 0;
+        uint2 rec = make_uint2(0xFFFFFFFFu, 0u);
+        if (sparse) {
+          if (!mbar_wait(recready_bar(it & (kRecSlots - 1)), static_cast<uint32_t>((it / kRecSlots) & 1), abort_flag, P.status)) break;
+          e0 = bound_ring[it & (kBoundSlots - 1)][0];
+          e1 = bound_ring[it & (kBoundSlots - 1)][1];
+          if (lane < e1 - e0) rec = rec_ring[it & (kRecSlots - 1)][lane];
+        }
         if (!mbar_wait(aempty_bar(a.idx), a.phase ^ 1u, abort_flag, P.status)) break;
 #pragma unroll
         for (int i = 0; i < kPasses; ++i) {
@@ -319,19 +377,19 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
           const uint4 v = dequant_word<kFast>(w[i], zs[i]);
           *reinterpret_cast<uint4*>(A + r * 128 + ((chunk ^ (r & 7)) << 4)) = v;
         }
-        if (sparse) {
+        if (e1 > e0) {
           // SparseAdd: add the bucket's fp32 values to this warp's rows of the bf16 tile
-          if (!mbar_wait(recready_bar(it & (kRecSlots - 1)), static_cast<uint32_t>((it / kRecSlots) & 1), abort_flag, P.status)) break;
           __syncwarp();
-          const int32_t e0 = bound_ring[it & (kBoundSlots - 1)][0], e1 = bound_ring[it & (kBoundSlots - 1)][1];
-          for (int32_t j = lane; j < e1 - e0; j += 32) {
-            const uint2 rec = (j < kRecCap) ? rec_ring[it & (kRecSlots - 1)][j] : __ldg(P.Sb + e0 + j);
-            const int r = static_cast<int>(rec.x >> 6), col = static_cast<int>(rec.x & 63);
+          auto apply = [&](uint2 rc) {
+            const int r = static_cast<int>(rc.x >> 6), col = static_cast<int>(rc.x & 63);
             if (r / kRowsPerWarp == wq) {
               __nv_bfloat16* el = reinterpret_cast<__nv_bfloat16*>(A + r * 128 + (((col >> 3) ^ (r & 7)) << 4) + (col & 7) * 2);
-              *el = __float2bfloat16_rn(__bfloat162float(*el) + __uint_as_float(rec.y));
+              *el = __float2bfloat16_rn(__bfloat162float(*el) + __uint_as_float(rc.y));
             }
-          }
+          };
+          if (lane < e1 - e0) apply(rec);
+          for (int32_t j = lane + 32; j < e1 - e0; j += 32)
+            apply((j < kRecCap) ? rec_ring[it & (kRecSlots - 1)][j] : __ldg(P.Sb + e0 + j));
         }
         fence_async_smem();
         __syncwarp();
