@@ -56,7 +56,7 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
   constexpr uint32_t kXBase = 0, kCBase = kXS * kXStageBytes, kABase = kCBase + (kDequant ? kCS * kCStageBytes : 0);
 
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[2 * kXS + 2 * kCS + 3 * kAS + 4 + kRecSlots];
+  __shared__ __align__(8) unsigned long long bars[2 * kXS + 2 * kCS + 3 * kAS + 4 + 2 * kRecSlots];
   __shared__ __align__(16) uint2 rec_ring[kRecSlots][kRecCap];      // sparse records, per k-block
   __shared__ __align__(8) int32_t bound_ring[kBoundSlots][2];
   __shared__ uint32_t tmem_base_slot;
@@ -77,6 +77,7 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
   auto accfull_bar = [&](int a) { return smem_u32(&bars[2 * kXS + 2 * kCS + 3 * kAS + a]); };
   auto accempty_bar = [&](int a) { return smem_u32(&bars[2 * kXS + 2 * kCS + 3 * kAS + 2 + a]); };
   auto recready_bar = [&](int r) { return smem_u32(&bars[2 * kXS + 2 * kCS + 3 * kAS + 4 + r]); };  // records of a k-block landed
+  auto recfree_bar = [&](int r) { return smem_u32(&bars[2 * kXS + 2 * kCS + 3 * kAS + 4 + kRecSlots + r]); };  // ... and consumed
   auto b_off = [&](int s) { return kXBase + static_cast<uint32_t>(s) * kXStageBytes; };
   auto c_off = [&](int c) { return kCBase + static_cast<uint32_t>(c) * kCStageBytes; };
   auto a_off = [&](int s, int t) {     // weight tile of iteration (X stage s, A slot t)
@@ -103,7 +104,10 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
       mbar_init(accfull_bar(a), 1);
       mbar_init(accempty_bar(a), 4);
     }
-    for (int r = 0; r < kRecSlots; ++r) mbar_init(recready_bar(r), 1);
+    for (int r = 0; r < kRecSlots; ++r) {
+      mbar_init(recready_bar(r), 1);
+      mbar_init(recfree_bar(r), kWarpsPerGroup);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), kTmemCols);
@@ -284,15 +288,16 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
         cb = sb;
         cr = sr;
       }
-      RingPos x{0, 0}, a{0, 0};
+      RingPos x{0, 0};
       // one iteration, on the register set that was loaded two iterations ago
       auto iteration = [&](int it, Loaded& L) -> bool {
         if constexpr (kDequant) {
-          // keep a ring slot from being refilled while its previous k-block is still being converted:
-          // records(it+3) reuse the slot of k-block it-5
+          // records(it+3) reuse the ring slot of k-block it-5: wait until its conversion warps have
+          // read it (that slot's previous phase, so the parity wait cannot alias)
           if (it >= 5) {
-            if (!mbar_wait(adone_bar(a.idx), a.phase, abort_flag, P.status)) return false;
-            a.advance(kAS);
+            const int prev = it - 5;
+            if (!mbar_wait(recfree_bar(prev & (kRecSlots - 1)), static_cast<uint32_t>((prev / kRecSlots) & 1), abort_flag, P.status))
+              return false;
           }
         }
         const int rec_it = cr.it;
@@ -396,6 +401,7 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
         if (lane == 0) {
           mbar_arrive(adone_bar(a.idx));
           mbar_arrive(cempty_bar(c.idx));
+          if (sparse) mbar_arrive(recfree_bar(it & (kRecSlots - 1)));
         }
 #pragma unroll
         for (int j = 0; j < kGroups; ++j) {
