@@ -97,7 +97,7 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
     }
     for (int t = 0; t < kAS; ++t) {
       mbar_init(adone_bar(t), kWarpsPerGroup);
-      mbar_init(aready_bar(t), 1);
+      mbar_init(aready_bar(t), kWarpsPerGroup);
       mbar_init(aempty_bar(t), 1);
     }
     for (int a = 0; a < 2; ++a) {
@@ -204,8 +204,8 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
     // Brings the bucket bounds and the sparse records (position in tile, fp32 value) of every
     // (tile, k-block) into two small rings in shared memory, a few k-blocks ahead of their use.
     // Plain global loads into registers, stored to shared memory two iterations later (two register
-    // sets in flight), so that no load latency sits on this warp's loop.  In dequantising mode the
-    // conversion warps add the values to the weight tile; for a dense bf16 weight this warp does.
+    // sets in flight), so that no load latency sits on this warp's loop.  Warps 4-11 add the values to
+    // the weight tile (after converting it, or after TMA delivered a dense bf16 tile).
     //   iteration it:  store {bounds(it+6), records(it+3)} loaded at it-2, signal recready(it+3),
     //                  load  {bounds(it+8), records(it+5)}    (records(it+5) are addressed by
     //                  bounds(it+5), stored at it-1)
@@ -226,7 +226,7 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
       };
       struct Loaded {
         int32_t bound;               // lanes 0,1: bucket_ptr[b], bucket_ptr[b+1]
-        uint2 rec[2];                // records lane and lane + 32 of the bucket
+        uint2 rec[kRecCap / 32];     // records lane, lane + 32, ... of the bucket
         int32_t n;                   // records of the bucket held in the ring (<= kRecCap)
       };
       Cursor cb = make_cursor(), cr = make_cursor();       // bounds stream, records stream
@@ -239,8 +239,9 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
         if (cr.it < my_iters) {
           const int32_t e0 = bound_ring[cr.it & (kBoundSlots - 1)][0], e1 = bound_ring[cr.it & (kBoundSlots - 1)][1];
           L.n = (e1 - e0 < kRecCap) ? e1 - e0 : kRecCap;
-          if (lane < L.n) L.rec[0] = __ldg(P.Sb + e0 + lane);
-          if (lane + 32 < L.n) L.rec[1] = __ldg(P.Sb + e0 + lane + 32);
+#pragma unroll
+          for (int q = 0; q < kRecCap / 32; ++q)
+            if (lane + 32 * q < L.n) L.rec[q] = __ldg(P.Sb + e0 + lane + 32 * q);
         }
       };
       auto store_set = [&](const Loaded& L) {              // then advance both streams
@@ -249,12 +250,13 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
           step(cb);
         }
         if (cr.it < my_iters) {
-          if (lane < L.n) rec_ring[cr.it & (kRecSlots - 1)][lane] = L.rec[0];
-          if (lane + 32 < L.n) rec_ring[cr.it & (kRecSlots - 1)][lane + 32] = L.rec[1];
+#pragma unroll
+          for (int q = 0; q < kRecCap / 32; ++q)
+            if (lane + 32 * q < L.n) rec_ring[cr.it & (kRecSlots - 1)][lane + 32 * q] = L.rec[q];
           step(cr);
         }
       };
-      static_assert(kRecCap == 64 && kRecSlots == 8 && kBoundSlots == 16, "ring sizes are part of the schedule");
+      static_assert(kRecSlots == 8 && kBoundSlots == 16, "ring sizes are part of the schedule");
       // prologue: bounds 0..5 and records 0..2 directly, then prime the two register sets
       Loaded set0, set1;
       for (int j = 0; j < 6; ++j) {                        // bounds only (the records stream idles)
@@ -274,7 +276,7 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
           const int32_t n = (e1 - e0 < kRecCap) ? e1 - e0 : kRecCap;
           for (int32_t q = lane; q < n; q += 32) rec_ring[cr.it & (kRecSlots - 1)][q] = __ldg(P.Sb + e0 + q);
           __syncwarp();
-          if (kDequant && lane == 0) mbar_arrive(recready_bar(cr.it & (kRecSlots - 1)));
+          if (lane == 0) mbar_arrive(recready_bar(cr.it & (kRecSlots - 1)));
           step(cr);
         }
       }
@@ -288,24 +290,19 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
         cb = sb;
         cr = sr;
       }
-      RingPos x{0, 0};
       // one iteration, on the register set that was loaded two iterations ago
       auto iteration = [&](int it, Loaded& L) -> bool {
-        if constexpr (kDequant) {
-          // records(it+3) reuse the ring slot of k-block it-5: wait until its conversion warps have
-          // read it (that slot's previous phase, so the parity wait cannot alias)
-          if (it >= 5) {
-            const int prev = it - 5;
-            if (!mbar_wait(recfree_bar(prev & (kRecSlots - 1)), static_cast<uint32_t>((prev / kRecSlots) & 1), abort_flag, P.status))
-              return false;
-          }
+        // records(it+3) reuse the ring slot of k-block it-5: wait until the warps that add them have
+        // read it (that slot's previous phase, so the parity wait cannot alias)
+        if (it >= 5) {
+          const int prev = it - 5;
+          if (!mbar_wait(recfree_bar(prev & (kRecSlots - 1)), static_cast<uint32_t>((prev / kRecSlots) & 1), abort_flag, P.status))
+            return false;
         }
         const int rec_it = cr.it;
         store_set(L);                                      // {bounds(it+6), records(it+3)}
         __syncwarp();
-        if constexpr (kDequant) {
-          if (lane == 0 && rec_it < my_iters) mbar_arrive(recready_bar(rec_it & (kRecSlots - 1)));
-        }
+        if (lane == 0 && rec_it < my_iters) mbar_arrive(recready_bar(rec_it & (kRecSlots - 1)));
         {                                                  // {bounds(it+8), records(it+5)}
           Cursor sb = cb, sr = cr;
           step(cb);
@@ -313,22 +310,6 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
           load_set(L);
           cb = sb;
           cr = sr;
-        }
-        if constexpr (!kDequant) {
-          // dense bf16 weight tile (written by TMA): add the records of k-block `it` here
-          const int32_t e0 = bound_ring[it & (kBoundSlots - 1)][0], e1 = bound_ring[it & (kBoundSlots - 1)][1];
-          if (!mbar_wait(xfull_bar(x.idx), x.phase, abort_flag, P.status, 0)) return false;
-          unsigned char* A = tiles_ptr + a_off(x.idx, x.idx);
-          for (int32_t j = lane; j < e1 - e0; j += 32) {
-            const uint2 rec = (j < kRecCap) ? rec_ring[it & (kRecSlots - 1)][j] : __ldg(P.Sb + e0 + j);
-            const int r = static_cast<int>(rec.x >> 6), c = static_cast<int>(rec.x & 63);
-            __nv_bfloat16* el = reinterpret_cast<__nv_bfloat16*>(A + r * 128 + (((c >> 3) ^ (r & 7)) << 4) + (c & 7) * 2);
-            *el = __float2bfloat16_rn(__bfloat162float(*el) + __uint_as_float(rec.y));
-          }
-          fence_async_smem();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(aready_bar(x.idx));
-          x.advance(kXS);
         }
         return true;
       };
@@ -408,6 +389,36 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
           c.advance(kCS);
           a.advance(kAS);
         }
+      }
+    } else if (sparse) {
+      // dense bf16 weight tile delivered by TMA: the same warps add the bucket's sparse values
+      const int dw = warp - kDeqWarp0;
+      const int gq = dw / kWarpsPerGroup, wq = dw % kWarpsPerGroup;
+      constexpr int kRowsPerWarp = kBM / kWarpsPerGroup;
+      RingPos x{0, 0};
+      for (int j = 0; j < gq; ++j) x.advance(kXS);
+      const int my_iters = my_tiles * nkb;
+      for (int it = gq; it < my_iters; it += kGroups) {
+        if (!mbar_wait(recready_bar(it & (kRecSlots - 1)), static_cast<uint32_t>((it / kRecSlots) & 1), abort_flag, P.status)) break;
+        const int32_t e0 = bound_ring[it & (kBoundSlots - 1)][0], e1 = bound_ring[it & (kBoundSlots - 1)][1];
+        if (!mbar_wait(xfull_bar(x.idx), x.phase, abort_flag, P.status)) break;
+        unsigned char* A = tiles_ptr + a_off(x.idx, x.idx);
+        for (int32_t j = lane; j < e1 - e0; j += 32) {
+          const uint2 rc = (j < kRecCap) ? rec_ring[it & (kRecSlots - 1)][j] : __ldg(P.Sb + e0 + j);
+          const int r = static_cast<int>(rc.x >> 6), col = static_cast<int>(rc.x & 63);
+          if (r / kRowsPerWarp == wq) {
+            __nv_bfloat16* el = reinterpret_cast<__nv_bfloat16*>(A + r * 128 + (((col >> 3) ^ (r & 7)) << 4) + (col & 7) * 2);
+            *el = __float2bfloat16_rn(__bfloat162float(*el) + __uint_as_float(rc.y));
+          }
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(aready_bar(x.idx));
+          mbar_arrive(recfree_bar(it & (kRecSlots - 1)));
+        }
+#pragma unroll
+        for (int j = 0; j < kGroups; ++j) x.advance(kXS);
       }
     }
   } else if (warp >= kEpiWarp0) {

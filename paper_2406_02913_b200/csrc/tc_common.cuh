@@ -19,7 +19,7 @@ constexpr int kATileBytes = kBM * kBK * 2;   // 16 KiB
 constexpr int kCodesBytes = kBM * kBK / 2;   // 4 KiB of packed codes per stage
 constexpr int kSzBytes = 2048;               // (scale, zero) fp32 pairs: 128 rows x up to 2 groups
 constexpr int kLook = 4;                     // SparseAdd look-ahead in k-blocks
-constexpr int kRecSlots = 8, kRecCap = 64;   // ring of per-k-block sparse records in shared memory
+constexpr int kRecSlots = 8, kRecCap = 128;  // ring of per-k-block sparse records in shared memory
 constexpr int kBoundSlots = 16;
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s of SM cycles
 
