@@ -46,6 +46,23 @@ __device__ __forceinline__ void load_tile(__nv_bfloat16* dst, const __nv_bfloat1
   }
 }
 
+// Same copy with cp.async (16 bytes per request, bypassing L1), for the double-buffered K/V tiles.
+template <int HD>
+__device__ __forceinline__ void load_tile_async(__nv_bfloat16* dst, const __nv_bfloat16* src, int64_t ld, int valid) {
+  constexpr int kChunks = HD / 8;
+  for (int i = threadIdx.x; i < 64 * kChunks; i += 128) {
+    const int r = i / kChunks, c = i % kChunks;
+    __nv_bfloat16* d = dst + r * (HD + 8) + c * 8;
+    if (r < valid) {
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(d))),
+                   "l"(src + r * ld + c * 8)
+                   : "memory");
+    } else {
+      *reinterpret_cast<uint4*>(d) = make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
+}
+
 template <int HD>
 __global__ void __launch_bounds__(128)
 flash_attn_bf16_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
@@ -54,10 +71,10 @@ flash_attn_bf16_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16*
   constexpr int LDS = HD + 8;
   extern __shared__ __align__(16) unsigned char smem_attn[];
   __nv_bfloat16* sQ = reinterpret_cast<__nv_bfloat16*>(smem_attn);
-  __nv_bfloat16* sK = sQ + kQT * LDS;
-  __nv_bfloat16* sV = sK + kKT * LDS;
+  __nv_bfloat16* sKV = sQ + kQT * LDS;          // two stages of (K tile, V tile)
 
-  const int qt = blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
+  // heavy query tiles (many key tiles) are scheduled first
+  const int qt = gridDim.x - 1 - blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
   const int hk = hq / (H / Hkv);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
@@ -82,13 +99,27 @@ flash_attn_bf16_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16*
   float mrow[2] = {-INFINITY, -INFINITY}, lrow[2] = {0.f, 0.f};
   const int row_a = q0 + warp * 16 + g, row_b = row_a + 8;     // the two query rows of this thread
 
+  auto issue_kv = [&](int kt) {                 // K and V tile kt into stage kt & 1
+    const int k0 = kt * kKT;
+    const int valid = S - k0 < kKT ? S - k0 : kKT;
+    __nv_bfloat16* dK = sKV + (kt & 1) * 2 * kKT * LDS;
+    load_tile_async<HD>(dK, k + (static_cast<int64_t>(b) * S + k0) * ldk + hk * HD, ldk, valid);
+    load_tile_async<HD>(dK + kKT * LDS, v + (static_cast<int64_t>(b) * S + k0) * ldk + hk * HD, ldk, valid);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  issue_kv(0);
   for (int kt = 0; kt <= qt; ++kt) {
     const int k0 = kt * kKT;
     const int valid = S - k0 < kKT ? S - k0 : kKT;
-    __syncthreads();                                            // previous tile fully consumed
-    load_tile<HD>(sK, k + (static_cast<int64_t>(b) * S + k0) * ldk + hk * HD, ldk, valid);
-    load_tile<HD>(sV, v + (static_cast<int64_t>(b) * S + k0) * ldk + hk * HD, ldk, valid);
-    __syncthreads();
+    if (kt + 1 <= qt) {
+      issue_kv(kt + 1);                                         // overlaps with the math on tile kt
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    __syncthreads();                                            // tile kt is visible to every warp
+    const __nv_bfloat16* sK = sKV + (kt & 1) * 2 * kKT * LDS;
+    const __nv_bfloat16* sV = sK + kKT * LDS;
 
     // scores: 16 rows x 64 keys per warp
     float sacc[kKT / 8][4];
@@ -172,6 +203,7 @@ flash_attn_bf16_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16*
         mma_bf16(oacc[2 * dp + 1], pa[ks], b2, b3);
       }
     }
+    __syncthreads();                                            // stage kt & 1 may be refilled now
   }
   // row sums across the quad, normalise, store
 #pragma unroll
@@ -196,12 +228,18 @@ szo_status launch_flash_attention_bf16(const void* q, const void* k, const void*
   SZO_REQUIRE(hd == 64 || hd == 128, SZO_ERR_UNSUPPORTED, "head dimension must be 64 or 128");
   const float scale_log2e = 1.4426950408889634f / sqrtf(static_cast<float>(hd));
   dim3 grid(static_cast<unsigned>(ceil_div(S, kQT)), H, B);
-  const size_t smem = static_cast<size_t>(3) * 64 * (hd + 8) * 2;
+  const size_t smem = static_cast<size_t>(5) * 64 * (hd + 8) * 2;      // Q + two (K, V) stages
   auto* qb = static_cast<const __nv_bfloat16*>(q);
   auto* kb = static_cast<const __nv_bfloat16*>(k);
   auto* vb = static_cast<const __nv_bfloat16*>(v);
   auto* ob = static_cast<__nv_bfloat16*>(o);
   if (hd == 64) {
+    static bool configured64 = false;
+    if (!configured64) {
+      SZO_CHECK_CUDA(cudaFuncSetAttribute(flash_attn_bf16_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(smem)));
+      configured64 = true;
+    }
     flash_attn_bf16_kernel<64><<<grid, 128, smem, st>>>(qb, kb, vb, ob, S, H, Hkv, scale_log2e);
   } else {
     static bool configured = false;

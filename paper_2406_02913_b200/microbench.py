@@ -114,9 +114,21 @@ def sparse_case(k, reps, n_total=12_582_912_000):
     return line
 
 
+def attention_case(Bn, S, H, Hkv, hd, reps):
+    g = torch.Generator(device="cuda")
+    g.manual_seed(1)
+    q = torch.randn(Bn * S, H * hd, generator=g, device="cuda").to(torch.bfloat16)
+    k = torch.randn(Bn * S, Hkv * hd, generator=g, device="cuda").to(torch.bfloat16)
+    v = torch.randn(Bn * S, Hkv * hd, generator=g, device="cuda").to(torch.bfloat16)
+    med, best = time_call(lambda: B.szo_attention(q, k, v, Bn, S, H, Hkv, hd), reps)
+    flops = 4.0 * Bn * H * S * S * hd / 2          # causal
+    print(json.dumps({"case": "attention", "B": Bn, "S": S, "H": H, "Hkv": Hkv, "hd": hd, "ms_median": med,
+                      "tflops_causal": flops / (med * 1e-3) / 1e12}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["linear", "sparse", "sweep"])
+    ap.add_argument("what", choices=["linear", "sparse", "sweep", "attention"])
     ap.add_argument("--M", type=int, default=8192)
     ap.add_argument("--N", type=int, default=4096)
     ap.add_argument("--K", type=int, default=4096)
@@ -131,6 +143,9 @@ def main():
         linear_case(a.M, a.N, a.K, a.G, a.mode, a.rho, a.reps)
     elif a.what == "sparse":
         sparse_case(a.k, a.reps)
+    elif a.what == "attention":
+        attention_case(16, 256, 32, 32, 128, a.reps)
+        attention_case(8, 512, 32, 8, 128, a.reps)
     else:
         for M in (16, 256, 8192):
             for mode in ("sparse_add", "spmm"):
