@@ -265,7 +265,7 @@ def run_ours(args):
         "e2e": {"value": world * 1e3 * args.steps / e2e_ms, "unit": "steps/s",
                 "h2d_bytes_per_step": BATCH * SEQ * 4 + BATCH * 4 + 8, "d2h_bytes_per_step": 24},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "tensor", "kernel": "szo_linear_tc_kernel", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "tensor", "kernel": "szo_linear_tc2_kernel", "achieved": achieved, "peak": peak,
                      "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
                      "peak_source": f"{peaks['source']} (sustained cuBLAS bf16)",
                      "launches": int(lin_launches), "avg_launch_ms": lin_ms / max(lin_launches, 1),

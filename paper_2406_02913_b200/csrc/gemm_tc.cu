@@ -601,14 +601,13 @@ szo_status linear_fwd_tc(const szo_linear* p, const void* x, int64_t M, const ui
   P.status = device_status_word();
   SZO_REQUIRE(P.status != nullptr, SZO_ERR_CUDA, "no device status word");
   const CUtensorMap& mw = t->w_map;
-  // SZO_LINEAR_KERNEL=2cta selects the pair-tile kernel for M > 128 (A/B measurement); the one-CTA
-  // kernel measured faster and is the default.
-  static const int forced = [] {
+  // M > 128: pair tiles of 256 weight rows x 256 tokens on two-CTA clusters.  SZO_LINEAR_KERNEL=1cta
+  // keeps the one-CTA kernel for every M (A/B measurement).
+  static const bool force_1cta = [] {
     const char* e = getenv("SZO_LINEAR_KERNEL");
-    return (e && e[0] == '1') ? 1 : (e && e[0] == '2') ? 2 : 0;
+    return e != nullptr && e[0] == '1';
   }();
-  if (M > 128 && forced == 2) {
-    // pair tiles of 256 weight rows x 256 tokens on two-CTA clusters
+  if (M > 128 && !force_1cta) {
     SZO_TRY(make_map(&mx, x, M, p->K, 128));
     P.m_tiles = ceil_div(M, 256);
     P.n_tiles = ceil_div(p->N, 256);

@@ -1,21 +1,24 @@
 // Two-CTA (cta_group::2) version of the fused linear for M > 128 tokens.
 //
 // A cluster of two CTAs on neighbouring SMs computes one 256 (weight rows) x 256 (tokens) tile:
-// each CTA owns 128 weight rows (its half of the MMA's M dimension, dequantised and SparseAdd-ed in
+// each CTA owns 128 weight rows (its half of the MMA's M dimension: dequantised and SparseAdd-ed in
 // its own shared memory, accumulated in its own TMEM) and loads only 128 of the 256 tokens (its half
-// of the N dimension); the tensor cores of both SMs read both halves.  Against the one-CTA kernel
-// this halves the activation bytes fetched from L2 per flop and shrinks a pipeline stage, so seven
-// raw stages (token tile + codes + scale/zero strip) and three dequantised weight slots fit.
+// of the N dimension); the tensor cores of both SMs read both halves.  Against the one-CTA kernel a
+// k-block moves 16 KiB instead of 32 KiB of tokens through each SM's shared memory, which is what
+// bounds the one-CTA kernel.
 //
-//   warp 0       TMA producer (own token half, own codes / scale-zero strip, or own bf16 weight tile)
+// Roles per CTA (same rings as the one-CTA kernel: X token tiles, C codes + scale/zero, A weights):
+//   warp 0       X producer: TMA of the CTA's own token half (and its bf16 weight tile in dense mode)
+//   warp 3       C producer: bulk copies of the CTA's code tile and scale/zero strip
 //   warp 1       TMEM allocation; in the leader CTA (cluster rank 0) one thread issues the
-//                tcgen05.mma.cta_group::2 instructions and commits, multicast, to the stage and
-//                accumulator barriers of both CTAs
-//   warp 2       stage finisher: waits for the dequantised (or TMA-loaded) weight tile, adds the
-//                bucket's sparse values in shared memory (records prefetched with cp.async), fences
-//                and arrives, with cluster scope, on the leader's ready[s] barrier (2 arrivals)
-//   warps 4-11   int4 -> bf16 conversion, shared -> shared, into the swizzled K-major layout
-//   warps 12-15  epilogue of the CTA's own 128 rows x 256 tokens (tcgen05.ld, bias, store)
+//                tcgen05.mma.cta_group::2 instructions and commits, multicast, to the barriers of
+//                both CTAs
+//   warp 2       sparse-record prefetch (register-pipelined loads into a ring in shared memory)
+//   warps 4-15   weight producers (three groups of four take k-blocks in turn): int4 -> bf16 conversion and SparseAdd of the CTA's own rows; when
+//                the tile is final and the CTA's token half has landed they arrive, with cluster
+//                scope, on the leader's aready barrier (8 arrivals: one group of each CTA).  In dense
+//                mode the same warps add the sparse values to the TMA-loaded tile and relay.
+//   warps 16-19  epilogue of the CTA's own 128 rows x 256 tokens (tcgen05.ld, bias, store)
 // All waits are bounded; no TMA load uses cluster multicast.
 #include "tc_common.cuh"
 
@@ -25,9 +28,17 @@ namespace {
 
 using namespace tc;
 
-constexpr int kBT2 = 256;                    // tokens per pair tile (UMMA N)
-constexpr int kBHalfBytes = 128 * kBK * 2;   // this CTA's half of the token tile: 16 KiB
-constexpr int kARing = 3;                    // dequantised weight slots
+constexpr int kPairBT = 256;                 // tokens per pair tile (UMMA N)
+constexpr int kXHalfBytes = 128 * kBK * 2;   // this CTA's half of the token tile: 16 KiB
+constexpr int kCStages2 = 6;
+constexpr int kASlots2 = 6;
+// 20 warps: four single-thread roles, three groups of four conversion warps, four epilogue warps
+constexpr int kGroups2 = 3, kWarpsPerGroup2 = 4;
+constexpr int kNumDeqWarps2 = kGroups2 * kWarpsPerGroup2;
+constexpr int kEpiWarp02 = kDeqWarp0 + kNumDeqWarps2;
+constexpr int kNumWarps2 = kEpiWarp02 + 4;
+// sparse records: ring of per-k-block slots, filled a chunk of four k-blocks at a time
+constexpr int kRecChunk = 4, kRecChunks = 3, kRecSlots2 = kRecChunk * kRecChunks;
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
@@ -38,11 +49,14 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-// Arrive (release, cluster scope) on the barrier at the same shared-memory offset in CTA `target`.
+// Arrive on the barrier at the same shared-memory offset in CTA `target`.  The data the arrival
+// publishes sits in this CTA's shared memory and is read by the tensor cores (async proxy), for
+// which the preceding fence.proxy.async orders the writes; a cluster-scope release on top of that
+// measured about a thousand cycles per arrival.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t local_bar, uint32_t target) {
   uint32_t remote;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_bar), "r"(target));
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -55,19 +69,21 @@ __device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t
       : "memory");
   return ok;
 }
+// Bounded wait on a barrier that the peer CTA also arrives on (acquire at cluster scope).
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                                   int32_t* status) {
-  for (int i = 0; i < 256; ++i)
-    if (mbar_try_wait_cluster(bar, parity)) return true;
+  if (mbar_try_wait_cluster(bar, parity)) return true;
   const long long t0 = clock64();
+  int polls = 0;
   while (true) {
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try_wait_cluster(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitCycles) {
-      *abort_flag = 1;
-      atomicExch(status, static_cast<int32_t>(SZO_ERR_TIMEOUT));
-      return false;
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    if ((++polls & 1023) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitLimitCycles) {
+        *abort_flag = 1;
+        atomicExch(status, static_cast<int32_t>(SZO_ERR_TIMEOUT));
+        return false;
+      }
     }
   }
 }
@@ -97,59 +113,71 @@ __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
       : "memory");
 }
 
-template <int kRaw, bool kDequant, bool kFast>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumWarps * 32, 1)
+template <int kXS, bool kDequant, bool kFast>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumWarps2 * 32, 1)
 szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                       const TcParams P) {
-  constexpr int kRawBytes = kBHalfBytes + (kDequant ? kCodesBytes + kSzBytes : kATileBytes);
-  constexpr uint32_t kTmemCols = 512;
-  constexpr uint32_t kIdesc = make_idesc(256, kBT2);
+  constexpr int kXStageBytes = kXHalfBytes + (kDequant ? 0 : kATileBytes);
+  constexpr int kCStageBytes = kCodesBytes + kSzBytes;
+  constexpr int kCS = kDequant ? kCStages2 : 1;
+  constexpr int kAS = kDequant ? kASlots2 : kXS;            // dense: the weight tile lives in the X stage
+  constexpr int kGroups = kGroups2, kWarpsPerGroup = kWarpsPerGroup2;
+  constexpr uint32_t kTmemCols = 512;                       // two accumulators of 256 columns
+  constexpr uint32_t kIdesc = make_idesc(256, kPairBT);
+  constexpr uint32_t kCBase = kXS * kXStageBytes, kABase = kCBase + (kDequant ? kCS * kCStageBytes : 0);
 
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[3 * kRaw + 2 * kARing + 4];
-  __shared__ __align__(16) uint2 rec_ring[kRecSlots][kRecCap];
-  __shared__ __align__(8) int32_t bound_ring[kBoundSlots][2];
+  __shared__ __align__(8) unsigned long long bars[2 * kXS + 2 * kCS + 2 * kAS + 4 + 2 * kRecSlots2];
+  __shared__ __align__(16) uint2 rec_ring[kRecSlots2][kRecCap];
+  __shared__ __align__(8) int32_t bound_ring[kRecSlots2][2];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
 
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* tiles_ptr = smem_raw + (tiles_base - smem_u32(smem_raw));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t rank = cluster_ctarank();
+  const int rank = static_cast<int>(cluster_ctarank());
   const bool leader = rank == 0;
   volatile int* abort_flag = &abort_flag_s;
 
-  auto full_bar = [&](int s) { return smem_u32(&bars[s]); };                    // local TMA bytes landed
-  auto ready_bar = [&](int s) { return smem_u32(&bars[kRaw + s]); };            // leader: both CTAs' tiles final
-  auto empty_bar = [&](int s) { return smem_u32(&bars[2 * kRaw + s]); };        // MMAs of the raw stage retired
-  auto deq_bar = [&](int t) { return smem_u32(&bars[3 * kRaw + t]); };          // weight slot t converted
-  auto aempty_bar = [&](int t) { return smem_u32(&bars[3 * kRaw + kARing + t]); };  // weight slot t consumed
-  auto accfull_bar = [&](int a) { return smem_u32(&bars[3 * kRaw + 2 * kARing + a]); };
-  auto accempty_bar = [&](int a) { return smem_u32(&bars[3 * kRaw + 2 * kARing + 2 + a]); };  // leader
-  // shared-memory carve-up: kRaw raw stages, then (dequant mode) kARing weight slots
-  auto raw_off = [&](int s) { return static_cast<uint32_t>(s) * kRawBytes; };
-  auto b_tile = [&](int s) { return tiles_base + raw_off(s); };
-  auto c_tile = [&](int s) { return tiles_base + raw_off(s) + kBHalfBytes; };   // codes (+ sz) or bf16 weight tile
+  auto xfull_bar = [&](int s) { return smem_u32(&bars[s]); };                  // own X stage landed (TMA)
+  auto xempty_bar = [&](int s) { return smem_u32(&bars[kXS + s]); };           // its MMAs retired (commit to both)
+  auto cfull_bar = [&](int c) { return smem_u32(&bars[2 * kXS + c]); };
+  auto cempty_bar = [&](int c) { return smem_u32(&bars[2 * kXS + kCS + c]); };
+  auto aready_bar = [&](int t) { return smem_u32(&bars[2 * kXS + 2 * kCS + t]); };          // leader: both CTAs' tiles final
+  auto aempty_bar = [&](int t) { return smem_u32(&bars[2 * kXS + 2 * kCS + kAS + t]); };    // MMAs retired (commit to both)
+  auto accfull_bar = [&](int a) { return smem_u32(&bars[2 * kXS + 2 * kCS + 2 * kAS + a]); };
+  auto accempty_bar = [&](int a) { return smem_u32(&bars[2 * kXS + 2 * kCS + 2 * kAS + 2 + a]); };   // leader
+  auto recready_bar = [&](int r) { return smem_u32(&bars[2 * kXS + 2 * kCS + 2 * kAS + 4 + r]); };
+  auto recfree_bar = [&](int r) { return smem_u32(&bars[2 * kXS + 2 * kCS + 2 * kAS + 4 + kRecSlots2 + r]); };
+  auto b_off = [&](int s) { return static_cast<uint32_t>(s) * kXStageBytes; };
+  auto c_off = [&](int c) { return kCBase + static_cast<uint32_t>(c) * kCStageBytes; };
   auto a_off = [&](int s, int t) {
-    return kDequant ? static_cast<uint32_t>(kRaw) * kRawBytes + static_cast<uint32_t>(t) * kATileBytes
-                    : raw_off(s) + kBHalfBytes;
+    return kDequant ? kABase + static_cast<uint32_t>(t) * kATileBytes : b_off(s) + kXHalfBytes;
   };
 
   const bool sparse = P.Sb != nullptr;
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
-    for (int s = 0; s < kRaw; ++s) {
-      mbar_init(full_bar(s), 1);
-      mbar_init(ready_bar(s), 2);
-      mbar_init(empty_bar(s), 1);
+    for (int s = 0; s < kXS; ++s) {
+      mbar_init(xfull_bar(s), 1);
+      mbar_init(xempty_bar(s), 1);
     }
-    for (int t = 0; t < kARing; ++t) {
-      mbar_init(deq_bar(t), kNumDeqWarps);
+    for (int c = 0; c < kCS; ++c) {
+      mbar_init(cfull_bar(c), 1);
+      mbar_init(cempty_bar(c), kWarpsPerGroup);
+    }
+    for (int t = 0; t < kAS; ++t) {
+      mbar_init(aready_bar(t), 2 * kWarpsPerGroup);
       mbar_init(aempty_bar(t), 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(accfull_bar(a), 1);
       mbar_init(accempty_bar(a), 8);
+    }
+    for (int r = 0; r < kRecSlots2; ++r) {
+      mbar_init(recready_bar(r), 1);
+      mbar_init(recfree_bar(r), kWarpsPerGroup);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -160,159 +188,294 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
 
-  const int64_t pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-  const int64_t total_tiles = P.m_tiles * P.n_tiles;
-  const int64_t my_tiles = (total_tiles > pair) ? (total_tiles - pair + n_pairs - 1) / n_pairs : 0;
-  const int64_t my_iters = my_tiles * P.nkb;
-  auto tile_of = [&](int64_t it) { return pair + (it / P.nkb) * n_pairs; };
+  // pair tiles of this cluster: tile(lt) = pair + lt * n_pairs, tile = n_pair_tile * m_tiles + m_tile;
+  // this CTA's 128-row weight tile is 2 * n_pair_tile + rank
+  const int pair = static_cast<int>(blockIdx.x >> 1), n_pairs = static_cast<int>(gridDim.x >> 1);
+  const int total_tiles = static_cast<int>(P.m_tiles * P.n_tiles), m_tiles = static_cast<int>(P.m_tiles);
+  const int my_tiles = (total_tiles > pair) ? (total_tiles - pair + n_pairs - 1) / n_pairs : 0;
+  const int nkb = P.nkb;
+  const int my_iters = my_tiles * nkb;
 
   if (warp == 0) {
-    // ---------------------------------------------------------------- TMA producer
+    // ---------------------------------------------------------------- X producer (own token half)
     if (lane == 0) {
-      const int groups_kb = (kDequant && P.G < kBK) ? kBK / P.G : 1;
-      for (int64_t it = 0; it < my_iters; ++it) {
-        const int64_t tile = tile_of(it);
-        const int kb = static_cast<int>(it % P.nkb);
-        const int64_t row0 = (tile / P.m_tiles) * 256 + rank * 128;       // this CTA's weight rows
-        const int64_t tok0 = (tile % P.m_tiles) * kBT2 + rank * 128;      // this CTA's half of the tokens
-        const int s = static_cast<int>(it % kRaw);
-        const uint32_t ph = static_cast<uint32_t>((it / kRaw) & 1);
-        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, P.status)) break;
-        if constexpr (kDequant) {
-          mbar_expect_tx(full_bar(s), kBHalfBytes + kCodesBytes + groups_kb * 1024);
-          bulk_load_1d(c_tile(s), P.codes + ((row0 / kBM) * P.nkb + kb) * static_cast<int64_t>(kCodesBytes), kCodesBytes,
-                       full_bar(s));
-          const int64_t g0 = (static_cast<int64_t>(kb) * kBK) / P.G;
-          for (int g = 0; g < groups_kb; ++g)
-            bulk_load_1d(c_tile(s) + kCodesBytes + g * 1024, P.sz + (g0 + g) * P.Npad + row0, 1024, full_bar(s));
-        } else {
-          mbar_expect_tx(full_bar(s), kBHalfBytes + kATileBytes);
-          tma_load_2d(c_tile(s), &tmap_w, kb * kBK, static_cast<int>(row0), full_bar(s));
+      RingPos x{0, 0};
+      bool ok = true;
+      for (int lt = 0; lt < my_tiles && ok; ++lt) {
+        const int tile = pair + lt * n_pairs;
+        const int tok0 = (tile % m_tiles) * kPairBT + rank * 128;
+        const int row0 = ((tile / m_tiles) * 2 + rank) * kBM;
+        for (int kb = 0; kb < nkb; ++kb) {
+          if (!mbar_wait(xempty_bar(x.idx), x.phase ^ 1u, abort_flag, P.status)) { ok = false; break; }
+          mbar_expect_tx(xfull_bar(x.idx), kXStageBytes);
+          tma_load_2d(tiles_base + b_off(x.idx), &tmap_x, kb * kBK, tok0, xfull_bar(x.idx));
+          if constexpr (!kDequant) tma_load_2d(tiles_base + a_off(x.idx, 0), &tmap_w, kb * kBK, row0, xfull_bar(x.idx));
+          x.advance(kXS);
         }
-        tma_load_2d(b_tile(s), &tmap_x, kb * kBK, static_cast<int>(tok0), full_bar(s));
+      }
+    }
+  } else if (warp == 3) {
+    // ---------------------------------------------------------------- C producer (codes, scale/zero)
+    if constexpr (kDequant) {
+      if (lane == 0) {
+        // Everything the loop needs advances by addition: this is one thread, and every dependent
+        // instruction of its loop body is several cycles of the k-block period.
+        const int groups_kb = (P.G < kBK) ? kBK / P.G : 1;     // scale groups per k-block
+        const int kb_per_group = (P.G > kBK) ? P.G / kBK : 1;  // k-blocks per scale group
+        const uint32_t tx_bytes = static_cast<uint32_t>(kCodesBytes + groups_kb * 1024);
+        const int64_t sz_step = static_cast<int64_t>(groups_kb) * P.Npad;
+        int cidx = 0;
+        uint32_t cphase = 0, dst = tiles_base + kCBase;
+        bool ok = true;
+        for (int lt = 0; lt < my_tiles && ok; ++lt) {
+          const int n_tile = ((pair + lt * n_pairs) / m_tiles) * 2 + rank;
+          const uint8_t* codes = P.codes + static_cast<int64_t>(n_tile) * nkb * kCodesBytes;
+          const float2* sz = P.sz + static_cast<int64_t>(n_tile) * kBM;
+          int kbg = 0;
+          for (int kb = 0; kb < nkb; ++kb) {
+            if (!mbar_wait(cempty_bar(cidx), cphase ^ 1u, abort_flag, P.status)) { ok = false; break; }
+            const uint32_t bar = cfull_bar(cidx);
+            mbar_expect_tx(bar, tx_bytes);
+            bulk_load_1d(dst, codes, kCodesBytes, bar);
+            bulk_load_1d(dst + kCodesBytes, sz, 1024, bar);
+            for (int g = 1; g < groups_kb; ++g) bulk_load_1d(dst + kCodesBytes + g * 1024, sz + g * P.Npad, 1024, bar);
+            codes += kCodesBytes;
+            if (++kbg == kb_per_group) {
+              kbg = 0;
+              sz += sz_step;
+            }
+            dst += kCStageBytes;
+            if (++cidx == kCS) {
+              cidx = 0;
+              cphase ^= 1u;
+              dst = tiles_base + kCBase;
+            }
+          }
+        }
       }
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer (leader CTA only)
     if (leader && lane == 0) {
+      RingPos x{0, 0}, a{0, 0};
       bool ok = true;
-      for (int64_t lt = 0; lt < my_tiles && ok; ++lt) {
-        const int as = static_cast<int>(lt & 1);
+      for (int lt = 0; lt < my_tiles && ok; ++lt) {
+        const int as = lt & 1;
         const uint32_t aph = static_cast<uint32_t>((lt >> 1) & 1);
-        if (!mbar_wait_cluster(accempty_bar(as), aph ^ 1u, abort_flag, P.status)) break;
+        if (!mbar_wait(accempty_bar(as), aph ^ 1u, abort_flag, P.status, 0)) break;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kBT2);
-        for (int kb = 0; kb < P.nkb; ++kb) {
-          const int64_t it = lt * P.nkb + kb;
-          const int s = static_cast<int>(it % kRaw), t = static_cast<int>(it % kARing);
-          const uint32_t ph = static_cast<uint32_t>((it / kRaw) & 1);
-          if (!mbar_wait_cluster(ready_bar(s), ph, abort_flag, P.status)) { ok = false; break; }
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kPairBT);
+        for (int kb = 0; kb < nkb; ++kb) {
+          // both CTAs' weight tiles final and both token halves landed
+          if (!mbar_wait(aready_bar(a.idx), a.phase, abort_flag, P.status, 0)) { ok = false; break; }
           tc_fence_after();
-          const uint64_t adesc = make_desc_sw128(tiles_base + a_off(s, t)), bdesc = make_desc_sw128(b_tile(s));
+          const uint64_t adesc = make_desc_sw128(tiles_base + a_off(x.idx, a.idx));
+          const uint64_t bdesc = make_desc_sw128(tiles_base + b_off(x.idx));
 #pragma unroll
           for (int k = 0; k < kBK / kUmmaK; ++k) umma2_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc, (kb | k) ? 1u : 0u);
-          umma2_commit_both(empty_bar(s));
-          if constexpr (kDequant) umma2_commit_both(aempty_bar(t));
+          umma2_commit_both(xempty_bar(x.idx));
+          if constexpr (kDequant) umma2_commit_both(aempty_bar(a.idx));
+          x.advance(kXS);
+          a.advance(kAS);
         }
         if (ok) umma2_commit_both(accfull_bar(as));
       }
     }
   } else if (warp == 2) {
-    // ---------------------------------------------------------------- stage finisher / SparseAdd
-    if (my_iters > 0) {
-      auto bucket_of = [&](int64_t it) { return ((tile_of(it) / P.m_tiles) * 2 + rank) * P.n_kblocks + (it % P.nkb); };
-      auto has_bucket = [&](int64_t it) { return (tile_of(it) / P.m_tiles) * 2 + rank < P.n_rowtiles; };
-      auto issue_bounds = [&](int64_t it) {
-        if (sparse && it < my_iters && lane < 2) {
-          if (has_bucket(it)) cp_async_4(smem_u32(&bound_ring[it % kBoundSlots][lane]), P.bucket_ptr + bucket_of(it) + lane);
-          else bound_ring[it % kBoundSlots][lane] = 0;
-        }
-      };
-      auto issue_records = [&](int64_t it) {
-        if (sparse && it < my_iters) {
-          const int32_t e0 = bound_ring[it % kBoundSlots][0], e1 = bound_ring[it % kBoundSlots][1];
-          const int32_t n = (e1 - e0 < kRecCap) ? e1 - e0 : kRecCap;
-          for (int32_t j = lane; j < n; j += 32) cp_async_8(smem_u32(&rec_ring[it % kRecSlots][j]), P.Sb + e0 + j);
-        }
-      };
-      for (int64_t j = 0; j < 2 * kLook; ++j) issue_bounds(j);
-      cp_async_commit();
-      cp_async_wait_all();
-      __syncwarp();
-      for (int64_t j = 0; j < kLook; ++j) {
-        issue_records(j);
-        cp_async_commit();
-      }
-      for (int64_t it = 0; it < my_iters; ++it) {
-        const int s = static_cast<int>(it % kRaw), t = static_cast<int>(it % kARing);
-        const uint32_t ph = static_cast<uint32_t>((it / kRaw) & 1), pht = static_cast<uint32_t>((it / kARing) & 1);
-        // group(j) = { bounds(j + 2 kLook), records(j + kLook) }: with at most kLook - 1 groups pending,
-        // group(it - kLook) has landed, i.e. records(it) and bounds(it + kLook)
-        cp_async_wait_group<kLook - 1>();
-        __syncwarp();
-        issue_bounds(it + 2 * kLook);
-        issue_records(it + kLook);
-        cp_async_commit();
-        if (!mbar_wait(kDequant ? deq_bar(t) : full_bar(s), kDequant ? pht : ph, abort_flag, P.status)) break;
-        if (sparse) {
-          const int32_t e0 = bound_ring[it % kBoundSlots][0], e1 = bound_ring[it % kBoundSlots][1];
-          unsigned char* A = tiles_ptr + a_off(s, t);
-          for (int32_t j = lane; j < e1 - e0; j += 32) {
-            const uint2 rec = (j < kRecCap) ? rec_ring[it % kRecSlots][j] : __ldg(P.Sb + e0 + j);
-            const int r = static_cast<int>(rec.x >> 6), c = static_cast<int>(rec.x & 63);
-            __nv_bfloat16* el = reinterpret_cast<__nv_bfloat16*>(A + r * 128 + (((c >> 3) ^ (r & 7)) << 4) + (c & 7) * 2);
-            *el = __float2bfloat16_rn(__bfloat162float(*el) + __uint_as_float(rec.y));
+    // ---------------------------------------------------------------- sparse-record warp
+    // Brings the bucket bounds and the sparse records (position in tile, fp32 value) of every
+    // k-block of this CTA into a ring of per-k-block slots in shared memory, a chunk of four
+    // k-blocks per loop iteration (lane j < 4 owns the bounds of k-block it0 + j), up to three chunks
+    // ahead of their use.  The bounds of the next chunk are fetched while this chunk's records are
+    // in flight, so one global-load latency is exposed per four k-blocks.
+    if (sparse && my_tiles > 0) {
+      const int n_kblocks = static_cast<int>(P.n_kblocks);
+      const int n_rowtiles = static_cast<int>(P.n_rowtiles);
+      auto load_bounds = [&](int it0, int32_t& e0, int32_t& e1) {
+        const int itl = it0 + (lane & (kRecChunk - 1));
+        e0 = 0;
+        e1 = 0;
+        if (itl < my_iters) {
+          const int lt = itl / nkb, kb = itl - lt * nkb;
+          const int n_tile = ((pair + lt * n_pairs) / m_tiles) * 2 + rank;
+          if (n_tile < n_rowtiles) {
+            const int32_t* bp = P.bucket_ptr + static_cast<int64_t>(n_tile) * n_kblocks + kb;
+            e0 = __ldg(bp);
+            e1 = __ldg(bp + 1);
           }
-          fence_async_smem();
-          __syncwarp();
         }
-        if (lane == 0) mbar_arrive_cluster(ready_bar(s), 0);
+      };
+      int32_t e0, e1;
+      load_bounds(0, e0, e1);
+      int cs = 0;                       // chunk slot: ring slots cs * 4 .. cs * 4 + 3
+      uint32_t cphase = 0;
+      bool first_pass = true;
+      bool ok = true;
+      for (int it0 = 0; it0 < my_iters && ok; it0 += kRecChunk) {
+        int32_t ne0, ne1;
+        load_bounds(it0 + kRecChunk, ne0, ne1);
+        if (!first_pass) {              // the slots' previous k-blocks must have been consumed
+#pragma unroll
+          for (int j = 0; j < kRecChunk; ++j)
+            if (it0 + j < my_iters && !mbar_wait(recfree_bar(cs * kRecChunk + j), cphase ^ 1u, abort_flag, P.status)) ok = false;
+          if (!ok) break;
+        }
+        uint2 r[kRecChunk][kRecCap / 32];
+        int32_t n[kRecChunk];
+#pragma unroll
+        for (int j = 0; j < kRecChunk; ++j) {
+          const int32_t b0 = __shfl_sync(0xFFFFFFFFu, e0, j), b1 = __shfl_sync(0xFFFFFFFFu, e1, j);
+          n[j] = (b1 - b0 < kRecCap) ? b1 - b0 : kRecCap;
+#pragma unroll
+          for (int q = 0; q < kRecCap / 32; ++q)
+            if (lane + 32 * q < n[j]) r[j][q] = __ldg(P.Sb + b0 + lane + 32 * q);
+        }
+        if (lane < kRecChunk) {
+          bound_ring[cs * kRecChunk + lane][0] = e0;
+          bound_ring[cs * kRecChunk + lane][1] = e1;
+        }
+#pragma unroll
+        for (int j = 0; j < kRecChunk; ++j) {
+#pragma unroll
+          for (int q = 0; q < kRecCap / 32; ++q)
+            if (lane + 32 * q < n[j]) rec_ring[cs * kRecChunk + j][lane + 32 * q] = r[j][q];
+        }
+        __syncwarp();
+        if (lane < kRecChunk && it0 + lane < my_iters) mbar_arrive(recready_bar(cs * kRecChunk + lane));
+        e0 = ne0;
+        e1 = ne1;
+        if (++cs == kRecChunks) {
+          cs = 0;
+          cphase ^= 1u;
+          first_pass = false;
+        }
       }
-      cp_async_wait_all();
     }
-  } else if (warp >= kDeqWarp0 && warp < kDeqWarp0 + kNumDeqWarps) {
-    // ---------------------------------------------------------------- dequantisation warps
+  } else if (warp >= kDeqWarp0 && warp < kEpiWarp02) {
+    // ---------------------------------------------------------------- weight producers
+    const int dw = warp - kDeqWarp0;
+    const int gq = dw / kWarpsPerGroup, wq = dw % kWarpsPerGroup;
+    constexpr int kRowsPerWarp = kBM / kWarpsPerGroup;
+    auto add_record = [&](unsigned char* A, uint2 rc) {
+      const int r = static_cast<int>(rc.x >> 6), col = static_cast<int>(rc.x & 63);
+      if (r / kRowsPerWarp == wq) {
+        __nv_bfloat16* el = reinterpret_cast<__nv_bfloat16*>(A + r * 128 + (((col >> 3) ^ (r & 7)) << 4) + (col & 7) * 2);
+        *el = __float2bfloat16_rn(__bfloat162float(*el) + __uint_as_float(rc.y));
+      }
+    };
     if constexpr (kDequant) {
-      const int dw = warp - kDeqWarp0;
+      constexpr int kPasses = kRowsPerWarp / 4;
       const int sub = lane >> 3, chunk = lane & 7;
       const int gsel = (P.G < kBK) ? (chunk * 8) / P.G : 0;
-      for (int64_t it = 0; it < my_iters; ++it) {
-        const int s = static_cast<int>(it % kRaw), t = static_cast<int>(it % kARing);
-        const uint32_t ph = static_cast<uint32_t>((it / kRaw) & 1), pht = static_cast<uint32_t>((it / kARing) & 1);
-        unsigned char* A = tiles_ptr + a_off(s, t);
-        const unsigned char* C = tiles_ptr + raw_off(s) + kBHalfBytes;
+      RingPos c{0, 0}, a{0, 0}, x{0, 0}, rr{0, 0};
+      for (int j = 0; j < gq; ++j) {
+        c.advance(kCS);
+        a.advance(kAS);
+        x.advance(kXS);
+        rr.advance(kRecSlots2);
+      }
+      for (int it = gq; it < my_iters; it += kGroups) {
+        unsigned char* A = tiles_ptr + a_off(0, a.idx);
+        const unsigned char* C = tiles_ptr + c_off(c.idx);
         const float2* SZ = reinterpret_cast<const float2*>(C + kCodesBytes) + gsel * kBM;
-        if (!mbar_wait(full_bar(s), ph, abort_flag, P.status)) break;
-        if (!mbar_wait(aempty_bar(t), pht ^ 1u, abort_flag, P.status)) break;
+        if (!mbar_wait(cfull_bar(c.idx), c.phase, abort_flag, P.status)) break;
+        uint32_t w[kPasses];
+        float2 zs[kPasses];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int r = dw * 16 + i * 4 + sub;
-          const uint32_t w = *reinterpret_cast<const uint32_t*>(C + r * 32 + chunk * 4);
-          const uint4 v = dequant_word<kFast>(w, SZ[r]);
+        for (int i = 0; i < kPasses; ++i) {
+          const int r = wq * kRowsPerWarp + i * 4 + sub;
+          w[i] = *reinterpret_cast<const uint32_t*>(C + r * 32 + chunk * 4);
+          zs[i] = SZ[r];
+        }
+        int32_t e0 = 0, e1 = 0;
+        uint2 rec = make_uint2(0xFFFFFFFFu, 0u);
+        if (sparse) {
+          if (!mbar_wait(recready_bar(rr.idx), rr.phase, abort_flag, P.status)) break;
+          e0 = bound_ring[rr.idx][0];
+          e1 = bound_ring[rr.idx][1];
+          if (lane < e1 - e0) rec = rec_ring[rr.idx][lane];
+        }
+        if (!mbar_wait(aempty_bar(a.idx), a.phase ^ 1u, abort_flag, P.status)) break;
+#pragma unroll
+        for (int i = 0; i < kPasses; ++i) {
+          const int r = wq * kRowsPerWarp + i * 4 + sub;
+          const uint4 v = dequant_word<kFast>(w[i], zs[i]);
           *reinterpret_cast<uint4*>(A + r * 128 + ((chunk ^ (r & 7)) << 4)) = v;
+        }
+        if (e1 > e0) {
+          __syncwarp();
+          if (lane < e1 - e0) add_record(A, rec);
+          for (int32_t j = lane + 32; j < e1 - e0; j += 32)
+            add_record(A, (j < kRecCap) ? rec_ring[rr.idx][j] : __ldg(P.Sb + e0 + j));
         }
         fence_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(deq_bar(t));
+        // the leader's MMA of this k-block also reads this CTA's token half: it has long landed
+        if (!mbar_wait(xfull_bar(x.idx), x.phase, abort_flag, P.status)) break;
+        if (lane == 0) {
+          mbar_arrive_cluster(aready_bar(a.idx), 0);
+          mbar_arrive(cempty_bar(c.idx));
+          if (sparse) mbar_arrive(recfree_bar(rr.idx));
+        }
+#pragma unroll
+        for (int j = 0; j < kGroups; ++j) {
+          c.advance(kCS);
+          a.advance(kAS);
+          x.advance(kXS);
+          rr.advance(kRecSlots2);
+        }
+      }
+    } else {
+      // dense bf16 weight tile delivered by TMA: add the bucket's sparse values (if any) and relay
+      // "this CTA's stage is final" to the leader
+      RingPos x{0, 0}, rr{0, 0};
+      for (int j = 0; j < gq; ++j) {
+        x.advance(kXS);
+        rr.advance(kRecSlots2);
+      }
+      for (int it = gq; it < my_iters; it += kGroups) {
+        int32_t e0 = 0, e1 = 0;
+        if (sparse) {
+          if (!mbar_wait(recready_bar(rr.idx), rr.phase, abort_flag, P.status)) break;
+          e0 = bound_ring[rr.idx][0];
+          e1 = bound_ring[rr.idx][1];
+        }
+        if (!mbar_wait(xfull_bar(x.idx), x.phase, abort_flag, P.status)) break;
+        if (e1 > e0) {
+          unsigned char* A = tiles_ptr + a_off(x.idx, x.idx);
+          for (int32_t j = lane; j < e1 - e0; j += 32)
+            add_record(A, (j < kRecCap) ? rec_ring[rr.idx][j] : __ldg(P.Sb + e0 + j));
+          fence_async_smem();
+        }
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive_cluster(aready_bar(x.idx), 0);
+          if (sparse) mbar_arrive(recfree_bar(rr.idx));
+        }
+#pragma unroll
+        for (int j = 0; j < kGroups; ++j) {
+          x.advance(kXS);
+          rr.advance(kRecSlots2);
+        }
       }
     }
-  } else if (warp >= kEpiWarp0) {
+  } else if (warp >= kEpiWarp02) {
     // ---------------------------------------------------------------- epilogue (own 128 rows)
     const int qd = warp & 3;
-    for (int64_t lt = 0; lt < my_tiles; ++lt) {
-      const int64_t tile = pair + lt * n_pairs;
-      const int64_t n_tile = tile / P.m_tiles, m_tile = tile % P.m_tiles;
-      const int as = static_cast<int>(lt & 1);
+    for (int lt = 0; lt < my_tiles; ++lt) {
+      const int tile = pair + lt * n_pairs;
+      const int64_t n_tile = static_cast<int64_t>(tile / m_tiles) * 2 + rank, m_tile = tile % m_tiles;
+      const int as = lt & 1;
       const uint32_t aph = static_cast<uint32_t>((lt >> 1) & 1);
-      if (!mbar_wait(accfull_bar(as), aph, abort_flag, P.status)) break;
+      if (!mbar_wait(accfull_bar(as), aph, abort_flag, P.status, 256)) break;
       tc_fence_after();
-      const int64_t n = n_tile * 256 + rank * 128 + qd * 32 + lane;
+      const int64_t n = n_tile * kBM + qd * 32 + lane;
       const float bias = (P.bias != nullptr && n < P.N) ? P.bias[n] : 0.f;
-      const int64_t m0 = m_tile * kBT2;
-      const int mlimit = static_cast<int>((P.M - m0 < kBT2) ? P.M - m0 : kBT2);
-      for (int c0 = 0; c0 < kBT2; c0 += 32) {
+      const int64_t m0 = m_tile * kPairBT;
+      const int mlimit = static_cast<int>((P.M - m0 < kPairBT) ? P.M - m0 : kPairBT);
+      for (int c0 = 0; c0 < kPairBT; c0 += 32) {
         uint32_t v[32];
-        tmem_ld32(tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + static_cast<uint32_t>(as * kBT2 + c0), v);
+        tmem_ld32(tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + static_cast<uint32_t>(as * kPairBT + c0), v);
         if (n < P.N && c0 < mlimit) {
           const int cnt = mlimit - c0;
           if (P.y_f32) {
@@ -349,11 +512,11 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
   if (warp == 1) tmem_dealloc2(tmem_base, kTmemCols);
 }
 
-template <int kRaw, bool kDequant, bool kFast>
+template <int kXS, bool kDequant, bool kFast>
 szo_status launch_tc2(const CUtensorMap& mx, const CUtensorMap& mw, const TcParams& P, int sms, cudaStream_t st) {
-  constexpr size_t raw = kBHalfBytes + (kDequant ? kCodesBytes + kSzBytes : kATileBytes);
-  constexpr size_t smem = kRaw * raw + (kDequant ? kARing * kATileBytes : 0) + 1024;
-  auto kern = szo_linear_tc2_kernel<kRaw, kDequant, kFast>;
+  constexpr size_t smem = static_cast<size_t>(kXS) * (kXHalfBytes + (kDequant ? 0 : kATileBytes)) +
+                          (kDequant ? kCStages2 * (kCodesBytes + kSzBytes) + kASlots2 * kATileBytes : 0) + 1024;
+  auto kern = szo_linear_tc2_kernel<kXS, kDequant, kFast>;
   static bool configured = false;
   if (!configured) {
     SZO_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
@@ -362,7 +525,7 @@ szo_status launch_tc2(const CUtensorMap& mx, const CUtensorMap& mw, const TcPara
   const int64_t tiles = P.m_tiles * P.n_tiles;
   const int64_t max_pairs = sms / 2;
   const unsigned grid = static_cast<unsigned>(2 * (tiles < max_pairs ? tiles : max_pairs));
-  kern<<<grid, kNumWarps * 32, smem, st>>>(mx, mw, P);
+  kern<<<grid, kNumWarps2 * 32, smem, st>>>(mx, mw, P);
   count_launch();
   SZO_CHECK_LAUNCH("szo_linear_tc2_kernel");
   return SZO_OK;
@@ -374,8 +537,8 @@ szo_status launch_tc2(const CUtensorMap& mx, const CUtensorMap& mw, const TcPara
 szo_status linear_fwd_tc2(const szo_linear* p, const CUtensorMap& mx, const CUtensorMap& mw, const tc::TcParams& P,
                           int sms, cudaStream_t st) {
   if (p->G == 0) return launch_tc2<6, false, false>(mx, mw, P, sms, st);
-  if (p->sz_dtype == SZO_BF16) return launch_tc2<7, true, true>(mx, mw, P, sms, st);
-  return launch_tc2<7, true, false>(mx, mw, P, sms, st);
+  if (p->sz_dtype == SZO_BF16) return launch_tc2<5, true, true>(mx, mw, P, sms, st);
+  return launch_tc2<5, true, false>(mx, mw, P, sms, st);
 }
 
 }  // namespace szo
