@@ -19,6 +19,10 @@
 //                scope, on the leader's aready barrier (8 arrivals: one group of each CTA).  In dense
 //                mode the same warps add the sparse values to the TMA-loaded tile and relay.
 //   warps 16-19  epilogue of the CTA's own 128 rows x 256 tokens (tcgen05.ld, bias, store)
+// Work units: a launch covers up to three weight matrices that share the activations (their pair
+// tiles are numbered consecutively), and the last, partial round of tiles is split along K into
+// up to four parts so that every cluster stays busy; the parts of a tile meet in an fp32 workspace
+// and the last one to finish adds them in part order (deterministic) and stores y.
 // All waits are bounded; no TMA load uses cluster multicast.
 #include "tc_common.cuh"
 
@@ -113,6 +117,123 @@ __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
       : "memory");
 }
 
+// One work unit of a cluster: k-blocks [kb0, kb1) of the pair tile (matrix s, this CTA's 128-row
+// tile n_tile of that matrix, token tile m_tile).
+struct Unit {
+  int s, n_tile, m_tile, kb0, kb1, part, parts, slot;
+};
+__device__ __forceinline__ int tail_kb_at(const TcParams& P, int i) {
+  return i == 0 ? P.tail_kb[0] : i == 1 ? P.tail_kb[1] : i == 2 ? P.tail_kb[2] : i == 3 ? P.tail_kb[3] : P.tail_kb[4];
+}
+__device__ __forceinline__ Unit decode_unit(const TcParams& P, int pair, int n_pairs, int rank, int lt) {
+  Unit u;
+  int tile;
+  if (lt < P.full_rounds) {
+    tile = lt * n_pairs + pair;
+    u.kb0 = 0;
+    u.kb1 = P.nkb;
+    u.part = 0;
+    u.parts = 1;
+    u.slot = 0;
+  } else {
+    u.part = pair / P.tail_tiles;
+    u.slot = pair - u.part * P.tail_tiles;
+    u.parts = P.tail_parts;
+    tile = P.full_rounds * n_pairs + u.slot;
+    u.kb0 = tail_kb_at(P, u.part);
+    u.kb1 = tail_kb_at(P, u.part + 1);
+  }
+  const int m_tiles = static_cast<int>(P.m_tiles);
+  int np = tile / m_tiles;
+  u.m_tile = tile - np * m_tiles;
+  u.s = 0;
+  if (P.nsub > 1 && np >= P.sub[0].n_tiles) {
+    np -= P.sub[0].n_tiles;
+    u.s = 1;
+    if (P.nsub > 2 && np >= P.sub[1].n_tiles) {
+      np -= P.sub[1].n_tiles;
+      u.s = 2;
+    }
+  }
+  u.n_tile = np * 2 + rank;
+  return u;
+}
+// Fields of matrix s, selected without indexing the parameter block dynamically.
+#define SZO_SUB(P, s, f) ((s) == 0 ? (P).sub[0].f : ((s) == 1 ? (P).sub[1].f : (P).sub[2].f))
+
+// Sum of the K-split parts of one CTA's 128 rows x 256 tokens, + bias, stored to y; run by every
+// thread of the CTA after its roles have finished.  A part is [token][128 rows] fp32, parts are
+// 2 * 256 * 128 floats apart; the sum runs in part order, so the result does not depend on which
+// part finished last.  Thread -> one float4 (4 rows of one token) per step of nthreads, seven in
+// flight per part.  Kept out of line: its registers would otherwise add to every role's.
+__device__ __noinline__ void reduce_parts(const float* part0, int parts, int64_t n0, int64_t N, const float* bias_p,
+                                          void* y, int y_f32, int64_t m0, int mlimit, int tid, int nthreads) {
+  constexpr int64_t kPartFloats = static_cast<int64_t>(kPairBT) * kBM;
+  constexpr int kBatch = 7;
+  const int total = mlimit * (kBM / 4);          // float4s of the valid tokens
+  for (int base = tid; base < total; base += nthreads * kBatch) {
+    float4 acc[kBatch];
+#pragma unroll
+    for (int i = 0; i < kBatch; ++i) {
+      const int f = base + i * nthreads;
+      if (f < total) acc[i] = __ldcg(reinterpret_cast<const float4*>(part0) + f);
+    }
+    for (int q = 1; q < parts; ++q) {
+      const float4* pq = reinterpret_cast<const float4*>(part0 + q * 2 * kPartFloats);
+      float4 tt[kBatch];
+#pragma unroll
+      for (int i = 0; i < kBatch; ++i) {
+        const int f = base + i * nthreads;
+        if (f < total) tt[i] = __ldcg(pq + f);
+      }
+#pragma unroll
+      for (int i = 0; i < kBatch; ++i) {
+        acc[i].x += tt[i].x;
+        acc[i].y += tt[i].y;
+        acc[i].z += tt[i].z;
+        acc[i].w += tt[i].w;
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < kBatch; ++i) {
+      const int f = base + i * nthreads;
+      if (f >= total) continue;
+      const int mm = f >> 5;
+      const int64_t n4 = n0 + ((f & 31) << 2);
+      if (n4 >= N) continue;
+      float o[4] = {acc[i].x, acc[i].y, acc[i].z, acc[i].w};
+      if (bias_p != nullptr) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (n4 + e < N) o[e] += __ldg(bias_p + n4 + e);
+      }
+      const bool vec_ok = (N % 4 == 0) && (n4 + 3 < N);
+      const int64_t off = (m0 + mm) * N + n4;
+      if (y_f32) {
+        float* yp = static_cast<float*>(y) + off;
+        if (vec_ok) {
+          *reinterpret_cast<float4*>(yp) = make_float4(o[0], o[1], o[2], o[3]);
+        } else {
+          for (int e = 0; e < 4; ++e)
+            if (n4 + e < N) yp[e] = o[e];
+        }
+      } else {
+        __nv_bfloat16* yp = static_cast<__nv_bfloat16*>(y) + off;
+        if (vec_ok) {
+          const __nv_bfloat162 lo = __floats2bfloat162_rn(o[0], o[1]), hi = __floats2bfloat162_rn(o[2], o[3]);
+          uint2 pk;
+          pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+          pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+          *reinterpret_cast<uint2*>(yp) = pk;
+        } else {
+          for (int e = 0; e < 4; ++e)
+            if (n4 + e < N) yp[e] = __float2bfloat16_rn(o[e]);
+        }
+      }
+    }
+  }
+}
+
 template <int kXS, bool kDequant, bool kFast>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumWarps2 * 32, 1)
 szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
@@ -129,9 +250,10 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) unsigned long long bars[2 * kXS + 2 * kCS + 2 * kAS + 4 + 2 * kRecSlots2];
   __shared__ __align__(16) uint2 rec_ring[kRecSlots2][kRecCap];
-  __shared__ __align__(8) int32_t bound_ring[kRecSlots2][2];
+  __shared__ __align__(16) int32_t bound_ring[kRecSlots2][4];   // e0, e1, matrix index
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
+  __shared__ int epi_count_s, reduce_flag_s;   // K-split tail: epilogue warps done, this CTA sums the parts
 
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* tiles_ptr = smem_raw + (tiles_base - smem_u32(smem_raw));
@@ -156,9 +278,11 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     return kDequant ? kABase + static_cast<uint32_t>(t) * kATileBytes : b_off(s) + kXHalfBytes;
   };
 
-  const bool sparse = P.Sb != nullptr;
+  const bool sparse = P.sub[0].Sb != nullptr || (P.nsub > 1 && P.sub[1].Sb != nullptr) || (P.nsub > 2 && P.sub[2].Sb != nullptr);
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
+    epi_count_s = 0;
+    reduce_flag_s = 0;
     for (int s = 0; s < kXS; ++s) {
       mbar_init(xfull_bar(s), 1);
       mbar_init(xempty_bar(s), 1);
@@ -188,24 +312,26 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
 
-  // pair tiles of this cluster: tile(lt) = pair + lt * n_pairs, tile = n_pair_tile * m_tiles + m_tile;
-  // this CTA's 128-row weight tile is 2 * n_pair_tile + rank
+  // work units of this cluster (see TcParams): full tiles first, then at most one unit of the tail
   const int pair = static_cast<int>(blockIdx.x >> 1), n_pairs = static_cast<int>(gridDim.x >> 1);
-  const int total_tiles = static_cast<int>(P.m_tiles * P.n_tiles), m_tiles = static_cast<int>(P.m_tiles);
-  const int my_tiles = (total_tiles > pair) ? (total_tiles - pair + n_pairs - 1) / n_pairs : 0;
   const int nkb = P.nkb;
-  const int my_iters = my_tiles * nkb;
+  const bool has_tail = pair < P.tail_tiles * P.tail_parts;
+  const int my_units = P.full_rounds + (has_tail ? 1 : 0);
+  const int full_iters = P.full_rounds * nkb;
+  const int tail_part = has_tail ? pair / P.tail_tiles : 0;
+  const int tail_kb0 = has_tail ? tail_kb_at(P, tail_part) : 0;
+  const int my_iters = full_iters + (has_tail ? tail_kb_at(P, tail_part + 1) - tail_kb0 : 0);
 
   if (warp == 0) {
     // ---------------------------------------------------------------- X producer (own token half)
     if (lane == 0) {
       RingPos x{0, 0};
       bool ok = true;
-      for (int lt = 0; lt < my_tiles && ok; ++lt) {
-        const int tile = pair + lt * n_pairs;
-        const int tok0 = (tile % m_tiles) * kPairBT + rank * 128;
-        const int row0 = ((tile / m_tiles) * 2 + rank) * kBM;
-        for (int kb = 0; kb < nkb; ++kb) {
+      for (int lt = 0; lt < my_units && ok; ++lt) {
+        const Unit u = decode_unit(P, pair, n_pairs, rank, lt);
+        const int tok0 = u.m_tile * kPairBT + rank * 128;
+        const int row0 = u.n_tile * kBM;
+        for (int kb = u.kb0; kb < u.kb1; ++kb) {
           if (!mbar_wait(xempty_bar(x.idx), x.phase ^ 1u, abort_flag, P.status)) { ok = false; break; }
           mbar_expect_tx(xfull_bar(x.idx), kXStageBytes);
           tma_load_2d(tiles_base + b_off(x.idx), &tmap_x, kb * kBK, tok0, xfull_bar(x.idx));
@@ -223,22 +349,24 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         const int groups_kb = (P.G < kBK) ? kBK / P.G : 1;     // scale groups per k-block
         const int kb_per_group = (P.G > kBK) ? P.G / kBK : 1;  // k-blocks per scale group
         const uint32_t tx_bytes = static_cast<uint32_t>(kCodesBytes + groups_kb * 1024);
-        const int64_t sz_step = static_cast<int64_t>(groups_kb) * P.Npad;
         int cidx = 0;
         uint32_t cphase = 0, dst = tiles_base + kCBase;
         bool ok = true;
-        for (int lt = 0; lt < my_tiles && ok; ++lt) {
-          const int n_tile = ((pair + lt * n_pairs) / m_tiles) * 2 + rank;
-          const uint8_t* codes = P.codes + static_cast<int64_t>(n_tile) * nkb * kCodesBytes;
-          const float2* sz = P.sz + static_cast<int64_t>(n_tile) * kBM;
+        for (int lt = 0; lt < my_units && ok; ++lt) {
+          const Unit u = decode_unit(P, pair, n_pairs, rank, lt);
+          const int64_t Npad = SZO_SUB(P, u.s, Npad);
+          const int64_t sz_step = static_cast<int64_t>(groups_kb) * Npad;
+          // a unit starts on a scale-group boundary (the host aligns the K split)
+          const uint8_t* codes = SZO_SUB(P, u.s, codes) + (static_cast<int64_t>(u.n_tile) * nkb + u.kb0) * kCodesBytes;
+          const float2* sz = SZO_SUB(P, u.s, sz) + static_cast<int64_t>(u.n_tile) * kBM + (u.kb0 / kb_per_group) * sz_step;
           int kbg = 0;
-          for (int kb = 0; kb < nkb; ++kb) {
+          for (int kb = u.kb0; kb < u.kb1; ++kb) {
             if (!mbar_wait(cempty_bar(cidx), cphase ^ 1u, abort_flag, P.status)) { ok = false; break; }
             const uint32_t bar = cfull_bar(cidx);
             mbar_expect_tx(bar, tx_bytes);
             bulk_load_1d(dst, codes, kCodesBytes, bar);
             bulk_load_1d(dst + kCodesBytes, sz, 1024, bar);
-            for (int g = 1; g < groups_kb; ++g) bulk_load_1d(dst + kCodesBytes + g * 1024, sz + g * P.Npad, 1024, bar);
+            for (int g = 1; g < groups_kb; ++g) bulk_load_1d(dst + kCodesBytes + g * 1024, sz + g * Npad, 1024, bar);
             codes += kCodesBytes;
             if (++kbg == kb_per_group) {
               kbg = 0;
@@ -259,13 +387,14 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     if (leader && lane == 0) {
       RingPos x{0, 0}, a{0, 0};
       bool ok = true;
-      for (int lt = 0; lt < my_tiles && ok; ++lt) {
+      for (int lt = 0; lt < my_units && ok; ++lt) {
         const int as = lt & 1;
         const uint32_t aph = static_cast<uint32_t>((lt >> 1) & 1);
+        const int n_kb = (lt < P.full_rounds) ? nkb : my_iters - full_iters;
         if (!mbar_wait(accempty_bar(as), aph ^ 1u, abort_flag, P.status, 0)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kPairBT);
-        for (int kb = 0; kb < nkb; ++kb) {
+        for (int kb = 0; kb < n_kb; ++kb) {
           // both CTAs' weight tiles final and both token halves landed
           if (!mbar_wait(aready_bar(a.idx), a.phase, abort_flag, P.status, 0)) { ok = false; break; }
           tc_fence_after();
@@ -288,32 +417,41 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     // k-blocks per loop iteration (lane j < 4 owns the bounds of k-block it0 + j), up to three chunks
     // ahead of their use.  The bounds of the next chunk are fetched while this chunk's records are
     // in flight, so one global-load latency is exposed per four k-blocks.
-    if (sparse && my_tiles > 0) {
-      const int n_kblocks = static_cast<int>(P.n_kblocks);
-      const int n_rowtiles = static_cast<int>(P.n_rowtiles);
-      auto load_bounds = [&](int it0, int32_t& e0, int32_t& e1) {
+    if (sparse && my_units > 0) {
+      auto load_bounds = [&](int it0, int32_t& e0, int32_t& e1, int& sm) {
         const int itl = it0 + (lane & (kRecChunk - 1));
         e0 = 0;
         e1 = 0;
+        sm = 0;
         if (itl < my_iters) {
-          const int lt = itl / nkb, kb = itl - lt * nkb;
-          const int n_tile = ((pair + lt * n_pairs) / m_tiles) * 2 + rank;
-          if (n_tile < n_rowtiles) {
-            const int32_t* bp = P.bucket_ptr + static_cast<int64_t>(n_tile) * n_kblocks + kb;
+          int lt, kb;
+          if (itl < full_iters) {
+            lt = itl / nkb;
+            kb = itl - lt * nkb;
+          } else {
+            lt = P.full_rounds;
+            kb = tail_kb0 + (itl - full_iters);
+          }
+          const Unit u = decode_unit(P, pair, n_pairs, rank, lt);
+          sm = u.s;
+          if (u.n_tile < SZO_SUB(P, u.s, n_rowtiles) && SZO_SUB(P, u.s, Sb) != nullptr) {
+            const int32_t* bp = SZO_SUB(P, u.s, bucket_ptr) + static_cast<int64_t>(u.n_tile) * nkb + kb;
             e0 = __ldg(bp);
             e1 = __ldg(bp + 1);
           }
         }
       };
       int32_t e0, e1;
-      load_bounds(0, e0, e1);
+      int sm;
+      load_bounds(0, e0, e1, sm);
       int cs = 0;                       // chunk slot: ring slots cs * 4 .. cs * 4 + 3
       uint32_t cphase = 0;
       bool first_pass = true;
       bool ok = true;
       for (int it0 = 0; it0 < my_iters && ok; it0 += kRecChunk) {
         int32_t ne0, ne1;
-        load_bounds(it0 + kRecChunk, ne0, ne1);
+        int nsm;
+        load_bounds(it0 + kRecChunk, ne0, ne1, nsm);
         if (!first_pass) {              // the slots' previous k-blocks must have been consumed
 #pragma unroll
           for (int j = 0; j < kRecChunk; ++j)
@@ -325,15 +463,14 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
 #pragma unroll
         for (int j = 0; j < kRecChunk; ++j) {
           const int32_t b0 = __shfl_sync(0xFFFFFFFFu, e0, j), b1 = __shfl_sync(0xFFFFFFFFu, e1, j);
+          const int sj = __shfl_sync(0xFFFFFFFFu, sm, j);
+          const uint2* Sb = SZO_SUB(P, sj, Sb);
           n[j] = (b1 - b0 < kRecCap) ? b1 - b0 : kRecCap;
 #pragma unroll
           for (int q = 0; q < kRecCap / 32; ++q)
-            if (lane + 32 * q < n[j]) r[j][q] = __ldg(P.Sb + b0 + lane + 32 * q);
+            if (lane + 32 * q < n[j]) r[j][q] = __ldg(Sb + b0 + lane + 32 * q);
         }
-        if (lane < kRecChunk) {
-          bound_ring[cs * kRecChunk + lane][0] = e0;
-          bound_ring[cs * kRecChunk + lane][1] = e1;
-        }
+        if (lane < kRecChunk) *reinterpret_cast<int4*>(bound_ring[cs * kRecChunk + lane]) = make_int4(e0, e1, sm, 0);
 #pragma unroll
         for (int j = 0; j < kRecChunk; ++j) {
 #pragma unroll
@@ -344,6 +481,7 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         if (lane < kRecChunk && it0 + lane < my_iters) mbar_arrive(recready_bar(cs * kRecChunk + lane));
         e0 = ne0;
         e1 = ne1;
+        sm = nsm;
         if (++cs == kRecChunks) {
           cs = 0;
           cphase ^= 1u;
@@ -406,7 +544,7 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
           __syncwarp();
           if (lane < e1 - e0) add_record(A, rec);
           for (int32_t j = lane + 32; j < e1 - e0; j += 32)
-            add_record(A, (j < kRecCap) ? rec_ring[rr.idx][j] : __ldg(P.Sb + e0 + j));
+            add_record(A, (j < kRecCap) ? rec_ring[rr.idx][j] : __ldg(SZO_SUB(P, bound_ring[rr.idx][2], Sb) + e0 + j));
         }
         fence_async_smem();
         __syncwarp();
@@ -444,7 +582,7 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         if (e1 > e0) {
           unsigned char* A = tiles_ptr + a_off(x.idx, x.idx);
           for (int32_t j = lane; j < e1 - e0; j += 32)
-            add_record(A, (j < kRecCap) ? rec_ring[rr.idx][j] : __ldg(P.Sb + e0 + j));
+            add_record(A, (j < kRecCap) ? rec_ring[rr.idx][j] : __ldg(SZO_SUB(P, bound_ring[rr.idx][2], Sb) + e0 + j));
           fence_async_smem();
         }
         __syncwarp();
@@ -462,42 +600,77 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
   } else if (warp >= kEpiWarp02) {
     // ---------------------------------------------------------------- epilogue (own 128 rows)
     const int qd = warp & 3;
-    for (int lt = 0; lt < my_tiles; ++lt) {
-      const int tile = pair + lt * n_pairs;
-      const int64_t n_tile = static_cast<int64_t>(tile / m_tiles) * 2 + rank, m_tile = tile % m_tiles;
+    for (int lt = 0; lt < my_units; ++lt) {
+      const Unit u = decode_unit(P, pair, n_pairs, rank, lt);
       const int as = lt & 1;
       const uint32_t aph = static_cast<uint32_t>((lt >> 1) & 1);
       if (!mbar_wait(accfull_bar(as), aph, abort_flag, P.status, 256)) break;
       tc_fence_after();
-      const int64_t n = n_tile * kBM + qd * 32 + lane;
-      const float bias = (P.bias != nullptr && n < P.N) ? P.bias[n] : 0.f;
-      const int64_t m0 = m_tile * kPairBT;
+      const int64_t N = SZO_SUB(P, u.s, N);
+      const float* bias_p = SZO_SUB(P, u.s, bias);
+      void* y = SZO_SUB(P, u.s, y);
+      const int64_t n = static_cast<int64_t>(u.n_tile) * kBM + qd * 32 + lane;
+      const float bias = (bias_p != nullptr && n < N) ? bias_p[n] : 0.f;
+      const int64_t m0 = static_cast<int64_t>(u.m_tile) * kPairBT;
       const int mlimit = static_cast<int>((P.M - m0 < kPairBT) ? P.M - m0 : kPairBT);
-      for (int c0 = 0; c0 < kPairBT; c0 += 32) {
-        uint32_t v[32];
-        tmem_ld32(tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + static_cast<uint32_t>(as * kPairBT + c0), v);
-        if (n < P.N && c0 < mlimit) {
+      // y[m0 + c0 + j, n] = v[j] + bias for the valid tokens of a 32-token chunk
+      auto store_chunk = [&](int c0, const uint32_t (&v)[32]) {
+        if (n < N && c0 < mlimit) {
           const int cnt = mlimit - c0;
           if (P.y_f32) {
-            float* yp = static_cast<float*>(P.y) + (m0 + c0) * P.N + n;
+            float* yp = static_cast<float*>(y) + (m0 + c0) * N + n;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
               if (j < cnt) *yp = __uint_as_float(v[j]) + bias;
-              yp += P.N;
+              yp += N;
             }
           } else {
-            __nv_bfloat16* yp = static_cast<__nv_bfloat16*>(P.y) + (m0 + c0) * P.N + n;
+            __nv_bfloat16* yp = static_cast<__nv_bfloat16*>(y) + (m0 + c0) * N + n;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
               if (j < cnt) *yp = __float2bfloat16_rn(__uint_as_float(v[j]) + bias);
-              yp += P.N;
+              yp += N;
             }
           }
         }
+      };
+      const uint32_t t_acc = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + static_cast<uint32_t>(as * kPairBT);
+      if (u.parts == 1) {
+        for (int c0 = 0; c0 < kPairBT; c0 += 32) {
+          uint32_t v[32];
+          tmem_ld32(t_acc + static_cast<uint32_t>(c0), v);
+          store_chunk(c0, v);
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(accempty_bar(as), 0);
+      } else {
+        // K-split tile (always this CTA's last unit): park this part's fp32 accumulator
+        // ([token][row], rows contiguous).  The last of the four epilogue warps takes the tile's
+        // ticket; the CTA holding the last part's ticket sums the parts after its roles are done.
+        constexpr int64_t kPartFloats = static_cast<int64_t>(kPairBT) * kBM;
+        float* mine = P.partial + (static_cast<int64_t>(u.slot * u.parts + u.part) * 2 + rank) * kPartFloats + qd * 32 + lane;
+        for (int c0 = 0; c0 < kPairBT; c0 += 32) {
+          uint32_t v[32];
+          tmem_ld32(t_acc + static_cast<uint32_t>(c0), v);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) __stcg(mine + (c0 + j) * kBM, __uint_as_float(v[j]));
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(accempty_bar(as), 0);
+        __threadfence();
+        __syncwarp();
+        if (lane == 0 && atomicAdd_block(&epi_count_s, 1) == 3) {
+          __threadfence();
+          int32_t* ticket = P.tickets + u.slot * 2 + rank;
+          if (atomicAdd(ticket, 1) == u.parts - 1) {
+            *ticket = 0;                       // ready for the next launch
+            __threadfence();                   // the other parts' tiles are read after this point
+            reduce_flag_s = 1;
+          }
+        }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(accempty_bar(as), 0);
     }
   }
 
@@ -507,13 +680,24 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
   }
   tc_fence_before();
   __syncthreads();
+  if (reduce_flag_s && !*abort_flag) {
+    // (the thread that took the last ticket fenced before raising the flag; the parts are read from
+    // L2 with ld.cg, and a fence by all 640 threads here measured about 7 us)
+    constexpr int64_t kPartFloats = static_cast<int64_t>(kPairBT) * kBM;
+    const Unit u = decode_unit(P, pair, n_pairs, rank, my_units - 1);
+    const int64_t m0 = static_cast<int64_t>(u.m_tile) * kPairBT;
+    const int mlimit = static_cast<int>((P.M - m0 < kPairBT) ? P.M - m0 : kPairBT);
+    reduce_parts(P.partial + (static_cast<int64_t>(u.slot * u.parts) * 2 + rank) * kPartFloats, u.parts,
+                 static_cast<int64_t>(u.n_tile) * kBM, SZO_SUB(P, u.s, N), SZO_SUB(P, u.s, bias), SZO_SUB(P, u.s, y), P.y_f32,
+                 m0, mlimit, static_cast<int>(threadIdx.x), kNumWarps2 * 32);
+  }
   cluster_sync_all();          // no CTA leaves while its peer may still signal it or read its tiles
   tc_fence_after();
   if (warp == 1) tmem_dealloc2(tmem_base, kTmemCols);
 }
 
 template <int kXS, bool kDequant, bool kFast>
-szo_status launch_tc2(const CUtensorMap& mx, const CUtensorMap& mw, const TcParams& P, int sms, cudaStream_t st) {
+szo_status launch_tc2(const CUtensorMap& mx, const CUtensorMap& mw, const TcParams& P, int n_pairs, cudaStream_t st) {
   constexpr size_t smem = static_cast<size_t>(kXS) * (kXHalfBytes + (kDequant ? 0 : kATileBytes)) +
                           (kDequant ? kCStages2 * (kCodesBytes + kSzBytes) + kASlots2 * kATileBytes : 0) + 1024;
   auto kern = szo_linear_tc2_kernel<kXS, kDequant, kFast>;
@@ -522,10 +706,7 @@ szo_status launch_tc2(const CUtensorMap& mx, const CUtensorMap& mw, const TcPara
     SZO_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
     configured = true;
   }
-  const int64_t tiles = P.m_tiles * P.n_tiles;
-  const int64_t max_pairs = sms / 2;
-  const unsigned grid = static_cast<unsigned>(2 * (tiles < max_pairs ? tiles : max_pairs));
-  kern<<<grid, kNumWarps2 * 32, smem, st>>>(mx, mw, P);
+  kern<<<static_cast<unsigned>(2 * n_pairs), kNumWarps2 * 32, smem, st>>>(mx, mw, P);
   count_launch();
   SZO_CHECK_LAUNCH("szo_linear_tc2_kernel");
   return SZO_OK;
@@ -533,12 +714,11 @@ szo_status launch_tc2(const CUtensorMap& mx, const CUtensorMap& mw, const TcPara
 
 }  // namespace
 
-// Pair-tile launch: tmap_x must have a [128 x 64] box; P.m_tiles / P.n_tiles count 256-wide tiles.
-szo_status linear_fwd_tc2(const szo_linear* p, const CUtensorMap& mx, const CUtensorMap& mw, const tc::TcParams& P,
-                          int sms, cudaStream_t st) {
-  if (p->G == 0) return launch_tc2<6, false, false>(mx, mw, P, sms, st);
-  if (p->sz_dtype == SZO_BF16) return launch_tc2<5, true, true>(mx, mw, P, sms, st);
-  return launch_tc2<5, true, false>(mx, mw, P, sms, st);
+szo_status launch_pair_kernel(bool dequant, bool bf16_tables, const CUtensorMap& mx, const CUtensorMap& mw,
+                              const tc::TcParams& P, int n_pairs, cudaStream_t st) {
+  if (!dequant) return launch_tc2<6, false, false>(mx, mw, P, n_pairs, st);
+  if (bf16_tables) return launch_tc2<5, true, true>(mx, mw, P, n_pairs, st);
+  return launch_tc2<5, true, false>(mx, mw, P, n_pairs, st);
 }
 
 }  // namespace szo

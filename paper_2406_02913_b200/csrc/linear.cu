@@ -332,17 +332,20 @@ szo_status linear_fwd_impl(const szo_linear* p, const void* x, int x_dtype, int6
   if (mode == SZO_MODE_FP32_VALIDATE)
     return linear_fwd_fp32(p, x, x_dtype, M, S_pert, y, y_dtype, workspace, workspace_bytes, st);
   if (mode == SZO_MODE_SPMM) {
-    SZO_TRY(linear_fwd_tc(p, x, M, nullptr, y, y_dtype, st));
+    SZO_TRY(linear_fwd_tc(p, x, M, nullptr, y, y_dtype, workspace, workspace_bytes, st));
     return linear_spmm(p, x, M, S_pert, y, y_dtype, st);
   }
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
   if (p->nnz > 0 && S_bucket == nullptr) {
     const size_t need = round_up(static_cast<size_t>(p->nnz) * sizeof(uint2), 256);
     SZO_REQUIRE(workspace && workspace_bytes >= need, SZO_ERR_WORKSPACE,
                 "SparseAdd needs a workspace of %zu bytes for the bucket-ordered values", need);
     SZO_TRY(gather_values(S_pert, p->bucket_eid, p->bucket_pos, p->nnz, static_cast<uint2*>(workspace), st));
     S_bucket = static_cast<const uint2*>(workspace);
+    ws += need;
+    workspace_bytes -= need;
   }
-  return linear_fwd_tc(p, x, M, S_bucket, y, y_dtype, st);
+  return linear_fwd_tc(p, x, M, S_bucket, y, y_dtype, workspace ? ws : nullptr, workspace ? workspace_bytes : 0, st);
 }
 
 static void free_plan(szo_linear* p) {
@@ -463,8 +466,10 @@ szo_status szo_linear_create(szo_linear_t** out, int64_t N, int64_t K, int32_t G
 size_t szo_linear_workspace_bytes(const szo_linear_t* p, int64_t M, int32_t mode) {
   if (!p) return 0;
   if (mode == SZO_MODE_FP32_VALIDATE) return linear_ws_fp32(p, M);
-  if (mode == SZO_MODE_SPMM) return 0;
-  return round_up(static_cast<size_t>(p->nnz) * sizeof(uint2), 256);   // bucket-ordered sparse records
+  const szo_linear* pp = p;
+  const size_t tail = tc_tail_ws_bytes(&pp, 1, M);                     // K-split tiles of the last round
+  if (mode == SZO_MODE_SPMM) return tail;
+  return round_up(static_cast<size_t>(p->nnz) * sizeof(uint2), 256) + tail;   // + bucket-ordered sparse records
 }
 
 szo_status szo_linear_fwd(const szo_linear_t* p, const void* x, szo_dtype x_dtype, int64_t M,

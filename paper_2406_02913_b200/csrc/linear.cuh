@@ -43,8 +43,18 @@ void tc_plan_destroy(szo_linear* p);
 // S_bucket: the sparse entries gathered into bucket order as records
 // (bucket_pos[p], bits of S[bucket_eid[p]]), or nullptr to leave the sparse term out (it is then
 // applied by linear_spmm).
+// ws: scratch of tc_tail_ws_bytes() bytes for the K-split tiles of the last round (may be nullptr:
+// no split).
 szo_status linear_fwd_tc(const szo_linear* p, const void* x, int64_t M, const uint2* S_bucket, void* y,
-                         int y_dtype, cudaStream_t st);
+                         int y_dtype, void* ws, size_t ws_bytes, cudaStream_t st);
+// Several layers that read the same x in one launch (q/k/v, gate/up): same K, G and table dtype,
+// G > 0, M > 128 (tc_can_fuse).  S_bucket[i] / y[i] belong to plans[i].
+bool tc_can_fuse(const szo_linear* const* plans, int n, int64_t M);
+szo_status linear_fwd_tc_group(const szo_linear* const* plans, int n, const void* x, int64_t M,
+                               const uint2* const* S_bucket, void* const* y, int y_dtype, void* ws, size_t ws_bytes,
+                               cudaStream_t st);
+size_t tc_tail_ws_bytes(const szo_linear* const* plans, int n, int64_t M);
+size_t tc_tail_ws_bound();   // enough for any M and any group
 // out[p] = (pos[p], bits of S[eid[p]]) for p in [0, n)
 szo_status gather_values(const float* S, const int32_t* eid, const uint16_t* pos, int64_t n, uint2* out,
                          cudaStream_t st);

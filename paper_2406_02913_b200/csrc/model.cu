@@ -419,6 +419,34 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
     }
     return rc;
   };
+  // layers j0 .. j0 + n - 1 read the same x: one fused launch when the tensor-core path allows it
+  auto lin_group = [&](int layer, int j0, int n, const void* x, void* const* outs) -> szo_status {
+    const int t0 = layer * m->n_lin + j0;
+    const szo_linear* plans[3];
+    const uint2* recs[3];
+    for (int i = 0; i < n; ++i) {
+      plans[i] = m->plans[t0 + i];
+      recs[i] = m->recs + m->offsets[t0 + i];
+    }
+    if (!(pregather && sizeof(T) == 2 && tc_can_fuse(plans, n, M))) {
+      for (int i = 0; i < n; ++i) SZO_TRY(lin(layer, j0 + i, x, outs[i]));
+      return SZO_OK;
+    }
+    if (m->timing) {
+      while (m->events.size() < m->events_used + 2) {
+        cudaEvent_t e;
+        SZO_CHECK_CUDA(cudaEventCreate(&e));
+        m->events.push_back(e);
+      }
+      SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used], st));
+    }
+    const szo_status rc = linear_fwd_tc_group(plans, n, x, M, recs, outs, act, m->ws, m->ws_bytes, st);
+    if (m->timing) {
+      SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used + 1], st));
+      m->events_used += 2;
+    }
+    return rc;
+  };
   embed_kernel<<<static_cast<unsigned>(M), 128, 0, st>>>(tokens, static_cast<const __nv_bfloat16*>(m->top.embed),
                                                         static_cast<const __nv_bfloat16*>(m->top.pos), S, d,
                                                         c.vocab, m->h);
@@ -431,9 +459,10 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
     add_norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, pending, L.attn_norm_g, L.attn_norm_b, d,
                                                                 c.norm_eps, opt, 1, 0, a);
     count_launch();
-    SZO_TRY(lin(l, 0, a, q));
-    SZO_TRY(lin(l, 1, a, k));
-    SZO_TRY(lin(l, 2, a, v));
+    {
+      void* const qkv[3] = {q, k, v};
+      SZO_TRY(lin_group(l, 0, 3, a, qkv));
+    }
     if (!opt) {
       const int64_t n_vec = M * (H + Hkv) * ((hd / 2) / Vec16<T>::kN);
       rope_kernel<T><<<blocks_for(n_vec, 256), 256, 0, st>>>(q, k, m->rope_tab, M, S, H, Hkv, hd);
@@ -453,8 +482,8 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
                                                                 opt, 1, 0, a);
     count_launch();
     if (!opt) {
-      SZO_TRY(lin(l, 4, a, gate));
-      SZO_TRY(lin(l, 5, a, up));
+      void* const gu[2] = {gate, up};
+      SZO_TRY(lin_group(l, 4, 2, a, gu));
       silu_mul_kernel<T><<<blocks_for(M * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, up, M * ff, gate);
       count_launch();
       SZO_TRY(lin(l, 6, gate, y));
@@ -566,6 +595,11 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
       const size_t need = szo_linear_workspace_bytes(p, m->Mmax, c.linear_mode);
       if (need > ws_need) ws_need = need;
     }
+  }
+  if (!m->plans.empty() && c.linear_mode != SZO_MODE_FP32_VALIDATE) {
+    // K-split scratch of the pair-tile kernel: at most one 256 x 256 fp32 tile per cluster
+    const size_t need = tc_tail_ws_bound();
+    if (need > ws_need) ws_need = need;
   }
   m->k_total = m->offsets.back();
   if (m->k_total > 0 && S_all == nullptr) return bail(fail(SZO_ERR_INVALID_ARG, "S_all is NULL"));

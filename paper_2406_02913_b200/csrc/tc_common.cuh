@@ -23,6 +23,20 @@ constexpr int kRecSlots = 8, kRecCap = 128;  // ring of per-k-block sparse recor
 constexpr int kBoundSlots = 16;
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s of SM cycles
 
+// One weight matrix of a fused launch (pair-tile kernel): several linear layers that read the same
+// activations (q/k/v, gate/up) are concatenated along their output rows.
+struct TcSub {
+  const uint8_t* codes;    // tile order, as TcParams::codes
+  const float2* sz;
+  const int32_t* bucket_ptr;
+  const uint2* Sb;         // may be nullptr when the matrix has no sparse entries
+  const float* bias;
+  void* y;
+  int64_t N, Npad;
+  int n_rowtiles;          // 128-row tiles that have buckets
+  int n_tiles;             // 256-row pair tiles
+};
+
 struct TcParams {
   int64_t M, N, K;
   int G;
@@ -39,6 +53,18 @@ struct TcParams {
   void* y;
   int y_f32;
   int32_t* status;
+  // ---- pair-tile kernel only
+  int nsub;
+  TcSub sub[3];
+  // Work units of pair p: full tiles p + lt * n_pairs for lt < full_rounds, then (p < tail_tiles *
+  // tail_parts) one unit of the tail: tile full_rounds * n_pairs + p % tail_tiles, k-blocks
+  // [tail_kb[part], tail_kb[part + 1]) with part = p / tail_tiles.  With tail_parts > 1 the parts of
+  // a tile meet in `partial` (fp32 [tail_tiles][tail_parts][2 ranks][256 tokens][128 rows]) and the
+  // last part to finish (tickets, self-resetting) adds them up in part order and stores y.
+  int full_rounds, tail_tiles, tail_parts;
+  int tail_kb[5];
+  float* partial;
+  int32_t* tickets;        // [tail_tiles][2 ranks]
 };
 
 // Position in a ring of n slots: slot index and the parity of the current pass over the ring.
@@ -227,9 +253,10 @@ __device__ __forceinline__ uint4 dequant_word(uint32_t w, float2 p) {
 
 }  // namespace tc
 
-// Two-CTA pair-tile kernel (gemm_tc2.cu): tmap_x has a [128 x 64] box; P.m_tiles / P.n_tiles count
-// 256-wide tiles.
-szo_status linear_fwd_tc2(const szo_linear* p, const CUtensorMap& mx, const CUtensorMap& mw, const tc::TcParams& P,
-                          int sms, cudaStream_t st);
+// Two-CTA pair-tile kernel (gemm_tc2.cu): tmap_x has a [128 x 64] box; P.m_tiles counts
+// 256-token tiles, P.n_tiles the 256-row tiles of all P.nsub matrices; n_pairs clusters are launched.
+// dequant == false: dense bf16 weight through mw (one matrix only).
+szo_status launch_pair_kernel(bool dequant, bool bf16_tables, const CUtensorMap& mx, const CUtensorMap& mw,
+                              const tc::TcParams& P, int n_pairs, cudaStream_t st);
 
 }  // namespace szo
