@@ -26,8 +26,20 @@ __global__ void widen_sz_kernel(const SZ* __restrict__ scales, const SZ* __restr
 }
 
 // Copy of the packed codes in tile order: block (t, kb) holds rows [128 t, 128 t + 128) x bytes
-// [32 kb, 32 kb + 32) of the caller's [N, K/2] array, 4 KiB contiguous, rows beyond N zero.  One thread
-// moves 16 bytes.
+// [32 kb, 32 kb + 32) of the caller's [N, K/2] array, 4 KiB contiguous, rows beyond N zero.  Inside
+// each 32-bit word (eight consecutive columns c .. c+7) the nibbles are re-ordered so that nibble i
+// holds column c + 2 i and nibble 4 + i column c + 2 i + 1: the pair (c + 2 i, c + 2 i + 1) is then
+// (w >> 4 i) & 0x000F000F, one code per 16-bit half, which is what the bf16 conversion wants.  One
+// thread moves 16 bytes.
+__device__ __forceinline__ uint32_t pair_order(uint32_t w) {
+  uint32_t o = 0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    o |= ((w >> (8 * i)) & 0xFu) << (4 * i);             // column 2 i: low nibble of byte i
+    o |= ((w >> (8 * i + 4)) & 0xFu) << (16 + 4 * i);    // column 2 i + 1: high nibble of byte i
+  }
+  return o;
+}
 __global__ void tile_codes_kernel(const uint8_t* __restrict__ codes, int64_t N, int64_t K, int64_t n_tiles,
                                   uint8_t* __restrict__ out) {
   const int64_t nkb = K / 64;
@@ -38,6 +50,7 @@ __global__ void tile_codes_kernel(const uint8_t* __restrict__ codes, int64_t N, 
   const int64_t row = t * 128 + r;
   uint4 v = make_uint4(0u, 0u, 0u, 0u);
   if (row < N) v = *reinterpret_cast<const uint4*>(codes + row * (K / 2) + kb * 32 + half * 16);
+  v = make_uint4(pair_order(v.x), pair_order(v.y), pair_order(v.z), pair_order(v.w));
   *reinterpret_cast<uint4*>(out + i * 16) = v;
 }
 

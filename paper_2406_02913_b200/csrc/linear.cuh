@@ -14,7 +14,8 @@ struct szo_linear {
   const int64_t* idx;
   const float* bias;
   // derived, owned by the plan (device memory)
-  uint8_t* codes_tiled;  // [Npad/128][K/64][128 rows][32 B]: the codes of one (128-row tile, k-block) contiguous
+  uint8_t* codes_tiled;  // [Npad/128][K/64][128 rows][32 B]: the codes of one (128-row tile, k-block) contiguous,
+                         // nibbles of each 32-bit word in pair order (see tile_codes_kernel)
   float2* sz;            // [K/G][Npad] (scale, zero) widened to fp32, group-major (G > 0)
   int64_t Npad;          // N rounded up to a multiple of 256
   int32_t* ent_col;      // [nnz] column of entry e

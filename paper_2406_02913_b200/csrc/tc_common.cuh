@@ -214,7 +214,9 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
   return d;
 }
 
-// Eight codes of one 32-bit word -> eight bf16 values q*scale+zero (one rounding each).
+// Eight codes of one 32-bit word of the plan's tile-ordered copy -> eight bf16 values q*scale+zero
+// (one rounding each).  The word holds the codes of columns c .. c+7 in pair order: nibble i is
+// column c + 2 i, nibble 4 + i is column c + 2 i + 1.
 // kFast (bf16 scales/zeros): p carries the bit patterns of the packed pairs (scale,scale) and
 // (zero,zero); the arithmetic is exact packed bf16: (128+q) as bf16 is 0x4300|q, minus 128, then
 // one fused multiply-add.  Otherwise p = (scale, zero) in fp32: fp32 fma, then one conversion.
@@ -227,13 +229,9 @@ __device__ __forceinline__ uint4 dequant_word(uint32_t w, float2 p) {
     const __nv_bfloat162 z2 = *reinterpret_cast<const __nv_bfloat162*>(&zb);
     const uint32_t magic = 0x43004300u;
     const __nv_bfloat162 m2 = *reinterpret_cast<const __nv_bfloat162*>(&magic);
-    const uint32_t lo = w & 0x0F0F0F0Fu;          // codes of the even columns, one per byte
-    const uint32_t hi = (w >> 4) & 0x0F0F0F0Fu;   // codes of the odd columns
-    // byte permute: [lo.byte[i], 0, hi.byte[i], 0]; selector bit 3 replicates the (zero) sign bit
-    const uint32_t sel[4] = {0x8480u, 0x9591u, 0xA6A2u, 0xB7B3u};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const uint32_t t = prmt(lo, hi, sel[i]) | magic;
+      const uint32_t t = ((w >> (4 * i)) & 0x000F000Fu) | magic;     // one shift and one three-input logic op
       const __nv_bfloat162 q2 = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&t), m2);
       const __nv_bfloat162 r = __hfma2(q2, s2, z2);
       o[i] = *reinterpret_cast<const uint32_t*>(&r);
@@ -242,7 +240,8 @@ __device__ __forceinline__ uint4 dequant_word(uint32_t w, float2 p) {
     float f[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-      const float q = __uint_as_float(0x4B000000u | ((w >> (4 * e)) & 0xFu)) - 8388608.0f;
+      const int nib = (e >> 1) + 4 * (e & 1);
+      const float q = __uint_as_float(0x4B000000u | ((w >> (4 * nib)) & 0xFu)) - 8388608.0f;
       f[e] = fmaf(q, p.x, p.y);
     }
 #pragma unroll
