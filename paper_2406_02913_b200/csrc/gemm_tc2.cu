@@ -9,12 +9,12 @@
 //
 // Roles per CTA (same rings as the one-CTA kernel: X token tiles, C codes + scale/zero, A weights):
 //   warp 0       X producer: TMA of the CTA's own token half (and its bf16 weight tile in dense mode)
-//   warp 3       C producer: bulk copies of the CTA's code tile and scale/zero strip
-//   warp 1       TMEM allocation; in the leader CTA (cluster rank 0) one thread issues the
+//   warp 4       C producer: bulk copies of the CTA's code tile and scale/zero strip
+//   warp 8       TMEM allocation; in the leader CTA (cluster rank 0) one thread issues the
 //                tcgen05.mma.cta_group::2 instructions and commits, multicast, to the barriers of
 //                both CTAs
-//   warp 2       sparse-record prefetch (register-pipelined loads into a ring in shared memory)
-//   warps 4-15   weight producers (three groups of four take k-blocks in turn): int4 -> bf16 conversion and SparseAdd of the CTA's own rows; when
+//   warp 12      sparse-record prefetch (register-pipelined loads into a ring in shared memory)
+//   12 warps     weight producers (w < 16, w % 4 != 0; three groups of four take k-blocks in turn): int4 -> bf16 conversion and SparseAdd of the CTA's own rows; when
 //                the tile is final and the CTA's token half has landed they arrive, with cluster
 //                scope, on the leader's aready barrier (8 arrivals: one group of each CTA).  In dense
 //                mode the same warps add the sparse values to the TMA-loaded tile and relay.
@@ -36,10 +36,14 @@ constexpr int kPairBT = 256;                 // tokens per pair tile (UMMA N)
 constexpr int kXHalfBytes = 128 * kBK * 2;   // this CTA's half of the token tile: 16 KiB
 constexpr int kCStages2 = 6;
 constexpr int kASlots2 = 6;
-// 20 warps: four single-thread roles, three groups of four conversion warps, four epilogue warps
+// 20 warps: four single-thread roles, three groups of four conversion warps, four epilogue warps.
+// Warp w issues on scheduler w % 4.  The single-thread roles (warps 0, 4, 8, 12) share scheduler 0
+// with one epilogue warp only, so the thread that issues the MMAs never competes with conversion
+// warps for issue slots; the twelve conversion warps are the warps < 16 with w % 4 != 0; the
+// epilogue warps 16-19 cover the four TMEM lane quarters.
 constexpr int kGroups2 = 3, kWarpsPerGroup2 = 4;
-constexpr int kNumDeqWarps2 = kGroups2 * kWarpsPerGroup2;
-constexpr int kEpiWarp02 = kDeqWarp0 + kNumDeqWarps2;
+constexpr int kWarpX = 0, kWarpC = 4, kWarpMma = 8, kWarpRec = 12;
+constexpr int kEpiWarp02 = 16;
 constexpr int kNumWarps2 = kEpiWarp02 + 4;
 // sparse records: ring of per-k-block slots, filled a chunk of four k-blocks at a time
 constexpr int kRecChunk = 4, kRecChunks = 3, kRecSlots2 = kRecChunk * kRecChunks;
@@ -305,7 +309,7 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) tmem_alloc2(smem_u32(&tmem_base_slot), kTmemCols);
+  if (warp == kWarpMma) tmem_alloc2(smem_u32(&tmem_base_slot), kTmemCols);
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();          // the peer's barriers exist before anyone arrives on them
@@ -322,7 +326,7 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
   const int tail_kb0 = has_tail ? tail_kb_at(P, tail_part) : 0;
   const int my_iters = full_iters + (has_tail ? tail_kb_at(P, tail_part + 1) - tail_kb0 : 0);
 
-  if (warp == 0) {
+  if (warp == kWarpX) {
     // ---------------------------------------------------------------- X producer (own token half)
     if (lane == 0) {
       RingPos x{0, 0};
@@ -340,7 +344,7 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         }
       }
     }
-  } else if (warp == 3) {
+  } else if (warp == kWarpC) {
     // ---------------------------------------------------------------- C producer (codes, scale/zero)
     if constexpr (kDequant) {
       if (lane == 0) {
@@ -382,7 +386,7 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         }
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == kWarpMma) {
     // ---------------------------------------------------------------- MMA issuer (leader CTA only)
     if (leader && lane == 0) {
       RingPos x{0, 0}, a{0, 0};
@@ -410,7 +414,7 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         if (ok) umma2_commit_both(accfull_bar(as));
       }
     }
-  } else if (warp == 2) {
+  } else if (warp == kWarpRec) {
     // ---------------------------------------------------------------- sparse-record warp
     // Brings the bucket bounds and the sparse records (position in tile, fp32 value) of every
     // k-block of this CTA into a ring of per-k-block slots in shared memory, a chunk of four
@@ -470,7 +474,9 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
           for (int q = 0; q < kRecCap / 32; ++q)
             if (lane + 32 * q < n[j]) r[j][q] = __ldg(Sb + b0 + lane + 32 * q);
         }
-        if (lane < kRecChunk) *reinterpret_cast<int4*>(bound_ring[cs * kRecChunk + lane]) = make_int4(e0, e1, sm, 0);
+        // (slots past the end of the stream still belong to k-blocks that may not have been consumed)
+        if (lane < kRecChunk && it0 + lane < my_iters)
+          *reinterpret_cast<int4*>(bound_ring[cs * kRecChunk + lane]) = make_int4(e0, e1, sm, 0);
 #pragma unroll
         for (int j = 0; j < kRecChunk; ++j) {
 #pragma unroll
@@ -489,9 +495,9 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         }
       }
     }
-  } else if (warp >= kDeqWarp0 && warp < kEpiWarp02) {
+  } else if ((warp & 3) != 0 && warp < kEpiWarp02) {
     // ---------------------------------------------------------------- weight producers
-    const int dw = warp - kDeqWarp0;
+    const int dw = (warp >> 2) * 3 + (warp & 3) - 1;
     const int gq = dw / kWarpsPerGroup, wq = dw % kWarpsPerGroup;
     constexpr int kRowsPerWarp = kBM / kWarpsPerGroup;
     auto add_record = [&](unsigned char* A, uint2 rc) {
@@ -693,7 +699,7 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
   }
   cluster_sync_all();          // no CTA leaves while its peer may still signal it or read its tiles
   tc_fence_after();
-  if (warp == 1) tmem_dealloc2(tmem_base, kTmemCols);
+  if (warp == kWarpMma) tmem_dealloc2(tmem_base, kTmemCols);
 }
 
 template <int kXS, bool kDequant, bool kFast>
