@@ -111,6 +111,21 @@ szo_status szo_select_mask_static(const float* scores, int64_t n, int64_t k, int
 szo_status szo_perturb(const float* S_in, float* S_out, const int64_t* idx, int64_t k,
                        int64_t idx_base, uint64_t seed, uint64_t step, float scale, void* stream);
 
+/* ---- The same passes with z kept in device memory.  Section 2.1's seed trick regenerates z so that
+ * no copy of a model-sized vector is held; with the Definition 4 mask only k values are needed
+ * (26 MB at the 7B shape), so the first pass of a step can keep them and the -2 eps pass, the
+ * restore and the update become plain 12-byte-per-entry streams with bit-identical results.
+ *   szo_perturb_keep_z : szo_perturb, and z_out[j] = z_j (fp32[k], 16-byte aligned, caller-owned)
+ *   szo_perturb_kept_z : S_out[j] = fma(scale, z[j], S_in[j])
+ *   szo_update_kept_z  : szo_update with z read from z[] */
+szo_status szo_perturb_keep_z(const float* S_in, float* S_out, const int64_t* idx, int64_t k,
+                              int64_t idx_base, uint64_t seed, uint64_t step, float scale, float* z_out,
+                              void* stream);
+szo_status szo_perturb_kept_z(const float* S_in, float* S_out, const float* z, int64_t k, float scale,
+                              void* stream);
+szo_status szo_update_kept_z(float* S, const float* z, int64_t k, float lr, const double* f_plus_dev,
+                             const double* f_minus_dev, float eps, void* stream);
+
 /* ---- Projected gradient (Definition 1, SPSA): *g_dev = (*f_plus_dev - *f_minus_dev) / (2 eps),
  * fp64, all on the device. */
 szo_status szo_projected_gradient(const double* f_plus_dev, const double* f_minus_dev, float eps,

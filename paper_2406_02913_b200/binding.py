@@ -69,6 +69,11 @@ _SIGS = {
     "szo_select_mask_static": (C.c_int32, [C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]),
     "szo_perturb": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
                                 C.c_uint64, C.c_uint64, C.c_float, C.c_void_p]),
+    "szo_perturb_keep_z": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
+                                       C.c_uint64, C.c_uint64, C.c_float, C.c_void_p, C.c_void_p]),
+    "szo_perturb_kept_z": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_float, C.c_void_p]),
+    "szo_update_kept_z": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int64, C.c_float, C.c_void_p, C.c_void_p,
+                                      C.c_float, C.c_void_p]),
     "szo_projected_gradient": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p]),
     "szo_update": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_uint64, C.c_uint64,
                                C.c_float, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]),
@@ -180,6 +185,19 @@ def szo_select_mask_static(scores: torch.Tensor, k: int, out: torch.Tensor) -> t
 def szo_perturb(S_in, S_out, idx, idx_base: int, seed: int, step: int, scale: float):
     _check(lib().szo_perturb(_ptr(S_in), _ptr(S_out), _ptr(idx), idx.numel(), idx_base, seed, step,
                              scale, _stream()))
+
+
+def szo_perturb_keep_z(S_in, S_out, idx, idx_base: int, seed: int, step: int, scale: float, z_out):
+    _check(lib().szo_perturb_keep_z(_ptr(S_in), _ptr(S_out), _ptr(idx), idx.numel(), idx_base, seed, step,
+                                    scale, _ptr(z_out), _stream()))
+
+
+def szo_perturb_kept_z(S_in, S_out, z, scale: float):
+    _check(lib().szo_perturb_kept_z(_ptr(S_in), _ptr(S_out), _ptr(z), z.numel(), scale, _stream()))
+
+
+def szo_update_kept_z(S, z, lr: float, f_plus, f_minus, eps: float):
+    _check(lib().szo_update_kept_z(_ptr(S), _ptr(z), z.numel(), lr, _ptr(f_plus), _ptr(f_minus), eps, _stream()))
 
 
 def szo_projected_gradient(f_plus, f_minus, eps: float, g_out):

@@ -63,9 +63,13 @@ struct ScaleArg {
   const double* f_plus;
   const double* f_minus;
 };
+// z_out != nullptr: also keep z_j in z_out[j]
 szo_status launch_sparse_axpy(const float* S_in, float* S_out, const int64_t* idx, int64_t k,
                               int64_t idx_base, uint64_t seed, uint64_t step, ScaleArg sa,
-                              cudaStream_t st);
+                              cudaStream_t st, float* z_out = nullptr);
+// S_out[j] = fma(scale, z[j], S_in[j]) with kept z
+szo_status launch_sparse_axpy_kept(const float* S_in, float* S_out, const float* z, int64_t k, ScaleArg sa,
+                                   cudaStream_t st);
 
 // Causal attention for bf16 activations (attention.cu); q, k, v, o are [B*S, heads*hd] row-major.
 szo_status launch_flash_attention_bf16(const void* q, const void* k, const void* v, void* o, int B, int S, int H,

@@ -344,6 +344,7 @@ struct szo_model {
   int32_t* geid = nullptr;      // [k_total] entry id in S_all of each bucket-ordered record
   uint16_t* gpos = nullptr;     // [k_total] in-tile position of each bucket-ordered record
   uint2* recs = nullptr;        // [k_total] (position, value) records of the current forward
+  float* zkept = nullptr;       // [k_total] z of the current step, kept by the first perturb pass
   int64_t Mmax = 0;
   // activations
   float* h = nullptr;
@@ -647,6 +648,7 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
   SZO_M_TRY(dev_alloc(m, &m->geid, m->k_total * sizeof(int32_t)));
   SZO_M_TRY(dev_alloc(m, &m->gpos, m->k_total * sizeof(uint16_t)));
   SZO_M_TRY(dev_alloc(m, &m->recs, m->k_total * sizeof(uint2)));
+  SZO_M_TRY(dev_alloc(m, &m->zkept, m->k_total * sizeof(float)));
   if (m->k_total >= (int64_t(1) << 31)) return bail(fail(SZO_ERR_SHAPE, "more than 2^31 sparse entries"));
   for (size_t t = 0; t < m->plans.size(); ++t) {
     const szo_linear* p = m->plans[t];
@@ -706,16 +708,17 @@ szo_status szo_model_zo_step(szo_model_t* m, const int32_t* tokens, const int32_
   const int64_t k = m->k_total;
   float* Sv = m->S_all;
   ScaleArg sa{eps, 0.f, 0.f, nullptr, nullptr};
-  SZO_TRY(launch_sparse_axpy(Sv, Sv, m->gidx, k, 0, seed, step, sa, st));                 // S += eps z
+  // z is generated once per step (first pass) and kept: the other three passes stream it
+  SZO_TRY(launch_sparse_axpy(Sv, Sv, m->gidx, k, 0, seed, step, sa, st, m->zkept));       // S += eps z
   SZO_TRY(run_loss(m, tokens, labels, cand, B, S, Sv, f_plus_dev, st));                   // f+
   sa.scale = -2.0f * eps;
-  SZO_TRY(launch_sparse_axpy(Sv, Sv, m->gidx, k, 0, seed, step, sa, st));                 // S -= 2 eps z
+  SZO_TRY(launch_sparse_axpy_kept(Sv, Sv, m->zkept, k, sa, st));                          // S -= 2 eps z
   SZO_TRY(run_loss(m, tokens, labels, cand, B, S, Sv, f_minus_dev, st));                  // f-
   sa.scale = eps;
-  SZO_TRY(launch_sparse_axpy(Sv, Sv, m->gidx, k, 0, seed, step, sa, st));                 // S += eps z
+  SZO_TRY(launch_sparse_axpy_kept(Sv, Sv, m->zkept, k, sa, st));                          // S += eps z
   SZO_TRY(szo_projected_gradient(f_plus_dev, f_minus_dev, eps, g_dev, stream));           // g
   ScaleArg su{0.f, lr, eps, f_plus_dev, f_minus_dev};
-  SZO_TRY(launch_sparse_axpy(Sv, Sv, m->gidx, k, 0, seed, step, su, st));                 // S -= lr g z
+  SZO_TRY(launch_sparse_axpy_kept(Sv, Sv, m->zkept, k, su, st));                          // S -= lr g z
   m->last_launches = g_launch_count - before;
   return SZO_OK;
 }

@@ -97,10 +97,12 @@ __device__ __forceinline__ float resolve_scale(const ScaleArg& a) {
 // ten-round chain.  The next iteration's loads are issued before the current values are computed.
 constexpr int kAxpyPer = 8;
 
+// kKeepZ: also store z_j to z_out[j], for the later passes of the same (seed, step).
+template <bool kKeepZ>
 __global__ void __launch_bounds__(256)
 sparse_axpy_kernel(const float* __restrict__ S_in, float* __restrict__ S_out,
                    const int64_t* __restrict__ idx, int64_t k, int64_t idx_base, const PhiloxKeys K,
-                   uint32_t step_lo, uint32_t step_hi, ScaleArg sa) {
+                   uint32_t step_lo, uint32_t step_hi, ScaleArg sa, float* __restrict__ z_out) {
   const float scale = resolve_scale(sa);
   const int64_t octs = k / kAxpyPer;
   const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
@@ -125,6 +127,8 @@ sparse_axpy_kernel(const float* __restrict__ S_in, float* __restrict__ S_out,
       o.z = fmaf(scale, z[4 * j + 2], s[j].z);
       o.w = fmaf(scale, z[4 * j + 3], s[j].w);
       reinterpret_cast<float4*>(S_out)[2 * p + j] = o;
+      if constexpr (kKeepZ)
+        reinterpret_cast<float4*>(z_out)[2 * p + j] = make_float4(z[4 * j], z[4 * j + 1], z[4 * j + 2], z[4 * j + 3]);
     }
   }
   // up to seven trailing entries
@@ -132,7 +136,47 @@ sparse_axpy_kernel(const float* __restrict__ S_in, float* __restrict__ S_out,
   if (blockIdx.x == 0 && threadIdx.x < kAxpyPer && j < k) {
     const float z = z_of(static_cast<uint64_t>(idx_base + idx[j]), step_lo, step_hi, K);
     S_out[j] = fmaf(scale, z, S_in[j]);
+    if constexpr (kKeepZ) z_out[j] = z;
   }
+}
+
+// The later passes of a step with z kept by the first one: S_out[j] = fma(scale, z[j], S_in[j]),
+// 12 bytes per entry and one fma: a plain stream.  Sixteen entries per thread and iteration, all
+// eight 16-byte loads issued before the first use (a pass over a few million entries lasts ~15 us:
+// memory-level parallelism per thread is what fills the pipe that quickly).
+constexpr int kKeptUnroll = 4;
+__global__ void __launch_bounds__(256)
+sparse_axpy_kept_kernel(const float* __restrict__ S_in, float* __restrict__ S_out, const float* __restrict__ z,
+                        int64_t k, ScaleArg sa) {
+  const float scale = resolve_scale(sa);
+  const int64_t quads = k / 4;
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  for (int64_t p0 = t; p0 < quads; p0 += stride * kKeptUnroll) {
+    float4 s[kKeptUnroll], zz[kKeptUnroll];
+#pragma unroll
+    for (int u = 0; u < kKeptUnroll; ++u) {
+      const int64_t p = p0 + u * stride;
+      if (p < quads) {
+        s[u] = reinterpret_cast<const float4*>(S_in)[p];
+        zz[u] = reinterpret_cast<const float4*>(z)[p];
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kKeptUnroll; ++u) {
+      const int64_t p = p0 + u * stride;
+      if (p < quads) {
+        float4 o;
+        o.x = fmaf(scale, zz[u].x, s[u].x);
+        o.y = fmaf(scale, zz[u].y, s[u].y);
+        o.z = fmaf(scale, zz[u].z, s[u].z);
+        o.w = fmaf(scale, zz[u].w, s[u].w);
+        reinterpret_cast<float4*>(S_out)[p] = o;
+      }
+    }
+  }
+  const int64_t j = quads * 4 + threadIdx.x;
+  if (blockIdx.x == 0 && threadIdx.x < 4 && j < k) S_out[j] = fmaf(scale, z[j], S_in[j]);
 }
 
 __global__ void projected_gradient_kernel(const double* f_plus, const double* f_minus, float eps,
@@ -140,9 +184,21 @@ __global__ void projected_gradient_kernel(const double* f_plus, const double* f_
   *g = (*f_plus - *f_minus) / (2.0 * static_cast<double>(eps));
 }
 
+szo_status launch_sparse_axpy_kept(const float* S_in, float* S_out, const float* z, int64_t k, ScaleArg sa,
+                                   cudaStream_t st) {
+  if (k == 0) return SZO_OK;
+  int64_t blocks = ceil_div(ceil_div(k, 4 * kKeptUnroll), 256);
+  const int64_t wave = 148 * 8;
+  if (blocks > wave) blocks = wave;
+  sparse_axpy_kept_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(S_in, S_out, z, k, sa);
+  count_launch();
+  SZO_CHECK_LAUNCH("sparse_axpy_kept_kernel");
+  return SZO_OK;
+}
+
 szo_status launch_sparse_axpy(const float* S_in, float* S_out, const int64_t* idx, int64_t k,
                               int64_t idx_base, uint64_t seed, uint64_t step, ScaleArg sa,
-                              cudaStream_t st) {
+                              cudaStream_t st, float* z_out) {
   if (k == 0) return SZO_OK;
   PhiloxKeys K;
   uint32_t k0 = static_cast<uint32_t>(seed), k1 = static_cast<uint32_t>(seed >> 32);
@@ -161,8 +217,12 @@ szo_status launch_sparse_axpy(const float* S_in, float* S_out, const int64_t* id
     blocks = ceil_div(ceil_div(quads, sweeps), 256);        // just enough threads for that many sweeps
     if (blocks > wave) blocks = wave;
   }
-  sparse_axpy_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(
-      S_in, S_out, idx, k, idx_base, K, static_cast<uint32_t>(step), static_cast<uint32_t>(step >> 32), sa);
+  if (z_out != nullptr)
+    sparse_axpy_kernel<true><<<static_cast<unsigned>(blocks), 256, 0, st>>>(
+        S_in, S_out, idx, k, idx_base, K, static_cast<uint32_t>(step), static_cast<uint32_t>(step >> 32), sa, z_out);
+  else
+    sparse_axpy_kernel<false><<<static_cast<unsigned>(blocks), 256, 0, st>>>(
+        S_in, S_out, idx, k, idx_base, K, static_cast<uint32_t>(step), static_cast<uint32_t>(step >> 32), sa, nullptr);
   count_launch();
   SZO_CHECK_LAUNCH("sparse_axpy_kernel");
   return SZO_OK;
@@ -183,6 +243,41 @@ szo_status szo_perturb(const float* S_in, float* S_out, const int64_t* idx, int6
   szo::ScaleArg sa{scale, 0.f, 0.f, nullptr, nullptr};
   return szo::launch_sparse_axpy(S_in, S_out, idx, k, idx_base, seed, step, sa,
                                  static_cast<cudaStream_t>(stream));
+}
+
+szo_status szo_perturb_keep_z(const float* S_in, float* S_out, const int64_t* idx, int64_t k, int64_t idx_base,
+                              uint64_t seed, uint64_t step, float scale, float* z_out, void* stream) {
+  SZO_REQUIRE(k >= 0, SZO_ERR_INVALID_ARG, "k < 0");
+  if (k == 0) return SZO_OK;
+  SZO_REQUIRE(S_in && S_out && idx && z_out, SZO_ERR_INVALID_ARG, "NULL pointer");
+  SZO_REQUIRE(idx_base >= 0, SZO_ERR_INVALID_ARG, "idx_base < 0");
+  SZO_REQUIRE(szo::aligned16(S_in) && szo::aligned16(S_out) && szo::aligned16(idx) && szo::aligned16(z_out),
+              SZO_ERR_ALIGNMENT, "S_in, S_out, idx and z_out must be 16-byte aligned");
+  szo::ScaleArg sa{scale, 0.f, 0.f, nullptr, nullptr};
+  return szo::launch_sparse_axpy(S_in, S_out, idx, k, idx_base, seed, step, sa, static_cast<cudaStream_t>(stream),
+                                 z_out);
+}
+
+szo_status szo_perturb_kept_z(const float* S_in, float* S_out, const float* z, int64_t k, float scale, void* stream) {
+  SZO_REQUIRE(k >= 0, SZO_ERR_INVALID_ARG, "k < 0");
+  if (k == 0) return SZO_OK;
+  SZO_REQUIRE(S_in && S_out && z, SZO_ERR_INVALID_ARG, "NULL pointer");
+  SZO_REQUIRE(szo::aligned16(S_in) && szo::aligned16(S_out) && szo::aligned16(z), SZO_ERR_ALIGNMENT,
+              "S_in, S_out and z must be 16-byte aligned");
+  szo::ScaleArg sa{scale, 0.f, 0.f, nullptr, nullptr};
+  return szo::launch_sparse_axpy_kept(S_in, S_out, z, k, sa, static_cast<cudaStream_t>(stream));
+}
+
+szo_status szo_update_kept_z(float* S, const float* z, int64_t k, float lr, const double* f_plus_dev,
+                             const double* f_minus_dev, float eps, void* stream) {
+  SZO_REQUIRE(k >= 0, SZO_ERR_INVALID_ARG, "k < 0");
+  SZO_REQUIRE(f_plus_dev && f_minus_dev, SZO_ERR_INVALID_ARG, "NULL loss pointer");
+  SZO_REQUIRE(eps != 0.f, SZO_ERR_INVALID_ARG, "eps == 0");
+  if (k == 0) return SZO_OK;
+  SZO_REQUIRE(S && z, SZO_ERR_INVALID_ARG, "NULL pointer");
+  SZO_REQUIRE(szo::aligned16(S) && szo::aligned16(z), SZO_ERR_ALIGNMENT, "S and z must be 16-byte aligned");
+  szo::ScaleArg sa{0.f, lr, eps, f_plus_dev, f_minus_dev};
+  return szo::launch_sparse_axpy_kept(S, S, z, k, sa, static_cast<cudaStream_t>(stream));
 }
 
 szo_status szo_update(float* S, const int64_t* idx, int64_t k, int64_t idx_base, uint64_t seed,

@@ -90,6 +90,37 @@ def test_update_and_projected_gradient(B):
     assert np.allclose(d_S.cpu().numpy(), full, rtol=0, atol=1e-12 + abs(float(sc)) * 1e-5)
 
 
+@pytest.mark.parametrize("k", [1, 3, 8, 4099, 250_001])
+def test_kept_z_passes_equal_the_regenerating_ones(B, k):
+    """First pass keeps z; the -2 eps pass, the restore and the update then read it.  Every result
+    must be bit-identical to the regenerating entry points (same z, same single fma)."""
+    n = 6_476_005_376
+    idx = torch.from_numpy(wl.sorted_random_indices(n, k, seed=21, i=k)).cuda()
+    S0 = torch.from_numpy(wl.rng(22, wl.PURPOSE_WEIGHTS, k).normal(0, 0.02, k).astype(np.float32)).cuda()
+    seed, step, eps, lr = 99, 7, 1e-3, 1e-4
+    f = torch.tensor([0.70, 0.69], dtype=torch.float64, device="cuda")
+    a, b = S0.clone(), S0.clone()
+    z = torch.full((k,), 123.0, device="cuda")
+    zref = torch.empty(k, device="cuda")
+    B.szo_perturb(torch.zeros(k, device="cuda"), zref, idx, 5, seed, step, 1.0)        # z itself
+    B.szo_perturb(a, a, idx, 5, seed, step, eps)
+    B.szo_perturb_keep_z(b, b, idx, 5, seed, step, eps, z)
+    assert torch.equal(a, b) and torch.equal(z, zref)
+    z_ref = so.gaussian(seed, step, idx.cpu().numpy() + 5)
+    assert np.all(np.abs(z.cpu().numpy().astype(np.float64) - z_ref) <= _z_tol(z_ref))
+    for sc in (-2e-3, 1e-3):
+        B.szo_perturb(a, a, idx, 5, seed, step, sc)
+        B.szo_perturb_kept_z(b, b, z, sc)
+        assert torch.equal(a, b)
+    B.szo_update(a, idx, 5, seed, step, lr, f[0:1], f[1:2], eps)
+    B.szo_update_kept_z(b, z, lr, f[0:1], f[1:2], eps)
+    assert torch.equal(a, b)
+    out = torch.empty_like(b)                                                          # out of place
+    B.szo_perturb_kept_z(b, out, z, 0.5)
+    assert np.array_equal(out.cpu().numpy().view(np.uint32),
+                          so.fmaf32(np.float32(0.5), z.cpu().numpy(), b.cpu().numpy()).view(np.uint32))
+
+
 def test_perturb_empty_and_bad_arguments(B):
     e = torch.empty(0, device="cuda")
     B.szo_perturb(e, e, torch.empty(0, dtype=torch.int64, device="cuda"), 0, 1, 1, 1.0)
