@@ -561,13 +561,11 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
           mbar_arrive(cempty_bar(c.idx));
           if (sparse) mbar_arrive(recfree_bar(rr.idx));
         }
-#pragma unroll
-        for (int j = 0; j < kGroups; ++j) {
-          c.advance(kCS);
-          a.advance(kAS);
-          x.advance(kXS);
-          rr.advance(kRecSlots2);
-        }
+        static_assert(kGroups <= kCS && kGroups <= kAS && kGroups <= kXS && kGroups <= kRecSlots2, "ring shorter than a stride");
+        c.advance_by(kGroups, kCS);
+        a.advance_by(kGroups, kAS);
+        x.advance_by(kGroups, kXS);
+        rr.advance_by(kGroups, kRecSlots2);
       }
     } else {
       // dense bf16 weight tile delivered by TMA: add the bucket's sparse values (if any) and relay
@@ -596,11 +594,8 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
           mbar_arrive_cluster(aready_bar(x.idx), 0);
           if (sparse) mbar_arrive(recfree_bar(rr.idx));
         }
-#pragma unroll
-        for (int j = 0; j < kGroups; ++j) {
-          x.advance(kXS);
-          rr.advance(kRecSlots2);
-        }
+        x.advance_by(kGroups, kXS);
+        rr.advance_by(kGroups, kRecSlots2);
       }
     }
   } else if (warp >= kEpiWarp02) {

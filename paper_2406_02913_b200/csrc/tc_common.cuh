@@ -80,6 +80,14 @@ struct RingPos {
       phase ^= 1u;
     }
   }
+  // steps <= n slots forward in one go
+  __device__ __forceinline__ void advance_by(int steps, int n) {
+    idx += steps;
+    if (idx >= n) {
+      idx -= n;
+      phase ^= 1u;
+    }
+  }
 };
 
 // ------------------------------------------------------------------------------ PTX wrappers
