@@ -367,9 +367,8 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
           // SparseAdd: add the bucket's fp32 values to this warp's rows of the bf16 tile
           __syncwarp();
           auto apply = [&](uint2 rc) {
-            const int r = static_cast<int>(rc.x >> 6), col = static_cast<int>(rc.x & 63);
-            if (r / kRowsPerWarp == wq) {
-              __nv_bfloat16* el = reinterpret_cast<__nv_bfloat16*>(A + r * 128 + (((col >> 3) ^ (r & 7)) << 4) + (col & 7) * 2);
+            if (static_cast<int>(rc.x >> 7) / kRowsPerWarp == wq) {     // rc.x: byte offset in the swizzled tile
+              __nv_bfloat16* el = reinterpret_cast<__nv_bfloat16*>(A + rc.x);
               *el = __float2bfloat16_rn(__bfloat162float(*el) + __uint_as_float(rc.y));
             }
           };
@@ -405,9 +404,8 @@ szo_linear_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
         unsigned char* A = tiles_ptr + a_off(x.idx, x.idx);
         for (int32_t j = lane; j < e1 - e0; j += 32) {
           const uint2 rc = (j < kRecCap) ? rec_ring[it & (kRecSlots - 1)][j] : __ldg(P.Sb + e0 + j);
-          const int r = static_cast<int>(rc.x >> 6), col = static_cast<int>(rc.x & 63);
-          if (r / kRowsPerWarp == wq) {
-            __nv_bfloat16* el = reinterpret_cast<__nv_bfloat16*>(A + r * 128 + (((col >> 3) ^ (r & 7)) << 4) + (col & 7) * 2);
+          if (static_cast<int>(rc.x >> 7) / kRowsPerWarp == wq) {
+            __nv_bfloat16* el = reinterpret_cast<__nv_bfloat16*>(A + rc.x);
             *el = __float2bfloat16_rn(__bfloat162float(*el) + __uint_as_float(rc.y));
           }
         }

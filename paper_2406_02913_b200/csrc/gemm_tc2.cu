@@ -501,9 +501,9 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     const int gq = dw / kWarpsPerGroup, wq = dw % kWarpsPerGroup;
     constexpr int kRowsPerWarp = kBM / kWarpsPerGroup;
     auto add_record = [&](unsigned char* A, uint2 rc) {
-      const int r = static_cast<int>(rc.x >> 6), col = static_cast<int>(rc.x & 63);
-      if (r / kRowsPerWarp == wq) {
-        __nv_bfloat16* el = reinterpret_cast<__nv_bfloat16*>(A + r * 128 + (((col >> 3) ^ (r & 7)) << 4) + (col & 7) * 2);
+      // rc.x: byte offset of the element in the swizzled tile (row = offset / 128)
+      if (static_cast<int>(rc.x >> 7) / kRowsPerWarp == wq) {
+        __nv_bfloat16* el = reinterpret_cast<__nv_bfloat16*>(A + rc.x);
         *el = __float2bfloat16_rn(__bfloat162float(*el) + __uint_as_float(rc.y));
       }
     };
@@ -535,8 +535,9 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         uint2 rec = make_uint2(0xFFFFFFFFu, 0u);
         if (sparse) {
           if (!mbar_wait(recready_bar(rr.idx), rr.phase, abort_flag, P.status)) break;
-          e0 = bound_ring[rr.idx][0];
-          e1 = bound_ring[rr.idx][1];
+          const int2 be = *reinterpret_cast<const int2*>(bound_ring[rr.idx]);
+          e0 = be.x;
+          e1 = be.y;
           if (lane < e1 - e0) rec = rec_ring[rr.idx][lane];
         }
         if (!mbar_wait(aempty_bar(a.idx), a.phase ^ 1u, abort_flag, P.status)) break;

@@ -123,7 +123,10 @@ __global__ void bucket_fill_kernel(const int64_t* __restrict__ idx, const int32_
     const int64_t b = g * nkb + (col >> 6);
     const int32_t pos = bucket_ptr[b] + cursor[b]++;
     bucket_eid[pos] = e;
-    bucket_pos[pos] = static_cast<uint16_t>(((row - r0) << 6) | (col & 63));
+    // byte offset of the element in the tile's shared-memory image: [128 rows x 64 bf16], rows of 128
+    // bytes whose 16-byte chunks are XOR-swizzled by (row & 7) (the layout the MMA descriptor reads)
+    const int rl = static_cast<int>(row - r0), cl = static_cast<int>(col & 63);
+    bucket_pos[pos] = static_cast<uint16_t>(rl * 128 + (((cl >> 3) ^ (rl & 7)) << 4) + (cl & 7) * 2);
   }
 }
 

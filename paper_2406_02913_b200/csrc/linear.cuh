@@ -22,7 +22,7 @@ struct szo_linear {
   int32_t* row_ptr;      // [N+1] entries of row r are [row_ptr[r], row_ptr[r+1])
   int32_t* bucket_ptr;   // [n_rowgroups * n_kblocks + 1]; bucket = (row/128, col/64)
   int32_t* bucket_eid;   // [nnz] entry id (index into S) in bucket order
-  uint16_t* bucket_pos;  // [nnz] (local_row << 6) | local_col in bucket order
+  uint16_t* bucket_pos;  // [nnz] byte offset of the element inside its swizzled [128 x 64] bf16 tile, bucket order
   int64_t n_rowgroups, n_kblocks;
   void* tc;              // tensor-core side data (tensor maps), owned; see gemm_tc.cu
 };
