@@ -394,7 +394,6 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
   const szo_model_config& c = m->cfg;
   const int64_t M = static_cast<int64_t>(B) * S;
   const int d = c.d_model, H = c.n_heads, Hkv = c.n_kv_heads, hd = d / H, ff = c.d_ff;
-  const int64_t dkv = static_cast<int64_t>(Hkv) * hd;
   const int act = c.act_dtype;
   const bool opt = c.arch == 1;
   T *a = static_cast<T*>(m->a), *q = static_cast<T*>(m->q), *k = static_cast<T*>(m->k), *v = static_cast<T*>(m->v),

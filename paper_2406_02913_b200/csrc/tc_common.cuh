@@ -1,5 +1,5 @@
-// Building blocks shared by the tensor-core kernels: tile constants, kernel parameters, the PTX
-// wrappers (mbarrier, TMA, cp.async, tcgen05 / TMEM), descriptor encoders and the int4 -> bf16
+// Building blocks of the tensor-core kernel and its host side: tile constants, kernel parameters,
+// the PTX wrappers (mbarrier, TMA, tcgen05 / TMEM), descriptor encoders and the int4 -> bf16
 // conversion of one 32-bit word of codes.
 #pragma once
 #include <cuda.h>
@@ -12,24 +12,19 @@ namespace tc {
 constexpr int kBM = 128;           // weight rows per tile (UMMA M)
 constexpr int kBK = 64;            // K per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int kUmmaK = 16;
-constexpr int kNumWarps = 16;
-constexpr int kDeqWarp0 = 4, kNumDeqWarps = 8;
-constexpr int kEpiWarp0 = 12;
 constexpr int kATileBytes = kBM * kBK * 2;   // 16 KiB
 constexpr int kCodesBytes = kBM * kBK / 2;   // 4 KiB of packed codes per stage
 constexpr int kSzBytes = 2048;               // (scale, zero) fp32 pairs: 128 rows x up to 2 groups
-constexpr int kLook = 4;                     // SparseAdd look-ahead in k-blocks
-constexpr int kRecSlots = 8, kRecCap = 128;  // ring of per-k-block sparse records in shared memory
-constexpr int kBoundSlots = 16;
+constexpr int kRecCap = 128;                 // sparse records of a k-block kept in the shared-memory ring
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s of SM cycles
 
-// One weight matrix of a fused launch (pair-tile kernel): several linear layers that read the same
-// activations (q/k/v, gate/up) are concatenated along their output rows.
+// One weight matrix of a launch: several linear layers that read the same activations (q/k/v,
+// gate/up) are concatenated along their output rows.
 struct TcSub {
-  const uint8_t* codes;    // tile order, as TcParams::codes
-  const float2* sz;
+  const uint8_t* codes;    // tile order: block (128-row tile t, k-block kb) = 4 KiB at (t * nkb + kb) * 4096
+  const float2* sz;        // [K/G][Npad]; fp32 (scale, zero), or packed bf16 pairs when kFast
   const int32_t* bucket_ptr;
-  const uint2* Sb;         // may be nullptr when the matrix has no sparse entries
+  const uint2* Sb;         // sparse records (byte offset in the tile, value bits) in bucket order; nullptr: none
   const float* bias;
   void* y;
   int64_t N, Npad;
@@ -38,22 +33,12 @@ struct TcSub {
 };
 
 struct TcParams {
-  int64_t M, N, K;
+  int64_t M, K;
   int G;
   int nkb;                 // K / 64
-  int64_t m_tiles, n_tiles;
-  const uint8_t* codes;    // tile order: block (128-row tile t, k-block kb) = 4 KiB at (t * nkb + kb) * 4096
-  const float2* sz;        // [K/G][Npad]; fp32 (scale, zero), or packed bf16 pairs when kFast
-  int64_t Npad;
-  const int32_t* bucket_ptr;
-  int64_t n_kblocks;       // buckets per 128-row tile
-  int64_t n_rowtiles;      // number of 128-row tiles that have buckets
-  const uint2* Sb;         // sparse records (position in tile, value bits) in bucket order; nullptr: none
-  const float* bias;
-  void* y;
+  int64_t m_tiles, n_tiles;   // 256-token tiles; 256-row pair tiles of all matrices together
   int y_f32;
   int32_t* status;
-  // ---- pair-tile kernel only
   int nsub;
   TcSub sub[3];
   // Work units of pair p: full tiles p + lt * n_pairs for lt < full_rounds, then (p < tail_tiles *
@@ -114,11 +99,6 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
       : "memory");
   return ok;
 }
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
 // Bounded wait: false when the limit expired or another role already gave up.  Between polls the
 // warp sleeps for `backoff_ns` so that waiting roles do not take issue slots from the few threads
 // that feed the tensor core; the SM cycle counter bounds the wait (kWaitLimitCycles is about two
@@ -152,40 +132,9 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint
                "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
                : "memory");
 }
-__device__ __forceinline__ void cp_async_4(uint32_t dst, const void* src) {
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_8(uint32_t dst, const void* src) {
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait_group() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void tmem_alloc(uint32_t result_smem, uint32_t ncols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(result_smem), "r"(ncols)
-               : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                          uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
