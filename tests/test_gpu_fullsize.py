@@ -1,5 +1,5 @@
-"""Parity at the benchmark's full sizes, in the launch configuration bench.py times: the fused
-linear at the Llama-2-7B shapes (M = 4096 tokens) and the sparse passes at k = 6.48 M, checked on
+"""Parity at full sizes, in the launch configuration bench.py times: the fused linear at the
+Llama-2-7B, Mistral-7B and OPT-13B shapes (M = 4096 tokens) and the sparse passes at k = 6.48 M, checked on
 sampled outputs that the oracle computes one by one (a full fp64 product would take minutes)."""
 import numpy as np
 import pytest
@@ -22,21 +22,35 @@ def _bf16_bits(t):
     return t.cpu().view(torch.int16).numpy().view(np.uint16)
 
 
-@pytest.mark.parametrize("N,K,mode", [(4096, 4096, "sparse_add"), (11008, 4096, "sparse_add"), (4096, 11008, "sparse_add"),
-                                      (4096, 4096, "spmm")])
-def test_llama7b_linear_sampled_outputs(B, N, K, mode):
-    M, G, rho = 4096, 128, 1e-3
+@pytest.mark.parametrize("N,K,G,rho,bias,mode", [
+    # Llama-2-7B shapes, int4 G=128, 0.1 % mask
+    (4096, 4096, 128, 1e-3, False, "sparse_add"), (11008, 4096, 128, 1e-3, False, "sparse_add"),
+    (4096, 11008, 128, 1e-3, False, "sparse_add"), (4096, 4096, 128, 1e-3, False, "spmm"),
+    # Mistral-7B shapes, dense bf16 weights, 1 % mask (k/v projections are 1024 wide: GQA)
+    (14336, 4096, 0, 1e-2, False, "sparse_add"), (4096, 14336, 0, 1e-2, False, "sparse_add"),
+    (1024, 4096, 0, 1e-2, False, "sparse_add"),
+    # OPT-13B shapes, int4 G=128, 0.1 % mask, biases
+    (5120, 5120, 128, 1e-3, True, "sparse_add"), (20480, 5120, 128, 1e-3, True, "sparse_add"),
+    (5120, 20480, 128, 1e-3, True, "sparse_add"),
+])
+def test_full_size_linear_sampled_outputs(B, N, K, G, rho, bias, mode):
+    M = 4096
     g = torch.Generator(device="cuda")
     g.manual_seed(N * 7 + K)
-    codes = torch.randint(0, 256, (N, K // 2), generator=g, device="cuda", dtype=torch.uint8)
-    sc = (0.004 + 0.002 * torch.rand(N, K // G, generator=g, device="cuda")).to(torch.bfloat16)
-    ze = (-7.5 * sc.float()).to(torch.bfloat16)
+    if G > 0:
+        codes = torch.randint(0, 256, (N, K // 2), generator=g, device="cuda", dtype=torch.uint8)
+        sc = (0.004 + 0.002 * torch.rand(N, K // G, generator=g, device="cuda")).to(torch.bfloat16)
+        ze = (-7.5 * sc.float()).to(torch.bfloat16)
+    else:
+        codes = (torch.randn(N, K, generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+        sc = ze = None
     nnz = int(rho * N * K)
     idx_np = wl.sorted_random_indices(N * K, nnz, seed=N + K)
     idx = torch.from_numpy(idx_np).cuda()
     S = (torch.randn(nnz, generator=g, device="cuda") * 0.02).contiguous()
     x = torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16)
-    plan = B.Linear(N, K, G, codes, sc, ze, "bf16", idx)
+    b = (torch.randn(N, generator=g, device="cuda") * 0.02) if bias else None
+    plan = B.Linear(N, K, G, codes, sc, ze, "bf16", idx, b)
     md = B.MODE_SPARSE_ADD if mode == "sparse_add" else B.MODE_SPMM
     y = plan.fwd(x, S, md, torch.float32)
     torch.cuda.synchronize()
@@ -46,14 +60,18 @@ def test_llama7b_linear_sampled_outputs(B, N, K, mode):
     r = wl.rng(5, wl.PURPOSE_INDICES, N + K)
     rows = np.unique(np.concatenate([r.integers(0, N, 24), [0, 127, 128, N - 129, N - 1]]))
     toks = np.unique(np.concatenate([r.integers(0, M, 24), [0, 255, 256, M - 257, M - 1]]))
-    codes_h = codes[rows].cpu().numpy()
-    deq = so.dequantize(codes_h, _bf16_bits(sc[rows]), _bf16_bits(ze[rows]), G, "bf16")       # [rows, K] fp64
+    if G > 0:
+        deq = so.dequantize(codes[rows].cpu().numpy(), _bf16_bits(sc[rows]), _bf16_bits(ze[rows]), G, "bf16")   # [rows, K] fp64
+    else:
+        deq = codes[rows].float().cpu().numpy().astype(np.float64)
     S_h = S.cpu().numpy().astype(np.float64)
     for i, n in enumerate(rows):
         lo, hi = np.searchsorted(idx_np, [n * K, (n + 1) * K])
         np.add.at(deq[i], idx_np[lo:hi] - n * K, S_h[lo:hi])
     xs = x[toks].float().cpu().numpy().astype(np.float64)
     ref = xs @ deq.T                                                                          # [toks, rows]
+    if bias:
+        ref = ref + b[rows].cpu().numpy().astype(np.float64)[None, :]
     got = y[toks][:, rows].cpu().numpy().astype(np.float64)
     scale = np.max(np.abs(ref))
     assert np.max(np.abs(got - ref)) <= 2e-2 * scale
