@@ -4,7 +4,7 @@
 // The loss path needs attention only as one block of the black-box loss f (Definition 1); it is a
 // few percent of a step's flops, so the legacy warp-level MMA is enough here and the tcgen05
 // machinery is kept for the linears.  One CTA = 64 queries of one (batch, head); 4 warps x 16 rows;
-// K/V tiles of 64 keys staged in padded shared memory; online softmax; grouped-query attention by
+// K/V tiles of 64 keys double-buffered in padded shared memory (cp.async); online softmax; grouped-query attention by
 // mapping query head h to KV head h / (H / Hkv).  q, k, v, o are [B*S, heads*HD] bf16 row-major.
 #include "common.cuh"
 
@@ -64,14 +64,16 @@ __device__ __forceinline__ void load_tile_async(__nv_bfloat16* dst, const __nv_b
 }
 
 template <int HD>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, 3)
 flash_attn_bf16_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                        const __nv_bfloat16* __restrict__ v, __nv_bfloat16* __restrict__ o, int S, int H, int Hkv,
                        float scale_log2e) {
   constexpr int LDS = HD + 8;
   extern __shared__ __align__(16) unsigned char smem_attn[];
-  __nv_bfloat16* sQ = reinterpret_cast<__nv_bfloat16*>(smem_attn);
-  __nv_bfloat16* sKV = sQ + kQT * LDS;          // two stages of (K tile, V tile)
+  // two stages of (K tile, V tile); the query tile first sits in stage 1's K slot and is moved to
+  // registers before that stage is filled (4 tiles of shared memory: three CTAs per SM)
+  __nv_bfloat16* sKV = reinterpret_cast<__nv_bfloat16*>(smem_attn);
+  __nv_bfloat16* sQ = sKV + 2 * kKT * LDS;
 
   // heavy query tiles (many key tiles) are scheduled first
   const int qt = gridDim.x - 1 - blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
@@ -81,7 +83,19 @@ flash_attn_bf16_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16*
   const int64_t ldq = static_cast<int64_t>(H) * HD, ldk = static_cast<int64_t>(Hkv) * HD;
   const int q0 = qt * kQT;
   const __nv_bfloat16* qbase = q + (static_cast<int64_t>(b) * S + q0) * ldq + hq * HD;
-  load_tile<HD>(sQ, qbase, ldq, S - q0 < kQT ? S - q0 : kQT);
+  auto issue_kv = [&](int kt) {                 // K and V tile kt into stage kt & 1
+    const int k0 = kt * kKT;
+    const int valid = S - k0 < kKT ? S - k0 : kKT;
+    __nv_bfloat16* dK = sKV + (kt & 1) * 2 * kKT * LDS;
+    load_tile_async<HD>(dK, k + (static_cast<int64_t>(b) * S + k0) * ldk + hk * HD, ldk, valid);
+    load_tile_async<HD>(dK + kKT * LDS, v + (static_cast<int64_t>(b) * S + k0) * ldk + hk * HD, ldk, valid);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  // the query tile and the first K/V tile travel together: one global-memory latency for both
+  load_tile_async<HD>(sQ, qbase, ldq, S - q0 < kQT ? S - q0 : kQT);
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  issue_kv(0);
+  asm volatile("cp.async.wait_group 1;" ::: "memory");          // the query tile has landed
   __syncthreads();
 
   // this warp's 16 query rows as A fragments, kept in registers
@@ -99,15 +113,7 @@ flash_attn_bf16_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16*
   float mrow[2] = {-INFINITY, -INFINITY}, lrow[2] = {0.f, 0.f};
   const int row_a = q0 + warp * 16 + g, row_b = row_a + 8;     // the two query rows of this thread
 
-  auto issue_kv = [&](int kt) {                 // K and V tile kt into stage kt & 1
-    const int k0 = kt * kKT;
-    const int valid = S - k0 < kKT ? S - k0 : kKT;
-    __nv_bfloat16* dK = sKV + (kt & 1) * 2 * kKT * LDS;
-    load_tile_async<HD>(dK, k + (static_cast<int64_t>(b) * S + k0) * ldk + hk * HD, ldk, valid);
-    load_tile_async<HD>(dK + kKT * LDS, v + (static_cast<int64_t>(b) * S + k0) * ldk + hk * HD, ldk, valid);
-    asm volatile("cp.async.commit_group;" ::: "memory");
-  };
-  issue_kv(0);
+  __syncthreads();                              // every warp holds its query fragments: stage 1 is free
   for (int kt = 0; kt <= qt; ++kt) {
     const int k0 = kt * kKT;
     const int valid = S - k0 < kKT ? S - k0 : kKT;
@@ -228,7 +234,7 @@ szo_status launch_flash_attention_bf16(const void* q, const void* k, const void*
   SZO_REQUIRE(hd == 64 || hd == 128, SZO_ERR_UNSUPPORTED, "head dimension must be 64 or 128");
   const float scale_log2e = 1.4426950408889634f / sqrtf(static_cast<float>(hd));
   dim3 grid(static_cast<unsigned>(ceil_div(S, kQT)), H, B);
-  const size_t smem = static_cast<size_t>(5) * 64 * (hd + 8) * 2;      // Q + two (K, V) stages
+  const size_t smem = static_cast<size_t>(4) * 64 * (hd + 8) * 2;      // two (K, V) stages; Q borrows one slot
   auto* qb = static_cast<const __nv_bfloat16*>(q);
   auto* kb = static_cast<const __nv_bfloat16*>(k);
   auto* vb = static_cast<const __nv_bfloat16*>(v);

@@ -126,6 +126,26 @@ def sparse_case(k, reps, n_total=12_582_912_000):
     return line
 
 
+def cold_case(N, K, G, reps):
+    """The two one-off steps: szo_quantize of one [N, K] fp32 weight and szo_select_mask of its
+    N*K scores (k = 0.1 %).  Reported, not part of the step."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(3)
+    W = torch.randn(N, K, generator=g, device="cuda") * 0.02
+    hbm, _, src = peaks()
+    med, _ = time_call(lambda: B.szo_quantize(W, G, "bf16"), reps)
+    q_bytes = 4.0 * N * K + 0.5 * N * K + 4.0 * N * K / G
+    scores = (W * W).reshape(-1).contiguous()
+    k = N * K // 1000
+    med_s, _ = time_call(lambda: B.szo_select_mask(scores, k), reps)
+    line = {"case": "cold", "N": N, "K": K, "G": G, "peaks": src,
+            "quantize": {"ms_median": med, "gbs": q_bytes / (med * 1e-3) / 1e9, "frac_hbm": q_bytes / (med * 1e-3) / 1e9 / hbm},
+            "select_mask": {"ms_median": med_s, "n": N * K, "k": k,
+                            "gbs_one_pass_equivalent": 4.0 * N * K / (med_s * 1e-3) / 1e9}}
+    print(json.dumps(line), flush=True)
+    return line
+
+
 def attention_case(Bn, S, H, Hkv, hd, reps):
     g = torch.Generator(device="cuda")
     g.manual_seed(1)
@@ -166,6 +186,8 @@ def main():
             linear_case(4096, N, K, 128, "sparse_add", 1e-3, a.reps)
         for k in (100_000, 1_000_000, 6_476_005, 12_582_912, 100_000_000):
             sparse_case(k, a.reps)
+        cold_case(11008, 4096, 128, a.reps)
+        attention_case(16, 256, 32, 32, 128, a.reps)
 
 
 if __name__ == "__main__":
