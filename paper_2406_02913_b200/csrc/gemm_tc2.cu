@@ -38,7 +38,7 @@ using namespace tc;
 
 constexpr int kPairBT = 256;                 // tokens per pair tile (UMMA N)
 constexpr int kXHalfBytes = 128 * kBK * 2;   // this CTA's half of the token tile: 16 KiB
-constexpr int kCStages2 = 6;
+constexpr int kCStages2 = 8;
 constexpr int kASlots2 = 6;
 // 20 warps: four single-thread roles, three groups of four conversion warps, four epilogue warps.
 // Warp w issues on scheduler w % 4.  The single-thread roles (warps 0, 4, 8, 12) share scheduler 0
@@ -694,8 +694,8 @@ szo_status launch_tc2(const CUtensorMap& mx, const CUtensorMap& mw, const TcPara
 szo_status launch_pair_kernel(bool dequant, bool bf16_tables, const CUtensorMap& mx, const CUtensorMap& mw,
                               const tc::TcParams& P, int n_pairs, cudaStream_t st) {
   if (!dequant) return launch_tc2<6, false, false>(mx, mw, P, n_pairs, st);
-  if (bf16_tables) return launch_tc2<5, true, true>(mx, mw, P, n_pairs, st);
-  return launch_tc2<5, true, false>(mx, mw, P, n_pairs, st);
+  if (bf16_tables) return launch_tc2<4, true, true>(mx, mw, P, n_pairs, st);
+  return launch_tc2<4, true, false>(mx, mw, P, n_pairs, st);
 }
 
 }  // namespace szo
