@@ -63,6 +63,10 @@ CASES = [
     (384, 512, 128, "bf16", 300, 1e-2, True),       # several tiles and a ragged tail in M and N
     (200, 320, 32, "bf16", 65, 5e-3, False),        # N not a multiple of the tile
     (256, 512, 0, "bf16", 130, 1e-2, False),        # dense bf16 weight (no quantization)
+    (128, 64, 64, "bf16", 1, 1e-2, True),           # one token, one k-block
+    (512, 4096, 128, "bf16", 16, 1e-3, False),      # few tiles, long K: every tile split along K in four parts
+    (300, 4160, 64, "f16", 257, 2e-3, True),        # K-split parts of unequal length, ragged N and M
+    (256, 256, 64, "bf16", 200, 5e-2, False),       # dense mask: buckets larger than the record ring
 ]
 
 
@@ -72,7 +76,8 @@ def test_fp32_validation_mode(B, N, K, G, fmt, M, rho, bias):
     plan, x, S = upload(B, c)
     ref = so.linear_fwd(c["x"], c["deq"], c["idx"], c["S"], c["bias"])
     y = plan.fwd(x, S, B.MODE_FP32_VALIDATE, torch.float32).cpu().numpy()
-    assert max_rel(y, ref) < 2e-6
+    # fp32 accumulation of K products: a random walk of roundings, 4 * 2^-24 * sqrt(K) bounds it with margin
+    assert max_rel(y, ref) < 4 * 2.0 ** -24 * np.sqrt(K)
     y16 = plan.fwd(x.to(torch.bfloat16), S, B.MODE_FP32_VALIDATE, torch.bfloat16).float().cpu().numpy()
     assert max_rel(y16, ref) < 4e-3                                    # only the output rounding
     plan.close()
@@ -94,6 +99,25 @@ def test_tensor_core_modes(B, N, K, G, fmt, M, rho, bias, mode):
     # determinism: bitwise-same output on a second launch
     y2 = plan.fwd(xb, S, md, torch.float32).cpu().numpy()
     assert np.array_equal(y, y2)
+    assert B.device_status() == 0
+    plan.close()
+
+
+def test_k_split_does_not_depend_on_the_scratch_contents(B):
+    """Tiles split along K meet in the caller's workspace; whatever it held before must not matter,
+    and two launches give the same bits."""
+    c = make_case(512, 4096, 128, "bf16", 48, 1e-3, seed=11)
+    plan, x, S = upload(B, c)
+    xb = x.to(torch.bfloat16)
+    y1 = plan.fwd(xb, S, B.MODE_SPARSE_ADD, torch.float32).clone()
+    assert plan._ws is not None and plan._ws.numel() > c["idx"].size * 8 + 4096      # records + split scratch
+    plan._ws.fill_(0x7F)
+    y2 = plan.fwd(xb, S, B.MODE_SPARSE_ADD, torch.float32).clone()
+    plan._ws.zero_()
+    y3 = plan.fwd(xb, S, B.MODE_SPARSE_ADD, torch.float32)
+    assert torch.equal(y1, y2) and torch.equal(y1, y3)
+    ref = so.linear_fwd(xb.float().cpu().numpy(), c["deq"], c["idx"], c["S"], c["bias"])
+    assert max_rel(y1.cpu().numpy(), ref) <= LINEAR_TOL
     assert B.device_status() == 0
     plan.close()
 
