@@ -208,6 +208,142 @@ szo_status linear_fwd_tc_group(const szo_linear* const* plans, int n, const void
   return launch_pair_kernel(p0->G != 0, p0->sz_dtype == SZO_BF16, mx, t->w_map, P, sc.n_pairs, st);
 }
 
+// ------------------------------------------------------------------------------ materialised form
+// For many tokens the appendix's DenseMM(SparseAdd(w_sparse, Dequantize(Q(w_dense))), x) is cheaper
+// taken literally: one pass writes the effective weight RN_bf16(q*scale+zero), RN_bf16(. + S) at the
+// masked positions, as a bf16 matrix into scratch (2.5 bytes per weight of HBM traffic), and the
+// tensor-core kernel runs in its dense mode, where no conversion competes with the MMAs for issue
+// slots.  The values are bit-identical to what the fused mode builds in shared memory.
+namespace {
+
+// thread -> one 32-bit word of the tile-ordered codes (8 weights) -> 16 bytes of the row-major output
+template <bool kFast>
+__global__ void materialise_kernel(const uint8_t* __restrict__ codes_tiled, const float2* __restrict__ sz, int64_t Npad,
+                                   int nkb, int G, __nv_bfloat16* __restrict__ out, int64_t K) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= (Npad / kBM) * nkb * 1024) return;
+  const int chunk = static_cast<int>(i & 7), r = static_cast<int>((i >> 3) & 127);
+  const int64_t blk = i >> 10;
+  const int64_t t = blk / nkb;
+  const int kb = static_cast<int>(blk - t * nkb);
+  const uint32_t w = *reinterpret_cast<const uint32_t*>(codes_tiled + blk * kCodesBytes + r * 32 + chunk * 4);
+  const int g = (kb * kBK + chunk * 8) / G;
+  const float2 p = sz[static_cast<int64_t>(g) * Npad + t * kBM + r];
+  *reinterpret_cast<uint4*>(out + (t * kBM + r) * K + kb * kBK + chunk * 8) = dequant_word<kFast>(w, p);
+}
+
+// SparseAdd on the materialised matrix: indices are unique, so no two threads touch one element
+__global__ void scatter_add_bf16_kernel(__nv_bfloat16* __restrict__ w, const int64_t* __restrict__ idx,
+                                        const float* __restrict__ S, int64_t nnz) {
+  const int64_t e = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (e >= nnz) return;
+  __nv_bfloat16* el = w + idx[e];
+  *el = __float2bfloat16_rn(__bfloat162float(*el) + S[e]);
+}
+
+// SZO_LINEAR_MATERIALISE=0 / 1 switches the form off / on for every M (A/B measurement)
+int materialise_override() {
+  static const int v = [] {
+    const char* e = getenv("SZO_LINEAR_MATERIALISE");
+    return e == nullptr ? -1 : (e[0] == '0' ? 0 : 1);
+  }();
+  return v;
+}
+
+}  // namespace
+
+bool tc_use_materialised(const szo_linear* p, int64_t M) {
+  if (p->G == 0 || p->tc == nullptr) return false;
+  const int o = materialise_override();
+  if (o >= 0) return o == 1;
+  // the extra pass costs about 2.5 N K bytes of traffic, the fused conversion 5-10 % of 2 M N K flop at
+  // the kernel's rate: measured break-even near M = 2048 (4096^2: 73 vs 75 us), 7 % ahead at M = 4096
+  return M >= 4096;
+}
+
+size_t tc_materialised_ws_bytes(const szo_linear* const* plans, int n, int64_t M) {
+  size_t rows = 0;
+  for (int i = 0; i < n; ++i) rows += static_cast<size_t>(plans[i]->Npad);
+  return round_up(rows * static_cast<size_t>(plans[0]->K) * sizeof(__nv_bfloat16), 256) + tc_tail_ws_bound();
+}
+
+// n matrices that share x (n == 1 or tc_can_fuse): materialise, SparseAdd, dense launch.
+szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, const void* x, int64_t M,
+                                      const float* const* S_pert, void* const* y, int y_dtype, void* ws,
+                                      size_t ws_bytes, cudaStream_t st) {
+  const szo_linear* p0 = plans[0];
+  const TcPlan* t = static_cast<const TcPlan*>(p0->tc);
+  SZO_REQUIRE(t != nullptr, SZO_ERR_INVALID_ARG, "plan has no tensor-core data");
+  SZO_REQUIRE(M < (int64_t(1) << 31), SZO_ERR_SHAPE, "M too large");
+  int64_t rows = 0;
+  for (int i = 0; i < n; ++i) rows += plans[i]->Npad;
+  const size_t w_bytes = round_up(static_cast<size_t>(rows) * p0->K * sizeof(__nv_bfloat16), 256);
+  SZO_REQUIRE(ws != nullptr && ws_bytes >= w_bytes, SZO_ERR_WORKSPACE,
+              "the materialised form needs a workspace of at least %zu bytes", w_bytes);
+  SZO_REQUIRE(rows < (int64_t(1) << 31), SZO_ERR_SHAPE, "too many weight rows in one launch");
+  __nv_bfloat16* W = static_cast<__nv_bfloat16*>(ws);
+  const int nkb = static_cast<int>(p0->K / kBK);
+  int64_t row0 = 0;
+  for (int i = 0; i < n; ++i) {
+    const szo_linear* p = plans[i];
+    const int64_t words = (p->Npad / kBM) * nkb * 1024;
+    __nv_bfloat16* Wi = W + row0 * p->K;
+    if (p->sz_dtype == SZO_BF16)
+      materialise_kernel<true><<<static_cast<unsigned>(ceil_div(words, 256)), 256, 0, st>>>(p->codes_tiled, p->sz, p->Npad, nkb,
+                                                                                         p->G, Wi, p->K);
+    else
+      materialise_kernel<false><<<static_cast<unsigned>(ceil_div(words, 256)), 256, 0, st>>>(p->codes_tiled, p->sz, p->Npad, nkb,
+                                                                                          p->G, Wi, p->K);
+    count_launch();
+    if (p->nnz > 0) {
+      scatter_add_bf16_kernel<<<static_cast<unsigned>(ceil_div(p->nnz, 256)), 256, 0, st>>>(Wi, p->idx, S_pert[i], p->nnz);
+      count_launch();
+    }
+    row0 += p->Npad;
+  }
+  SZO_CHECK_LAUNCH("materialise_kernel");
+  CUtensorMap mx, mw;
+  SZO_TRY(make_map(&mx, x, M, p0->K, 128));
+  SZO_TRY(make_map(&mw, W, rows, p0->K, kBM));
+  TcParams P{};
+  P.M = M; P.K = p0->K; P.G = 0; P.nkb = nkb;
+  P.m_tiles = ceil_div(M, 256);
+  P.nsub = n;
+  int64_t n_tiles = 0;
+  for (int i = 0; i < n; ++i) {
+    const szo_linear* p = plans[i];
+    TcSub& sb = P.sub[i];
+    sb.codes = nullptr;
+    sb.sz = nullptr;
+    sb.bucket_ptr = nullptr;
+    sb.Sb = nullptr;
+    sb.bias = p->bias;
+    sb.y = y[i];
+    sb.N = p->N;
+    sb.Npad = p->Npad;
+    sb.n_rowtiles = 0;
+    sb.n_tiles = static_cast<int>(p->Npad / 256);     // the buffer pads every matrix to whole pair tiles
+    n_tiles += sb.n_tiles;
+  }
+  P.n_tiles = n_tiles;
+  P.y_f32 = (y_dtype == SZO_F32) ? 1 : 0;
+  P.status = device_status_word();
+  SZO_REQUIRE(P.status != nullptr, SZO_ERR_CUDA, "no device status word");
+  const int64_t tiles = P.m_tiles * P.n_tiles;
+  SZO_REQUIRE(tiles < (int64_t(1) << 30), SZO_ERR_SHAPE, "too many tiles");
+  void* tail = static_cast<unsigned char*>(ws) + w_bytes;
+  const size_t tail_bytes = ws_bytes - w_bytes;
+  PairSchedule sc = pair_schedule(tiles, P.nkb, 0, t->sms, true);
+  if (sc.ws_bytes > tail_bytes) sc = pair_schedule(tiles, P.nkb, 0, t->sms, false);
+  P.full_rounds = sc.full_rounds;
+  P.tail_tiles = sc.tail_tiles;
+  P.tail_parts = sc.tail_parts;
+  for (int i = 0; i < 5; ++i) P.tail_kb[i] = sc.tail_kb[i];
+  P.partial = static_cast<float*>(tail);
+  P.tickets = t->tickets;
+  return launch_pair_kernel(false, false, mx, mw, P, sc.n_pairs, st);
+}
+
 szo_status linear_fwd_tc(const szo_linear* p, const void* x, int64_t M, const uint2* S_bucket, void* y,
                          int y_dtype, void* ws, size_t ws_bytes, cudaStream_t st) {
   return linear_fwd_tc_group(&p, 1, x, M, &S_bucket, &y, y_dtype, ws, ws_bytes, st);

@@ -100,6 +100,7 @@ __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
 // tile n_tile of that matrix, token tile m_tile).
 struct Unit {
   int s, n_tile, m_tile, kb0, kb1, part, parts, slot;
+  int g_tile;      // 128-row tile counted over all matrices of the launch (rows of a shared dense weight buffer)
 };
 __device__ __forceinline__ int tail_kb_at(const TcParams& P, int i) {
   return i == 0 ? P.tail_kb[0] : i == 1 ? P.tail_kb[1] : i == 2 ? P.tail_kb[2] : i == 3 ? P.tail_kb[3] : P.tail_kb[4];
@@ -125,6 +126,7 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& P, int pair, int n_p
   const int m_tiles = static_cast<int>(P.m_tiles);
   int np = tile / m_tiles;
   u.m_tile = tile - np * m_tiles;
+  u.g_tile = np * 2 + rank;
   u.s = 0;
   if (P.nsub > 1 && np >= P.sub[0].n_tiles) {
     np -= P.sub[0].n_tiles;
@@ -309,7 +311,7 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
       for (int lt = 0; lt < my_units && ok; ++lt) {
         const Unit u = decode_unit(P, pair, n_pairs, rank, lt);
         const int tok0 = u.m_tile * kPairBT + rank * 128;
-        const int row0 = u.n_tile * kBM;
+        const int row0 = u.g_tile * kBM;   // dense weights of a launch are one buffer, each matrix padded to 256 rows
         for (int kb = u.kb0; kb < u.kb1; ++kb) {
           if (!mbar_wait(xempty_bar(x.idx), x.phase ^ 1u, abort_flag, P.status)) { ok = false; break; }
           mbar_expect_tx(xfull_bar(x.idx), kXStageBytes);

@@ -351,6 +351,8 @@ szo_status linear_fwd_impl(const szo_linear* p, const void* x, int x_dtype, int6
     SZO_TRY(linear_fwd_tc(p, x, M, nullptr, y, y_dtype, workspace, workspace_bytes, st));
     return linear_spmm(p, x, M, S_pert, y, y_dtype, st);
   }
+  if (tc_use_materialised(p, M))
+    return linear_fwd_tc_materialised(&p, 1, x, M, &S_pert, &y, y_dtype, workspace, workspace_bytes, st);
   unsigned char* ws = static_cast<unsigned char*>(workspace);
   if (p->nnz > 0 && S_bucket == nullptr) {
     const size_t need = round_up(static_cast<size_t>(p->nnz) * sizeof(uint2), 256);
@@ -485,6 +487,7 @@ size_t szo_linear_workspace_bytes(const szo_linear_t* p, int64_t M, int32_t mode
   const szo_linear* pp = p;
   const size_t tail = tc_tail_ws_bytes(&pp, 1, M);                     // K-split tiles of the last round
   if (mode == SZO_MODE_SPMM) return tail;
+  if (tc_use_materialised(p, M)) return tc_materialised_ws_bytes(&pp, 1, M);
   return round_up(static_cast<size_t>(p->nnz) * sizeof(uint2), 256) + tail;   // + bucket-ordered sparse records
 }
 

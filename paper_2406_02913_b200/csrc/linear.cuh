@@ -56,6 +56,13 @@ szo_status linear_fwd_tc_group(const szo_linear* const* plans, int n, const void
                                cudaStream_t st);
 size_t tc_tail_ws_bytes(const szo_linear* const* plans, int n, int64_t M);
 size_t tc_tail_ws_bound();   // enough for any M and any group
+// Materialised form (gemm_tc.cu): the effective bf16 weight is written to scratch, then the dense
+// mode of the kernel runs.  Chosen for int4 plans when M is large (tc_use_materialised).
+bool tc_use_materialised(const szo_linear* p, int64_t M);
+size_t tc_materialised_ws_bytes(const szo_linear* const* plans, int n, int64_t M);
+szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, const void* x, int64_t M,
+                                      const float* const* S_pert, void* const* y, int y_dtype, void* ws,
+                                      size_t ws_bytes, cudaStream_t st);
 // out[p] = (pos[p], bits of S[eid[p]]) for p in [0, n)
 szo_status gather_values(const float* S, const int32_t* eid, const uint16_t* pos, int64_t n, uint2* out,
                          cudaStream_t st);

@@ -432,6 +432,9 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
       for (int i = 0; i < n; ++i) SZO_TRY(lin(layer, j0 + i, x, outs[i]));
       return SZO_OK;
     }
+    const bool mat = tc_use_materialised(plans[0], M);
+    const float* spert[3];
+    for (int i = 0; i < n; ++i) spert[i] = Sv + m->offsets[t0 + i];
     if (m->timing) {
       while (m->events.size() < m->events_used + 2) {
         cudaEvent_t e;
@@ -440,7 +443,8 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
       }
       SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used], st));
     }
-    const szo_status rc = linear_fwd_tc_group(plans, n, x, M, recs, outs, act, m->ws, m->ws_bytes, st);
+    const szo_status rc = mat ? linear_fwd_tc_materialised(plans, n, x, M, spert, outs, act, m->ws, m->ws_bytes, st)
+                              : linear_fwd_tc_group(plans, n, x, M, recs, outs, act, m->ws, m->ws_bytes, st);
     if (m->timing) {
       SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used + 1], st));
       m->events_used += 2;
@@ -452,7 +456,8 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
                                                         c.vocab, m->h);
   count_launch();
   // One gather of all sparse values into the bucket order of every linear (SparseAdd mode)
-  if (pregather) SZO_TRY(gather_values(Sv, m->geid, m->gpos, m->k_total, m->recs, st));
+  if (pregather && !(m->plans.size() > 0 && tc_use_materialised(m->plans[0], M)))
+    SZO_TRY(gather_values(Sv, m->geid, m->gpos, m->k_total, m->recs, st));
   const T* pending = nullptr;     // projection output still to be added to the residual stream
   for (int l = 0; l < c.n_layers; ++l) {
     const szo_layer_weights& L = m->layers[l];
@@ -600,6 +605,21 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
     // K-split scratch of the pair-tile kernel: at most one 256 x 256 fp32 tile per cluster
     const size_t need = tc_tail_ws_bound();
     if (need > ws_need) ws_need = need;
+    // scratch of the materialised form: the largest group of layers that share their input
+    if (tc_use_materialised(m->plans[0], m->Mmax)) {
+      for (int l = 0; l < c.n_layers; ++l) {
+        const szo_linear* const* pl = m->plans.data() + static_cast<size_t>(l) * m->n_lin;
+        const size_t g0 = tc_materialised_ws_bytes(pl, 3, m->Mmax);                       // q, k, v
+        const size_t g1 = c.arch == 0 ? tc_materialised_ws_bytes(pl + 4, 2, m->Mmax) : 0;  // gate, up
+        size_t g2 = 0;
+        for (int j = 0; j < m->n_lin; ++j) {
+          const size_t one = tc_materialised_ws_bytes(pl + j, 1, m->Mmax);
+          if (one > g2) g2 = one;
+        }
+        const size_t mx = g0 > g1 ? (g0 > g2 ? g0 : g2) : (g1 > g2 ? g1 : g2);
+        if (mx > ws_need) ws_need = mx;
+      }
+    }
   }
   m->k_total = m->offsets.back();
   if (m->k_total > 0 && S_all == nullptr) return bail(fail(SZO_ERR_INVALID_ARG, "S_all is NULL"));

@@ -122,6 +122,22 @@ def test_k_split_does_not_depend_on_the_scratch_contents(B):
     plan.close()
 
 
+def test_materialised_and_fused_forms_give_the_same_bits(B):
+    """M >= 4096 tokens take the materialised form (effective bf16 weight written to scratch, dense
+    kernel), fewer tokens the fused form; both build the same bf16 weights and accumulate in the
+    same order (K = 512: no tile is split along K), so the rows they share are bit-identical."""
+    c = make_case(1024, 512, 64, "bf16", 4096, 2e-3, seed=13, bias=True)
+    plan, x, S = upload(B, c)
+    xb = x.to(torch.bfloat16)
+    y_mat = plan.fwd(xb, S, B.MODE_SPARSE_ADD, torch.float32).clone()
+    y_fused = plan.fwd(xb[:2000], S, B.MODE_SPARSE_ADD, torch.float32)
+    assert torch.equal(y_mat[:2000], y_fused)
+    ref = so.linear_fwd(xb.float().cpu().numpy(), c["deq"], c["idx"], c["S"], c["bias"])
+    assert max_rel(y_mat.cpu().numpy(), ref) <= LINEAR_TOL
+    assert B.device_status() == 0
+    plan.close()
+
+
 def test_special_cases_identity_input_and_sparse_only(B):
     # x = I returns W_eff^T tile by tile (exposes layout mistakes); zero codes leave the sparse term
     N, K, G = 256, 256, 64
