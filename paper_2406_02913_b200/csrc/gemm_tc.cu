@@ -216,28 +216,54 @@ szo_status linear_fwd_tc_group(const szo_linear* const* plans, int n, const void
 // slots.  The values are bit-identical to what the fused mode builds in shared memory.
 namespace {
 
+// Up to three matrices (the layers of one launch) per kernel call.
+struct MatSub {
+  const uint8_t* codes_tiled;
+  const float2* sz;
+  int64_t Npad;
+  __nv_bfloat16* out;         // [Npad, K] row-major
+  const int64_t* idx;         // sparse entries: flat indices n * K + c, values S
+  const float* S;
+  int64_t words_end, nnz_end; // running totals over the matrices: work items of this and the earlier ones
+};
+struct MatArgs {
+  MatSub sub[3];
+  int n, nkb, G;
+  int64_t K;
+};
+
 // thread -> one 32-bit word of the tile-ordered codes (8 weights) -> 16 bytes of the row-major output
 template <bool kFast>
-__global__ void materialise_kernel(const uint8_t* __restrict__ codes_tiled, const float2* __restrict__ sz, int64_t Npad,
-                                   int nkb, int G, __nv_bfloat16* __restrict__ out, int64_t K) {
-  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (i >= (Npad / kBM) * nkb * 1024) return;
+__global__ void materialise_kernel(const MatArgs a) {
+  int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= a.sub[a.n - 1].words_end) return;
+  int s = 0;
+  if (i >= a.sub[0].words_end) s = (a.n > 2 && i >= a.sub[1].words_end) ? 2 : 1;
+  if (s > 0) i -= a.sub[s - 1].words_end;
+  const uint8_t* codes_tiled = s == 0 ? a.sub[0].codes_tiled : (s == 1 ? a.sub[1].codes_tiled : a.sub[2].codes_tiled);
+  const float2* sz = s == 0 ? a.sub[0].sz : (s == 1 ? a.sub[1].sz : a.sub[2].sz);
+  const int64_t Npad = s == 0 ? a.sub[0].Npad : (s == 1 ? a.sub[1].Npad : a.sub[2].Npad);
+  __nv_bfloat16* out = s == 0 ? a.sub[0].out : (s == 1 ? a.sub[1].out : a.sub[2].out);
   const int chunk = static_cast<int>(i & 7), r = static_cast<int>((i >> 3) & 127);
   const int64_t blk = i >> 10;
-  const int64_t t = blk / nkb;
-  const int kb = static_cast<int>(blk - t * nkb);
+  const int64_t t = blk / a.nkb;
+  const int kb = static_cast<int>(blk - t * a.nkb);
   const uint32_t w = *reinterpret_cast<const uint32_t*>(codes_tiled + blk * kCodesBytes + r * 32 + chunk * 4);
-  const int g = (kb * kBK + chunk * 8) / G;
+  const int g = (kb * kBK + chunk * 8) / a.G;
   const float2 p = sz[static_cast<int64_t>(g) * Npad + t * kBM + r];
-  *reinterpret_cast<uint4*>(out + (t * kBM + r) * K + kb * kBK + chunk * 8) = dequant_word<kFast>(w, p);
+  *reinterpret_cast<uint4*>(out + (t * kBM + r) * a.K + kb * kBK + chunk * 8) = dequant_word<kFast>(w, p);
 }
 
-// SparseAdd on the materialised matrix: indices are unique, so no two threads touch one element
-__global__ void scatter_add_bf16_kernel(__nv_bfloat16* __restrict__ w, const int64_t* __restrict__ idx,
-                                        const float* __restrict__ S, int64_t nnz) {
-  const int64_t e = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (e >= nnz) return;
-  __nv_bfloat16* el = w + idx[e];
+// SparseAdd on the materialised matrices: indices are unique, so no two threads touch one element
+__global__ void scatter_add_bf16_kernel(const MatArgs a) {
+  int64_t e = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (e >= a.sub[a.n - 1].nnz_end) return;
+  int s = 0;
+  if (e >= a.sub[0].nnz_end) s = (a.n > 2 && e >= a.sub[1].nnz_end) ? 2 : 1;
+  if (s > 0) e -= a.sub[s - 1].nnz_end;
+  const int64_t* idx = s == 0 ? a.sub[0].idx : (s == 1 ? a.sub[1].idx : a.sub[2].idx);
+  const float* S = s == 0 ? a.sub[0].S : (s == 1 ? a.sub[1].S : a.sub[2].S);
+  __nv_bfloat16* el = (s == 0 ? a.sub[0].out : (s == 1 ? a.sub[1].out : a.sub[2].out)) + idx[e];
   *el = __float2bfloat16_rn(__bfloat162float(*el) + S[e]);
 }
 
@@ -283,23 +309,22 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
   SZO_REQUIRE(rows < (int64_t(1) << 31), SZO_ERR_SHAPE, "too many weight rows in one launch");
   __nv_bfloat16* W = static_cast<__nv_bfloat16*>(ws);
   const int nkb = static_cast<int>(p0->K / kBK);
-  int64_t row0 = 0;
+  MatArgs a{};
+  a.n = n; a.nkb = nkb; a.G = p0->G; a.K = p0->K;
+  int64_t row0 = 0, words = 0, nnz = 0;
   for (int i = 0; i < n; ++i) {
     const szo_linear* p = plans[i];
-    const int64_t words = (p->Npad / kBM) * nkb * 1024;
-    __nv_bfloat16* Wi = W + row0 * p->K;
-    if (p->sz_dtype == SZO_BF16)
-      materialise_kernel<true><<<static_cast<unsigned>(ceil_div(words, 256)), 256, 0, st>>>(p->codes_tiled, p->sz, p->Npad, nkb,
-                                                                                         p->G, Wi, p->K);
-    else
-      materialise_kernel<false><<<static_cast<unsigned>(ceil_div(words, 256)), 256, 0, st>>>(p->codes_tiled, p->sz, p->Npad, nkb,
-                                                                                          p->G, Wi, p->K);
-    count_launch();
-    if (p->nnz > 0) {
-      scatter_add_bf16_kernel<<<static_cast<unsigned>(ceil_div(p->nnz, 256)), 256, 0, st>>>(Wi, p->idx, S_pert[i], p->nnz);
-      count_launch();
-    }
+    words += (p->Npad / kBM) * nkb * 1024;
+    nnz += p->nnz;
+    a.sub[i] = MatSub{p->codes_tiled, p->sz, p->Npad, W + row0 * p->K, p->idx, S_pert[i], words, nnz};
     row0 += p->Npad;
+  }
+  if (p0->sz_dtype == SZO_BF16) materialise_kernel<true><<<static_cast<unsigned>(ceil_div(words, 256)), 256, 0, st>>>(a);
+  else materialise_kernel<false><<<static_cast<unsigned>(ceil_div(words, 256)), 256, 0, st>>>(a);
+  count_launch();
+  if (nnz > 0) {
+    scatter_add_bf16_kernel<<<static_cast<unsigned>(ceil_div(nnz, 256)), 256, 0, st>>>(a);
+    count_launch();
   }
   SZO_CHECK_LAUNCH("materialise_kernel");
   CUtensorMap mx, mw;
