@@ -232,9 +232,10 @@ struct MatArgs {
   int64_t K;
 };
 
-// thread -> one 32-bit word of the tile-ordered codes (8 weights) -> 16 bytes of the row-major output.
-// A warp covers four k-blocks of one row: 32-byte reads from four code blocks, one 512-byte
-// contiguous write.  Work items per matrix: (Npad / 128) * ceil(nkb / 4) * 4096.
+// thread -> four 32-bit words of the tile-ordered codes (8 weights each, rows r, r + 32, r + 64, r + 96
+// of one tile) -> four 16-byte pieces of the row-major output; the four loads are issued before the
+// first use.  A warp covers four k-blocks of one row at a time: 32-byte reads from four code
+// blocks, one 512-byte contiguous write.  Work items per matrix: (Npad / 128) * ceil(nkb / 4) * 1024.
 template <bool kFast>
 __global__ void materialise_kernel(const MatArgs a) {
   int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -246,16 +247,25 @@ __global__ void materialise_kernel(const MatArgs a) {
   const float2* sz = s == 0 ? a.sub[0].sz : (s == 1 ? a.sub[1].sz : a.sub[2].sz);
   const int64_t Npad = s == 0 ? a.sub[0].Npad : (s == 1 ? a.sub[1].Npad : a.sub[2].Npad);
   __nv_bfloat16* out = s == 0 ? a.sub[0].out : (s == 1 ? a.sub[1].out : a.sub[2].out);
-  const int chunk = static_cast<int>(i & 7), kbo = static_cast<int>((i >> 3) & 3), r = static_cast<int>((i >> 5) & 127);
+  const int chunk = static_cast<int>(i & 7), kbo = static_cast<int>((i >> 3) & 3), r0 = static_cast<int>((i >> 5) & 31);
   const int nkb4 = (a.nkb + 3) >> 2;
-  const int64_t grp = i >> 12;
+  const int64_t grp = i >> 10;
   const int64_t t = grp / nkb4;
   const int kb = static_cast<int>(grp - t * nkb4) * 4 + kbo;
   if (kb >= a.nkb) return;
-  const uint32_t w = *reinterpret_cast<const uint32_t*>(codes_tiled + (t * a.nkb + kb) * kCodesBytes + r * 32 + chunk * 4);
+  const uint8_t* src = codes_tiled + (t * a.nkb + kb) * kCodesBytes + r0 * 32 + chunk * 4;
   const int g = (kb * kBK + chunk * 8) / a.G;
-  const float2 p = sz[static_cast<int64_t>(g) * Npad + t * kBM + r];
-  *reinterpret_cast<uint4*>(out + (t * kBM + r) * a.K + kb * kBK + chunk * 8) = dequant_word<kFast>(w, p);
+  const float2* szp = sz + static_cast<int64_t>(g) * Npad + t * kBM + r0;
+  uint32_t w[4];
+  float2 p[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    w[j] = *reinterpret_cast<const uint32_t*>(src + j * 32 * 32);
+    p[j] = szp[j * 32];
+  }
+  __nv_bfloat16* dst = out + (t * kBM + r0) * a.K + kb * kBK + chunk * 8;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(dst + static_cast<int64_t>(j) * 32 * a.K) = dequant_word<kFast>(w[j], p[j]);
 }
 
 // SparseAdd on the materialised matrices: indices are unique, so no two threads touch one element
@@ -318,7 +328,7 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
   int64_t row0 = 0, words = 0, nnz = 0;
   for (int i = 0; i < n; ++i) {
     const szo_linear* p = plans[i];
-    words += (p->Npad / kBM) * ((nkb + 3) / 4) * 4096;
+    words += (p->Npad / kBM) * ((nkb + 3) / 4) * 1024;
     nnz += p->nnz;
     a.sub[i] = MatSub{p->codes_tiled, p->sz, p->Npad, W + row0 * p->K, p->idx, S_pert[i], words, nnz};
     row0 += p->Npad;
