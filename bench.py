@@ -30,7 +30,7 @@ BATCH, SEQ = 16, 256
 EPS, LR, SEED = 1e-3, 1e-6, 1234
 # dram__bytes_read.sum + dram__bytes_write.sum of one szo_linear_tc2_kernel launch (ncu, see profiles/);
 # set to None when that kernel changes until the counters are taken again
-TC2_GATE_TRAFFIC_BYTES = 135.6e6
+TC2_GATE_TRAFFIC_BYTES = 224.4e6
 
 
 def measured_peaks():
@@ -270,8 +270,9 @@ def run_ours(args):
         "gpu_launches": int(launches),
         "roofline": {"bound": "tensor", "kernel": "szo_linear_tc2_kernel", "achieved": achieved, "peak": peak,
                      "unit": "TFLOP/s", "frac": achieved / peak, "traffic": TC2_GATE_TRAFFIC_BYTES,
-                     "traffic_of": "one gate-shape launch (M=4096, N=11008, K=4096) of the same kernel under ncu: "
-                                   "profiles/szo_linear_tc2_kernel_gate_proj_M4096.md (149.4e6 algorithmic)",
+                     "traffic_of": "one gate-shape launch (M=4096, N=11008, K=4096) of the same kernel (dense mode, as the "
+                                   "step runs it) under ncu: profiles/szo_linear_tc2_kernel_dense_mode_gate_proj_M4096.md "
+                                   "(214e6 algorithmic for that launch; the materialising pass before it moves 112.7e6)",
                      "peak_source": f"{peaks['source']} (sustained cuBLAS bf16)",
                      "launches": int(lin_launches), "avg_launch_ms": lin_ms / max(lin_launches, 1),
                      "linear_ms_per_step": lin_ms / args.steps},
