@@ -177,18 +177,14 @@ def run_ours(args):
     from paper_2406_02913_b200 import build as build_mod
     from paper_2406_02913_b200 import workloads as wl
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl")
+    from paper_2406_02913_b200.replicas import Replicas
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    rep = Replicas("nccl")
+    world, rank, local = rep.world, rep.rank, rep.local_rank
     if rank == 0:
         build_mod.build()
-    if dist is not None:
-        dist.barrier()
+    if rep.dist is not None:
+        rep.dist.barrier()
     B.lib()
 
     shape = wl.MODEL_SHAPES[WORKLOAD]
@@ -204,18 +200,7 @@ def run_ours(args):
     labs_dev = [t.cuda() for t in labs_host]
     cand_dev = cand_host.cuda()
 
-    def barrier():
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def max_over_ranks(ms):
-        if dist is None:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    barrier, max_over_ranks = rep.barrier, rep.max_over_ranks
 
     # ---- device-resident inputs (the headline value)
     for i in range(args.warmup):
@@ -254,7 +239,7 @@ def run_ours(args):
     peaks = measured_peaks()
     M = BATCH * SEQ
     ms_per_step = ms_total / args.steps
-    steps_per_s = world * 1e3 / ms_per_step
+    steps_per_s = rep.whole_job_rate(1.0, ms_per_step)
     flops_fwd = linear_flops_per_forward(shape, M)
     lin_flops_total = 2 * flops_fwd * args.steps
     achieved = lin_flops_total / (lin_ms * 1e-3) / 1e12 if lin_ms > 0 else 0.0
@@ -265,7 +250,7 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(shape),
         "tokens_per_s": steps_per_s * M,
-        "e2e": {"value": world * 1e3 * args.steps / e2e_ms, "unit": "steps/s",
+        "e2e": {"value": rep.whole_job_rate(args.steps, e2e_ms), "unit": "steps/s",
                 "h2d_bytes_per_step": BATCH * SEQ * 4 + BATCH * 4 + 8, "d2h_bytes_per_step": 24},
         "gpu_launches": int(launches),
         "roofline": {"bound": "tensor", "kernel": "szo_linear_tc2_kernel", "achieved": achieved, "peak": peak,
