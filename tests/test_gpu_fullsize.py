@@ -109,3 +109,47 @@ def test_sparse_passes_at_7b_scale(B):
     got = S.cpu().numpy()[samp].astype(np.float64)
     ref = s3[samp].astype(np.float64) + float(sc) * z_ref.astype(np.float64)
     assert np.all(np.abs(got - ref) <= abs(float(sc)) * 1e-6 * np.maximum(1, np.abs(z_ref)) + 1.5e-8)   # + one fp32 ulp of the sum
+
+
+def test_two_full_width_layers_in_the_bench_configuration(B):
+    """Two decoder layers at the Llama-2-7B width with the bench's batch (16 x 256 tokens, so every
+    linear group takes the launch configuration bench.py times: fused q/k/v and gate/up groups, the
+    materialised form).  The fp64 oracle cannot run this size; what holds at any size is checked:
+    the bf16 tensor-core loss agrees with the library's own fp32 validation path (which the small
+    tests pin to the oracle), a step is repeatable bit for bit, and a step with lr = 0 leaves the
+    sparse values where they were up to the rounding of +eps, -2 eps, +eps."""
+    shape = dict(wl.MODEL_SHAPES["llama2_7b"], n_layers=2)
+    tensors, S_all = wl.device_decoder_tensors(shape, seed=3)
+    names = wl.linear_names(shape)
+    Bn, S = 16, 256
+    toks = torch.from_numpy(wl.token_batch(shape["vocab"], Bn, S, 3, wl.PURPOSE_TRAIN_BATCH, 0)).cuda()
+    labs = torch.from_numpy(wl.binary_labels(Bn, 3, 0)).cuda()
+    cand = torch.tensor([9906, 13], dtype=torch.int32, device="cuda")
+    S_tc, S_ref = S_all.clone(), S_all.clone()
+    m_tc = B.Model(shape, names, tensors, S_tc, act_dtype=B.SZO_BF16, linear_mode=B.MODE_SPARSE_ADD,
+                   loss_kind=B.LOSS_CLS2, max_batch=Bn, max_seq=S)
+    m_ref = B.Model(shape, names, tensors, S_ref, act_dtype=B.SZO_F32, linear_mode=B.MODE_FP32_VALIDATE,
+                    loss_kind=B.LOSS_CLS2, max_batch=Bn, max_seq=S)
+    f_tc = float(m_tc.loss(toks, labs, cand).item())
+    f_ref = float(m_ref.loss(toks, labs, cand).item())
+    assert np.isfinite(f_tc) and np.isfinite(f_ref)
+    # bf16 path: between the embedding and the last norm a state passes about ten bf16 roundings
+    # (2^-9 relative each: x, q/k/v, P, o, gate/up, their product, ...), i.e. ~6e-3 of relative noise;
+    # the loss reads it through a logit difference of standard deviation 0.02 sqrt(2 * 4096) = 1.8 and
+    # |dL/dlogit| <= 1/2, averaged over only 16 sequences: about 5e-3, bounded here by 1.5e-2
+    assert abs(f_tc - f_ref) <= 1.5e-2 * abs(f_ref)
+    # one step twice from the same state
+    eps = 1e-3
+    S0 = S_tc.clone()
+    out1 = m_tc.zo_step(toks, 1234, 7, eps, 0.0, labs, cand).clone()
+    S1 = S_tc.clone()
+    S_tc.copy_(S0)
+    out2 = m_tc.zo_step(toks, 1234, 7, eps, 0.0, labs, cand).clone()
+    torch.cuda.synchronize()
+    assert B.device_status() == 0
+    assert torch.equal(out1, out2) and torch.equal(S1, S_tc)
+    assert float((S1 - S0).abs().max()) <= 2 * float(np.spacing(np.float32(0.25)))     # lr = 0: restored
+    fp, fm, g = (float(v) for v in out1.cpu())
+    assert abs(g - (fp - fm) / (2 * float(np.float32(eps)))) <= 1e-9 * max(1.0, abs(g))    # eps is an fp32 value
+    # the perturbed losses bracket the unperturbed one to first order
+    assert abs(0.5 * (fp + fm) - f_tc) <= 1.5e-2 * abs(f_tc)
