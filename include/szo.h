@@ -152,7 +152,13 @@ szo_status szo_linear_create(szo_linear_t** out, int64_t N, int64_t K, int32_t G
 /* x: x_dtype [M,K] (SZO_BF16; SZO_F32 also accepted in SZO_MODE_FP32_VALIDATE);
  * S_pert: fp32 [nnz] current (already perturbed) sparse values; y: y_dtype [M,N] (SZO_BF16 or
  * SZO_F32).  workspace: at least szo_linear_workspace_bytes(plan, M, mode) bytes (may be NULL
- * when that is 0). */
+ * when that is 0), device memory, contents irrelevant on entry and undefined on return.  In the
+ * tensor-core modes it holds the bucket-ordered sparse records and the fp32 scratch of tiles that
+ * are split along K; for an int4 plan and M >= 4096 tokens it holds instead the effective bf16
+ * weight Dequantize(Q) + w_sparse of this layer (2 N K bytes, rows padded to 256), which is written
+ * first and then multiplied: the appendix's DenseMM(SparseAdd(w_sparse, Dequantize(Q)), x) literally.
+ * Both forms give the same bits.  A plan must not run on two streams at once (its K-split
+ * tickets are shared). */
 szo_status szo_linear_fwd(const szo_linear_t* plan, const void* x, szo_dtype x_dtype, int64_t M,
                           const float* S_pert, void* y, szo_dtype y_dtype, int32_t mode,
                           void* workspace, size_t workspace_bytes, void* stream);
