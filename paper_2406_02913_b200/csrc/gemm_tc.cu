@@ -225,11 +225,13 @@ struct MatSub {
   const int64_t* idx;         // sparse entries: flat indices n * K + c, values S
   const float* S;
   int64_t words_end, nnz_end; // running totals over the matrices: work items of this and the earlier ones
+  __nv_bfloat16* saved;       // [nnz] dense values at the masked positions (two-set form)
 };
 struct MatArgs {
   MatSub sub[3];
   int n, nkb, G;
   int64_t K;
+  int scatter_mode;           // 0: w += S; 1: saved = w, w += S; 2: w = saved + S (second set of sparse values)
 };
 
 // thread -> four 32-bit words of the tile-ordered codes (8 weights each, rows r, r + 32, r + 64, r + 96
@@ -268,7 +270,9 @@ __global__ void materialise_kernel(const MatArgs a) {
   for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(dst + static_cast<int64_t>(j) * 32 * a.K) = dequant_word<kFast>(w[j], p[j]);
 }
 
-// SparseAdd on the materialised matrices: indices are unique, so no two threads touch one element
+// SparseAdd on the materialised matrices: indices are unique, so no two threads touch one element.
+// With two sets of sparse values for one weight pass (the two perturbed forwards of a ZO step) the
+// dense values at the masked positions are kept aside by the first scatter and reused by the second.
 __global__ void scatter_add_bf16_kernel(const MatArgs a) {
   int64_t e = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (e >= a.sub[a.n - 1].nnz_end) return;
@@ -277,8 +281,12 @@ __global__ void scatter_add_bf16_kernel(const MatArgs a) {
   if (s > 0) e -= a.sub[s - 1].nnz_end;
   const int64_t* idx = s == 0 ? a.sub[0].idx : (s == 1 ? a.sub[1].idx : a.sub[2].idx);
   const float* S = s == 0 ? a.sub[0].S : (s == 1 ? a.sub[1].S : a.sub[2].S);
+  __nv_bfloat16* saved = s == 0 ? a.sub[0].saved : (s == 1 ? a.sub[1].saved : a.sub[2].saved);
   __nv_bfloat16* el = (s == 0 ? a.sub[0].out : (s == 1 ? a.sub[1].out : a.sub[2].out)) + idx[e];
-  *el = __float2bfloat16_rn(__bfloat162float(*el) + S[e]);
+  __nv_bfloat16 base = *el;
+  if (a.scatter_mode == 1) saved[e] = base;
+  if (a.scatter_mode == 2) base = saved[e];
+  *el = __float2bfloat16_rn(__bfloat162float(base) + S[e]);
 }
 
 // SZO_LINEAR_MATERIALISE=0 / 1 switches the form off / on for every M (A/B measurement)
@@ -304,24 +312,35 @@ bool tc_use_materialised(const szo_linear* p, int64_t M) {
 size_t tc_materialised_ws_bytes(const szo_linear* const* plans, int n, int64_t M) {
   size_t rows = 0;
   for (int i = 0; i < n; ++i) rows += static_cast<size_t>(plans[i]->Npad);
-  return round_up(rows * static_cast<size_t>(plans[0]->K) * sizeof(__nv_bfloat16), 256) + tc_tail_ws_bound();
+  size_t nnz = 0;
+  for (int i = 0; i < n; ++i) nnz += static_cast<size_t>(plans[i]->nnz);
+  return round_up(rows * static_cast<size_t>(plans[0]->K) * sizeof(__nv_bfloat16), 256) +
+         round_up(nnz * sizeof(__nv_bfloat16), 256) + tc_tail_ws_bound();
 }
 
-// n matrices that share x (n == 1 or tc_can_fuse): materialise, SparseAdd, dense launch.
+// n matrices that share x (n == 1 or tc_can_fuse): materialise, SparseAdd, dense launch.  With
+// S_second != nullptr the weight pass serves two sets of sparse values (S_pert and S_second) and two
+// sets of M tokens each: x and every y[i] then hold 2 M rows, set 0 first.
 szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, const void* x, int64_t M,
                                       const float* const* S_pert, void* const* y, int y_dtype, void* ws,
-                                      size_t ws_bytes, cudaStream_t st) {
+                                      size_t ws_bytes, cudaStream_t st, const float* const* S_second) {
   const szo_linear* p0 = plans[0];
   const TcPlan* t = static_cast<const TcPlan*>(p0->tc);
   SZO_REQUIRE(t != nullptr, SZO_ERR_INVALID_ARG, "plan has no tensor-core data");
   SZO_REQUIRE(M < (int64_t(1) << 31), SZO_ERR_SHAPE, "M too large");
   int64_t rows = 0;
-  for (int i = 0; i < n; ++i) rows += plans[i]->Npad;
+  size_t nnz_all = 0;
+  for (int i = 0; i < n; ++i) {
+    rows += plans[i]->Npad;
+    nnz_all += static_cast<size_t>(plans[i]->nnz);
+  }
   const size_t w_bytes = round_up(static_cast<size_t>(rows) * p0->K * sizeof(__nv_bfloat16), 256);
-  SZO_REQUIRE(ws != nullptr && ws_bytes >= w_bytes, SZO_ERR_WORKSPACE,
-              "the materialised form needs a workspace of at least %zu bytes", w_bytes);
+  const size_t saved_bytes = round_up(nnz_all * sizeof(__nv_bfloat16), 256);
+  SZO_REQUIRE(ws != nullptr && ws_bytes >= w_bytes + saved_bytes, SZO_ERR_WORKSPACE,
+              "the materialised form needs a workspace of at least %zu bytes", w_bytes + saved_bytes);
   SZO_REQUIRE(rows < (int64_t(1) << 31), SZO_ERR_SHAPE, "too many weight rows in one launch");
   __nv_bfloat16* W = static_cast<__nv_bfloat16*>(ws);
+  __nv_bfloat16* saved = reinterpret_cast<__nv_bfloat16*>(static_cast<unsigned char*>(ws) + w_bytes);
   const int nkb = static_cast<int>(p0->K / kBK);
   MatArgs a{};
   a.n = n; a.nkb = nkb; a.G = p0->G; a.K = p0->K;
@@ -329,20 +348,15 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
   for (int i = 0; i < n; ++i) {
     const szo_linear* p = plans[i];
     words += (p->Npad / kBM) * ((nkb + 3) / 4) * 1024;
+    a.sub[i] = MatSub{p->codes_tiled, p->sz, p->Npad, W + row0 * p->K, p->idx, S_pert[i], words, nnz + p->nnz, saved + nnz};
     nnz += p->nnz;
-    a.sub[i] = MatSub{p->codes_tiled, p->sz, p->Npad, W + row0 * p->K, p->idx, S_pert[i], words, nnz};
     row0 += p->Npad;
   }
   if (p0->sz_dtype == SZO_BF16) materialise_kernel<true><<<static_cast<unsigned>(ceil_div(words, 256)), 256, 0, st>>>(a);
   else materialise_kernel<false><<<static_cast<unsigned>(ceil_div(words, 256)), 256, 0, st>>>(a);
   count_launch();
-  if (nnz > 0) {
-    scatter_add_bf16_kernel<<<static_cast<unsigned>(ceil_div(nnz, 256)), 256, 0, st>>>(a);
-    count_launch();
-  }
   SZO_CHECK_LAUNCH("materialise_kernel");
-  CUtensorMap mx, mw;
-  SZO_TRY(make_map(&mx, x, M, p0->K, 128));
+  CUtensorMap mw;
   SZO_TRY(make_map(&mw, W, rows, p0->K, kBM));
   TcParams P{};
   P.M = M; P.K = p0->K; P.G = 0; P.nkb = nkb;
@@ -357,7 +371,6 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
     sb.bucket_ptr = nullptr;
     sb.Sb = nullptr;
     sb.bias = p->bias;
-    sb.y = y[i];
     sb.N = p->N;
     sb.Npad = p->Npad;
     sb.n_rowtiles = 0;
@@ -370,8 +383,8 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
   SZO_REQUIRE(P.status != nullptr, SZO_ERR_CUDA, "no device status word");
   const int64_t tiles = P.m_tiles * P.n_tiles;
   SZO_REQUIRE(tiles < (int64_t(1) << 30), SZO_ERR_SHAPE, "too many tiles");
-  void* tail = static_cast<unsigned char*>(ws) + w_bytes;
-  const size_t tail_bytes = ws_bytes - w_bytes;
+  void* tail = static_cast<unsigned char*>(ws) + w_bytes + saved_bytes;
+  const size_t tail_bytes = ws_bytes - w_bytes - saved_bytes;
   PairSchedule sc = pair_schedule(tiles, P.nkb, 0, t->sms, true);
   if (sc.ws_bytes > tail_bytes) sc = pair_schedule(tiles, P.nkb, 0, t->sms, false);
   P.full_rounds = sc.full_rounds;
@@ -380,7 +393,23 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
   for (int i = 0; i < 5; ++i) P.tail_kb[i] = sc.tail_kb[i];
   P.partial = static_cast<float*>(tail);
   P.tickets = t->tickets;
-  return launch_pair_kernel(false, false, mx, mw, P, sc.n_pairs, st);
+  const size_t y_elt = (y_dtype == SZO_F32) ? 4 : 2;
+  const int n_sets = S_second != nullptr ? 2 : 1;
+  for (int set = 0; set < n_sets; ++set) {
+    if (nnz > 0) {
+      a.scatter_mode = n_sets == 1 ? 0 : set + 1;
+      if (set == 1)
+        for (int i = 0; i < n; ++i) a.sub[i].S = S_second[i];
+      scatter_add_bf16_kernel<<<static_cast<unsigned>(ceil_div(nnz, 256)), 256, 0, st>>>(a);
+      count_launch();
+    }
+    CUtensorMap mx;
+    SZO_TRY(make_map(&mx, static_cast<const __nv_bfloat16*>(x) + static_cast<int64_t>(set) * M * p0->K, M, p0->K, 128));
+    for (int i = 0; i < n; ++i)
+      P.sub[i].y = static_cast<unsigned char*>(y[i]) + static_cast<size_t>(set) * M * plans[i]->N * y_elt;
+    SZO_TRY(launch_pair_kernel(false, false, mx, mw, P, sc.n_pairs, st));
+  }
+  return SZO_OK;
 }
 
 szo_status linear_fwd_tc(const szo_linear* p, const void* x, int64_t M, const uint2* S_bucket, void* y,

@@ -62,7 +62,9 @@ bool tc_use_materialised(const szo_linear* p, int64_t M);
 size_t tc_materialised_ws_bytes(const szo_linear* const* plans, int n, int64_t M);
 szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, const void* x, int64_t M,
                                       const float* const* S_pert, void* const* y, int y_dtype, void* ws,
-                                      size_t ws_bytes, cudaStream_t st);
+                                      size_t ws_bytes, cudaStream_t st, const float* const* S_second = nullptr);
+// S_second: a second set of sparse values and of M tokens served by the same weight pass (x and
+// y[i] hold 2 M rows).
 // out[p] = (pos[p], bits of S[eid[p]]) for p in [0, n)
 szo_status gather_values(const float* S, const int32_t* eid, const uint16_t* pos, int64_t n, uint2* out,
                          cudaStream_t st);

@@ -360,6 +360,8 @@ struct szo_model {
   uint16_t* gpos = nullptr;     // [k_total] in-tile position of each bucket-ordered record
   uint2* recs = nullptr;        // [k_total] (position, value) records of the current forward
   float* zkept = nullptr;       // [k_total] z of the current step, kept by the first perturb pass
+  float *Splus = nullptr, *Sminus = nullptr;   // [k_total] the two perturbed copies of S (two forwards side by side)
+  bool dual_rows = false;       // the activation buffers hold 2 * Mmax rows
   int64_t Mmax = 0;
   // activations
   float* h = nullptr;
@@ -403,11 +405,19 @@ void linear_shape(const szo_model_config& c, int j, int64_t* N, int64_t* K) {
 
 unsigned blocks_for(int64_t n, int t) { return static_cast<unsigned>(ceil_div(n, t)); }
 
+// One forward, or (Sv2 != nullptr) the two forwards of a ZO step side by side: the same tokens with
+// two sets of sparse values.  Every activation buffer then holds 2 M rows (set 0 first), the
+// elementwise, norm and attention kernels run once over both sets, and each linear group makes one
+// weight pass for both (materialised form only).
 template <typename T>
 szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand, int B,
-                      int S, const float* Sv, double* loss_dev, cudaStream_t st) {
+                      int S, const float* Sv, double* loss_dev, cudaStream_t st, const float* Sv2 = nullptr,
+                      double* loss_dev2 = nullptr) {
   const szo_model_config& c = m->cfg;
   const int64_t M = static_cast<int64_t>(B) * S;
+  const int nsets = Sv2 != nullptr ? 2 : 1;
+  const int64_t Mr = nsets * M;                 // rows of the activation buffers
+  const int Br = nsets * B;                     // sequences
   const int d = c.d_model, H = c.n_heads, Hkv = c.n_kv_heads, hd = d / H, ff = c.d_ff;
   const int act = c.act_dtype;
   const bool opt = c.arch == 1;
@@ -415,7 +425,7 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
     *o = static_cast<T*>(m->o), *y = static_cast<T*>(m->y), *gate = static_cast<T*>(m->gate),
     *up = static_cast<T*>(m->up);
   const bool pregather = c.linear_mode != SZO_MODE_FP32_VALIDATE && c.linear_mode != SZO_MODE_SPMM && m->k_total > 0;
-  auto lin = [&](int layer, int j, const void* x, void* out) -> szo_status {
+  auto lin_single = [&](int layer, int j, const void* x, void* out) -> szo_status {
     const int t = layer * m->n_lin + j;
     if (m->timing) {
       while (m->events.size() < m->events_used + 2) {
@@ -443,13 +453,18 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
       plans[i] = m->plans[t0 + i];
       recs[i] = m->recs + m->offsets[t0 + i];
     }
-    if (!(pregather && sizeof(T) == 2 && tc_can_fuse(plans, n, M))) {
-      for (int i = 0; i < n; ++i) SZO_TRY(lin(layer, j0 + i, x, outs[i]));
+    if (nsets == 1 && !(pregather && sizeof(T) == 2 && (n == 1 || tc_can_fuse(plans, n, M)))) {
+      for (int i = 0; i < n; ++i) SZO_TRY(lin_single(layer, j0 + i, x, outs[i]));
       return SZO_OK;
     }
-    const bool mat = tc_use_materialised(plans[0], M);
+    if (nsets == 1 && n == 1) return lin_single(layer, j0, x, outs[0]);
+    const bool mat = nsets == 2 || tc_use_materialised(plans[0], M);
     const float* spert[3];
-    for (int i = 0; i < n; ++i) spert[i] = Sv + m->offsets[t0 + i];
+    const float* spert2[3];
+    for (int i = 0; i < n; ++i) {
+      spert[i] = Sv + m->offsets[t0 + i];
+      spert2[i] = nsets == 2 ? Sv2 + m->offsets[t0 + i] : nullptr;
+    }
     if (m->timing) {
       while (m->events.size() < m->events_used + 2) {
         cudaEvent_t e;
@@ -458,7 +473,8 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
       }
       SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used], st));
     }
-    const szo_status rc = mat ? linear_fwd_tc_materialised(plans, n, x, M, spert, outs, act, m->ws, m->ws_bytes, st)
+    const szo_status rc = mat ? linear_fwd_tc_materialised(plans, n, x, M, spert, outs, act, m->ws, m->ws_bytes, st,
+                                                           nsets == 2 ? spert2 : nullptr)
                               : linear_fwd_tc_group(plans, n, x, M, recs, outs, act, m->ws, m->ws_bytes, st);
     if (m->timing) {
       SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used + 1], st));
@@ -466,74 +482,88 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
     }
     return rc;
   };
-  embed_kernel<<<static_cast<unsigned>(M), 128, 0, st>>>(tokens, static_cast<const __nv_bfloat16*>(m->top.embed),
-                                                        static_cast<const __nv_bfloat16*>(m->top.pos), S, d,
-                                                        c.vocab, m->h);
-  count_launch();
+  auto lin = [&](int layer, int j, const void* x, void* out) -> szo_status {
+    void* const outs[1] = {out};
+    return lin_group(layer, j, 1, x, outs);
+  };
+  for (int set = 0; set < nsets; ++set) {
+    embed_kernel<<<static_cast<unsigned>(M), 128, 0, st>>>(tokens, static_cast<const __nv_bfloat16*>(m->top.embed),
+                                                          static_cast<const __nv_bfloat16*>(m->top.pos), S, d,
+                                                          c.vocab, m->h + set * M * d);
+    count_launch();
+  }
   // One gather of all sparse values into the bucket order of every linear (SparseAdd mode)
-  if (pregather && !(m->plans.size() > 0 && tc_use_materialised(m->plans[0], M)))
+  if (nsets == 1 && pregather && !(m->plans.size() > 0 && tc_use_materialised(m->plans[0], M)))
     SZO_TRY(gather_values(Sv, m->geid, m->gpos, m->k_total, m->recs, st));
   const T* pending = nullptr;     // projection output still to be added to the residual stream
   for (int l = 0; l < c.n_layers; ++l) {
     const szo_layer_weights& L = m->layers[l];
-    add_norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, pending, L.attn_norm_g, L.attn_norm_b, d,
-                                                                c.norm_eps, opt, 1, 0, a);
+    add_norm_kernel<T><<<static_cast<unsigned>(Mr), 256, 0, st>>>(m->h, pending, L.attn_norm_g, L.attn_norm_b, d,
+                                                                 c.norm_eps, opt, 1, 0, a);
     count_launch();
     {
       void* const qkv[3] = {q, k, v};
       SZO_TRY(lin_group(l, 0, 3, a, qkv));
     }
     if (!opt) {
-      const int64_t n_vec = M * (H + Hkv) * ((hd / 2) / Vec16<T>::kN);
-      rope_kernel<T><<<blocks_for(n_vec, 256), 256, 0, st>>>(q, k, m->rope_tab, M, S, H, Hkv, hd);
+      const int64_t n_vec = Mr * (H + Hkv) * ((hd / 2) / Vec16<T>::kN);
+      rope_kernel<T><<<blocks_for(n_vec, 256), 256, 0, st>>>(q, k, m->rope_tab, Mr, S, H, Hkv, hd);
       count_launch();
     }
     if constexpr (sizeof(T) == 2) {
-      SZO_TRY(launch_flash_attention_bf16(q, k, v, o, B, S, H, Hkv, hd, st));
+      SZO_TRY(launch_flash_attention_bf16(q, k, v, o, Br, S, H, Hkv, hd, st));
     } else {
-      dim3 grid(static_cast<unsigned>(ceil_div(S, 4)), H, B);
+      dim3 grid(static_cast<unsigned>(ceil_div(S, 4)), H, Br);
       const float scale = 1.0f / sqrtf(static_cast<float>(hd));
       if (hd == 64) attn_warp_kernel<T, 64><<<grid, 128, 0, st>>>(q, k, v, o, S, H, Hkv, scale);
       else attn_warp_kernel<T, 128><<<grid, 128, 0, st>>>(q, k, v, o, S, H, Hkv, scale);
       count_launch();
     }
     SZO_TRY(lin(l, 3, o, y));
-    add_norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, y, L.mlp_norm_g, L.mlp_norm_b, d, c.norm_eps,
-                                                                opt, 1, 0, a);
+    add_norm_kernel<T><<<static_cast<unsigned>(Mr), 256, 0, st>>>(m->h, y, L.mlp_norm_g, L.mlp_norm_b, d, c.norm_eps,
+                                                                 opt, 1, 0, a);
     count_launch();
     if (!opt) {
       void* const gu[2] = {gate, up};
       SZO_TRY(lin_group(l, 4, 2, a, gu));
-      silu_mul_kernel<T><<<blocks_for(M * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, up, M * ff, gate);
+      silu_mul_kernel<T><<<blocks_for(Mr * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, up, Mr * ff, gate);
       count_launch();
       SZO_TRY(lin(l, 6, gate, y));
     } else {
       SZO_TRY(lin(l, 4, a, gate));
-      relu_kernel<T><<<blocks_for(M * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, M * ff);
+      relu_kernel<T><<<blocks_for(Mr * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, Mr * ff);
       count_launch();
       SZO_TRY(lin(l, 5, gate, y));
     }
     pending = y;                  // added by the next norm (next layer's, or the final one)
   }
+  double* const loss_out[2] = {loss_dev, loss_dev2};
   if (c.loss_kind == 0) {
-    add_norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, pending, m->top.final_norm_g,
-                                                                m->top.final_norm_b, d, c.norm_eps, opt, 1, 0, a);
+    add_norm_kernel<T><<<static_cast<unsigned>(Mr), 256, 0, st>>>(m->h, pending, m->top.final_norm_g,
+                                                                 m->top.final_norm_b, d, c.norm_eps, opt, 1, 0, a);
     count_launch();
     const int mode = c.linear_mode == SZO_MODE_FP32_VALIDATE ? SZO_MODE_FP32_VALIDATE : SZO_MODE_SPARSE_ADD;
-    SZO_TRY(szo_linear_fwd(m->lm_head_plan, a, static_cast<szo_dtype>(act), M, nullptr, m->logits, SZO_F32, mode,
+    SZO_TRY(szo_linear_fwd(m->lm_head_plan, a, static_cast<szo_dtype>(act), Mr, nullptr, m->logits, SZO_F32, mode,
                            m->ws, m->ws_bytes, st));
-    ce_rows_kernel<<<static_cast<unsigned>(M), 256, 0, st>>>(m->logits, tokens, S, c.vocab, m->tok_loss);
-    mean_f64_kernel<<<1, 1024, 0, st>>>(m->tok_loss, M, static_cast<double>(B) * (S - 1), loss_dev);
-    count_launch(2);
+    for (int set = 0; set < nsets; ++set) {
+      ce_rows_kernel<<<static_cast<unsigned>(M), 256, 0, st>>>(m->logits + set * M * c.vocab, tokens, S, c.vocab,
+                                                              m->tok_loss + set * M);
+      mean_f64_kernel<<<1, 1024, 0, st>>>(m->tok_loss + set * M, M, static_cast<double>(B) * (S - 1), loss_out[set]);
+      count_launch(2);
+    }
   } else {
-    // only B rows feed this loss: keep their normalised states in fp32 (the q buffer is free here)
+    // only B rows per set feed this loss: keep their normalised states in fp32 (the q buffer is free here)
     float* a_last = reinterpret_cast<float*>(m->q);
-    add_norm_kernel<T, float><<<static_cast<unsigned>(B), 256, 0, st>>>(
+    add_norm_kernel<T, float><<<static_cast<unsigned>(Br), 256, 0, st>>>(
         m->h, pending, m->top.final_norm_g, m->top.final_norm_b, d, c.norm_eps, opt, S, S - 1, a_last);
-    cls2_kernel<float><<<static_cast<unsigned>(B), 256, 0, st>>>(
-        a_last, static_cast<const __nv_bfloat16*>(m->top.lm_head), cand, labels, d, c.vocab, m->tok_loss);
-    mean_f64_kernel<<<1, 1024, 0, st>>>(m->tok_loss, B, static_cast<double>(B), loss_dev);
-    count_launch(3);
+    count_launch();
+    for (int set = 0; set < nsets; ++set) {
+      cls2_kernel<float><<<static_cast<unsigned>(B), 256, 0, st>>>(
+          a_last + static_cast<int64_t>(set) * B * d, static_cast<const __nv_bfloat16*>(m->top.lm_head), cand, labels, d,
+          c.vocab, m->tok_loss + set * B);
+      mean_f64_kernel<<<1, 1024, 0, st>>>(m->tok_loss + set * B, B, static_cast<double>(B), loss_out[set]);
+      count_launch(2);
+    }
   }
   SZO_CHECK_LAUNCH("model kernels");
   return SZO_OK;
@@ -543,6 +573,14 @@ szo_status run_loss(szo_model* m, const int32_t* tokens, const int32_t* labels, 
                     const float* Sv, double* loss_dev, cudaStream_t st) {
   if (m->cfg.act_dtype == SZO_F32) return run_loss_t<float>(m, tokens, labels, cand, B, S, Sv, loss_dev, st);
   return run_loss_t<__nv_bfloat16>(m, tokens, labels, cand, B, S, Sv, loss_dev, st);
+}
+
+// Both perturbed forwards of a step side by side (see run_loss_t); bf16 tensor-core path with the
+// materialised form only: the caller checks dual_forward_applies().
+bool dual_forward_applies(const szo_model* m, int64_t M) {
+  return m->dual_rows && m->cfg.act_dtype != SZO_F32 && m->cfg.linear_mode != SZO_MODE_FP32_VALIDATE &&
+         m->cfg.linear_mode != SZO_MODE_SPMM && !m->plans.empty() && m->k_total > 0 &&
+         tc_use_materialised(m->plans[0], M);
 }
 
 szo_status check_batch(const szo_model* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand, int B,
@@ -646,7 +684,21 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
   }
   // buffers
   const size_t e = c.act_dtype == SZO_F32 ? 4 : 2;
-  const int64_t Mx = m->Mmax, d = c.d_model, dkv = static_cast<int64_t>(c.n_kv_heads) * hd, ff = c.d_ff;
+  // When the step can run its two forwards side by side (bf16 tensor-core path in the materialised
+  // form; SZO_DUAL_FORWARD=0 at creation switches it off for A/B), every activation buffer holds
+  // two sets of Mmax rows.
+  {
+    const char* env = getenv("SZO_DUAL_FORWARD");
+    m->dual_rows = !(env != nullptr && env[0] == '0') && c.act_dtype != SZO_F32 &&
+                   c.linear_mode != SZO_MODE_FP32_VALIDATE && c.linear_mode != SZO_MODE_SPMM && !m->plans.empty() &&
+                   m->k_total > 0 && tc_use_materialised(m->plans[0], m->Mmax);
+  }
+  const int64_t Mx = m->Mmax * (m->dual_rows ? 2 : 1), d = c.d_model, dkv = static_cast<int64_t>(c.n_kv_heads) * hd,
+                ff = c.d_ff;
+  if (m->dual_rows) {
+    SZO_M_TRY(dev_alloc(m, &m->Splus, m->k_total * sizeof(float)));
+    SZO_M_TRY(dev_alloc(m, &m->Sminus, m->k_total * sizeof(float)));
+  }
   SZO_M_TRY(dev_alloc(m, &m->gidx, m->k_total * sizeof(int64_t)));
   SZO_M_TRY(dev_alloc(m, &m->h, Mx * d * sizeof(float)));
   SZO_M_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->a), Mx * d * e));
@@ -662,7 +714,7 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
   SZO_M_TRY(dev_alloc(m, &m->rope_tab, static_cast<size_t>(c.max_seq) * (hd / 2) * sizeof(float2)));
   if (ws_need) SZO_M_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->ws), ws_need));
   m->ws_bytes = ws_need;
-  SZO_M_TRY(dev_alloc(m, &m->d_tokens, Mx * sizeof(int32_t)));
+  SZO_M_TRY(dev_alloc(m, &m->d_tokens, m->Mmax * sizeof(int32_t)));
   SZO_M_TRY(dev_alloc(m, &m->d_labels, c.max_batch * sizeof(int32_t)));
   SZO_M_TRY(dev_alloc(m, &m->d_cand, 16));
   SZO_M_TRY(dev_alloc(m, &m->d_scalars, 4 * sizeof(double)));
@@ -742,6 +794,22 @@ szo_status szo_model_zo_step(szo_model_t* m, const int32_t* tokens, const int32_
   const int64_t k = m->k_total;
   float* Sv = m->S_all;
   ScaleArg sa{eps, 0.f, 0.f, nullptr, nullptr};
+  if (dual_forward_applies(m, static_cast<int64_t>(B) * S)) {
+    // both forwards side by side: the same arithmetic on S as the in-place sequence below
+    // (+eps, -2 eps, +eps), written to two copies, so that every linear makes one weight pass
+    SZO_TRY(launch_sparse_axpy(Sv, m->Splus, m->gidx, k, 0, seed, step, sa, st, m->zkept));   // S+ = S + eps z
+    sa.scale = -2.0f * eps;
+    SZO_TRY(launch_sparse_axpy_kept(m->Splus, m->Sminus, m->zkept, k, sa, st));               // S- = S+ - 2 eps z
+    sa.scale = eps;
+    SZO_TRY(launch_sparse_axpy_kept(m->Sminus, Sv, m->zkept, k, sa, st));                     // S = S- + eps z
+    SZO_TRY(run_loss_t<__nv_bfloat16>(m, tokens, labels, cand, B, S, m->Splus, f_plus_dev, st, m->Sminus,
+                                      f_minus_dev));                                          // f+, f-
+    SZO_TRY(szo_projected_gradient(f_plus_dev, f_minus_dev, eps, g_dev, stream));             // g
+    ScaleArg su2{0.f, lr, eps, f_plus_dev, f_minus_dev};
+    SZO_TRY(launch_sparse_axpy_kept(Sv, Sv, m->zkept, k, su2, st));                           // S -= lr g z
+    m->last_launches = g_launch_count - before;
+    return SZO_OK;
+  }
   // z is generated once per step (first pass) and kept: the other three passes stream it
   SZO_TRY(launch_sparse_axpy(Sv, Sv, m->gidx, k, 0, seed, step, sa, st, m->zkept));       // S += eps z
   SZO_TRY(run_loss(m, tokens, labels, cand, B, S, Sv, f_plus_dev, st));                   // f+

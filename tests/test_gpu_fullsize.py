@@ -153,3 +153,20 @@ def test_two_full_width_layers_in_the_bench_configuration(B):
     assert abs(g - (fp - fm) / (2 * float(np.float32(eps)))) <= 1e-9 * max(1.0, abs(g))    # eps is an fp32 value
     # the perturbed losses bracket the unperturbed one to first order
     assert abs(0.5 * (fp + fm) - f_tc) <= 1.5e-2 * abs(f_tc)
+    # the step runs its two forwards side by side (one weight pass per linear for both); the
+    # sequential form (one forward after the other) must give the same bits
+    import os
+    os.environ["SZO_DUAL_FORWARD"] = "0"
+    try:
+        S_seq = S0.clone()
+        m_seq = B.Model(shape, names, tensors, S_seq, act_dtype=B.SZO_BF16, linear_mode=B.MODE_SPARSE_ADD,
+                        loss_kind=B.LOSS_CLS2, max_batch=Bn, max_seq=S)
+    finally:
+        del os.environ["SZO_DUAL_FORWARD"]
+    S_tc.copy_(S0)
+    out_dual = m_tc.zo_step(toks, 99, 3, eps, 1e-4, labs, cand).clone()
+    out_seq = m_seq.zo_step(toks, 99, 3, eps, 1e-4, labs, cand).clone()
+    torch.cuda.synchronize()
+    assert m_tc.last_launches() < m_seq.last_launches()            # it really took the other route
+    assert torch.equal(out_dual, out_seq) and torch.equal(S_tc, S_seq)
+    assert not torch.equal(S_tc, S0)                               # and the update moved S
