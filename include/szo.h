@@ -47,7 +47,11 @@ typedef enum { SZO_F32 = 0, SZO_BF16 = 1, SZO_F16 = 2 } szo_dtype;
 /* How szo_linear_fwd evaluates y = x Dequantize(Q)^T + x S^T (the paper's appendix
  * "Implementation of Sparse Operations in Linear Layers" gives the two orders). */
 typedef enum {
-  SZO_MODE_AUTO = 0,          /* SPARSE_ADD */
+  SZO_MODE_AUTO = 0,          /* SPARSE_ADD, except for an int4 plan with M <= 16 tokens and K % 128 == 0:
+                                 there the layer is bound by reading the codes once, and a
+                                 weight-streaming kernel evaluates SparseAddMM(Dequantize(Q) x, S, x)
+                                 with the sparse term in fp32 (the order the appendix finds faster
+                                 for few tokens); it needs no workspace */
   SZO_MODE_SPARSE_ADD = 1,    /* DenseMM(SparseAdd(S, Dequantize(Q)), x): S is added to the
                                  dequantised bf16 tile in shared memory before the tensor-core MMA */
   SZO_MODE_SPMM = 2,          /* SparseAddMM(Dequantize(Q) x, S, x): tensor-core GEMM on the dense

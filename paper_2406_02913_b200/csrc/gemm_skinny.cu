@@ -1,0 +1,588 @@
+// Weight-streaming form of the decomposed linear for a handful of tokens (M <= 16):
+//   y[m, n] = sum_k x[m,k] * Dequantize(Q)[n,k] + sum_{(n,c) in mask} x[m,c] * S[n,c] + bias[n]
+// (appendix "Implementation of Sparse Operations in Linear Layers": the SparseAddMM form, which
+// the paper finds the faster one when few tokens are processed).  With so few tokens the layer is
+// bound by reading the int4 weights once from HBM, so the kernel is built around that stream, not
+// around the tensor cores' peak:
+//   * persistent clusters of 8 CTAs: a cluster takes 128-row tiles of the weight in turn and splits
+//     K between its CTAs, so that a CTA always works on the same columns and keeps its slice of the
+//     activations (8 or 16 tokens) in shared memory for the whole launch, 16-byte chunks permuted
+//     so that the lanes' 128-bit reads are free of bank conflicts;
+//   * one producer thread per CTA streams the CTA's part of the tiled codes (8 KB per 128-column
+//     step, contiguous) and the (scale, zero) entries of the step through an 8-stage ring of bulk
+//     copies that complete on mbarriers; it runs ahead across tile boundaries, so the stream never
+//     drains;
+//   * 8 weight warps own 16 rows each; per step a lane takes 16 bytes (32 codes) of each of its two
+//     rows from the stage.  The product runs on warp-level MMAs (m16n8k16: 16 weight rows x 8
+//     tokens, the weight as the A operand).  A dot product does not care about the order of k, so
+//     lane t uses its own four consecutive columns where the fragment layout names columns
+//     (2t, 2t+1, 2t+8, 2t+9), for the weights and the tokens alike;
+//   * when the quantization group covers whole steps (G a multiple of 128) the codes are not
+//     dequantised one by one: with q the codes of a group, scale s and zero z,
+//         sum_k x_k (q_k s + z) = s * sum_k x_k (128 + q_k) + (z - 128 s) * sum_k x_k,
+//     where 128 + q_k as bf16 is the code OR-ed into a constant (two instructions per pair of codes),
+//     the first sum is the MMA of the codes, the second is formed once per CTA when the activations
+//     are staged; scale and zero are applied once per step to the fp32 accumulators.  This is the
+//     exact (unrounded) Dequantize(Q).  Smaller groups (32, 64) take the packed-bf16 conversion of
+//     the large-M kernel instead;
+//   * a ninth warp forms the sparse term of 16 rows of the tile in fp32: its loads from global
+//     memory are pipelined over tiles, and the activations at the entries' columns come from the
+//     shared memory of the CTA that staged them (distributed shared memory, no trip through L2);
+//   * the K-split partial sums meet through distributed shared memory too: a tenth warp of CTA c
+//     adds the eight partials of rows 16c .. 16c+15 in CTA order (deterministic), then the sparse
+//     term and the bias, and stores y.  Partials and sparse terms are double-buffered and everyone
+//     waits only for the barrier of the tile before, so nobody stands still for the sum.
+// Waits on mbarriers are bounded (status SZO_ERR_TIMEOUT); after a failed wait a thread keeps the
+// control flow, and with it the cluster barriers, but skips waiting and copying.
+#include "tc_common.cuh"
+
+namespace szo {
+
+namespace {
+
+constexpr int kRowsWarp = 16;    // weight rows per warp (MMA M)
+constexpr int kWarps = 8;        // weight warps; then one warp each: sparse term, sum over the K-parts, producer
+constexpr int kWarpSparse = kWarps, kWarpSum = kWarps + 1, kWarpProducer = kWarps + 2;
+constexpr int kRowsCta = kRowsWarp * kWarps;   // 128: one tile of the plan's tiled codes
+constexpr int kSplit = 8;        // CTAs per cluster = parts K is split in
+constexpr int kTok = 8;          // tokens per token tile (MMA N)
+constexpr int kStepK = 128;      // columns per step: 4 lanes x 32 codes per row
+constexpr int kStages = 8;       // ring of steps in flight per CTA
+constexpr int kSpChunk = 128;    // sparse entries the sparse warp takes at a time
+constexpr int kPad = 32;         // elements added to a token row in shared memory: row stride = 16 words mod 32
+constexpr int kThreads = (kWarps + 3) * 32;
+constexpr int kWorkers = (kWarps + 2) * 32;    // all but the producer warp
+constexpr int kBlk1 = 4096 + 64; // offset of the step's second k-block in a stage: 16 banks away from the first
+constexpr int kSzOff = kBlk1 + 4096;           // (scale, zero) entries of the step: 1 KB per group
+constexpr size_t kMaxDynSmem = 190 * 1024;
+
+// Where the 16-byte chunk c (columns 8c .. 8c+7 of the CTA's slice) of a token row sits in shared
+// memory.  Inside a 128-column step, lane t works on chunks 4t .. 4t+3, one per turn; storing chunk
+// 4t+w at position 4w+t puts the four lanes' chunks of one turn side by side (64 contiguous bytes
+// per token), and with the row stride above the eight lanes of a quarter warp touch every bank once.
+__device__ __forceinline__ int chunk_pos(int c) { return (c & ~15) | ((c & 3) << 2) | ((c >> 2) & 3); }
+
+// D = A B + C, C given
+__device__ __forceinline__ void mma_acc(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// D = A B
+__device__ __forceinline__ void mma_new(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
+}
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address of `local` (a pointer into this CTA's shared memory) in CTA `cta` of the cluster
+__device__ __forceinline__ uint32_t cluster_addr(const void* local, uint32_t cta) {
+  const uint32_t a = static_cast<uint32_t>(__cvta_generic_to_shared(local));
+  uint32_t ra;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(a), "r"(cta));
+  return ra;
+}
+// Loads from the cluster's shared memory.  (volatile keeps them after the cluster barrier's wait,
+// which is volatile too; no memory clobber, so that the compiler may keep several in flight.)
+__device__ __forceinline__ uint4 ld_cluster_v4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared::cluster.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+  return v;
+}
+
+// (scale, zero) of one table entry as fp32; bf16 tables are stored as packed pairs (s,s), (z,z)
+template <bool kBf16Tables>
+__device__ __forceinline__ float2 sz_f32(float2 p) {
+  if constexpr (kBf16Tables)
+    return make_float2(__uint_as_float(__float_as_uint(p.x) & 0xFFFF0000u), __uint_as_float(__float_as_uint(p.y) & 0xFFFF0000u));
+  else
+    return p;
+}
+
+// A release at cluster scope measured about a microsecond per use here, so exactly one warp per CTA
+// (the summing warp) arrives with release, after a CTA-level barrier with the warps whose writes it
+// publishes; everybody else arrives relaxed.
+__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
+// CTA-level barrier 2: the weight warps and the sparse warp arrive, the summing warp waits
+__device__ __forceinline__ void tile_written_arrive() { asm volatile("bar.arrive 2, %0;" ::"n"((kWarps + 2) * 32) : "memory"); }
+__device__ __forceinline__ void tile_written_sync() { asm volatile("bar.sync 2, %0;" ::"n"((kWarps + 2) * 32) : "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+__device__ __forceinline__ void workers_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory"); }
+
+// kNT: token tiles per CTA (1: up to 8 tokens, 2: up to 16).  kGroupMma: G is a multiple of 128.
+// Grid: kSplit * n_clusters CTAs, clusters of kSplit along x; cluster c takes tiles c, c + n_clusters, ...
+// Cluster barriers, the same sequence for every thread (no early exit): number 0 says that every
+// CTA has staged its activations, number it + 1 that part and sparse term of the cluster's tile it
+// are written, the last one that nobody reads a peer any more.  A thread arrives at number k + 1
+// only after it is done with what number k - 1 published (the buffers alternate).
+template <bool kBf16Tables, bool kGroupMma, typename TY, int kNT>
+__global__ void __cluster_dims__(kSplit, 1, 1) __launch_bounds__(kThreads, kNT == 1 ? 2 : 1)
+szo_linear_skinny_kernel(const uint8_t* __restrict__ codes_tiled, const float2* __restrict__ sz, int64_t Npad,
+                         const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ row_ptr,
+                         const int32_t* __restrict__ ent_col, const float* __restrict__ S, const float* __restrict__ bias,
+                         TY* __restrict__ y, int M, int64_t N, int64_t K, int G, int n_tiles, int32_t* status) {
+  constexpr int kT = kTok * kNT;                       // tokens per CTA
+  extern __shared__ __align__(128) unsigned char smem_sk[];
+  __shared__ float part[2][kRowsCta * kT];             // this CTA's K-part of a 128-row tile: [row][token]
+  __shared__ float spart[2][kRowsWarp * kT];           // sparse term of the 16 rows this CTA sums: [row][token]
+  __shared__ float sp_x[kT * kSpChunk];                // sparse warp: activations at the chunk's columns, [token][entry]
+  __shared__ float sp_val[kSpChunk];                   //              values of the chunk's entries
+  __shared__ __align__(8) uint64_t bars[2 * kStages];  // full[kStages], empty[kStages]
+  __shared__ int abort_flag_s;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int rank = static_cast<int>(cluster_rank());
+  const int cid = static_cast<int>(blockIdx.x / kSplit), n_clusters = static_cast<int>(gridDim.x / kSplit);
+  const int n_steps = static_cast<int>(K / kStepK);
+  const int s_begin = rank * n_steps / kSplit, my_steps = (rank + 1) * n_steps / kSplit - s_begin;
+  const int ld = ((n_steps + kSplit - 1) / kSplit) * kStepK + kPad;    // the same in every CTA: peers index each other's rows
+  const int64_t nkb = K / 64;
+  const int ngs = (G >= kStepK) ? 1 : kStepK / G;       // (scale, zero) groups per step
+  const uint32_t stage_bytes = (static_cast<uint32_t>(kSzOff + ngs * 1024) + 127u) & ~127u;
+  unsigned char* ring = smem_sk;
+  __nv_bfloat16* sx = reinterpret_cast<__nv_bfloat16*>(smem_sk + kStages * stage_bytes);   // [kT][ld]: the CTA's columns of x
+  float* xsum = reinterpret_cast<float*>(sx + kT * ld);                                    // [my_steps][kT]
+  __nv_bfloat16* xt = reinterpret_cast<__nv_bfloat16*>(xsum + (ld - kPad) / kStepK * kT);  // [column of the slice][kT]: for the sparse warps
+  auto full_bar = [&](int i) { return tc::smem_u32(&bars[i]); };
+  auto empty_bar = [&](int i) { return tc::smem_u32(&bars[kStages + i]); };
+  volatile int* abort_flag = &abort_flag_s;
+
+  if (threadIdx.x == 0) {
+    abort_flag_s = 0;
+    for (int i = 0; i < kStages; ++i) {
+      tc::mbar_init(full_bar(i), 1);
+      tc::mbar_init(empty_bar(i), kWarps);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  bool failed = false;
+
+  if (warp == kWarpProducer) {
+    // ---------------------------------------------------------------- producer
+    tc::RingPos p{0, 0};
+    int it = 0;
+    const uint32_t tx_bytes = 8192u + static_cast<uint32_t>(ngs) * 1024u;
+    const uint32_t steps_per_group = (G >= kStepK) ? static_cast<uint32_t>(G / kStepK) : 0u;   // 0: several groups per step
+    cluster_arrive_relaxed();                           // number 0 (it stages nothing)
+    // It takes its turn at barrier number it only after tile it + 1 is issued (as far as the ring lets
+    // it), so that the stream does not stop while the cluster meets.
+    auto issue_tile = [&](int tile) {
+      if (lane == 0) {
+        // (a lone thread runs a dependent instruction every few cycles: no 64-bit division in here)
+        const uint8_t* src = codes_tiled + (static_cast<int64_t>(tile) * nkb + 2 * s_begin) * 4096;
+        const float2* zsrc = sz + static_cast<int64_t>(tile) * kRowsCta;
+        for (int i = 0; i < my_steps; ++i) {
+          if (!failed && !tc::mbar_wait(empty_bar(p.idx), p.phase ^ 1u, abort_flag, status)) failed = true;
+          if (!failed) {
+            const uint32_t dst = tc::smem_u32(ring + p.idx * stage_bytes);
+            const uint32_t bar = full_bar(p.idx);
+            tc::mbar_expect_tx(bar, tx_bytes);
+            tc::bulk_load_1d(dst, src, 4096, bar);
+            tc::bulk_load_1d(dst + kBlk1, src + 4096, 4096, bar);
+            const uint32_t grp0 = (steps_per_group > 0) ? static_cast<uint32_t>(s_begin + i) / steps_per_group
+                                                        : static_cast<uint32_t>(s_begin + i) * static_cast<uint32_t>(ngs);
+            const float2* z = zsrc + static_cast<int64_t>(grp0) * Npad;
+            for (int q = 0; q < ngs; ++q, z += Npad) tc::bulk_load_1d(dst + kSzOff + q * 1024, z, 1024, bar);
+          }
+          src += 8192;
+          p.advance(kStages);
+        }
+      }
+      __syncwarp();
+    };
+    issue_tile(cid);
+    for (int tile = cid; tile < n_tiles; tile += n_clusters, ++it) {
+      if (tile + n_clusters < n_tiles) issue_tile(tile + n_clusters);
+      cluster_wait();
+      cluster_arrive_relaxed();
+    }
+    cluster_wait();
+    if (lane == 0 && (failed || *abort_flag)) {
+      for (int i = 0; i < 200; ++i) __nanosleep(1000);      // copies in flight land before the CTA leaves
+    }
+  } else {
+    // the sparse warp's first row pointers (tiles it, it + 1) are on their way while the activations are staged
+    const int sp_r = lane >> 1;
+    const int64_t sp_row = rank * kRowsWarp + sp_r;                       // its lane's row inside a tile
+    auto load_rp = [&](int tile, int32_t& rb, int32_t& re) {
+      rb = re = 0;
+      if (row_ptr != nullptr && tile < n_tiles) {
+        const int64_t n = static_cast<int64_t>(tile) * kRowsCta + sp_row;
+        rb = row_ptr[(n < N) ? n : N];                                   // rows beyond N: empty
+        re = row_ptr[(n + 1 < N) ? n + 1 : N];
+      }
+    };
+    int32_t b0 = 0, e0 = 0, b1 = 0, e1 = 0;
+    if (warp == kWarpSparse) {
+      load_rp(cid, b0, e0);
+      load_rp(cid + n_clusters, b1, e1);
+    }
+    // ---------------------------------------------------------------- workers: stage the activations
+    {
+      // a thread takes one 16-byte chunk (8 columns) of every token: kT loads, the same chunks into the
+      // [token][column] tile, and their 8 x kT transpose into the [column][token] copy
+      const int chunks = my_steps * (kStepK / 8);
+      const __nv_bfloat16* xsrc = x + static_cast<int64_t>(s_begin) * kStepK;
+      for (int c = threadIdx.x; c < chunks; c += kWorkers) {
+        uint4 v[kT];
+#pragma unroll
+        for (int r = 0; r < kT; ++r)
+          v[r] = (r < M) ? __ldg(reinterpret_cast<const uint4*>(xsrc + static_cast<int64_t>(r) * K + c * 8)) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int r = 0; r < kT; ++r) *reinterpret_cast<uint4*>(sx + r * ld + chunk_pos(c) * 8) = v[r];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {                     // column c * 8 + e: tokens (2p, 2p + 1) share a word
+          const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;
+#pragma unroll
+          for (int j = 0; j < kNT; ++j) {
+            uint32_t o[4];
+#pragma unroll
+            for (int p2 = 0; p2 < 4; ++p2) {
+              const uint4& lo = v[8 * j + 2 * p2];
+              const uint4& hi = v[8 * j + 2 * p2 + 1];
+              const uint32_t wl = (e >> 1) == 0 ? lo.x : (e >> 1) == 1 ? lo.y : (e >> 1) == 2 ? lo.z : lo.w;
+              const uint32_t wh = (e >> 1) == 0 ? hi.x : (e >> 1) == 1 ? hi.y : (e >> 1) == 2 ? hi.z : hi.w;
+              o[p2] = tc::prmt(wl, wh, sel);
+            }
+            *reinterpret_cast<uint4*>(xt + (c * 8 + e) * kT + 8 * j) = make_uint4(o[0], o[1], o[2], o[3]);
+          }
+        }
+      }
+      workers_sync();
+      if (warp == kWarpSum) cluster_arrive_release();   // number 0: the CTA's activations are staged
+      else cluster_arrive_relaxed();
+      // sum of a token's activations over each step (the chunk permutation stays inside a step)
+      // half a warp per (step, token): a lane adds the eight values of one chunk, a fixed shuffle tree the rest
+      for (int i0 = warp * 2; i0 < my_steps * kT; i0 += (kWorkers / 32) * 2) {
+        const int i = i0 + (lane >> 4);
+        float acc = 0.f;
+        if (i < my_steps * kT) {
+          const int st = i / kT, m = i % kT;
+          const uint4 v = *reinterpret_cast<const uint4*>(sx + m * ld + st * kStepK + (lane & 15) * 8);
+          const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) acc += __uint_as_float(w[e] << 16) + __uint_as_float(w[e] & 0xFFFF0000u);
+        }
+#pragma unroll
+        for (int o = 8; o >= 1; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (i < my_steps * kT && (lane & 15) == 0) xsum[i] = acc;
+      }
+      workers_sync();
+    }
+
+    if (warp == kWarpSparse) {
+      // -------------------------------------------------------------- sparse warp
+      // Sparse term of rows 16 rank .. 16 rank + 15 of each tile.  The entries of the 16 rows are one
+      // contiguous CSR range, taken in chunks of kSpChunk: every lane fetches (column, value) of its
+      // entries, then the tokens' activations at those columns from the shared memory of the CTA
+      // that staged them, all loads independent; then lane = (row, token parity) adds its row's
+      // entries in ascending order, one fma each, from shared memory.  The dependent loads from
+      // global memory (row pointers, then entries) are software-pipelined over tiles: the row
+      // pointers of tile it + 2 and the first chunk of entries of tile it + 1 are in flight while
+      // tile it is summed.
+      constexpr int kGatherQ = kSpChunk / 32;                            // entries per lane whose activations are fetched at once
+      const int r = sp_r, h = lane & 1;
+      auto load_entries = [&](int32_t base, int32_t end, int (&col)[kSpChunk / 32], float (&val)[kSpChunk / 32]) {
+#pragma unroll
+        for (int q = 0; q < kSpChunk / 32; ++q) {
+          const int32_t e = base + lane + 32 * q;
+          col[q] = (e < end) ? ent_col[e] : -1;
+          val[q] = (e < end) ? S[e] : 0.f;
+        }
+      };
+      int32_t b2, e2;                                                    // row pointers of tile it + 2
+      int col0[kSpChunk / 32], col1[kSpChunk / 32];
+      float val0[kSpChunk / 32], val1[kSpChunk / 32];
+      load_entries(__shfl_sync(0xffffffffu, b0, 0), __shfl_sync(0xffffffffu, e0, 31), col0, val0);
+      int it = 0;
+      for (int tile = cid; tile < n_tiles; tile += n_clusters, ++it) {
+        load_rp(tile + 2 * n_clusters, b2, e2);
+        load_entries(__shfl_sync(0xffffffffu, b1, 0), __shfl_sync(0xffffffffu, e1, 31), col1, val1);
+        const int32_t tile_b = __shfl_sync(0xffffffffu, b0, 0), tile_e = __shfl_sync(0xffffffffu, e0, 31);
+        if (it == 0) cluster_wait();         // number 0: the peers' activations are staged
+        float sp[kT / 2];
+#pragma unroll
+        for (int j = 0; j < kT / 2; ++j) sp[j] = 0.f;
+        for (int32_t base = tile_b; base < tile_e; base += kSpChunk) {
+          if (base > tile_b) load_entries(base, tile_e, col0, val0);     // rows with more entries than one chunk
+          // (all loads of a pass first, then the stores: a store to shared memory between two loads
+          // from the cluster's shared memory would keep the second load waiting for the first)
+#pragma unroll
+          for (int q0 = 0; q0 < kSpChunk / 32; q0 += kGatherQ) {
+            uint4 xv[kGatherQ][kNT];
+#pragma unroll
+            for (int q = 0; q < kGatherQ; ++q) {
+              // column -> the CTA whose K-part holds it, and the position inside that CTA's slice
+              const int colq = col0[q0 + q] >= 0 ? col0[q0 + q] : 0;
+              const int step = colq >> 7;
+              const int owner = (kSplit * (step + 1) - 1) / n_steps;
+              const int lc = colq - (owner * n_steps / kSplit) * kStepK;
+              const uint32_t src = cluster_addr(xt + lc * kT, static_cast<uint32_t>(owner));
+#pragma unroll
+              for (int j = 0; j < kNT; ++j) xv[q][j] = ld_cluster_v4(src + 16u * j);     // 8 tokens per load
+            }
+#pragma unroll
+            for (int q = 0; q < kGatherQ; ++q) {
+              const bool live = col0[q0 + q] >= 0;       // (rows of x beyond M are staged as zeros)
+              sp_val[lane + 32 * (q0 + q)] = val0[q0 + q];
+#pragma unroll
+              for (int j = 0; j < kNT; ++j) {
+                const uint32_t w[4] = {xv[q][j].x, xv[q][j].y, xv[q][j].z, xv[q][j].w};
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                  sp_x[(8 * j + e) * kSpChunk + lane + 32 * (q0 + q)] =
+                      live ? __uint_as_float((e & 1) ? (w[e >> 1] & 0xFFFF0000u) : (w[e >> 1] << 16)) : 0.f;
+              }
+            }
+          }
+          __syncwarp();
+          const int lo = ((b0 > base) ? b0 : base) - base;
+          const int hi = ((e0 < base + kSpChunk) ? e0 : base + kSpChunk) - base;
+#pragma unroll 4
+          for (int i = lo; i < hi; ++i) {
+            const float sv = sp_val[i];
+#pragma unroll
+            for (int j = 0; j < kT / 2; ++j) sp[j] = fmaf(sp_x[(2 * j + h) * kSpChunk + i], sv, sp[j]);
+          }
+          __syncwarp();
+        }
+        if (it > 0) cluster_wait();          // number it: the tile of two turns ago is summed, its buffer free
+#pragma unroll
+        for (int j = 0; j < kT / 2; ++j) spart[it & 1][r * kT + 2 * j + h] = sp[j];
+        tile_written_arrive();
+        cluster_arrive_relaxed();            // number it + 1
+        b0 = b1; e0 = e1; b1 = b2; e1 = e2;
+#pragma unroll
+        for (int q = 0; q < kSpChunk / 32; ++q) {
+          col0[q] = col1[q];
+          val0[q] = val1[q];
+        }
+      }
+      cluster_wait();
+    } else if (warp == kWarpSum) {
+      // -------------------------------------------------------------- sum over the cluster's K-parts
+      // Rows 16 rank .. 16 rank + 15 of each tile: the eight CTAs' parts in CTA order, then the
+      // sparse term and the bias.  lane = (row, token parity) as in the sparse warp.
+      const int r = lane >> 1, h = lane & 1;
+      cluster_wait();                        // number 0
+      int it = 0;
+      for (int tile = cid; tile < n_tiles; tile += n_clusters, ++it) {
+        tile_written_sync();                 // this CTA's part and sparse term of the tile are written
+        cluster_arrive_release();            // number it + 1 (and: the tile before is summed and stored)
+        cluster_wait();
+        const int64_t n = static_cast<int64_t>(tile) * kRowsCta + rank * kRowsWarp + r;
+        const float bv = (bias != nullptr && n < N) ? bias[n] : 0.f;
+        float pv[kSplit][kT / 2], v[kT / 2];
+#pragma unroll
+        for (int cta = 0; cta < kSplit; ++cta) {                       // all loads first, then the sums in CTA order
+          const uint32_t src = cluster_addr(part[it & 1] + (rank * kRowsWarp + r) * kT + h, static_cast<uint32_t>(cta));
+#pragma unroll
+          for (int j = 0; j < kT / 2; ++j) pv[cta][j] = ld_cluster_f32(src + 8u * j);
+        }
+#pragma unroll
+        for (int j = 0; j < kT / 2; ++j) {
+          v[j] = pv[0][j];
+#pragma unroll
+          for (int cta = 1; cta < kSplit; ++cta) v[j] += pv[cta][j];
+        }
+#pragma unroll
+        for (int j = 0; j < kT / 2; ++j) {
+          const int m = 2 * j + h;
+          const float out = v[j] + spart[it & 1][r * kT + m] + bv;
+          if (n < N && m < M) {
+            if constexpr (sizeof(TY) == 2) y[static_cast<int64_t>(m) * N + n] = __float2bfloat16_rn(out);
+            else y[static_cast<int64_t>(m) * N + n] = out;
+          }
+        }
+      }
+    } else {
+      // -------------------------------------------------------------- weight warps
+      tc::RingPos c{0, 0};
+      const uint32_t w_off = static_cast<uint32_t>((t >> 1) * kBlk1 + (warp * kRowsWarp + g) * 32 + (t & 1) * 16);
+      const uint32_t z_off = static_cast<uint32_t>(kSzOff + ((G >= kStepK) ? 0 : (t * 32 / G)) * 1024 + (warp * kRowsWarp + g) * 8);
+      int it = 0;
+      for (int tile = cid; tile < n_tiles; tile += n_clusters, ++it) {
+        float tot[kNT][4];
+#pragma unroll
+        for (int j = 0; j < kNT; ++j) tot[j][0] = tot[j][1] = tot[j][2] = tot[j][3] = 0.f;
+        // one step: 16 rows x 128 columns of this warp against the staged tokens
+        auto step_body = [&](int i, const unsigned char* stg) {
+          const uint4 wa = *reinterpret_cast<const uint4*>(stg + w_off);
+          const uint4 wb = *reinterpret_cast<const uint4*>(stg + w_off + 8 * 32);
+          const float2 pa = *reinterpret_cast<const float2*>(stg + z_off);
+          const float2 pb = *reinterpret_cast<const float2*>(stg + z_off + 8 * 8);
+          const uint32_t qa[4] = {wa.x, wa.y, wa.z, wa.w}, qb[4] = {wb.x, wb.y, wb.z, wb.w};
+          const __nv_bfloat16* xs = sx + g * ld + i * kStepK + t * 8;      // token g; word wd of this lane: + wd * 32
+          if constexpr (kGroupMma) {
+            float accq[kNT][2][4];                                         // even and odd words: two shorter chains
+#pragma unroll
+            for (int wd = 0; wd < 4; ++wd) {                                // one 32-bit word = 8 columns = two k16 MMAs
+              uint32_t a0[4], a1[4];
+              a0[0] = (qa[wd] & 0x000F000Fu) | 0x43004300u;
+              a0[1] = (qb[wd] & 0x000F000Fu) | 0x43004300u;
+              a0[2] = ((qa[wd] >> 4) & 0x000F000Fu) | 0x43004300u;
+              a0[3] = ((qb[wd] >> 4) & 0x000F000Fu) | 0x43004300u;
+              a1[0] = ((qa[wd] >> 8) & 0x000F000Fu) | 0x43004300u;
+              a1[1] = ((qb[wd] >> 8) & 0x000F000Fu) | 0x43004300u;
+              a1[2] = ((qa[wd] >> 12) & 0x000F000Fu) | 0x43004300u;
+              a1[3] = ((qb[wd] >> 12) & 0x000F000Fu) | 0x43004300u;
+#pragma unroll
+              for (int j = 0; j < kNT; ++j) {
+                const uint4 xv = *reinterpret_cast<const uint4*>(xs + j * kTok * ld + wd * 32);
+                if (wd < 2) mma_new(accq[j][wd & 1], a0, xv.x, xv.y);
+                else mma_acc(accq[j][wd & 1], a0, xv.x, xv.y);
+                mma_acc(accq[j][wd & 1], a1, xv.z, xv.w);
+              }
+            }
+            const float2 fa = sz_f32<kBf16Tables>(pa), fb = sz_f32<kBf16Tables>(pb);
+            const float za = fmaf(-128.f, fa.x, fa.y), zb = fmaf(-128.f, fb.x, fb.y);
+#pragma unroll
+            for (int j = 0; j < kNT; ++j) {
+              const float2 xs2 = *reinterpret_cast<const float2*>(xsum + i * kT + kTok * j + 2 * t);   // tokens 2t, 2t+1
+              tot[j][0] = fmaf(fa.x, accq[j][0][0] + accq[j][1][0], fmaf(za, xs2.x, tot[j][0]));
+              tot[j][1] = fmaf(fa.x, accq[j][0][1] + accq[j][1][1], fmaf(za, xs2.y, tot[j][1]));
+              tot[j][2] = fmaf(fb.x, accq[j][0][2] + accq[j][1][2], fmaf(zb, xs2.x, tot[j][2]));
+              tot[j][3] = fmaf(fb.x, accq[j][0][3] + accq[j][1][3], fmaf(zb, xs2.y, tot[j][3]));
+            }
+          } else {
+#pragma unroll
+            for (int wd = 0; wd < 4; ++wd) {
+              const uint4 da = tc::dequant_word<kBf16Tables>(qa[wd], pa);
+              const uint4 db = tc::dequant_word<kBf16Tables>(qb[wd], pb);
+              const uint32_t a0[4] = {da.x, db.x, da.y, db.y};
+              const uint32_t a1[4] = {da.z, db.z, da.w, db.w};
+#pragma unroll
+              for (int j = 0; j < kNT; ++j) {
+                const uint4 xv = *reinterpret_cast<const uint4*>(xs + j * kTok * ld + wd * 32);
+                mma_acc(tot[j], a0, xv.x, xv.y);
+                mma_acc(tot[j], a1, xv.z, xv.w);
+              }
+            }
+          }
+        };
+        // two steps at a time: their instruction streams are independent and interleave
+        for (int i = 0; i < my_steps; i += 2) {
+          const bool two = i + 1 < my_steps;
+          tc::RingPos c1 = c;
+          c1.advance(kStages);
+          if (!failed && !tc::mbar_wait(full_bar(c.idx), c.phase, abort_flag, status)) failed = true;
+          if (two && !failed && !tc::mbar_wait(full_bar(c1.idx), c1.phase, abort_flag, status)) failed = true;
+          step_body(i, ring + c.idx * stage_bytes);
+          if (two) step_body(i + 1, ring + c1.idx * stage_bytes);
+          __syncwarp();
+          if (lane == 0 && !failed) {                      // the stages' data are in registers and used
+            tc::mbar_arrive(empty_bar(c.idx));
+            if (two) tc::mbar_arrive(empty_bar(c1.idx));
+          }
+          c = c1;
+          if (two) c.advance(kStages);
+        }
+        // accumulator layout: [0], [1] = (row g, tokens 2t, 2t+1); [2], [3] = (row g+8, same tokens)
+        cluster_wait();                                   // number it: the tile of two turns ago is summed, its buffer free
+#pragma unroll
+        for (int j = 0; j < kNT; ++j) {
+          float* mine = part[it & 1] + (warp * kRowsWarp + g) * kT + kTok * j + 2 * t;
+          mine[0] = tot[j][0];
+          mine[1] = tot[j][1];
+          mine[8 * kT] = tot[j][2];
+          mine[8 * kT + 1] = tot[j][3];
+        }
+        tile_written_arrive();
+        cluster_arrive_relaxed();                         // number it + 1
+      }
+      cluster_wait();
+    }
+  }
+  cluster_arrive_relaxed();                             // nobody leaves while its shared memory may still be read
+  cluster_wait();
+}
+
+size_t skinny_dyn_smem(int64_t K, int G, int kT) {
+  const int64_t n_steps = K / kStepK, max_steps = ceil_div(n_steps, kSplit);
+  const size_t ngs = (G >= kStepK) ? 1 : kStepK / G;
+  const size_t stage = (static_cast<size_t>(kSzOff) + ngs * 1024 + 127) & ~static_cast<size_t>(127);
+  return kStages * stage + static_cast<size_t>(kT) * (max_steps * kStepK + kPad) * 2 + static_cast<size_t>(max_steps) * kT * 4 +
+         static_cast<size_t>(max_steps) * kStepK * kT * 2;     // ring, x [token][column], step sums, x [column][token]
+}
+
+template <bool kBf16Tables, bool kGroupMma, typename TY, int kNT>
+szo_status launch_skinny(const szo_linear* p, const void* x, int64_t M, const float* S, void* y, cudaStream_t st) {
+  auto kern = szo_linear_skinny_kernel<kBf16Tables, kGroupMma, TY, kNT>;
+  const size_t smem = skinny_dyn_smem(p->K, p->G, kTok * kNT);
+  static bool configured = false;
+  if (!configured) {
+    SZO_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynSmem)));
+    configured = true;
+  }
+  int32_t* status = device_status_word();
+  SZO_REQUIRE(status != nullptr, SZO_ERR_CUDA, "no device status word");
+  const int n_tiles = static_cast<int>(ceil_div(p->N, kRowsCta));
+  // as many clusters as fit at once with this much shared memory (asked from the driver), no more than tiles
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(kSplit * n_tiles));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  static size_t asked_smem = ~static_cast<size_t>(0);
+  static int max_clusters = 0;
+  if (smem != asked_smem) {
+    SZO_CHECK_CUDA(cudaOccupancyMaxActiveClusters(&max_clusters, kern, &cfg));
+    if (max_clusters < 1) max_clusters = 1;
+    asked_smem = smem;
+  }
+  const int n_clusters = n_tiles < max_clusters ? n_tiles : max_clusters;
+  kern<<<static_cast<unsigned>(kSplit * n_clusters), kThreads, smem, st>>>(
+      p->codes_tiled, p->sz, p->Npad, static_cast<const __nv_bfloat16*>(x), p->nnz > 0 ? p->row_ptr : nullptr, p->ent_col,
+      S, p->bias, static_cast<TY*>(y), static_cast<int>(M), p->N, p->K, p->G, n_tiles, status);
+  count_launch();
+  SZO_CHECK_LAUNCH("szo_linear_skinny_kernel");
+  return SZO_OK;
+}
+
+template <bool kBf16Tables, typename TY>
+szo_status launch_skinny_nt(const szo_linear* p, const void* x, int64_t M, const float* S, void* y, cudaStream_t st) {
+  const bool group = p->G % kStepK == 0;
+  if (M <= kTok) {
+    if (group) return launch_skinny<kBf16Tables, true, TY, 1>(p, x, M, S, y, st);
+    return launch_skinny<kBf16Tables, false, TY, 1>(p, x, M, S, y, st);
+  }
+  if (group) return launch_skinny<kBf16Tables, true, TY, 2>(p, x, M, S, y, st);
+  return launch_skinny<kBf16Tables, false, TY, 2>(p, x, M, S, y, st);
+}
+
+}  // namespace
+
+// The shapes the weight-streaming kernel takes: int4 plans with groups of 32, 64 or a multiple of
+// 128 columns, at most 16 tokens, K a multiple of 128 whose per-CTA slice of the tokens fits shared memory.
+bool skinny_applies(const szo_linear* p, int64_t M) {
+  return p->G > 0 && (p->G == 32 || p->G == 64 || p->G % kStepK == 0) && M >= 1 && M <= 2 * kTok &&
+         p->K % kStepK == 0 && skinny_dyn_smem(p->K, p->G, 2 * kTok) <= kMaxDynSmem;
+}
+
+szo_status linear_fwd_skinny(const szo_linear* p, const void* x, int64_t M, const float* S_pert, void* y, int y_dtype,
+                             cudaStream_t st) {
+  SZO_REQUIRE(skinny_applies(p, M), SZO_ERR_UNSUPPORTED, "shape not covered by the weight-streaming kernel");
+  const bool bf = p->sz_dtype == SZO_BF16;
+  if (y_dtype == SZO_F32) {
+    if (bf) return launch_skinny_nt<true, float>(p, x, M, S_pert, y, st);
+    return launch_skinny_nt<false, float>(p, x, M, S_pert, y, st);
+  }
+  if (bf) return launch_skinny_nt<true, __nv_bfloat16>(p, x, M, S_pert, y, st);
+  return launch_skinny_nt<false, __nv_bfloat16>(p, x, M, S_pert, y, st);
+}
+
+}  // namespace szo

@@ -38,6 +38,12 @@ size_t linear_ws_fp32(const szo_linear* p, int64_t M);
 szo_status linear_spmm(const szo_linear* p, const void* x, int64_t M, const float* S, void* y,
                        int y_dtype, cudaStream_t st);
 
+// Weight-streaming kernel for at most 16 tokens (gemm_skinny.cu): int4 plans, K a multiple of 128;
+// the sparse term is added in fp32 from the CSR rows (SparseAddMM).  Needs no workspace.
+bool skinny_applies(const szo_linear* p, int64_t M);
+szo_status linear_fwd_skinny(const szo_linear* p, const void* x, int64_t M, const float* S_pert, void* y, int y_dtype,
+                             cudaStream_t st);
+
 // tensor-core path (gemm_tc.cu)
 szo_status tc_plan_create(szo_linear* p, cudaStream_t st);
 void tc_plan_destroy(szo_linear* p);

@@ -103,6 +103,48 @@ def test_tensor_core_modes(B, N, K, G, fmt, M, rho, bias, mode):
     plan.close()
 
 
+SKINNY_CASES = [
+    # N, K, G, fmt, M, rho, bias: at most 16 tokens, K a multiple of 128 -> the weight-streaming kernel
+    (256, 256, 64, "f16", 1, 1e-3, False),
+    (200, 640, 32, "bf16", 5, 5e-3, True),          # N not a multiple of the 128-row tile; 5 K steps for 8 CTAs
+    (512, 4096, 128, "bf16", 8, 1e-3, False),       # every CTA takes four steps
+    (300, 4224, 64, "f16", 13, 2e-3, True),         # two token tiles, the second ragged; 33 K steps
+    (1024, 11008, 128, "bf16", 16, 1e-3, False),    # the longest K of the 7B shapes
+    (128, 128, 128, "bf16", 3, 5e-2, True),         # one K step: seven CTAs of the cluster idle; dense mask
+    (512, 1024, 256, "f16", 7, 1e-3, False),        # a quantization group spans two steps
+    (640, 2048, 64, "bf16", 16, 3e-2, True),        # small groups; more sparse entries per 16 rows than one chunk
+]
+
+
+@pytest.mark.parametrize("N,K,G,fmt,M,rho,bias", SKINNY_CASES)
+def test_auto_mode_few_tokens(B, N, K, G, fmt, M, rho, bias):
+    """SZO_MODE_AUTO with M <= 16: weight-streaming kernel, sparse term in fp32 (SparseAddMM)."""
+    c = make_case(N, K, G, fmt, M, rho, seed=N + K + M, bias=bias)
+    plan, x, S = upload(B, c)
+    xb = x.to(torch.bfloat16)
+    ref = so.linear_fwd(xb.float().cpu().numpy(), c["deq"], c["idx"], c["S"], c["bias"])
+    assert plan.workspace_bytes(M, B.MODE_AUTO) == 0                   # the streaming kernel needs none
+    assert plan.workspace_bytes(M, B.MODE_SPARSE_ADD) > 0
+    y = plan.fwd(xb, S, B.MODE_AUTO, torch.float32).cpu().numpy()
+    assert max_rel(y, ref) < LINEAR_TOL
+    assert max_rel(y, ref) < 5e-3          # at most the bf16 rounding of the dequantised weight
+    if G % 128 == 0:
+        # scale and zero are applied to the fp32 sums of a group, the weight is never rounded to bf16:
+        # what is left is fp32 accumulation
+        assert max_rel(y, ref) < 1e-4
+    else:
+        # same bf16 weights as the pair-tile kernel: the two differ by accumulation order and by the
+        # sparse term (fp32 here and in SZO_MODE_SPMM)
+        y_pair = plan.fwd(xb, S, B.MODE_SPMM, torch.float32).cpu().numpy()
+        assert max_rel(y, y_pair) < 1e-4
+    yb = plan.fwd(xb, S, B.MODE_AUTO, torch.bfloat16).float().cpu().numpy()
+    assert max_rel(yb, ref) < LINEAR_TOL
+    y2 = plan.fwd(xb, S, B.MODE_AUTO, torch.float32).cpu().numpy()
+    assert np.array_equal(y, y2)
+    assert B.device_status() == 0
+    plan.close()
+
+
 def test_k_split_does_not_depend_on_the_scratch_contents(B):
     """Tiles split along K meet in the caller's workspace; whatever it held before must not matter,
     and two launches give the same bits."""
