@@ -567,10 +567,11 @@ szo_status launch_skinny_nt(const szo_linear* p, const void* x, int64_t M, const
 }  // namespace
 
 // The shapes the weight-streaming kernel takes: int4 plans with groups of 32, 64 or a multiple of
-// 128 columns, at most 16 tokens, K a multiple of 128 whose per-CTA slice of the tokens fits shared memory.
+// 128 columns, at most 16 tokens, K a multiple of 128 whose per-CTA slice of the tokens fits shared
+// memory (K up to about 25 000 for 8 tokens, 14 000 for 16).
 bool skinny_applies(const szo_linear* p, int64_t M) {
   return p->G > 0 && (p->G == 32 || p->G == 64 || p->G % kStepK == 0) && M >= 1 && M <= 2 * kTok &&
-         p->K % kStepK == 0 && skinny_dyn_smem(p->K, p->G, 2 * kTok) <= kMaxDynSmem;
+         p->K % kStepK == 0 && skinny_dyn_smem(p->K, p->G, M <= kTok ? kTok : 2 * kTok) <= kMaxDynSmem;
 }
 
 szo_status linear_fwd_skinny(const szo_linear* p, const void* x, int64_t M, const float* S_pert, void* y, int y_dtype,

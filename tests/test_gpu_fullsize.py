@@ -83,6 +83,56 @@ def test_full_size_linear_sampled_outputs(B, N, K, G, rho, bias, mode):
     plan.close()
 
 
+@pytest.mark.parametrize("N,K,bias", [
+    (4096, 4096, False), (11008, 4096, False), (4096, 11008, False),      # Llama-2-7B shapes
+    (20480, 5120, True), (5120, 20480, True),                             # OPT-13B MLP shapes, biases
+])
+@pytest.mark.parametrize("M", [1, 8, 16])
+def test_full_size_linear_few_tokens(B, N, K, bias, M):
+    """SZO_MODE_AUTO with at most 16 tokens (the weight-streaming kernel) at full width: every token,
+    sampled weight rows (all their columns) from the oracle; exact Dequantize(Q), so only fp32
+    accumulation separates the two."""
+    G = 128
+    g = torch.Generator(device="cuda")
+    g.manual_seed(N * 11 + K + M)
+    codes = torch.randint(0, 256, (N, K // 2), generator=g, device="cuda", dtype=torch.uint8)
+    sc = (0.004 + 0.002 * torch.rand(N, K // G, generator=g, device="cuda")).to(torch.bfloat16)
+    ze = (-7.5 * sc.float()).to(torch.bfloat16)
+    nnz = int(1e-3 * N * K)
+    idx_np = wl.sorted_random_indices(N * K, nnz, seed=N + K + M)
+    idx = torch.from_numpy(idx_np).cuda()
+    S = (torch.randn(nnz, generator=g, device="cuda") * 0.02).contiguous()
+    x = torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16)
+    b = (torch.randn(N, generator=g, device="cuda") * 0.02) if bias else None
+    plan = B.Linear(N, K, G, codes, sc, ze, "bf16", idx, b)
+    # no workspace = the weight-streaming kernel; 16 tokens x K = 20480 do not fit its shared memory
+    # and stay on the pair-tile kernel (bf16-rounded weights)
+    streaming = plan.workspace_bytes(M, B.MODE_AUTO) == 0
+    assert streaming == (not (K == 20480 and M > 8))
+    y = plan.fwd(x, S, B.MODE_AUTO, torch.float32)
+    torch.cuda.synchronize()
+    assert B.device_status() == 0
+    r = wl.rng(6, wl.PURPOSE_INDICES, N + K + M)
+    rows = np.unique(np.concatenate([r.integers(0, N, 40), [0, 15, 16, 127, 128, N - 129, N - 17, N - 1]]))
+    deq = so.dequantize(codes[rows].cpu().numpy(), _bf16_bits(sc[rows]), _bf16_bits(ze[rows]), G, "bf16")
+    S_h = S.cpu().numpy().astype(np.float64)
+    for i, n in enumerate(rows):
+        lo, hi = np.searchsorted(idx_np, [n * K, (n + 1) * K])
+        np.add.at(deq[i], idx_np[lo:hi] - n * K, S_h[lo:hi])
+    ref = x.float().cpu().numpy().astype(np.float64) @ deq.T
+    if bias:
+        ref = ref + b[rows].cpu().numpy().astype(np.float64)[None, :]
+    got = y[:, rows].cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(got - ref)) <= (1e-4 if streaming else 4e-3) * np.max(np.abs(ref))
+    assert torch.isfinite(y).all()
+    y2 = plan.fwd(x, S, B.MODE_AUTO, torch.float32)
+    assert torch.equal(y, y2)
+    # and the bf16 output path
+    yb = plan.fwd(x, S, B.MODE_AUTO, torch.bfloat16).float()
+    assert np.max(np.abs(yb[:, rows].cpu().numpy() - ref)) <= 5e-3 * np.max(np.abs(ref))
+    plan.close()
+
+
 def test_sparse_passes_at_7b_scale(B):
     """k = 0.1 % of the Llama-2-7B linear parameters: the +eps, -2eps, +eps sequence and an update,
     checked on a sample of entries (z and the fp32 fma), with the unsampled rest checked for the
