@@ -47,7 +47,7 @@ constexpr int kRowsCta = kRowsWarp * kWarps;   // 128: one tile of the plan's ti
 constexpr int kSplit = 8;        // CTAs per cluster = parts K is split in
 constexpr int kTok = 8;          // tokens per token tile (MMA N)
 constexpr int kStepK = 128;      // columns per step: 4 lanes x 32 codes per row
-constexpr int kStages = 8;       // ring of steps in flight per CTA
+constexpr int kStages = 8;       // most steps in flight per CTA (the launch may ask for fewer: n_stages)
 constexpr int kSpChunk = 128;    // sparse entries the sparse warp takes at a time
 constexpr int kPad = 32;         // elements added to a token row in shared memory: row stride = 16 words mod 32
 constexpr int kThreads = (kWarps + 3) * 32;
@@ -129,11 +129,11 @@ __device__ __forceinline__ void workers_sync() { asm volatile("bar.sync 1, %0;" 
 // are written, the last one that nobody reads a peer any more.  A thread arrives at number k + 1
 // only after it is done with what number k - 1 published (the buffers alternate).
 template <bool kBf16Tables, bool kGroupMma, typename TY, int kNT>
-__global__ void __cluster_dims__(kSplit, 1, 1) __launch_bounds__(kThreads, kNT == 1 ? 2 : 1)
+__global__ void __cluster_dims__(kSplit, 1, 1) __launch_bounds__(kThreads, 2)
 szo_linear_skinny_kernel(const uint8_t* __restrict__ codes_tiled, const float2* __restrict__ sz, int64_t Npad,
                          const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ row_ptr,
                          const int32_t* __restrict__ ent_col, const float* __restrict__ S, const float* __restrict__ bias,
-                         TY* __restrict__ y, int M, int64_t N, int64_t K, int G, int n_tiles, int32_t* status) {
+                         TY* __restrict__ y, int M, int64_t N, int64_t K, int G, int n_tiles, int n_stages, int32_t* status) {
   constexpr int kT = kTok * kNT;                       // tokens per CTA
   extern __shared__ __align__(128) unsigned char smem_sk[];
   __shared__ float part[2][kRowsCta * kT];             // this CTA's K-part of a 128-row tile: [row][token]
@@ -154,7 +154,7 @@ szo_linear_skinny_kernel(const uint8_t* __restrict__ codes_tiled, const float2* 
   const int ngs = (G >= kStepK) ? 1 : kStepK / G;       // (scale, zero) groups per step
   const uint32_t stage_bytes = (static_cast<uint32_t>(kSzOff + ngs * 1024) + 127u) & ~127u;
   unsigned char* ring = smem_sk;
-  __nv_bfloat16* sx = reinterpret_cast<__nv_bfloat16*>(smem_sk + kStages * stage_bytes);   // [kT][ld]: the CTA's columns of x
+  __nv_bfloat16* sx = reinterpret_cast<__nv_bfloat16*>(smem_sk + n_stages * stage_bytes);   // [kT][ld]: the CTA's columns of x
   float* xsum = reinterpret_cast<float*>(sx + kT * ld);                                    // [my_steps][kT]
   __nv_bfloat16* xt = reinterpret_cast<__nv_bfloat16*>(xsum + (ld - kPad) / kStepK * kT);  // [column of the slice][kT]: for the sparse warps
   auto full_bar = [&](int i) { return tc::smem_u32(&bars[i]); };
@@ -200,7 +200,7 @@ szo_linear_skinny_kernel(const uint8_t* __restrict__ codes_tiled, const float2* 
             for (int q = 0; q < ngs; ++q, z += Npad) tc::bulk_load_1d(dst + kSzOff + q * 1024, z, 1024, bar);
           }
           src += 8192;
-          p.advance(kStages);
+          p.advance(n_stages);
         }
       }
       __syncwarp();
@@ -234,33 +234,32 @@ szo_linear_skinny_kernel(const uint8_t* __restrict__ codes_tiled, const float2* 
     }
     // ---------------------------------------------------------------- workers: stage the activations
     {
-      // a thread takes one 16-byte chunk (8 columns) of every token: kT loads, the same chunks into the
-      // [token][column] tile, and their 8 x kT transpose into the [column][token] copy
+      // a thread takes one 16-byte chunk (8 columns) of the 8 tokens of a token tile: 8 loads, the same chunks into the
+      // [token][column] tile, and their 8 x 8 transpose into the [column][token] copy
       const int chunks = my_steps * (kStepK / 8);
       const __nv_bfloat16* xsrc = x + static_cast<int64_t>(s_begin) * kStepK;
-      for (int c = threadIdx.x; c < chunks; c += kWorkers) {
-        uint4 v[kT];
+      for (int cj = threadIdx.x; cj < chunks * kNT; cj += kWorkers) {
+        const int c = cj / kNT, j = cj % kNT;               // chunk, token tile
+        uint4 v[kTok];
 #pragma unroll
-        for (int r = 0; r < kT; ++r)
-          v[r] = (r < M) ? __ldg(reinterpret_cast<const uint4*>(xsrc + static_cast<int64_t>(r) * K + c * 8)) : make_uint4(0u, 0u, 0u, 0u);
+        for (int r = 0; r < kTok; ++r)
+          v[r] = (8 * j + r < M) ? __ldg(reinterpret_cast<const uint4*>(xsrc + static_cast<int64_t>(8 * j + r) * K + c * 8))
+                                 : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-        for (int r = 0; r < kT; ++r) *reinterpret_cast<uint4*>(sx + r * ld + chunk_pos(c) * 8) = v[r];
+        for (int r = 0; r < kTok; ++r) *reinterpret_cast<uint4*>(sx + (8 * j + r) * ld + chunk_pos(c) * 8) = v[r];
 #pragma unroll
         for (int e = 0; e < 8; ++e) {                     // column c * 8 + e: tokens (2p, 2p + 1) share a word
           const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;
+          uint32_t o[4];
 #pragma unroll
-          for (int j = 0; j < kNT; ++j) {
-            uint32_t o[4];
-#pragma unroll
-            for (int p2 = 0; p2 < 4; ++p2) {
-              const uint4& lo = v[8 * j + 2 * p2];
-              const uint4& hi = v[8 * j + 2 * p2 + 1];
-              const uint32_t wl = (e >> 1) == 0 ? lo.x : (e >> 1) == 1 ? lo.y : (e >> 1) == 2 ? lo.z : lo.w;
-              const uint32_t wh = (e >> 1) == 0 ? hi.x : (e >> 1) == 1 ? hi.y : (e >> 1) == 2 ? hi.z : hi.w;
-              o[p2] = tc::prmt(wl, wh, sel);
-            }
-            *reinterpret_cast<uint4*>(xt + (c * 8 + e) * kT + 8 * j) = make_uint4(o[0], o[1], o[2], o[3]);
+          for (int p2 = 0; p2 < 4; ++p2) {
+            const uint4& lo = v[2 * p2];
+            const uint4& hi = v[2 * p2 + 1];
+            const uint32_t wl = (e >> 1) == 0 ? lo.x : (e >> 1) == 1 ? lo.y : (e >> 1) == 2 ? lo.z : lo.w;
+            const uint32_t wh = (e >> 1) == 0 ? hi.x : (e >> 1) == 1 ? hi.y : (e >> 1) == 2 ? hi.z : hi.w;
+            o[p2] = tc::prmt(wl, wh, sel);
           }
+          *reinterpret_cast<uint4*>(xt + (c * 8 + e) * kT + 8 * j) = make_uint4(o[0], o[1], o[2], o[3]);
         }
       }
       workers_sync();
@@ -295,7 +294,7 @@ szo_linear_skinny_kernel(const uint8_t* __restrict__ codes_tiled, const float2* 
       // global memory (row pointers, then entries) are software-pipelined over tiles: the row
       // pointers of tile it + 2 and the first chunk of entries of tile it + 1 are in flight while
       // tile it is summed.
-      constexpr int kGatherQ = kSpChunk / 32;                            // entries per lane whose activations are fetched at once
+      constexpr int kGatherQ = kSpChunk / 32 / kNT;                      // entries per lane whose activations are fetched at once
       const int r = sp_r, h = lane & 1;
       auto load_entries = [&](int32_t base, int32_t end, int (&col)[kSpChunk / 32], float (&val)[kSpChunk / 32]) {
 #pragma unroll
@@ -387,18 +386,22 @@ szo_linear_skinny_kernel(const uint8_t* __restrict__ codes_tiled, const float2* 
         cluster_wait();
         const int64_t n = static_cast<int64_t>(tile) * kRowsCta + rank * kRowsWarp + r;
         const float bv = (bias != nullptr && n < N) ? bias[n] : 0.f;
-        float pv[kSplit][kT / 2], v[kT / 2];
+        float v[kT / 2];
 #pragma unroll
-        for (int cta = 0; cta < kSplit; ++cta) {                       // all loads first, then the sums in CTA order
-          const uint32_t src = cluster_addr(part[it & 1] + (rank * kRowsWarp + r) * kT + h, static_cast<uint32_t>(cta));
+        for (int j0 = 0; j0 < kT / 2; j0 += 4) {                       // four tokens at a time
+          float pv[kSplit][4];
 #pragma unroll
-          for (int j = 0; j < kT / 2; ++j) pv[cta][j] = ld_cluster_f32(src + 8u * j);
-        }
+          for (int cta = 0; cta < kSplit; ++cta) {                     // all loads first, then the sums in CTA order
+            const uint32_t src = cluster_addr(part[it & 1] + (rank * kRowsWarp + r) * kT + h, static_cast<uint32_t>(cta));
 #pragma unroll
-        for (int j = 0; j < kT / 2; ++j) {
-          v[j] = pv[0][j];
+            for (int j = 0; j < 4; ++j) pv[cta][j] = ld_cluster_f32(src + 8u * (j0 + j));
+          }
 #pragma unroll
-          for (int cta = 1; cta < kSplit; ++cta) v[j] += pv[cta][j];
+          for (int j = 0; j < 4; ++j) {
+            v[j0 + j] = pv[0][j];
+#pragma unroll
+            for (int cta = 1; cta < kSplit; ++cta) v[j0 + j] += pv[cta][j];
+          }
         }
 #pragma unroll
         for (int j = 0; j < kT / 2; ++j) {
@@ -479,7 +482,7 @@ szo_linear_skinny_kernel(const uint8_t* __restrict__ codes_tiled, const float2* 
         for (int i = 0; i < my_steps; i += 2) {
           const bool two = i + 1 < my_steps;
           tc::RingPos c1 = c;
-          c1.advance(kStages);
+          c1.advance(n_stages);
           if (!failed && !tc::mbar_wait(full_bar(c.idx), c.phase, abort_flag, status)) failed = true;
           if (two && !failed && !tc::mbar_wait(full_bar(c1.idx), c1.phase, abort_flag, status)) failed = true;
           step_body(i, ring + c.idx * stage_bytes);
@@ -490,7 +493,7 @@ szo_linear_skinny_kernel(const uint8_t* __restrict__ codes_tiled, const float2* 
             if (two) tc::mbar_arrive(empty_bar(c1.idx));
           }
           c = c1;
-          if (two) c.advance(kStages);
+          if (two) c.advance(n_stages);
         }
         // accumulator layout: [0], [1] = (row g, tokens 2t, 2t+1); [2], [3] = (row g+8, same tokens)
         cluster_wait();                                   // number it: the tile of two turns ago is summed, its buffer free
@@ -512,18 +515,26 @@ szo_linear_skinny_kernel(const uint8_t* __restrict__ codes_tiled, const float2* 
   cluster_wait();
 }
 
-size_t skinny_dyn_smem(int64_t K, int G, int kT) {
+size_t skinny_dyn_smem(int64_t K, int G, int kT, int n_stages = kStages) {
   const int64_t n_steps = K / kStepK, max_steps = ceil_div(n_steps, kSplit);
   const size_t ngs = (G >= kStepK) ? 1 : kStepK / G;
   const size_t stage = (static_cast<size_t>(kSzOff) + ngs * 1024 + 127) & ~static_cast<size_t>(127);
-  return kStages * stage + static_cast<size_t>(kT) * (max_steps * kStepK + kPad) * 2 + static_cast<size_t>(max_steps) * kT * 4 +
+  return n_stages * stage + static_cast<size_t>(kT) * (max_steps * kStepK + kPad) * 2 + static_cast<size_t>(max_steps) * kT * 4 +
          static_cast<size_t>(max_steps) * kStepK * kT * 2;     // ring, x [token][column], step sums, x [column][token]
 }
 
 template <bool kBf16Tables, bool kGroupMma, typename TY, int kNT>
 szo_status launch_skinny(const szo_linear* p, const void* x, int64_t M, const float* S, void* y, cudaStream_t st) {
   auto kern = szo_linear_skinny_kernel<kBf16Tables, kGroupMma, TY, kNT>;
-  const size_t smem = skinny_dyn_smem(p->K, p->G, kTok * kNT);
+  // A ring of 8 steps when two CTAs of that size still share an SM (or when 4 would not change that
+  // either), else 4: two CTAs with 4 steps in flight each hide more than one with 8.
+  constexpr size_t kStaticSmem = (kNT == 1) ? 14 * 1024 : 28 * 1024;            // upper bounds of the kernel's static arrays
+  constexpr size_t kTwoPerSm = (227 * 1024) / 2 - 1024;                         // per CTA, 1 KB reserved by the driver each
+  int n_stages = kStages;
+  if (skinny_dyn_smem(p->K, p->G, kTok * kNT, kStages) + kStaticSmem > kTwoPerSm &&
+      skinny_dyn_smem(p->K, p->G, kTok * kNT, kStages / 2) + kStaticSmem <= kTwoPerSm)
+    n_stages = kStages / 2;
+  const size_t smem = skinny_dyn_smem(p->K, p->G, kTok * kNT, n_stages);
   static bool configured = false;
   if (!configured) {
     SZO_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynSmem)));
@@ -547,7 +558,7 @@ szo_status launch_skinny(const szo_linear* p, const void* x, int64_t M, const fl
   const int n_clusters = n_tiles < max_clusters ? n_tiles : max_clusters;
   kern<<<static_cast<unsigned>(kSplit * n_clusters), kThreads, smem, st>>>(
       p->codes_tiled, p->sz, p->Npad, static_cast<const __nv_bfloat16*>(x), p->nnz > 0 ? p->row_ptr : nullptr, p->ent_col,
-      S, p->bias, static_cast<TY*>(y), static_cast<int>(M), p->N, p->K, p->G, n_tiles, status);
+      S, p->bias, static_cast<TY*>(y), static_cast<int>(M), p->N, p->K, p->G, n_tiles, n_stages, status);
   count_launch();
   SZO_CHECK_LAUNCH("szo_linear_skinny_kernel");
   return SZO_OK;
