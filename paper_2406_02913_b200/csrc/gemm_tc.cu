@@ -318,13 +318,78 @@ size_t tc_materialised_ws_bytes(const szo_linear* const* plans, int n, int64_t M
          round_up(nnz * sizeof(__nv_bfloat16), 256) + tc_tail_ws_bound();
 }
 
+// Resident form (dense bf16 plans, G == 0).  With nothing to dequantise, the effective weight of a
+// launch group can stay in device memory across calls: a private copy [sum Npad, K] of the group's
+// frozen weights, made once, plus the frozen values at the masked positions.  A forward then only
+// rewrites the masked entries (RN_bf16(frozen + S), the SparseAdd of the appendix on sparse
+// operations) and runs the dense mode of the kernel; no entry needs restoring afterwards, because the
+// next scatter writes every masked position again from the saved frozen value.
+bool tc_use_resident(const szo_linear* p, int64_t M) {
+  if (p->G != 0 || p->tc == nullptr) return false;
+  const int o = materialise_override();
+  if (o >= 0) return o == 1;
+  return M >= 4096;
+}
+
+bool tc_can_stack(const szo_linear* const* plans, int n) {
+  if (n < 1 || n > 3) return false;
+  for (int i = 0; i < n; ++i)
+    if (plans[i]->G != 0 || plans[i]->tc == nullptr || plans[i]->K != plans[0]->K) return false;
+  return true;
+}
+
+void tc_resident_bytes(const szo_linear* const* plans, int n, size_t* w_bytes, size_t* saved_bytes) {
+  size_t rows = 0, nnz = 0;
+  for (int i = 0; i < n; ++i) {
+    rows += static_cast<size_t>(plans[i]->Npad);
+    nnz += static_cast<size_t>(plans[i]->nnz);
+  }
+  *w_bytes = round_up(rows * static_cast<size_t>(plans[0]->K) * sizeof(__nv_bfloat16), 256);
+  *saved_bytes = round_up(nnz * sizeof(__nv_bfloat16), 256);
+}
+
+namespace {
+__global__ void gather_bf16_kernel(const __nv_bfloat16* __restrict__ W, const int64_t* __restrict__ idx, int64_t nnz,
+                                   __nv_bfloat16* __restrict__ out) {
+  const int64_t e = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (e < nnz) out[e] = W[idx[e]];
+}
+}  // namespace
+
+// Fills the resident buffers of one launch group: rows [0, N) of every matrix copied from the frozen
+// weight, the padding rows zero, saved[e] = the frozen value at masked position e.
+szo_status tc_resident_init(const szo_linear* const* plans, int n, __nv_bfloat16* W, __nv_bfloat16* saved,
+                            cudaStream_t st) {
+  SZO_REQUIRE(tc_can_stack(plans, n), SZO_ERR_INVALID_ARG, "resident form: dense bf16 plans with one K only");
+  int64_t row0 = 0, nnz = 0;
+  for (int i = 0; i < n; ++i) {
+    const szo_linear* p = plans[i];
+    __nv_bfloat16* dst = W + row0 * p->K;
+    SZO_CHECK_CUDA(cudaMemcpyAsync(dst, p->codes, static_cast<size_t>(p->N) * p->K * sizeof(__nv_bfloat16),
+                                   cudaMemcpyDeviceToDevice, st));
+    if (p->Npad > p->N)
+      SZO_CHECK_CUDA(cudaMemsetAsync(dst + p->N * p->K, 0, static_cast<size_t>(p->Npad - p->N) * p->K * sizeof(__nv_bfloat16), st));
+    if (p->nnz > 0) {
+      gather_bf16_kernel<<<static_cast<unsigned>(ceil_div(p->nnz, 256)), 256, 0, st>>>(
+          static_cast<const __nv_bfloat16*>(p->codes), p->idx, p->nnz, saved + nnz);
+      count_launch();
+    }
+    nnz += p->nnz;
+    row0 += p->Npad;
+  }
+  SZO_CHECK_LAUNCH("gather_bf16_kernel");
+  return SZO_OK;
+}
+
 // n matrices that share x (n == 1 or tc_can_fuse): materialise, SparseAdd, dense launch.  With
 // S_second != nullptr the weight pass serves two sets of sparse values (S_pert and S_second) and two
 // sets of M tokens each: x and every y[i] then hold 2 M rows, set 0 first.
 szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, const void* x, int64_t M,
                                       const float* const* S_pert, void* const* y, int y_dtype, void* ws,
-                                      size_t ws_bytes, cudaStream_t st, const float* const* S_second) {
+                                      size_t ws_bytes, cudaStream_t st, const float* const* S_second,
+                                      __nv_bfloat16* W_resident, __nv_bfloat16* saved_resident) {
   const szo_linear* p0 = plans[0];
+  const bool resident = W_resident != nullptr;
   const TcPlan* t = static_cast<const TcPlan*>(p0->tc);
   SZO_REQUIRE(t != nullptr, SZO_ERR_INVALID_ARG, "plan has no tensor-core data");
   SZO_REQUIRE(M < (int64_t(1) << 31), SZO_ERR_SHAPE, "M too large");
@@ -334,13 +399,17 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
     rows += plans[i]->Npad;
     nnz_all += static_cast<size_t>(plans[i]->nnz);
   }
-  const size_t w_bytes = round_up(static_cast<size_t>(rows) * p0->K * sizeof(__nv_bfloat16), 256);
-  const size_t saved_bytes = round_up(nnz_all * sizeof(__nv_bfloat16), 256);
-  SZO_REQUIRE(ws != nullptr && ws_bytes >= w_bytes + saved_bytes, SZO_ERR_WORKSPACE,
+  // resident form: the weight and the dense values at the masked positions live in the caller's buffers
+  const size_t w_bytes = resident ? 0 : round_up(static_cast<size_t>(rows) * p0->K * sizeof(__nv_bfloat16), 256);
+  const size_t saved_bytes = resident ? 0 : round_up(nnz_all * sizeof(__nv_bfloat16), 256);
+  SZO_REQUIRE(resident || (ws != nullptr && ws_bytes >= w_bytes + saved_bytes), SZO_ERR_WORKSPACE,
               "the materialised form needs a workspace of at least %zu bytes", w_bytes + saved_bytes);
+  SZO_REQUIRE(!resident || nnz_all == 0 || saved_resident != nullptr, SZO_ERR_INVALID_ARG,
+              "resident form without the saved dense values");
   SZO_REQUIRE(rows < (int64_t(1) << 31), SZO_ERR_SHAPE, "too many weight rows in one launch");
-  __nv_bfloat16* W = static_cast<__nv_bfloat16*>(ws);
-  __nv_bfloat16* saved = reinterpret_cast<__nv_bfloat16*>(static_cast<unsigned char*>(ws) + w_bytes);
+  __nv_bfloat16* W = resident ? W_resident : static_cast<__nv_bfloat16*>(ws);
+  __nv_bfloat16* saved = resident ? saved_resident
+                                  : reinterpret_cast<__nv_bfloat16*>(static_cast<unsigned char*>(ws) + w_bytes);
   const int nkb = static_cast<int>(p0->K / kBK);
   MatArgs a{};
   a.n = n; a.nkb = nkb; a.G = p0->G; a.K = p0->K;
@@ -352,10 +421,12 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
     nnz += p->nnz;
     row0 += p->Npad;
   }
-  if (p0->sz_dtype == SZO_BF16) materialise_kernel<true><<<static_cast<unsigned>(ceil_div(words, 256)), 256, 0, st>>>(a);
-  else materialise_kernel<false><<<static_cast<unsigned>(ceil_div(words, 256)), 256, 0, st>>>(a);
-  count_launch();
-  SZO_CHECK_LAUNCH("materialise_kernel");
+  if (!resident) {
+    if (p0->sz_dtype == SZO_BF16) materialise_kernel<true><<<static_cast<unsigned>(ceil_div(words, 256)), 256, 0, st>>>(a);
+    else materialise_kernel<false><<<static_cast<unsigned>(ceil_div(words, 256)), 256, 0, st>>>(a);
+    count_launch();
+    SZO_CHECK_LAUNCH("materialise_kernel");
+  }
   CUtensorMap mw;
   SZO_TRY(make_map(&mw, W, rows, p0->K, kBM));
   TcParams P{};
@@ -383,9 +454,9 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
   SZO_REQUIRE(P.status != nullptr, SZO_ERR_CUDA, "no device status word");
   const int64_t tiles = P.m_tiles * P.n_tiles;
   SZO_REQUIRE(tiles < (int64_t(1) << 30), SZO_ERR_SHAPE, "too many tiles");
-  void* tail = static_cast<unsigned char*>(ws) + w_bytes + saved_bytes;
-  const size_t tail_bytes = ws_bytes - w_bytes - saved_bytes;
-  PairSchedule sc = pair_schedule(tiles, P.nkb, 0, t->sms, true);
+  void* tail = ws == nullptr ? nullptr : static_cast<unsigned char*>(ws) + w_bytes + saved_bytes;
+  const size_t tail_bytes = ws == nullptr ? 0 : ws_bytes - w_bytes - saved_bytes;
+  PairSchedule sc = pair_schedule(tiles, P.nkb, 0, t->sms, tail != nullptr);
   if (sc.ws_bytes > tail_bytes) sc = pair_schedule(tiles, P.nkb, 0, t->sms, false);
   P.full_rounds = sc.full_rounds;
   P.tail_tiles = sc.tail_tiles;
@@ -397,7 +468,7 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
   const int n_sets = S_second != nullptr ? 2 : 1;
   for (int set = 0; set < n_sets; ++set) {
     if (nnz > 0) {
-      a.scatter_mode = n_sets == 1 ? 0 : set + 1;
+      a.scatter_mode = resident ? 2 : (n_sets == 1 ? 0 : set + 1);
       if (set == 1)
         for (int i = 0; i < n; ++i) a.sub[i].S = S_second[i];
       scatter_add_bf16_kernel<<<static_cast<unsigned>(ceil_div(nnz, 256)), 256, 0, st>>>(a);

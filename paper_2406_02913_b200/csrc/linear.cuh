@@ -68,7 +68,16 @@ bool tc_use_materialised(const szo_linear* p, int64_t M);
 size_t tc_materialised_ws_bytes(const szo_linear* const* plans, int n, int64_t M);
 szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, const void* x, int64_t M,
                                       const float* const* S_pert, void* const* y, int y_dtype, void* ws,
-                                      size_t ws_bytes, cudaStream_t st, const float* const* S_second = nullptr);
+                                      size_t ws_bytes, cudaStream_t st, const float* const* S_second = nullptr,
+                                      __nv_bfloat16* W_resident = nullptr, __nv_bfloat16* saved_resident = nullptr);
+// Resident form for dense bf16 plans (G == 0): W_resident [sum Npad, K] and saved_resident [sum nnz]
+// are filled once by tc_resident_init and passed to linear_fwd_tc_materialised, which then skips the
+// weight pass and writes every masked entry as RN_bf16(saved + S); ws is only the K-split scratch.
+bool tc_use_resident(const szo_linear* p, int64_t M);
+bool tc_can_stack(const szo_linear* const* plans, int n);
+void tc_resident_bytes(const szo_linear* const* plans, int n, size_t* w_bytes, size_t* saved_bytes);
+szo_status tc_resident_init(const szo_linear* const* plans, int n, __nv_bfloat16* W, __nv_bfloat16* saved,
+                            cudaStream_t st);
 // S_second: a second set of sparse values and of M tokens served by the same weight pass (x and
 // y[i] hold 2 M rows).
 // out[p] = (pos[p], bits of S[eid[p]]) for p in [0, n)

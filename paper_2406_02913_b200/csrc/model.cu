@@ -362,6 +362,10 @@ struct szo_model {
   float* zkept = nullptr;       // [k_total] z of the current step, kept by the first perturb pass
   float *Splus = nullptr, *Sminus = nullptr;   // [k_total] the two perturbed copies of S (two forwards side by side)
   bool dual_rows = false;       // the activation buffers hold 2 * Mmax rows
+  // dense bf16 weights (group == 0) with many tokens: every launch group keeps its effective weight
+  // resident (a private copy of the frozen matrices, masked entries rewritten per forward)
+  bool resident = false;
+  std::vector<__nv_bfloat16*> res_W, res_saved;   // indexed by the first linear of a group; else nullptr
   int64_t Mmax = 0;
   // activations
   float* h = nullptr;
@@ -453,12 +457,13 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
       plans[i] = m->plans[t0 + i];
       recs[i] = m->recs + m->offsets[t0 + i];
     }
-    if (nsets == 1 && !(pregather && sizeof(T) == 2 && (n == 1 || tc_can_fuse(plans, n, M)))) {
+    const bool res = m->resident && sizeof(T) == 2;
+    if (!res && nsets == 1 && !(pregather && sizeof(T) == 2 && (n == 1 || tc_can_fuse(plans, n, M)))) {
       for (int i = 0; i < n; ++i) SZO_TRY(lin_single(layer, j0 + i, x, outs[i]));
       return SZO_OK;
     }
-    if (nsets == 1 && n == 1) return lin_single(layer, j0, x, outs[0]);
-    const bool mat = nsets == 2 || tc_use_materialised(plans[0], M);
+    if (!res && nsets == 1 && n == 1) return lin_single(layer, j0, x, outs[0]);
+    const bool mat = res || nsets == 2 || tc_use_materialised(plans[0], M);
     const float* spert[3];
     const float* spert2[3];
     for (int i = 0; i < n; ++i) {
@@ -474,7 +479,8 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
       SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used], st));
     }
     const szo_status rc = mat ? linear_fwd_tc_materialised(plans, n, x, M, spert, outs, act, m->ws, m->ws_bytes, st,
-                                                           nsets == 2 ? spert2 : nullptr)
+                                                           nsets == 2 ? spert2 : nullptr, res ? m->res_W[t0] : nullptr,
+                                                           res ? m->res_saved[t0] : nullptr)
                               : linear_fwd_tc_group(plans, n, x, M, recs, outs, act, m->ws, m->ws_bytes, st);
     if (m->timing) {
       SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used + 1], st));
@@ -493,7 +499,7 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
     count_launch();
   }
   // One gather of all sparse values into the bucket order of every linear (SparseAdd mode)
-  if (nsets == 1 && pregather && !(m->plans.size() > 0 && tc_use_materialised(m->plans[0], M)))
+  if (nsets == 1 && pregather && !m->resident && !(m->plans.size() > 0 && tc_use_materialised(m->plans[0], M)))
     SZO_TRY(gather_values(Sv, m->geid, m->gpos, m->k_total, m->recs, st));
   const T* pending = nullptr;     // projection output still to be added to the residual stream
   for (int l = 0; l < c.n_layers; ++l) {
@@ -580,7 +586,7 @@ szo_status run_loss(szo_model* m, const int32_t* tokens, const int32_t* labels, 
 bool dual_forward_applies(const szo_model* m, int64_t M) {
   return m->dual_rows && m->cfg.act_dtype != SZO_F32 && m->cfg.linear_mode != SZO_MODE_FP32_VALIDATE &&
          m->cfg.linear_mode != SZO_MODE_SPMM && !m->plans.empty() && m->k_total > 0 &&
-         tc_use_materialised(m->plans[0], M);
+         (m->resident || tc_use_materialised(m->plans[0], M));
 }
 
 szo_status check_batch(const szo_model* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand, int B,
@@ -676,6 +682,28 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
   }
   m->k_total = m->offsets.back();
   if (m->k_total > 0 && S_all == nullptr) return bail(fail(SZO_ERR_INVALID_ARG, "S_all is NULL"));
+  // resident effective weights of the launch groups (dense bf16 weights, many tokens)
+  m->resident = c.group == 0 && c.act_dtype == SZO_BF16 && c.linear_mode != SZO_MODE_FP32_VALIDATE &&
+                c.linear_mode != SZO_MODE_SPMM && !m->plans.empty() && tc_use_resident(m->plans[0], m->Mmax);
+  if (m->resident) {
+    m->res_W.assign(m->plans.size(), nullptr);
+    m->res_saved.assign(m->plans.size(), nullptr);
+    const int n_groups = 4;
+    const int g_first[4] = {0, 3, 4, c.arch == 0 ? 6 : 5};
+    const int g_count[4] = {3, 1, c.arch == 0 ? 2 : 1, 1};
+    for (int l = 0; l < c.n_layers; ++l) {
+      for (int g = 0; g < n_groups; ++g) {
+        const size_t t0 = static_cast<size_t>(l) * m->n_lin + g_first[g];
+        const szo_linear* const* pl = m->plans.data() + t0;
+        if (!tc_can_stack(pl, g_count[g])) return bail(fail(SZO_ERR_UNSUPPORTED, "resident form: group cannot be stacked"));
+        size_t wb = 0, sb = 0;
+        tc_resident_bytes(pl, g_count[g], &wb, &sb);
+        SZO_M_TRY(dev_alloc(m, &m->res_W[t0], wb));
+        SZO_M_TRY(dev_alloc(m, &m->res_saved[t0], sb));
+        SZO_M_TRY(tc_resident_init(pl, g_count[g], m->res_W[t0], m->res_saved[t0], st));
+      }
+    }
+  }
   if (c.loss_kind == 0) {
     SZO_M_TRY(szo_linear_create(&m->lm_head_plan, c.vocab, c.d_model, 0, top->lm_head, nullptr, nullptr, SZO_BF16,
                                 nullptr, 0, nullptr, st));
@@ -691,7 +719,7 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
     const char* env = getenv("SZO_DUAL_FORWARD");
     m->dual_rows = !(env != nullptr && env[0] == '0') && c.act_dtype != SZO_F32 &&
                    c.linear_mode != SZO_MODE_FP32_VALIDATE && c.linear_mode != SZO_MODE_SPMM && !m->plans.empty() &&
-                   m->k_total > 0 && tc_use_materialised(m->plans[0], m->Mmax);
+                   m->k_total > 0 && (m->resident || tc_use_materialised(m->plans[0], m->Mmax));
   }
   const int64_t Mx = m->Mmax * (m->dual_rows ? 2 : 1), d = c.d_model, dkv = static_cast<int64_t>(c.n_kv_heads) * hd,
                 ff = c.d_ff;

@@ -4,6 +4,7 @@
     python -m paper_2406_02913_b200.microbench sparse --k 6476005
     python -m paper_2406_02913_b200.microbench steady --M 8 --N 11008 --K 4096 --mode auto
     python -m paper_2406_02913_b200.microbench sweep            # the single-linear and k-sweep cases
+    python -m paper_2406_02913_b200.microbench step --model opt_13b --batch 8 --seq 512 --loss lm
 
 linear: x bf16 [M,K] ~ N(0,1); W [N,K] int4 group-128 with bf16 scales/zeros quantized (by the
 library) from N(0,0.02); 0.1 % sparse entries chosen as the top-k of squared Student-t(3) scores
@@ -216,9 +217,58 @@ def attention_case(Bn, S, H, Hkv, hd, reps):
                       "tflops_causal": flops / (med * 1e-3) / 1e12}), flush=True)
 
 
+def step_case(name, Bn, S, loss, steps, eps, lr):
+    """A full ZO step of a whole decoder shape (random-init weights in device memory), timed like
+    bench.py: CUDA events around `steps` back-to-back steps after three warm-up steps; the weights
+    streamed per forward exceed L2."""
+    shape = wl.MODEL_SHAPES[name]
+    tensors, S_all = wl.device_decoder_tensors(shape, seed=0)
+    loss_kind = B.LOSS_CLS2 if loss == "cls2" else B.LOSS_LM
+    model = B.Model(shape, wl.linear_names(shape), tensors, S_all, act_dtype=B.SZO_BF16,
+                    linear_mode=B.MODE_SPARSE_ADD, loss_kind=loss_kind, max_batch=Bn, max_seq=S)
+    n = 3 + steps
+    toks = [torch.from_numpy(wl.token_batch(shape["vocab"], Bn, S, 0, wl.PURPOSE_TRAIN_BATCH, i)).cuda() for i in range(n)]
+    labs = [torch.from_numpy(wl.binary_labels(Bn, 0, i)).cuda() for i in range(n)] if loss == "cls2" else [None] * n
+    cand = torch.tensor([9906, 13], dtype=torch.int32).cuda() if loss == "cls2" else None
+    for i in range(3):
+        model.zo_step(toks[i], 1234, i, eps, lr, labs[i], cand)
+    torch.cuda.synchronize()
+    model.enable_timing(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(3, n):
+        model.zo_step(toks[i], 1234, i, eps, lr, labs[i], cand)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    lin_ms, lin_launches = model.linear_time()
+    model.enable_timing(False)
+    M = Bn * S
+    flops = 2 * steps * shape["n_layers"] * sum(2 * M * nn * kk for nn, kk in
+                                                 (wl.linear_shape(shape, nm) for nm in wl.linear_names(shape)))
+    sus = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))).get("bf16_tflops_sustained") \
+        if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else 1400.0
+    last = model._scalars[:3].cpu().numpy()
+    ach = flops / (lin_ms * 1e-3) / 1e12
+    print(json.dumps({"case": "step", "model": name, "batch": Bn, "seq": S, "loss": loss, "k": int(model.k_total),
+                      "ms_per_step": ms, "steps_per_s": 1e3 / ms, "tokens_per_s": 1e3 / ms * M,
+                      "linear_ms_per_step": lin_ms / steps, "linear_launches_per_step": lin_launches / steps,
+                      "linear_tflops": ach, "frac_of_sustained_peak": ach / sus,
+                      "roofline_ms_per_step": flops / steps / sus / 1e9, "device_status": B.device_status(),
+                      "f_plus": float(last[0]), "f_minus": float(last[1]), "g": float(last[2])}))
+    model.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["linear", "steady", "sparse", "sweep", "attention"])
+    ap.add_argument("what", choices=["linear", "steady", "sparse", "sweep", "attention", "step"])
+    ap.add_argument("--model", default="mistral_7b", choices=sorted(wl.MODEL_SHAPES))
+    ap.add_argument("--batch", type=int, default=8)
+    ap.add_argument("--seq", type=int, default=512)
+    ap.add_argument("--loss", default="lm", choices=["lm", "cls2"])
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--eps", type=float, default=1e-3)
+    ap.add_argument("--lr", type=float, default=1e-6)
     ap.add_argument("--M", type=int, default=8192)
     ap.add_argument("--N", type=int, default=4096)
     ap.add_argument("--K", type=int, default=4096)
@@ -235,6 +285,8 @@ def main():
         steady_case(a.M, a.N, a.K, a.G, a.mode, a.rho, a.reps)
     elif a.what == "sparse":
         sparse_case(a.k, a.reps)
+    elif a.what == "step":
+        step_case(a.model, a.batch, a.seq, a.loss, a.steps, a.eps, a.lr)
     elif a.what == "attention":
         attention_case(16, 256, 32, 32, 128, a.reps)
         attention_case(8, 512, 32, 8, 128, a.reps)

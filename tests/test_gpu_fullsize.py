@@ -220,3 +220,55 @@ def test_two_full_width_layers_in_the_bench_configuration(B):
     assert m_tc.last_launches() < m_seq.last_launches()            # it really took the other route
     assert torch.equal(out_dual, out_seq) and torch.equal(S_tc, S_seq)
     assert not torch.equal(S_tc, S0)                               # and the update moved S
+
+
+def test_two_mistral_width_layers_resident_form(B):
+    """Two decoder layers at the Mistral-7B width (GQA 32/8, d_ff 14336, dense bf16 weights, 1 % mask)
+    with 8 x 512 tokens and the full-sequence loss.  At this token count the model keeps the effective
+    weight of every launch group resident and runs the two forwards of a step side by side.  Checked:
+    the loss against the library's fp32 validation path (pinned to the oracle by the small tests),
+    against the fused form of the same weights (a model created for fewer tokens), repeatability bit
+    for bit, and that a second step starts from clean weights (no masked entry keeps an old value)."""
+    shape = dict(wl.MODEL_SHAPES["mistral_7b"], n_layers=2)
+    tensors, S_all = wl.device_decoder_tensors(shape, seed=5)
+    names = wl.linear_names(shape)
+    Bn, S = 8, 512
+    toks = torch.from_numpy(wl.token_batch(shape["vocab"], Bn, S, 5, wl.PURPOSE_TRAIN_BATCH, 0)).cuda()
+    S_res, S_fused, S_ref = S_all.clone(), S_all.clone(), S_all.clone()
+    m_res = B.Model(shape, names, tensors, S_res, act_dtype=B.SZO_BF16, linear_mode=B.MODE_SPARSE_ADD,
+                    loss_kind=B.LOSS_LM, max_batch=Bn, max_seq=S)
+    m_fused = B.Model(shape, names, tensors, S_fused, act_dtype=B.SZO_BF16, linear_mode=B.MODE_SPARSE_ADD,
+                      loss_kind=B.LOSS_LM, max_batch=Bn - 1, max_seq=S)          # 3584 tokens: fused form
+    m_ref = B.Model(shape, names, tensors, S_ref, act_dtype=B.SZO_F32, linear_mode=B.MODE_FP32_VALIDATE,
+                    loss_kind=B.LOSS_LM, max_batch=Bn, max_seq=S)
+    f_res = float(m_res.loss(toks).item())
+    f_ref = float(m_ref.loss(toks).item())
+    assert np.isfinite(f_res) and np.isfinite(f_ref)
+    assert abs(f_res - f_ref) <= 1e-3 * abs(f_ref)                 # mean over 4088 positions
+    # the same 7 sequences through both forms: same bf16 weights, a different order of fp32 sums at most
+    sub = toks[:Bn - 1].contiguous()
+    a, b = float(m_res.loss(sub).item()), float(m_fused.loss(sub).item())
+    assert abs(a - b) <= 2e-4 * abs(b)
+    eps = 1e-4
+    S0 = S_res.clone()
+    out1 = m_res.zo_step(toks, 1234, 7, eps, 0.0).clone()
+    S_res.copy_(S0)
+    out2 = m_res.zo_step(toks, 1234, 7, eps, 0.0).clone()
+    torch.cuda.synchronize()
+    assert B.device_status() == 0
+    assert torch.equal(out1, out2)
+    fp, fm, g = (float(v) for v in out1.cpu())
+    assert abs(g - (fp - fm) / (2 * float(np.float32(eps)))) <= 1e-9 * max(1.0, abs(g))
+    assert abs(0.5 * (fp + fm) - f_res) <= 1e-3 * abs(f_res)
+    # after steps with other sparse values the unperturbed loss is reproduced bit for bit
+    S_res.copy_(S0)
+    assert float(m_res.loss(toks).item()) == f_res
+    # and the step of the fused form agrees on the smaller batch
+    o_res = m_res.zo_step(sub, 99, 3, eps, 1e-6).clone()
+    o_fused = m_fused.zo_step(sub, 99, 3, eps, 1e-6).clone()
+    torch.cuda.synchronize()
+    assert abs(float(o_res[0]) - float(o_fused[0])) <= 2e-4 * abs(float(o_fused[0]))
+    assert abs(float(o_res[1]) - float(o_fused[1])) <= 2e-4 * abs(float(o_fused[1]))
+    assert not torch.equal(S_res, S0)                              # the update moved S
+    for m in (m_res, m_fused, m_ref):
+        m.close()

@@ -200,3 +200,22 @@ def test_other_architectures_bf16_tensor_core_path(B, name, loss_kind, mode):
     assert abs(out[0] - fp) <= tol * abs(fp) and abs(out[1] - fm) <= tol * abs(fm)
     assert np.isfinite(out[2]) and B.device_status() == 0
     m.close()
+
+
+def test_resident_and_materialised_forms_at_test_size():
+    """The forms that large token counts select (int4: effective weight materialised per launch group;
+    dense bf16: effective weight resident per launch group, masked entries rewritten per forward) are
+    forced at test size, where the oracle can check them: SZO_LINEAR_MATERIALISE=1 is read once per
+    process, so the oracle-parity tests of the three architectures run again in a child process."""
+    import os
+    import subprocess
+    import sys
+    env = dict(os.environ, SZO_LINEAR_MATERIALISE="1")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", "-p", "no:cacheprovider",
+                          os.path.join(root, "tests", "test_gpu_model.py"), "-k",
+                          "test_other_architectures_bf16_tensor_core_path or test_bf16_tensor_core_path_losses "
+                          "or test_host_buffer_step_equals_device_step"],
+                         cwd=root, env=env, capture_output=True, text=True, timeout=900)
+    assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-2000:]
+    assert " passed" in res.stdout
