@@ -17,6 +17,9 @@ quantize_int4     Section 3.5 "Integration with quantization": a 4-bit quantizer
                   The paper allows any post-training quantizer; the convention here (uniform,
                   asymmetric, group-wise, round-half-even) is parity unpinned by the paper.
 dequantize        the inverse map, exact in fp64.
+dequantize_lut    Section 4 / appendix on hyperparameters: the experiments quantize with a non-uniform
+                  4-bit format (SqueezeLLM), i.e. a code selects one of 16 per-output-channel
+                  values.  The inverse map is that table look-up, exact in fp64.
 effective_weight  Appendix "Implementation of Sparse Operations in Linear Layers":
                   Dequantize(Q(w_dense)) + w_sparse.
 linear_fwd        the same appendix: y = x (Dequantize(Q(w_dense)) + w_sparse)^T.
@@ -218,6 +221,20 @@ def dequantize(codes, s_bits, z_bits, G: int, fmt: str) -> np.ndarray:
     s = bits16_to_f32(s_bits, fmt).astype(np.float64)
     z = bits16_to_f32(z_bits, fmt).astype(np.float64)
     return q * np.repeat(s, G, axis=1) + np.repeat(z, G, axis=1)
+
+
+def dequantize_lut(codes, lut_bits, fmt: str) -> np.ndarray:
+    """Non-uniform 4-bit format: Dequantize(Q(w_dense))[n,c] = lut[n][q[n,c]], where row n of the
+    weight (one output channel) has its own table of 16 values stored in a 16-bit float format
+    (lut_bits: uint16 [N,16]).  Exact in fp64."""
+    q = unpack_codes(codes)
+    lut = bits16_to_f32(lut_bits, fmt).astype(np.float64)
+    N, K = q.shape
+    W = np.empty((N, K), dtype=np.float64)
+    for n in range(N):
+        for c in range(K):
+            W[n, c] = lut[n, q[n, c]]
+    return W
 
 
 # --------------------------------------------------------------------------- linear layer

@@ -214,6 +214,40 @@ def test_quantize_rejects_bad_input():
 
 
 # ------------------------------------------------------------------ sensitive mask
+def test_dequantize_lut_hand_values_and_reduction_to_the_uniform_format():
+    """Non-uniform 4-bit format (a code selects one of 16 per-row values).  Pinned by values written
+    out by hand (nibble order: low nibble = even column; the table is per row) and by the special case
+    of an arithmetic table j*s + z, where the look-up must equal the uniform format with one group
+    per row, which the quantizer tests pin."""
+    codes = np.array([[0x21, 0x43], [0xF0, 0x0F]], np.uint8)            # q = [1,2,3,4], [0,15,15,0]
+    lut = np.stack([10.0 + np.arange(16), -np.arange(16) / 4.0]).astype(np.float32)
+    for fmt in ("f16", "bf16"):
+        bits, vals = so.round_to_16(lut, fmt)
+        assert np.array_equal(vals, lut)                                   # representable in both formats
+        W = so.dequantize_lut(codes, bits, fmt)
+        assert np.array_equal(W, np.array([[11.0, 12.0, 13.0, 14.0], [0.0, -3.75, -3.75, 0.0]]))
+    r = np.random.default_rng(5)
+    N, K = 6, 64
+    codes = r.integers(0, 256, (N, K // 2), dtype=np.uint8)
+    s = (2.0 ** -r.integers(4, 8, N)).astype(np.float32)                   # powers of two: j*s + z is exact
+    z = (-8.0 * s).astype(np.float32)
+    lut = (np.arange(16, dtype=np.float32)[None, :] * s[:, None] + z[:, None]).astype(np.float32)
+    for fmt in ("f16", "bf16"):
+        lb, lv = so.round_to_16(lut, fmt)
+        assert np.array_equal(lv, lut)
+        sb, _ = so.round_to_16(s[:, None], fmt)
+        zb, _ = so.round_to_16(z[:, None], fmt)
+        assert np.array_equal(so.dequantize_lut(codes, lb, fmt), so.dequantize(codes, sb, zb, K, fmt))
+    # a table that is not arithmetic: every element is one of its row's 16 values, chosen by its code
+    lut = np.sort(r.normal(0, 0.02, (N, 16)).astype(np.float32), axis=1)
+    lb, lv = so.round_to_16(lut, "f16")
+    W = so.dequantize_lut(codes, lb, "f16")
+    q = so.unpack_codes(codes)
+    for n in range(N):
+        assert set(np.unique(W[n])) <= set(lv[n].astype(np.float64))
+        assert np.all(np.diff(W[n][np.argsort(q[n], kind="stable")]) >= 0)   # ascending table: monotone in the code
+
+
 def test_select_mask_brute_force_subsets():
     g = np.random.default_rng(3)
     for trial in range(30):
