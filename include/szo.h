@@ -153,6 +153,18 @@ szo_status szo_linear_create(szo_linear_t** out, int64_t N, int64_t K, int32_t G
                              const void* codes_or_bf16_W, const void* scales, const void* zeros,
                              szo_dtype sz_dtype, const int64_t* idx, int64_t nnz, const float* bias,
                              void* stream);
+/* Non-uniform 4-bit format (Section 4 and the hyperparameter appendix: the 4-bit experiments use
+ * SqueezeLLM, whose codes index a table of 16 values per output channel instead of a scale and a
+ * zero): Dequantize(Q(w_dense))[n,c] = lut[n][q[n,c]].  codes uint8 [N,K/2] as for szo_quantize
+ * (low nibble = even column); lut lut_dtype (SZO_F16 or SZO_BF16) [N,16], caller-owned like the
+ * codes; everything else as szo_linear_create.  How the table and the codes are fitted is the
+ * quantizer's business (the paper takes any post-training quantizer) and not part of this library.
+ * Such a plan runs in SZO_MODE_AUTO / SZO_MODE_SPARSE_ADD (for every M the effective bf16 weight
+ * RN_bf16(lut[n][q]) , RN_bf16(. + S) at the masked positions, is written to the workspace and then
+ * multiplied) and in SZO_MODE_FP32_VALIDATE; SZO_MODE_SPMM returns SZO_ERR_UNSUPPORTED. */
+szo_status szo_linear_create_lut(szo_linear_t** out, int64_t N, int64_t K, const uint8_t* codes,
+                                 const void* lut, szo_dtype lut_dtype, const int64_t* idx, int64_t nnz,
+                                 const float* bias, void* stream);
 /* x: x_dtype [M,K] (SZO_BF16; SZO_F32 also accepted in SZO_MODE_FP32_VALIDATE);
  * S_pert: fp32 [nnz] current (already perturbed) sparse values; y: y_dtype [M,N] (SZO_BF16 or
  * SZO_F32).  workspace: at least szo_linear_workspace_bytes(plan, M, mode) bytes (may be NULL

@@ -80,6 +80,8 @@ _SIGS = {
     "szo_linear_create": (C.c_int32, [C.POINTER(C.c_void_p), C.c_int64, C.c_int64, C.c_int32,
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
                                       C.c_int64, C.c_void_p, C.c_void_p]),
+    "szo_linear_create_lut": (C.c_int32, [C.POINTER(C.c_void_p), C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
+                                          C.c_int, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]),
     "szo_linear_fwd": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_void_p, C.c_void_p,
                                    C.c_int, C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p]),
     "szo_linear_workspace_bytes": (C.c_size_t, [C.c_void_p, C.c_int64, C.c_int32]),
@@ -213,14 +215,20 @@ def szo_update(S, idx, idx_base: int, seed: int, step: int, lr: float, f_plus, f
 class Linear:
     """Plan for one decomposed linear (szo_linear_create / szo_linear_fwd)."""
 
-    def __init__(self, N, K, G, codes_or_W, scales, zeros, sz_fmt, idx, bias=None):
-        self.N, self.K, self.G = N, K, G
-        self._keep = (codes_or_W, scales, zeros, idx, bias)      # plan borrows these buffers
+    def __init__(self, N, K, G, codes_or_W, scales, zeros, sz_fmt, idx, bias=None, lut=None):
+        """lut (16-bit float CUDA tensor [N,16]) selects the non-uniform 4-bit format
+        (szo_linear_create_lut); G, scales and zeros are then ignored."""
+        self.N, self.K, self.G = N, K, (-1 if lut is not None else G)
+        self._keep = (codes_or_W, scales, zeros, idx, bias, lut)      # plan borrows these buffers
         self.nnz = 0 if idx is None else idx.numel()
         h = C.c_void_p()
-        _check(lib().szo_linear_create(C.byref(h), N, K, G, _ptr(codes_or_W), _ptr(scales), _ptr(zeros),
-                                       SZ_FMT[sz_fmt][0], _ptr(idx) if self.nnz else None, self.nnz,
-                                       _ptr(bias), _stream()))
+        if lut is not None:
+            _check(lib().szo_linear_create_lut(C.byref(h), N, K, _ptr(codes_or_W), _ptr(lut), _DT[lut.dtype],
+                                               _ptr(idx) if self.nnz else None, self.nnz, _ptr(bias), _stream()))
+        else:
+            _check(lib().szo_linear_create(C.byref(h), N, K, G, _ptr(codes_or_W), _ptr(scales), _ptr(zeros),
+                                           SZ_FMT[sz_fmt][0], _ptr(idx) if self.nnz else None, self.nnz,
+                                           _ptr(bias), _stream()))
         self.h = h
         self._ws = None
 

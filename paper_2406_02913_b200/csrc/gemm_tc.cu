@@ -226,6 +226,7 @@ struct MatSub {
   const float* S;
   int64_t words_end, nnz_end; // running totals over the matrices: work items of this and the earlier ones
   __nv_bfloat16* saved;       // [nnz] dense values at the masked positions (two-set form)
+  const __nv_bfloat16* lut;   // [Npad][16] per-row table of the non-uniform 4-bit format (G == -1), else nullptr
 };
 struct MatArgs {
   MatSub sub[3];
@@ -238,7 +239,10 @@ struct MatArgs {
 // of one tile) -> four 16-byte pieces of the row-major output; the four loads are issued before the
 // first use.  A warp covers four k-blocks of one row at a time: 32-byte reads from four code
 // blocks, one 512-byte contiguous write.  Work items per matrix: (Npad / 128) * ceil(nkb / 4) * 1024.
-template <bool kFast>
+// kKind 0: fp32 (scale, zero) pairs; 1: packed bf16 pairs (exact bf16 arithmetic); 2: the non-uniform
+// format, where the code selects one of the 16 bf16 values of its row (a warp works on one row per
+// load, so the 32 look-ups of an instruction hit one 32-byte line).
+template <int kKind>
 __global__ void materialise_kernel(const MatArgs a) {
   int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i >= a.sub[a.n - 1].words_end) return;
@@ -256,18 +260,38 @@ __global__ void materialise_kernel(const MatArgs a) {
   const int kb = static_cast<int>(grp - t * nkb4) * 4 + kbo;
   if (kb >= a.nkb) return;
   const uint8_t* src = codes_tiled + (t * a.nkb + kb) * kCodesBytes + r0 * 32 + chunk * 4;
-  const int g = (kb * kBK + chunk * 8) / a.G;
-  const float2* szp = sz + static_cast<int64_t>(g) * Npad + t * kBM + r0;
-  uint32_t w[4];
-  float2 p[4];
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    w[j] = *reinterpret_cast<const uint32_t*>(src + j * 32 * 32);
-    p[j] = szp[j * 32];
-  }
   __nv_bfloat16* dst = out + (t * kBM + r0) * a.K + kb * kBK + chunk * 8;
+  uint32_t w[4];
+  if constexpr (kKind == 2) {
+    const __nv_bfloat16* lut = s == 0 ? a.sub[0].lut : (s == 1 ? a.sub[1].lut : a.sub[2].lut);
+    const unsigned short* row = reinterpret_cast<const unsigned short*>(lut) + (t * kBM + r0) * 16;
 #pragma unroll
-  for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(dst + static_cast<int64_t>(j) * 32 * a.K) = dequant_word<kFast>(w[j], p[j]);
+    for (int j = 0; j < 4; ++j) w[j] = *reinterpret_cast<const uint32_t*>(src + j * 32 * 32);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const unsigned short* rj = row + j * 32 * 16;
+      uint32_t o[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {       // nibble i is column 2 i, nibble 4 + i column 2 i + 1 (pair order)
+        const uint32_t lo = __ldg(rj + ((w[j] >> (4 * i)) & 0xFu));
+        const uint32_t hi = __ldg(rj + ((w[j] >> (16 + 4 * i)) & 0xFu));
+        o[i] = lo | (hi << 16);
+      }
+      *reinterpret_cast<uint4*>(dst + static_cast<int64_t>(j) * 32 * a.K) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+  } else {
+    const int g = (kb * kBK + chunk * 8) / a.G;
+    const float2* szp = sz + static_cast<int64_t>(g) * Npad + t * kBM + r0;
+    float2 p[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      w[j] = *reinterpret_cast<const uint32_t*>(src + j * 32 * 32);
+      p[j] = szp[j * 32];
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      *reinterpret_cast<uint4*>(dst + static_cast<int64_t>(j) * 32 * a.K) = dequant_word<kKind == 1>(w[j], p[j]);
+  }
 }
 
 // SparseAdd on the materialised matrices: indices are unique, so no two threads touch one element.
@@ -302,6 +326,7 @@ int materialise_override() {
 
 bool tc_use_materialised(const szo_linear* p, int64_t M) {
   if (p->G == 0 || p->tc == nullptr) return false;
+  if (p->G < 0) return true;      // table-coded weights have this form only
   const int o = materialise_override();
   if (o >= 0) return o == 1;
   // the extra pass costs about 2.5 N K bytes of traffic, the fused conversion 5-10 % of 2 M N K flop at
@@ -417,13 +442,17 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
   for (int i = 0; i < n; ++i) {
     const szo_linear* p = plans[i];
     words += (p->Npad / kBM) * ((nkb + 3) / 4) * 1024;
-    a.sub[i] = MatSub{p->codes_tiled, p->sz, p->Npad, W + row0 * p->K, p->idx, S_pert[i], words, nnz + p->nnz, saved + nnz};
+    SZO_REQUIRE(p->G == p0->G && p->K == p0->K, SZO_ERR_INVALID_ARG, "matrices of one launch must share K and format");
+    a.sub[i] = MatSub{p->codes_tiled, p->sz, p->Npad, W + row0 * p->K, p->idx, S_pert[i], words, nnz + p->nnz, saved + nnz,
+                      p->lut_bf16};
     nnz += p->nnz;
     row0 += p->Npad;
   }
   if (!resident) {
-    if (p0->sz_dtype == SZO_BF16) materialise_kernel<true><<<static_cast<unsigned>(ceil_div(words, 256)), 256, 0, st>>>(a);
-    else materialise_kernel<false><<<static_cast<unsigned>(ceil_div(words, 256)), 256, 0, st>>>(a);
+    const unsigned blocks = static_cast<unsigned>(ceil_div(words, 256));
+    if (p0->G < 0) materialise_kernel<2><<<blocks, 256, 0, st>>>(a);
+    else if (p0->sz_dtype == SZO_BF16) materialise_kernel<1><<<blocks, 256, 0, st>>>(a);
+    else materialise_kernel<0><<<blocks, 256, 0, st>>>(a);
     count_launch();
     SZO_CHECK_LAUNCH("materialise_kernel");
   }

@@ -215,6 +215,24 @@ sgemm_nt_kernel(const TA* __restrict__ A, const float* __restrict__ B, const flo
   }
 }
 
+// Non-uniform 4-bit format: W[n, c] = lut[n][q[n, c]] (fp32 holds a 16-bit float exactly).
+template <typename T>
+__global__ void dequant_lut_f32_kernel(const uint8_t* __restrict__ codes, const T* __restrict__ lut, int64_t N,
+                                       int64_t K, float* __restrict__ W) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;   // one byte: two columns
+  if (i >= N * (K / 2)) return;
+  const int64_t n = i / (K / 2);
+  const uint8_t b = codes[i];
+  W[2 * i] = static_cast<float>(lut[n * 16 + (b & 0xF)]);
+  W[2 * i + 1] = static_cast<float>(lut[n * 16 + (b >> 4)]);
+}
+
+template <typename T>
+__global__ void lut_to_bf16_kernel(const T* __restrict__ lut, int64_t n, __nv_bfloat16* __restrict__ out) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = __float2bfloat16_rn(static_cast<float>(lut[i]));
+}
+
 size_t linear_ws_fp32(const szo_linear* p, int64_t) {
   return round_up(static_cast<size_t>(p->N) * p->K * sizeof(float), 256);
 }
@@ -225,7 +243,14 @@ szo_status linear_fwd_fp32(const szo_linear* p, const void* x, int x_dtype, int6
               "fp32 path needs a workspace of %zu bytes", linear_ws_fp32(p, M));
   float* W = static_cast<float*>(ws);
   const int64_t NK = p->N * p->K;
-  if (p->G > 0) {
+  if (p->G < 0) {
+    if (p->sz_dtype == SZO_BF16)
+      dequant_lut_f32_kernel<__nv_bfloat16><<<static_cast<unsigned>(ceil_div(NK / 2, 256)), 256, 0, st>>>(
+          static_cast<const uint8_t*>(p->codes), static_cast<const __nv_bfloat16*>(p->lut), p->N, p->K, W);
+    else
+      dequant_lut_f32_kernel<__half><<<static_cast<unsigned>(ceil_div(NK / 2, 256)), 256, 0, st>>>(
+          static_cast<const uint8_t*>(p->codes), static_cast<const __half*>(p->lut), p->N, p->K, W);
+  } else if (p->G > 0) {
     if (p->sz_dtype == SZO_BF16)
       dequant_f32_kernel<__nv_bfloat16><<<static_cast<unsigned>(ceil_div(NK / 2, 256)), 256, 0, st>>>(
           static_cast<const uint8_t*>(p->codes), static_cast<const __nv_bfloat16*>(p->scales),
@@ -347,6 +372,8 @@ szo_status linear_fwd_impl(const szo_linear* p, const void* x, int x_dtype, int6
                            size_t workspace_bytes, cudaStream_t st) {
   if (mode == SZO_MODE_FP32_VALIDATE)
     return linear_fwd_fp32(p, x, x_dtype, M, S_pert, y, y_dtype, workspace, workspace_bytes, st);
+  SZO_REQUIRE(!(p->G < 0 && mode == SZO_MODE_SPMM), SZO_ERR_UNSUPPORTED,
+              "table-coded weights take the SparseAdd order only (SZO_MODE_AUTO or SZO_MODE_SPARSE_ADD)");
   if (mode == SZO_MODE_SPMM) {
     SZO_TRY(linear_fwd_tc(p, x, M, nullptr, y, y_dtype, workspace, workspace_bytes, st));
     return linear_spmm(p, x, M, S_pert, y, y_dtype, st);
@@ -371,6 +398,7 @@ static void free_plan(szo_linear* p) {
   if (!p) return;
   tc_plan_destroy(p);
   cudaFree(p->sz);
+  cudaFree(p->lut_bf16);
   cudaFree(p->codes_tiled);
   cudaFree(p->ent_col);
   cudaFree(p->row_ptr);
@@ -384,24 +412,25 @@ static void free_plan(szo_linear* p) {
 
 using namespace szo;
 
-extern "C" {
-
-szo_status szo_linear_create(szo_linear_t** out, int64_t N, int64_t K, int32_t G,
-                             const void* codes_or_bf16_W, const void* scales, const void* zeros,
-                             szo_dtype sz_dtype, const int64_t* idx, int64_t nnz, const float* bias,
-                             void* stream) {
+// G == -1: codes into the per-row table `lut` (type sz_dtype), scales/zeros unused.
+static szo_status create_plan(szo_linear_t** out, int64_t N, int64_t K, int32_t G,
+                              const void* codes_or_bf16_W, const void* scales, const void* zeros,
+                              const void* lut, szo_dtype sz_dtype, const int64_t* idx, int64_t nnz,
+                              const float* bias, void* stream) {
   SZO_REQUIRE(out != nullptr, SZO_ERR_INVALID_ARG, "out is NULL");
   *out = nullptr;
   SZO_REQUIRE(N > 0 && K > 0, SZO_ERR_SHAPE, "N and K must be positive");
   SZO_REQUIRE(K % 64 == 0, SZO_ERR_SHAPE, "K (%lld) must be a multiple of 64", (long long)K);
-  SZO_REQUIRE(G >= 0 && (G == 0 || ((G == 32 || G % 64 == 0) && K % G == 0)), SZO_ERR_SHAPE,
+  SZO_REQUIRE(G >= -1 && (G <= 0 || ((G == 32 || G % 64 == 0) && K % G == 0)), SZO_ERR_SHAPE,
               "G (%d) must be 0, 32 or a multiple of 64, and divide K", G);
+  SZO_REQUIRE(G != -1 || lut != nullptr, SZO_ERR_INVALID_ARG, "lut is NULL");
+  SZO_REQUIRE(aligned16(lut), SZO_ERR_ALIGNMENT, "lut must be 16-byte aligned");
   SZO_REQUIRE(N * K < (int64_t(1) << 40), SZO_ERR_SHAPE, "tensor too large");
   SZO_REQUIRE(nnz >= 0 && nnz <= N * K && nnz < (int64_t(1) << 31), SZO_ERR_INVALID_ARG, "bad nnz");
   SZO_REQUIRE(codes_or_bf16_W != nullptr, SZO_ERR_INVALID_ARG, "weight pointer is NULL");
-  SZO_REQUIRE(G == 0 || (scales && zeros), SZO_ERR_INVALID_ARG, "scales/zeros are NULL");
+  SZO_REQUIRE(G <= 0 || (scales && zeros), SZO_ERR_INVALID_ARG, "scales/zeros are NULL");
   SZO_REQUIRE(G == 0 || sz_dtype == SZO_BF16 || sz_dtype == SZO_F16, SZO_ERR_UNSUPPORTED,
-              "sz_dtype must be bf16 or f16");
+              "the 16-bit table type must be bf16 or f16");
   SZO_REQUIRE(nnz == 0 || idx != nullptr, SZO_ERR_INVALID_ARG, "idx is NULL");
   SZO_REQUIRE(aligned16(codes_or_bf16_W) && aligned16(scales) && aligned16(zeros) && aligned16(idx) &&
                   aligned16(bias),
@@ -411,6 +440,7 @@ szo_status szo_linear_create(szo_linear_t** out, int64_t N, int64_t K, int32_t G
   *p = szo_linear{};
   p->N = N; p->K = K; p->G = G; p->sz_dtype = sz_dtype; p->nnz = nnz;
   p->codes = codes_or_bf16_W; p->scales = scales; p->zeros = zeros; p->idx = idx; p->bias = bias;
+  p->lut = lut;
   p->n_rowgroups = ceil_div(N, 128);
   p->Npad = ceil_div(N, 256) * 256;   // the pair-tile kernel copies 128-row strips up to this bound
   p->n_kblocks = K / 64;
@@ -441,7 +471,17 @@ szo_status szo_linear_create(szo_linear_t** out, int64_t N, int64_t K, int32_t G
       widen_sz_kernel<__half><<<static_cast<unsigned>(ceil_div(ng, 256)), 256, 0, st>>>(
           static_cast<const __half*>(scales), static_cast<const __half*>(zeros), N, K / G, p->Npad, p->sz);
   }
-  if (G > 0) {
+  if (G < 0) {
+    SZO_PLAN_CUDA(cudaMalloc(&p->lut_bf16, p->Npad * 16 * sizeof(__nv_bfloat16)));
+    SZO_PLAN_CUDA(cudaMemsetAsync(p->lut_bf16, 0, p->Npad * 16 * sizeof(__nv_bfloat16), st));
+    if (sz_dtype == SZO_BF16)
+      lut_to_bf16_kernel<__nv_bfloat16><<<static_cast<unsigned>(ceil_div(N * 16, 256)), 256, 0, st>>>(
+          static_cast<const __nv_bfloat16*>(lut), N * 16, p->lut_bf16);
+    else
+      lut_to_bf16_kernel<__half><<<static_cast<unsigned>(ceil_div(N * 16, 256)), 256, 0, st>>>(
+          static_cast<const __half*>(lut), N * 16, p->lut_bf16);
+  }
+  if (G != 0) {
     const int64_t n_code_tiles = p->Npad / 128;      // padded to an even count for the pair-tile kernel
     const int64_t units = n_code_tiles * (K / 64) * 256;
     SZO_PLAN_CUDA(cudaMalloc(&p->codes_tiled, units * 16));
@@ -480,6 +520,22 @@ szo_status szo_linear_create(szo_linear_t** out, int64_t N, int64_t K, int32_t G
   cleanup(SZO_OK);
   *out = p;
   return SZO_OK;
+}
+
+extern "C" {
+
+szo_status szo_linear_create(szo_linear_t** out, int64_t N, int64_t K, int32_t G,
+                             const void* codes_or_bf16_W, const void* scales, const void* zeros,
+                             szo_dtype sz_dtype, const int64_t* idx, int64_t nnz, const float* bias,
+                             void* stream) {
+  SZO_REQUIRE(G >= 0, SZO_ERR_SHAPE, "G (%d) must be 0, 32 or a multiple of 64, and divide K", G);
+  return create_plan(out, N, K, G, codes_or_bf16_W, scales, zeros, nullptr, sz_dtype, idx, nnz, bias, stream);
+}
+
+szo_status szo_linear_create_lut(szo_linear_t** out, int64_t N, int64_t K, const uint8_t* codes,
+                                 const void* lut, szo_dtype lut_dtype, const int64_t* idx, int64_t nnz,
+                                 const float* bias, void* stream) {
+  return create_plan(out, N, K, -1, codes, nullptr, nullptr, lut, lut_dtype, idx, nnz, bias, stream);
 }
 
 size_t szo_linear_workspace_bytes(const szo_linear_t* p, int64_t M, int32_t mode) {

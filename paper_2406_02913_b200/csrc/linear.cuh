@@ -4,7 +4,7 @@
 
 struct szo_linear {
   int64_t N, K;
-  int32_t G;          // 0: dense bf16 weight
+  int32_t G;          // 0: dense bf16 weight; -1: 4-bit codes into a per-row table of 16 values (lut)
   int32_t sz_dtype;
   int64_t nnz;
   // caller-owned
@@ -25,6 +25,8 @@ struct szo_linear {
   uint16_t* bucket_pos;  // [nnz] byte offset of the element inside its swizzled [128 x 64] bf16 tile, bucket order
   int64_t n_rowgroups, n_kblocks;
   void* tc;              // tensor-core side data (tensor maps), owned; see gemm_tc.cu
+  const void* lut;           // caller-owned table [N][16] (G == -1), 16-bit floats of type sz_dtype
+  __nv_bfloat16* lut_bf16;   // owned: [Npad][16], RN_bf16 of the table, padding rows zero
 };
 
 namespace szo {

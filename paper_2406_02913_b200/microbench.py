@@ -76,13 +76,16 @@ def linear_case(M, N, K, G, mode, rho, reps, out_dtype=torch.bfloat16):
     idx = B.szo_select_mask(g * g, nnz)
     S = W.view(-1)[idx].contiguous()
     W.view(-1)[idx] = 0.0
-    plan_args = None
+    plan_args, lut = None, None
     if G > 0:
         codes, sc, ze = B.szo_quantize(W, G, "bf16")
         plan_args = (codes, sc, ze)
+    elif G < 0:    # non-uniform 4-bit format: random codes into per-row tables of 16 fp16 values
+        plan_args = (torch.from_numpy(wl.random_codes(N, K, seed=0, i=4)).cuda(), None, None)
+        lut = torch.from_numpy(wl.random_lut(N, seed=0, i=5)).cuda().to(torch.float16)
     else:
         plan_args = (W.to(torch.bfloat16), None, None)
-    plan = B.Linear(N, K, G, plan_args[0], plan_args[1], plan_args[2], "bf16", idx)
+    plan = B.Linear(N, K, G, plan_args[0], plan_args[1], plan_args[2], "bf16", idx, lut=lut)
     x = torch.from_numpy(wl.activation(M, K, seed=0, i=3)).cuda().to(torch.bfloat16)
     S_pert = torch.empty_like(S)
     B.szo_perturb(S, S_pert, idx, 0, 1234, 0, 1e-3)
@@ -91,7 +94,8 @@ def linear_case(M, N, K, G, mode, rho, reps, out_dtype=torch.bfloat16):
     med, best = time_call(lambda: plan.fwd(x, S_pert, md, out_dtype, y=y), reps)
     hbm, tf, src = peaks()
     flops = 2.0 * M * N * K
-    byts = (N * K / 2 + 4 * N * K / max(G, 1) if G > 0 else 2 * N * K) + 2 * M * K + y.element_size() * M * N + 8 * nnz
+    w_bytes = N * K / 2 + 4 * N * K / G if G > 0 else (N * K / 2 + 32 * N if G < 0 else 2 * N * K)
+    byts = w_bytes + 2 * M * K + y.element_size() * M * N + 8 * nnz
     t_roof = max(flops / (tf * 1e12), byts / (hbm * 1e9))
     line = {"case": "linear", "M": M, "N": N, "K": K, "G": G, "mode": mode, "nnz": nnz, "ms_median": med,
             "ms_min": best, "tflops": flops / (med * 1e-3) / 1e12, "gbs": byts / (med * 1e-3) / 1e9,
@@ -272,7 +276,7 @@ def main():
     ap.add_argument("--M", type=int, default=8192)
     ap.add_argument("--N", type=int, default=4096)
     ap.add_argument("--K", type=int, default=4096)
-    ap.add_argument("--G", type=int, default=128)
+    ap.add_argument("--G", type=int, default=128, help="group size; 0: dense bf16 weight; -1: non-uniform 4-bit (table) format")
     ap.add_argument("--rho", type=float, default=1e-3)
     ap.add_argument("--mode", default="sparse_add")
     ap.add_argument("--k", type=int, default=6_476_005)

@@ -142,6 +142,13 @@ def random_codes(N: int, K: int, seed: int = 0, i: int = 0) -> np.ndarray:
     return rng(seed, PURPOSE_CODES, i).integers(0, 256, (N, K // 2), dtype=np.uint8)
 
 
+def random_lut(N: int, seed: int = 0, i: int = 0, std: float = 0.02) -> np.ndarray:
+    """Per-row tables of the non-uniform 4-bit format, fp32 [N,16]: 16 ascending draws from
+    N(0, std) per row (the shape a sensitivity-weighted k-means over a Gaussian row produces:
+    dense near zero, sparse in the tails).  Input generator only; the caller rounds to fp16/bf16."""
+    return np.sort(rng(seed, PURPOSE_WEIGHTS, 900 + i).normal(0.0, std, (N, 16)), axis=1).astype(np.float32)
+
+
 # ------------------------------------------------------------------------------ large workloads
 # Full-size decoders (billions of parameters) are generated directly in device memory with a seeded
 # torch generator: quantizing 6.5 G fp32 weights on the host only to time a step would take

@@ -32,15 +32,22 @@ def _bf16_bits(t):
     # OPT-13B shapes, int4 G=128, 0.1 % mask, biases
     (5120, 5120, 128, 1e-3, True, "sparse_add"), (20480, 5120, 128, 1e-3, True, "sparse_add"),
     (5120, 20480, 128, 1e-3, True, "sparse_add"),
+    # non-uniform 4-bit format (G = -1 here: a per-row table of 16 fp16 values), Llama-2-7B MLP shapes
+    (11008, 4096, -1, 1e-3, False, "sparse_add"), (4096, 11008, -1, 1e-3, False, "sparse_add"),
 ])
 def test_full_size_linear_sampled_outputs(B, N, K, G, rho, bias, mode):
     M = 4096
     g = torch.Generator(device="cuda")
     g.manual_seed(N * 7 + K)
+    lut = None
     if G > 0:
         codes = torch.randint(0, 256, (N, K // 2), generator=g, device="cuda", dtype=torch.uint8)
         sc = (0.004 + 0.002 * torch.rand(N, K // G, generator=g, device="cuda")).to(torch.bfloat16)
         ze = (-7.5 * sc.float()).to(torch.bfloat16)
+    elif G < 0:
+        codes = torch.randint(0, 256, (N, K // 2), generator=g, device="cuda", dtype=torch.uint8)
+        lut = torch.sort(torch.randn(N, 16, generator=g, device="cuda") * 0.02, dim=1).values.to(torch.float16).contiguous()
+        sc = ze = None
     else:
         codes = (torch.randn(N, K, generator=g, device="cuda") * 0.02).to(torch.bfloat16)
         sc = ze = None
@@ -50,7 +57,7 @@ def test_full_size_linear_sampled_outputs(B, N, K, G, rho, bias, mode):
     S = (torch.randn(nnz, generator=g, device="cuda") * 0.02).contiguous()
     x = torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16)
     b = (torch.randn(N, generator=g, device="cuda") * 0.02) if bias else None
-    plan = B.Linear(N, K, G, codes, sc, ze, "bf16", idx, b)
+    plan = B.Linear(N, K, G, codes, sc, ze, "bf16", idx, b, lut=lut)
     md = B.MODE_SPARSE_ADD if mode == "sparse_add" else B.MODE_SPMM
     y = plan.fwd(x, S, md, torch.float32)
     torch.cuda.synchronize()
@@ -62,6 +69,8 @@ def test_full_size_linear_sampled_outputs(B, N, K, G, rho, bias, mode):
     toks = np.unique(np.concatenate([r.integers(0, M, 24), [0, 255, 256, M - 257, M - 1]]))
     if G > 0:
         deq = so.dequantize(codes[rows].cpu().numpy(), _bf16_bits(sc[rows]), _bf16_bits(ze[rows]), G, "bf16")   # [rows, K] fp64
+    elif G < 0:
+        deq = so.dequantize_lut(codes[rows].cpu().numpy(), lut[rows].cpu().view(torch.int16).numpy().view(np.uint16), "f16")
     else:
         deq = codes[rows].float().cpu().numpy().astype(np.float64)
     S_h = S.cpu().numpy().astype(np.float64)

@@ -221,3 +221,52 @@ def test_linear_argument_errors(B):
     y = plan.fwd(x[:0].to(torch.bfloat16), S, B.MODE_SPARSE_ADD, torch.float32)     # M = 0
     assert y.shape == (0, 64)
     plan.close()
+
+
+LUT_CASES = [
+    # N, K, fmt, M, rho, bias: non-uniform 4-bit format (codes into a per-row table of 16 values)
+    (256, 256, "f16", 256, 1e-3, False),
+    (384, 512, "bf16", 300, 1e-2, True),            # several tiles and a ragged tail in M and N
+    (200, 320, "f16", 65, 5e-3, False),             # N not a multiple of the tile: padded table rows
+    (512, 4096, "f16", 16, 1e-3, True),             # long K, few tokens: K-split tiles
+    (128, 64, "bf16", 1, 0.0, False),               # one token, one k-block, no sparse entries
+]
+
+
+def make_lut_case(N, K, fmt, M, rho, seed, bias):
+    codes = wl.random_codes(N, K, seed=seed, i=4)
+    lut_bits, _ = so.round_to_16(wl.random_lut(N, seed=seed, i=5), fmt)
+    deq = so.dequantize_lut(codes, lut_bits, fmt)
+    nnz = int(rho * N * K)
+    idx = wl.sorted_random_indices(N * K, nnz, seed=seed, i=6)
+    S0 = wl.rng(seed, wl.PURPOSE_WEIGHTS, 7).normal(0, 0.02, nnz).astype(np.float32)
+    S = so.perturb(S0, idx, 1234, 0, np.float32(1e-3)) if nnz else S0
+    x = wl.activation(M, K, seed=seed, i=3)
+    b = wl.rng(seed, wl.PURPOSE_WEIGHTS, 77).normal(0, 0.02, N).astype(np.float32) if bias else None
+    return dict(codes=codes, lut_bits=lut_bits, deq=deq, idx=idx, S=S, x=x, bias=b)
+
+
+@pytest.mark.parametrize("N,K,fmt,M,rho,bias", LUT_CASES)
+def test_lut_format_validation_and_tensor_core_modes(B, N, K, fmt, M, rho, bias):
+    c = make_lut_case(N, K, fmt, M, rho, seed=N + K + M + 1, bias=bias)
+    dt = torch.bfloat16 if fmt == "bf16" else torch.float16
+    lut = torch.from_numpy(c["lut_bits"].view(np.int16)).cuda().view(dt)
+    idx = torch.from_numpy(c["idx"]).cuda() if len(c["idx"]) else None
+    b = None if c["bias"] is None else torch.from_numpy(c["bias"]).cuda()
+    plan = B.Linear(N, K, 0, torch.from_numpy(c["codes"]).cuda(), None, None, fmt, idx, b, lut=lut)
+    x, S = torch.from_numpy(c["x"]).cuda(), torch.from_numpy(c["S"]).cuda()
+    ref = so.linear_fwd(c["x"], c["deq"], c["idx"], c["S"], c["bias"])
+    y = plan.fwd(x, S, B.MODE_FP32_VALIDATE, torch.float32).cpu().numpy()
+    assert max_rel(y, ref) < 4 * 2.0 ** -24 * np.sqrt(K)               # exact table values, fp32 accumulation
+    xb = x.to(torch.bfloat16)
+    for md in (B.MODE_SPARSE_ADD, B.MODE_AUTO):
+        yt = plan.fwd(xb, S, md, torch.float32).cpu().numpy()
+        assert max_rel(yt, ref) < LINEAR_TOL
+        assert max_rel(yt, ref) < 5e-3                                 # bf16 rounding of the table values only
+        assert np.array_equal(yt, plan.fwd(xb, S, md, torch.float32).cpu().numpy())
+    yb = plan.fwd(xb, S, B.MODE_SPARSE_ADD, torch.bfloat16).float().cpu().numpy()
+    assert max_rel(yb, ref) < LINEAR_TOL
+    with pytest.raises(B.SzoError):
+        plan.fwd(xb, S, B.MODE_SPMM, torch.float32)
+    assert B.device_status() == 0
+    plan.close()
