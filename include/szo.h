@@ -191,8 +191,9 @@ typedef struct {
   int32_t arch;
   int32_t n_layers, d_model, n_heads, n_kv_heads, d_ff, vocab, max_pos;
   float norm_eps, rope_base;
-  int32_t group;       /* int4 group size; 0 = dense bf16 linears */
-  int32_t sz_dtype;    /* szo_dtype of scales/zeros */
+  int32_t group;       /* int4 group size; 0 = dense bf16 linears; -1 = non-uniform 4-bit format
+                          (szo_linear_create_lut) */
+  int32_t sz_dtype;    /* szo_dtype of scales/zeros (of the tables when group == -1) */
   int32_t act_dtype;   /* SZO_BF16 (tensor-core path) or SZO_F32 (validation path) */
   int32_t linear_mode; /* szo_linear_mode used by every linear */
   int32_t loss_kind;   /* 0: mean next-token cross-entropy over B*(S-1) positions;
@@ -202,7 +203,7 @@ typedef struct {
 
 typedef struct {
   const void* codes;     /* uint8 [N,K/2], or bf16 [N,K] when group == 0 */
-  const void* scales;    /* sz_dtype [N,K/G] or NULL */
+  const void* scales;    /* sz_dtype [N,K/G] or NULL; when group == -1 the table [N,16] */
   const void* zeros;
   const int64_t* idx;    /* [nnz] ascending tensor-local flat indices */
   int64_t nnz;

@@ -300,7 +300,7 @@ class Model:
                 p = f"l{l}.{nm}."
                 idx = tensors.get(p + "idx")
                 lw.lin[j].codes = _ptr(tensors[p + "codes"])
-                lw.lin[j].scales = _ptr(tensors.get(p + "scales"))
+                lw.lin[j].scales = _ptr(tensors.get(p + ("lut" if shape["group"] == -1 else "scales")))
                 lw.lin[j].zeros = _ptr(tensors.get(p + "zeros"))
                 lw.lin[j].nnz = 0 if idx is None else idx.numel()
                 lw.lin[j].idx = _ptr(idx) if lw.lin[j].nnz else None

@@ -652,8 +652,12 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
       linear_shape(c, j, &N, &K);
       const szo_linear_weights& w = m->layers[l].lin[j];
       szo_linear_t* p = nullptr;
-      SZO_M_TRY(szo_linear_create(&p, N, K, c.group, w.codes, w.scales, w.zeros, static_cast<szo_dtype>(c.sz_dtype),
-                                  w.idx, w.nnz, w.bias, st));
+      if (c.group == -1)   // non-uniform 4-bit format: `scales` is the per-row table [N,16]
+        SZO_M_TRY(szo_linear_create_lut(&p, N, K, static_cast<const uint8_t*>(w.codes), w.scales,
+                                        static_cast<szo_dtype>(c.sz_dtype), w.idx, w.nnz, w.bias, st));
+      else
+        SZO_M_TRY(szo_linear_create(&p, N, K, c.group, w.codes, w.scales, w.zeros, static_cast<szo_dtype>(c.sz_dtype),
+                                    w.idx, w.nnz, w.bias, st));
       m->plans.push_back(p);
       m->offsets.push_back(m->offsets.back() + w.nnz);
       const size_t need = szo_linear_workspace_bytes(p, m->Mmax, c.linear_mode);

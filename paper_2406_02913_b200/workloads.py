@@ -42,6 +42,10 @@ MODEL_SHAPES = {
                      vocab=512, max_pos=0, group=0, sz_fmt="bf16", rho=1e-2),
     "tiny_opt": dict(arch="opt", n_layers=2, d_model=256, n_heads=4, n_kv_heads=4, d_ff=1024,
                      vocab=1024, max_pos=128, group=128, sz_fmt="bf16", rho=1e-3),
+    "tiny_lut": dict(arch="llama", n_layers=2, d_model=256, n_heads=4, n_kv_heads=4, d_ff=1024,
+                     vocab=1024, max_pos=0, group=-1, sz_fmt="f16", rho=1e-3),
+    "llama2_7b_lut": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, n_kv_heads=32,
+                          d_ff=11008, vocab=32000, max_pos=0, group=-1, sz_fmt="f16", rho=1e-3),
     "llama2_7b": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, n_kv_heads=32,
                       d_ff=11008, vocab=32000, max_pos=0, group=128, sz_fmt="bf16", rho=1e-3),
     "mistral_7b": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, n_kv_heads=8,
@@ -186,6 +190,9 @@ def device_decoder_tensors(shape: dict, seed: int = 0, device: str = "cuda"):
                 sc = (0.004 + 0.002 * torch.rand(N, K // G, generator=g, device=device)).to(sz_dt)
                 t[p + "scales"] = sc
                 t[p + "zeros"] = (-7.5 * sc.float()).to(sz_dt)
+            elif G < 0:     # non-uniform 4-bit format: uniform codes into 16 ascending N(0, 0.02) draws per row
+                t[p + "codes"] = torch.randint(0, 256, (N, K // 2), generator=g, device=device, dtype=torch.uint8)
+                t[p + "lut"] = torch.sort(randn(N, 16) * 0.02, dim=1).values.to(sz_dt).contiguous()
             else:
                 t[p + "codes"] = (randn(N, K) * 0.02).to(torch.bfloat16)
             k = int(shape["rho"] * N * K)

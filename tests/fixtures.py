@@ -15,6 +15,17 @@ def decoder_config(shape: dict) -> mo.DecoderConfig:
                             vocab=shape["vocab"], max_pos=shape["max_pos"])
 
 
+def table_coded(Wd: np.ndarray, fmt: str):
+    """A stand-in for a non-uniform 4-bit quantizer (fitting the tables is outside the library): per
+    row the 16 values are the (i + 1/2)/16 quantiles of the row, rounded to `fmt`; each weight takes
+    the code of its nearest value.  Returns (packed codes uint8 [N,K/2], table bits uint16 [N,16])."""
+    q = (np.arange(16) + 0.5) / 16.0
+    lut = np.quantile(Wd.astype(np.float64), q, axis=1).T.astype(np.float32)           # [N,16], ascending
+    lb, lv = so.round_to_16(lut, fmt)
+    code = np.argmin(np.abs(Wd[:, :, None].astype(np.float64) - lv[:, None, :].astype(np.float64)), axis=2).astype(np.uint8)
+    return (code[:, 0::2] | (code[:, 1::2] << 4)).astype(np.uint8), lb
+
+
 class DecoderFixture:
     """Weights -> mask (top-k of accumulated squared gradients, or a random sample) -> decompose ->
     quantize, all with the oracle; keeps every intermediate for comparison."""
@@ -55,6 +66,10 @@ class DecoderFixture:
                     codes, sb, zb = so.quantize_int4(Wd, G, fmt)
                     dq = so.dequantize(codes, sb, zb, G, fmt)
                     ql[nm] = (codes, sb, zb)
+                elif G < 0:
+                    codes, lb = table_coded(Wd, fmt)
+                    dq = so.dequantize_lut(codes, lb, fmt)
+                    ql[nm] = (codes, lb, None)
                 else:
                     Wd = wl.bf16_round(Wd)
                     dq = Wd.astype(np.float64)
@@ -101,7 +116,11 @@ class DecoderFixture:
                     t[f"l{l}.{nm}_b"] = up(self.params[f"l{l}.{nm}_b"])
             for nm in self.names:
                 p = f"l{l}.{nm}."
-                if G > 0:
+                if G < 0:
+                    codes, lb, _ = self.q[l][nm]
+                    dt = torch.bfloat16 if fmt == "bf16" else torch.float16
+                    t[p + "codes"], t[p + "lut"] = up(codes), up(lb.view(np.int16)).view(dt)
+                elif G > 0:
                     if quantize_on_gpu is not None:
                         codes, sc, ze = quantize_on_gpu(up(self.W_dense[l][nm]), G, fmt)
                     else:

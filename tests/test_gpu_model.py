@@ -101,7 +101,7 @@ def test_ten_zo_steps_fp32_validation(B, tiny):
     m.close()
 
 
-@pytest.mark.parametrize("name,loss_kind", [("tiny_opt", 0), ("tiny_gqa", 1)])
+@pytest.mark.parametrize("name,loss_kind", [("tiny_opt", 0), ("tiny_gqa", 1), ("tiny_lut", 0)])
 def test_other_architectures_fp32_validation(B, name, loss_kind):
     fx = DecoderFixture(name, seed=1, mask="random", B=3, S=32)
     m, S, _ = build_gpu(B, fx, B.SZO_F32, B.MODE_FP32_VALIDATE, loss_kind, quantize_on_gpu=fx.shape["group"] > 0)
@@ -177,10 +177,11 @@ def test_attention_matches_oracle(B, B_, S, H, Hkv, hd, dtype):
 
 
 @pytest.mark.parametrize("name,loss_kind,mode", [("tiny_opt", 0, "sparse_add"), ("tiny_gqa", 1, "sparse_add"),
-                                                 ("tiny_gqa", 0, "spmm")])
+                                                 ("tiny_gqa", 0, "spmm"), ("tiny_lut", 0, "sparse_add")])
 def test_other_architectures_bf16_tensor_core_path(B, name, loss_kind, mode):
     """OPT-shaped (LayerNorm, biases, ReLU, learned positions, int4) and Mistral-shaped (GQA, dense bf16
-    weights, 1 % mask) decoders on the tensor-core path: losses within 1e-3 of the oracle."""
+    weights, 1 % mask) decoders, and the tiny decoder in the non-uniform 4-bit format, on the
+    tensor-core path: losses within 1e-3 of the oracle."""
     fx = DecoderFixture(name, seed=2, mask="random", B=3, S=48)
     md = B.MODE_SPARSE_ADD if mode == "sparse_add" else B.MODE_SPMM
     m, S, _ = build_gpu(B, fx, B.SZO_BF16, md, loss_kind, quantize_on_gpu=fx.shape["group"] > 0)
