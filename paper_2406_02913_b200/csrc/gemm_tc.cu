@@ -324,14 +324,16 @@ int materialise_override() {
 
 }  // namespace
 
-bool tc_use_materialised(const szo_linear* p, int64_t M) {
+bool tc_use_materialised(const szo_linear* p, int64_t M, bool two_sets) {
   if (p->G == 0 || p->tc == nullptr) return false;
   if (p->G < 0) return true;      // table-coded weights have this form only
   const int o = materialise_override();
   if (o >= 0) return o == 1;
   // the extra pass costs about 2.5 N K bytes of traffic, the fused conversion 5-10 % of 2 M N K flop at
-  // the kernel's rate: measured break-even near M = 2048 (4096^2: 73 vs 75 us), 7 % ahead at M = 4096
-  return M >= 4096;
+  // the kernel's rate: measured break-even near M = 2048 (4096^2: 73 vs 75 us), 7 % ahead at M = 4096.
+  // When one weight pass serves the two perturbed forwards of a step, the break-even halves
+  // (Llama-2-7B-shaped step: 54.2 vs 57.5 ms at 2048 tokens, 31.3 vs 31.6 at 1024, 21.1 vs 20.8 at 512).
+  return M >= (two_sets ? 2048 : 4096);
 }
 
 size_t tc_materialised_ws_bytes(const szo_linear* const* plans, int n, int64_t M) {
@@ -349,11 +351,12 @@ size_t tc_materialised_ws_bytes(const szo_linear* const* plans, int n, int64_t M
 // rewrites the masked entries (RN_bf16(frozen + S), the SparseAdd of the appendix on sparse
 // operations) and runs the dense mode of the kernel; no entry needs restoring afterwards, because the
 // next scatter writes every masked position again from the saved frozen value.
-bool tc_use_resident(const szo_linear* p, int64_t M) {
+// Measured on the Mistral-7B shape (1 % mask) it is ahead of the fused form at every token count tried
+// (step at 4096 / 2048 / 1024 / 512 tokens: 115 / 60 / 35 / 23 ms against 132 / 72 / 42 / 31), so it is
+// taken for every M; SZO_LINEAR_MATERIALISE=0 switches it off.
+bool tc_use_resident(const szo_linear* p, int64_t) {
   if (p->G != 0 || p->tc == nullptr) return false;
-  const int o = materialise_override();
-  if (o >= 0) return o == 1;
-  return M >= 4096;
+  return materialise_override() != 0;
 }
 
 bool tc_can_stack(const szo_linear* const* plans, int n) {

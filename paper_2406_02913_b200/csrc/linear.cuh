@@ -66,7 +66,7 @@ size_t tc_tail_ws_bytes(const szo_linear* const* plans, int n, int64_t M);
 size_t tc_tail_ws_bound();   // enough for any M and any group
 // Materialised form (gemm_tc.cu): the effective bf16 weight is written to scratch, then the dense
 // mode of the kernel runs.  Chosen for int4 plans when M is large (tc_use_materialised).
-bool tc_use_materialised(const szo_linear* p, int64_t M);
+bool tc_use_materialised(const szo_linear* p, int64_t M, bool two_sets = false);   // two_sets: one weight pass for two forwards
 size_t tc_materialised_ws_bytes(const szo_linear* const* plans, int n, int64_t M);
 szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, const void* x, int64_t M,
                                       const float* const* S_pert, void* const* y, int y_dtype, void* ws,

@@ -586,7 +586,7 @@ szo_status run_loss(szo_model* m, const int32_t* tokens, const int32_t* labels, 
 bool dual_forward_applies(const szo_model* m, int64_t M) {
   return m->dual_rows && m->cfg.act_dtype != SZO_F32 && m->cfg.linear_mode != SZO_MODE_FP32_VALIDATE &&
          m->cfg.linear_mode != SZO_MODE_SPMM && !m->plans.empty() && m->k_total > 0 &&
-         (m->resident || tc_use_materialised(m->plans[0], M));
+         (m->resident || tc_use_materialised(m->plans[0], M, true));
 }
 
 szo_status check_batch(const szo_model* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand, int B,
@@ -669,7 +669,7 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
     const size_t need = tc_tail_ws_bound();
     if (need > ws_need) ws_need = need;
     // scratch of the materialised form: the largest group of layers that share their input
-    if (tc_use_materialised(m->plans[0], m->Mmax)) {
+    if (tc_use_materialised(m->plans[0], m->Mmax, true)) {
       for (int l = 0; l < c.n_layers; ++l) {
         const szo_linear* const* pl = m->plans.data() + static_cast<size_t>(l) * m->n_lin;
         const size_t g0 = tc_materialised_ws_bytes(pl, 3, m->Mmax);                       // q, k, v
@@ -687,8 +687,11 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
   m->k_total = m->offsets.back();
   if (m->k_total > 0 && S_all == nullptr) return bail(fail(SZO_ERR_INVALID_ARG, "S_all is NULL"));
   // resident effective weights of the launch groups (dense bf16 weights, many tokens)
-  m->resident = c.group == 0 && c.act_dtype == SZO_BF16 && c.linear_mode != SZO_MODE_FP32_VALIDATE &&
-                c.linear_mode != SZO_MODE_SPMM && !m->plans.empty() && tc_use_resident(m->plans[0], m->Mmax);
+  // (SZO_MODEL_RESIDENT=0 at creation keeps the fused form, for A/B and for tests that compare the two)
+  const char* res_env = getenv("SZO_MODEL_RESIDENT");
+  m->resident = !(res_env != nullptr && res_env[0] == '0') && c.group == 0 && c.act_dtype == SZO_BF16 &&
+                c.linear_mode != SZO_MODE_FP32_VALIDATE && c.linear_mode != SZO_MODE_SPMM && !m->plans.empty() &&
+                tc_use_resident(m->plans[0], m->Mmax);
   if (m->resident) {
     m->res_W.assign(m->plans.size(), nullptr);
     m->res_saved.assign(m->plans.size(), nullptr);
@@ -723,7 +726,7 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
     const char* env = getenv("SZO_DUAL_FORWARD");
     m->dual_rows = !(env != nullptr && env[0] == '0') && c.act_dtype != SZO_F32 &&
                    c.linear_mode != SZO_MODE_FP32_VALIDATE && c.linear_mode != SZO_MODE_SPMM && !m->plans.empty() &&
-                   m->k_total > 0 && (m->resident || tc_use_materialised(m->plans[0], m->Mmax));
+                   m->k_total > 0 && (m->resident || tc_use_materialised(m->plans[0], m->Mmax, true));
   }
   const int64_t Mx = m->Mmax * (m->dual_rows ? 2 : 1), d = c.d_model, dkv = static_cast<int64_t>(c.n_kv_heads) * hd,
                 ff = c.d_ff;

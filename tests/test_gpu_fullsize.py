@@ -233,10 +233,10 @@ def test_two_full_width_layers_in_the_bench_configuration(B):
 
 def test_two_mistral_width_layers_resident_form(B):
     """Two decoder layers at the Mistral-7B width (GQA 32/8, d_ff 14336, dense bf16 weights, 1 % mask)
-    with 8 x 512 tokens and the full-sequence loss.  At this token count the model keeps the effective
+    with 8 x 512 tokens and the full-sequence loss.  With dense bf16 weights the model keeps the effective
     weight of every launch group resident and runs the two forwards of a step side by side.  Checked:
     the loss against the library's fp32 validation path (pinned to the oracle by the small tests),
-    against the fused form of the same weights (a model created for fewer tokens), repeatability bit
+    against the fused form of the same weights (a model created with SZO_MODEL_RESIDENT=0), repeatability bit
     for bit, and that a second step starts from clean weights (no masked entry keeps an old value)."""
     shape = dict(wl.MODEL_SHAPES["mistral_7b"], n_layers=2)
     tensors, S_all = wl.device_decoder_tensors(shape, seed=5)
@@ -246,8 +246,13 @@ def test_two_mistral_width_layers_resident_form(B):
     S_res, S_fused, S_ref = S_all.clone(), S_all.clone(), S_all.clone()
     m_res = B.Model(shape, names, tensors, S_res, act_dtype=B.SZO_BF16, linear_mode=B.MODE_SPARSE_ADD,
                     loss_kind=B.LOSS_LM, max_batch=Bn, max_seq=S)
-    m_fused = B.Model(shape, names, tensors, S_fused, act_dtype=B.SZO_BF16, linear_mode=B.MODE_SPARSE_ADD,
-                      loss_kind=B.LOSS_LM, max_batch=Bn - 1, max_seq=S)          # 3584 tokens: fused form
+    import os
+    os.environ["SZO_MODEL_RESIDENT"] = "0"                                       # read at creation: fused form
+    try:
+        m_fused = B.Model(shape, names, tensors, S_fused, act_dtype=B.SZO_BF16, linear_mode=B.MODE_SPARSE_ADD,
+                          loss_kind=B.LOSS_LM, max_batch=Bn - 1, max_seq=S)
+    finally:
+        del os.environ["SZO_MODEL_RESIDENT"]
     m_ref = B.Model(shape, names, tensors, S_ref, act_dtype=B.SZO_F32, linear_mode=B.MODE_FP32_VALIDATE,
                     loss_kind=B.LOSS_LM, max_batch=Bn, max_seq=S)
     f_res = float(m_res.loss(toks).item())
