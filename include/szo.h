@@ -233,7 +233,10 @@ szo_status szo_attention(const void* q, const void* k, const void* v, void* o, s
 typedef struct szo_model szo_model_t;
 /* layers_host: host array of n_layers entries holding device pointers.  S_all: fp32 [k_total],
  * the trainable sparse values of all linears concatenated in model order (the only mutable
- * state; caller-owned, updated in place by szo_model_zo_step).  Synchronises the stream. */
+ * state; caller-owned, updated in place by szo_model_zo_step).  Synchronises the stream.
+ * The weights are frozen by the method (Section 3.4: only w_sparse is trained) and must not change
+ * after this call: with dense bf16 linears (group == 0) the model keeps its own copy of them
+ * (2 bytes per weight more device memory), in which it rewrites the masked entries per forward. */
 szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg,
                             const szo_model_weights* top, const szo_layer_weights* layers_host,
                             float* S_all, void* stream);
