@@ -221,7 +221,7 @@ def attention_case(Bn, S, H, Hkv, hd, reps):
                       "tflops_causal": flops / (med * 1e-3) / 1e12}), flush=True)
 
 
-def step_case(name, Bn, S, loss, steps, eps, lr):
+def step_case(name, Bn, S, loss, steps, eps, lr, profile_range=False):
     """A full ZO step of a whole decoder shape (random-init weights in device memory), timed like
     bench.py: CUDA events around `steps` back-to-back steps after three warm-up steps; the weights
     streamed per forward exceed L2."""
@@ -239,11 +239,15 @@ def step_case(name, Bn, S, loss, steps, eps, lr):
     torch.cuda.synchronize()
     model.enable_timing(True)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if profile_range:       # for ncu --profile-from-start off: exactly the timed steps are listed
+        torch.cuda.profiler.start()
     e0.record()
     for i in range(3, n):
         model.zo_step(toks[i], 1234, i, eps, lr, labs[i], cand)
     e1.record()
     torch.cuda.synchronize()
+    if profile_range:
+        torch.cuda.profiler.stop()
     ms = e0.elapsed_time(e1) / steps
     lin_ms, lin_launches = model.linear_time()
     model.enable_timing(False)
@@ -273,6 +277,8 @@ def main():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--eps", type=float, default=1e-3)
     ap.add_argument("--lr", type=float, default=1e-6)
+    ap.add_argument("--profile-range", action="store_true",
+                    help="step: bracket the timed steps with cudaProfilerStart/Stop")
     ap.add_argument("--M", type=int, default=8192)
     ap.add_argument("--N", type=int, default=4096)
     ap.add_argument("--K", type=int, default=4096)
@@ -290,7 +296,7 @@ def main():
     elif a.what == "sparse":
         sparse_case(a.k, a.reps)
     elif a.what == "step":
-        step_case(a.model, a.batch, a.seq, a.loss, a.steps, a.eps, a.lr)
+        step_case(a.model, a.batch, a.seq, a.loss, a.steps, a.eps, a.lr, a.profile_range)
     elif a.what == "attention":
         attention_case(16, 256, 32, 32, 128, a.reps)
         attention_case(8, 512, 32, 8, 128, a.reps)
