@@ -415,7 +415,7 @@ szo_status tc_resident_init(const szo_linear* const* plans, int n, __nv_bfloat16
 szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, const void* x, int64_t M,
                                       const float* const* S_pert, void* const* y, int y_dtype, void* ws,
                                       size_t ws_bytes, cudaStream_t st, const float* const* S_second,
-                                      __nv_bfloat16* W_resident, __nv_bfloat16* saved_resident) {
+                                      __nv_bfloat16* W_resident, __nv_bfloat16* saved_resident, bool relu) {
   const szo_linear* p0 = plans[0];
   const bool resident = W_resident != nullptr;
   const TcPlan* t = static_cast<const TcPlan*>(p0->tc);
@@ -463,6 +463,7 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
   SZO_TRY(make_map(&mw, W, rows, p0->K, kBM));
   TcParams P{};
   P.M = M; P.K = p0->K; P.G = 0; P.nkb = nkb;
+  P.relu = relu ? 1 : 0;
   P.m_tiles = ceil_div(M, 256);
   P.nsub = n;
   int64_t n_tiles = 0;

@@ -148,7 +148,7 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& P, int pair, int n_p
 // part finished last.  Thread -> one float4 (4 rows of one token) per step of nthreads, seven in
 // flight per part.  Kept out of line: its registers would otherwise add to every role's.
 __device__ __noinline__ void reduce_parts(const float* part0, int parts, int64_t n0, int64_t N, const float* bias_p,
-                                          void* y, int y_f32, int64_t m0, int mlimit, int tid, int nthreads) {
+                                          void* y, int y_f32, int relu, int64_t m0, int mlimit, int tid, int nthreads) {
   constexpr int64_t kPartFloats = static_cast<int64_t>(kPairBT) * kBM;
   constexpr int kBatch = 7;
   const int total = mlimit * (kBM / 4);          // float4s of the valid tokens
@@ -187,6 +187,10 @@ __device__ __noinline__ void reduce_parts(const float* part0, int parts, int64_t
 #pragma unroll
         for (int e = 0; e < 4; ++e)
           if (n4 + e < N) o[e] += __ldg(bias_p + n4 + e);
+      }
+      if (relu) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) o[e] = fmaxf(o[e], 0.f);
       }
       const bool vec_ok = (N % 4 == 0) && (n4 + 3 < N);
       const int64_t off = (m0 + mm) * N + n4;
@@ -593,6 +597,8 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
       const int64_t m0 = static_cast<int64_t>(u.m_tile) * kPairBT;
       const int mlimit = static_cast<int>((P.M - m0 < kPairBT) ? P.M - m0 : kPairBT);
       // y[m0 + c0 + j, n] = v[j] + bias for the valid tokens of a 32-token chunk
+      const bool relu = P.relu != 0;
+      auto act = [&](float t) { return relu ? fmaxf(t, 0.f) : t; };
       auto store_chunk = [&](int c0, const uint32_t (&v)[32]) {
         if (n < N && c0 < mlimit) {
           const int cnt = mlimit - c0;
@@ -600,14 +606,14 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             float* yp = static_cast<float*>(y) + (m0 + c0) * N + n;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-              if (j < cnt) *yp = __uint_as_float(v[j]) + bias;
+              if (j < cnt) *yp = act(__uint_as_float(v[j]) + bias);
               yp += N;
             }
           } else {
             __nv_bfloat16* yp = static_cast<__nv_bfloat16*>(y) + (m0 + c0) * N + n;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-              if (j < cnt) *yp = __float2bfloat16_rn(__uint_as_float(v[j]) + bias);
+              if (j < cnt) *yp = __float2bfloat16_rn(act(__uint_as_float(v[j]) + bias));
               yp += N;
             }
           }
@@ -668,7 +674,7 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     const int mlimit = static_cast<int>((P.M - m0 < kPairBT) ? P.M - m0 : kPairBT);
     reduce_parts(P.partial + (static_cast<int64_t>(u.slot * u.parts) * 2 + rank) * kPartFloats, u.parts,
                  static_cast<int64_t>(u.n_tile) * kBM, SZO_SUB(P, u.s, N), SZO_SUB(P, u.s, bias), SZO_SUB(P, u.s, y), P.y_f32,
-                 m0, mlimit, static_cast<int>(threadIdx.x), kNumWarps2 * 32);
+                 P.relu, m0, mlimit, static_cast<int>(threadIdx.x), kNumWarps2 * 32);
   }
   cluster_sync_all();          // no CTA leaves while its peer may still signal it or read its tiles
   tc_fence_after();

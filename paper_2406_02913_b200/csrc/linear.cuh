@@ -71,7 +71,8 @@ size_t tc_materialised_ws_bytes(const szo_linear* const* plans, int n, int64_t M
 szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, const void* x, int64_t M,
                                       const float* const* S_pert, void* const* y, int y_dtype, void* ws,
                                       size_t ws_bytes, cudaStream_t st, const float* const* S_second = nullptr,
-                                      __nv_bfloat16* W_resident = nullptr, __nv_bfloat16* saved_resident = nullptr);
+                                      __nv_bfloat16* W_resident = nullptr, __nv_bfloat16* saved_resident = nullptr,
+                                      bool relu = false);   // relu: y = max(y, 0) applied in the epilogue
 // Resident form for dense bf16 plans (G == 0): W_resident [sum Npad, K] and saved_resident [sum nnz]
 // are filled once by tc_resident_init and passed to linear_fwd_tc_materialised, which then skips the
 // weight pass and writes every masked entry as RN_bf16(saved + S); ws is only the K-split scratch.

@@ -449,7 +449,9 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
     return rc;
   };
   // layers j0 .. j0 + n - 1 read the same x: one fused launch when the tensor-core path allows it
-  auto lin_group = [&](int layer, int j0, int n, const void* x, void* const* outs) -> szo_status {
+  // relu_applied (n == 1 only): asks for y = max(y, 0); set when the launch applied it in its epilogue
+  auto lin_group = [&](int layer, int j0, int n, const void* x, void* const* outs,
+                       bool* relu_applied = nullptr) -> szo_status {
     const int t0 = layer * m->n_lin + j0;
     const szo_linear* plans[3];
     const uint2* recs[3];
@@ -480,8 +482,9 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
     }
     const szo_status rc = mat ? linear_fwd_tc_materialised(plans, n, x, M, spert, outs, act, m->ws, m->ws_bytes, st,
                                                            nsets == 2 ? spert2 : nullptr, res ? m->res_W[t0] : nullptr,
-                                                           res ? m->res_saved[t0] : nullptr)
+                                                           res ? m->res_saved[t0] : nullptr, relu_applied != nullptr)
                               : linear_fwd_tc_group(plans, n, x, M, recs, outs, act, m->ws, m->ws_bytes, st);
+    if (mat && relu_applied != nullptr) *relu_applied = true;
     if (m->timing) {
       SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used + 1], st));
       m->events_used += 2;
@@ -536,9 +539,15 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
       count_launch();
       SZO_TRY(lin(l, 6, gate, y));
     } else {
-      SZO_TRY(lin(l, 4, a, gate));
-      relu_kernel<T><<<blocks_for(Mr * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, Mr * ff);
-      count_launch();
+      bool relu_applied = false;
+      {
+        void* const fc1_out[1] = {gate};
+        SZO_TRY(lin_group(l, 4, 1, a, fc1_out, &relu_applied));
+      }
+      if (!relu_applied) {
+        relu_kernel<T><<<blocks_for(Mr * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, Mr * ff);
+        count_launch();
+      }
       SZO_TRY(lin(l, 5, gate, y));
     }
     pending = y;                  // added by the next norm (next layer's, or the final one)

@@ -38,6 +38,7 @@ struct TcParams {
   int nkb;                 // K / 64
   int64_t m_tiles, n_tiles;   // 256-token tiles; 256-row pair tiles of all matrices together
   int y_f32;
+  int relu;                // y = max(y, 0) in the epilogue (the ReLU of an OPT-style MLP after its first matrix)
   int32_t* status;
   int nsub;
   TcSub sub[3];

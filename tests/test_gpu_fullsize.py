@@ -286,3 +286,47 @@ def test_two_mistral_width_layers_resident_form(B):
     assert not torch.equal(S_res, S0)                              # the update moved S
     for m in (m_res, m_fused, m_ref):
         m.close()
+
+
+def test_two_opt_width_layers_relu_in_the_epilogue(B):
+    """Two decoder layers at the OPT-13B width (LayerNorm, biases, learned positions, ReLU MLP of width
+    20480, int4 group-128, 0.1 % mask) with 8 x 512 tokens and the full-sequence loss.  The step runs
+    its two forwards side by side and applies the ReLU in the epilogue of the first MLP matrix (tiles
+    of its last round are split along K, so the sum of the parts applies it too); the sequential form
+    runs the ReLU as a kernel of its own.  Both must agree (to the order of the LM head's fp32 sums);
+    the loss is also checked against the library's fp32 validation path."""
+    import os
+    shape = dict(wl.MODEL_SHAPES["opt_13b"], n_layers=2)
+    tensors, S_all = wl.device_decoder_tensors(shape, seed=7)
+    names = wl.linear_names(shape)
+    Bn, S = 8, 512
+    toks = torch.from_numpy(wl.token_batch(shape["vocab"], Bn, S, 7, wl.PURPOSE_TRAIN_BATCH, 0)).cuda()
+    S_dual, S_seq, S_ref = S_all.clone(), S_all.clone(), S_all.clone()
+    m_dual = B.Model(shape, names, tensors, S_dual, act_dtype=B.SZO_BF16, linear_mode=B.MODE_SPARSE_ADD,
+                     loss_kind=B.LOSS_LM, max_batch=Bn, max_seq=S)
+    os.environ["SZO_DUAL_FORWARD"] = "0"
+    try:
+        m_seq = B.Model(shape, names, tensors, S_seq, act_dtype=B.SZO_BF16, linear_mode=B.MODE_SPARSE_ADD,
+                        loss_kind=B.LOSS_LM, max_batch=Bn, max_seq=S)
+    finally:
+        del os.environ["SZO_DUAL_FORWARD"]
+    m_ref = B.Model(shape, names, tensors, S_ref, act_dtype=B.SZO_F32, linear_mode=B.MODE_FP32_VALIDATE,
+                    loss_kind=B.LOSS_LM, max_batch=Bn, max_seq=S)
+    f_ref = float(m_ref.loss(toks).item())
+    f_seq = float(m_seq.loss(toks).item())
+    assert np.isfinite(f_ref) and abs(f_seq - f_ref) <= 1e-3 * abs(f_ref)
+    out_dual = m_dual.zo_step(toks, 99, 3, 1e-3, 1e-6).clone()
+    out_seq = m_seq.zo_step(toks, 99, 3, 1e-3, 1e-6).clone()
+    torch.cuda.synchronize()
+    assert B.device_status() == 0
+    assert m_dual.last_launches() < m_seq.last_launches()
+    # everything up to the last norm has the same bits in both forms; the LM head runs over 8192 rows
+    # in one form and twice over 4096 in the other, so other tiles of it are split along K and their
+    # fp32 sums run in another order: the losses agree to ~1e-9, not bit for bit
+    for i in (0, 1):
+        assert abs(float(out_dual[i]) - float(out_seq[i])) <= 1e-7 * abs(float(out_seq[i]))
+    assert float((S_dual - S_seq).abs().max()) <= 4e-9            # at most an fp32 ulp of values ~0.02
+    fp, fm = float(out_dual[0]), float(out_dual[1])
+    assert abs(0.5 * (fp + fm) - f_seq) <= 1e-3 * abs(f_seq)
+    for m in (m_dual, m_seq, m_ref):
+        m.close()
