@@ -61,9 +61,61 @@ quantize_kernel(const WT* __restrict__ W, int64_t N, int64_t K, int G, uint8_t* 
   }
 }
 
+// G in {32, 64, 128} with fp32 weights: a warp takes 128 consecutive elements of a row (one 16-byte
+// load per lane, kept in registers for the second step), i.e. 128 / G groups of G / 4 lanes each; the
+// min/max shuffles stay inside a group's lanes, a lane writes its four codes as one 16-bit store.
+// Same arithmetic, instruction by instruction, as the general kernel: the same bits.
+template <typename SZ>
+__global__ void __launch_bounds__(256)
+quantize_f32_vec_kernel(const float* __restrict__ W, int64_t N, int64_t K, int G, uint8_t* __restrict__ codes,
+                        SZ* __restrict__ scales, SZ* __restrict__ zeros) {
+  const int lane = threadIdx.x & 31;
+  const int lanes_per_group = G >> 2;
+  const int64_t chunks = N * K / 128;          // K % G == 0 and G | 128, K % 128 == 0 (checked by the caller)
+  const int64_t warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
+  for (int64_t ch = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5; ch < chunks; ch += warps) {
+    const int64_t e0 = ch * 128 + lane * 4;    // flat element index of this lane's first weight
+    const float4 w4 = *reinterpret_cast<const float4*>(W + e0);
+    const float w[4] = {w4.x, w4.y, w4.z, w4.w};
+    float mn = fminf(fminf(w[0], w[1]), fminf(w[2], w[3]));
+    float mx = fmaxf(fmaxf(w[0], w[1]), fmaxf(w[2], w[3]));
+    for (int o = lanes_per_group >> 1; o; o >>= 1) {
+      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    }
+    const SZ s16 = round16<SZ>(__fdiv_rn(__fsub_rn(mx, mn), 15.0f));
+    const SZ z16 = round16<SZ>(mn);
+    const float s = widen(s16), z0 = widen(z16);
+    if ((lane & (lanes_per_group - 1)) == 0) {
+      const int64_t g = e0 / G;                // groups are numbered row-major, like the elements
+      scales[g] = s16;
+      zeros[g] = z16;
+    }
+    uint32_t packed = 0;
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      float r = (s == 0.0f) ? 0.0f : rintf(__fdiv_rn(__fsub_rn(w[t], z0), s));
+      r = fminf(fmaxf(r, 0.0f), 15.0f);
+      packed |= static_cast<uint32_t>(static_cast<int>(r)) << (4 * t);
+    }
+    *reinterpret_cast<uint16_t*>(codes + (e0 >> 1)) = static_cast<uint16_t>(packed);
+  }
+}
+
 template <typename WT, typename SZ>
 szo_status launch_quantize(const void* W, int64_t N, int64_t K, int G, uint8_t* codes, void* scales,
                            void* zeros, cudaStream_t st) {
+  if constexpr (sizeof(WT) == 4) {
+    if ((G == 32 || G == 64 || G == 128) && K % 128 == 0) {
+      int64_t blocks = ceil_div(N * K / 128, 8);
+      if (blocks > 148 * 32) blocks = 148 * 32;
+      quantize_f32_vec_kernel<SZ><<<static_cast<unsigned>(blocks), 256, 0, st>>>(
+          static_cast<const float*>(W), N, K, G, codes, static_cast<SZ*>(scales), static_cast<SZ*>(zeros));
+      count_launch();
+      SZO_CHECK_LAUNCH("quantize_f32_vec_kernel");
+      return SZO_OK;
+    }
+  }
   const int64_t total_warps = N * (K / G);
   int64_t blocks = ceil_div(total_warps, 8);
   if (blocks > 148 * 16) blocks = 148 * 16;

@@ -134,7 +134,8 @@ def test_perturb_empty_and_bad_arguments(B):
 
 
 @pytest.mark.parametrize("N,K,G,fmt,wdt", [(64, 256, 64, "f16", torch.float32), (96, 4096, 128, "bf16", torch.float32),
-                                           (33, 320, 32, "bf16", torch.float32), (16, 512, 128, "bf16", torch.bfloat16)])
+                                           (33, 320, 32, "bf16", torch.float32), (16, 512, 128, "bf16", torch.bfloat16),
+                                           (40, 384, 32, "f16", torch.float32), (8, 512, 256, "bf16", torch.float32)])
 def test_quantize_bit_exact(B, N, K, G, fmt, wdt):
     W = wl.gaussian_matrix(N, K, 0.02, seed=7, i=N)
     if wdt == torch.bfloat16:
