@@ -307,9 +307,13 @@ __global__ void scatter_add_bf16_kernel(const MatArgs a) {
   const float* S = s == 0 ? a.sub[0].S : (s == 1 ? a.sub[1].S : a.sub[2].S);
   __nv_bfloat16* saved = s == 0 ? a.sub[0].saved : (s == 1 ? a.sub[1].saved : a.sub[2].saved);
   __nv_bfloat16* el = (s == 0 ? a.sub[0].out : (s == 1 ? a.sub[1].out : a.sub[2].out)) + idx[e];
-  __nv_bfloat16 base = *el;
-  if (a.scatter_mode == 1) saved[e] = base;
-  if (a.scatter_mode == 2) base = saved[e];
+  __nv_bfloat16 base;
+  if (a.scatter_mode == 2) {
+    base = saved[e];              // the element itself is not read: it holds the other set's value
+  } else {
+    base = *el;
+    if (a.scatter_mode == 1) saved[e] = base;
+  }
   *el = __float2bfloat16_rn(__bfloat162float(base) + S[e]);
 }
 
