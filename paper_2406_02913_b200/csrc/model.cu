@@ -260,6 +260,9 @@ __global__ void residual_add_kernel(float* __restrict__ h, const T* __restrict__
 }
 
 // Next-token cross-entropy of row m (position s < S-1 predicts tok[m+1]); 0 for the last position.
+// One pass over the row: every thread keeps a running maximum and the sum of exp(x - maximum) of its
+// elements (16-byte loads when the row allows it), the block then brings the partial sums to the
+// common maximum.
 __global__ void __launch_bounds__(256)
 ce_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__ tok, int S, int V,
                double* __restrict__ tok_loss) {
@@ -270,21 +273,39 @@ ce_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__ tok
     return;
   }
   const float* row = logits + m * V;
-  float mx = -INFINITY;
-  for (int c = threadIdx.x; c < V; c += blockDim.x) mx = fmaxf(mx, row[c]);
+  float mx = -INFINITY, s = 0.f;
+  auto fold = [&](float cmax, float csum_at_cmax) {      // merge a chunk given at its own maximum
+    if (cmax > mx) {
+      s = s * __expf(mx - cmax) + csum_at_cmax;
+      mx = cmax;
+    } else {
+      s += csum_at_cmax * __expf(cmax - mx);
+    }
+  };
+  if ((V & 3) == 0) {
+    const float4* row4 = reinterpret_cast<const float4*>(row);
+    for (int c = threadIdx.x; c < (V >> 2); c += blockDim.x) {
+      const float4 x = row4[c];
+      const float cm = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
+      fold(cm, __expf(x.x - cm) + __expf(x.y - cm) + __expf(x.z - cm) + __expf(x.w - cm));
+    }
+  } else {
+    for (int c = threadIdx.x; c < V; c += blockDim.x) fold(row[c], 1.f);
+  }
+  // block maximum, then every partial sum rescaled to it
+  float bm = mx;
 #pragma unroll
-  for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  for (int o = 16; o; o >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, o));
   __syncthreads();
-  if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = mx;
+  if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = bm;
   __syncthreads();
-  for (int i = 0; i < (blockDim.x >> 5); ++i) mx = fmaxf(mx, scratch[i]);
-  float s = 0.f;
-  for (int c = threadIdx.x; c < V; c += blockDim.x) s += expf(row[c] - mx);
+  for (int i = 0; i < (blockDim.x >> 5); ++i) bm = fmaxf(bm, scratch[i]);
+  s = (mx == -INFINITY) ? 0.f : s * __expf(mx - bm);
   s = block_sum(s, scratch);
   if (threadIdx.x == 0) {
     int32_t t = tok[m + 1];
     t = t < 0 ? 0 : (t >= V ? V - 1 : t);
-    tok_loss[m] = (static_cast<double>(mx) + log(static_cast<double>(s))) - static_cast<double>(row[t]);
+    tok_loss[m] = (static_cast<double>(bm) + log(static_cast<double>(s))) - static_cast<double>(row[t]);
   }
 }
 
