@@ -19,7 +19,10 @@ quantize_int4     Section 3.5 "Integration with quantization": a 4-bit quantizer
 dequantize        the inverse map, exact in fp64.
 dequantize_lut    Section 4 / appendix on hyperparameters: the experiments quantize with a non-uniform
                   4-bit format (SqueezeLLM), i.e. a code selects one of 16 per-output-channel
-                  values.  The inverse map is that table look-up, exact in fp64.
+                  values.  The inverse map is that table look-up, exact in fp64.  The paper does
+                  not spell the format out: the convention here (per-row table of 16 values in a
+                  16-bit float format, codes packed like the uniform format) is parity unpinned by
+                  the paper.
 effective_weight  Appendix "Implementation of Sparse Operations in Linear Layers":
                   Dequantize(Q(w_dense)) + w_sparse.
 linear_fwd        the same appendix: y = x (Dequantize(Q(w_dense)) + w_sparse)^T.
