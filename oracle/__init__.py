@@ -18,6 +18,6 @@ The paper prints no worked numeric example of a step, a mask or a quantized tens
 so absolute end-to-end values are "parity unpinned"; every function is pinned by
 closed forms, invariants, brute force or library routines in tests/test_oracle_*.py.
 The int4 rounding convention (uniform asymmetric, zero = group minimum, round half
-to even) is this build's reading: the paper allows any post-training quantizer, so
+to even) is the reading taken here: the paper allows any post-training quantizer, so
 that convention is "parity unpinned" by the paper and pinned only by its invariants.
 """

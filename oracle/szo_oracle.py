@@ -8,7 +8,7 @@ What each function restates
 philox4x32_10     Philox4x32-10 counter-based generator of Salmon, Moraes, Dror & Shaw
                   (SC'11), the published definition.  The paper only asks that z be
                   reproducible from a seed (Section 2.1, the "random seed trick"; Section 3.5,
-                  "Gradients"); keying it by (seed, step, parameter index) is this build's reading.
+                  "Gradients"); keying it by (seed, step, parameter index) is the reading taken here.
 gaussian          z ~ N(0,1) per parameter (Definition 1, SPSA): Box-Muller in fp64.
 select_mask       Definition 3 (sensitive parameter mask): the k coordinates with the largest
                   squared gradient, ties broken by lowest index.
