@@ -31,10 +31,12 @@ class DecoderFixture:
     quantize, all with the oracle; keeps every intermediate for comparison."""
 
     def __init__(self, name: str, seed: int = 0, mask: str = "gradient", n_mask_batches: int = 4,
-                 B: int = 4, S: int = 64, n_layers: int | None = None):
+                 B: int = 4, S: int = 64, n_layers: int | None = None, rho: float | None = None):
         shape = dict(wl.MODEL_SHAPES[name])
         if n_layers:
             shape["n_layers"] = n_layers
+        if rho is not None:
+            shape["rho"] = rho
         self.shape, self.seed, self.B, self.S = shape, seed, B, S
         self.cfg = decoder_config(shape)
         self.names = wl.linear_names(shape)

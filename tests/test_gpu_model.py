@@ -220,3 +220,32 @@ def test_resident_and_materialised_forms_at_test_size():
                          cwd=root, env=env, capture_output=True, text=True, timeout=900)
     assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-2000:]
     assert " passed" in res.stdout
+
+
+@pytest.mark.parametrize("name,rho", [("tiny_gqa", 1.6e-5), ("tiny", 1.6e-5), ("tiny", 0.0), ("tiny_gqa", 0.0)])
+def test_degenerate_masks(B, name, rho):
+    """Linears without a single sensitive entry next to linears with one or two (rho * n < 1 for the
+    narrow k/v projections), and a model with no sensitive entry at all (k = 0: both perturbed losses
+    equal the unperturbed one, g = 0, nothing to update), on the fp32 validation path against the
+    oracle and on the tensor-core path."""
+    fx = DecoderFixture(name, seed=1, mask="random", B=2, S=32, rho=rho)
+    om = fx.oracle_model()
+    toks = fx.batch(0)
+    fp, fm, g = mo.zo_step(om, toks, 7, 3, 1e-3, 1e-4, "lm", None, None)
+    d = lambda a: torch.from_numpy(a).cuda()
+    for act, mode, tol in ((B.SZO_F32, B.MODE_FP32_VALIDATE, 3e-6), (B.SZO_BF16, B.MODE_SPARSE_ADD, LOSS_TOL)):
+        t = fx.gpu_tensors(torch, None)
+        for key in [k for k, v in t.items() if k.endswith(".idx") and v.numel() == 0]:
+            del t[key]                                  # a linear without entries passes no index list
+        S = torch.from_numpy(fx.S_init.copy()).cuda() if len(fx.S_init) else torch.zeros(0, device="cuda")
+        m = B.Model(fx.shape, fx.names, t, S, act_dtype=act, linear_mode=mode, loss_kind=0, max_batch=fx.B, max_seq=fx.S)
+        assert m.k_total == len(fx.S_init)
+        out = m.zo_step(d(toks), 7, 3, 1e-3, 1e-4).cpu().numpy()
+        assert abs(out[0] - fp) <= tol * abs(fp) and abs(out[1] - fm) <= tol * abs(fm)
+        if rho == 0.0:
+            assert out[0] == out[1] and out[2] == 0.0
+        elif mode == B.MODE_FP32_VALIDATE:
+            assert abs(out[2] - g) <= g_tol(g, fp, 1e-3)
+            assert np.allclose(S.cpu().numpy(), om.S, rtol=0, atol=2e-7)
+        assert B.device_status() == 0
+        m.close()
