@@ -219,7 +219,9 @@ __device__ __noinline__ void reduce_parts(const float* part0, int parts, int64_t
   }
 }
 
-template <int kXS, bool kDequant, bool kFast>
+// kRelu: y = max(y, 0) in the epilogue (dense mode only: its own instantiation, so that the other
+// launches' store loops stay as they are)
+template <int kXS, bool kDequant, bool kFast, bool kRelu = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumWarps2 * 32, 1)
 szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                       const TcParams P) {
@@ -597,8 +599,10 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
       const int64_t m0 = static_cast<int64_t>(u.m_tile) * kPairBT;
       const int mlimit = static_cast<int>((P.M - m0 < kPairBT) ? P.M - m0 : kPairBT);
       // y[m0 + c0 + j, n] = v[j] + bias for the valid tokens of a 32-token chunk
-      const bool relu = P.relu != 0;
-      auto act = [&](float t) { return relu ? fmaxf(t, 0.f) : t; };
+      auto act = [&](float t) {
+        if constexpr (kRelu) return fmaxf(t, 0.f);
+        else return t;
+      };
       auto store_chunk = [&](int c0, const uint32_t (&v)[32]) {
         if (n < N && c0 < mlimit) {
           const int cnt = mlimit - c0;
@@ -674,18 +678,18 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     const int mlimit = static_cast<int>((P.M - m0 < kPairBT) ? P.M - m0 : kPairBT);
     reduce_parts(P.partial + (static_cast<int64_t>(u.slot * u.parts) * 2 + rank) * kPartFloats, u.parts,
                  static_cast<int64_t>(u.n_tile) * kBM, SZO_SUB(P, u.s, N), SZO_SUB(P, u.s, bias), SZO_SUB(P, u.s, y), P.y_f32,
-                 P.relu, m0, mlimit, static_cast<int>(threadIdx.x), kNumWarps2 * 32);
+                 kRelu ? 1 : 0, m0, mlimit, static_cast<int>(threadIdx.x), kNumWarps2 * 32);
   }
   cluster_sync_all();          // no CTA leaves while its peer may still signal it or read its tiles
   tc_fence_after();
   if (warp == kWarpMma) tmem_dealloc2(tmem_base, kTmemCols);
 }
 
-template <int kXS, bool kDequant, bool kFast>
+template <int kXS, bool kDequant, bool kFast, bool kRelu = false>
 szo_status launch_tc2(const CUtensorMap& mx, const CUtensorMap& mw, const TcParams& P, int n_pairs, cudaStream_t st) {
   constexpr size_t smem = static_cast<size_t>(kXS) * (kXHalfBytes + (kDequant ? 0 : kATileBytes)) +
                           (kDequant ? kCStages2 * (kCodesBytes + kSzBytes) + kASlots2 * kATileBytes : 0) + 1024;
-  auto kern = szo_linear_tc2_kernel<kXS, kDequant, kFast>;
+  auto kern = szo_linear_tc2_kernel<kXS, kDequant, kFast, kRelu>;
   static bool configured = false;
   if (!configured) {
     SZO_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
@@ -701,7 +705,9 @@ szo_status launch_tc2(const CUtensorMap& mx, const CUtensorMap& mw, const TcPara
 
 szo_status launch_pair_kernel(bool dequant, bool bf16_tables, const CUtensorMap& mx, const CUtensorMap& mw,
                               const tc::TcParams& P, int n_pairs, cudaStream_t st) {
+  if (!dequant && P.relu) return launch_tc2<6, false, false, true>(mx, mw, P, n_pairs, st);
   if (!dequant) return launch_tc2<6, false, false>(mx, mw, P, n_pairs, st);
+  SZO_REQUIRE(!P.relu, SZO_ERR_UNSUPPORTED, "the ReLU epilogue exists in the dense mode only");
   if (bf16_tables) return launch_tc2<4, true, true>(mx, mw, P, n_pairs, st);
   return launch_tc2<4, true, false>(mx, mw, P, n_pairs, st);
 }
