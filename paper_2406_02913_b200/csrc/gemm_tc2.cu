@@ -615,10 +615,22 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             }
           } else {
             __nv_bfloat16* yp = static_cast<__nv_bfloat16*>(y) + (m0 + c0) * N + n;
+            if (cnt >= 32) {
+              // a full chunk: no per-token predicate, two tokens per conversion
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              if (j < cnt) *yp = __float2bfloat16_rn(act(__uint_as_float(v[j]) + bias));
-              yp += N;
+              for (int j = 0; j < 32; j += 2) {
+                const __nv_bfloat162 pr = __floats2bfloat162_rn(act(__uint_as_float(v[j]) + bias),
+                                                                act(__uint_as_float(v[j + 1]) + bias));
+                yp[0] = pr.x;
+                yp[N] = pr.y;
+                yp += 2 * N;
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                if (j < cnt) *yp = __float2bfloat16_rn(act(__uint_as_float(v[j]) + bias));
+                yp += N;
+              }
             }
           }
         }
