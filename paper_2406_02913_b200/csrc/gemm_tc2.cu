@@ -608,10 +608,18 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
           const int cnt = mlimit - c0;
           if (P.y_f32) {
             float* yp = static_cast<float*>(y) + (m0 + c0) * N + n;
+            if (cnt >= 32) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              if (j < cnt) *yp = act(__uint_as_float(v[j]) + bias);
-              yp += N;
+              for (int j = 0; j < 32; ++j) {
+                *yp = act(__uint_as_float(v[j]) + bias);
+                yp += N;
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                if (j < cnt) *yp = act(__uint_as_float(v[j]) + bias);
+                yp += N;
+              }
             }
           } else {
             __nv_bfloat16* yp = static_cast<__nv_bfloat16*>(y) + (m0 + c0) * N + n;
