@@ -623,8 +623,16 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             }
           } else {
             __nv_bfloat16* yp = static_cast<__nv_bfloat16*>(y) + (m0 + c0) * N + n;
-            if (cnt >= 32) {
-              // a full chunk: no per-token predicate, two tokens per conversion
+            if (cnt >= 32 && bias_p == nullptr) {
+              // a full chunk: no per-token predicate, two tokens per conversion (and nothing to add)
+#pragma unroll
+              for (int j = 0; j < 32; j += 2) {
+                const __nv_bfloat162 pr = __floats2bfloat162_rn(act(__uint_as_float(v[j])), act(__uint_as_float(v[j + 1])));
+                yp[0] = pr.x;
+                yp[N] = pr.y;
+                yp += 2 * N;
+              }
+            } else if (cnt >= 32) {
 #pragma unroll
               for (int j = 0; j < 32; j += 2) {
                 const __nv_bfloat162 pr = __floats2bfloat162_rn(act(__uint_as_float(v[j]) + bias),
