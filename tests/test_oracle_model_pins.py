@@ -157,6 +157,91 @@ def test_decoder_blocks_against_an_independent_einsum_statement():
     assert np.allclose(got, ref, rtol=0, atol=1e-12)
 
 
+def _opt_layer_numpy(params, W, tokens, H, eps=1e-5, act=lambda t: np.maximum(t, 0.0)):
+    """One OPT decoder layer + final LayerNorm written with numpy loops and einsum (no torch, nothing
+    from the oracle): token + learned-position embedding from position 0, pre-LayerNorm with gain and
+    shift, a bias on each of q/k/v/o/fc1/fc2, causal softmax attention without rotary positions,
+    fc2(relu(fc1 x + b1)) + b2, residuals around both blocks."""
+    f64 = lambda a: np.asarray(a, dtype=np.float64)
+    B, S = tokens.shape
+    d = params["embed"].shape[1]
+    hd = d // H
+    h = np.empty((B, S, d))
+    for b in range(B):
+        for s in range(S):
+            h[b, s] = f64(params["embed"])[tokens[b, s]] + f64(params["pos"])[s]
+
+    def ln(x, name):
+        mu = x.sum(-1, keepdims=True) / d
+        var = ((x - mu) ** 2).sum(-1, keepdims=True) / d
+        return (x - mu) / np.sqrt(var + eps) * f64(params[name]) + f64(params[name + "_b"])
+
+    def lin(x, nm):
+        return np.einsum("bsk,nk->bsn", x, f64(W[nm])) + f64(params[f"l0.{nm}_b"])
+
+    a = ln(h, "l0.attn_norm")
+    q, k, v = (lin(a, nm).reshape(B, S, H, hd) for nm in ("wq", "wk", "wv"))
+    o = np.zeros((B, S, H, hd))
+    for b in range(B):
+        for hh in range(H):
+            for s in range(S):
+                sc = np.array([q[b, s, hh] @ k[b, t, hh] / np.sqrt(hd) for t in range(s + 1)])
+                p = np.exp(sc - sc.max())
+                p /= p.sum()
+                o[b, s, hh] = sum(p[t] * v[b, t, hh] for t in range(s + 1))
+    h = h + lin(o.reshape(B, S, d), "wo")
+    m = ln(h, "l0.mlp_norm")
+    h = h + lin(act(lin(m, "fc1")), "fc2")
+    return ln(h, "final_norm")
+
+
+def _opt_case():
+    cfg, params, lin_W, tokens = _small("opt")
+    params = dict(params)
+    g = np.random.default_rng(5)
+    for k in list(params):                        # a different gain and shift for every norm
+        if k.endswith("norm"):
+            params[k] = (1 + 0.2 * g.standard_normal(32)).astype(np.float32)
+        if k.endswith("norm_b"):
+            params[k] = (0.3 * g.standard_normal(32)).astype(np.float32)
+    cfg1 = mo.DecoderConfig(**{**cfg.__dict__, "n_layers": 1})
+    return cfg1, params, lin_W[:1], tokens
+
+
+def test_opt_blocks_against_an_independent_numpy_statement():
+    """The OPT branch of hidden_states (learned positions, LayerNorm with shift, biases, ReLU MLP)
+    against a restatement that shares nothing with it."""
+    cfg1, params, lin_W, tokens = _opt_case()
+    got = mo.hidden_states(cfg1, params, lin_W, tokens).numpy()
+    ref = _opt_layer_numpy(params, lin_W[0], tokens, H=4)
+    assert np.allclose(got, ref, rtol=0, atol=1e-12)
+
+
+def test_opt_statement_notices_a_dropped_bias_a_position_shift_and_post_norm():
+    """The pin above has teeth: handing the oracle inputs that stand for a plausible mistake (fc2's
+    bias missing, positions starting at 1, a zeroed norm shift, no ReLU effect) moves its output far
+    beyond the comparison's tolerance, so such a mistake inside the oracle would be seen."""
+    cfg1, params, lin_W, tokens = _opt_case()
+    ref = _opt_layer_numpy(params, lin_W[0], tokens, H=4)
+
+    def oracle_with(**changes):
+        p = dict(params)
+        p.update(changes)
+        return mo.hidden_states(cfg1, p, lin_W, tokens).numpy()
+
+    for nm in ("wq", "wk", "wv", "wo", "fc1", "fc2"):
+        key = f"l0.{nm}_b"
+        if nm == "wk":
+            continue           # a bias on k shifts every score of a row equally: softmax removes it
+        assert np.abs(oracle_with(**{key: np.zeros_like(params[key])}) - ref).max() > 1e-6, nm
+    assert np.abs(oracle_with(pos=np.roll(params["pos"], -1, axis=0)) - ref).max() > 1e-6
+    for key in ("l0.attn_norm_b", "l0.mlp_norm_b", "final_norm_b"):
+        assert np.abs(oracle_with(**{key: np.zeros_like(params[key])}) - ref).max() > 1e-6, key
+    # the ReLU matters on these inputs: a statement without the clamp is far from the oracle
+    got = mo.hidden_states(cfg1, params, lin_W, tokens).numpy()
+    assert np.abs(_opt_layer_numpy(params, lin_W[0], tokens, H=4, act=lambda t: t) - got).max() > 1e-6
+
+
 def test_gqa_reduces_to_mha_when_kv_heads_are_duplicated():
     cfg, params, lin_W, tokens = _small("llama", kv=2)
     full = mo.DecoderConfig(**{**cfg.__dict__, "n_kv_heads": 4})
