@@ -189,8 +189,9 @@ def run_ours(args):
 
     shape = wl.MODEL_SHAPES[WORKLOAD]
     tensors, S_all = wl.device_decoder_tensors(shape, seed=rank)
+    mode = {"paired": B.MODE_PAIRED, "sparse_add": B.MODE_SPARSE_ADD}[args.mode]
     model = B.Model(shape, wl.linear_names(shape), tensors, S_all, act_dtype=B.SZO_BF16,
-                    linear_mode=B.MODE_SPARSE_ADD, loss_kind=B.LOSS_CLS2, max_batch=BATCH, max_seq=SEQ)
+                    linear_mode=mode, loss_kind=B.LOSS_CLS2, max_batch=BATCH, max_seq=SEQ)
     n_steps = args.warmup + args.steps
     toks_host = [torch.from_numpy(wl.token_batch(shape["vocab"], BATCH, SEQ, rank, wl.PURPOSE_TRAIN_BATCH, i)).pin_memory()
                  for i in range(n_steps)]
@@ -275,6 +276,9 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--mode", default="paired", choices=["paired", "sparse_add"],
+                    help="paired: both forwards of a step in one pass as centre / half-difference (the default: "
+                         "the form whose projected gradient meets the tested bound); sparse_add: two bf16 forwards")
     ap.add_argument("--profile-range", action="store_true",
                     help="bracket the timed region with cudaProfilerStart/Stop (for ncu --profile-from-start off)")
     args = ap.parse_args()

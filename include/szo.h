@@ -56,8 +56,12 @@ typedef enum {
                                  dequantised bf16 tile in shared memory before the tensor-core MMA */
   SZO_MODE_SPMM = 2,          /* SparseAddMM(Dequantize(Q) x, S, x): tensor-core GEMM on the dense
                                  part, then a row-bucketed CSR SpMM with fp32 values */
-  SZO_MODE_FP32_VALIDATE = 3  /* fp32 CUDA-core evaluation of the same expression (exact fp32
+  SZO_MODE_FP32_VALIDATE = 3, /* fp32 CUDA-core evaluation of the same expression (exact fp32
                                  sparse term); slow, for checking losses and projected gradients */
+  SZO_MODE_PAIRED = 4         /* szo_model_config.linear_mode only: the two forwards of a ZO step run as
+                                 ONE pass that carries the centre (x+ + x-)/2 and the half-difference
+                                 (x+ - x-)/2 of every activation (see szo_linear_fwd_paired); lone
+                                 forwards (szo_model_loss) run as SZO_MODE_SPARSE_ADD */
 } szo_linear_mode;
 
 const char* szo_status_string(szo_status s);   /* static storage */
@@ -179,6 +183,29 @@ szo_status szo_linear_fwd(const szo_linear_t* plan, const void* x, szo_dtype x_d
                           const float* S_pert, void* y, szo_dtype y_dtype, int32_t mode,
                           void* workspace, size_t workspace_bytes, void* stream);
 size_t szo_linear_workspace_bytes(const szo_linear_t* plan, int64_t M, int32_t mode);
+
+/* ---- The same layer for BOTH forwards of a ZO step at once, in the paired form.  Definition 1 (SPSA)
+ * needs the loss at w + eps zbar and at w - eps zbar on the same batch; only the difference of the
+ * two enters the projected gradient.  The perturbation moves an activation by less than one bf16 ulp,
+ * so two forwards whose activations are each rounded to bf16 lose that difference in rounding.  Here
+ * the pair (x+, x-) travels as centre xc = (x+ + x-)/2 and half-difference xd = (x+ - x-)/2, each
+ * in bf16 with its own exponent.  With W = RN_bf16(Dequantize(Q(w_dense)) + S) (Section 3.4's
+ * decomposition, S unperturbed; the appendix's SparseAdd order) and Zbar = z at the sensitive
+ * entries (Definition 4):
+ *     yc = xc W^T (+ bias)            yd = xd W^T + eps * xc Zbar^T
+ * which are centre and half-difference of x+ (W + eps Zbar)^T and x- (W - eps Zbar)^T except for the
+ * term eps * xd Zbar^T in yc, of relative order eps^2 and left out.  The dense products run on the
+ * tensor cores; eps * xc Zbar^T is accumulated in fp32 onto the fp32 accumulator before the one
+ * rounding of the store (the appendix's SparseAddMM order, for the perturbation only).
+ *   x   bf16 [M0 + M, K]: rows [0, M) = xc, rows [M0, M0 + M) = xd, M0 = M rounded up to a multiple of
+ *       256 (rows in between are ignored)            y   y_dtype [M0 + M, N], same row layout
+ *   S   fp32 [nnz] current sparse values             z   fp32 [nnz] z of this step at the entries of idx
+ *   workspace  szo_linear_paired_workspace_bytes(plan, M) bytes (effective weight, x^T, K-split scratch)
+ * Every plan format is accepted (int4 groups, per-row tables, dense bf16). */
+size_t szo_linear_paired_workspace_bytes(const szo_linear_t* plan, int64_t M);
+szo_status szo_linear_fwd_paired(const szo_linear_t* plan, const void* x, int64_t M, const float* S, const float* z,
+                                 float eps, void* y, szo_dtype y_dtype, void* workspace, size_t workspace_bytes,
+                                 void* stream);
 void szo_linear_destroy(szo_linear_t* plan);
 
 /* ---- Whole loss path and ZO step on one GPU (Definition 1 evaluates the loss twice per step;
@@ -230,6 +257,13 @@ typedef struct {
 szo_status szo_attention(const void* q, const void* k, const void* v, void* o, szo_dtype dtype, int32_t B, int32_t S,
                          int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, void* stream);
 
+/* The same attention in the paired form of szo_linear_fwd_paired: every buffer holds the B*S centre rows
+ * first and the half-difference rows from row `row0` (>= B*S) on; the outputs are the exact centre and
+ * half-difference of attention(q+, k+, v+) and attention(q-, k-, v-) (nothing of higher order is left
+ * out), bf16 only. */
+szo_status szo_attention_paired(const void* q, const void* k, const void* v, void* o, int64_t row0, int32_t B,
+                                int32_t S, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, void* stream);
+
 typedef struct szo_model szo_model_t;
 /* layers_host: host array of n_layers entries holding device pointers.  S_all: fp32 [k_total],
  * the trainable sparse values of all linears concatenated in model order (the only mutable
@@ -249,7 +283,11 @@ szo_status szo_model_loss(szo_model_t* m, const int32_t* tokens, const int32_t* 
                           const int32_t* cand, int32_t B, int32_t S, const float* S_vals,
                           double* loss_dev, void* stream);
 /* One step in the seed trick's in-place order: S += eps z; f+; S -= 2 eps z; f-; S += eps z;
- * g = (f+ - f-)/(2 eps); S -= lr g z.  Outputs are device scalars (fp64); no host read-back. */
+ * g = (f+ - f-)/(2 eps); S -= lr g z.  Outputs are device scalars (fp64); no host read-back.
+ * With linear_mode SZO_MODE_PAIRED, S goes through the same three passes first and both losses are then
+ * evaluated in one pass in the paired form (z kept in device memory, +- eps z applied inside the linears
+ * in fp32): f+ and f- are the same two function values, with their difference resolved far below the
+ * bf16 rounding of the activations. */
 szo_status szo_model_zo_step(szo_model_t* m, const int32_t* tokens, const int32_t* labels,
                              const int32_t* cand, int32_t B, int32_t S, uint64_t seed,
                              uint64_t step, float eps, float lr, double* f_plus_dev,

@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libszo.so")
 
 SZO_F32, SZO_BF16, SZO_F16 = 0, 1, 2
-MODE_AUTO, MODE_SPARSE_ADD, MODE_SPMM, MODE_FP32_VALIDATE = 0, 1, 2, 3
+MODE_AUTO, MODE_SPARSE_ADD, MODE_SPMM, MODE_FP32_VALIDATE, MODE_PAIRED = 0, 1, 2, 3, 4
 LOSS_LM, LOSS_CLS2 = 0, 1
 ARCH_LLAMA, ARCH_OPT = 0, 1
 
@@ -85,7 +85,12 @@ _SIGS = {
     "szo_linear_fwd": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_void_p, C.c_void_p,
                                    C.c_int, C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p]),
     "szo_linear_workspace_bytes": (C.c_size_t, [C.c_void_p, C.c_int64, C.c_int32]),
+    "szo_linear_paired_workspace_bytes": (C.c_size_t, [C.c_void_p, C.c_int64]),
+    "szo_linear_fwd_paired": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_float,
+                                          C.c_void_p, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]),
     "szo_linear_destroy": (None, [C.c_void_p]),
+    "szo_attention_paired": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int32,
+                                         C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]),
     "szo_attention": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int32, C.c_int32,
                                   C.c_int32, C.c_int32, C.c_int32, C.c_void_p]),
     "szo_model_create": (C.c_int32, [C.POINTER(C.c_void_p), C.POINTER(ModelConfig),
@@ -247,6 +252,20 @@ class Linear:
                                     _stream()))
         return y
 
+    def fwd_paired(self, x, M, S, z, eps, out_dtype=torch.bfloat16):
+        """x: bf16 [paired_row0(M) + M, K] (centre rows, then half-difference rows); returns y in the
+        same row layout."""
+        rows = paired_row0(M) + M
+        assert x.shape[0] == rows
+        y = torch.zeros((rows, self.N), dtype=out_dtype, device=x.device)
+        need = lib().szo_linear_paired_workspace_bytes(self.h, M)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty((need,), dtype=torch.uint8, device=x.device)
+        _check(lib().szo_linear_fwd_paired(self.h, _ptr(x), M, _ptr(S) if self.nnz else None,
+                                           _ptr(z) if self.nnz else None, eps, _ptr(y), _DT[y.dtype], _ptr(self._ws),
+                                           need, _stream()))
+        return y
+
     def close(self):
         if getattr(self, "h", None):
             lib().szo_linear_destroy(self.h)
@@ -257,6 +276,20 @@ class Linear:
             self.close()
         except Exception:
             pass
+
+
+def paired_row0(M: int) -> int:
+    """First half-difference row of a paired buffer with M centre rows."""
+    return (M + 255) // 256 * 256
+
+
+def szo_attention_paired(q, k, v, row0: int, B: int, S: int, n_heads: int, n_kv_heads: int, head_dim: int):
+    """Paired causal attention; every tensor holds B*S centre rows and, from row row0 on, B*S
+    half-difference rows (bf16).  Returns o like q."""
+    o = torch.zeros_like(q)
+    _check(lib().szo_attention_paired(_ptr(q), _ptr(k), _ptr(v), _ptr(o), row0, B, S, n_heads, n_kv_heads,
+                                      head_dim, _stream()))
+    return o
 
 
 def szo_attention(q, k, v, B: int, S: int, n_heads: int, n_kv_heads: int, head_dim: int):

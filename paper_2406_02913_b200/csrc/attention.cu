@@ -227,6 +227,236 @@ flash_attn_bf16_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16*
   }
 }
 
+// ------------------------------------------------------------------------------ paired form
+// Causal attention of the two forwards of a ZO step given as centre and half-difference (see
+// model.cu): inputs qc, qd, kc, kd, vc, vd; with s+- = (qc +- qd)(kc +- kd)^T = sc +- sd,
+//   sc = qc kc^T + qd kd^T,  sd = qc kd^T + qd kc^T,
+//   p+- = exp(sc - m) exp(+-sd):  pc = exp(sc - m) cosh(sd),  pd = exp(sc - m) sinh(sd)   (m >= sc + |sd|),
+//   Oc = pc vc + pd vd,  Od = pc vd + pd vc,  lc = sum pc,  ld = sum pd,
+//   o+- = (Oc +- Od) / (lc +- ld):  oc = (Oc lc - Od ld) / (lc^2 - ld^2),  od = (Od lc - Oc ld) / (lc^2 - ld^2).
+// Nothing is dropped: the result is the exact centre and half-difference of the two attentions, up
+// to the rounding of pc, pd to bf16 and the fp32 accumulation.  Same tiling as above with 32-key
+// tiles (twice the accumulators); the query tiles stay in shared memory.
+constexpr int kKT2 = 32;
+
+__device__ __forceinline__ float sinh_small(float a) {
+  const float a2 = a * a;
+  if (a2 < 0.25f) return a * (1.0f + a2 * (1.0f / 6.0f + a2 * (1.0f / 120.0f + a2 * (1.0f / 5040.0f + a2 * (1.0f / 362880.0f)))));
+  const float u = __expf(a);
+  return 0.5f * (u - 1.0f / u);
+}
+
+template <int HD>
+__device__ __forceinline__ void load_tile_async_rows(__nv_bfloat16* dst, const __nv_bfloat16* src, int64_t ld, int rows,
+                                                     int valid) {
+  constexpr int kChunks = HD / 8;
+  for (int i = threadIdx.x; i < rows * kChunks; i += 128) {
+    const int r = i / kChunks, c = i % kChunks;
+    __nv_bfloat16* d = dst + r * (HD + 8) + c * 8;
+    if (r < valid) {
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(d))),
+                   "l"(src + r * ld + c * 8)
+                   : "memory");
+    } else {
+      *reinterpret_cast<uint4*>(d) = make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
+}
+
+template <int HD>
+__global__ void __launch_bounds__(128, 2)
+flash_attn_pair_bf16_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                            const __nv_bfloat16* __restrict__ v, __nv_bfloat16* __restrict__ o, int64_t row0, int S,
+                            int H, int Hkv, float scale, float scale_log2e) {
+  constexpr int LDS = HD + 8;
+  extern __shared__ __align__(16) unsigned char smem_attn[];
+  __nv_bfloat16* sQc = reinterpret_cast<__nv_bfloat16*>(smem_attn);
+  __nv_bfloat16* sQd = sQc + kQT * LDS;
+  __nv_bfloat16* sKV = sQd + kQT * LDS;          // two stages of (Kc, Kd, Vc, Vd), kKT2 rows each
+
+  const int qt = gridDim.x - 1 - blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
+  const int hk = hq / (H / Hkv);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int64_t ldq = static_cast<int64_t>(H) * HD, ldk = static_cast<int64_t>(Hkv) * HD;
+  const int q0 = qt * kQT;
+  const int64_t offq = row0 * ldq, offk = row0 * ldk;           // the half-difference rows
+  const __nv_bfloat16* qbase = q + (static_cast<int64_t>(b) * S + q0) * ldq + hq * HD;
+  const int n_kt = (((q0 + kQT < S) ? q0 + kQT : S) + kKT2 - 1) / kKT2;
+  auto issue_kv = [&](int kt) {
+    const int k0 = kt * kKT2;
+    const int valid = S - k0 < kKT2 ? S - k0 : kKT2;
+    __nv_bfloat16* st = sKV + (kt & 1) * 4 * kKT2 * LDS;
+    const __nv_bfloat16* kp = k + (static_cast<int64_t>(b) * S + k0) * ldk + hk * HD;
+    const __nv_bfloat16* vp = v + (static_cast<int64_t>(b) * S + k0) * ldk + hk * HD;
+    load_tile_async_rows<HD>(st, kp, ldk, kKT2, valid);
+    load_tile_async_rows<HD>(st + kKT2 * LDS, kp + offk, ldk, kKT2, valid);
+    load_tile_async_rows<HD>(st + 2 * kKT2 * LDS, vp, ldk, kKT2, valid);
+    load_tile_async_rows<HD>(st + 3 * kKT2 * LDS, vp + offk, ldk, kKT2, valid);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  {
+    const int valid = S - q0 < kQT ? S - q0 : kQT;
+    load_tile_async_rows<HD>(sQc, qbase, ldq, kQT, valid);
+    load_tile_async_rows<HD>(sQd, qbase + offq, ldq, kQT, valid);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
+  issue_kv(0);
+
+  float oc[HD / 8][4], od[HD / 8][4];
+#pragma unroll
+  for (int i = 0; i < HD / 8; ++i) {
+    oc[i][0] = oc[i][1] = oc[i][2] = oc[i][3] = 0.f;
+    od[i][0] = od[i][1] = od[i][2] = od[i][3] = 0.f;
+  }
+  float mrow[2] = {-INFINITY, -INFINITY}, lc[2] = {0.f, 0.f}, ldr[2] = {0.f, 0.f};
+  const int row_a = q0 + warp * 16 + g, row_b = row_a + 8;
+
+  for (int kt = 0; kt < n_kt; ++kt) {
+    const int k0 = kt * kKT2;
+    if (kt + 1 < n_kt) {
+      issue_kv(kt + 1);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    __syncthreads();
+    const __nv_bfloat16* sKc = sKV + (kt & 1) * 4 * kKT2 * LDS;
+    const __nv_bfloat16* sKd = sKc + kKT2 * LDS;
+    const __nv_bfloat16* sVc = sKd + kKT2 * LDS;
+    const __nv_bfloat16* sVd = sVc + kKT2 * LDS;
+
+    float sc[kKT2 / 8][4], sd[kKT2 / 8][4];
+#pragma unroll
+    for (int i = 0; i < kKT2 / 8; ++i) {
+      sc[i][0] = sc[i][1] = sc[i][2] = sc[i][3] = 0.f;
+      sd[i][0] = sd[i][1] = sd[i][2] = sd[i][3] = 0.f;
+    }
+#pragma unroll
+    for (int ks = 0; ks < HD / 16; ++ks) {
+      uint32_t ac[4], ad[4];
+      const int qoff = (warp * 16 + (lane & 15)) * LDS + ks * 16 + (lane >> 4) * 8;
+      ldsm_x4(static_cast<uint32_t>(__cvta_generic_to_shared(sQc + qoff)), ac[0], ac[1], ac[2], ac[3]);
+      ldsm_x4(static_cast<uint32_t>(__cvta_generic_to_shared(sQd + qoff)), ad[0], ad[1], ad[2], ad[3]);
+#pragma unroll
+      for (int np = 0; np < kKT2 / 16; ++np) {
+        const int koff = (np * 16 + (lane & 7) + (lane >> 4) * 8) * LDS + ks * 16 + ((lane >> 3) & 1) * 8;
+        uint32_t b0, b1, b2, b3, d0, d1, d2, d3;
+        ldsm_x4(static_cast<uint32_t>(__cvta_generic_to_shared(sKc + koff)), b0, b1, b2, b3);
+        ldsm_x4(static_cast<uint32_t>(__cvta_generic_to_shared(sKd + koff)), d0, d1, d2, d3);
+        mma_bf16(sc[2 * np], ac, b0, b1);
+        mma_bf16(sc[2 * np + 1], ac, b2, b3);
+        mma_bf16(sc[2 * np], ad, d0, d1);
+        mma_bf16(sc[2 * np + 1], ad, d2, d3);
+        mma_bf16(sd[2 * np], ac, d0, d1);
+        mma_bf16(sd[2 * np + 1], ac, d2, d3);
+        mma_bf16(sd[2 * np], ad, b0, b1);
+        mma_bf16(sd[2 * np + 1], ad, b2, b3);
+      }
+    }
+    // causal mask and keys beyond the sequence
+    if (k0 + kKT2 > q0 || k0 + kKT2 > S) {
+#pragma unroll
+      for (int i = 0; i < kKT2 / 8; ++i) {
+        const int c = k0 + i * 8 + 2 * t;
+        if (c > row_a || c >= S) { sc[i][0] = -INFINITY; sd[i][0] = 0.f; }
+        if (c + 1 > row_a || c + 1 >= S) { sc[i][1] = -INFINITY; sd[i][1] = 0.f; }
+        if (c > row_b || c >= S) { sc[i][2] = -INFINITY; sd[i][2] = 0.f; }
+        if (c + 1 > row_b || c + 1 >= S) { sc[i][3] = -INFINITY; sd[i][3] = 0.f; }
+      }
+    }
+    // reference value per row: >= sc + |sd| of every key seen so far (raw score units)
+    float mx[2] = {mrow[0], mrow[1]};
+#pragma unroll
+    for (int i = 0; i < kKT2 / 8; ++i) {
+      mx[0] = fmaxf(mx[0], fmaxf(sc[i][0] + fabsf(sd[i][0]), sc[i][1] + fabsf(sd[i][1])));
+      mx[1] = fmaxf(mx[1], fmaxf(sc[i][2] + fabsf(sd[i][2]), sc[i][3] + fabsf(sd[i][3])));
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+    }
+    float corr[2], msc[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      msc[r] = (mx[r] == -INFINITY) ? 0.f : mx[r] * scale_log2e;
+      corr[r] = (mrow[r] == -INFINITY) ? 0.f : exp2f(mrow[r] * scale_log2e - msc[r]);
+      mrow[r] = mx[r];
+      lc[r] *= corr[r];
+      ldr[r] *= corr[r];
+    }
+    uint32_t pac[kKT2 / 16][4], pad[kKT2 / 16][4];
+#pragma unroll
+    for (int i = 0; i < kKT2 / 8; ++i) {
+      float pc4[4], pd4[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float e = exp2f(sc[i][j] * scale_log2e - msc[j >> 1]);
+        const float a = sd[i][j] * scale;
+        const float u = exp2f(sd[i][j] * scale_log2e);
+        pc4[j] = e * 0.5f * (u + 1.0f / u);
+        pd4[j] = e * sinh_small(a);
+      }
+      lc[0] += pc4[0] + pc4[1];
+      lc[1] += pc4[2] + pc4[3];
+      ldr[0] += pd4[0] + pd4[1];
+      ldr[1] += pd4[2] + pd4[3];
+      pac[i >> 1][(i & 1) * 2 + 0] = pack2(pc4[0], pc4[1]);
+      pac[i >> 1][(i & 1) * 2 + 1] = pack2(pc4[2], pc4[3]);
+      pad[i >> 1][(i & 1) * 2 + 0] = pack2(pd4[0], pd4[1]);
+      pad[i >> 1][(i & 1) * 2 + 1] = pack2(pd4[2], pd4[3]);
+    }
+#pragma unroll
+    for (int i = 0; i < HD / 8; ++i) {
+      oc[i][0] *= corr[0]; oc[i][1] *= corr[0]; oc[i][2] *= corr[1]; oc[i][3] *= corr[1];
+      od[i][0] *= corr[0]; od[i][1] *= corr[0]; od[i][2] *= corr[1]; od[i][3] *= corr[1];
+    }
+#pragma unroll
+    for (int ks = 0; ks < kKT2 / 16; ++ks) {
+#pragma unroll
+      for (int dp = 0; dp < HD / 16; ++dp) {
+        const int voff = (ks * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * LDS + dp * 16 + (lane >> 4) * 8;
+        uint32_t b0, b1, b2, b3, d0, d1, d2, d3;
+        ldsm_x4_trans(static_cast<uint32_t>(__cvta_generic_to_shared(sVc + voff)), b0, b1, b2, b3);
+        ldsm_x4_trans(static_cast<uint32_t>(__cvta_generic_to_shared(sVd + voff)), d0, d1, d2, d3);
+        mma_bf16(oc[2 * dp], pac[ks], b0, b1);
+        mma_bf16(oc[2 * dp + 1], pac[ks], b2, b3);
+        mma_bf16(oc[2 * dp], pad[ks], d0, d1);
+        mma_bf16(oc[2 * dp + 1], pad[ks], d2, d3);
+        mma_bf16(od[2 * dp], pac[ks], d0, d1);
+        mma_bf16(od[2 * dp + 1], pac[ks], d2, d3);
+        mma_bf16(od[2 * dp], pad[ks], b0, b1);
+        mma_bf16(od[2 * dp + 1], pad[ks], b2, b3);
+      }
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    lc[r] += __shfl_xor_sync(0xffffffffu, lc[r], 1);
+    lc[r] += __shfl_xor_sync(0xffffffffu, lc[r], 2);
+    ldr[r] += __shfl_xor_sync(0xffffffffu, ldr[r], 1);
+    ldr[r] += __shfl_xor_sync(0xffffffffu, ldr[r], 2);
+  }
+  const float inv_a = 1.0f / (lc[0] * lc[0] - ldr[0] * ldr[0]), inv_b = 1.0f / (lc[1] * lc[1] - ldr[1] * ldr[1]);
+  __nv_bfloat16* obase = o + static_cast<int64_t>(b) * S * ldq + hq * HD;
+#pragma unroll
+  for (int i = 0; i < HD / 8; ++i) {
+    const int c = i * 8 + 2 * t;
+    if (row_a < S) {
+      __nv_bfloat16* p = obase + row_a * ldq + c;
+      *reinterpret_cast<uint32_t*>(p) = pack2((oc[i][0] * lc[0] - od[i][0] * ldr[0]) * inv_a, (oc[i][1] * lc[0] - od[i][1] * ldr[0]) * inv_a);
+      *reinterpret_cast<uint32_t*>(p + offq) = pack2((od[i][0] * lc[0] - oc[i][0] * ldr[0]) * inv_a, (od[i][1] * lc[0] - oc[i][1] * ldr[0]) * inv_a);
+    }
+    if (row_b < S) {
+      __nv_bfloat16* p = obase + row_b * ldq + c;
+      *reinterpret_cast<uint32_t*>(p) = pack2((oc[i][2] * lc[1] - od[i][2] * ldr[1]) * inv_b, (oc[i][3] * lc[1] - od[i][3] * ldr[1]) * inv_b);
+      *reinterpret_cast<uint32_t*>(p + offq) = pack2((od[i][2] * lc[1] - oc[i][2] * ldr[1]) * inv_b, (od[i][3] * lc[1] - oc[i][3] * ldr[1]) * inv_b);
+    }
+  }
+}
+
 }  // namespace
 
 szo_status launch_flash_attention_bf16(const void* q, const void* k, const void* v, void* o, int B, int S, int H,
@@ -258,6 +488,38 @@ szo_status launch_flash_attention_bf16(const void* q, const void* k, const void*
   }
   count_launch();
   SZO_CHECK_LAUNCH("flash_attn_bf16_kernel");
+  return SZO_OK;
+}
+
+}  // namespace szo
+
+namespace szo {
+
+// Paired form: every buffer holds the B*S centre rows first and the half-difference rows from row
+// `row0` on.
+szo_status launch_flash_attention_pair_bf16(const void* q, const void* k, const void* v, void* o, int64_t row0, int B,
+                                            int S, int H, int Hkv, int hd, cudaStream_t st) {
+  SZO_REQUIRE(hd == 64 || hd == 128, SZO_ERR_UNSUPPORTED, "head dimension must be 64 or 128");
+  const float scale = 1.0f / sqrtf(static_cast<float>(hd));
+  const float scale_log2e = 1.4426950408889634f * scale;
+  dim3 grid(static_cast<unsigned>(ceil_div(S, kQT)), H, B);
+  const size_t smem = static_cast<size_t>(2 * kQT + 8 * kKT2) * (hd + 8) * 2;
+  auto* qb = static_cast<const __nv_bfloat16*>(q);
+  auto* kb = static_cast<const __nv_bfloat16*>(k);
+  auto* vb = static_cast<const __nv_bfloat16*>(v);
+  auto* ob = static_cast<__nv_bfloat16*>(o);
+  // (the attribute is per device; setting it before every launch costs a host call, no device work)
+  if (hd == 64) {
+    SZO_CHECK_CUDA(cudaFuncSetAttribute(flash_attn_pair_bf16_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(smem)));
+    flash_attn_pair_bf16_kernel<64><<<grid, 128, smem, st>>>(qb, kb, vb, ob, row0, S, H, Hkv, scale, scale_log2e);
+  } else {
+    SZO_CHECK_CUDA(cudaFuncSetAttribute(flash_attn_pair_bf16_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(smem)));
+    flash_attn_pair_bf16_kernel<128><<<grid, 128, smem, st>>>(qb, kb, vb, ob, row0, S, H, Hkv, scale, scale_log2e);
+  }
+  count_launch();
+  SZO_CHECK_LAUNCH("flash_attn_pair_bf16_kernel");
   return SZO_OK;
 }
 

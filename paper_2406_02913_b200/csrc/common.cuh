@@ -75,4 +75,9 @@ szo_status launch_sparse_axpy_kept(const float* S_in, float* S_out, const float*
 szo_status launch_flash_attention_bf16(const void* q, const void* k, const void* v, void* o, int B, int S, int H,
                                        int Hkv, int hd, cudaStream_t st);
 
+// The same for the paired form of a ZO step's two forwards: centre rows first, half-difference rows
+// from row `row0` on in every buffer.
+szo_status launch_flash_attention_pair_bf16(const void* q, const void* k, const void* v, void* o, int64_t row0, int B,
+                                            int S, int H, int Hkv, int hd, cudaStream_t st);
+
 }  // namespace szo

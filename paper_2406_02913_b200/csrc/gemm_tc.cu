@@ -317,6 +317,32 @@ __global__ void scatter_add_bf16_kernel(const MatArgs a) {
   *el = __float2bfloat16_rn(__bfloat162float(base) + S[e]);
 }
 
+// xT[c][t] = x[t][c] for t < M, c < K (bf16; x row-major [M][K], xT row stride ldT >= M): the centre
+// activations by column, for the sparse product of the paired form.  64 x 64 tiles through shared
+// memory, 16-byte loads and stores.
+__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* __restrict__ x, int64_t M, int64_t K,
+                                                            __nv_bfloat16* __restrict__ xT, int64_t ldT) {
+  __shared__ __align__(16) __nv_bfloat16 tile[64][72];
+  const int64_t t0 = static_cast<int64_t>(blockIdx.x) * 64, c0 = static_cast<int64_t>(blockIdx.y) * 64;
+  const int r = threadIdx.x >> 3, ch = threadIdx.x & 7;          // 32 rows x 8 chunks of 8 elements per pass
+#pragma unroll
+  for (int p = 0; p < 2; ++p) {
+    const int tr = r + p * 32;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (t0 + tr < M) v = *reinterpret_cast<const uint4*>(x + (t0 + tr) * K + c0 + ch * 8);   // K % 64 == 0
+    *reinterpret_cast<uint4*>(&tile[tr][ch * 8]) = v;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int p = 0; p < 2; ++p) {
+    const int cr = r + p * 32;                                    // column of x = row of xT
+    __nv_bfloat16 o[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) o[j] = tile[ch * 8 + j][cr];
+    *reinterpret_cast<uint4*>(xT + (c0 + cr) * ldT + t0 + ch * 8) = *reinterpret_cast<const uint4*>(o);   // ldT % 64 == 0
+  }
+}
+
 // SZO_LINEAR_MATERIALISE=0 / 1 switches the form off / on for every M (A/B measurement)
 int materialise_override() {
   static const int v = [] {
@@ -419,9 +445,15 @@ szo_status tc_resident_init(const szo_linear* const* plans, int n, __nv_bfloat16
 szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, const void* x, int64_t M,
                                       const float* const* S_pert, void* const* y, int y_dtype, void* ws,
                                       size_t ws_bytes, cudaStream_t st, const float* const* S_second,
-                                      __nv_bfloat16* W_resident, __nv_bfloat16* saved_resident, bool relu) {
+                                      __nv_bfloat16* W_resident, __nv_bfloat16* saved_resident, bool relu,
+                                      const PairedArgs* paired) {
   const szo_linear* p0 = plans[0];
   const bool resident = W_resident != nullptr;
+  SZO_REQUIRE(paired == nullptr || (S_second == nullptr && !relu), SZO_ERR_INVALID_ARG,
+              "the paired form takes one set of sparse values and no ReLU epilogue");
+  // paired form: M centre rows, then M half-difference rows from row Mp (a multiple of 256) on
+  const int64_t Mp = paired != nullptr ? static_cast<int64_t>(round_up(static_cast<size_t>(M), 256)) : 0;
+  const int64_t M_rows = paired != nullptr ? Mp + M : M;
   const TcPlan* t = static_cast<const TcPlan*>(p0->tc);
   SZO_REQUIRE(t != nullptr, SZO_ERR_INVALID_ARG, "plan has no tensor-core data");
   SZO_REQUIRE(M < (int64_t(1) << 31), SZO_ERR_SHAPE, "M too large");
@@ -455,7 +487,18 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
     nnz += p->nnz;
     row0 += p->Npad;
   }
-  if (!resident) {
+  if (!resident && p0->G == 0) {
+    // dense bf16 plans outside a model (which keeps them resident): copy the frozen weight
+    int64_t r0 = 0;
+    for (int i = 0; i < n; ++i) {
+      const szo_linear* p = plans[i];
+      SZO_CHECK_CUDA(cudaMemcpyAsync(W + r0 * p->K, p->codes, static_cast<size_t>(p->N) * p->K * sizeof(__nv_bfloat16),
+                                     cudaMemcpyDeviceToDevice, st));
+      if (p->Npad > p->N)
+        SZO_CHECK_CUDA(cudaMemsetAsync(W + (r0 + p->N) * p->K, 0, static_cast<size_t>(p->Npad - p->N) * p->K * sizeof(__nv_bfloat16), st));
+      r0 += p->Npad;
+    }
+  } else if (!resident) {
     const unsigned blocks = static_cast<unsigned>(ceil_div(words, 256));
     if (p0->G < 0) materialise_kernel<2><<<blocks, 256, 0, st>>>(a);
     else if (p0->sz_dtype == SZO_BF16) materialise_kernel<1><<<blocks, 256, 0, st>>>(a);
@@ -466,14 +509,32 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
   CUtensorMap mw;
   SZO_TRY(make_map(&mw, W, rows, p0->K, kBM));
   TcParams P{};
-  P.M = M; P.K = p0->K; P.G = 0; P.nkb = nkb;
+  P.M = M_rows; P.K = p0->K; P.G = 0; P.nkb = nkb;
   P.relu = relu ? 1 : 0;
-  P.m_tiles = ceil_div(M, 256);
+  P.m_tiles = ceil_div(M_rows, 256);
   P.nsub = n;
+  if (paired != nullptr) {
+    SZO_REQUIRE(paired->xT != nullptr && paired->eps != 0.f, SZO_ERR_INVALID_ARG, "paired form: xT scratch and eps needed");
+    P.pair_eps = paired->eps;
+    P.pair_row0 = Mp;
+    P.xT = paired->xT;
+    P.ldT = Mp;
+    P.mt_c = static_cast<int>(Mp / 256);
+    P.mt_d = static_cast<int>(ceil_div(M, 256));
+    dim3 grid(static_cast<unsigned>(Mp / 64), static_cast<unsigned>(p0->K / 64));
+    transpose_bf16_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), M, p0->K, paired->xT, Mp);
+    count_launch();
+    SZO_CHECK_LAUNCH("transpose_bf16_kernel");
+  }
   int64_t n_tiles = 0;
   for (int i = 0; i < n; ++i) {
     const szo_linear* p = plans[i];
     TcSub& sb = P.sub[i];
+    if (paired != nullptr && p->nnz > 0) {
+      sb.row_ptr = p->row_ptr;
+      sb.ent_col = p->ent_col;
+      sb.zc = paired->z[i];
+    }
     sb.codes = nullptr;
     sb.sz = nullptr;
     sb.bucket_ptr = nullptr;
@@ -512,7 +573,7 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
       count_launch();
     }
     CUtensorMap mx;
-    SZO_TRY(make_map(&mx, static_cast<const __nv_bfloat16*>(x) + static_cast<int64_t>(set) * M * p0->K, M, p0->K, 128));
+    SZO_TRY(make_map(&mx, static_cast<const __nv_bfloat16*>(x) + static_cast<int64_t>(set) * M * p0->K, M_rows, p0->K, 128));
     for (int i = 0; i < n; ++i)
       P.sub[i].y = static_cast<unsigned char*>(y[i]) + static_cast<size_t>(set) * M * plans[i]->N * y_elt;
     SZO_TRY(launch_pair_kernel(false, false, mx, mw, P, sc.n_pairs, st));

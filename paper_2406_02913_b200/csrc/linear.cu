@@ -568,6 +568,36 @@ szo_status szo_linear_fwd(const szo_linear_t* p, const void* x, szo_dtype x_dtyp
   return linear_fwd_impl(p, x, x_dtype, M, S_pert, nullptr, y, y_dtype, mode, workspace, workspace_bytes, st);
 }
 
+size_t szo_linear_paired_workspace_bytes(const szo_linear_t* p, int64_t M) {
+  if (!p || M <= 0 || p->tc == nullptr) return 0;
+  const szo_linear* pp = p;
+  return tc_materialised_ws_bytes(&pp, 1, M) + round_up(static_cast<size_t>(M), 256) * p->K * sizeof(__nv_bfloat16);
+}
+
+szo_status szo_linear_fwd_paired(const szo_linear_t* p, const void* x, int64_t M, const float* S, const float* z,
+                                 float eps, void* y, szo_dtype y_dtype, void* workspace, size_t workspace_bytes,
+                                 void* stream) {
+  SZO_REQUIRE(p != nullptr, SZO_ERR_INVALID_ARG, "plan is NULL");
+  SZO_REQUIRE(M >= 0 && M < (int64_t(1) << 30), SZO_ERR_SHAPE, "bad M");
+  SZO_REQUIRE(y_dtype == SZO_BF16 || y_dtype == SZO_F32, SZO_ERR_UNSUPPORTED, "y must be bf16 or f32");
+  SZO_REQUIRE(eps != 0.f, SZO_ERR_INVALID_ARG, "eps == 0");
+  if (M == 0) return SZO_OK;
+  SZO_REQUIRE(x && y, SZO_ERR_INVALID_ARG, "x or y is NULL");
+  SZO_REQUIRE(p->nnz == 0 || (S && z), SZO_ERR_INVALID_ARG, "S or z is NULL");
+  SZO_REQUIRE(aligned16(x) && aligned16(y) && aligned16(workspace), SZO_ERR_ALIGNMENT,
+              "x, y and workspace must be 16-byte aligned");
+  SZO_REQUIRE(((reinterpret_cast<uintptr_t>(S) | reinterpret_cast<uintptr_t>(z)) & 3u) == 0, SZO_ERR_ALIGNMENT,
+              "S and z must be 4-byte aligned");
+  const size_t need = szo_linear_paired_workspace_bytes(p, M);
+  SZO_REQUIRE(workspace != nullptr && workspace_bytes >= need, SZO_ERR_WORKSPACE,
+              "the paired form needs a workspace of %zu bytes", need);
+  const size_t xt_bytes = round_up(static_cast<size_t>(M), 256) * p->K * sizeof(__nv_bfloat16);
+  const szo_linear* pp = p;
+  const PairedArgs pa{&z, eps, reinterpret_cast<__nv_bfloat16*>(static_cast<unsigned char*>(workspace) + (need - xt_bytes))};
+  return linear_fwd_tc_materialised(&pp, 1, x, M, &S, &y, y_dtype, workspace, need - xt_bytes,
+                                    static_cast<cudaStream_t>(stream), nullptr, nullptr, nullptr, false, &pa);
+}
+
 void szo_linear_destroy(szo_linear_t* p) { free_plan(p); }
 
 }  // extern "C"

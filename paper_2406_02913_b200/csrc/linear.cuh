@@ -68,11 +68,20 @@ size_t tc_tail_ws_bound();   // enough for any M and any group
 // mode of the kernel runs.  Chosen for int4 plans when M is large (tc_use_materialised).
 bool tc_use_materialised(const szo_linear* p, int64_t M, bool two_sets = false);   // two_sets: one weight pass for two forwards
 size_t tc_materialised_ws_bytes(const szo_linear* const* plans, int n, int64_t M);
+// Paired form of a ZO step's two forwards (see tc::TcParams): x and every y[i] hold the M centre rows
+// first and the M half-difference rows from row round_up(M, 256) on; S_pert are the unperturbed sparse
+// values; z[i] the z of plans[i]'s entries; xT scratch of K * round_up(M, 256) bf16.
+struct PairedArgs {
+  const float* const* z;
+  float eps;
+  __nv_bfloat16* xT;
+};
 szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, const void* x, int64_t M,
                                       const float* const* S_pert, void* const* y, int y_dtype, void* ws,
                                       size_t ws_bytes, cudaStream_t st, const float* const* S_second = nullptr,
                                       __nv_bfloat16* W_resident = nullptr, __nv_bfloat16* saved_resident = nullptr,
-                                      bool relu = false);   // relu: y = max(y, 0) applied in the epilogue
+                                      bool relu = false,    // relu: y = max(y, 0) applied in the epilogue
+                                      const PairedArgs* paired = nullptr);
 // Resident form for dense bf16 plans (G == 0): W_resident [sum Npad, K] and saved_resident [sum nnz]
 // are filled once by tc_resident_init and passed to linear_fwd_tc_materialised, which then skips the
 // weight pass and writes every masked entry as RN_bf16(saved + S); ws is only the K-split scratch.

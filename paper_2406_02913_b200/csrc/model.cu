@@ -337,6 +337,280 @@ cls2_kernel(const T* __restrict__ a_last, const __nv_bfloat16* __restrict__ lm_h
   }
 }
 
+
+// ------------------------------------------------------------------------------ paired form
+// The two forwards of a ZO step (Definition 1: the loss at w + eps zbar and at w - eps zbar, same
+// batch) carried through the network as centre c = (x+ + x-)/2 and half-difference d = (x+ - x-)/2
+// instead of x+ and x-.  The perturbation changes an activation by less than a bf16 ulp; stored as
+// x+ and x-, each rounded on its own, the difference f+ - f- (all that the projected gradient uses)
+// drowns in rounding, whereas d has its own exponent and keeps 8 significant bits whatever its size.
+// Every kernel below evaluates its function at c + d and c - d in fp32 and returns centre and
+// half-difference of the two results, with the half-difference formed from expressions that do not
+// cancel.  Buffers hold the centre rows first and the half-difference rows from row `row0` on.
+
+// sinh(a) without cancellation for small |a|
+__device__ __forceinline__ float sinh_stable(float a) {
+  const float a2 = a * a;
+  if (a2 < 0.25f) return a * (1.0f + a2 * (1.0f / 6.0f + a2 * (1.0f / 120.0f + a2 * (1.0f / 5040.0f + a2 * (1.0f / 362880.0f)))));
+  const float u = __expf(a);
+  return 0.5f * (u - 1.0f / u);
+}
+
+// Block-wide sums of two values at once (same tree as block_sum).
+__device__ __forceinline__ float2 block_sum2(float a, float b, float2* scratch) {
+#pragma unroll
+  for (int o = 16; o; o >>= 1) {
+    a += __shfl_xor_sync(0xffffffffu, a, o);
+    b += __shfl_xor_sync(0xffffffffu, b, o);
+  }
+  const int w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) scratch[w] = make_float2(a, b);
+  __syncthreads();
+  float2 t = make_float2(0.f, 0.f);
+  for (int i = 0; i < nw; ++i) {
+    t.x += scratch[i].x;
+    t.y += scratch[i].y;
+  }
+  return t;
+}
+
+// add_norm_kernel in the paired form.  Residual add of both parts (linear), then with
+// x+- = c +- d:  mean(x+-^2) = mean(c^2 + d^2) +- 2 mean(c d) = sc +- sx, a+- = sqrt(sc +- sx + eps),
+// r+- = 1/a+-:  rc = (r+ + r-)/2,  rd = (r+ - r-)/2 = -sx / ((a+ + a-) a+ a-);
+// out_c = (c rc + d rd) gamma (+ beta),  out_d = (c rd + d rc) gamma.  LayerNorm: the same on c - mean(c),
+// d - mean(d).  One block per token; h_d = h + row0 * d_model etc.
+template <typename T, typename TO = T>
+__global__ void __launch_bounds__(256)
+add_norm_pair_kernel(float* __restrict__ h, const T* __restrict__ y, int64_t row0, const float* __restrict__ gamma,
+                     const float* __restrict__ beta, int d, float eps, bool layer_norm, int64_t row_stride,
+                     int64_t row_offset, TO* __restrict__ out, int64_t out_row0) {
+  constexpr int kMaxV = 8;
+  __shared__ float2 scratch[32];
+  const int64_t m = static_cast<int64_t>(blockIdx.x) * row_stride + row_offset;
+  float* xc = h + m * d;
+  float* xd = h + (row0 + m) * d;
+  const int nv = d >> 2;
+  float4 vc[kMaxV], vd[kMaxV];
+  float s1 = 0.f, s2 = 0.f;
+  auto add4 = [](float4& v, const T* yp) {
+    if constexpr (sizeof(T) == 2) {
+      const uint2 raw = *reinterpret_cast<const uint2*>(yp);
+      v.x += __uint_as_float(raw.x << 16);
+      v.y += __uint_as_float(raw.x & 0xFFFF0000u);
+      v.z += __uint_as_float(raw.y << 16);
+      v.w += __uint_as_float(raw.y & 0xFFFF0000u);
+    } else {
+      v.x += to_f32<T>(yp[0]);
+      v.y += to_f32<T>(yp[1]);
+      v.z += to_f32<T>(yp[2]);
+      v.w += to_f32<T>(yp[3]);
+    }
+  };
+#pragma unroll
+  for (int i = 0; i < kMaxV; ++i) {
+    const int c = threadIdx.x + i * 256;
+    vc[i] = vd[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (c < nv) {
+      vc[i] = reinterpret_cast<const float4*>(xc)[c];
+      vd[i] = reinterpret_cast<const float4*>(xd)[c];
+      if (y != nullptr) {
+        add4(vc[i], y + m * d + c * 4);
+        add4(vd[i], y + (row0 + m) * d + c * 4);
+        if (row_stride == 1) {
+          reinterpret_cast<float4*>(xc)[c] = vc[i];
+          reinterpret_cast<float4*>(xd)[c] = vd[i];
+        }
+      }
+      s1 += (vc[i].x + vc[i].y) + (vc[i].z + vc[i].w);
+      s2 += (vd[i].x + vd[i].y) + (vd[i].z + vd[i].w);
+    }
+  }
+  float mc = 0.f, md = 0.f;
+  if (layer_norm) {
+    const float2 mu = block_sum2(s1, s2, scratch);
+    mc = mu.x / d;
+    md = mu.y / d;
+  }
+  float qc = 0.f, qx = 0.f;
+#pragma unroll
+  for (int i = 0; i < kMaxV; ++i) {
+    if (threadIdx.x + i * 256 < nv) {
+      const float c0 = vc[i].x - mc, c1 = vc[i].y - mc, c2 = vc[i].z - mc, c3 = vc[i].w - mc;
+      const float d0 = vd[i].x - md, d1 = vd[i].y - md, d2 = vd[i].z - md, d3 = vd[i].w - md;
+      qc += ((c0 * c0 + d0 * d0) + (c1 * c1 + d1 * d1)) + ((c2 * c2 + d2 * d2) + (c3 * c3 + d3 * d3));
+      qx += (c0 * d0 + c1 * d1) + (c2 * d2 + c3 * d3);
+    }
+  }
+  const float2 q = block_sum2(qc, qx, scratch);
+  const float sc = q.x / d, sx = 2.0f * q.y / d;
+  const float ap = sqrtf(sc + sx + eps), am = sqrtf(sc - sx + eps);
+  const float rc = 0.5f * (1.0f / ap + 1.0f / am);
+  const float rd = -sx / ((ap + am) * ap * am);
+  TO* oc = out + static_cast<int64_t>(blockIdx.x) * d;
+  TO* od = out + (out_row0 + static_cast<int64_t>(blockIdx.x)) * d;
+  auto put4 = [](TO* op, float o0, float o1, float o2, float o3) {
+    if constexpr (sizeof(TO) == 2) {
+      const __nv_bfloat162 lo = __floats2bfloat162_rn(o0, o1), hi = __floats2bfloat162_rn(o2, o3);
+      uint2 pk;
+      pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+      pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+      *reinterpret_cast<uint2*>(op) = pk;
+    } else {
+      *reinterpret_cast<float4*>(op) = make_float4(o0, o1, o2, o3);
+    }
+  };
+#pragma unroll
+  for (int i = 0; i < kMaxV; ++i) {
+    const int c = threadIdx.x + i * 256;
+    if (c < nv) {
+      const float4 g = reinterpret_cast<const float4*>(gamma)[c];
+      float4 bt = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (beta) bt = reinterpret_cast<const float4*>(beta)[c];
+      const float c0 = vc[i].x - mc, c1 = vc[i].y - mc, c2 = vc[i].z - mc, c3 = vc[i].w - mc;
+      const float d0 = vd[i].x - md, d1 = vd[i].y - md, d2 = vd[i].z - md, d3 = vd[i].w - md;
+      put4(oc + c * 4, (c0 * rc + d0 * rd) * g.x + bt.x, (c1 * rc + d1 * rd) * g.y + bt.y,
+           (c2 * rc + d2 * rd) * g.z + bt.z, (c3 * rc + d3 * rd) * g.w + bt.w);
+      put4(od + c * 4, (c0 * rd + d0 * rc) * g.x, (c1 * rd + d1 * rc) * g.y, (c2 * rd + d2 * rc) * g.z,
+           (c3 * rd + d3 * rc) * g.w);
+    }
+  }
+}
+
+// silu(g) * u in the paired form, in place on gate.  With g+- = gc +- gd and s(x) = 1/(1+exp(-x)):
+// s+ - s- = 2 exp(-gc) sinh(gd) s+ s-  (for gc < 0 written with 1 - s, so that nothing overflows);
+// silu: tc = gc sc + gd sd, td = gc sd + gd sc;  out_c = tc uc + td ud,  out_d = tc ud + td uc.
+template <typename T>
+__global__ void silu_mul_pair_kernel(T* __restrict__ gate, const T* __restrict__ up, int64_t n, int64_t off_d) {
+  constexpr int kN = Vec16<T>::kN;
+  const int64_t i = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) * kN;
+  if (i >= n) return;
+  const Vec16<T> gc = load16(gate + i), gd = load16(gate + off_d + i), uc = load16(up + i), ud = load16(up + off_d + i);
+  Vec16<T> rc, rd;
+#pragma unroll
+  for (int j = 0; j < kN; ++j) {
+    const float c = to_f32<T>(gc.v[j]), d = to_f32<T>(gd.v[j]);
+    const float sp = 1.0f / (1.0f + __expf(-(c + d))), sm = 1.0f / (1.0f + __expf(-(c - d)));
+    const float q = __expf(-fabsf(c)) * sinh_stable(d);
+    const float sd = c >= 0.f ? q * sp * sm : q * (1.0f - sp) * (1.0f - sm);
+    const float sc = 0.5f * (sp + sm);
+    const float tc = c * sc + d * sd, td = c * sd + d * sc;
+    const float a = to_f32<T>(uc.v[j]), b = to_f32<T>(ud.v[j]);
+    rc.v[j] = from_f32<T>(tc * a + td * b);
+    rd.v[j] = from_f32<T>(tc * b + td * a);
+  }
+  store16(gate + i, rc);
+  store16(gate + off_d + i, rd);
+}
+
+// max(x, 0) in the paired form, in place.
+template <typename T>
+__global__ void relu_pair_kernel(T* __restrict__ x, int64_t n, int64_t off_d) {
+  constexpr int kN = Vec16<T>::kN;
+  const int64_t i = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) * kN;
+  if (i >= n) return;
+  Vec16<T> c = load16(x + i), d = load16(x + off_d + i);
+#pragma unroll
+  for (int j = 0; j < kN; ++j) {
+    const float a = to_f32<T>(c.v[j]), b = to_f32<T>(d.v[j]);
+    const float p = a + b, q = a - b;
+    if (p > 0.f && q > 0.f) continue;                   // both sides pass: (a, b) unchanged
+    const float rp = fmaxf(p, 0.f), rq = fmaxf(q, 0.f); // at least one side is clamped: no cancellation to fear
+    c.v[j] = from_f32<T>(0.5f * (rp + rq));
+    d.v[j] = from_f32<T>(0.5f * (rp - rq));
+  }
+  store16(x + i, c);
+  store16(x + off_d + i, d);
+}
+
+// ce_rows_kernel in the paired form: logits lc (row m) and ld (row row0 + m).  With reference value R >=
+// every lc + |ld|:  P = sum exp(lc - R) cosh(ld),  D = sum exp(lc - R) sinh(ld), so that
+// logsumexp(lc +- ld) = R + log(P +- D).  Centre and half-difference of the two cross-entropies:
+//   cc = R + (log(P + D) + log(P - D)) / 2 - lc[t],   cd = log1p(2 D / (P - D)) / 2 - ld[t];
+// loss_plus[m] = cc + cd, loss_minus[m] = cc - cd in fp64.
+__global__ void __launch_bounds__(256)
+ce_rows_pair_kernel(const float* __restrict__ logits, int64_t row0, const int32_t* __restrict__ tok, int S, int V,
+                    double* __restrict__ loss_plus, double* __restrict__ loss_minus) {
+  __shared__ float2 scratch2[32];
+  __shared__ float scratch[32];
+  const int64_t m = blockIdx.x;
+  if ((m % S) == S - 1) {
+    if (threadIdx.x == 0) {
+      loss_plus[m] = 0.0;
+      loss_minus[m] = 0.0;
+    }
+    return;
+  }
+  const float* lc = logits + m * V;
+  const float* ld = logits + (row0 + m) * V;
+  float R = -INFINITY, Ps = 0.f, Ds = 0.f;
+  for (int c = threadIdx.x; c < V; c += blockDim.x) {
+    const float a = lc[c], b = ld[c];
+    const float ref = a + fabsf(b);
+    if (ref > R) {
+      const float sc = __expf(R - ref);     // exp(-inf) = 0 on the first element
+      Ps *= sc;
+      Ds *= sc;
+      R = ref;
+    }
+    const float e = __expf(a - R), u = __expf(b);
+    Ps += e * 0.5f * (u + 1.0f / u);
+    Ds += e * sinh_stable(b);
+  }
+  float bm = R;
+#pragma unroll
+  for (int o = 16; o; o >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, o));
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = bm;
+  __syncthreads();
+  for (int i = 0; i < (blockDim.x >> 5); ++i) bm = fmaxf(bm, scratch[i]);
+  const float sc = (R == -INFINITY) ? 0.f : __expf(R - bm);
+  const float2 t = block_sum2(Ps * sc, Ds * sc, scratch2);
+  if (threadIdx.x == 0) {
+    int32_t tg = tok[m + 1];
+    tg = tg < 0 ? 0 : (tg >= V ? V - 1 : tg);
+    const double P = t.x, D = t.y;
+    const double cc = static_cast<double>(bm) + 0.5 * (log(P + D) + log(P - D)) - static_cast<double>(lc[tg]);
+    const double cd = 0.5 * log1p(2.0 * D / (P - D)) - static_cast<double>(ld[tg]);
+    loss_plus[m] = cc + cd;
+    loss_minus[m] = cc - cd;
+  }
+}
+
+// cls2_kernel in the paired form: a_last holds the B centre states, then the B half-differences.
+__global__ void __launch_bounds__(256)
+cls2_pair_kernel(const float* __restrict__ a_last, int B, const __nv_bfloat16* __restrict__ lm_head,
+                 const int32_t* __restrict__ cand, const int32_t* __restrict__ labels, int d, int V,
+                 double* __restrict__ loss_plus, double* __restrict__ loss_minus) {
+  __shared__ float2 scratch[32];
+  const int b = blockIdx.x;
+  const float* ac = a_last + static_cast<int64_t>(b) * d;
+  const float* ad = a_last + static_cast<int64_t>(B + b) * d;
+  int32_t c0 = cand[0], c1 = cand[1];
+  c0 = c0 < 0 ? 0 : (c0 >= V ? V - 1 : c0);
+  c1 = c1 < 0 ? 0 : (c1 >= V ? V - 1 : c1);
+  const __nv_bfloat16* e0 = lm_head + static_cast<int64_t>(c0) * d;
+  const __nv_bfloat16* e1 = lm_head + static_cast<int64_t>(c1) * d;
+  float s0c = 0.f, s1c = 0.f, s0d = 0.f, s1d = 0.f;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    const float w0 = __bfloat162float(e0[c]), w1 = __bfloat162float(e1[c]);
+    s0c = fmaf(ac[c], w0, s0c);
+    s1c = fmaf(ac[c], w1, s1c);
+    s0d = fmaf(ad[c], w0, s0d);
+    s1d = fmaf(ad[c], w1, s1d);
+  }
+  const float2 tc = block_sum2(s0c, s1c, scratch);
+  const float2 td = block_sum2(s0d, s1d, scratch);
+  if (threadIdx.x == 0) {
+    for (int sgn = 0; sgn < 2; ++sgn) {
+      const double f = sgn ? -1.0 : 1.0;
+      const double l0 = tc.x + f * td.x, l1 = tc.y + f * td.y, mx = l0 > l1 ? l0 : l1;
+      const double lse = mx + log(exp(l0 - mx) + exp(l1 - mx));
+      (sgn ? loss_minus : loss_plus)[b] = lse - (labels[b] ? l1 : l0);
+    }
+  }
+}
+
 // *out = (sum of v[0..n)) / denom, fixed order, fp64.
 __global__ void __launch_bounds__(1024) mean_f64_kernel(const double* __restrict__ v, int64_t n, double denom,
                                                         double* __restrict__ out) {
@@ -383,6 +657,8 @@ struct szo_model {
   float* zkept = nullptr;       // [k_total] z of the current step, kept by the first perturb pass
   float *Splus = nullptr, *Sminus = nullptr;   // [k_total] the two perturbed copies of S (two forwards side by side)
   bool dual_rows = false;       // the activation buffers hold 2 * Mmax rows
+  bool paired = false;          // SZO_MODE_PAIRED: a step's two forwards as centre and half-difference
+  __nv_bfloat16* xT = nullptr;  // paired form: the centre activations of the current linear by column
   // dense bf16 weights (group == 0) with many tokens: every launch group keeps its effective weight
   // resident (a private copy of the frozen matrices, masked entries rewritten per forward)
   bool resident = false;
@@ -449,7 +725,9 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
   T *a = static_cast<T*>(m->a), *q = static_cast<T*>(m->q), *k = static_cast<T*>(m->k), *v = static_cast<T*>(m->v),
     *o = static_cast<T*>(m->o), *y = static_cast<T*>(m->y), *gate = static_cast<T*>(m->gate),
     *up = static_cast<T*>(m->up);
-  const bool pregather = c.linear_mode != SZO_MODE_FP32_VALIDATE && c.linear_mode != SZO_MODE_SPMM && m->k_total > 0;
+  // a lone forward of a model in the paired mode (szo_model_loss) is a SparseAdd forward
+  const int32_t lmode = c.linear_mode == SZO_MODE_PAIRED ? SZO_MODE_SPARSE_ADD : c.linear_mode;
+  const bool pregather = lmode != SZO_MODE_FP32_VALIDATE && lmode != SZO_MODE_SPMM && m->k_total > 0;
   auto lin_single = [&](int layer, int j, const void* x, void* out) -> szo_status {
     const int t = layer * m->n_lin + j;
     if (m->timing) {
@@ -461,7 +739,7 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
       SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used], st));
     }
     const szo_status rc = linear_fwd_impl(m->plans[t], x, act, M, Sv + m->offsets[t],
-                                          pregather ? m->recs + m->offsets[t] : nullptr, out, act, c.linear_mode,
+                                          pregather ? m->recs + m->offsets[t] : nullptr, out, act, lmode,
                                           m->ws, m->ws_bytes, st);
     if (m->timing) {
       SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used + 1], st));
@@ -578,7 +856,7 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
     add_norm_kernel<T><<<static_cast<unsigned>(Mr), 256, 0, st>>>(m->h, pending, m->top.final_norm_g,
                                                                  m->top.final_norm_b, d, c.norm_eps, opt, 1, 0, a);
     count_launch();
-    const int mode = c.linear_mode == SZO_MODE_FP32_VALIDATE ? SZO_MODE_FP32_VALIDATE : SZO_MODE_SPARSE_ADD;
+    const int mode = lmode == SZO_MODE_FP32_VALIDATE ? SZO_MODE_FP32_VALIDATE : SZO_MODE_SPARSE_ADD;
     SZO_TRY(szo_linear_fwd(m->lm_head_plan, a, static_cast<szo_dtype>(act), Mr, nullptr, m->logits, SZO_F32, mode,
                            m->ws, m->ws_bytes, st));
     for (int set = 0; set < nsets; ++set) {
@@ -605,6 +883,122 @@ szo_status run_loss_t(szo_model* m, const int32_t* tokens, const int32_t* labels
   return SZO_OK;
 }
 
+
+// Both forwards of a ZO step in the paired form (see the kernels above): bf16 activations, dense
+// mode of the tensor-core kernel on W = RN_bf16(Dequantize(Q) + S) (written per launch group, or
+// resident for dense bf16 weights), eps * xc Zbar^T added to the half-difference rows in the
+// epilogue.  Rows [0, M) of every activation buffer are the centre, rows [Mp, Mp + M) the
+// half-difference, Mp = M rounded up to 256 (rows in between are never read as results).
+szo_status run_loss_paired(szo_model* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand, int B, int S,
+                           const float* Sv, const float* z, float eps, double* loss_plus_dev, double* loss_minus_dev,
+                           cudaStream_t st) {
+  using T = __nv_bfloat16;
+  const szo_model_config& c = m->cfg;
+  const int64_t M = static_cast<int64_t>(B) * S;
+  const int64_t Mp = static_cast<int64_t>(round_up(static_cast<size_t>(M), 256));
+  const int64_t Mr = Mp + M;
+  const int d = c.d_model, H = c.n_heads, Hkv = c.n_kv_heads, hd = d / H, ff = c.d_ff;
+  const int64_t dkv = static_cast<int64_t>(Hkv) * hd;
+  const bool opt = c.arch == 1;
+  T *a = static_cast<T*>(m->a), *q = static_cast<T*>(m->q), *k = static_cast<T*>(m->k), *v = static_cast<T*>(m->v),
+    *o = static_cast<T*>(m->o), *y = static_cast<T*>(m->y), *gate = static_cast<T*>(m->gate), *up = static_cast<T*>(m->up);
+  auto lin_group = [&](int layer, int j0, int n, const void* x, void* const* outs) -> szo_status {
+    const int t0 = layer * m->n_lin + j0;
+    const szo_linear* plans[3];
+    const float* sv[3];
+    const float* zz[3];
+    for (int i = 0; i < n; ++i) {
+      plans[i] = m->plans[t0 + i];
+      sv[i] = Sv + m->offsets[t0 + i];
+      zz[i] = z + m->offsets[t0 + i];
+    }
+    if (m->timing) {
+      while (m->events.size() < m->events_used + 2) {
+        cudaEvent_t e;
+        SZO_CHECK_CUDA(cudaEventCreate(&e));
+        m->events.push_back(e);
+      }
+      SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used], st));
+    }
+    const PairedArgs pa{zz, eps, m->xT};
+    const bool res = m->resident;
+    const szo_status rc = linear_fwd_tc_materialised(plans, n, x, M, sv, outs, SZO_BF16, m->ws, m->ws_bytes, st, nullptr,
+                                                     res ? m->res_W[t0] : nullptr, res ? m->res_saved[t0] : nullptr,
+                                                     false, &pa);
+    if (m->timing) {
+      SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used + 1], st));
+      m->events_used += 2;
+    }
+    return rc;
+  };
+  auto lin = [&](int layer, int j, const void* x, void* out) -> szo_status {
+    void* const outs[1] = {out};
+    return lin_group(layer, j, 1, x, outs);
+  };
+  embed_kernel<<<static_cast<unsigned>(M), 128, 0, st>>>(tokens, static_cast<const __nv_bfloat16*>(m->top.embed),
+                                                        static_cast<const __nv_bfloat16*>(m->top.pos), S, d, c.vocab, m->h);
+  SZO_CHECK_CUDA(cudaMemsetAsync(m->h + Mp * d, 0, static_cast<size_t>(M) * d * sizeof(float), st));   // both forwards embed alike
+  count_launch();
+  const T* pending = nullptr;
+  for (int l = 0; l < c.n_layers; ++l) {
+    const szo_layer_weights& L = m->layers[l];
+    add_norm_pair_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, pending, Mp, L.attn_norm_g, L.attn_norm_b, d,
+                                                                     c.norm_eps, opt, 1, 0, a, Mp);
+    count_launch();
+    {
+      void* const qkv[3] = {q, k, v};
+      SZO_TRY(lin_group(l, 0, 3, a, qkv));
+    }
+    if (!opt) {        // the rotation is linear: the same kernel on both parts
+      const int64_t n_vec = M * (H + Hkv) * ((hd / 2) / Vec16<T>::kN);
+      rope_kernel<T><<<blocks_for(n_vec, 256), 256, 0, st>>>(q, k, m->rope_tab, M, S, H, Hkv, hd);
+      rope_kernel<T><<<blocks_for(n_vec, 256), 256, 0, st>>>(q + Mp * d, k + Mp * dkv, m->rope_tab, M, S, H, Hkv, hd);
+      count_launch(2);
+    }
+    SZO_TRY(launch_flash_attention_pair_bf16(q, k, v, o, Mp, B, S, H, Hkv, hd, st));
+    SZO_TRY(lin(l, 3, o, y));
+    add_norm_pair_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, y, Mp, L.mlp_norm_g, L.mlp_norm_b, d, c.norm_eps,
+                                                                     opt, 1, 0, a, Mp);
+    count_launch();
+    if (!opt) {
+      void* const gu[2] = {gate, up};
+      SZO_TRY(lin_group(l, 4, 2, a, gu));
+      silu_mul_pair_kernel<T><<<blocks_for(M * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, up, M * ff, Mp * ff);
+      count_launch();
+      SZO_TRY(lin(l, 6, gate, y));
+    } else {
+      SZO_TRY(lin(l, 4, a, gate));
+      relu_pair_kernel<T><<<blocks_for(M * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, M * ff, Mp * ff);
+      count_launch();
+      SZO_TRY(lin(l, 5, gate, y));
+    }
+    pending = y;
+  }
+  if (c.loss_kind == 0) {
+    add_norm_pair_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, pending, Mp, m->top.final_norm_g,
+                                                                     m->top.final_norm_b, d, c.norm_eps, opt, 1, 0, a, Mp);
+    count_launch();
+    SZO_TRY(szo_linear_fwd(m->lm_head_plan, a, SZO_BF16, Mr, nullptr, m->logits, SZO_F32, SZO_MODE_SPARSE_ADD, m->ws,
+                           m->ws_bytes, st));
+    ce_rows_pair_kernel<<<static_cast<unsigned>(M), 256, 0, st>>>(m->logits, Mp, tokens, S, c.vocab, m->tok_loss,
+                                                                 m->tok_loss + M);
+    mean_f64_kernel<<<1, 1024, 0, st>>>(m->tok_loss, M, static_cast<double>(B) * (S - 1), loss_plus_dev);
+    mean_f64_kernel<<<1, 1024, 0, st>>>(m->tok_loss + M, M, static_cast<double>(B) * (S - 1), loss_minus_dev);
+    count_launch(3);
+  } else {
+    float* a_last = reinterpret_cast<float*>(m->q);       // B centre states, then B half-differences, fp32
+    add_norm_pair_kernel<T, float><<<static_cast<unsigned>(B), 256, 0, st>>>(
+        m->h, pending, Mp, m->top.final_norm_g, m->top.final_norm_b, d, c.norm_eps, opt, S, S - 1, a_last, B);
+    cls2_pair_kernel<<<static_cast<unsigned>(B), 256, 0, st>>>(a_last, B, static_cast<const __nv_bfloat16*>(m->top.lm_head),
+                                                              cand, labels, d, c.vocab, m->tok_loss, m->tok_loss + B);
+    mean_f64_kernel<<<1, 1024, 0, st>>>(m->tok_loss, B, static_cast<double>(B), loss_plus_dev);
+    mean_f64_kernel<<<1, 1024, 0, st>>>(m->tok_loss + B, B, static_cast<double>(B), loss_minus_dev);
+    count_launch(4);
+  }
+  SZO_CHECK_LAUNCH("model kernels (paired form)");
+  return SZO_OK;
+}
+
 szo_status run_loss(szo_model* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand, int B, int S,
                     const float* Sv, double* loss_dev, cudaStream_t st) {
   if (m->cfg.act_dtype == SZO_F32) return run_loss_t<float>(m, tokens, labels, cand, B, S, Sv, loss_dev, st);
@@ -614,7 +1008,7 @@ szo_status run_loss(szo_model* m, const int32_t* tokens, const int32_t* labels, 
 // Both perturbed forwards of a step side by side (see run_loss_t); bf16 tensor-core path with the
 // materialised form only: the caller checks dual_forward_applies().
 bool dual_forward_applies(const szo_model* m, int64_t M) {
-  return m->dual_rows && m->cfg.act_dtype != SZO_F32 && m->cfg.linear_mode != SZO_MODE_FP32_VALIDATE &&
+  return m->dual_rows && !m->paired && m->cfg.act_dtype != SZO_F32 && m->cfg.linear_mode != SZO_MODE_FP32_VALIDATE &&
          m->cfg.linear_mode != SZO_MODE_SPMM && !m->plans.empty() && m->k_total > 0 &&
          (m->resident || tc_use_materialised(m->plans[0], M, true));
 }
@@ -652,6 +1046,8 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
   SZO_REQUIRE(c.act_dtype == SZO_BF16 || c.act_dtype == SZO_F32, SZO_ERR_UNSUPPORTED, "act_dtype must be bf16 or f32");
   SZO_REQUIRE(c.act_dtype == SZO_BF16 || c.linear_mode == SZO_MODE_FP32_VALIDATE, SZO_ERR_UNSUPPORTED,
               "fp32 activations need the fp32 validation mode");
+  SZO_REQUIRE(c.linear_mode >= SZO_MODE_AUTO && c.linear_mode <= SZO_MODE_PAIRED, SZO_ERR_INVALID_ARG,
+              "unknown linear_mode %d", c.linear_mode);
   SZO_REQUIRE(c.loss_kind == 0 || c.loss_kind == 1, SZO_ERR_INVALID_ARG, "loss_kind must be 0 or 1");
   SZO_REQUIRE(c.max_batch > 0 && c.max_seq > 1, SZO_ERR_SHAPE, "max_batch/max_seq");
   SZO_REQUIRE(c.arch == 0 || (top->pos && c.max_pos >= c.max_seq), SZO_ERR_INVALID_ARG, "position table missing/short");
@@ -664,6 +1060,8 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
   m->layers.assign(layers_host, layers_host + c.n_layers);
   m->S_all = S_all;
   m->Mmax = static_cast<int64_t>(c.max_batch) * c.max_seq;
+  m->paired = c.linear_mode == SZO_MODE_PAIRED;
+  const int32_t lmode = m->paired ? SZO_MODE_SPARSE_ADD : c.linear_mode;   // mode of a lone forward
   auto bail = [&](szo_status s) {
     szo_model_destroy(m);
     return s;
@@ -690,7 +1088,7 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
                                     w.idx, w.nnz, w.bias, st));
       m->plans.push_back(p);
       m->offsets.push_back(m->offsets.back() + w.nnz);
-      const size_t need = szo_linear_workspace_bytes(p, m->Mmax, c.linear_mode);
+      const size_t need = szo_linear_workspace_bytes(p, m->Mmax, lmode);
       if (need > ws_need) ws_need = need;
     }
   }
@@ -699,7 +1097,7 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
     const size_t need = tc_tail_ws_bound();
     if (need > ws_need) ws_need = need;
     // scratch of the materialised form: the largest group of layers that share their input
-    if (tc_use_materialised(m->plans[0], m->Mmax, true)) {
+    if (tc_use_materialised(m->plans[0], m->Mmax, true) || (m->paired && c.group != 0)) {
       for (int l = 0; l < c.n_layers; ++l) {
         const szo_linear* const* pl = m->plans.data() + static_cast<size_t>(l) * m->n_lin;
         const size_t g0 = tc_materialised_ws_bytes(pl, 3, m->Mmax);                       // q, k, v
@@ -744,7 +1142,7 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
   if (c.loss_kind == 0) {
     SZO_M_TRY(szo_linear_create(&m->lm_head_plan, c.vocab, c.d_model, 0, top->lm_head, nullptr, nullptr, SZO_BF16,
                                 nullptr, 0, nullptr, st));
-    const size_t need = szo_linear_workspace_bytes(m->lm_head_plan, m->Mmax, c.linear_mode);
+    const size_t need = szo_linear_workspace_bytes(m->lm_head_plan, 2 * m->Mmax + 256, lmode);
     if (need > ws_need) ws_need = need;
   }
   // buffers
@@ -754,12 +1152,18 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
   // two sets of Mmax rows.
   {
     const char* env = getenv("SZO_DUAL_FORWARD");
-    m->dual_rows = !(env != nullptr && env[0] == '0') && c.act_dtype != SZO_F32 &&
+    m->dual_rows = !(env != nullptr && env[0] == '0') && !m->paired && c.act_dtype != SZO_F32 &&
                    c.linear_mode != SZO_MODE_FP32_VALIDATE && c.linear_mode != SZO_MODE_SPMM && !m->plans.empty() &&
                    m->k_total > 0 && (m->resident || tc_use_materialised(m->plans[0], m->Mmax, true));
   }
-  const int64_t Mx = m->Mmax * (m->dual_rows ? 2 : 1), d = c.d_model, dkv = static_cast<int64_t>(c.n_kv_heads) * hd,
-                ff = c.d_ff;
+  // paired form: centre rows, then the half-difference rows from a multiple of 256 on
+  const int64_t Mpmax = static_cast<int64_t>(round_up(static_cast<size_t>(m->Mmax), 256));
+  const int64_t Mx = m->paired ? Mpmax + m->Mmax : m->Mmax * (m->dual_rows ? 2 : 1), d = c.d_model,
+                dkv = static_cast<int64_t>(c.n_kv_heads) * hd, ff = c.d_ff;
+  if (m->paired) {
+    const int64_t Kmax = d > ff ? d : ff;
+    SZO_M_TRY(dev_alloc(m, &m->xT, static_cast<size_t>(Kmax) * Mpmax * sizeof(__nv_bfloat16)));
+  }
   if (m->dual_rows) {
     SZO_M_TRY(dev_alloc(m, &m->Splus, m->k_total * sizeof(float)));
     SZO_M_TRY(dev_alloc(m, &m->Sminus, m->k_total * sizeof(float)));
@@ -837,6 +1241,17 @@ szo_status szo_attention(const void* q, const void* k, const void* v, void* o, s
   return SZO_OK;
 }
 
+szo_status szo_attention_paired(const void* q, const void* k, const void* v, void* o, int64_t row0, int32_t B,
+                                int32_t S, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, void* stream) {
+  SZO_REQUIRE(q && k && v && o, SZO_ERR_INVALID_ARG, "NULL pointer");
+  SZO_REQUIRE(B > 0 && S > 0 && n_heads > 0 && n_kv_heads > 0 && n_heads % n_kv_heads == 0, SZO_ERR_SHAPE, "bad shape");
+  SZO_REQUIRE(row0 >= static_cast<int64_t>(B) * S, SZO_ERR_SHAPE, "row0 must leave room for the B*S centre rows");
+  SZO_REQUIRE(head_dim == 64 || head_dim == 128, SZO_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
+  SZO_REQUIRE(aligned16(q) && aligned16(k) && aligned16(v) && aligned16(o), SZO_ERR_ALIGNMENT, "buffers must be 16-byte aligned");
+  return launch_flash_attention_pair_bf16(q, k, v, o, row0, B, S, n_heads, n_kv_heads, head_dim,
+                                          static_cast<cudaStream_t>(stream));
+}
+
 int64_t szo_model_k_total(const szo_model_t* m) { return m ? m->k_total : 0; }
 const int64_t* szo_model_gidx(const szo_model_t* m) { return m ? m->gidx : nullptr; }
 int64_t szo_model_last_launches(const szo_model_t* m) { return m ? m->last_launches : 0; }
@@ -859,6 +1274,22 @@ szo_status szo_model_zo_step(szo_model_t* m, const int32_t* tokens, const int32_
   const int64_t k = m->k_total;
   float* Sv = m->S_all;
   ScaleArg sa{eps, 0.f, 0.f, nullptr, nullptr};
+  if (m->paired) {
+    // S goes through the seed trick's +eps, -2 eps, +eps sequence (so that it ends where the
+    // in-place order leaves it) while z is kept; the two forwards then run in the paired form on the
+    // restored S, with +-eps z applied inside the linears in fp32
+    SZO_TRY(launch_sparse_axpy(Sv, Sv, m->gidx, k, 0, seed, step, sa, st, m->zkept));
+    sa.scale = -2.0f * eps;
+    SZO_TRY(launch_sparse_axpy_kept(Sv, Sv, m->zkept, k, sa, st));
+    sa.scale = eps;
+    SZO_TRY(launch_sparse_axpy_kept(Sv, Sv, m->zkept, k, sa, st));
+    SZO_TRY(run_loss_paired(m, tokens, labels, cand, B, S, Sv, m->zkept, eps, f_plus_dev, f_minus_dev, st));
+    SZO_TRY(szo_projected_gradient(f_plus_dev, f_minus_dev, eps, g_dev, stream));
+    ScaleArg su3{0.f, lr, eps, f_plus_dev, f_minus_dev};
+    SZO_TRY(launch_sparse_axpy_kept(Sv, Sv, m->zkept, k, su3, st));
+    m->last_launches = g_launch_count - before;
+    return SZO_OK;
+  }
   if (dual_forward_applies(m, static_cast<int64_t>(B) * S)) {
     // both forwards side by side: the same arithmetic on S as the in-place sequence below
     // (+eps, -2 eps, +eps), written to two copies, so that every linear makes one weight pass
