@@ -200,7 +200,7 @@ size_t szo_linear_workspace_bytes(const szo_linear_t* plan, int64_t M, int32_t m
  *   x   bf16 [M0 + M, K]: rows [0, M) = xc, rows [M0, M0 + M) = xd, M0 = M rounded up to a multiple of
  *       256 (rows in between are ignored)            y   y_dtype [M0 + M, N], same row layout
  *   S   fp32 [nnz] current sparse values             z   fp32 [nnz] z of this step at the entries of idx
- *   workspace  szo_linear_paired_workspace_bytes(plan, M) bytes (effective weight, x^T, K-split scratch)
+ *   workspace  szo_linear_paired_workspace_bytes(plan, M) bytes (effective weight, K-split scratch)
  * Every plan format is accepted (int4 groups, per-row tables, dense bf16). */
 size_t szo_linear_paired_workspace_bytes(const szo_linear_t* plan, int64_t M);
 szo_status szo_linear_fwd_paired(const szo_linear_t* plan, const void* x, int64_t M, const float* S, const float* z,

@@ -317,31 +317,202 @@ __global__ void scatter_add_bf16_kernel(const MatArgs a) {
   *el = __float2bfloat16_rn(__bfloat162float(base) + S[e]);
 }
 
-// xT[c][t] = x[t][c] for t < M, c < K (bf16; x row-major [M][K], xT row stride ldT >= M): the centre
-// activations by column, for the sparse product of the paired form.  64 x 64 tiles through shared
-// memory, 16-byte loads and stores.
-__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* __restrict__ x, int64_t M, int64_t K,
-                                                            __nv_bfloat16* __restrict__ xT, int64_t ldT) {
-  __shared__ __align__(16) __nv_bfloat16 tile[64][72];
-  const int64_t t0 = static_cast<int64_t>(blockIdx.x) * 64, c0 = static_cast<int64_t>(blockIdx.y) * 64;
-  const int r = threadIdx.x >> 3, ch = threadIdx.x & 7;          // 32 rows x 8 chunks of 8 elements per pass
+// Sparse product of the paired form: yd[t][n] += eps * sum_e z_e * xc[t][col_e] over the sensitive entries e
+// of weight row n (Zbar of Definition 4 times the centre activations), for the M half-difference
+// rows of up to three matrices that share x; runs after the tensor-core launch that wrote xd W^T into
+// those rows.  The sum is formed in fp32 and added to the stored value, one rounding (the
+// half-difference has its own exponent, so a second bf16 rounding costs 2^-9 of ITS size, not of
+// the centre's).
+// A block owns TM tokens and a share of the weight rows: it stages xc[those tokens][all K columns] in
+// shared memory transposed, xs[c][TM] (16-byte reads along the token rows, 2-byte stores rotated so
+// that the four column groups of a warp hit different banks), then each thread walks weight rows:
+// every entry is one 16-byte (TM = 8) read of shared memory and TM fused multiply-adds; y is read and
+// written 64 contiguous bytes per token and warp.  Tried first: columns of a transposed copy of xc
+// read from L2 per entry (8 KB per entry, 2.6 TB/s: 20 ms of a Llama-2-7B-shaped step), and the slab
+// copied from that transposed copy (16 bytes every 8 KB: the strided reads camp on a few L2 slices,
+// 25 ms).  The epilogue of the tensor-core kernel is on that kernel's critical path
+// (adding this sum there, from xT or from a buffer, made the decoder-block linears 45 % slower), which
+// is why it is a pass of its own.
+struct CrossSub {
+  const int32_t* row_ptr;
+  const uint32_t* rec;   // per entry: column in the low col_bits bits, the leading bits of fp32(eps * z) above them
+  void* yd;              // first half-difference row of this matrix's y
+  int64_t N;
+};
+struct CrossArgs {
+  CrossSub sub[3];
+  int n;
+  const __nv_bfloat16* x;   // centre rows [M][K]
+  int64_t M, K;
+  uint32_t col_mask;        // (1 << col_bits) - 1, col_bits = bits needed for K - 1
+};
+template <int TM> struct SlabVec;
+template <> struct SlabVec<16> { using type = uint4; };   // two per column
+template <> struct SlabVec<8> { using type = uint4; };
+template <> struct SlabVec<4> { using type = uint2; };
+template <> struct SlabVec<2> { using type = uint32_t; };
+
+// R weight rows per thread (2 when N is even: y is then read and written four bytes per lane)
+template <int TM, int R, typename TY>
+__global__ void __launch_bounds__(TM == 16 ? 1024 : 512) pair_cross_kernel(const CrossArgs a) {
+  using V = typename SlabVec<TM>::type;
+  constexpr int kVecs = TM * 2 / static_cast<int>(sizeof(V));    // vectors per column
+  extern __shared__ __align__(16) unsigned char cross_smem[];
+  const V* xs = reinterpret_cast<const V*>(cross_smem);          // [K][kVecs]
+  const int64_t m0 = static_cast<int64_t>(blockIdx.x) * TM;
+  {
+    // lane = (column group cg, token t): one 16-byte load of 8 columns of token t, then 8 two-byte
+    // stores xs[c][t]; group cg starts its 8 stores at element cg so that groups use different banks
+    unsigned short* xs16 = reinterpret_cast<unsigned short*>(cross_smem);
+    constexpr int kLaneTok = TM < 32 ? TM : 32;
+    const int t = threadIdx.x % kLaneTok, cg = (threadIdx.x / kLaneTok) & 7;
+    const int64_t per_pass = static_cast<int64_t>(blockDim.x / kLaneTok) * 8;       // columns per pass of the block
+    const bool valid = m0 + t < a.M;
+    const __nv_bfloat16* row = a.x + (m0 + t) * a.K;
+    for (int64_t c8 = static_cast<int64_t>(threadIdx.x / kLaneTok) * 8; c8 < a.K; c8 += per_pass) {
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (valid) v = *reinterpret_cast<const uint4*>(row + c8);
 #pragma unroll
-  for (int p = 0; p < 2; ++p) {
-    const int tr = r + p * 32;
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (t0 + tr < M) v = *reinterpret_cast<const uint4*>(x + (t0 + tr) * K + c0 + ch * 8);   // K % 64 == 0
-    *reinterpret_cast<uint4*>(&tile[tr][ch * 8]) = v;
+      for (int i = 0; i < 8; ++i) {
+        const int el = (i + cg) & 7;
+        const uint32_t w = el < 4 ? (el < 2 ? v.x : v.y) : (el < 6 ? v.z : v.w);      // selects, not an indexed array
+        xs16[(c8 + el) * TM + t] = static_cast<unsigned short>((el & 1) ? w >> 16 : w & 0xFFFFu);
+      }
+    }
   }
   __syncthreads();
+  const int cnt = static_cast<int>(a.M - m0 < TM ? a.M - m0 : TM);
+  for (int s = 0; s < a.n; ++s) {
+    const int32_t* row_ptr = s == 0 ? a.sub[0].row_ptr : (s == 1 ? a.sub[1].row_ptr : a.sub[2].row_ptr);
+    if (row_ptr == nullptr) continue;
+    const uint32_t* rec = s == 0 ? a.sub[0].rec : (s == 1 ? a.sub[1].rec : a.sub[2].rec);
+    TY* yd = static_cast<TY*>(s == 0 ? a.sub[0].yd : (s == 1 ? a.sub[1].yd : a.sub[2].yd));
+    const int64_t N = s == 0 ? a.sub[0].N : (s == 1 ? a.sub[1].N : a.sub[2].N);
+    // the row shares of the gridDim.y blocks of a token group interleave in units of the block size
+    for (int64_t n = (static_cast<int64_t>(blockIdx.y) * blockDim.x + threadIdx.x) * R; n < N;
+         n += static_cast<int64_t>(gridDim.y) * blockDim.x * R) {
+      int32_t eb[R + 1];
 #pragma unroll
-  for (int p = 0; p < 2; ++p) {
-    const int cr = r + p * 32;                                    // column of x = row of xT
-    __nv_bfloat16 o[8];
+      for (int r = 0; r <= R; ++r) eb[r] = __ldg(row_ptr + (n + r <= N ? n + r : N));
+      if (eb[0] == eb[R]) continue;
+      float acc[R][TM];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) o[j] = tile[ch * 8 + j][cr];
-    *reinterpret_cast<uint4*>(xT + (c0 + cr) * ldT + t0 + ch * 8) = *reinterpret_cast<const uint4*>(o);   // ldT % 64 == 0
+      for (int r = 0; r < R; ++r) {
+#pragma unroll
+        for (int j = 0; j < TM; ++j) acc[r][j] = 0.f;
+        for (int32_t e = eb[r]; e < eb[r + 1]; ++e) {
+          const uint32_t rc = __ldg(rec + e);
+          const float zz = __uint_as_float(rc & ~a.col_mask);
+          const uint32_t col = rc & a.col_mask;
+#pragma unroll
+          for (int q = 0; q < kVecs; ++q) {
+            const V v = xs[col * kVecs + q];
+            const uint32_t* w = reinterpret_cast<const uint32_t*>(&v);
+            constexpr int kW = static_cast<int>(sizeof(V)) / 4;
+#pragma unroll
+            for (int h = 0; h < kW; ++h) {
+              acc[r][q * kW * 2 + 2 * h] = fmaf(zz, __uint_as_float(w[h] << 16), acc[r][q * kW * 2 + 2 * h]);
+              acc[r][q * kW * 2 + 2 * h + 1] = fmaf(zz, __uint_as_float(w[h] & 0xFFFF0000u), acc[r][q * kW * 2 + 2 * h + 1]);
+            }
+          }
+        }
+      }
+      TY* yp = yd + m0 * N + n;
+      if constexpr (R == 2 && sizeof(TY) == 2) {
+        uint32_t old[TM];
+#pragma unroll
+        for (int j = 0; j < TM; ++j) old[j] = (j < cnt) ? *reinterpret_cast<const uint32_t*>(yp + j * N) : 0u;
+#pragma unroll
+        for (int j = 0; j < TM; ++j) {
+          if (j < cnt) {
+            const __nv_bfloat162 o = __floats2bfloat162_rn(__uint_as_float(old[j] << 16) + acc[0][j],
+                                                            __uint_as_float(old[j] & 0xFFFF0000u) + acc[1][j]);
+            *reinterpret_cast<__nv_bfloat162*>(yp + j * N) = o;
+          }
+        }
+      } else {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          if (n + r >= N) continue;
+          float old[TM];
+#pragma unroll
+          for (int j = 0; j < TM; ++j) old[j] = (j < cnt) ? static_cast<float>(yp[j * N + r]) : 0.f;
+#pragma unroll
+          for (int j = 0; j < TM; ++j) {
+            if (j < cnt) {
+              if constexpr (sizeof(TY) == 2) yp[j * N + r] = __float2bfloat16_rn(old[j] + acc[r][j]);
+              else yp[j * N + r] = old[j] + acc[r][j];
+            }
+          }
+        }
+      }
+    }
   }
 }
+
+// rec[e] = the column of entry e in the low col_bits bits and, above them, fp32(eps * z[e]) rounded to
+// the nearest value with 32 - col_bits bits (sign, exponent and at least 9 bits of mantissa for K up
+// to 16384: 2^-10 relative, a quarter of a bf16 rounding, on a term that ends in a bf16 value)
+__global__ void pack_cross_records_kernel(const int32_t* __restrict__ col, const float* __restrict__ z, float eps,
+                                          int64_t n, uint32_t col_mask, uint32_t* __restrict__ rec) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  uint32_t b = __float_as_uint(eps * z[i]);
+  b += (col_mask >> 1) + ((b >> (32 - __clz(col_mask))) & 1u);       // to nearest, ties to even, at bit col_bits
+  rec[i] = (b & ~col_mask) | static_cast<uint32_t>(col[i]);
+}
+
+template <int TM, int R, typename TY>
+szo_status launch_pair_cross(const CrossArgs& ca, int64_t max_N, cudaStream_t st) {
+  const size_t smem = static_cast<size_t>(ca.K) * TM * sizeof(__nv_bfloat16);
+  SZO_CHECK_CUDA(cudaFuncSetAttribute(pair_cross_kernel<TM, R, TY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      static_cast<int>(smem)));
+  // few token groups: the rows of a group go to several blocks (each stages the slab again), so that
+  // the grid covers the SMs
+  const int64_t groups = ceil_div(ca.M, TM);
+  int row_split = static_cast<int>(ceil_div(296, groups));
+  constexpr int kThreads = TM == 16 ? 1024 : 512;
+  const int64_t max_split = ceil_div(max_N, kThreads * R);
+  if (row_split > max_split) row_split = static_cast<int>(max_split);
+  if (row_split < 1) row_split = 1;
+  dim3 grid(static_cast<unsigned>(groups), static_cast<unsigned>(row_split));
+  pair_cross_kernel<TM, R, TY><<<grid, kThreads, smem, st>>>(ca);
+  count_launch();
+  SZO_CHECK_LAUNCH("pair_cross_kernel");
+  return SZO_OK;
+}
+template <int TM>
+szo_status launch_pair_cross_tm(const CrossArgs& ca, int64_t max_N, bool even, bool f32, cudaStream_t st) {
+  if (f32) return launch_pair_cross<TM, 1, float>(ca, max_N, st);
+  if (even) return launch_pair_cross<TM, 2, __nv_bfloat16>(ca, max_N, st);
+  return launch_pair_cross<TM, 1, __nv_bfloat16>(ca, max_N, st);
+}
+
+}  // namespace
+
+size_t tc_paired_rec_bytes(const szo_linear* const* plans, int n) {
+  size_t nnz = 0;
+  for (int i = 0; i < n; ++i) nnz += static_cast<size_t>(plans[i]->nnz);
+  return round_up(nnz * sizeof(uint32_t), 256);
+}
+
+uint32_t cross_col_mask(int64_t K) {
+  uint32_t bits = 1;
+  while ((int64_t(1) << bits) < K) ++bits;
+  return (1u << bits) - 1u;
+}
+
+szo_status pack_cross_records(const int32_t* col, const float* z, float eps, int64_t n, int64_t K, uint32_t* rec,
+                              cudaStream_t st) {
+  if (n == 0) return SZO_OK;
+  SZO_REQUIRE(K <= (int64_t(1) << 18), SZO_ERR_UNSUPPORTED, "K = %lld too large for the paired form", (long long)K);
+  pack_cross_records_kernel<<<static_cast<unsigned>(ceil_div(n, 256)), 256, 0, st>>>(col, z, eps, n, cross_col_mask(K), rec);
+  count_launch();
+  SZO_CHECK_LAUNCH("pack_cross_records_kernel");
+  return SZO_OK;
+}
+
+namespace {
 
 // SZO_LINEAR_MATERIALISE=0 / 1 switches the form off / on for every M (A/B measurement)
 int materialise_override() {
@@ -514,27 +685,12 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
   P.m_tiles = ceil_div(M_rows, 256);
   P.nsub = n;
   if (paired != nullptr) {
-    SZO_REQUIRE(paired->xT != nullptr && paired->eps != 0.f, SZO_ERR_INVALID_ARG, "paired form: xT scratch and eps needed");
-    P.pair_eps = paired->eps;
     P.pair_row0 = Mp;
-    P.xT = paired->xT;
-    P.ldT = Mp;
-    P.mt_c = static_cast<int>(Mp / 256);
-    P.mt_d = static_cast<int>(ceil_div(M, 256));
-    dim3 grid(static_cast<unsigned>(Mp / 64), static_cast<unsigned>(p0->K / 64));
-    transpose_bf16_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), M, p0->K, paired->xT, Mp);
-    count_launch();
-    SZO_CHECK_LAUNCH("transpose_bf16_kernel");
   }
   int64_t n_tiles = 0;
   for (int i = 0; i < n; ++i) {
     const szo_linear* p = plans[i];
     TcSub& sb = P.sub[i];
-    if (paired != nullptr && p->nnz > 0) {
-      sb.row_ptr = p->row_ptr;
-      sb.ent_col = p->ent_col;
-      sb.zc = paired->z[i];
-    }
     sb.codes = nullptr;
     sb.sz = nullptr;
     sb.bucket_ptr = nullptr;
@@ -577,6 +733,30 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
     for (int i = 0; i < n; ++i)
       P.sub[i].y = static_cast<unsigned char*>(y[i]) + static_cast<size_t>(set) * M * plans[i]->N * y_elt;
     SZO_TRY(launch_pair_kernel(false, false, mx, mw, P, sc.n_pairs, st));
+  }
+  if (paired != nullptr && nnz_all > 0) {
+    CrossArgs ca{};
+    ca.n = n; ca.x = static_cast<const __nv_bfloat16*>(x); ca.M = M; ca.K = p0->K;
+    ca.col_mask = cross_col_mask(p0->K);
+    const size_t y_el = (y_dtype == SZO_F32) ? 4 : 2;
+    int64_t max_N = 0;
+    bool even = true;
+    for (int i = 0; i < n; ++i) {
+      const szo_linear* p = plans[i];
+      if (p->N > max_N) max_N = p->N;
+      if (p->N & 1) even = false;
+      ca.sub[i] = CrossSub{p->nnz > 0 ? p->row_ptr : nullptr, paired->rec[i],
+                           static_cast<unsigned char*>(y[i]) + static_cast<size_t>(Mp) * p->N * y_el, p->N};
+    }
+    const size_t per_token = static_cast<size_t>(p0->K) * sizeof(__nv_bfloat16);
+    const bool f32 = y_dtype == SZO_F32;
+    if (16 * per_token <= 200 * 1024 && M >= 2048) SZO_TRY(launch_pair_cross_tm<16>(ca, max_N, even, f32, st));
+    else if (8 * per_token <= 200 * 1024) SZO_TRY(launch_pair_cross_tm<8>(ca, max_N, even, f32, st));
+    else if (4 * per_token <= 200 * 1024) SZO_TRY(launch_pair_cross_tm<4>(ca, max_N, even, f32, st));
+    else {
+      SZO_REQUIRE(2 * per_token <= 200 * 1024, SZO_ERR_UNSUPPORTED, "K = %lld too large for the paired form", (long long)p0->K);
+      SZO_TRY(launch_pair_cross_tm<2>(ca, max_N, even, f32, st));
+    }
   }
   return SZO_OK;
 }

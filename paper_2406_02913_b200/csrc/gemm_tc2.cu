@@ -126,24 +126,9 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& P, int pair, int n_p
     u.kb0 = tail_kb_at(P, u.part);
     u.kb1 = tail_kb_at(P, u.part + 1);
   }
-  int np;
-  if (P.mt_d > 0) {
-    // paired launch: every half-difference token tile (of every row tile) comes before the centre
-    // tiles, so that the last round holds tiles with the short epilogue only
-    const int first = static_cast<int>(P.n_tiles) * P.mt_d;
-    if (tile < first) {
-      np = tile / P.mt_d;
-      u.m_tile = P.mt_c + (tile - np * P.mt_d);
-    } else {
-      const int t2 = tile - first;
-      np = t2 / P.mt_c;
-      u.m_tile = t2 - np * P.mt_c;
-    }
-  } else {
-    const int m_tiles = static_cast<int>(P.m_tiles);
-    np = tile / m_tiles;
-    u.m_tile = tile - np * m_tiles;
-  }
+  const int m_tiles = static_cast<int>(P.m_tiles);
+  int np = tile / m_tiles;
+  u.m_tile = tile - np * m_tiles;
   u.g_tile = np * 2 + rank;
   u.s = 0;
   if (P.nsub > 1 && np >= P.sub[0].n_tiles) {
@@ -240,7 +225,7 @@ __device__ __noinline__ void reduce_parts(const float* part0, int parts, int64_t
 // kRelu: y = max(y, 0) in the epilogue (dense mode only: its own instantiation, so that the other
 // launches' store loops stay as they are)
 // kPaired: the paired form of a ZO step's two forwards (dense mode only, see TcParams): bias on the
-// centre rows only, eps * xc Zbar^T added to the half-difference rows in the epilogue
+// centre rows only
 template <int kXS, bool kDequant, bool kFast, bool kRelu = false, bool kPaired = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumWarps2 * 32, 1)
 szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
@@ -675,50 +660,10 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         }
       };
       const uint32_t t_acc = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + static_cast<uint32_t>(as * kPairBT);
-      // Paired form, half-difference token tile: v[j] += eps * sum_e z_e * xc[token j][col_e] over the
-      // sensitive entries e of this thread's weight row, in fp32, before the one rounding of the store.
-      // Column col_e of xc is contiguous in xT, so a chunk of 32 tokens is four 16-byte loads per entry.
-      // (A tile split along K adds it in its first part only.)
-      int32_t ce0 = 0, ce1 = 0;
-      const int32_t* ent_col = nullptr;
-      const float* zc = nullptr;
-      if constexpr (kPaired) {
-        if (m0 >= P.pair_row0 && u.part == 0 && n < N && SZO_SUB(P, u.s, row_ptr) != nullptr) {
-          const int32_t* rp = SZO_SUB(P, u.s, row_ptr) + n;
-          ce0 = __ldg(rp);
-          ce1 = __ldg(rp + 1);
-          ent_col = SZO_SUB(P, u.s, ent_col);
-          zc = SZO_SUB(P, u.s, zc);
-        }
-      }
-      auto cross_chunk = [&](int c0, uint32_t (&v)[32]) {
-        if constexpr (kPaired) {
-          if (c0 >= mlimit) return;
-          const __nv_bfloat16* xt = P.xT + (m0 - P.pair_row0 + c0);
-          for (int32_t e = ce0; e < ce1; ++e) {
-            const float zz = __ldg(zc + e) * P.pair_eps;
-            const uint4* src = reinterpret_cast<const uint4*>(xt + static_cast<int64_t>(__ldg(ent_col + e)) * P.ldT);
-            uint4 a[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) a[i] = __ldg(src + i);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const uint32_t w4[4] = {a[i].x, a[i].y, a[i].z, a[i].w};
-#pragma unroll
-              for (int h = 0; h < 4; ++h) {
-                const int j = i * 8 + h * 2;
-                v[j] = __float_as_uint(fmaf(zz, __uint_as_float(w4[h] << 16), __uint_as_float(v[j])));
-                v[j + 1] = __float_as_uint(fmaf(zz, __uint_as_float(w4[h] & 0xFFFF0000u), __uint_as_float(v[j + 1])));
-              }
-            }
-          }
-        }
-      };
       if (u.parts == 1) {
         for (int c0 = 0; c0 < kPairBT; c0 += 32) {
           uint32_t v[32];
           tmem_ld32(t_acc + static_cast<uint32_t>(c0), v);
-          cross_chunk(c0, v);
           store_chunk(c0, v);
         }
         tc_fence_before();
@@ -733,7 +678,6 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         for (int c0 = 0; c0 < kPairBT; c0 += 32) {
           uint32_t v[32];
           tmem_ld32(t_acc + static_cast<uint32_t>(c0), v);
-          cross_chunk(c0, v);
 #pragma unroll
           for (int j = 0; j < 32; ++j) __stcg(mine + (c0 + j) * kBM, __uint_as_float(v[j]));
         }
@@ -809,7 +753,7 @@ szo_status launch_tc2(const CUtensorMap& mx, const CUtensorMap& mw, const TcPara
 
 szo_status launch_pair_kernel(bool dequant, bool bf16_tables, const CUtensorMap& mx, const CUtensorMap& mw,
                               const tc::TcParams& P, int n_pairs, cudaStream_t st) {
-  if (P.mt_d > 0) {
+  if (P.pair_row0 > 0) {
     SZO_REQUIRE(!dequant && !P.relu, SZO_ERR_UNSUPPORTED, "the paired form exists in the dense mode without ReLU only");
     return launch_tc2<6, false, false, false, true>(mx, mw, P, n_pairs, st);
   }

@@ -70,12 +70,16 @@ bool tc_use_materialised(const szo_linear* p, int64_t M, bool two_sets = false);
 size_t tc_materialised_ws_bytes(const szo_linear* const* plans, int n, int64_t M);
 // Paired form of a ZO step's two forwards (see tc::TcParams): x and every y[i] hold the M centre rows
 // first and the M half-difference rows from row round_up(M, 256) on; S_pert are the unperturbed sparse
-// values; z[i] the z of plans[i]'s entries; xT scratch of K * round_up(M, 256) bf16.
+// values; rec[i][e] = column of entry e of plans[i] and eps * z_e in one word (pack_cross_records; the
+// split depends on K only, so one call may pack the entries of matrices with different K one after another
+// only if called per K).
 struct PairedArgs {
-  const float* const* z;
-  float eps;
-  __nv_bfloat16* xT;
+  const uint32_t* const* rec;
 };
+szo_status pack_cross_records(const int32_t* col, const float* z, float eps, int64_t n, int64_t K, uint32_t* rec,
+                              cudaStream_t st);
+uint32_t cross_col_mask(int64_t K);
+size_t tc_paired_rec_bytes(const szo_linear* const* plans, int n);
 szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, const void* x, int64_t M,
                                       const float* const* S_pert, void* const* y, int y_dtype, void* ws,
                                       size_t ws_bytes, cudaStream_t st, const float* const* S_second = nullptr,

@@ -653,12 +653,11 @@ struct szo_model {
   int64_t* gidx = nullptr;
   int32_t* geid = nullptr;      // [k_total] entry id in S_all of each bucket-ordered record
   uint16_t* gpos = nullptr;     // [k_total] in-tile position of each bucket-ordered record
-  uint2* recs = nullptr;        // [k_total] (position, value) records of the current forward
+  uint2* recs = nullptr;        // [k_total] (position, value) records of the current forward; paired form: (column, eps z)
   float* zkept = nullptr;       // [k_total] z of the current step, kept by the first perturb pass
   float *Splus = nullptr, *Sminus = nullptr;   // [k_total] the two perturbed copies of S (two forwards side by side)
   bool dual_rows = false;       // the activation buffers hold 2 * Mmax rows
   bool paired = false;          // SZO_MODE_PAIRED: a step's two forwards as centre and half-difference
-  __nv_bfloat16* xT = nullptr;  // paired form: the centre activations of the current linear by column
   // dense bf16 weights (group == 0) with many tokens: every launch group keeps its effective weight
   // resident (a private copy of the frozen matrices, masked entries rewritten per forward)
   bool resident = false;
@@ -906,11 +905,11 @@ szo_status run_loss_paired(szo_model* m, const int32_t* tokens, const int32_t* l
     const int t0 = layer * m->n_lin + j0;
     const szo_linear* plans[3];
     const float* sv[3];
-    const float* zz[3];
+    const uint32_t* crec[3];
     for (int i = 0; i < n; ++i) {
       plans[i] = m->plans[t0 + i];
       sv[i] = Sv + m->offsets[t0 + i];
-      zz[i] = z + m->offsets[t0 + i];
+      crec[i] = reinterpret_cast<const uint32_t*>(m->recs) + m->offsets[t0 + i];
     }
     if (m->timing) {
       while (m->events.size() < m->events_used + 2) {
@@ -920,7 +919,7 @@ szo_status run_loss_paired(szo_model* m, const int32_t* tokens, const int32_t* l
       }
       SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used], st));
     }
-    const PairedArgs pa{zz, eps, m->xT};
+    const PairedArgs pa{crec};
     const bool res = m->resident;
     const szo_status rc = linear_fwd_tc_materialised(plans, n, x, M, sv, outs, SZO_BF16, m->ws, m->ws_bytes, st, nullptr,
                                                      res ? m->res_W[t0] : nullptr, res ? m->res_saved[t0] : nullptr,
@@ -935,6 +934,11 @@ szo_status run_loss_paired(szo_model* m, const int32_t* tokens, const int32_t* l
     void* const outs[1] = {out};
     return lin_group(layer, j, 1, x, outs);
   };
+  // (column, eps * z) of every sensitive entry, once for all linears of the step (the record layout
+  // depends on K: one call per linear)
+  for (size_t t = 0; t < m->plans.size(); ++t)
+    SZO_TRY(pack_cross_records(m->plans[t]->ent_col, z + m->offsets[t], eps, m->plans[t]->nnz, m->plans[t]->K,
+                               reinterpret_cast<uint32_t*>(m->recs) + m->offsets[t], st));
   embed_kernel<<<static_cast<unsigned>(M), 128, 0, st>>>(tokens, static_cast<const __nv_bfloat16*>(m->top.embed),
                                                         static_cast<const __nv_bfloat16*>(m->top.pos), S, d, c.vocab, m->h);
   SZO_CHECK_CUDA(cudaMemsetAsync(m->h + Mp * d, 0, static_cast<size_t>(M) * d * sizeof(float), st));   // both forwards embed alike
@@ -1160,10 +1164,6 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
   const int64_t Mpmax = static_cast<int64_t>(round_up(static_cast<size_t>(m->Mmax), 256));
   const int64_t Mx = m->paired ? Mpmax + m->Mmax : m->Mmax * (m->dual_rows ? 2 : 1), d = c.d_model,
                 dkv = static_cast<int64_t>(c.n_kv_heads) * hd, ff = c.d_ff;
-  if (m->paired) {
-    const int64_t Kmax = d > ff ? d : ff;
-    SZO_M_TRY(dev_alloc(m, &m->xT, static_cast<size_t>(Kmax) * Mpmax * sizeof(__nv_bfloat16)));
-  }
   if (m->dual_rows) {
     SZO_M_TRY(dev_alloc(m, &m->Splus, m->k_total * sizeof(float)));
     SZO_M_TRY(dev_alloc(m, &m->Sminus, m->k_total * sizeof(float)));

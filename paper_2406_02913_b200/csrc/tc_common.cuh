@@ -30,10 +30,6 @@ struct TcSub {
   int64_t N, Npad;
   int n_rowtiles;          // 128-row tiles that have buckets
   int n_tiles;             // 256-row pair tiles
-  // paired form (TcParams::pair_eps != 0): the sensitive entries of this matrix by row, and their z
-  const int32_t* row_ptr;  // [N + 1]
-  const int32_t* ent_col;  // [nnz] column of entry e (entries ascending by row, then column)
-  const float* zc;         // [nnz] z of entry e
 };
 
 struct TcParams {
@@ -61,14 +57,10 @@ struct TcParams {
   //   centre rows:           y = xc W^T + bias
   //   half-difference rows:  y = xd W^T + eps * xc Zbar^T          (Zbar: z at the sensitive entries)
   // so x+- (W +- eps Zbar)^T = (centre) +- (half-difference) up to the term eps xd Zbar^T, which is of
-  // relative order eps^2.  The sparse product is added to the fp32 accumulator in the epilogue from
-  // xT = xc^T ([K][ldT] bf16, column t = token t).  The half-difference token tiles are visited first
-  // (their epilogue is the long one), mt_c / mt_d count the token tiles of the two kinds.
-  float pair_eps;          // 0: not a paired launch
-  int64_t pair_row0;       // first half-difference row; bias is added to rows below it only
-  const __nv_bfloat16* xT;
-  int64_t ldT;
-  int mt_c, mt_d;
+  // relative order eps^2.  This kernel computes the dense products of both kinds of rows in one launch
+  // and leaves the bias out of the half-difference rows; the sparse product is added to those rows by
+  // pair_cross_kernel after it.
+  int64_t pair_row0;       // first half-difference row (0: not a paired launch)
 };
 
 // Position in a ring of n slots: slot index and the parity of the current pass over the ring.
