@@ -6,7 +6,8 @@
  *
  * Conventions (all entry points)
  *   pointers   Device pointers unless the name ends in _host.  The caller owns every buffer it
- *              passes; the library allocates only inside *_create (freed by *_destroy).
+ *              passes; the library allocates inside *_create (freed by *_destroy) and, once per
+ *              device, a 4-byte status word on the first call that may report a device-side problem.
  *              Buffers must be 16-byte aligned (SZO_ERR_ALIGNMENT otherwise).
  *   stream     `void* stream` is a cudaStream_t (NULL = default stream).  Calls enqueue work and
  *              return; none synchronises unless its comment says so.
@@ -69,8 +70,15 @@ const char* szo_last_error(void);              /* thread-local; valid until the 
 int szo_version(void);
 
 /* Reads and clears the device status word (0 = no kernel reported a problem, else a negative
- * szo_status).  Synchronises the device. */
+ * szo_status).  Synchronises the device.  After a non-zero status every plan clears the tickets of
+ * its K-split tiles before its next launch (a kernel that gave up may have left them set). */
 szo_status szo_device_status(int32_t* status_host);
+
+/* Self-test of the bounded waits inside the kernels (no counterpart in the paper): launches one tiny
+ * kernel whose only wait, limited to limit_ms milliseconds of SM clock, is on a barrier that nothing
+ * ever signals.  The wait must give up: *gave_up_host = 1, the kernel returns, and the next
+ * szo_device_status reports SZO_ERR_TIMEOUT.  Synchronises the stream. */
+szo_status szo_selftest_wait_timeout(double limit_ms, int32_t* gave_up_host, void* stream);
 
 /* ---- Quantizer Q for w_dense (Section 3.5, "Integration with quantization": the dense part is
  * stored in 4 bits; the paper leaves the choice of quantizer open).  Uniform asymmetric,
@@ -97,11 +105,14 @@ szo_status szo_select_mask(const float* scores, int64_t n, int64_t k, int64_t* i
  * for example a plug-in running inside a host application that owns the allocator and hands out only
  * the input and output buffers, or a process whose memory budget is fixed before it starts.  The
  * scratch that szo_select_mask takes as a workspace lives here in a fixed array inside the library
- * (about 194 KiB of device memory on every GPU that loads the library, until the process exits), so
- * the call performs no cudaMalloc/cudaFree and needs no workspace query.
+ * (196 864 bytes = 192.25 KiB of device memory on every GPU that loads the library, until the process
+ * exits), so the call performs no cudaMalloc/cudaFree and needs no workspace query.
  *   limit     n <= 67 108 864 (2^26) scores; larger n returns SZO_ERR_WORKSPACE and touches nothing.
  *   set-up    the first call on each device looks up the array's device address (the device must be
- *             current, as for every call); make that first call before starting any stream capture.
+ *             current, as for every call) and keeps it for the life of the process; it belongs to the
+ *             device's primary context, so a cudaDeviceReset in the same process invalidates it.
+ *   capture   like szo_select_mask the call ends in a stream synchronisation (it reads the NaN flag
+ *             back), so it cannot be issued on a stream that is being captured.
  *   sharing   every call on a device uses the same array and finds the previous call's contents in
  *             it; the function clears what it needs.  Two calls that overlap on the GPU (different
  *             streams or threads) race on it: serialise them.

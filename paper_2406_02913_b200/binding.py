@@ -62,6 +62,7 @@ _SIGS = {
     "szo_last_error": (C.c_char_p, []),
     "szo_version": (C.c_int, []),
     "szo_device_status": (C.c_int32, [C.POINTER(C.c_int32)]),
+    "szo_selftest_wait_timeout": (C.c_int32, [C.c_double, C.POINTER(C.c_int32), C.c_void_p]),
     "szo_quantize": (C.c_int32, [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int32, C.c_int,
                                  C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "szo_select_mask": (C.c_int32, [C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
@@ -155,6 +156,13 @@ def _stream():
 def device_status() -> int:
     v = C.c_int32(0)
     _check(lib().szo_device_status(C.byref(v)))
+    return v.value
+
+
+def selftest_wait_timeout(limit_ms: float = 2.0) -> int:
+    """1 when the kernel's bounded wait gave up (as it must); the status word then holds SZO_ERR_TIMEOUT."""
+    v = C.c_int32(0)
+    _check(lib().szo_selftest_wait_timeout(limit_ms, C.byref(v), _stream()))
     return v.value
 
 

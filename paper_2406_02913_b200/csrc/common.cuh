@@ -19,6 +19,8 @@ szo_status fail(szo_status code, const char* fmt, ...);
 
 // Device status word (one per device, allocated on first use on the current device).
 int32_t* device_status_word();
+// Host-side count of non-zero status reads (see status.cu).
+uint64_t abort_epoch();
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t dtype_size(int dt) { return dt == SZO_F32 ? 4 : 2; }

@@ -50,6 +50,7 @@ struct TcPlan {
   CUtensorMap w_map;    // dense bf16 weight (G == 0) or the packed codes as bytes (G > 0)
   int sms;
   int32_t* tickets;     // device, [sms / 2][2][4], zero between launches (K-split tiles of the pair kernel)
+  uint64_t clean_epoch; // abort_epoch() when the tickets were last known to be zero
 };
 
 // Work schedule of the pair-tile kernel over `tiles` pair tiles (see TcParams).  The last, partial
@@ -103,6 +104,19 @@ szo_status make_codes_map(CUtensorMap* map, const void* base, int64_t rows, int6
 
 }  // namespace
 
+// A kernel that gave up on a bounded wait leaves the tickets of its K-split tiles non-zero (only the
+// part that finishes last resets them).  Once the host has seen that status (szo_device_status), every
+// plan clears its tickets before its next launch.
+static szo_status refresh_tickets(const TcPlan* tc, cudaStream_t st) {
+  TcPlan* t = const_cast<TcPlan*>(tc);
+  const uint64_t now = abort_epoch();
+  if (t->clean_epoch != now) {
+    SZO_CHECK_CUDA(cudaMemsetAsync(t->tickets, 0, static_cast<size_t>(t->sms / 2) * 8 * sizeof(int32_t), st));
+    t->clean_epoch = now;
+  }
+  return SZO_OK;
+}
+
 szo_status tc_plan_create(szo_linear* p, cudaStream_t) {
   TcPlan* t = new TcPlan();
   int dev = 0;
@@ -122,6 +136,7 @@ szo_status tc_plan_create(szo_linear* p, cudaStream_t) {
     delete t;
     return fail(SZO_ERR_CUDA, "cannot allocate the K-split tickets");
   }
+  t->clean_epoch = abort_epoch();
   p->tc = t;
   return SZO_OK;
 }
@@ -205,6 +220,7 @@ szo_status linear_fwd_tc_group(const szo_linear* const* plans, int n, const void
   for (int i = 0; i < 5; ++i) P.tail_kb[i] = sc.tail_kb[i];
   P.partial = static_cast<float*>(ws);
   P.tickets = t->tickets;
+  SZO_TRY(refresh_tickets(t, st));
   return launch_pair_kernel(p0->G != 0, p0->sz_dtype == SZO_BF16, mx, t->w_map, P, sc.n_pairs, st);
 }
 
@@ -718,6 +734,7 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
   for (int i = 0; i < 5; ++i) P.tail_kb[i] = sc.tail_kb[i];
   P.partial = static_cast<float*>(tail);
   P.tickets = t->tickets;
+  SZO_TRY(refresh_tickets(t, st));
   const size_t y_elt = (y_dtype == SZO_F32) ? 4 : 2;
   const int n_sets = S_second != nullptr ? 2 : 1;
   for (int set = 0; set < n_sets; ++set) {
@@ -767,3 +784,22 @@ szo_status linear_fwd_tc(const szo_linear* p, const void* x, int64_t M, const ui
 }
 
 }  // namespace szo
+
+extern "C" szo_status szo_selftest_wait_timeout(double limit_ms, int32_t* gave_up_host, void* stream) {
+  using namespace szo;
+  SZO_REQUIRE(gave_up_host != nullptr, SZO_ERR_INVALID_ARG, "gave_up_host is NULL");
+  SZO_REQUIRE(limit_ms > 0.0 && limit_ms <= 100.0, SZO_ERR_INVALID_ARG, "limit_ms must be in (0, 100]");
+  int dev = 0, khz = 0;
+  SZO_CHECK_CUDA(cudaGetDevice(&dev));
+  SZO_CHECK_CUDA(cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, dev));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int32_t* flag = nullptr;
+  SZO_CHECK_CUDA(cudaMalloc(&flag, sizeof(int32_t)));
+  cudaMemsetAsync(flag, 0, sizeof(int32_t), st);
+  szo_status rc = launch_wait_timeout_selftest(static_cast<long long>(limit_ms * khz), flag, st);
+  if (rc == SZO_OK && (cudaMemcpyAsync(gave_up_host, flag, sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+                       cudaStreamSynchronize(st) != cudaSuccess))
+    rc = fail(SZO_ERR_CUDA, "self-test read-back failed");
+  cudaFree(flag);
+  return rc;
+}

@@ -751,6 +751,32 @@ szo_status launch_tc2(const CUtensorMap& mx, const CUtensorMap& mw, const TcPara
 
 }  // namespace
 
+namespace {
+// One thread waits, with a limit of `limit_cycles` SM cycles, on an mbarrier that nothing ever arrives
+// on: the wait must give up, record SZO_ERR_TIMEOUT in the status word and let the kernel return.
+__global__ void wait_timeout_selftest_kernel(long long limit_cycles, int32_t* status, int32_t* gave_up) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_flag_s;
+  if (threadIdx.x == 0) {
+    abort_flag_s = 0;
+    tc::mbar_init(tc::smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    volatile int* abort_flag = &abort_flag_s;
+    const bool ok = tc::mbar_wait(tc::smem_u32(&bar), 0u, abort_flag, status, 32, limit_cycles);
+    *gave_up = ok ? 0 : 1;
+  }
+}
+}  // namespace
+
+szo_status launch_wait_timeout_selftest(long long limit_cycles, int32_t* gave_up_dev, cudaStream_t st) {
+  int32_t* status = device_status_word();
+  SZO_REQUIRE(status != nullptr, SZO_ERR_CUDA, "no device status word");
+  wait_timeout_selftest_kernel<<<1, 32, 0, st>>>(limit_cycles, status, gave_up_dev);
+  count_launch();
+  SZO_CHECK_LAUNCH("wait_timeout_selftest_kernel");
+  return SZO_OK;
+}
+
 szo_status launch_pair_kernel(bool dequant, bool bf16_tables, const CUtensorMap& mx, const CUtensorMap& mw,
                               const tc::TcParams& P, int n_pairs, cudaStream_t st) {
   if (P.pair_row0 > 0) {

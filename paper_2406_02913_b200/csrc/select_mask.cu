@@ -6,6 +6,8 @@
 // and how many keys equal to T are still needed, (3) an ordered two-level compaction writes, in
 // index order, every i with key > T and the first `need` indices with key == T.
 // Everything stays on the device; the host only reads a NaN flag at the end.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace szo {
@@ -221,6 +223,33 @@ select_write_kernel(const float* __restrict__ scores, int64_t n, const SelectSta
 
 }  // namespace szo
 
+// The selection proper, shared by both entry points: four radix passes on the float bits, per-block
+// counts, their scan, the ordered write; then the NaN flag is read back (synchronises the stream).
+// Every word of scratch that is read has been written by an earlier kernel of this sequence.
+static szo_status run_select(const float* scores, int64_t n, int64_t k, int64_t* idx_out, szo::SelectState* state,
+                             uint32_t* blk_gt, uint32_t* blk_eq, unsigned long long* off_gt, unsigned long long* off_eq,
+                             int64_t nblocks, cudaStream_t st) {
+  using namespace szo;
+  select_init_kernel<<<1, 256, 0, st>>>(state, static_cast<unsigned long long>(k));
+  int64_t hist_blocks = ceil_div(n, kSelBlock * 8);
+  if (hist_blocks > 148 * 8) hist_blocks = 148 * 8;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    select_hist_kernel<<<static_cast<unsigned>(hist_blocks), kSelBlock, 0, st>>>(scores, n, shift, state);
+    select_pick_kernel<<<1, 32, 0, st>>>(state, shift);
+  }
+  select_count_kernel<<<static_cast<unsigned>(nblocks), kSelBlock, 0, st>>>(scores, n, state, blk_gt, blk_eq);
+  select_scan_kernel<<<1, 1024, 0, st>>>(blk_gt, blk_eq, nblocks, off_gt, off_eq);
+  select_write_kernel<<<static_cast<unsigned>(nblocks), kSelBlock, 0, st>>>(scores, n, state, off_gt, off_eq,
+                                                                          idx_out, k);
+  count_launch(12);
+  SZO_CHECK_LAUNCH("select_mask kernels");
+  int32_t nan_flag = 0;
+  SZO_CHECK_CUDA(cudaMemcpyAsync(&nan_flag, &state->nan_flag, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  SZO_CHECK_CUDA(cudaStreamSynchronize(st));
+  SZO_REQUIRE(nan_flag == 0, SZO_ERR_NONFINITE, "scores contain NaN");
+  return SZO_OK;
+}
+
 extern "C" szo_status szo_select_mask(const float* scores, int64_t n, int64_t k, int64_t* idx_out,
                                       void* workspace, size_t* workspace_bytes, void* stream) {
   using namespace szo;
@@ -249,24 +278,7 @@ extern "C" szo_status szo_select_mask(const float* scores, int64_t n, int64_t k,
   unsigned long long* off_gt = reinterpret_cast<unsigned long long*>(ws + state_bytes + 2 * cnt_bytes);
   unsigned long long* off_eq = reinterpret_cast<unsigned long long*>(ws + state_bytes + 2 * cnt_bytes + off_bytes);
 
-  select_init_kernel<<<1, 256, 0, st>>>(state, static_cast<unsigned long long>(k));
-  int64_t hist_blocks = ceil_div(n, kSelBlock * 8);
-  if (hist_blocks > 148 * 8) hist_blocks = 148 * 8;
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    select_hist_kernel<<<static_cast<unsigned>(hist_blocks), kSelBlock, 0, st>>>(scores, n, shift, state);
-    select_pick_kernel<<<1, 32, 0, st>>>(state, shift);
-  }
-  select_count_kernel<<<static_cast<unsigned>(nblocks), kSelBlock, 0, st>>>(scores, n, state, blk_gt, blk_eq);
-  select_scan_kernel<<<1, 1024, 0, st>>>(blk_gt, blk_eq, nblocks, off_gt, off_eq);
-  select_write_kernel<<<static_cast<unsigned>(nblocks), kSelBlock, 0, st>>>(scores, n, state, off_gt, off_eq,
-                                                                          idx_out, k);
-  count_launch(12);
-  SZO_CHECK_LAUNCH("select_mask kernels");
-  int32_t nan_flag = 0;
-  SZO_CHECK_CUDA(cudaMemcpyAsync(&nan_flag, &state->nan_flag, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-  SZO_CHECK_CUDA(cudaStreamSynchronize(st));
-  SZO_REQUIRE(nan_flag == 0, SZO_ERR_NONFINITE, "scores contain NaN");
-  return SZO_OK;
+  return run_select(scores, n, k, idx_out, state, blk_gt, blk_eq, off_gt, off_eq, nblocks, st);
 }
 
 
@@ -284,9 +296,13 @@ static __device__ __align__(256) unsigned char g_select_scratch[kStaticScratchBy
 
 // Device address of g_select_scratch on the current device, looked up once per device.  In host
 // code the symbol name is only a handle; the address a kernel can use comes from
-// cudaGetSymbolAddress, with the device that will run the kernels current.
+// cudaGetSymbolAddress, with the device that will run the kernels current.  The cached address
+// belongs to the device's primary context and is valid as long as that context lives (a
+// cudaDeviceReset in the same process would make it stale).
 static szo_status static_scratch_address(unsigned char** out) {
   static unsigned char* cached[64] = {nullptr};
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
   int dev = 0;
   SZO_CHECK_CUDA(cudaGetDevice(&dev));
   SZO_REQUIRE(dev >= 0 && dev < 64, SZO_ERR_UNSUPPORTED, "device ordinal %d not supported", dev);
@@ -325,22 +341,5 @@ extern "C" szo_status szo_select_mask_static(const float* scores, int64_t n, int
   unsigned long long* off_eq = off_gt + kStaticBlocks;
   // The array keeps whatever the previous call left: the state and histogram are cleared here, the
   // per-block counts and offsets of the nblocks in use are fully overwritten before they are read.
-  select_init_kernel<<<1, 256, 0, st>>>(state, static_cast<unsigned long long>(k));
-  int64_t hist_blocks = ceil_div(n, kSelBlock * 8);
-  if (hist_blocks > 148 * 8) hist_blocks = 148 * 8;
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    select_hist_kernel<<<static_cast<unsigned>(hist_blocks), kSelBlock, 0, st>>>(scores, n, shift, state);
-    select_pick_kernel<<<1, 32, 0, st>>>(state, shift);
-  }
-  select_count_kernel<<<static_cast<unsigned>(nblocks), kSelBlock, 0, st>>>(scores, n, state, blk_gt, blk_eq);
-  select_scan_kernel<<<1, 1024, 0, st>>>(blk_gt, blk_eq, nblocks, off_gt, off_eq);
-  select_write_kernel<<<static_cast<unsigned>(nblocks), kSelBlock, 0, st>>>(scores, n, state, off_gt, off_eq,
-                                                                          idx_out, k);
-  count_launch(12);
-  SZO_CHECK_LAUNCH("select_mask kernels (static scratch)");
-  int32_t nan_flag = 0;
-  SZO_CHECK_CUDA(cudaMemcpyAsync(&nan_flag, &state->nan_flag, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-  SZO_CHECK_CUDA(cudaStreamSynchronize(st));
-  SZO_REQUIRE(nan_flag == 0, SZO_ERR_NONFINITE, "scores contain NaN");
-  return SZO_OK;
+  return run_select(scores, n, k, idx_out, state, blk_gt, blk_eq, off_gt, off_eq, nblocks, st);
 }

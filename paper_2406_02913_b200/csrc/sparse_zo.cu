@@ -45,8 +45,8 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
 //   ln u1:  u1 = f 2^e with f in [sqrt(1/2), sqrt(2)), s = f - 1, ln(1+s) = s - s^2/2 + s^3 P(s)
 //   cos(2 pi u2) = -cos(pi y), y = 2 u2 - 1; with a = |y| and b = min(a, 1 - a) in [0, 1/2]:
 //                  cos(pi a) = +-cos(pi b) = +-C(b^2)
-// P (degree 7) and C (degree 6) are least-squares fits on Chebyshev nodes (fit_gauss_polys.py, which
-// also checks |z - z_fp64| <= 5e-7 max(1,|z|) for this arithmetic).
+// P (degree 7) and C (degree 6) are least-squares fits on Chebyshev nodes; tests/test_gauss_polynomials.py
+// reads the coefficients below, refits them and checks |z - z_fp64| <= 5e-7 max(1,|z|) for this arithmetic.
 __device__ __forceinline__ float gaussian_from_words(uint32_t r0, uint32_t r1) {
   const float u1 = static_cast<float>((r0 >> 8) + 1u) * 5.9604644775390625e-8f;
   const int bits = __float_as_int(u1);
@@ -100,7 +100,7 @@ constexpr int kAxpyPer = 8;
 // kKeepZ: also store z_j to z_out[j], for the later passes of the same (seed, step).
 template <bool kKeepZ>
 __global__ void __launch_bounds__(256)
-sparse_axpy_kernel(const float* __restrict__ S_in, float* __restrict__ S_out,
+sparse_axpy_kernel(const float* S_in, float* S_out,      // may alias (in-place passes): no __restrict__
                    const int64_t* __restrict__ idx, int64_t k, int64_t idx_base, const PhiloxKeys K,
                    uint32_t step_lo, uint32_t step_hi, ScaleArg sa, float* __restrict__ z_out) {
   const float scale = resolve_scale(sa);
@@ -146,7 +146,7 @@ sparse_axpy_kernel(const float* __restrict__ S_in, float* __restrict__ S_out,
 // memory-level parallelism per thread is what fills the pipe that quickly).
 constexpr int kKeptUnroll = 4;
 __global__ void __launch_bounds__(256)
-sparse_axpy_kept_kernel(const float* __restrict__ S_in, float* __restrict__ S_out, const float* __restrict__ z,
+sparse_axpy_kept_kernel(const float* S_in, float* S_out /* may alias S_in */, const float* __restrict__ z,
                         int64_t k, ScaleArg sa) {
   const float scale = resolve_scale(sa);
   const int64_t quads = k / 4;

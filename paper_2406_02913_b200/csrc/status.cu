@@ -1,9 +1,17 @@
 // Status strings, thread-local error text and the device status word.
+#include <atomic>
+#include <mutex>
+
 #include "common.cuh"
 
 namespace szo {
 
 thread_local int64_t g_launch_count = 0;
+
+// Bumped whenever szo_device_status reads a non-zero status word: a kernel that gave up may have left
+// the self-resetting K-split tickets of its plan non-zero; plans compare their own copy of this
+// counter before a launch and clear their tickets when it has moved (gemm_tc.cu).
+std::atomic<uint64_t> g_abort_epoch{0};
 
 char* last_error_buffer() {
   static thread_local char buf[512] = {0};
@@ -18,10 +26,14 @@ szo_status fail(szo_status code, const char* fmt, ...) {
   return code;
 }
 
+uint64_t abort_epoch() { return g_abort_epoch.load(); }
+
 int32_t* device_status_word() {
   static int32_t* words[64] = {nullptr};
+  static std::mutex mu;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
   if (!words[dev]) {
     int32_t* p = nullptr;
     if (cudaMalloc(&p, sizeof(int32_t)) != cudaSuccess) return nullptr;
@@ -61,6 +73,7 @@ szo_status szo_device_status(int32_t* status_host) {
   SZO_CHECK_CUDA(cudaDeviceSynchronize());
   SZO_CHECK_CUDA(cudaMemcpy(status_host, w, sizeof(int32_t), cudaMemcpyDeviceToHost));
   SZO_CHECK_CUDA(cudaMemset(w, 0, sizeof(int32_t)));
+  if (*status_host != 0) szo::g_abort_epoch.fetch_add(1);
   return SZO_OK;
 }
 

@@ -115,7 +115,7 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 // that feed the tensor core; the SM cycle counter bounds the wait (kWaitLimitCycles is about two
 // seconds at 2 GHz).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
-                                          unsigned backoff_ns = 32) {
+                                          unsigned backoff_ns = 32, long long limit_cycles = kWaitLimitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   int polls = 0;
@@ -124,7 +124,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try_wait(bar, parity)) return true;
     if ((++polls & 1023) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitLimitCycles) {
+      if (clock64() - t0 > limit_cycles) {
         *abort_flag = 1;
         atomicExch(status, static_cast<int32_t>(SZO_ERR_TIMEOUT));
         return false;
@@ -225,5 +225,8 @@ __device__ __forceinline__ uint4 dequant_word(uint32_t w, float2 p) {
 // dequant == false: dense bf16 weight through mw (one matrix only).
 szo_status launch_pair_kernel(bool dequant, bool bf16_tables, const CUtensorMap& mx, const CUtensorMap& mw,
                               const tc::TcParams& P, int n_pairs, cudaStream_t st);
+
+// Self-test of the bounded waits (gemm_tc2.cu): *gave_up_dev = 1 when the wait expired.
+szo_status launch_wait_timeout_selftest(long long limit_cycles, int32_t* gave_up_dev, cudaStream_t st);
 
 }  // namespace szo

@@ -183,3 +183,25 @@ def test_select_mask_ties_zero_k_and_nan(B):
     assert ei.value.name == "SZO_ERR_NONFINITE"
     with pytest.raises(B.SzoError):
         B.szo_select_mask(torch.from_numpy(same).cuda(), same.size + 1)
+
+
+def test_bounded_wait_gives_up_and_reports_a_timeout(B):
+    """A wait inside a kernel that nothing will ever satisfy (a barrier without an arrival, limit 2 ms):
+    the kernel returns, the device status word holds SZO_ERR_TIMEOUT once, and the library keeps
+    working afterwards (the K-split tickets of every plan are cleared before its next launch)."""
+    import numpy as np
+    from oracle import szo_oracle as so
+    from tests.test_gpu_linear import make_case, max_rel, upload
+    assert B.device_status() == 0
+    c = make_case(512, 4096, 128, "bf16", 16, 1e-3, seed=5)           # every tile split along K: uses tickets
+    plan, x, S = upload(B, c)
+    ref = so.linear_fwd(c["x"], c["deq"], c["idx"], c["S"], c["bias"])
+    xb = x.to(torch.bfloat16)
+    y0 = plan.fwd(xb, S, B.MODE_SPARSE_ADD, torch.float32).cpu().numpy()
+    assert B.selftest_wait_timeout(2.0) == 1
+    assert B.device_status() == -8
+    assert B.device_status() == 0
+    y1 = plan.fwd(xb, S, B.MODE_SPARSE_ADD, torch.float32).cpu().numpy()
+    assert np.array_equal(y0, y1) and max_rel(y1, ref) < 5e-3
+    assert B.device_status() == 0
+    plan.close()

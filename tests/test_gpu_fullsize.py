@@ -330,3 +330,97 @@ def test_two_opt_width_layers_relu_in_the_epilogue(B):
     assert abs(0.5 * (fp + fm) - f_seq) <= 1e-3 * abs(f_seq)
     for m in (m_dual, m_seq, m_ref):
         m.close()
+
+
+def test_one_full_width_layer_against_the_oracle(B):
+    """One decoder layer at the Llama-2-7B width (d 4096, 32 heads, d_ff 11008, vocab 32000, int4 G=128,
+    0.1 % mask) on 2 x 32 tokens, a size the fp64 oracle still runs: both loss kinds and the projected
+    gradient of a step against the oracle itself, on the fp32 validation path and on the bf16
+    tensor-core path in the paired form (the kernels and the launch form of the 7B-shape workload)."""
+    from oracle import model_oracle as mo
+    from tests.fixtures import DecoderFixture
+    fx = DecoderFixture("llama2_7b", seed=4, mask="random", B=2, S=32, n_layers=1)
+    om = fx.oracle_model()
+    toks = fx.batch(0)
+    labels = wl.binary_labels(fx.B, 4, 0)
+    cand = np.array([9906, 13], np.int32)
+    d = lambda a: torch.from_numpy(a).cuda()
+    t = fx.gpu_tensors(torch, None)
+    eps, lr = 1e-3, 1e-6
+    for kind, loss_kind in (("lm", B.LOSS_LM), ("cls2", B.LOSS_CLS2)):
+        ref_model = fx.oracle_model()
+        f0 = ref_model.loss(ref_model.S, toks, kind, labels, cand)
+        fp, fm, g = mo.zo_step(ref_model, toks, 1234, 0, eps, lr, kind, labels, cand)
+        # bf16 path: 1e-3 for the loss averaged over 62 positions; the 2-candidate loss of TWO sequences
+        # reads a logit difference of standard deviation 0.02 sqrt(2 * 4096) = 1.8 (random-init head at
+        # this width) that carries ~6e-3 of relative bf16 noise, |dL/dlogit| <= 1/2: bounded by 1.5e-2
+        # (tests/test_gpu_paired.py holds 1e-3 for this loss kind over 64 sequences)
+        for act, mode, ltol in ((B.SZO_F32, B.MODE_FP32_VALIDATE, 5e-6), (B.SZO_BF16, B.MODE_PAIRED, 1e-3 if kind == "lm" else 1.5e-2)):
+            S = d(fx.S_init.copy())
+            m = B.Model(fx.shape, fx.names, t, S, act_dtype=act, linear_mode=mode, loss_kind=loss_kind,
+                        max_batch=fx.B, max_seq=fx.S)
+            got0 = m.loss(d(toks), d(labels), d(cand)).item()
+            out = m.zo_step(d(toks), 1234, 0, eps, lr, d(labels), d(cand)).cpu().numpy()
+            assert abs(got0 - f0) <= ltol * abs(f0), (kind, mode, got0, f0)
+            assert abs(out[0] - fp) <= ltol * abs(fp) and abs(out[1] - fm) <= ltol * abs(fm), (kind, mode, out, fp, fm)
+            if mode == B.MODE_FP32_VALIDATE:
+                assert abs(out[2] - g) <= 1e-3 * abs(g) + 0.25 * float(np.spacing(np.float32(fp))) / (2 * eps), (kind, out[2], g)
+            else:
+                # one step, no averaging over steps: 5 % of |g| plus 5 % of the scale of g for this model
+                assert abs(out[2] - g) <= 0.05 * abs(g) + 0.05 * abs(fp) * 0.1, (kind, out[2], g)
+            assert B.device_status() == 0
+            m.close()
+
+
+def test_two_full_width_layers_paired_form_in_the_bench_configuration(B):
+    """The step bench.py times (paired form, 16 x 256 tokens, 2-candidate loss) on two full-width layers:
+    the fp64 oracle cannot run this size, so the projected gradient of the bf16 tensor-core path is held
+    against the library's own fp32 validation path (which the smaller tests pin to the oracle), over
+    four steps with different z; the two-forward mode is run beside it for the record."""
+    shape = dict(wl.MODEL_SHAPES["llama2_7b"], n_layers=2)
+    tensors, S_all = wl.device_decoder_tensors(shape, seed=5)
+    names = wl.linear_names(shape)
+    Bn, S = 16, 256
+    toks = torch.from_numpy(wl.token_batch(shape["vocab"], Bn, S, 5, wl.PURPOSE_TRAIN_BATCH, 0)).cuda()
+    labs = torch.from_numpy(wl.binary_labels(Bn, 5, 0)).cuda()
+    cand = torch.tensor([9906, 13], dtype=torch.int32, device="cuda")
+    res = {}
+    for name, act, mode in (("fp32", B.SZO_F32, B.MODE_FP32_VALIDATE), ("paired", B.SZO_BF16, B.MODE_PAIRED),
+                            ("sparse_add", B.SZO_BF16, B.MODE_SPARSE_ADD)):
+        Sm = S_all.clone()
+        m = B.Model(shape, names, tensors, Sm, act_dtype=act, linear_mode=mode, loss_kind=B.LOSS_CLS2,
+                    max_batch=Bn, max_seq=S)
+        rows = []
+        for step in range(4):
+            Sm.copy_(S_all)
+            rows.append(m.zo_step(toks, 1234, step, 1e-3, 0.0, labs, cand).cpu().numpy().copy())
+        assert B.device_status() == 0
+        m.close()
+        res[name] = np.array(rows)
+    g_ref, g_p, g_sa = res["fp32"][:, 2], res["paired"][:, 2], res["sparse_add"][:, 2]
+    rms = np.sqrt(np.mean(g_ref ** 2))
+    print("G_FULLWIDTH ref", g_ref, "paired", g_p, "sparse_add", g_sa)
+    assert np.max(np.abs(res["paired"][:, :2] - res["fp32"][:, :2]) / res["fp32"][:, :2]) <= 1.5e-2
+    assert np.sqrt(np.mean((g_p - g_ref) ** 2)) <= 0.05 * rms
+    assert np.all(np.sign(g_p) == np.sign(g_ref))
+
+
+def test_select_mask_at_the_largest_tensor_of_the_workloads(B):
+    """n = 104 857 600 scores (the fc1 matrix of the OPT-13B shape), k = floor(1e-3 n): the mask against
+    Definition 3 restated with a partition instead of a sort (threshold = k-th largest score; every index
+    above it, then the lowest indices equal to it), bit-exact."""
+    n = 20480 * 5120
+    k = n // 1000
+    g = wl.rng(11, wl.PURPOSE_SCORES, 0)
+    scores = np.empty(n, np.float32)
+    for i in range(0, n, 1 << 24):                              # squared Student-t(3) draws, in chunks
+        m = min(1 << 24, n - i)
+        t = g.standard_normal(m) / np.sqrt(g.chisquare(3.0, m) / 3.0)
+        scores[i:i + m] = np.round((t * t).astype(np.float32), 3)       # rounding makes ties at the threshold likely
+    thr = np.partition(scores, n - k)[n - k]
+    above = np.flatnonzero(scores > thr)
+    equal = np.flatnonzero(scores == thr)[:k - above.size]
+    ref = np.sort(np.concatenate([above, equal]))
+    assert ref.size == k
+    got = B.szo_select_mask(torch.from_numpy(scores).cuda(), k).cpu().numpy()
+    assert np.array_equal(got, ref)
