@@ -303,6 +303,22 @@ szo_status szo_model_zo_step(szo_model_t* m, const int32_t* tokens, const int32_
                              const int32_t* cand, int32_t B, int32_t S, uint64_t seed,
                              uint64_t step, float eps, float lr, double* f_plus_dev,
                              double* f_minus_dev, double* g_dev, void* stream);
+/* The step in two halves, for data-parallel replicas (Definition 1 evaluates f on a batch: replicas that
+ * hold the same weights, mask and S and use the same (seed, step) draw the same z, evaluate f+ and f-
+ * on their own share of the batch and need to exchange only sums of losses before each applies the
+ * identical update of Definition 2).
+ *   szo_model_zo_losses: draws and keeps z, evaluates both losses on this replica's B sequences, leaves S
+ *     where the +eps, -2 eps, +eps sequence leaves it, and writes sums_dev[3] (fp64, device) =
+ *     (sum of the per-position losses of f+, the same for f-, number of positions).
+ *   szo_model_zo_apply: takes sums_dev[3] ADDED UP OVER ALL REPLICAS (the caller's all-reduce: 24 bytes;
+ *     with one replica, its own sums), forms f+- = sum / count, g = (f+ - f-)/(2 eps) and
+ *     S -= lr g z with the kept z.  It must follow a szo_model_zo_losses on the same model.
+ * szo_model_zo_step is the first followed by the second on one replica. */
+szo_status szo_model_zo_losses(szo_model_t* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand,
+                               int32_t B, int32_t S, uint64_t seed, uint64_t step, float eps, double* sums_dev,
+                               void* stream);
+szo_status szo_model_zo_apply(szo_model_t* m, float eps, float lr, const double* sums_dev, double* f_plus_dev,
+                              double* f_minus_dev, double* g_dev, void* stream);
 /* Same step through HOST buffers: copies tokens (and labels, cand) to the device, runs the step
  * and copies (f+, f-, g) back into out3_host[3]; synchronises the stream. */
 szo_status szo_model_zo_step_host(szo_model_t* m, const int32_t* tokens_host,

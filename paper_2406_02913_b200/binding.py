@@ -104,6 +104,10 @@ _SIGS = {
     "szo_model_zo_step": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                       C.c_int32, C.c_uint64, C.c_uint64, C.c_float, C.c_float,
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "szo_model_zo_losses": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                        C.c_uint64, C.c_uint64, C.c_float, C.c_void_p, C.c_void_p]),
+    "szo_model_zo_apply": (C.c_int32, [C.c_void_p, C.c_float, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
+                                       C.c_void_p, C.c_void_p]),
     "szo_model_zo_step_host": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                            C.c_int32, C.c_uint64, C.c_uint64, C.c_float, C.c_float,
                                            C.c_void_p, C.c_void_p]),
@@ -375,6 +379,23 @@ class Model:
         _check(lib().szo_model_zo_step(self.h, _ptr(tokens), _ptr(labels), _ptr(cand), B, S, seed, step,
                                        eps, lr, sc[0:1].data_ptr(), sc[1:2].data_ptr(),
                                        sc[2:3].data_ptr(), _stream()))
+        return sc[:3]
+
+    def zo_losses(self, tokens, seed, step, eps, labels=None, cand=None, sums=None) -> torch.Tensor:
+        """First half of a step on this replica's share of the batch: returns the device tensor
+        (sum of losses of f+, of f-, number of positions) (fp64 [3]); z stays in the model."""
+        B, S = tokens.shape
+        if sums is None:
+            sums = torch.zeros(3, dtype=torch.float64, device=self.S_all.device)
+        _check(lib().szo_model_zo_losses(self.h, _ptr(tokens), _ptr(labels), _ptr(cand), B, S, seed, step, eps,
+                                         _ptr(sums), _stream()))
+        return sums
+
+    def zo_apply(self, eps, lr, sums) -> torch.Tensor:
+        """Second half: `sums` added up over all replicas; returns the device tensor (f+, f-, g)."""
+        sc = self._scalars
+        _check(lib().szo_model_zo_apply(self.h, eps, lr, _ptr(sums), sc[0:1].data_ptr(), sc[1:2].data_ptr(),
+                                        sc[2:3].data_ptr(), _stream()))
         return sc[:3]
 
     def zo_step_host(self, tokens_host, seed, step, eps, lr, labels_host=None, cand_host=None):

@@ -626,6 +626,19 @@ __global__ void __launch_bounds__(1024) mean_f64_kernel(const double* __restrict
   if (threadIdx.x == 0) *out = s[0] / denom;
 }
 
+// sums = (f+ * count, f- * count, count): what data-parallel replicas add up
+__global__ void loss_sums_kernel(const double* __restrict__ fp, const double* __restrict__ fm, double count,
+                                 double* __restrict__ sums) {
+  sums[0] = *fp * count;
+  sums[1] = *fm * count;
+  sums[2] = count;
+}
+// (f+, f-) = (sums[0], sums[1]) / sums[2]
+__global__ void loss_means_kernel(const double* __restrict__ sums, double* __restrict__ fp, double* __restrict__ fm) {
+  *fp = sums[0] / sums[2];
+  *fm = sums[1] / sums[2];
+}
+
 __global__ void offset_eid_kernel(const int32_t* __restrict__ eid, int64_t n, int32_t off, int32_t* __restrict__ out) {
   const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i < n) out[i] = eid[i] + off;
@@ -675,6 +688,7 @@ struct szo_model {
   int32_t *d_tokens = nullptr, *d_labels = nullptr, *d_cand = nullptr;
   double* d_scalars = nullptr;
   int64_t last_launches = 0;
+  bool z_valid = false;         // zkept holds the z of the last szo_model_zo_losses, not yet consumed
   std::vector<void*> owned;
   // measurement aid: CUDA events around every decoder-block linear launch
   bool timing = false;
@@ -1263,14 +1277,11 @@ szo_status szo_model_loss(szo_model_t* m, const int32_t* tokens, const int32_t* 
   return run_loss(m, tokens, labels, cand, B, S, S_vals ? S_vals : m->S_all, loss_dev, static_cast<cudaStream_t>(stream));
 }
 
-szo_status szo_model_zo_step(szo_model_t* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand,
-                             int32_t B, int32_t S, uint64_t seed, uint64_t step, float eps, float lr,
-                             double* f_plus_dev, double* f_minus_dev, double* g_dev, void* stream) {
-  SZO_TRY(check_batch(m, tokens, labels, cand, B, S));
-  SZO_REQUIRE(f_plus_dev && f_minus_dev && g_dev, SZO_ERR_INVALID_ARG, "NULL output scalar");
-  SZO_REQUIRE(eps != 0.f, SZO_ERR_INVALID_ARG, "eps == 0");
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int64_t before = g_launch_count;
+// First half of a step: z is drawn (and kept), both perturbed losses are evaluated, S is back where the
+// in-place +eps, -2 eps, +eps sequence leaves it.
+static szo_status zo_losses_impl(szo_model* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand,
+                                 int32_t B, int32_t S, uint64_t seed, uint64_t step, float eps, double* f_plus_dev,
+                                 double* f_minus_dev, cudaStream_t st) {
   const int64_t k = m->k_total;
   float* Sv = m->S_all;
   ScaleArg sa{eps, 0.f, 0.f, nullptr, nullptr};
@@ -1283,12 +1294,7 @@ szo_status szo_model_zo_step(szo_model_t* m, const int32_t* tokens, const int32_
     SZO_TRY(launch_sparse_axpy_kept(Sv, Sv, m->zkept, k, sa, st));
     sa.scale = eps;
     SZO_TRY(launch_sparse_axpy_kept(Sv, Sv, m->zkept, k, sa, st));
-    SZO_TRY(run_loss_paired(m, tokens, labels, cand, B, S, Sv, m->zkept, eps, f_plus_dev, f_minus_dev, st));
-    SZO_TRY(szo_projected_gradient(f_plus_dev, f_minus_dev, eps, g_dev, stream));
-    ScaleArg su3{0.f, lr, eps, f_plus_dev, f_minus_dev};
-    SZO_TRY(launch_sparse_axpy_kept(Sv, Sv, m->zkept, k, su3, st));
-    m->last_launches = g_launch_count - before;
-    return SZO_OK;
+    return run_loss_paired(m, tokens, labels, cand, B, S, Sv, m->zkept, eps, f_plus_dev, f_minus_dev, st);
   }
   if (dual_forward_applies(m, static_cast<int64_t>(B) * S)) {
     // both forwards side by side: the same arithmetic on S as the in-place sequence below
@@ -1298,26 +1304,71 @@ szo_status szo_model_zo_step(szo_model_t* m, const int32_t* tokens, const int32_
     SZO_TRY(launch_sparse_axpy_kept(m->Splus, m->Sminus, m->zkept, k, sa, st));               // S- = S+ - 2 eps z
     sa.scale = eps;
     SZO_TRY(launch_sparse_axpy_kept(m->Sminus, Sv, m->zkept, k, sa, st));                     // S = S- + eps z
-    SZO_TRY(run_loss_t<__nv_bfloat16>(m, tokens, labels, cand, B, S, m->Splus, f_plus_dev, st, m->Sminus,
-                                      f_minus_dev));                                          // f+, f-
-    SZO_TRY(szo_projected_gradient(f_plus_dev, f_minus_dev, eps, g_dev, stream));             // g
-    ScaleArg su2{0.f, lr, eps, f_plus_dev, f_minus_dev};
-    SZO_TRY(launch_sparse_axpy_kept(Sv, Sv, m->zkept, k, su2, st));                           // S -= lr g z
-    m->last_launches = g_launch_count - before;
-    return SZO_OK;
+    return run_loss_t<__nv_bfloat16>(m, tokens, labels, cand, B, S, m->Splus, f_plus_dev, st, m->Sminus, f_minus_dev);
   }
-  // z is generated once per step (first pass) and kept: the other three passes stream it
+  // z is generated once per step (first pass) and kept: the other passes stream it
   SZO_TRY(launch_sparse_axpy(Sv, Sv, m->gidx, k, 0, seed, step, sa, st, m->zkept));       // S += eps z
   SZO_TRY(run_loss(m, tokens, labels, cand, B, S, Sv, f_plus_dev, st));                   // f+
   sa.scale = -2.0f * eps;
   SZO_TRY(launch_sparse_axpy_kept(Sv, Sv, m->zkept, k, sa, st));                          // S -= 2 eps z
   SZO_TRY(run_loss(m, tokens, labels, cand, B, S, Sv, f_minus_dev, st));                  // f-
   sa.scale = eps;
-  SZO_TRY(launch_sparse_axpy_kept(Sv, Sv, m->zkept, k, sa, st));                          // S += eps z
-  SZO_TRY(szo_projected_gradient(f_plus_dev, f_minus_dev, eps, g_dev, stream));           // g
+  return launch_sparse_axpy_kept(Sv, Sv, m->zkept, k, sa, st);                            // S += eps z
+}
+
+// Second half: g from the two losses, then S -= lr g z with the kept z.
+static szo_status zo_apply_impl(szo_model* m, float eps, float lr, const double* f_plus_dev, const double* f_minus_dev,
+                                double* g_dev, cudaStream_t st) {
+  SZO_TRY(szo_projected_gradient(f_plus_dev, f_minus_dev, eps, g_dev, st));
   ScaleArg su{0.f, lr, eps, f_plus_dev, f_minus_dev};
-  SZO_TRY(launch_sparse_axpy_kept(Sv, Sv, m->zkept, k, su, st));                          // S -= lr g z
+  return launch_sparse_axpy_kept(m->S_all, m->S_all, m->zkept, m->k_total, su, st);
+}
+
+szo_status szo_model_zo_step(szo_model_t* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand,
+                             int32_t B, int32_t S, uint64_t seed, uint64_t step, float eps, float lr,
+                             double* f_plus_dev, double* f_minus_dev, double* g_dev, void* stream) {
+  SZO_TRY(check_batch(m, tokens, labels, cand, B, S));
+  SZO_REQUIRE(f_plus_dev && f_minus_dev && g_dev, SZO_ERR_INVALID_ARG, "NULL output scalar");
+  SZO_REQUIRE(eps != 0.f, SZO_ERR_INVALID_ARG, "eps == 0");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t before = g_launch_count;
+  SZO_TRY(zo_losses_impl(m, tokens, labels, cand, B, S, seed, step, eps, f_plus_dev, f_minus_dev, st));
+  SZO_TRY(zo_apply_impl(m, eps, lr, f_plus_dev, f_minus_dev, g_dev, st));
+  m->z_valid = false;
   m->last_launches = g_launch_count - before;
+  return SZO_OK;
+}
+
+szo_status szo_model_zo_losses(szo_model_t* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand,
+                               int32_t B, int32_t S, uint64_t seed, uint64_t step, float eps, double* sums_dev,
+                               void* stream) {
+  SZO_TRY(check_batch(m, tokens, labels, cand, B, S));
+  SZO_REQUIRE(sums_dev != nullptr, SZO_ERR_INVALID_ARG, "sums_dev is NULL");
+  SZO_REQUIRE(eps != 0.f, SZO_ERR_INVALID_ARG, "eps == 0");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t before = g_launch_count;
+  SZO_TRY(zo_losses_impl(m, tokens, labels, cand, B, S, seed, step, eps, m->d_scalars, m->d_scalars + 1, st));
+  const double count = m->cfg.loss_kind == 0 ? static_cast<double>(B) * (S - 1) : static_cast<double>(B);
+  loss_sums_kernel<<<1, 1, 0, st>>>(m->d_scalars, m->d_scalars + 1, count, sums_dev);
+  count_launch();
+  SZO_CHECK_LAUNCH("loss_sums_kernel");
+  m->z_valid = true;
+  m->last_launches = g_launch_count - before;
+  return SZO_OK;
+}
+
+szo_status szo_model_zo_apply(szo_model_t* m, float eps, float lr, const double* sums_dev, double* f_plus_dev,
+                              double* f_minus_dev, double* g_dev, void* stream) {
+  SZO_REQUIRE(m != nullptr, SZO_ERR_INVALID_ARG, "model is NULL");
+  SZO_REQUIRE(sums_dev && f_plus_dev && f_minus_dev && g_dev, SZO_ERR_INVALID_ARG, "NULL scalar pointer");
+  SZO_REQUIRE(eps != 0.f, SZO_ERR_INVALID_ARG, "eps == 0");
+  SZO_REQUIRE(m->z_valid, SZO_ERR_INVALID_ARG, "szo_model_zo_apply needs the z kept by a preceding szo_model_zo_losses");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  loss_means_kernel<<<1, 1, 0, st>>>(sums_dev, f_plus_dev, f_minus_dev);
+  count_launch();
+  SZO_CHECK_LAUNCH("loss_means_kernel");
+  SZO_TRY(zo_apply_impl(m, eps, lr, f_plus_dev, f_minus_dev, g_dev, st));
+  m->z_valid = false;
   return SZO_OK;
 }
 

@@ -249,3 +249,36 @@ def test_degenerate_masks(B, name, rho):
             assert np.allclose(S.cpu().numpy(), om.S, rtol=0, atol=2e-7)
         assert B.device_status() == 0
         m.close()
+
+
+@pytest.mark.parametrize("act,mode", [("f32", "fp32"), ("bf16", "paired")])
+def test_two_half_batches_through_losses_and_apply_equal_the_full_batch_step(B, tiny, act, mode):
+    """Data-parallel replicas emulated in one process: szo_model_zo_losses on each half of the batch
+    (both from the same S, as two replicas would), the two (sum f+, sum f-, count) added, then
+    szo_model_zo_apply, against szo_model_zo_step on the whole batch.  fp32 validation path: the same
+    per-position losses in another summation order.  Paired bf16 path: the same kernels on other tile
+    shapes, compared at the loss tolerance."""
+    fx = tiny
+    a, md = (B.SZO_F32, B.MODE_FP32_VALIDATE) if mode == "fp32" else (B.SZO_BF16, B.MODE_PAIRED)
+    toks = torch.from_numpy(fx.batch(0)).cuda()
+    eps, lr = 1e-3, 1e-3
+    m_full, S_full, _ = build_gpu(B, fx, a, md)
+    out_full = m_full.zo_step(toks, 1234, 3, eps, lr).cpu().numpy().copy()
+    m_dp, S_dp, _ = build_gpu(B, fx, a, md)
+    S0 = S_dp.clone()
+    sums = torch.zeros(3, dtype=torch.float64, device="cuda")
+    for half in (toks[:2].contiguous(), toks[2:].contiguous()):
+        S_dp.copy_(S0)                                   # every replica starts the step from the same S
+        sums += m_dp.zo_losses(half, 1234, 3, eps)
+    assert float(sums[2]) == fx.B * (fx.S - 1)
+    out_dp = m_dp.zo_apply(eps, lr, sums).cpu().numpy().copy()
+    tol = 1e-12 if mode == "fp32" else 2e-5
+    assert abs(out_dp[0] - out_full[0]) <= tol * abs(out_full[0]) and abs(out_dp[1] - out_full[1]) <= tol * abs(out_full[1])
+    gtol = 1e-8 if mode == "fp32" else 2e-2
+    assert abs(out_dp[2] - out_full[2]) <= gtol * abs(out_full[2]), (out_dp, out_full)
+    assert torch.allclose(S_dp, S_full, rtol=0, atol=1e-9 if mode == "fp32" else abs(lr * out_full[2]) * 0.1)
+    with pytest.raises(B.SzoError):                      # apply without a preceding losses call
+        m_dp.zo_apply(eps, lr, sums)
+    assert B.device_status() == 0
+    m_full.close()
+    m_dp.close()
