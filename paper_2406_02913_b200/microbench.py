@@ -221,7 +221,31 @@ def attention_case(Bn, S, H, Hkv, hd, reps):
                       "tflops_causal": flops / (med * 1e-3) / 1e12}), flush=True)
 
 
-def step_case(name, Bn, S, loss, steps, eps, lr, profile_range=False):
+def paired_case(M, N, K, G, rho, reps):
+    """One linear in the paired form (szo_linear_fwd_paired): M centre rows and M half-difference rows
+    in one call: weight pass, SparseAdd scatter, one tensor-core launch over both kinds of rows, the
+    sparse product pass.  Timed whole, L2 flushed between repetitions."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(0)
+    codes = torch.randint(0, 256, (N, K // 2), generator=g, device="cuda", dtype=torch.uint8)
+    sc = (0.004 + 0.002 * torch.rand(N, K // G, generator=g, device="cuda")).to(torch.bfloat16)
+    ze = (-7.5 * sc.float()).to(torch.bfloat16)
+    nnz = int(rho * N * K)
+    idx = torch.from_numpy(wl.sorted_random_indices(N * K, nnz, seed=1)).cuda()
+    plan = B.Linear(N, K, G, codes, sc, ze, "bf16", idx)
+    S = torch.randn(nnz, generator=g, device="cuda") * 0.02
+    z = torch.randn(nnz, generator=g, device="cuda")
+    row0 = B.paired_row0(M)
+    x = torch.randn(row0 + M, K, generator=g, device="cuda").to(torch.bfloat16)
+    x[row0:] *= 1e-3
+    ms, ms_min = time_call(lambda: plan.fwd_paired(x, M, S, z, 1e-3), reps)
+    flops = 2 * 2 * M * N * K
+    print(json.dumps({"case": "paired_linear", "M": M, "N": N, "K": K, "G": G, "rho": rho, "nnz": nnz, "ms": ms,
+                      "ms_min": ms_min, "tflops_both_row_kinds": flops / ms / 1e9, "device_status": B.device_status()}))
+    plan.close()
+
+
+def step_case(name, Bn, S, loss, steps, eps, lr, profile_range=False, form="paired"):
     """A full ZO step of a whole decoder shape (random-init weights in device memory), timed like
     bench.py: CUDA events around `steps` back-to-back steps after three warm-up steps; the weights
     streamed per forward exceed L2."""
@@ -229,7 +253,8 @@ def step_case(name, Bn, S, loss, steps, eps, lr, profile_range=False):
     tensors, S_all = wl.device_decoder_tensors(shape, seed=0)
     loss_kind = B.LOSS_CLS2 if loss == "cls2" else B.LOSS_LM
     model = B.Model(shape, wl.linear_names(shape), tensors, S_all, act_dtype=B.SZO_BF16,
-                    linear_mode=B.MODE_SPARSE_ADD, loss_kind=loss_kind, max_batch=Bn, max_seq=S)
+                    linear_mode=B.MODE_PAIRED if form == "paired" else B.MODE_SPARSE_ADD, loss_kind=loss_kind,
+                    max_batch=Bn, max_seq=S)
     n = 3 + steps
     toks = [torch.from_numpy(wl.token_batch(shape["vocab"], Bn, S, 0, wl.PURPOSE_TRAIN_BATCH, i)).cuda() for i in range(n)]
     labs = [torch.from_numpy(wl.binary_labels(Bn, 0, i)).cuda() for i in range(n)] if loss == "cls2" else [None] * n
@@ -258,7 +283,7 @@ def step_case(name, Bn, S, loss, steps, eps, lr, profile_range=False):
         if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else 1400.0
     last = model._scalars[:3].cpu().numpy()
     ach = flops / (lin_ms * 1e-3) / 1e12
-    print(json.dumps({"case": "step", "model": name, "batch": Bn, "seq": S, "loss": loss, "k": int(model.k_total),
+    print(json.dumps({"case": "step", "model": name, "form": form, "batch": Bn, "seq": S, "loss": loss, "k": int(model.k_total),
                       "ms_per_step": ms, "steps_per_s": 1e3 / ms, "tokens_per_s": 1e3 / ms * M,
                       "linear_ms_per_step": lin_ms / steps, "linear_launches_per_step": lin_launches / steps,
                       "linear_tflops": ach, "frac_of_sustained_peak": ach / sus,
@@ -269,7 +294,7 @@ def step_case(name, Bn, S, loss, steps, eps, lr, profile_range=False):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["linear", "steady", "sparse", "sweep", "attention", "step"])
+    ap.add_argument("what", choices=["linear", "paired", "steady", "sparse", "sweep", "attention", "step"])
     ap.add_argument("--model", default="mistral_7b", choices=sorted(wl.MODEL_SHAPES))
     ap.add_argument("--batch", type=int, default=8)
     ap.add_argument("--seq", type=int, default=512)
@@ -285,18 +310,22 @@ def main():
     ap.add_argument("--G", type=int, default=128, help="group size; 0: dense bf16 weight; -1: non-uniform 4-bit (table) format")
     ap.add_argument("--rho", type=float, default=1e-3)
     ap.add_argument("--mode", default="sparse_add")
+    ap.add_argument("--form", default="paired", choices=["paired", "sparse_add"],
+                    help="step: both forwards in one paired pass (centre / half-difference), or two bf16 forwards")
     ap.add_argument("--k", type=int, default=6_476_005)
     ap.add_argument("--reps", type=int, default=20)
     a = ap.parse_args()
     B.lib()
     if a.what == "linear":
         linear_case(a.M, a.N, a.K, a.G, a.mode, a.rho, a.reps)
+    elif a.what == "paired":
+        paired_case(a.M, a.N, a.K, a.G, a.rho, a.reps)
     elif a.what == "steady":
         steady_case(a.M, a.N, a.K, a.G, a.mode, a.rho, a.reps)
     elif a.what == "sparse":
         sparse_case(a.k, a.reps)
     elif a.what == "step":
-        step_case(a.model, a.batch, a.seq, a.loss, a.steps, a.eps, a.lr, a.profile_range)
+        step_case(a.model, a.batch, a.seq, a.loss, a.steps, a.eps, a.lr, a.profile_range, a.form)
     elif a.what == "attention":
         attention_case(16, 256, 32, 32, 128, a.reps)
         attention_case(8, 512, 32, 8, 128, a.reps)
