@@ -368,7 +368,11 @@ template <> struct SlabVec<8> { using type = uint4; };
 template <> struct SlabVec<4> { using type = uint2; };
 template <> struct SlabVec<2> { using type = uint32_t; };
 
-// R weight rows per thread (2 when N is even: y is then read and written four bytes per lane)
+// R weight rows per thread (2 when N is even: y is then read and written four bytes per lane).  The rows of
+// a lane are walked one after the other, and a warp runs each walk as long as its longest row: at 4
+// entries per row that is about twice the mean.  Giving lane l the l-th longest and the l-th shortest
+// row of a 64-row group instead (so that lanes finish together) measured 16 % slower: the walks are
+// still separate loops, and the two rows of a lane are then no longer adjacent (two-byte accesses to y).
 template <int TM, int R, typename TY>
 __global__ void __launch_bounds__(TM == 16 ? 1024 : 512) pair_cross_kernel(const CrossArgs a) {
   using V = typename SlabVec<TM>::type;
