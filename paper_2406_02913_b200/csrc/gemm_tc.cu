@@ -248,6 +248,7 @@ struct MatArgs {
   MatSub sub[3];
   int n, nkb, G;
   int64_t K;
+  int64_t ld;                 // row stride of the output buffers in elements (K, or 2 K when eps * Zbar sits beside W)
   int scatter_mode;           // 0: w += S; 1: saved = w, w += S; 2: w = saved + S (second set of sparse values)
 };
 
@@ -276,7 +277,7 @@ __global__ void materialise_kernel(const MatArgs a) {
   const int kb = static_cast<int>(grp - t * nkb4) * 4 + kbo;
   if (kb >= a.nkb) return;
   const uint8_t* src = codes_tiled + (t * a.nkb + kb) * kCodesBytes + r0 * 32 + chunk * 4;
-  __nv_bfloat16* dst = out + (t * kBM + r0) * a.K + kb * kBK + chunk * 8;
+  __nv_bfloat16* dst = out + (t * kBM + r0) * a.ld + kb * kBK + chunk * 8;
   uint32_t w[4];
   if constexpr (kKind == 2) {
     const __nv_bfloat16* lut = s == 0 ? a.sub[0].lut : (s == 1 ? a.sub[1].lut : a.sub[2].lut);
@@ -293,7 +294,7 @@ __global__ void materialise_kernel(const MatArgs a) {
         const uint32_t hi = __ldg(rj + ((w[j] >> (16 + 4 * i)) & 0xFu));
         o[i] = lo | (hi << 16);
       }
-      *reinterpret_cast<uint4*>(dst + static_cast<int64_t>(j) * 32 * a.K) = make_uint4(o[0], o[1], o[2], o[3]);
+      *reinterpret_cast<uint4*>(dst + static_cast<int64_t>(j) * 32 * a.ld) = make_uint4(o[0], o[1], o[2], o[3]);
     }
   } else {
     const int g = (kb * kBK + chunk * 8) / a.G;
@@ -306,7 +307,7 @@ __global__ void materialise_kernel(const MatArgs a) {
     }
 #pragma unroll
     for (int j = 0; j < 4; ++j)
-      *reinterpret_cast<uint4*>(dst + static_cast<int64_t>(j) * 32 * a.K) = dequant_word<kKind == 1>(w[j], p[j]);
+      *reinterpret_cast<uint4*>(dst + static_cast<int64_t>(j) * 32 * a.ld) = dequant_word<kKind == 1>(w[j], p[j]);
   }
 }
 
@@ -322,7 +323,9 @@ __global__ void scatter_add_bf16_kernel(const MatArgs a) {
   const int64_t* idx = s == 0 ? a.sub[0].idx : (s == 1 ? a.sub[1].idx : a.sub[2].idx);
   const float* S = s == 0 ? a.sub[0].S : (s == 1 ? a.sub[1].S : a.sub[2].S);
   __nv_bfloat16* saved = s == 0 ? a.sub[0].saved : (s == 1 ? a.sub[1].saved : a.sub[2].saved);
-  __nv_bfloat16* el = (s == 0 ? a.sub[0].out : (s == 1 ? a.sub[1].out : a.sub[2].out)) + idx[e];
+  const int64_t flat = idx[e];
+  const int64_t row = flat / a.K;
+  __nv_bfloat16* el = (s == 0 ? a.sub[0].out : (s == 1 ? a.sub[1].out : a.sub[2].out)) + row * a.ld + (flat - row * a.K);
   __nv_bfloat16 base;
   if (a.scatter_mode == 2) {
     base = saved[e];              // the element itself is not read: it holds the other set's value
@@ -534,6 +537,22 @@ szo_status pack_cross_records(const int32_t* col, const float* z, float eps, int
 
 namespace {
 
+// Dense form of the sparse product (TcParams::pair_ext): eps * z written as bf16 into the second half
+// [K, 2 K) of the weight rows, which is zero elsewhere.
+__global__ void scatter_z_bf16_kernel(const MatArgs a, float eps) {
+  int64_t e = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (e >= a.sub[a.n - 1].nnz_end) return;
+  int s = 0;
+  if (e >= a.sub[0].nnz_end) s = (a.n > 2 && e >= a.sub[1].nnz_end) ? 2 : 1;
+  if (s > 0) e -= a.sub[s - 1].nnz_end;
+  const int64_t* idx = s == 0 ? a.sub[0].idx : (s == 1 ? a.sub[1].idx : a.sub[2].idx);
+  const float* z = s == 0 ? a.sub[0].S : (s == 1 ? a.sub[1].S : a.sub[2].S);     // the S slot carries z here
+  const int64_t flat = idx[e];
+  const int64_t row = flat / a.K;
+  __nv_bfloat16* el = (s == 0 ? a.sub[0].out : (s == 1 ? a.sub[1].out : a.sub[2].out)) + row * a.ld + a.K + (flat - row * a.K);
+  *el = __float2bfloat16_rn(eps * z[e]);
+}
+
 // SZO_LINEAR_MATERIALISE=0 / 1 switches the form off / on for every M (A/B measurement)
 int materialise_override() {
   static const int v = [] {
@@ -557,13 +576,32 @@ bool tc_use_materialised(const szo_linear* p, int64_t M, bool two_sets) {
   return M >= (two_sets ? 2048 : 4096);
 }
 
-size_t tc_materialised_ws_bytes(const szo_linear* const* plans, int n, int64_t M) {
+size_t tc_materialised_ws_bytes(const szo_linear* const* plans, int n, int64_t M, bool ext) {
   size_t rows = 0;
   for (int i = 0; i < n; ++i) rows += static_cast<size_t>(plans[i]->Npad);
   size_t nnz = 0;
   for (int i = 0; i < n; ++i) nnz += static_cast<size_t>(plans[i]->nnz);
-  return round_up(rows * static_cast<size_t>(plans[0]->K) * sizeof(__nv_bfloat16), 256) +
+  return round_up(rows * static_cast<size_t>(plans[0]->K) * (ext ? 2 : 1) * sizeof(__nv_bfloat16), 256) +
          round_up(nnz * sizeof(__nv_bfloat16), 256) + tc_tail_ws_bound();
+}
+
+// Paired form: where does eps * xc Zbar^T run?  On the CUDA cores (pair_cross_kernel) its cost grows
+// with the number of entries (18.8 ms of a Llama-2-7B-shaped step at 0.1 %, 200 ms of a Mistral-7B-shaped
+// one at 1 %); on the tensor cores it is half the dense flops again whatever the mask.  The break-even
+// is near a density of 0.2 %.  SZO_PAIRED_CROSS=sparse|dense forces either (A/B, tests).
+bool tc_paired_dense_cross(const szo_linear* const* plans, int n) {
+  static const int forced = [] {
+    const char* e = getenv("SZO_PAIRED_CROSS");
+    return e == nullptr ? -1 : (e[0] == 'd' ? 1 : 0);
+  }();
+  double nnz = 0, elems = 0;
+  for (int i = 0; i < n; ++i) {
+    nnz += static_cast<double>(plans[i]->nnz);
+    elems += static_cast<double>(plans[i]->N) * static_cast<double>(plans[i]->K);
+  }
+  if (nnz == 0) return false;
+  if (forced >= 0) return forced == 1;
+  return nnz >= 0.002 * elems;
 }
 
 // Resident form (dense bf16 plans, G == 0).  With nothing to dequantise, the effective weight of a
@@ -587,13 +625,13 @@ bool tc_can_stack(const szo_linear* const* plans, int n) {
   return true;
 }
 
-void tc_resident_bytes(const szo_linear* const* plans, int n, size_t* w_bytes, size_t* saved_bytes) {
+void tc_resident_bytes(const szo_linear* const* plans, int n, size_t* w_bytes, size_t* saved_bytes, bool ext) {
   size_t rows = 0, nnz = 0;
   for (int i = 0; i < n; ++i) {
     rows += static_cast<size_t>(plans[i]->Npad);
     nnz += static_cast<size_t>(plans[i]->nnz);
   }
-  *w_bytes = round_up(rows * static_cast<size_t>(plans[0]->K) * sizeof(__nv_bfloat16), 256);
+  *w_bytes = round_up(rows * static_cast<size_t>(plans[0]->K) * (ext ? 2 : 1) * sizeof(__nv_bfloat16), 256);
   *saved_bytes = round_up(nnz * sizeof(__nv_bfloat16), 256);
 }
 
@@ -608,16 +646,17 @@ __global__ void gather_bf16_kernel(const __nv_bfloat16* __restrict__ W, const in
 // Fills the resident buffers of one launch group: rows [0, N) of every matrix copied from the frozen
 // weight, the padding rows zero, saved[e] = the frozen value at masked position e.
 szo_status tc_resident_init(const szo_linear* const* plans, int n, __nv_bfloat16* W, __nv_bfloat16* saved,
-                            cudaStream_t st) {
+                            cudaStream_t st, bool ext) {
   SZO_REQUIRE(tc_can_stack(plans, n), SZO_ERR_INVALID_ARG, "resident form: dense bf16 plans with one K only");
   int64_t row0 = 0, nnz = 0;
+  const int64_t ld = plans[0]->K * (ext ? 2 : 1);       // ext: columns [K, 2 K) hold eps * Zbar, zero outside the mask
   for (int i = 0; i < n; ++i) {
     const szo_linear* p = plans[i];
-    __nv_bfloat16* dst = W + row0 * p->K;
-    SZO_CHECK_CUDA(cudaMemcpyAsync(dst, p->codes, static_cast<size_t>(p->N) * p->K * sizeof(__nv_bfloat16),
-                                   cudaMemcpyDeviceToDevice, st));
-    if (p->Npad > p->N)
-      SZO_CHECK_CUDA(cudaMemsetAsync(dst + p->N * p->K, 0, static_cast<size_t>(p->Npad - p->N) * p->K * sizeof(__nv_bfloat16), st));
+    __nv_bfloat16* dst = W + row0 * ld;
+    if (ext || p->Npad > p->N)
+      SZO_CHECK_CUDA(cudaMemsetAsync(dst, 0, static_cast<size_t>(p->Npad) * ld * sizeof(__nv_bfloat16), st));
+    SZO_CHECK_CUDA(cudaMemcpy2DAsync(dst, ld * sizeof(__nv_bfloat16), p->codes, p->K * sizeof(__nv_bfloat16),
+                                     p->K * sizeof(__nv_bfloat16), p->N, cudaMemcpyDeviceToDevice, st));
     if (p->nnz > 0) {
       gather_bf16_kernel<<<static_cast<unsigned>(ceil_div(p->nnz, 256)), 256, 0, st>>>(
           static_cast<const __nv_bfloat16*>(p->codes), p->idx, p->nnz, saved + nnz);
@@ -654,8 +693,11 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
     rows += plans[i]->Npad;
     nnz_all += static_cast<size_t>(plans[i]->nnz);
   }
+  // dense form of the paired sparse product: eps * Zbar beside W, rows 2 K wide
+  const bool ext = paired != nullptr && paired->dense && nnz_all > 0;
+  const int64_t ld = p0->K * (ext ? 2 : 1);
   // resident form: the weight and the dense values at the masked positions live in the caller's buffers
-  const size_t w_bytes = resident ? 0 : round_up(static_cast<size_t>(rows) * p0->K * sizeof(__nv_bfloat16), 256);
+  const size_t w_bytes = resident ? 0 : round_up(static_cast<size_t>(rows) * ld * sizeof(__nv_bfloat16), 256);
   const size_t saved_bytes = resident ? 0 : round_up(nnz_all * sizeof(__nv_bfloat16), 256);
   SZO_REQUIRE(resident || (ws != nullptr && ws_bytes >= w_bytes + saved_bytes), SZO_ERR_WORKSPACE,
               "the materialised form needs a workspace of at least %zu bytes", w_bytes + saved_bytes);
@@ -667,13 +709,13 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
                                   : reinterpret_cast<__nv_bfloat16*>(static_cast<unsigned char*>(ws) + w_bytes);
   const int nkb = static_cast<int>(p0->K / kBK);
   MatArgs a{};
-  a.n = n; a.nkb = nkb; a.G = p0->G; a.K = p0->K;
+  a.n = n; a.nkb = nkb; a.G = p0->G; a.K = p0->K; a.ld = ld;
   int64_t row0 = 0, words = 0, nnz = 0;
   for (int i = 0; i < n; ++i) {
     const szo_linear* p = plans[i];
     words += (p->Npad / kBM) * ((nkb + 3) / 4) * 1024;
     SZO_REQUIRE(p->G == p0->G && p->K == p0->K, SZO_ERR_INVALID_ARG, "matrices of one launch must share K and format");
-    a.sub[i] = MatSub{p->codes_tiled, p->sz, p->Npad, W + row0 * p->K, p->idx, S_pert[i], words, nnz + p->nnz, saved + nnz,
+    a.sub[i] = MatSub{p->codes_tiled, p->sz, p->Npad, W + row0 * ld, p->idx, S_pert[i], words, nnz + p->nnz, saved + nnz,
                       p->lut_bf16};
     nnz += p->nnz;
     row0 += p->Npad;
@@ -683,10 +725,10 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
     int64_t r0 = 0;
     for (int i = 0; i < n; ++i) {
       const szo_linear* p = plans[i];
-      SZO_CHECK_CUDA(cudaMemcpyAsync(W + r0 * p->K, p->codes, static_cast<size_t>(p->N) * p->K * sizeof(__nv_bfloat16),
-                                     cudaMemcpyDeviceToDevice, st));
+      SZO_CHECK_CUDA(cudaMemcpy2DAsync(W + r0 * ld, ld * sizeof(__nv_bfloat16), p->codes, p->K * sizeof(__nv_bfloat16),
+                                       p->K * sizeof(__nv_bfloat16), p->N, cudaMemcpyDeviceToDevice, st));
       if (p->Npad > p->N)
-        SZO_CHECK_CUDA(cudaMemsetAsync(W + (r0 + p->N) * p->K, 0, static_cast<size_t>(p->Npad - p->N) * p->K * sizeof(__nv_bfloat16), st));
+        SZO_CHECK_CUDA(cudaMemsetAsync(W + (r0 + p->N) * ld, 0, static_cast<size_t>(p->Npad - p->N) * ld * sizeof(__nv_bfloat16), st));
       r0 += p->Npad;
     }
   } else if (!resident) {
@@ -697,8 +739,11 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
     count_launch();
     SZO_CHECK_LAUNCH("materialise_kernel");
   }
+  if (ext && !resident)        // the eps * Zbar half starts from zero (the resident buffer keeps its zeros: the
+                               // entries sit at the same positions every step)
+    SZO_CHECK_CUDA(cudaMemset2DAsync(W + p0->K, ld * sizeof(__nv_bfloat16), 0, p0->K * sizeof(__nv_bfloat16), rows, st));
   CUtensorMap mw;
-  SZO_TRY(make_map(&mw, W, rows, p0->K, kBM));
+  SZO_TRY(make_map(&mw, W, rows, ld, kBM));
   TcParams P{};
   P.M = M_rows; P.K = p0->K; P.G = 0; P.nkb = nkb;
   P.relu = relu ? 1 : 0;
@@ -706,6 +751,7 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
   P.nsub = n;
   if (paired != nullptr) {
     P.pair_row0 = Mp;
+    P.pair_ext = ext ? 1 : 0;
   }
   int64_t n_tiles = 0;
   for (int i = 0; i < n; ++i) {
@@ -741,6 +787,13 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
   SZO_TRY(refresh_tickets(t, st));
   const size_t y_elt = (y_dtype == SZO_F32) ? 4 : 2;
   const int n_sets = S_second != nullptr ? 2 : 1;
+  if (ext) {
+    MatArgs az = a;
+    for (int i = 0; i < n; ++i) az.sub[i].S = paired->z[i];
+    scatter_z_bf16_kernel<<<static_cast<unsigned>(ceil_div(nnz, 256)), 256, 0, st>>>(az, paired->eps);
+    count_launch();
+    SZO_CHECK_LAUNCH("scatter_z_bf16_kernel");
+  }
   for (int set = 0; set < n_sets; ++set) {
     if (nnz > 0) {
       a.scatter_mode = resident ? 2 : (n_sets == 1 ? 0 : set + 1);
@@ -755,7 +808,7 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
       P.sub[i].y = static_cast<unsigned char*>(y[i]) + static_cast<size_t>(set) * M * plans[i]->N * y_elt;
     SZO_TRY(launch_pair_kernel(false, false, mx, mw, P, sc.n_pairs, st));
   }
-  if (paired != nullptr && nnz_all > 0) {
+  if (paired != nullptr && nnz_all > 0 && !ext) {
     CrossArgs ca{};
     ca.n = n; ca.x = static_cast<const __nv_bfloat16*>(x); ca.M = M; ca.K = p0->K;
     ca.col_mask = cross_col_mask(p0->K);

@@ -129,6 +129,10 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& P, int pair, int n_p
   const int m_tiles = static_cast<int>(P.m_tiles);
   int np = tile / m_tiles;
   u.m_tile = tile - np * m_tiles;
+  if (P.pair_ext && static_cast<int64_t>(u.m_tile) * 256 >= P.pair_row0) {
+    u.kb0 *= 2;          // half-difference token tile: twice the k-blocks (xd W^T, then xc (eps Zbar)^T)
+    u.kb1 *= 2;
+  }
   u.g_tile = np * 2 + rank;
   u.s = 0;
   if (P.nsub > 1 && np >= P.sub[0].n_tiles) {
@@ -312,7 +316,16 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
   const int full_iters = P.full_rounds * nkb;
   const int tail_part = has_tail ? pair / P.tail_tiles : 0;
   const int tail_kb0 = has_tail ? tail_kb_at(P, tail_part) : 0;
-  const int my_iters = full_iters + (has_tail ? tail_kb_at(P, tail_part + 1) - tail_kb0 : 0);
+  int my_iters = full_iters + (has_tail ? tail_kb_at(P, tail_part + 1) - tail_kb0 : 0);
+  if constexpr (kPaired) {
+    if (P.pair_ext) {      // units differ in length: add them up
+      my_iters = 0;
+      for (int lt = 0; lt < my_units; ++lt) {
+        const Unit u = decode_unit(P, pair, n_pairs, rank, lt);
+        my_iters += u.kb1 - u.kb0;
+      }
+    }
+  }
 
   if (warp == kWarpX) {
     // ---------------------------------------------------------------- X producer (own token half)
@@ -326,7 +339,14 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         for (int kb = u.kb0; kb < u.kb1; ++kb) {
           if (!mbar_wait(xempty_bar(x.idx), x.phase ^ 1u, abort_flag, P.status)) { ok = false; break; }
           mbar_expect_tx(xfull_bar(x.idx), kXStageBytes);
-          tma_load_2d(tiles_base + b_off(x.idx), &tmap_x, kb * kBK, tok0, xfull_bar(x.idx));
+          int xk = kb * kBK, xt = tok0;
+          if constexpr (kPaired) {
+            if (kb >= nkb) {            // second half of a half-difference tile: the centre rows of the same tokens
+              xk -= nkb * kBK;
+              xt -= static_cast<int>(P.pair_row0);
+            }
+          }
+          tma_load_2d(tiles_base + b_off(x.idx), &tmap_x, xk, xt, xfull_bar(x.idx));
           if constexpr (!kDequant) tma_load_2d(tiles_base + a_off(x.idx, 0), &tmap_w, kb * kBK, row0, xfull_bar(x.idx));
           x.advance(kXS);
         }
@@ -382,7 +402,13 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
       for (int lt = 0; lt < my_units && ok; ++lt) {
         const int as = lt & 1;
         const uint32_t aph = static_cast<uint32_t>((lt >> 1) & 1);
-        const int n_kb = (lt < P.full_rounds) ? nkb : my_iters - full_iters;
+        int n_kb = (lt < P.full_rounds) ? nkb : my_iters - full_iters;
+        if constexpr (kPaired) {
+          if (P.pair_ext) {
+            const Unit u = decode_unit(P, pair, n_pairs, rank, lt);
+            n_kb = u.kb1 - u.kb0;
+          }
+        }
         if (!mbar_wait(accempty_bar(as), aph ^ 1u, abort_flag, P.status, 0)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kPairBT);

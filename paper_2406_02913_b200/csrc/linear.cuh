@@ -67,15 +67,21 @@ size_t tc_tail_ws_bound();   // enough for any M and any group
 // Materialised form (gemm_tc.cu): the effective bf16 weight is written to scratch, then the dense
 // mode of the kernel runs.  Chosen for int4 plans when M is large (tc_use_materialised).
 bool tc_use_materialised(const szo_linear* p, int64_t M, bool two_sets = false);   // two_sets: one weight pass for two forwards
-size_t tc_materialised_ws_bytes(const szo_linear* const* plans, int n, int64_t M);
+size_t tc_materialised_ws_bytes(const szo_linear* const* plans, int n, int64_t M, bool ext = false);   // ext: rows 2 K wide
 // Paired form of a ZO step's two forwards (see tc::TcParams): x and every y[i] hold the M centre rows
 // first and the M half-difference rows from row round_up(M, 256) on; S_pert are the unperturbed sparse
 // values; rec[i][e] = column of entry e of plans[i] and eps * z_e in one word (pack_cross_records; the
 // split depends on K only, so one call may pack the entries of matrices with different K one after another
 // only if called per K).
+// dense: the product runs on the tensor cores instead (eps * z written as a bf16 matrix beside W; z, eps
+// are used, rec is not).
 struct PairedArgs {
   const uint32_t* const* rec;
+  const float* const* z;
+  float eps;
+  bool dense;
 };
+bool tc_paired_dense_cross(const szo_linear* const* plans, int n);
 szo_status pack_cross_records(const int32_t* col, const float* z, float eps, int64_t n, int64_t K, uint32_t* rec,
                               cudaStream_t st);
 uint32_t cross_col_mask(int64_t K);
@@ -91,9 +97,9 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
 // weight pass and writes every masked entry as RN_bf16(saved + S); ws is only the K-split scratch.
 bool tc_use_resident(const szo_linear* p, int64_t M);
 bool tc_can_stack(const szo_linear* const* plans, int n);
-void tc_resident_bytes(const szo_linear* const* plans, int n, size_t* w_bytes, size_t* saved_bytes);
+void tc_resident_bytes(const szo_linear* const* plans, int n, size_t* w_bytes, size_t* saved_bytes, bool ext = false);
 szo_status tc_resident_init(const szo_linear* const* plans, int n, __nv_bfloat16* W, __nv_bfloat16* saved,
-                            cudaStream_t st);
+                            cudaStream_t st, bool ext = false);
 // S_second: a second set of sparse values and of M tokens served by the same weight pass (x and
 // y[i] hold 2 M rows).
 // out[p] = (pos[p], bits of S[eid[p]]) for p in [0, n)

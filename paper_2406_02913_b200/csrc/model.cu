@@ -920,10 +920,12 @@ szo_status run_loss_paired(szo_model* m, const int32_t* tokens, const int32_t* l
     const szo_linear* plans[3];
     const float* sv[3];
     const uint32_t* crec[3];
+    const float* zz[3];
     for (int i = 0; i < n; ++i) {
       plans[i] = m->plans[t0 + i];
       sv[i] = Sv + m->offsets[t0 + i];
       crec[i] = reinterpret_cast<const uint32_t*>(m->recs) + m->offsets[t0 + i];
+      zz[i] = z + m->offsets[t0 + i];
     }
     if (m->timing) {
       while (m->events.size() < m->events_used + 2) {
@@ -933,7 +935,7 @@ szo_status run_loss_paired(szo_model* m, const int32_t* tokens, const int32_t* l
       }
       SZO_CHECK_CUDA(cudaEventRecord(m->events[m->events_used], st));
     }
-    const PairedArgs pa{crec};
+    const PairedArgs pa{crec, zz, eps, tc_paired_dense_cross(plans, n)};
     const bool res = m->resident;
     const szo_status rc = linear_fwd_tc_materialised(plans, n, x, M, sv, outs, SZO_BF16, m->ws, m->ws_bytes, st, nullptr,
                                                      res ? m->res_W[t0] : nullptr, res ? m->res_saved[t0] : nullptr,
@@ -950,9 +952,11 @@ szo_status run_loss_paired(szo_model* m, const int32_t* tokens, const int32_t* l
   };
   // (column, eps * z) of every sensitive entry, once for all linears of the step (the record layout
   // depends on K: one call per linear)
-  for (size_t t = 0; t < m->plans.size(); ++t)
-    SZO_TRY(pack_cross_records(m->plans[t]->ent_col, z + m->offsets[t], eps, m->plans[t]->nnz, m->plans[t]->K,
+  for (size_t t = 0; t < m->plans.size(); ++t) {
+    const szo_linear* pl = m->plans[t];
+    SZO_TRY(pack_cross_records(pl->ent_col, z + m->offsets[t], eps, pl->nnz, pl->K,
                                reinterpret_cast<uint32_t*>(m->recs) + m->offsets[t], st));
+  }
   embed_kernel<<<static_cast<unsigned>(M), 128, 0, st>>>(tokens, static_cast<const __nv_bfloat16*>(m->top.embed),
                                                         static_cast<const __nv_bfloat16*>(m->top.pos), S, d, c.vocab, m->h);
   SZO_CHECK_CUDA(cudaMemsetAsync(m->h + Mp * d, 0, static_cast<size_t>(M) * d * sizeof(float), st));   // both forwards embed alike
@@ -1118,11 +1122,12 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
     if (tc_use_materialised(m->plans[0], m->Mmax, true) || (m->paired && c.group != 0)) {
       for (int l = 0; l < c.n_layers; ++l) {
         const szo_linear* const* pl = m->plans.data() + static_cast<size_t>(l) * m->n_lin;
-        const size_t g0 = tc_materialised_ws_bytes(pl, 3, m->Mmax);                       // q, k, v
-        const size_t g1 = c.arch == 0 ? tc_materialised_ws_bytes(pl + 4, 2, m->Mmax) : 0;  // gate, up
+        const bool px = m->paired;
+        const size_t g0 = tc_materialised_ws_bytes(pl, 3, m->Mmax, px && tc_paired_dense_cross(pl, 3));   // q, k, v
+        const size_t g1 = c.arch == 0 ? tc_materialised_ws_bytes(pl + 4, 2, m->Mmax, px && tc_paired_dense_cross(pl + 4, 2)) : 0;  // gate, up
         size_t g2 = 0;
         for (int j = 0; j < m->n_lin; ++j) {
-          const size_t one = tc_materialised_ws_bytes(pl + j, 1, m->Mmax);
+          const size_t one = tc_materialised_ws_bytes(pl + j, 1, m->Mmax, px && tc_paired_dense_cross(pl + j, 1));
           if (one > g2) g2 = one;
         }
         const size_t mx = g0 > g1 ? (g0 > g2 ? g0 : g2) : (g1 > g2 ? g1 : g2);
@@ -1150,10 +1155,11 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
         const szo_linear* const* pl = m->plans.data() + t0;
         if (!tc_can_stack(pl, g_count[g])) return bail(fail(SZO_ERR_UNSUPPORTED, "resident form: group cannot be stacked"));
         size_t wb = 0, sb = 0;
-        tc_resident_bytes(pl, g_count[g], &wb, &sb);
+        const bool ext = m->paired && tc_paired_dense_cross(pl, g_count[g]);
+        tc_resident_bytes(pl, g_count[g], &wb, &sb, ext);
         SZO_M_TRY(dev_alloc(m, &m->res_W[t0], wb));
         SZO_M_TRY(dev_alloc(m, &m->res_saved[t0], sb));
-        SZO_M_TRY(tc_resident_init(pl, g_count[g], m->res_W[t0], m->res_saved[t0], st));
+        SZO_M_TRY(tc_resident_init(pl, g_count[g], m->res_W[t0], m->res_saved[t0], st, ext));
       }
     }
   }

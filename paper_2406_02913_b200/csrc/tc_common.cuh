@@ -61,6 +61,11 @@ struct TcParams {
   // and leaves the bias out of the half-difference rows; the sparse product is added to those rows by
   // pair_cross_kernel after it.
   int64_t pair_row0;       // first half-difference row (0: not a paired launch)
+  // pair_ext != 0: the sparse product runs on the tensor cores too.  The weight buffer is [rows][2 K]:
+  // W in columns [0, K), eps * Zbar as a dense bf16 matrix in columns [K, 2 K).  A half-difference
+  // token tile then runs 2 K / 64 k-blocks: the first K / 64 multiply xd by W, the others multiply the
+  // CENTRE rows of the same tokens (token row - pair_row0) by eps * Zbar, into the same accumulator.
+  int pair_ext;
 };
 
 // Position in a ring of n slots: slot index and the parity of the current pass over the ring.

@@ -73,13 +73,15 @@ def test_linear_paired_matches_oracle(B, N, K, G, fmt, M, rho, bias):
     assert max_rel(y[row0:], ref_d) < 5e-3
     yb = plan.fwd_paired(x, M, d(S), d(z), float(eps), torch.bfloat16).float().cpu().numpy()
     assert max_rel(yb[:M], ref_c) < 2e-2 and max_rel(yb[row0:], ref_d) < 2e-2
-    # with xd = 0 the half-difference rows are eps * xc Zbar^T alone: an fp32 sum of a few products, of
-    # eps * z kept with 23 - ceil(log2 K) mantissa bits (one word holds the column and eps * z)
+    # with xd = 0 the half-difference rows are eps * xc Zbar^T alone.  Sparse masks (below 0.2 %): an fp32 sum
+    # of a few products, of eps * z kept with 23 - ceil(log2 K) mantissa bits (one word holds the column and
+    # eps * z).  Denser masks: the product runs on the tensor cores with eps * z rounded to bf16.
     x0, _ = paired_rows(B, xc, np.zeros_like(xd))
     y0 = plan.fwd_paired(x0, M, d(S), d(z), float(eps), torch.float32).cpu().numpy()
     Zs = so.effective_weight(np.zeros_like(c["deq"]), c["idx"], ez)
     ref0 = xc.astype(np.float64) @ Zs.T
-    assert max_rel(y0[row0:], ref0) < 2e-6 + 2.0 ** -(24 - int(np.ceil(np.log2(K))))
+    dense_cross = len(c["idx"]) >= 0.002 * N * K
+    assert max_rel(y0[row0:], ref0) < (2.0 ** -8 if dense_cross else 2e-6 + 2.0 ** -(24 - int(np.ceil(np.log2(K)))))
     y1 = plan.fwd_paired(x0, M, d(S), d(z), float(eps), torch.float32).cpu().numpy()
     assert np.array_equal(y0[:M], y1[:M]) and np.array_equal(y0[row0:], y1[row0:])     # bit-repeatable
     assert B.device_status() == 0
