@@ -156,6 +156,16 @@ szo_status szo_update(float* S, const int64_t* idx, int64_t k, int64_t idx_base,
                       uint64_t step, float lr, const double* f_plus_dev, const double* f_minus_dev,
                       float eps, void* stream);
 
+/* ---- Replay of a run from its log (Section 2.1, the seed trick: z_t is a function of (seed, step_t), so
+ * the scalars g_t are a complete record of what a run did to the sparse values:
+ * S_T = S_0 - sum_t lr g_t z_t; a checkpoint is S at some step plus the (step, g) pairs since).
+ * For every logged step, in order: when eps != 0, the +eps, -2 eps, +eps passes of the in-place order
+ * (so that S takes exactly the roundings of the original step; eps == 0 skips them), then
+ * S[j] = fma(-(float)(lr * g_t), z_j, S[j]).  steps_host, g_host: HOST arrays of n entries.
+ * Reproduces the S of szo_model_zo_step / szo_update runs bit for bit. */
+szo_status szo_replay(float* S, const int64_t* idx, int64_t k, int64_t idx_base, uint64_t seed,
+                      const uint64_t* steps_host, const double* g_host, int64_t n, float eps, float lr, void* stream);
+
 /* ---- Decomposed linear layer (Section 3.4: w = w_sparse + w_dense; appendix on sparse
  * operations: y = x Dequantize(Q(w_dense))^T + x w_sparse^T).
  * A plan owns only derived, immutable data (kernel-layout scale/zero table, tile buckets and

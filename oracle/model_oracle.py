@@ -154,6 +154,80 @@ def hidden_states(cfg: DecoderConfig, params: dict, lin_W: list, tokens):
     return rms_norm(h, _t(params["final_norm"]), cfg.norm_eps)
 
 
+def rope_at(x, base, positions):
+    """rope for rows at the given positions: x [B, T, H, hd], positions [T]."""
+    B, T, H, hd = x.shape
+    half = hd // 2
+    inv = base ** (-(torch.arange(half, dtype=torch.float64) * 2.0) / hd)
+    ang = torch.as_tensor(positions, dtype=torch.float64)[:, None] * inv[None, :]
+    cos, sin = torch.cos(ang)[None, :, None, :], torch.sin(ang)[None, :, None, :]
+    x1, x2 = x[..., :half], x[..., half:]
+    return torch.cat([x1 * cos - x2 * sin, x2 * cos + x1 * sin], dim=-1)
+
+
+class KVCache:
+    """Keys and values of the positions decoded so far, per layer: lists of [B, n, Hkv, hd] tensors."""
+
+    def __init__(self, n_layers):
+        self.k = [None] * n_layers
+        self.v = [None] * n_layers
+        self.n = 0
+
+
+def decode_step(cfg: DecoderConfig, params: dict, lin_W: list, new_tokens, cache: KVCache):
+    """Token generation with a KV cache (the regime of the paper's inference measurements: Section 1's
+    speed figure and the appendix on sparse operations): processes T new tokens per sequence
+    (new_tokens [B, T]) that follow the cache.n positions already in the cache, appends their keys and
+    values, and returns the logits of the LAST new token, [B, V].  Each new position attends to every
+    cached position and to the new positions up to itself.  Same blocks as hidden_states."""
+    tok = torch.as_tensor(np.asarray(new_tokens), dtype=torch.long)
+    B, T = tok.shape
+    H, Hkv, hd = cfg.n_heads, cfg.n_kv_heads, cfg.head_dim
+    opt = cfg.arch == "opt"
+    pos = list(range(cache.n, cache.n + T))
+    h = _t(params["embed"])[tok]
+    if opt:
+        h = h + _t(params["pos"])[pos][None, :, :]
+    rep = H // Hkv
+    for l in range(cfg.n_layers):
+        W = lin_W[l]
+        P = lambda nm: _t(params[f"l{l}.{nm}"])
+
+        def lin(x, nm):
+            y = x @ _t(W[nm]).T
+            return y + P(nm + "_b") if opt else y
+
+        a = layer_norm(h, P("attn_norm"), P("attn_norm_b"), cfg.norm_eps) if opt else rms_norm(h, P("attn_norm"), cfg.norm_eps)
+        q = lin(a, "wq").view(B, T, H, hd)
+        k = lin(a, "wk").view(B, T, Hkv, hd)
+        v = lin(a, "wv").view(B, T, Hkv, hd)
+        if not opt:
+            q, k = rope_at(q, cfg.rope_base, pos), rope_at(k, cfg.rope_base, pos)
+        cache.k[l] = k if cache.k[l] is None else torch.cat([cache.k[l], k], dim=1)
+        cache.v[l] = v if cache.v[l] is None else torch.cat([cache.v[l], v], dim=1)
+        o = torch.empty(B, T, H, hd, dtype=torch.float64)
+        for t in range(T):
+            n_keys = cache.n + t + 1
+            for hh in range(H):
+                kh, vh = cache.k[l][:, :n_keys, hh // rep, :], cache.v[l][:, :n_keys, hh // rep, :]
+                sc = torch.einsum("bd,bnd->bn", q[:, t, hh, :], kh) / math.sqrt(hd)
+                o[:, t, hh, :] = torch.einsum("bn,bnd->bd", torch.softmax(sc, dim=-1), vh)
+        h = h + lin(o.reshape(B, T, H * hd), "wo")
+        if opt:
+            m = layer_norm(h, P("mlp_norm"), P("mlp_norm_b"), cfg.norm_eps)
+            h = h + lin(torch.relu(lin(m, "fc1")), "fc2")
+        else:
+            m = rms_norm(h, P("mlp_norm"), cfg.norm_eps)
+            h = h + lin(torch.nn.functional.silu(lin(m, "w_gate")) * lin(m, "w_up"), "w_down")
+    cache.n += T
+    last = h[:, -1, :]
+    if opt:
+        last = layer_norm(last, _t(params["final_norm"]), _t(params["final_norm_b"]), cfg.norm_eps)
+    else:
+        last = rms_norm(last, _t(params["final_norm"]), cfg.norm_eps)
+    return last @ _t(params["lm_head"]).T
+
+
 def _log_softmax(x):
     m = x.max(dim=-1, keepdim=True).values
     return x - m - torch.log(torch.exp(x - m).sum(dim=-1, keepdim=True))

@@ -293,6 +293,22 @@ def zo_update_scale(f_plus: float, f_minus: float, eps, lr) -> np.float32:
     return np.float32(-(float(np.float32(lr)) * g))
 
 
+def replay(S0, gidx, seed: int, log, eps, lr) -> np.ndarray:
+    """Section 2.1: the run's effect on the sparse values from its log [(step_t, g_t), ...] alone.  For
+    every logged step, in order: the +eps, -2 eps, +eps passes (when eps != 0: they leave S within an
+    ulp or two of where it was, and a replay that wants the same bits takes the same roundings), then
+    the update S <- S - lr g_t z_t of Definitions 2 and 4, z_t regenerated from (seed, step_t)."""
+    S = np.asarray(S0, dtype=np.float32).copy()
+    e = np.float32(eps)
+    for step, g in log:
+        if e != 0:
+            S = perturb(S, gidx, seed, step, e)
+            S = perturb(S, gidx, seed, step, np.float32(-2.0) * e)
+            S = perturb(S, gidx, seed, step, e)
+        S = perturb(S, gidx, seed, step, np.float32(-(float(np.float32(lr)) * float(g))))
+    return S
+
+
 def zo_sgd_step(loss, S, gidx, seed: int, step: int, eps, lr):
     """One sensitive-sparse ZO-SGD step on the k trainable values S for a loss callable
     loss(S) -> float, in the in-place order of the seed trick (Section 2.1):

@@ -78,6 +78,8 @@ _SIGS = {
     "szo_projected_gradient": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p]),
     "szo_update": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_uint64, C.c_uint64,
                                C.c_float, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]),
+    "szo_replay": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_uint64, C.POINTER(C.c_uint64),
+                               C.POINTER(C.c_double), C.c_int64, C.c_float, C.c_float, C.c_void_p]),
     "szo_linear_create": (C.c_int32, [C.POINTER(C.c_void_p), C.c_int64, C.c_int64, C.c_int32,
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
                                       C.c_int64, C.c_void_p, C.c_void_p]),
@@ -226,6 +228,14 @@ def szo_projected_gradient(f_plus, f_minus, eps: float, g_out):
 def szo_update(S, idx, idx_base: int, seed: int, step: int, lr: float, f_plus, f_minus, eps: float):
     _check(lib().szo_update(_ptr(S), _ptr(idx), idx.numel(), idx_base, seed, step, lr, _ptr(f_plus),
                             _ptr(f_minus), eps, _stream()))
+
+
+def szo_replay(S, idx, idx_base: int, seed: int, log, eps: float, lr: float):
+    """Applies the logged steps [(step, g), ...] to S in place (szo_replay)."""
+    n = len(log)
+    steps = (C.c_uint64 * max(n, 1))(*[int(s) for s, _ in log])
+    gs = (C.c_double * max(n, 1))(*[float(g) for _, g in log])
+    _check(lib().szo_replay(_ptr(S), _ptr(idx), idx.numel(), idx_base, seed, steps, gs, n, eps, lr, _stream()))
 
 
 # ------------------------------------------------------------------------------ linear layer

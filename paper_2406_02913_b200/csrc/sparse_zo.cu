@@ -296,6 +296,28 @@ szo_status szo_update(float* S, const int64_t* idx, int64_t k, int64_t idx_base,
                                  static_cast<cudaStream_t>(stream));
 }
 
+szo_status szo_replay(float* S, const int64_t* idx, int64_t k, int64_t idx_base, uint64_t seed,
+                      const uint64_t* steps_host, const double* g_host, int64_t n, float eps, float lr, void* stream) {
+  SZO_REQUIRE(k >= 0 && n >= 0, SZO_ERR_INVALID_ARG, "k < 0 or n < 0");
+  if (k == 0 || n == 0) return SZO_OK;
+  SZO_REQUIRE(S && idx && steps_host && g_host, SZO_ERR_INVALID_ARG, "NULL pointer");
+  SZO_REQUIRE(idx_base >= 0, SZO_ERR_INVALID_ARG, "idx_base < 0");
+  SZO_REQUIRE(szo::aligned16(S) && szo::aligned16(idx), SZO_ERR_ALIGNMENT, "S and idx must be 16-byte aligned");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  for (int64_t t = 0; t < n; ++t) {
+    if (eps != 0.f) {     // the roundings of the original step's +eps, -2 eps, +eps passes
+      const float sc[3] = {eps, -2.0f * eps, eps};
+      for (int i = 0; i < 3; ++i) {
+        szo::ScaleArg sa{sc[i], 0.f, 0.f, nullptr, nullptr};
+        SZO_TRY(szo::launch_sparse_axpy(S, S, idx, k, idx_base, seed, steps_host[t], sa, st));
+      }
+    }
+    szo::ScaleArg su{-static_cast<float>(static_cast<double>(lr) * g_host[t]), 0.f, 0.f, nullptr, nullptr};
+    SZO_TRY(szo::launch_sparse_axpy(S, S, idx, k, idx_base, seed, steps_host[t], su, st));
+  }
+  return SZO_OK;
+}
+
 szo_status szo_projected_gradient(const double* f_plus_dev, const double* f_minus_dev, float eps,
                                   double* g_dev, void* stream) {
   SZO_REQUIRE(f_plus_dev && f_minus_dev && g_dev, SZO_ERR_INVALID_ARG, "NULL pointer");

@@ -282,3 +282,26 @@ def test_two_half_batches_through_losses_and_apply_equal_the_full_batch_step(B, 
     assert B.device_status() == 0
     m_full.close()
     m_dp.close()
+
+
+def test_replay_from_the_g_log_reproduces_the_sparse_values(B, tiny):
+    """Five steps on the fp32 validation path, their (step, g) pairs logged; szo_replay from S_0 gives the
+    run's final S bit for bit (with the +-eps passes replayed), and the oracle's replay of the same log
+    agrees to the accuracy of z."""
+    fx = tiny
+    m, S, _ = build_gpu(B, fx, B.SZO_F32, B.MODE_FP32_VALIDATE)
+    S0 = S.clone()
+    eps, lr = 1e-3, 1e-3
+    log = []
+    for step in (0, 1, 2, 7, 8):
+        out = m.zo_step(torch.from_numpy(fx.batch(step)).cuda(), 1234, step, eps, lr).cpu().numpy()
+        log.append((step, float(out[2])))
+    S_rep = S0.clone()
+    B.szo_replay(S_rep, m.gidx(), 0, 1234, log, eps, lr)
+    assert torch.equal(S_rep, S)
+    ref = so.replay(S0.cpu().numpy(), fx.gidx, 1234, log, eps, lr)
+    assert np.allclose(S_rep.cpu().numpy(), ref, rtol=0, atol=5e-7)
+    S_plain = S0.clone()
+    B.szo_replay(S_plain, m.gidx(), 0, 1234, log, 0.0, lr)
+    assert torch.allclose(S_plain, S, rtol=0, atol=1e-6) and not torch.equal(S_plain, S0)
+    m.close()

@@ -242,6 +242,23 @@ def test_opt_statement_notices_a_dropped_bias_a_position_shift_and_post_norm():
     assert np.abs(_opt_layer_numpy(params, lin_W[0], tokens, H=4, act=lambda t: t) - got).max() > 1e-6
 
 
+def test_incremental_decode_equals_the_full_forward():
+    """decode_step with a KV cache (prefill of 3 tokens, then a chunk of 2, then one token at a time)
+    gives, at every stop, the logits that the full forward gives at that position: both architectures,
+    grouped-query attention included."""
+    for arch in ("llama", "opt"):
+        cfg, params, lin_W, tokens = _small(arch)
+        hs = mo.hidden_states(cfg, params, lin_W, tokens)
+        full = (hs @ torch.as_tensor(params["lm_head"], dtype=torch.float64).T).numpy()      # [B, S, V]
+        cache = mo.KVCache(cfg.n_layers)
+        at = 0
+        for T in (3, 2, 1, 1, 1):
+            logits = mo.decode_step(cfg, params, lin_W, tokens[:, at:at + T], cache).numpy()
+            at += T
+            assert cache.n == at
+            assert np.allclose(logits, full[:, at - 1, :], rtol=0, atol=1e-11), (arch, at)
+
+
 def test_gqa_reduces_to_mha_when_kv_heads_are_duplicated():
     cfg, params, lin_W, tokens = _small("llama", kv=2)
     full = mo.DecoderConfig(**{**cfg.__dict__, "n_kv_heads": 4})

@@ -383,6 +383,30 @@ def test_zo_sgd_update_and_replay_identity():
     assert np.allclose(S, S0 - acc, rtol=0, atol=1e-6)        # S_T = S_0 - sum_t lr g_t z_t
 
 
+def test_replay_from_the_log_reproduces_the_run():
+    """so.replay against the run it replays (itself pinned above): the same bits when the +-eps passes
+    are replayed too, and S_0 - sum_t lr g_t z_t up to their drift when they are skipped."""
+    A, w, idx = _quad_problem(d=64, k=10)
+    state = w.copy()
+
+    def loss(S):
+        v = state.astype(np.float64).copy()
+        v[idx] = S
+        return 0.5 * v @ A @ v
+
+    eps, lr = np.float32(1e-3), np.float32(1e-2)
+    S, log, acc = state[idx].copy(), [], np.zeros(10)
+    for step in (3, 4, 9, 10, 11, 40):                       # the log need not be contiguous
+        S, fp, fm, g = so.zo_sgd_step(loss, S, idx, 77, step, eps, lr)
+        log.append((step, g))
+        acc += float(lr) * g * so.gaussian(77, step, idx).astype(np.float64)
+    again = so.replay(state[idx], idx, 77, log, eps, lr)
+    assert np.array_equal(again.view(np.uint32), S.view(np.uint32))
+    plain = so.replay(state[idx], idx, 77, log, 0.0, lr)
+    assert np.allclose(plain, state[idx].astype(np.float64) - acc, rtol=0, atol=1e-6)
+    assert np.allclose(plain, S, rtol=0, atol=1e-6) and so.replay(state[idx], idx, 77, [], eps, lr).tolist() == state[idx].tolist()
+
+
 def test_sparse_step_touches_only_masked_coordinates():
     A, w, idx = _quad_problem(d=64, k=8)
     state = w.copy()
