@@ -335,6 +335,25 @@ szo_status szo_model_zo_step_host(szo_model_t* m, const int32_t* tokens_host,
                                   const int32_t* labels_host, const int32_t* cand_host, int32_t B,
                                   int32_t S, uint64_t seed, uint64_t step, float eps, float lr,
                                   double* out3_host, void* stream);
+/* ---- Token generation with a KV cache (the regime of the paper's inference measurements: the speed
+ * figure of Section 1, 128 generated tokens; the appendix on sparse operations finds the SparseAddMM
+ * order the faster one there).
+ *   szo_model_enable_decode: allocates the cache, act_dtype [n_layers][max_batch][max_seq][n_kv_heads *
+ *     head_dim] for keys and for values (and an LM-head plan when the model's loss does not use one); once.
+ *   szo_model_decode_step: T new tokens per sequence (tokens int32 [B, T]) that follow the pos0 positions
+ *     already cached: their keys and values are appended at positions pos0 .. pos0 + T - 1, every new
+ *     position attends to the cached ones and to the new ones up to itself, and logits_dev receives the
+ *     fp32 logits [B, vocab] of the LAST new token.  A prompt is one call with pos0 = 0; generation is
+ *     one call per token with T = 1.  The caller keeps pos0 (the cache is not cleared: positions at or
+ *     beyond pos0 + T are simply not read).  Linears run in SZO_MODE_AUTO (the weight-streaming kernel
+ *     with the sparse term in fp32 for at most 16 rows), or in the validation mode for an fp32 model.
+ *     S_vals: fp32 [k_total] or NULL for the model's S.  On a stream other than the default one the
+ *     several hundred launches of a step are captured once per (B, T, S_vals) into a CUDA graph and
+ *     replayed (SZO_DECODE_GRAPH=0 at szo_model_enable_decode keeps the launch-by-launch form); the
+ *     call itself must not be issued inside a capture of the caller's. */
+szo_status szo_model_enable_decode(szo_model_t* m, void* stream);
+szo_status szo_model_decode_step(szo_model_t* m, const int32_t* tokens, int32_t B, int32_t T, int32_t pos0,
+                                 const float* S_vals, float* logits_dev, void* stream);
 /* Number of kernel launches the last szo_model_zo_step on this model enqueued. */
 int64_t szo_model_last_launches(const szo_model_t* m);
 /* Measurement aid (no counterpart in the paper): when enabled, the model brackets every

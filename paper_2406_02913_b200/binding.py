@@ -113,6 +113,9 @@ _SIGS = {
     "szo_model_zo_step_host": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                            C.c_int32, C.c_uint64, C.c_uint64, C.c_float, C.c_float,
                                            C.c_void_p, C.c_void_p]),
+    "szo_model_enable_decode": (C.c_int32, [C.c_void_p, C.c_void_p]),
+    "szo_model_decode_step": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
+                                          C.c_void_p, C.c_void_p]),
     "szo_model_last_launches": (C.c_int64, [C.c_void_p]),
     "szo_model_enable_timing": (C.c_int32, [C.c_void_p, C.c_int32]),
     "szo_model_linear_time": (C.c_int32, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
@@ -416,6 +419,17 @@ class Model:
         _check(lib().szo_model_zo_step_host(self.h, hp(tokens_host), hp(labels_host), hp(cand_host), B, S,
                                             seed, step, eps, lr, C.cast(out, C.c_void_p), _stream()))
         return out[0], out[1], out[2]
+
+    def enable_decode(self):
+        _check(lib().szo_model_enable_decode(self.h, _stream()))
+
+    def decode_step(self, tokens, pos0: int, logits=None, S_vals=None) -> torch.Tensor:
+        """tokens int32 [B, T] following pos0 cached positions; returns fp32 logits [B, vocab] of the last one."""
+        B, T = tokens.shape
+        if logits is None:
+            logits = torch.empty((B, self.cfg.vocab), dtype=torch.float32, device=tokens.device)
+        _check(lib().szo_model_decode_step(self.h, _ptr(tokens), B, T, pos0, _ptr(S_vals), _ptr(logits), _stream()))
+        return logits
 
     def enable_timing(self, on: bool = True):
         _check(lib().szo_model_enable_timing(self.h, 1 if on else 0))

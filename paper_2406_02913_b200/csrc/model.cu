@@ -32,15 +32,16 @@ __device__ __forceinline__ float block_sum(float v, float* scratch) {
   return t;
 }
 
-// h[m, :] = embed[tok[m], :] (+ pos[m % S, :])
+// h[m, :] = embed[tok[m], :] (+ pos[pos0 + m % S, :]); pos0 > 0 when the rows continue a cached prefix
 __global__ void embed_kernel(const int32_t* __restrict__ tok, const __nv_bfloat16* __restrict__ embed,
                              const __nv_bfloat16* __restrict__ pos, int S, int d, int vocab,
-                             float* __restrict__ h) {
+                             float* __restrict__ h, int pos0 = 0, const int32_t* __restrict__ pos_dev = nullptr) {
+  if (pos_dev != nullptr) pos0 = *pos_dev;
   const int64_t m = blockIdx.x;
   int32_t t = tok[m];
   t = t < 0 ? 0 : (t >= vocab ? vocab - 1 : t);
   const __nv_bfloat16* e = embed + static_cast<int64_t>(t) * d;
-  const __nv_bfloat16* p = pos ? pos + static_cast<int64_t>(m % S) * d : nullptr;
+  const __nv_bfloat16* p = pos ? pos + static_cast<int64_t>(pos0 + m % S) * d : nullptr;
   for (int c = threadIdx.x; c < d; c += blockDim.x)
     h[m * d + c] = __bfloat162float(e[c]) + (p ? __bfloat162float(p[c]) : 0.f);
 }
@@ -135,7 +136,8 @@ __global__ void rope_table_kernel(int max_seq, int half, double base, float2* __
 // launch.  A thread rotates kN consecutive pairs (one 16-byte vector from each half of a head).
 template <typename T>
 __global__ void rope_kernel(T* __restrict__ q, T* __restrict__ k, const float2* __restrict__ tab, int64_t M, int S,
-                            int H, int Hkv, int hd) {
+                            int H, int Hkv, int hd, int pos0 = 0, const int32_t* __restrict__ pos_dev = nullptr) {
+  if (pos_dev != nullptr) pos0 = *pos_dev;
   constexpr int kN = 16 / sizeof(T);
   const int half = hd >> 1, vec_per_head = half / kN;
   const int64_t per_token = static_cast<int64_t>(H + Hkv) * vec_per_head;
@@ -145,7 +147,7 @@ __global__ void rope_kernel(T* __restrict__ q, T* __restrict__ k, const float2* 
   int r = static_cast<int>(i % per_token);
   const int head = r / vec_per_head, j0 = (r % vec_per_head) * kN;
   T* p = (head < H) ? q + (m * H + head) * hd : k + (m * Hkv + (head - H)) * hd;
-  const float2* cs = tab + static_cast<int64_t>(m % S) * half + j0;
+  const float2* cs = tab + static_cast<int64_t>(pos0 + m % S) * half + j0;
   T lo[kN], hi[kN];
   *reinterpret_cast<uint4*>(lo) = *reinterpret_cast<const uint4*>(p + j0);
   *reinterpret_cast<uint4*>(hi) = *reinterpret_cast<const uint4*>(p + half + j0);
@@ -337,6 +339,105 @@ cls2_kernel(const T* __restrict__ a_last, const __nv_bfloat16* __restrict__ lm_h
   }
 }
 
+
+
+// ------------------------------------------------------------------------------ token generation
+// cache[b][pos0 + t][:] = new[b * T + t][:] for the keys AND the values of T new tokens per sequence
+// (cache layout [B][Smax][width]); 16-byte vectors; the first n_vec threads copy keys, the others values.
+template <typename T>
+__global__ void kv_append_kernel(const T* __restrict__ k_new, const T* __restrict__ v_new, T* __restrict__ k_cache,
+                                 T* __restrict__ v_cache, int Tn, const int32_t* __restrict__ pos_dev, int64_t Smax,
+                                 int64_t width, int64_t n_vec) {
+  constexpr int kN = Vec16<T>::kN;
+  const int pos0 = *pos_dev;
+  int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= 2 * n_vec) return;
+  const bool is_v = i >= n_vec;
+  if (is_v) i -= n_vec;
+  const T* src = is_v ? v_new : k_new;
+  T* dst = is_v ? v_cache : k_cache;
+  const int64_t per_row = width / kN;
+  const int64_t row = i / per_row, c = (i - row * per_row) * kN;
+  const int64_t b = row / Tn, t = row - b * Tn;
+  store16(dst + (b * Smax + pos0 + t) * width + c, load16(src + row * width + c));
+}
+
+// Attention of T new tokens per sequence against the cache: query (b, t) attends to the cached
+// positions 0 .. pos0 + t (its own key included: the cache already holds the new keys).  One block of
+// four warps per (query, head): warp w takes the keys n = w, w + 4, ... (lanes split the head
+// dimension, online softmax per warp), then the four partial (maximum, sum, output) triples are merged
+// in warp order.  q, o: [B * T, H * HD]; kc, vc: [B][Smax][Hkv * HD].  The number of cached positions is
+// read from device memory, so that one captured graph of a token step serves every position.
+template <typename T, int HD>
+__global__ void __launch_bounds__(128)
+attn_decode_kernel(const T* __restrict__ q, const T* __restrict__ kc, const T* __restrict__ vc, T* __restrict__ o,
+                   int Tn, const int32_t* __restrict__ pos_dev, int64_t Smax, int H, int Hkv, float scale) {
+  constexpr int E = HD / 32;
+  __shared__ float part_acc[4][HD];
+  __shared__ float part_m[4], part_l[4];
+  const int pos0 = *pos_dev;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int t = blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
+  const int hk = hq / (H / Hkv);
+  const int64_t dq = static_cast<int64_t>(H) * HD, dk = static_cast<int64_t>(Hkv) * HD;
+  const T* qp = q + (static_cast<int64_t>(b) * Tn + t) * dq + hq * HD;
+  float qr[E], acc[E];
+#pragma unroll
+  for (int j = 0; j < E; ++j) {
+    qr[j] = to_f32<T>(qp[lane + 32 * j]) * scale;
+    acc[j] = 0.f;
+  }
+  float mx = -INFINITY, l = 0.f;
+  const T* kb = kc + static_cast<int64_t>(b) * Smax * dk + hk * HD;
+  const T* vb = vc + static_cast<int64_t>(b) * Smax * dk + hk * HD;
+  for (int n = w; n <= pos0 + t; n += 4) {
+    const T* kp = kb + n * dk;
+    const T* vp = vb + n * dk;
+    float kv[E], vv[E];
+#pragma unroll
+    for (int j = 0; j < E; ++j) {
+      kv[j] = to_f32<T>(kp[lane + 32 * j]);
+      vv[j] = to_f32<T>(vp[lane + 32 * j]);
+    }
+    float dot = 0.f;
+#pragma unroll
+    for (int j = 0; j < E; ++j) dot = fmaf(qr[j], kv[j], dot);
+#pragma unroll
+    for (int off = 16; off; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+    const float mn = fmaxf(mx, dot);
+    const float corr = expf(mx - mn), p = expf(dot - mn);
+    l = l * corr + p;
+#pragma unroll
+    for (int j = 0; j < E; ++j) acc[j] = fmaf(p, vv[j], acc[j] * corr);
+    mx = mn;
+  }
+#pragma unroll
+  for (int j = 0; j < E; ++j) part_acc[w][lane + 32 * j] = acc[j];
+  if (lane == 0) {
+    part_m[w] = mx;
+    part_l[w] = l;
+  }
+  __syncthreads();
+  if (w == 0) {
+    float M = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) M = fmaxf(M, part_m[i]);
+    float L = 0.f, out[E];
+#pragma unroll
+    for (int j = 0; j < E; ++j) out[j] = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float f = part_m[i] == -INFINITY ? 0.f : expf(part_m[i] - M);     // a warp without keys contributes nothing
+      L += part_l[i] * f;
+#pragma unroll
+      for (int j = 0; j < E; ++j) out[j] = fmaf(part_acc[i][lane + 32 * j], f, out[j]);
+    }
+    T* op = o + (static_cast<int64_t>(b) * Tn + t) * dq + hq * HD;
+    const float inv = 1.0f / L;
+#pragma unroll
+    for (int j = 0; j < E; ++j) op[lane + 32 * j] = from_f32<T>(out[j] * inv);
+  }
+}
 
 // ------------------------------------------------------------------------------ paired form
 // The two forwards of a ZO step (Definition 1: the loss at w + eps zbar and at w - eps zbar, same
@@ -611,6 +712,8 @@ cls2_pair_kernel(const float* __restrict__ a_last, int B, const __nv_bfloat16* _
   }
 }
 
+__global__ void set_i32_kernel(int32_t* p, int32_t v) { *p = v; }
+
 // *out = (sum of v[0..n)) / denom, fixed order, fp64.
 __global__ void __launch_bounds__(1024) mean_f64_kernel(const double* __restrict__ v, int64_t n, double denom,
                                                         double* __restrict__ out) {
@@ -688,6 +791,18 @@ struct szo_model {
   int32_t *d_tokens = nullptr, *d_labels = nullptr, *d_cand = nullptr;
   double* d_scalars = nullptr;
   int64_t last_launches = 0;
+  void *kcache = nullptr, *vcache = nullptr;     // [n_layers][max_batch][max_seq][n_kv_heads * head_dim], act dtype
+  szo_linear_t* decode_head = nullptr;           // LM head plan of the decode path when the loss path has none
+  int32_t* d_pos = nullptr;                      // cached positions before the current decode call
+  int32_t* dec_tokens = nullptr;                 // the call's tokens, at an address that a captured graph can keep
+  float* dec_logits = nullptr;                   // [max_batch][vocab]
+  struct DecodeGraph {
+    int B, T;
+    const float* Sv;
+    cudaGraphExec_t exec;
+  };
+  std::vector<DecodeGraph> dec_graphs;           // one captured token step per (B, T, sparse values)
+  bool dec_use_graph = true;
   bool z_valid = false;         // zkept holds the z of the last szo_model_zo_losses, not yet consumed
   std::vector<void*> owned;
   // measurement aid: CUDA events around every decoder-block linear launch
@@ -1018,6 +1133,82 @@ szo_status run_loss_paired(szo_model* m, const int32_t* tokens, const int32_t* l
     count_launch(4);
   }
   SZO_CHECK_LAUNCH("model kernels (paired form)");
+  return SZO_OK;
+}
+
+
+// T new tokens per sequence after pos0 cached positions (see szo_model_decode_step).
+template <typename T>
+szo_status run_decode_t(szo_model* m, const int32_t* tokens, int B, int Tn, const float* Sv, float* logits,
+                        cudaStream_t st) {
+  const int32_t* pos_dev = m->d_pos;                 // cached positions before this call, set by the caller
+  const szo_model_config& c = m->cfg;
+  const int64_t M = static_cast<int64_t>(B) * Tn;
+  const int d = c.d_model, H = c.n_heads, Hkv = c.n_kv_heads, hd = d / H, ff = c.d_ff;
+  const int64_t dkv = static_cast<int64_t>(Hkv) * hd, Smax = c.max_seq;
+  const int act = c.act_dtype;
+  const bool opt = c.arch == 1;
+  // few tokens: SZO_MODE_AUTO takes the weight-streaming kernel where it applies (the appendix's
+  // SparseAddMM order, the faster one for token generation)
+  const int32_t lmode = c.linear_mode == SZO_MODE_FP32_VALIDATE ? SZO_MODE_FP32_VALIDATE : SZO_MODE_AUTO;
+  T *a = static_cast<T*>(m->a), *q = static_cast<T*>(m->q), *k = static_cast<T*>(m->k), *v = static_cast<T*>(m->v),
+    *o = static_cast<T*>(m->o), *y = static_cast<T*>(m->y), *gate = static_cast<T*>(m->gate), *up = static_cast<T*>(m->up);
+  auto lin = [&](int layer, int j, const void* x, void* out) -> szo_status {
+    const int t = layer * m->n_lin + j;
+    return linear_fwd_impl(m->plans[t], x, act, M, Sv + m->offsets[t], nullptr, out, act, lmode, m->ws, m->ws_bytes, st);
+  };
+  embed_kernel<<<static_cast<unsigned>(M), 128, 0, st>>>(tokens, static_cast<const __nv_bfloat16*>(m->top.embed),
+                                                        static_cast<const __nv_bfloat16*>(m->top.pos), Tn, d, c.vocab, m->h, 0, pos_dev);
+  count_launch();
+  const T* pending = nullptr;
+  const int64_t layer_cache = static_cast<int64_t>(c.max_batch) * Smax * dkv;
+  for (int l = 0; l < c.n_layers; ++l) {
+    const szo_layer_weights& L = m->layers[l];
+    add_norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, pending, L.attn_norm_g, L.attn_norm_b, d, c.norm_eps,
+                                                                opt, 1, 0, a);
+    count_launch();
+    SZO_TRY(lin(l, 0, a, q));
+    SZO_TRY(lin(l, 1, a, k));
+    SZO_TRY(lin(l, 2, a, v));
+    if (!opt) {
+      const int64_t n_vec = M * (H + Hkv) * ((hd / 2) / Vec16<T>::kN);
+      rope_kernel<T><<<blocks_for(n_vec, 256), 256, 0, st>>>(q, k, m->rope_tab, M, Tn, H, Hkv, hd, 0, pos_dev);
+      count_launch();
+    }
+    T* kc = static_cast<T*>(m->kcache) + l * layer_cache;
+    T* vc = static_cast<T*>(m->vcache) + l * layer_cache;
+    const int64_t n_vec = M * dkv / Vec16<T>::kN;
+    kv_append_kernel<T><<<blocks_for(2 * n_vec, 256), 256, 0, st>>>(k, v, kc, vc, Tn, pos_dev, Smax, dkv, n_vec);
+    dim3 grid(static_cast<unsigned>(Tn), H, B);
+    const float scale = 1.0f / sqrtf(static_cast<float>(hd));
+    if (hd == 64) attn_decode_kernel<T, 64><<<grid, 128, 0, st>>>(q, kc, vc, o, Tn, pos_dev, Smax, H, Hkv, scale);
+    else attn_decode_kernel<T, 128><<<grid, 128, 0, st>>>(q, kc, vc, o, Tn, pos_dev, Smax, H, Hkv, scale);
+    count_launch(2);
+    SZO_TRY(lin(l, 3, o, y));
+    add_norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, y, L.mlp_norm_g, L.mlp_norm_b, d, c.norm_eps, opt, 1, 0, a);
+    count_launch();
+    if (!opt) {
+      SZO_TRY(lin(l, 4, a, gate));
+      SZO_TRY(lin(l, 5, a, up));
+      silu_mul_kernel<T><<<blocks_for(M * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, up, M * ff, gate);
+      count_launch();
+      SZO_TRY(lin(l, 6, gate, y));
+    } else {
+      SZO_TRY(lin(l, 4, a, gate));
+      relu_kernel<T><<<blocks_for(M * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, M * ff);
+      count_launch();
+      SZO_TRY(lin(l, 5, gate, y));
+    }
+    pending = y;
+  }
+  // the last new token of every sequence: final norm, LM head
+  add_norm_kernel<T><<<static_cast<unsigned>(B), 256, 0, st>>>(m->h, pending, m->top.final_norm_g, m->top.final_norm_b, d,
+                                                              c.norm_eps, opt, Tn, Tn - 1, a);
+  count_launch();
+  szo_linear_t* head = m->lm_head_plan != nullptr ? m->lm_head_plan : m->decode_head;
+  const int hmode = lmode == SZO_MODE_FP32_VALIDATE ? SZO_MODE_FP32_VALIDATE : SZO_MODE_SPARSE_ADD;
+  SZO_TRY(szo_linear_fwd(head, a, static_cast<szo_dtype>(act), B, nullptr, logits, SZO_F32, hmode, m->ws, m->ws_bytes, st));
+  SZO_CHECK_LAUNCH("decode kernels");
   return SZO_OK;
 }
 
@@ -1397,6 +1588,101 @@ szo_status szo_model_zo_step_host(szo_model_t* m, const int32_t* tokens_host, co
   return SZO_OK;
 }
 
+szo_status szo_model_enable_decode(szo_model_t* m, void* stream) {
+  SZO_REQUIRE(m != nullptr, SZO_ERR_INVALID_ARG, "model is NULL");
+  if (m->kcache != nullptr) return SZO_OK;
+  const szo_model_config& c = m->cfg;
+  const size_t e = c.act_dtype == SZO_F32 ? 4 : 2;
+  const size_t bytes = static_cast<size_t>(c.n_layers) * c.max_batch * c.max_seq * c.n_kv_heads * (c.d_model / c.n_heads) * e;
+  SZO_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->kcache), bytes));
+  SZO_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->vcache), bytes));
+  SZO_TRY(dev_alloc(m, &m->d_pos, sizeof(int32_t)));
+  SZO_TRY(dev_alloc(m, &m->dec_tokens, static_cast<size_t>(m->Mmax) * sizeof(int32_t)));
+  SZO_TRY(dev_alloc(m, &m->dec_logits, static_cast<size_t>(c.max_batch) * c.vocab * sizeof(float)));
+  SZO_REQUIRE(device_status_word() != nullptr, SZO_ERR_CUDA, "no device status word");    // allocated outside any capture
+  {
+    const char* env = getenv("SZO_DECODE_GRAPH");
+    m->dec_use_graph = !(env != nullptr && env[0] == '0');
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (m->lm_head_plan == nullptr) {
+    SZO_TRY(szo_linear_create(&m->decode_head, c.vocab, c.d_model, 0, m->top.lm_head, nullptr, nullptr, SZO_BF16, nullptr,
+                              0, nullptr, st));
+    const int32_t hmode = c.linear_mode == SZO_MODE_FP32_VALIDATE ? SZO_MODE_FP32_VALIDATE : SZO_MODE_SPARSE_ADD;
+    const size_t need = szo_linear_workspace_bytes(m->decode_head, c.max_batch, hmode);
+    if (need > m->ws_bytes) {
+      SZO_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->ws), need));      // the earlier workspace stays owned and is freed with the model
+      m->ws_bytes = need;
+    }
+  }
+  // the few-token linears of the decode path (SZO_MODE_AUTO) may want more workspace than the loss path's mode
+  if (c.linear_mode != SZO_MODE_FP32_VALIDATE) {
+    size_t need = m->ws_bytes;
+    for (szo_linear_t* p : m->plans) {
+      const size_t w = szo_linear_workspace_bytes(p, m->Mmax, SZO_MODE_AUTO);
+      if (w > need) need = w;
+    }
+    if (need > m->ws_bytes) {
+      SZO_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->ws), need));
+      m->ws_bytes = need;
+    }
+  }
+  return SZO_OK;
+}
+
+szo_status szo_model_decode_step(szo_model_t* m, const int32_t* tokens, int32_t B, int32_t T, int32_t pos0,
+                                 const float* S_vals, float* logits_dev, void* stream) {
+  SZO_REQUIRE(m != nullptr && tokens != nullptr && logits_dev != nullptr, SZO_ERR_INVALID_ARG, "NULL argument");
+  SZO_REQUIRE(m->kcache != nullptr, SZO_ERR_INVALID_ARG, "call szo_model_enable_decode first");
+  SZO_REQUIRE(B >= 1 && B <= m->cfg.max_batch && T >= 1 && pos0 >= 0 && pos0 + T <= m->cfg.max_seq, SZO_ERR_SHAPE,
+              "need 1 <= B <= %d, T >= 1 and pos0 + T <= %d (got B=%d, T=%d, pos0=%d)", m->cfg.max_batch, m->cfg.max_seq, B,
+              T, pos0);
+  SZO_REQUIRE(static_cast<int64_t>(B) * T <= m->Mmax, SZO_ERR_SHAPE, "B * T exceeds max_batch * max_seq");
+  SZO_REQUIRE(m->cfg.arch == 0 || pos0 + T <= m->cfg.max_pos, SZO_ERR_SHAPE, "position beyond the position table");
+  const float* Sv = S_vals ? S_vals : m->S_all;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  auto run = [&](const int32_t* toks, float* out) -> szo_status {
+    if (m->cfg.act_dtype == SZO_F32) return run_decode_t<float>(m, toks, B, T, Sv, out, st);
+    return run_decode_t<__nv_bfloat16>(m, toks, B, T, Sv, out, st);
+  };
+  set_i32_kernel<<<1, 1, 0, st>>>(m->d_pos, pos0);
+  count_launch();
+  // A token step is several hundred short launches: on a stream that can be captured it is recorded once
+  // per (B, T, sparse values) as a CUDA graph and replayed (the position comes from device memory, the
+  // tokens and logits pass through buffers of the model); the legacy default stream runs it launch by launch.
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  const bool capturable = m->dec_use_graph && st != nullptr && st != cudaStreamLegacy &&
+                          cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone;
+  if (!capturable) return run(tokens, logits_dev);
+  SZO_CHECK_CUDA(cudaMemcpyAsync(m->dec_tokens, tokens, static_cast<size_t>(B) * T * sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
+  cudaGraphExec_t exec = nullptr;
+  for (const auto& g : m->dec_graphs)
+    if (g.B == B && g.T == T && g.Sv == Sv) exec = g.exec;
+  if (exec == nullptr) {
+    SZO_CHECK_CUDA(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+    const szo_status rc = run(m->dec_tokens, m->dec_logits);
+    cudaGraph_t graph = nullptr;
+    const cudaError_t ce = cudaStreamEndCapture(st, &graph);
+    if (rc != SZO_OK) {
+      if (graph) cudaGraphDestroy(graph);
+      return rc;
+    }
+    SZO_REQUIRE(ce == cudaSuccess && graph != nullptr, SZO_ERR_CUDA, "capture of the token step failed: %s", cudaGetErrorString(ce));
+    const cudaError_t ie = cudaGraphInstantiate(&exec, graph, 0);
+    cudaGraphDestroy(graph);
+    SZO_REQUIRE(ie == cudaSuccess, SZO_ERR_CUDA, "cudaGraphInstantiate failed: %s", cudaGetErrorString(ie));
+    if (m->dec_graphs.size() >= 8) {            // a small cache: drop the oldest
+      cudaGraphExecDestroy(m->dec_graphs.front().exec);
+      m->dec_graphs.erase(m->dec_graphs.begin());
+    }
+    m->dec_graphs.push_back({B, T, Sv, exec});
+  }
+  SZO_CHECK_CUDA(cudaGraphLaunch(exec, st));
+  SZO_CHECK_CUDA(cudaMemcpyAsync(logits_dev, m->dec_logits, static_cast<size_t>(B) * m->cfg.vocab * sizeof(float),
+                                 cudaMemcpyDeviceToDevice, st));
+  return SZO_OK;
+}
+
 szo_status szo_model_enable_timing(szo_model_t* m, int32_t on) {
   SZO_REQUIRE(m != nullptr, SZO_ERR_INVALID_ARG, "model is NULL");
   m->timing = on != 0;
@@ -1424,6 +1710,8 @@ void szo_model_destroy(szo_model_t* m) {
   for (cudaEvent_t e : m->events) cudaEventDestroy(e);
   for (szo_linear_t* p : m->plans) szo_linear_destroy(p);
   szo_linear_destroy(m->lm_head_plan);
+  szo_linear_destroy(m->decode_head);
+  for (auto& g : m->dec_graphs) cudaGraphExecDestroy(g.exec);
   for (void* p : m->owned) cudaFree(p);
   delete m;
 }

@@ -292,9 +292,62 @@ def step_case(name, Bn, S, loss, steps, eps, lr, profile_range=False, form="pair
     model.close()
 
 
+def decode_case(name, Bn, prompt, gen):
+    """Token generation with a KV cache (szo_model_decode_step): a prompt of `prompt` tokens in one
+    call, then `gen` calls of one token per sequence, timed with CUDA events over the generation loop.
+    Every step streams all linear weights once, so the roofline is the weight bytes over the HBM
+    bandwidth."""
+    shape = wl.MODEL_SHAPES[name]
+    tensors, S_all = wl.device_decoder_tensors(shape, seed=0)
+    model = B.Model(shape, wl.linear_names(shape), tensors, S_all, act_dtype=B.SZO_BF16, linear_mode=B.MODE_SPARSE_ADD,
+                    loss_kind=B.LOSS_LM, max_batch=Bn, max_seq=prompt + gen)
+    model.enable_decode()
+    g = torch.Generator(device="cuda")
+    g.manual_seed(1)
+    toks = torch.randint(0, shape["vocab"], (Bn, prompt), generator=g, device="cuda", dtype=torch.int32)
+    logits = torch.empty((Bn, shape["vocab"]), dtype=torch.float32, device="cuda")
+    nxt = torch.empty((Bn, 1), dtype=torch.int32, device="cuda")
+
+    def run():
+        model.decode_step(toks, 0, logits)
+        for i in range(gen):
+            nxt.copy_(torch.argmax(logits, dim=1, keepdim=True))          # greedy choice, on the device
+            model.decode_step(nxt, prompt + i, logits)
+
+    stream = torch.cuda.Stream()          # a token step is replayed as a CUDA graph on a non-default stream
+    with torch.cuda.stream(stream):
+        run()
+        stream.synchronize()
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        e0.record(stream)
+        model.decode_step(toks, 0, logits)
+        e1.record(stream)
+        for i in range(gen):
+            nxt.copy_(torch.argmax(logits, dim=1, keepdim=True))
+            model.decode_step(nxt, prompt + i, logits)
+        e2.record(stream)
+        stream.synchronize()
+    ms_gen = e1.elapsed_time(e2)
+    weight_bytes = 0
+    for nm in wl.linear_names(shape):
+        N, K = wl.linear_shape(shape, nm)
+        weight_bytes += (N * K // 2 + 4 * N * K // shape["group"]) if shape["group"] > 0 else 2 * N * K
+    weight_bytes = weight_bytes * shape["n_layers"] + 2 * shape["vocab"] * shape["d_model"]
+    hbm = peaks()[0]
+    per_step_ms = ms_gen / gen
+    print(json.dumps({"case": "decode", "model": name, "batch": Bn, "prompt": prompt, "generated": gen,
+                      "prompt_ms": e0.elapsed_time(e1), "ms_per_token_step": per_step_ms,
+                      "tokens_per_s": Bn * gen / ms_gen * 1e3, "weight_bytes_per_step": weight_bytes,
+                      "roofline_ms_per_step": weight_bytes / hbm / 1e6, "frac_of_hbm": weight_bytes / hbm / 1e6 / per_step_ms,
+                      "device_status": B.device_status()}))
+    model.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["linear", "paired", "steady", "sparse", "sweep", "attention", "step"])
+    ap.add_argument("what", choices=["linear", "paired", "steady", "sparse", "sweep", "attention", "step", "decode"])
+    ap.add_argument("--prompt", type=int, default=16)
+    ap.add_argument("--gen", type=int, default=128)
     ap.add_argument("--model", default="mistral_7b", choices=sorted(wl.MODEL_SHAPES))
     ap.add_argument("--batch", type=int, default=8)
     ap.add_argument("--seq", type=int, default=512)
@@ -318,6 +371,8 @@ def main():
     B.lib()
     if a.what == "linear":
         linear_case(a.M, a.N, a.K, a.G, a.mode, a.rho, a.reps)
+    elif a.what == "decode":
+        decode_case(a.model, a.batch, a.prompt, a.gen)
     elif a.what == "paired":
         paired_case(a.M, a.N, a.K, a.G, a.rho, a.reps)
     elif a.what == "steady":
