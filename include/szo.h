@@ -313,6 +313,13 @@ szo_status szo_model_zo_step(szo_model_t* m, const int32_t* tokens, const int32_
                              const int32_t* cand, int32_t B, int32_t S, uint64_t seed,
                              uint64_t step, float eps, float lr, double* f_plus_dev,
                              double* f_minus_dev, double* g_dev, void* stream);
+/* n-sample SPSA (Definition 1 averaged over n independent perturbations; the paper's runs use n = 1, for
+ * which this is szo_model_zo_step): for i = 0 .. n-1, z_i is drawn for the counter step * n + i and both
+ * losses are evaluated around the same S; then S -= (lr / n) g_i z_i for i = 0 .. n-1 in turn.
+ * f_plus_dev, f_minus_dev, g_dev: fp64 device arrays of n entries. */
+szo_status szo_model_zo_step_n(szo_model_t* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand,
+                               int32_t B, int32_t S, uint64_t seed, uint64_t step, int32_t n, float eps, float lr,
+                               double* f_plus_dev, double* f_minus_dev, double* g_dev, void* stream);
 /* The step in two halves, for data-parallel replicas (Definition 1 evaluates f on a batch: replicas that
  * hold the same weights, mask and S and use the same (seed, step) draw the same z, evaluate f+ and f-
  * on their own share of the batch and need to exchange only sums of losses before each applies the

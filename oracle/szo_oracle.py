@@ -293,6 +293,30 @@ def zo_update_scale(f_plus: float, f_minus: float, eps, lr) -> np.float32:
     return np.float32(-(float(np.float32(lr)) * g))
 
 
+def zo_sgd_step_n(loss, S, gidx, seed: int, step: int, n: int, eps, lr):
+    """n-sample SPSA (Definition 1 averaged over n independent perturbations, the usual variance
+    reduction of a ZO estimate; the paper's runs use n = 1): for i = 0 .. n-1, z_i is drawn for the
+    counter step * n + i, both losses are evaluated around the SAME S (in the in-place order
+    +eps, -2 eps, +eps, which returns S to within an ulp or two), g_i = (f+_i - f-_i) / (2 eps); then
+    S <- S - (lr / n) g_i z_i for i = 0 .. n-1 in turn.  Returns (S_new, [f+_i], [f-_i], [g_i]).
+    n = 1 is zo_sgd_step."""
+    e = np.float32(eps)
+    S = np.asarray(S, dtype=np.float32)
+    fps, fms, gs = [], [], []
+    for i in range(n):
+        c = step * n + i
+        S = perturb(S, gidx, seed, c, e)
+        fps.append(float(loss(S)))
+        S = perturb(S, gidx, seed, c, np.float32(-2.0) * e)
+        fms.append(float(loss(S)))
+        S = perturb(S, gidx, seed, c, e)
+        gs.append(projected_gradient(fps[-1], fms[-1], e))
+    lr_n = float(np.float32(lr)) / n
+    for i in range(n):
+        S = perturb(S, gidx, seed, step * n + i, np.float32(-(lr_n * gs[i])))
+    return S, fps, fms, gs
+
+
 def replay(S0, gidx, seed: int, log, eps, lr) -> np.ndarray:
     """Section 2.1: the run's effect on the sparse values from its log [(step_t, g_t), ...] alone.  For
     every logged step, in order: the +eps, -2 eps, +eps passes (when eps != 0: they leave S within an

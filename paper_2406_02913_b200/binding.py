@@ -106,6 +106,9 @@ _SIGS = {
     "szo_model_zo_step": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                       C.c_int32, C.c_uint64, C.c_uint64, C.c_float, C.c_float,
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "szo_model_zo_step_n": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                        C.c_uint64, C.c_uint64, C.c_int32, C.c_float, C.c_float, C.c_void_p,
+                                        C.c_void_p, C.c_void_p, C.c_void_p]),
     "szo_model_zo_losses": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                         C.c_uint64, C.c_uint64, C.c_float, C.c_void_p, C.c_void_p]),
     "szo_model_zo_apply": (C.c_int32, [C.c_void_p, C.c_float, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -393,6 +396,14 @@ class Model:
                                        eps, lr, sc[0:1].data_ptr(), sc[1:2].data_ptr(),
                                        sc[2:3].data_ptr(), _stream()))
         return sc[:3]
+
+    def zo_step_n(self, tokens, seed, step, n, eps, lr, labels=None, cand=None) -> torch.Tensor:
+        """n-sample SPSA step; returns the device tensor [3, n] of (f+_i, f-_i, g_i) (fp64)."""
+        B, S = tokens.shape
+        out = torch.zeros((3, n), dtype=torch.float64, device=self.S_all.device)
+        _check(lib().szo_model_zo_step_n(self.h, _ptr(tokens), _ptr(labels), _ptr(cand), B, S, seed, step, n, eps, lr,
+                                         out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr(), _stream()))
+        return out
 
     def zo_losses(self, tokens, seed, step, eps, labels=None, cand=None, sums=None) -> torch.Tensor:
         """First half of a step on this replica's share of the batch: returns the device tensor

@@ -1536,6 +1536,32 @@ szo_status szo_model_zo_step(szo_model_t* m, const int32_t* tokens, const int32_
   return SZO_OK;
 }
 
+szo_status szo_model_zo_step_n(szo_model_t* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand,
+                               int32_t B, int32_t S, uint64_t seed, uint64_t step, int32_t n, float eps, float lr,
+                               double* f_plus_dev, double* f_minus_dev, double* g_dev, void* stream) {
+  SZO_TRY(check_batch(m, tokens, labels, cand, B, S));
+  SZO_REQUIRE(f_plus_dev && f_minus_dev && g_dev, SZO_ERR_INVALID_ARG, "NULL output array");
+  SZO_REQUIRE(eps != 0.f && n >= 1 && n <= 1024, SZO_ERR_INVALID_ARG, "need eps != 0 and 1 <= n <= 1024");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t before = g_launch_count;
+  // every sample's losses around the same S (each call returns S to where the +eps, -2 eps, +eps order leaves it)
+  for (int32_t i = 0; i < n; ++i) {
+    const uint64_t c = step * static_cast<uint64_t>(n) + static_cast<uint64_t>(i);
+    SZO_TRY(zo_losses_impl(m, tokens, labels, cand, B, S, seed, c, eps, f_plus_dev + i, f_minus_dev + i, st));
+    SZO_TRY(szo_projected_gradient(f_plus_dev + i, f_minus_dev + i, eps, g_dev + i, st));
+  }
+  // S -= (lr / n) g_i z_i, i in turn; z_i is regenerated (only the last sample's z is still kept)
+  const float lr_n = static_cast<float>(static_cast<double>(lr) / n);
+  for (int32_t i = 0; i < n; ++i) {
+    const uint64_t c = step * static_cast<uint64_t>(n) + static_cast<uint64_t>(i);
+    ScaleArg su{0.f, lr_n, eps, f_plus_dev + i, f_minus_dev + i};
+    SZO_TRY(launch_sparse_axpy(m->S_all, m->S_all, m->gidx, m->k_total, 0, seed, c, su, st));
+  }
+  m->z_valid = false;
+  m->last_launches = g_launch_count - before;
+  return SZO_OK;
+}
+
 szo_status szo_model_zo_losses(szo_model_t* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand,
                                int32_t B, int32_t S, uint64_t seed, uint64_t step, float eps, double* sums_dev,
                                void* stream) {

@@ -305,3 +305,26 @@ def test_replay_from_the_g_log_reproduces_the_sparse_values(B, tiny):
     B.szo_replay(S_plain, m.gidx(), 0, 1234, log, 0.0, lr)
     assert torch.allclose(S_plain, S, rtol=0, atol=1e-6) and not torch.equal(S_plain, S0)
     m.close()
+
+
+def test_n_sample_spsa_step_matches_the_oracle(B, tiny):
+    """szo_model_zo_step_n with n = 3 on the fp32 validation path against the oracle's n-sample step
+    (losses, the three projected gradients, the updated S); n = 1 equals szo_model_zo_step."""
+    fx = tiny
+    toks = fx.batch(0)
+    eps, lr = 1e-3, 1e-3
+    om = fx.oracle_model()
+    S_ref, fps, fms, gs = so.zo_sgd_step_n(lambda S_: om.loss(S_, toks), om.S, om.gidx, 1234, 2, 3, eps, lr)
+    m, S, _ = build_gpu(B, fx, B.SZO_F32, B.MODE_FP32_VALIDATE)
+    out = m.zo_step_n(torch.from_numpy(toks).cuda(), 1234, 2, 3, eps, lr).cpu().numpy()
+    for i in range(3):
+        assert abs(out[0, i] - fps[i]) <= 2e-6 * abs(fps[i]) and abs(out[1, i] - fms[i]) <= 2e-6 * abs(fms[i])
+        assert abs(out[2, i] - gs[i]) <= g_tol(gs[i], fps[i], eps)
+    assert np.allclose(S.cpu().numpy(), S_ref, rtol=0, atol=3e-7)
+    m1, S1, _ = build_gpu(B, fx, B.SZO_F32, B.MODE_FP32_VALIDATE)
+    m2, S2, _ = build_gpu(B, fx, B.SZO_F32, B.MODE_FP32_VALIDATE)
+    a = m1.zo_step_n(torch.from_numpy(toks).cuda(), 1234, 5, 1, eps, lr).cpu().numpy()[:, 0]
+    b = m2.zo_step(torch.from_numpy(toks).cuda(), 1234, 5, eps, lr).cpu().numpy()
+    assert tuple(a) == tuple(b) and torch.equal(S1, S2)
+    for mm in (m, m1, m2):
+        mm.close()

@@ -383,6 +383,50 @@ def test_zo_sgd_update_and_replay_identity():
     assert np.allclose(S, S0 - acc, rtol=0, atol=1e-6)        # S_T = S_0 - sum_t lr g_t z_t
 
 
+def test_n_sample_spsa_reduces_to_one_sample_and_averages():
+    """zo_sgd_step_n: n = 1 is zo_sgd_step bit for bit; for a linear loss a.w the update is exactly
+    -(lr/n) sum_i (zbar_i . a) zbar_i with the z of counters step*n + i; and the estimate's spread around
+    the true masked gradient shrinks like 1/sqrt(n)."""
+    A, w, idx = _quad_problem(d=64, k=10)
+    state = w.copy()
+
+    def quad(S):
+        v = state.astype(np.float64).copy()
+        v[idx] = S
+        return 0.5 * v @ A @ v
+
+    one = so.zo_sgd_step(quad, state[idx], idx, 3, 11, 1e-3, 1e-2)
+    n1 = so.zo_sgd_step_n(quad, state[idx], idx, 3, 11, 1, 1e-3, 1e-2)
+    assert np.array_equal(one[0].view(np.uint32), n1[0].view(np.uint32)) and one[3] == n1[3][0]
+    g = np.random.default_rng(4)
+    a = g.standard_normal(64)
+
+    def lin(S):
+        v = state.astype(np.float64).copy()
+        v[idx] = S
+        return float(a @ v)
+
+    eps, lr, n = np.float32(1e-3), np.float32(1e-3), 4
+    S_new, fps, fms, gs = so.zo_sgd_step_n(lin, state[idx], idx, 9, 5, n, eps, lr)
+    exp = state[idx].astype(np.float64)
+    for i in range(n):
+        z = so.gaussian(9, 5 * n + i, idx).astype(np.float64)
+        assert abs(gs[i] - z @ a[idx]) < 1e-3 * abs(z @ a[idx]) + 1e-4          # fp32 S limits the difference quotient
+        exp = exp - float(lr) / n * gs[i] * z
+    assert np.allclose(S_new, exp, rtol=0, atol=1e-6)
+    # spread of the estimate (sum_i g_i z_i / n) around a[idx]: n = 16 against n = 1 over 400 draws each
+    def spread(n):
+        err = []
+        for t in range(400):
+            est = np.zeros(10)
+            for i in range(n):
+                z = so.gaussian(21, t * n + i, idx).astype(np.float64)
+                est += (z @ a[idx]) * z / n
+            err.append(np.sum((est - a[idx]) ** 2))
+        return np.mean(err)
+    assert 10.0 < spread(1) / spread(16) < 24.0
+
+
 def test_replay_from_the_log_reproduces_the_run():
     """so.replay against the run it replays (itself pinned above): the same bits when the +-eps passes
     are replayed too, and S_0 - sum_t lr g_t z_t up to their drift when they are skipped."""
