@@ -769,6 +769,16 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
     n_tiles += sb.n_tiles;
   }
   P.n_tiles = n_tiles;
+  // bands of token tiles that fit L2 with room to spare (about 32 MB of tokens per band)
+  {
+    static const int band_env = [] {
+      const char* e = getenv("SZO_TILE_BAND");
+      return e == nullptr ? -1 : atoi(e);
+    }();
+    int band = static_cast<int>((32ll << 20) / (256 * p0->K * 2));
+    if (band_env >= 0) band = band_env;
+    P.m_band = (band > 0 && P.m_tiles > band) ? band : 0;
+  }
   P.y_f32 = (y_dtype == SZO_F32) ? 1 : 0;
   P.status = device_status_word();
   SZO_REQUIRE(P.status != nullptr, SZO_ERR_CUDA, "no device status word");

@@ -127,8 +127,19 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& P, int pair, int n_p
     u.kb1 = tail_kb_at(P, u.part + 1);
   }
   const int m_tiles = static_cast<int>(P.m_tiles);
-  int np = tile / m_tiles;
-  u.m_tile = tile - np * m_tiles;
+  int np;
+  if (P.m_band > 0) {
+    const int per_band = static_cast<int>(P.n_tiles) * P.m_band;
+    const int band = tile / per_band;
+    const int r = tile - band * per_band;
+    const int m_first = band * P.m_band;
+    const int width = (m_tiles - m_first < P.m_band) ? m_tiles - m_first : P.m_band;      // the last band may be narrower
+    np = r / width;
+    u.m_tile = m_first + (r - np * width);
+  } else {
+    np = tile / m_tiles;
+    u.m_tile = tile - np * m_tiles;
+  }
   if (P.pair_ext && static_cast<int64_t>(u.m_tile) * 256 >= P.pair_row0) {
     u.kb0 *= 2;          // half-difference token tile: twice the k-blocks (xd W^T, then xc (eps Zbar)^T)
     u.kb1 *= 2;
@@ -332,6 +343,7 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     if (lane == 0) {
       RingPos x{0, 0};
       bool ok = true;
+      const uint64_t keep = l2_policy_evict_last();
       for (int lt = 0; lt < my_units && ok; ++lt) {
         const Unit u = decode_unit(P, pair, n_pairs, rank, lt);
         const int tok0 = u.m_tile * kPairBT + rank * 128;
@@ -346,7 +358,7 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
               xt -= static_cast<int>(P.pair_row0);
             }
           }
-          tma_load_2d(tiles_base + b_off(x.idx), &tmap_x, xk, xt, xfull_bar(x.idx));
+          tma_load_2d_hint(tiles_base + b_off(x.idx), &tmap_x, xk, xt, xfull_bar(x.idx), keep);
           if constexpr (!kDequant) tma_load_2d(tiles_base + a_off(x.idx, 0), &tmap_w, kb * kBK, row0, xfull_bar(x.idx));
           x.advance(kXS);
         }
@@ -616,6 +628,7 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
   } else if (warp >= kEpiWarp02) {
     // ---------------------------------------------------------------- epilogue (own 128 rows)
     const int qd = warp & 3;
+    const uint64_t stream_out = l2_policy_evict_first();
     for (int lt = 0; lt < my_units; ++lt) {
       const Unit u = decode_unit(P, pair, n_pairs, rank, lt);
       const int as = lt & 1;
@@ -662,8 +675,8 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
 #pragma unroll
               for (int j = 0; j < 32; j += 2) {
                 const __nv_bfloat162 pr = __floats2bfloat162_rn(act(__uint_as_float(v[j])), act(__uint_as_float(v[j + 1])));
-                yp[0] = pr.x;
-                yp[N] = pr.y;
+                st_bf16_hint(yp, pr.x, stream_out);
+                st_bf16_hint(yp + N, pr.y, stream_out);
                 yp += 2 * N;
               }
             } else if (cnt >= 32) {
@@ -671,8 +684,8 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
               for (int j = 0; j < 32; j += 2) {
                 const __nv_bfloat162 pr = __floats2bfloat162_rn(act(__uint_as_float(v[j]) + bias),
                                                                 act(__uint_as_float(v[j + 1]) + bias));
-                yp[0] = pr.x;
-                yp[N] = pr.y;
+                st_bf16_hint(yp, pr.x, stream_out);
+                st_bf16_hint(yp + N, pr.y, stream_out);
                 yp += 2 * N;
               }
             } else {

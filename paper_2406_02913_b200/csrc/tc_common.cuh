@@ -37,6 +37,12 @@ struct TcParams {
   int G;
   int nkb;                 // K / 64
   int64_t m_tiles, n_tiles;   // 256-token tiles; 256-row pair tiles of all matrices together
+  // Tile order.  0: weight tile slowest, token tile fastest (a weight tile meets every token tile while it
+  // is hot).  m_band > 0: the token tiles are taken in bands of m_band; inside a band the order is as before.
+  // The tokens of a band (m_band x 256 x K bf16) then stay in L2 across the rounds of tiles, at the
+  // price of one more pass over the weights per band: with 8192 token rows of K = 4096 the whole token
+  // matrix (67 MB) was re-read from DRAM by most rounds (1.6 GB per launch against 0.6 GB algorithmic).
+  int m_band;
   int y_f32;
   int relu;                // y = max(y, 0) in the epilogue (the ReLU of an OPT-style MLP after its first matrix)
   int32_t* status;
@@ -142,6 +148,29 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
       : "memory");
+}
+// L2 eviction priorities: the token matrix is re-read by every round of tiles and should stay, the output
+// is written once and should not push it out.
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar,
+                                                 uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void st_bf16_hint(__nv_bfloat16* p, __nv_bfloat16 v, uint64_t policy) {
+  asm volatile("st.global.L2::cache_hint.b16 [%0], %1, %2;" ::"l"(p), "h"(*reinterpret_cast<const unsigned short*>(&v)), "l"(policy)
+               : "memory");
 }
 __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
