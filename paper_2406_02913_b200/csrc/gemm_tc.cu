@@ -220,6 +220,7 @@ szo_status linear_fwd_tc_group(const szo_linear* const* plans, int n, const void
   for (int i = 0; i < 5; ++i) P.tail_kb[i] = sc.tail_kb[i];
   P.partial = static_cast<float*>(ws);
   P.tickets = t->tickets;
+  P.tickets_done = t->tickets + (t->sms / 2) * 4;
   SZO_TRY(refresh_tickets(t, st));
   return launch_pair_kernel(p0->G != 0, p0->sz_dtype == SZO_BF16, mx, t->w_map, P, sc.n_pairs, st);
 }
@@ -794,6 +795,7 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
   for (int i = 0; i < 5; ++i) P.tail_kb[i] = sc.tail_kb[i];
   P.partial = static_cast<float*>(tail);
   P.tickets = t->tickets;
+  P.tickets_done = t->tickets + (t->sms / 2) * 4;
   SZO_TRY(refresh_tickets(t, st));
   const size_t y_elt = (y_dtype == SZO_F32) ? 4 : 2;
   const int n_sets = S_second != nullptr ? 2 : 1;
@@ -834,7 +836,12 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
     }
     const size_t per_token = static_cast<size_t>(p0->K) * sizeof(__nv_bfloat16);
     const bool f32 = y_dtype == SZO_F32;
-    if (16 * per_token <= 200 * 1024 && M >= 2048) SZO_TRY(launch_pair_cross_tm<16>(ca, max_N, even, f32, st));
+    static const int tm_env = [] {
+      const char* e = getenv("SZO_CROSS_TM");
+      return e == nullptr ? 0 : atoi(e);
+    }();
+    if (tm_env == 8 && 8 * per_token <= 200 * 1024) SZO_TRY(launch_pair_cross_tm<8>(ca, max_N, even, f32, st));
+    else if (16 * per_token <= 200 * 1024 && M >= 2048) SZO_TRY(launch_pair_cross_tm<16>(ca, max_N, even, f32, st));
     else if (8 * per_token <= 200 * 1024) SZO_TRY(launch_pair_cross_tm<8>(ca, max_N, even, f32, st));
     else if (4 * per_token <= 200 * 1024) SZO_TRY(launch_pair_cross_tm<4>(ca, max_N, even, f32, st));
     else {

@@ -160,17 +160,18 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& P, int pair, int n_p
 // Fields of matrix s, selected without indexing the parameter block dynamically.
 #define SZO_SUB(P, s, f) ((s) == 0 ? (P).sub[0].f : ((s) == 1 ? (P).sub[1].f : (P).sub[2].f))
 
-// Sum of the K-split parts of one CTA's 128 rows x 256 tokens, + bias, stored to y; run by every
-// thread of the CTA after its roles have finished.  A part is [token][128 rows] fp32, parts are
+// Sum of the K-split parts of one CTA's 128 rows, tokens [t_begin, mlimit) of the tile, + bias, stored to
+// y; run by every thread of the CTA after its roles have finished.  A part is [token][128 rows] fp32, parts are
 // 2 * 256 * 128 floats apart; the sum runs in part order, so the result does not depend on which
 // part finished last.  Thread -> one float4 (4 rows of one token) per step of nthreads, seven in
 // flight per part.  Kept out of line: its registers would otherwise add to every role's.
 __device__ __noinline__ void reduce_parts(const float* part0, int parts, int64_t n0, int64_t N, const float* bias_p,
-                                          void* y, int y_f32, int relu, int64_t m0, int mlimit, int tid, int nthreads) {
+                                          void* y, int y_f32, int relu, int64_t m0, int t_begin, int mlimit, int tid,
+                                          int nthreads) {
   constexpr int64_t kPartFloats = static_cast<int64_t>(kPairBT) * kBM;
   constexpr int kBatch = 7;
-  const int total = mlimit * (kBM / 4);          // float4s of the valid tokens
-  for (int base = tid; base < total; base += nthreads * kBatch) {
+  const int total = mlimit * (kBM / 4);          // float4s up to the last token of this share
+  for (int base = t_begin * (kBM / 4) + tid; base < total; base += nthreads * kBatch) {
     float4 acc[kBatch];
 #pragma unroll
     for (int i = 0; i < kBatch; ++i) {
@@ -727,12 +728,8 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         __syncwarp();
         if (lane == 0 && atomicAdd_block(&epi_count_s, 1) == 3) {
           __threadfence();
-          int32_t* ticket = P.tickets + u.slot * 2 + rank;
-          if (atomicAdd(ticket, 1) == u.parts - 1) {
-            *ticket = 0;                       // ready for the next launch
-            __threadfence();                   // the other parts' tiles are read after this point
-            reduce_flag_s = 1;
-          }
+          atomicAdd(P.tickets + u.slot * 2 + rank, 1);      // this part is parked
+          reduce_flag_s = 1;                                 // this CTA sums a share of the tile's tokens
         }
       }
     }
@@ -745,19 +742,43 @@ szo_linear_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
   tc_fence_before();
   __syncthreads();
   if (reduce_flag_s && !*abort_flag) {
-    // (the thread that took the last ticket fenced before raising the flag; the parts are read from
-    // L2 with ld.cg, and a fence by all 640 threads here measured about 7 us)
     constexpr int64_t kPartFloats = static_cast<int64_t>(kPairBT) * kBM;
     const Unit u = decode_unit(P, pair, n_pairs, rank, my_units - 1);
-    const int64_t m0 = static_cast<int64_t>(u.m_tile) * kPairBT;
-    const int mlimit = static_cast<int>((P.M - m0 < kPairBT) ? P.M - m0 : kPairBT);
-    const float* bias_p = SZO_SUB(P, u.s, bias);
-    if constexpr (kPaired) {
-      if (m0 >= P.pair_row0) bias_p = nullptr;
+    int32_t* ticket = P.tickets + u.slot * 2 + rank;
+    int32_t* done = P.tickets_done + u.slot * 2 + rank;
+    if (threadIdx.x == 0) {
+      // all parts of the tile parked?  Their clusters are resident and running: a bounded wait
+      const long long t0 = clock64();
+      while (*reinterpret_cast<volatile int32_t*>(ticket) < u.parts) {
+        __nanosleep(64);
+        if (clock64() - t0 > kWaitLimitCycles) {
+          *abort_flag = 1;
+          atomicExch(P.status, static_cast<int32_t>(SZO_ERR_TIMEOUT));
+          break;
+        }
+      }
+      __threadfence();               // the other parts' tiles are read after this point (from L2, ld.cg)
     }
-    reduce_parts(P.partial + (static_cast<int64_t>(u.slot * u.parts) * 2 + rank) * kPartFloats, u.parts,
-                 static_cast<int64_t>(u.n_tile) * kBM, SZO_SUB(P, u.s, N), bias_p, SZO_SUB(P, u.s, y), P.y_f32,
-                 kRelu ? 1 : 0, m0, mlimit, static_cast<int>(threadIdx.x), kNumWarps2 * 32);
+    __syncthreads();
+    if (!*abort_flag) {
+      const int64_t m0 = static_cast<int64_t>(u.m_tile) * kPairBT;
+      const int mlimit = static_cast<int>((P.M - m0 < kPairBT) ? P.M - m0 : kPairBT);
+      const int t_begin = (kPairBT * u.part) / u.parts, t_end = (kPairBT * (u.part + 1)) / u.parts;
+      const float* bias_p = SZO_SUB(P, u.s, bias);
+      if constexpr (kPaired) {
+        if (m0 >= P.pair_row0) bias_p = nullptr;
+      }
+      if (t_begin < mlimit)
+        reduce_parts(P.partial + (static_cast<int64_t>(u.slot * u.parts) * 2 + rank) * kPartFloats, u.parts,
+                     static_cast<int64_t>(u.n_tile) * kBM, SZO_SUB(P, u.s, N), bias_p, SZO_SUB(P, u.s, y), P.y_f32,
+                     kRelu ? 1 : 0, m0, t_begin, t_end < mlimit ? t_end : mlimit, static_cast<int>(threadIdx.x),
+                     kNumWarps2 * 32);
+      __syncthreads();
+      if (threadIdx.x == 0 && atomicAdd(done, 1) == u.parts - 1) {      // the last share: ready for the next launch
+        *ticket = 0;
+        *done = 0;
+      }
+    }
   }
   cluster_sync_all();          // no CTA leaves while its peer may still signal it or read its tiles
   tc_fence_after();

@@ -51,12 +51,15 @@ struct TcParams {
   // Work units of pair p: full tiles p + lt * n_pairs for lt < full_rounds, then (p < tail_tiles *
   // tail_parts) one unit of the tail: tile full_rounds * n_pairs + p % tail_tiles, k-blocks
   // [tail_kb[part], tail_kb[part + 1]) with part = p / tail_tiles.  With tail_parts > 1 the parts of
-  // a tile meet in `partial` (fp32 [tail_tiles][tail_parts][2 ranks][256 tokens][128 rows]) and the
-  // last part to finish (tickets, self-resetting) adds them up in part order and stores y.
+  // a tile meet in `partial` (fp32 [tail_tiles][tail_parts][2 ranks][256 tokens][128 rows]); when all
+  // are parked (tickets; every cluster of the launch is resident, so the wait is for running code,
+  // and it is bounded) each part's CTA adds up, in part order, its share of the tile's tokens and
+  // stores y; the last one to finish resets the counters.
   int full_rounds, tail_tiles, tail_parts;
   int tail_kb[5];
   float* partial;
-  int32_t* tickets;        // [tail_tiles][2 ranks]
+  int32_t* tickets;        // [tail_tiles][2 ranks]: parts of the tile parked so far
+  int32_t* tickets_done;   // [tail_tiles][2 ranks]: parts that have finished their share of the sum
   // Paired form of the two forwards of a ZO step (dense mode only).  The token rows hold the centre
   // xc = (x+ + x-)/2 in rows [0, M_c) and the half-difference xd = (x+ - x-)/2 from row pair_row0 (a
   // multiple of 256) on.  With W = RN_bf16(Dequantize(Q) + S) unperturbed,
