@@ -32,8 +32,14 @@
 //     adds the eight partials of rows 16c .. 16c+15 in CTA order (deterministic), then the sparse
 //     term and the bias, and stores y.  Partials and sparse terms are double-buffered and everyone
 //     waits only for the barrier of the tile before, so nobody stands still for the sum.
+// One launch may serve up to three matrices that read the same activations (q/k/v, gate/up of a decoder
+// layer): their 128-row tiles are numbered one after the other, and a tile's number names its matrix.
+// The activations may be formed while they are staged: silu(x) * x_mul, rounded to bf16 (the
+// gated MLP's product, which then never goes through device memory).
 // Waits on mbarriers are bounded (status SZO_ERR_TIMEOUT); after a failed wait a thread keeps the
 // control flow, and with it the cluster barriers, but skips waiting and copying.
+#include <mutex>
+
 #include "tc_common.cuh"
 
 namespace szo {
@@ -122,6 +128,46 @@ __device__ __forceinline__ void tile_written_sync() { asm volatile("bar.sync 2, 
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 __device__ __forceinline__ void workers_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory"); }
 
+struct SkinnySub {
+  const uint8_t* codes_tiled;
+  const float2* sz;
+  int64_t Npad;
+  const int32_t* row_ptr;   // NULL: no sparse entries
+  const int32_t* ent_col;
+  const float* S;
+  const float* bias;
+  void* y;
+  int64_t N;
+  int tile_begin;           // number of this matrix's first tile
+};
+struct SkinnyArgs {
+  SkinnySub sub[3];
+  int n;
+  const __nv_bfloat16* x;
+  const __nv_bfloat16* x_mul;   // not NULL: the activations are silu(x) * x_mul
+  int M;
+  int64_t K;
+  int G, n_tiles, n_stages;
+  int32_t* status;
+};
+// silu(g) * u of eight bf16 pairs, each product rounded to bf16 (the arithmetic of the model's own
+// SiLU-gating kernel, so that either route gives the same bits)
+__device__ __forceinline__ uint4 silu_mul_bf16x8(uint4 g, uint4 u) {
+  const uint32_t gw[4] = {g.x, g.y, g.z, g.w}, uw[4] = {u.x, u.y, u.z, u.w};
+  uint32_t o[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float g0 = __uint_as_float(gw[i] << 16), g1 = __uint_as_float(gw[i] & 0xFFFF0000u);
+    const float u0 = __uint_as_float(uw[i] << 16), u1 = __uint_as_float(uw[i] & 0xFFFF0000u);
+    const __nv_bfloat162 r = __floats2bfloat162_rn(g0 / (1.0f + expf(-g0)) * u0, g1 / (1.0f + expf(-g1)) * u1);
+    o[i] = *reinterpret_cast<const uint32_t*>(&r);
+  }
+  return make_uint4(o[0], o[1], o[2], o[3]);
+}
+__device__ __forceinline__ int sub_of_tile(const SkinnyArgs& a, int tile) {
+  return (a.n > 1 && tile >= a.sub[1].tile_begin) + (a.n > 2 && tile >= a.sub[2].tile_begin);
+}
+
 // kNT: token tiles per CTA (1: up to 8 tokens, 2: up to 16).  kGroupMma: G is a multiple of 128.
 // Grid: kSplit * n_clusters CTAs, clusters of kSplit along x; cluster c takes tiles c, c + n_clusters, ...
 // Cluster barriers, the same sequence for every thread (no early exit): number 0 says that every
@@ -130,11 +176,12 @@ __device__ __forceinline__ void workers_sync() { asm volatile("bar.sync 1, %0;" 
 // only after it is done with what number k - 1 published (the buffers alternate).
 template <bool kBf16Tables, bool kGroupMma, typename TY, int kNT>
 __global__ void __cluster_dims__(kSplit, 1, 1) __launch_bounds__(kThreads, 2)
-szo_linear_skinny_kernel(const uint8_t* __restrict__ codes_tiled, const float2* __restrict__ sz, int64_t Npad,
-                         const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ row_ptr,
-                         const int32_t* __restrict__ ent_col, const float* __restrict__ S, const float* __restrict__ bias,
-                         TY* __restrict__ y, int M, int64_t N, int64_t K, int G, int n_tiles, int n_stages, int32_t* status) {
+szo_linear_skinny_kernel(const __grid_constant__ SkinnyArgs a) {
   constexpr int kT = kTok * kNT;                       // tokens per CTA
+  const int M = a.M, G = a.G, n_tiles = a.n_tiles, n_stages = a.n_stages;
+  const int64_t K = a.K;
+  int32_t* const status = a.status;
+  const __nv_bfloat16* __restrict__ x = a.x;
   extern __shared__ __align__(128) unsigned char smem_sk[];
   __shared__ float part[2][kRowsCta * kT];             // this CTA's K-part of a 128-row tile: [row][token]
   __shared__ float spart[2][kRowsWarp * kT];           // sparse term of the 16 rows this CTA sums: [row][token]
@@ -184,8 +231,11 @@ szo_linear_skinny_kernel(const uint8_t* __restrict__ codes_tiled, const float2* 
     auto issue_tile = [&](int tile) {
       if (lane == 0) {
         // (a lone thread runs a dependent instruction every few cycles: no 64-bit division in here)
-        const uint8_t* src = codes_tiled + (static_cast<int64_t>(tile) * nkb + 2 * s_begin) * 4096;
-        const float2* zsrc = sz + static_cast<int64_t>(tile) * kRowsCta;
+        const SkinnySub& sb = a.sub[sub_of_tile(a, tile)];
+        const int64_t Npad = sb.Npad;
+        const int ltile = tile - sb.tile_begin;
+        const uint8_t* src = sb.codes_tiled + (static_cast<int64_t>(ltile) * nkb + 2 * s_begin) * 4096;
+        const float2* zsrc = sb.sz + static_cast<int64_t>(ltile) * kRowsCta;
         for (int i = 0; i < my_steps; ++i) {
           if (!failed && !tc::mbar_wait(empty_bar(p.idx), p.phase ^ 1u, abort_flag, status)) failed = true;
           if (!failed) {
@@ -221,10 +271,13 @@ szo_linear_skinny_kernel(const uint8_t* __restrict__ codes_tiled, const float2* 
     const int64_t sp_row = rank * kRowsWarp + sp_r;                       // its lane's row inside a tile
     auto load_rp = [&](int tile, int32_t& rb, int32_t& re) {
       rb = re = 0;
-      if (row_ptr != nullptr && tile < n_tiles) {
-        const int64_t n = static_cast<int64_t>(tile) * kRowsCta + sp_row;
-        rb = row_ptr[(n < N) ? n : N];                                   // rows beyond N: empty
-        re = row_ptr[(n + 1 < N) ? n + 1 : N];
+      if (tile < n_tiles) {
+        const SkinnySub& sb = a.sub[sub_of_tile(a, tile)];
+        if (sb.row_ptr != nullptr) {
+          const int64_t n = static_cast<int64_t>(tile - sb.tile_begin) * kRowsCta + sp_row, N = sb.N;
+          rb = sb.row_ptr[(n < N) ? n : N];                              // rows beyond N: empty
+          re = sb.row_ptr[(n + 1 < N) ? n + 1 : N];
+        }
       }
     };
     int32_t b0 = 0, e0 = 0, b1 = 0, e1 = 0;
@@ -245,6 +298,13 @@ szo_linear_skinny_kernel(const uint8_t* __restrict__ codes_tiled, const float2* 
         for (int r = 0; r < kTok; ++r)
           v[r] = (8 * j + r < M) ? __ldg(reinterpret_cast<const uint4*>(xsrc + static_cast<int64_t>(8 * j + r) * K + c * 8))
                                  : make_uint4(0u, 0u, 0u, 0u);
+        if (a.x_mul != nullptr) {
+          const __nv_bfloat16* usrc = a.x_mul + static_cast<int64_t>(s_begin) * kStepK;
+#pragma unroll
+          for (int r = 0; r < kTok; ++r)
+            if (8 * j + r < M)
+              v[r] = silu_mul_bf16x8(v[r], __ldg(reinterpret_cast<const uint4*>(usrc + static_cast<int64_t>(8 * j + r) * K + c * 8)));
+        }
 #pragma unroll
         for (int r = 0; r < kTok; ++r) *reinterpret_cast<uint4*>(sx + (8 * j + r) * ld + chunk_pos(c) * 8) = v[r];
 #pragma unroll
@@ -296,29 +356,31 @@ szo_linear_skinny_kernel(const uint8_t* __restrict__ codes_tiled, const float2* 
       // tile it is summed.
       constexpr int kGatherQ = kSpChunk / 32 / kNT;                      // entries per lane whose activations are fetched at once
       const int r = sp_r, h = lane & 1;
-      auto load_entries = [&](int32_t base, int32_t end, int (&col)[kSpChunk / 32], float (&val)[kSpChunk / 32]) {
+      // entries [base, end) of the matrix that tile `tile` belongs to (an empty range for a tile past the last)
+      auto load_entries = [&](int tile, int32_t base, int32_t end, int (&col)[kSpChunk / 32], float (&val)[kSpChunk / 32]) {
+        const SkinnySub& sb = a.sub[tile < n_tiles ? sub_of_tile(a, tile) : 0];
 #pragma unroll
         for (int q = 0; q < kSpChunk / 32; ++q) {
           const int32_t e = base + lane + 32 * q;
-          col[q] = (e < end) ? ent_col[e] : -1;
-          val[q] = (e < end) ? S[e] : 0.f;
+          col[q] = (e < end) ? sb.ent_col[e] : -1;
+          val[q] = (e < end) ? sb.S[e] : 0.f;
         }
       };
       int32_t b2, e2;                                                    // row pointers of tile it + 2
       int col0[kSpChunk / 32], col1[kSpChunk / 32];
       float val0[kSpChunk / 32], val1[kSpChunk / 32];
-      load_entries(__shfl_sync(0xffffffffu, b0, 0), __shfl_sync(0xffffffffu, e0, 31), col0, val0);
+      load_entries(cid, __shfl_sync(0xffffffffu, b0, 0), __shfl_sync(0xffffffffu, e0, 31), col0, val0);
       int it = 0;
       for (int tile = cid; tile < n_tiles; tile += n_clusters, ++it) {
         load_rp(tile + 2 * n_clusters, b2, e2);
-        load_entries(__shfl_sync(0xffffffffu, b1, 0), __shfl_sync(0xffffffffu, e1, 31), col1, val1);
+        load_entries(tile + n_clusters, __shfl_sync(0xffffffffu, b1, 0), __shfl_sync(0xffffffffu, e1, 31), col1, val1);
         const int32_t tile_b = __shfl_sync(0xffffffffu, b0, 0), tile_e = __shfl_sync(0xffffffffu, e0, 31);
         if (it == 0) cluster_wait();         // number 0: the peers' activations are staged
         float sp[kT / 2];
 #pragma unroll
         for (int j = 0; j < kT / 2; ++j) sp[j] = 0.f;
         for (int32_t base = tile_b; base < tile_e; base += kSpChunk) {
-          if (base > tile_b) load_entries(base, tile_e, col0, val0);     // rows with more entries than one chunk
+          if (base > tile_b) load_entries(tile, base, tile_e, col0, val0);     // rows with more entries than one chunk
           // (all loads of a pass first, then the stores: a store to shared memory between two loads
           // from the cluster's shared memory would keep the second load waiting for the first)
 #pragma unroll
@@ -384,8 +446,11 @@ szo_linear_skinny_kernel(const uint8_t* __restrict__ codes_tiled, const float2* 
         tile_written_sync();                 // this CTA's part and sparse term of the tile are written
         cluster_arrive_release();            // number it + 1 (and: the tile before is summed and stored)
         cluster_wait();
-        const int64_t n = static_cast<int64_t>(tile) * kRowsCta + rank * kRowsWarp + r;
-        const float bv = (bias != nullptr && n < N) ? bias[n] : 0.f;
+        const SkinnySub& sb = a.sub[sub_of_tile(a, tile)];
+        const int64_t N = sb.N;
+        const int64_t n = static_cast<int64_t>(tile - sb.tile_begin) * kRowsCta + rank * kRowsWarp + r;
+        const float bv = (sb.bias != nullptr && n < N) ? sb.bias[n] : 0.f;
+        TY* __restrict__ y = static_cast<TY*>(sb.y);
         float v[kT / 2];
 #pragma unroll
         for (int j0 = 0; j0 < kT / 2; j0 += 4) {                       // four tokens at a time
@@ -524,8 +589,10 @@ size_t skinny_dyn_smem(int64_t K, int G, int kT, int n_stages = kStages) {
 }
 
 template <bool kBf16Tables, bool kGroupMma, typename TY, int kNT>
-szo_status launch_skinny(const szo_linear* p, const void* x, int64_t M, const float* S, void* y, cudaStream_t st) {
+szo_status launch_skinny(const szo_linear* const* plans, int n, const void* x, const void* x_mul, int64_t M,
+                         const float* const* S, void* const* y, cudaStream_t st) {
   auto kern = szo_linear_skinny_kernel<kBf16Tables, kGroupMma, TY, kNT>;
+  const szo_linear* p = plans[0];
   // A ring of 8 steps when two CTAs of that size still share an SM (or when 4 would not change that
   // either), else 4: two CTAs with 4 steps in flight each hide more than one with 8.
   constexpr size_t kStaticSmem = (kNT == 1) ? 14 * 1024 : 28 * 1024;            // upper bounds of the kernel's static arrays
@@ -535,44 +602,71 @@ szo_status launch_skinny(const szo_linear* p, const void* x, int64_t M, const fl
       skinny_dyn_smem(p->K, p->G, kTok * kNT, kStages / 2) + kStaticSmem <= kTwoPerSm)
     n_stages = kStages / 2;
   const size_t smem = skinny_dyn_smem(p->K, p->G, kTok * kNT, n_stages);
-  static bool configured = false;
-  if (!configured) {
-    SZO_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynSmem)));
-    configured = true;
+  // per device: the attribute, and how many clusters fit at once with this much shared memory
+  struct PerDevice {
+    bool configured = false;
+    size_t asked_smem = ~static_cast<size_t>(0);
+    int max_clusters = 0;
+  };
+  static PerDevice per_device[64];
+  static std::mutex mu;
+  int dev = 0;
+  SZO_CHECK_CUDA(cudaGetDevice(&dev));
+  SZO_REQUIRE(dev >= 0 && dev < 64, SZO_ERR_UNSUPPORTED, "device ordinal %d", dev);
+  int max_clusters = 0;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    PerDevice& pd = per_device[dev];
+    if (!pd.configured) {
+      SZO_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynSmem)));
+      pd.configured = true;
+    }
+    if (smem != pd.asked_smem) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(static_cast<unsigned>(kSplit * 64));
+      cfg.blockDim = dim3(kThreads);
+      cfg.dynamicSmemBytes = smem;
+      SZO_CHECK_CUDA(cudaOccupancyMaxActiveClusters(&pd.max_clusters, kern, &cfg));
+      if (pd.max_clusters < 1) pd.max_clusters = 1;
+      pd.asked_smem = smem;
+    }
+    max_clusters = pd.max_clusters;
   }
-  int32_t* status = device_status_word();
-  SZO_REQUIRE(status != nullptr, SZO_ERR_CUDA, "no device status word");
-  const int n_tiles = static_cast<int>(ceil_div(p->N, kRowsCta));
-  // as many clusters as fit at once with this much shared memory (asked from the driver), no more than tiles
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(static_cast<unsigned>(kSplit * n_tiles));
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = smem;
-  static size_t asked_smem = ~static_cast<size_t>(0);
-  static int max_clusters = 0;
-  if (smem != asked_smem) {
-    SZO_CHECK_CUDA(cudaOccupancyMaxActiveClusters(&max_clusters, kern, &cfg));
-    if (max_clusters < 1) max_clusters = 1;
-    asked_smem = smem;
+  SkinnyArgs a{};
+  a.n = n;
+  a.x = static_cast<const __nv_bfloat16*>(x);
+  a.x_mul = static_cast<const __nv_bfloat16*>(x_mul);
+  a.M = static_cast<int>(M);
+  a.K = p->K;
+  a.G = p->G;
+  a.n_stages = n_stages;
+  a.status = device_status_word();
+  SZO_REQUIRE(a.status != nullptr, SZO_ERR_CUDA, "no device status word");
+  int n_tiles = 0;
+  for (int i = 0; i < n; ++i) {
+    const szo_linear* q = plans[i];
+    a.sub[i] = SkinnySub{q->codes_tiled, q->sz, q->Npad, q->nnz > 0 ? q->row_ptr : nullptr, q->ent_col, S[i], q->bias, y[i],
+                         q->N, n_tiles};
+    n_tiles += static_cast<int>(ceil_div(q->N, kRowsCta));
   }
+  a.n_tiles = n_tiles;
   const int n_clusters = n_tiles < max_clusters ? n_tiles : max_clusters;
-  kern<<<static_cast<unsigned>(kSplit * n_clusters), kThreads, smem, st>>>(
-      p->codes_tiled, p->sz, p->Npad, static_cast<const __nv_bfloat16*>(x), p->nnz > 0 ? p->row_ptr : nullptr, p->ent_col,
-      S, p->bias, static_cast<TY*>(y), static_cast<int>(M), p->N, p->K, p->G, n_tiles, n_stages, status);
+  kern<<<static_cast<unsigned>(kSplit * n_clusters), kThreads, smem, st>>>(a);
   count_launch();
   SZO_CHECK_LAUNCH("szo_linear_skinny_kernel");
   return SZO_OK;
 }
 
 template <bool kBf16Tables, typename TY>
-szo_status launch_skinny_nt(const szo_linear* p, const void* x, int64_t M, const float* S, void* y, cudaStream_t st) {
-  const bool group = p->G % kStepK == 0;
+szo_status launch_skinny_nt(const szo_linear* const* plans, int n, const void* x, const void* x_mul, int64_t M,
+                            const float* const* S, void* const* y, cudaStream_t st) {
+  const bool group = plans[0]->G % kStepK == 0;
   if (M <= kTok) {
-    if (group) return launch_skinny<kBf16Tables, true, TY, 1>(p, x, M, S, y, st);
-    return launch_skinny<kBf16Tables, false, TY, 1>(p, x, M, S, y, st);
+    if (group) return launch_skinny<kBf16Tables, true, TY, 1>(plans, n, x, x_mul, M, S, y, st);
+    return launch_skinny<kBf16Tables, false, TY, 1>(plans, n, x, x_mul, M, S, y, st);
   }
-  if (group) return launch_skinny<kBf16Tables, true, TY, 2>(p, x, M, S, y, st);
-  return launch_skinny<kBf16Tables, false, TY, 2>(p, x, M, S, y, st);
+  if (group) return launch_skinny<kBf16Tables, true, TY, 2>(plans, n, x, x_mul, M, S, y, st);
+  return launch_skinny<kBf16Tables, false, TY, 2>(plans, n, x, x_mul, M, S, y, st);
 }
 
 }  // namespace
@@ -585,16 +679,31 @@ bool skinny_applies(const szo_linear* p, int64_t M) {
          p->K % kStepK == 0 && skinny_dyn_smem(p->K, p->G, M <= kTok ? kTok : 2 * kTok) <= kMaxDynSmem;
 }
 
+// Up to three matrices with the same K, group size and table type in one launch
+bool skinny_group_applies(const szo_linear* const* plans, int n, int64_t M) {
+  if (n < 1 || n > 3) return false;
+  for (int i = 0; i < n; ++i)
+    if (!skinny_applies(plans[i], M) || plans[i]->K != plans[0]->K || plans[i]->G != plans[0]->G ||
+        plans[i]->sz_dtype != plans[0]->sz_dtype)
+      return false;
+  return true;
+}
+
+szo_status linear_fwd_skinny_group(const szo_linear* const* plans, int n, const void* x, const void* x_mul, int64_t M,
+                                   const float* const* S_pert, void* const* y, int y_dtype, cudaStream_t st) {
+  SZO_REQUIRE(skinny_group_applies(plans, n, M), SZO_ERR_UNSUPPORTED, "shapes not covered by the weight-streaming kernel");
+  const bool bf = plans[0]->sz_dtype == SZO_BF16;
+  if (y_dtype == SZO_F32) {
+    if (bf) return launch_skinny_nt<true, float>(plans, n, x, x_mul, M, S_pert, y, st);
+    return launch_skinny_nt<false, float>(plans, n, x, x_mul, M, S_pert, y, st);
+  }
+  if (bf) return launch_skinny_nt<true, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st);
+  return launch_skinny_nt<false, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st);
+}
+
 szo_status linear_fwd_skinny(const szo_linear* p, const void* x, int64_t M, const float* S_pert, void* y, int y_dtype,
                              cudaStream_t st) {
-  SZO_REQUIRE(skinny_applies(p, M), SZO_ERR_UNSUPPORTED, "shape not covered by the weight-streaming kernel");
-  const bool bf = p->sz_dtype == SZO_BF16;
-  if (y_dtype == SZO_F32) {
-    if (bf) return launch_skinny_nt<true, float>(p, x, M, S_pert, y, st);
-    return launch_skinny_nt<false, float>(p, x, M, S_pert, y, st);
-  }
-  if (bf) return launch_skinny_nt<true, __nv_bfloat16>(p, x, M, S_pert, y, st);
-  return launch_skinny_nt<false, __nv_bfloat16>(p, x, M, S_pert, y, st);
+  return linear_fwd_skinny_group(&p, 1, x, nullptr, M, &S_pert, &y, y_dtype, st);
 }
 
 }  // namespace szo

@@ -439,6 +439,115 @@ attn_decode_kernel(const T* __restrict__ q, const T* __restrict__ kc, const T* _
   }
 }
 
+// The same attention with the two kernels before it folded in, for a handful of new tokens (a token
+// step is a chain of short dependent launches: two fewer per layer).  q and k_new arrive unrotated.
+// Block (t, hq, b) rotates its query at position pos0 + t, reads the keys and values of the new
+// tokens 0 .. t from k_new / v_new (rotating each key at its position) and the older ones from the
+// cache; the first query head of every key/value head also stores the rotated key and the value of
+// token t in the cache.  No block reads a cache row that this launch writes.  Rotated values are
+// rounded to T exactly where rope_kernel and the cache would round them: same bits as the three
+// separate kernels.
+template <typename T, int HD>
+__global__ void __launch_bounds__(128)
+attn_decode_fused_kernel(const T* __restrict__ q, const T* __restrict__ k_new, const T* __restrict__ v_new,
+                         T* __restrict__ kc, T* __restrict__ vc, T* __restrict__ o, const float2* __restrict__ rope_tab,
+                         int Tn, const int32_t* __restrict__ pos_dev, int64_t Smax, int H, int Hkv, float scale) {
+  constexpr int E = HD / 32, half = HD / 2;
+  __shared__ float part_acc[4][HD];
+  __shared__ float part_m[4], part_l[4];
+  const int pos0 = *pos_dev;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int t = blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
+  const int hk = hq / (H / Hkv);
+  const int64_t dq = static_cast<int64_t>(H) * HD, dk = static_cast<int64_t>(Hkv) * HD;
+  // element lane + 32 j pairs with lane + 32 (j + E/2): both in this lane
+  auto rotate = [&](float (&x)[E], int pos) {
+    if (rope_tab == nullptr) return;
+#pragma unroll
+    for (int j = 0; j < E / 2; ++j) {
+      const float2 cs = rope_tab[static_cast<int64_t>(pos) * half + lane + 32 * j];
+      const float a0 = x[j], b0 = x[j + E / 2];
+      x[j] = to_f32<T>(from_f32<T>(a0 * cs.x - b0 * cs.y));
+      x[j + E / 2] = to_f32<T>(from_f32<T>(b0 * cs.x + a0 * cs.y));
+    }
+  };
+  const T* qp = q + (static_cast<int64_t>(b) * Tn + t) * dq + hq * HD;
+  float qr[E], acc[E];
+#pragma unroll
+  for (int j = 0; j < E; ++j) qr[j] = to_f32<T>(qp[lane + 32 * j]);
+  rotate(qr, pos0 + t);
+#pragma unroll
+  for (int j = 0; j < E; ++j) {
+    qr[j] *= scale;
+    acc[j] = 0.f;
+  }
+  const T* knb = k_new + static_cast<int64_t>(b) * Tn * dk + hk * HD;
+  const T* vnb = v_new + static_cast<int64_t>(b) * Tn * dk + hk * HD;
+  T* kb = kc + static_cast<int64_t>(b) * Smax * dk + hk * HD;
+  T* vb = vc + static_cast<int64_t>(b) * Smax * dk + hk * HD;
+  if (w == 3 && hq % (H / Hkv) == 0) {          // (the warp with the fewest keys when few are cached)
+    float kv[E];
+#pragma unroll
+    for (int j = 0; j < E; ++j) kv[j] = to_f32<T>(knb[t * dk + lane + 32 * j]);
+    rotate(kv, pos0 + t);
+#pragma unroll
+    for (int j = 0; j < E; ++j) {
+      kb[(pos0 + t) * dk + lane + 32 * j] = from_f32<T>(kv[j]);
+      vb[(pos0 + t) * dk + lane + 32 * j] = vnb[t * dk + lane + 32 * j];
+    }
+  }
+  float mx = -INFINITY, l = 0.f;
+  for (int n = w; n <= pos0 + t; n += 4) {
+    const bool fresh = n >= pos0;
+    const T* kp = fresh ? knb + (n - pos0) * dk : kb + n * dk;
+    const T* vp = fresh ? vnb + (n - pos0) * dk : vb + n * dk;
+    float kv[E], vv[E];
+#pragma unroll
+    for (int j = 0; j < E; ++j) {
+      kv[j] = to_f32<T>(kp[lane + 32 * j]);
+      vv[j] = to_f32<T>(vp[lane + 32 * j]);
+    }
+    if (fresh) rotate(kv, n);
+    float dot = 0.f;
+#pragma unroll
+    for (int j = 0; j < E; ++j) dot = fmaf(qr[j], kv[j], dot);
+#pragma unroll
+    for (int off = 16; off; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+    const float mn = fmaxf(mx, dot);
+    const float corr = expf(mx - mn), p = expf(dot - mn);
+    l = l * corr + p;
+#pragma unroll
+    for (int j = 0; j < E; ++j) acc[j] = fmaf(p, vv[j], acc[j] * corr);
+    mx = mn;
+  }
+#pragma unroll
+  for (int j = 0; j < E; ++j) part_acc[w][lane + 32 * j] = acc[j];
+  if (lane == 0) {
+    part_m[w] = mx;
+    part_l[w] = l;
+  }
+  __syncthreads();
+  if (w == 0) {
+    float M = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) M = fmaxf(M, part_m[i]);
+    float L = 0.f, out[E];
+#pragma unroll
+    for (int j = 0; j < E; ++j) out[j] = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float f = part_m[i] == -INFINITY ? 0.f : expf(part_m[i] - M);
+      L += part_l[i] * f;
+#pragma unroll
+      for (int j = 0; j < E; ++j) out[j] = fmaf(part_acc[i][lane + 32 * j], f, out[j]);
+    }
+    T* op = o + (static_cast<int64_t>(b) * Tn + t) * dq + hq * HD;
+    const float inv = 1.0f / L;
+#pragma unroll
+    for (int j = 0; j < E; ++j) op[lane + 32 * j] = from_f32<T>(out[j] * inv);
+  }
+}
+
 // ------------------------------------------------------------------------------ paired form
 // The two forwards of a ZO step (Definition 1: the loss at w + eps zbar and at w - eps zbar, same
 // batch) carried through the network as centre c = (x+ + x-)/2 and half-difference d = (x+ - x-)/2
@@ -1157,6 +1266,21 @@ szo_status run_decode_t(szo_model* m, const int32_t* tokens, int B, int Tn, cons
     const int t = layer * m->n_lin + j;
     return linear_fwd_impl(m->plans[t], x, act, M, Sv + m->offsets[t], nullptr, out, act, lmode, m->ws, m->ws_bytes, st);
   };
+  // n matrices that read the same activations: one launch of the weight-streaming kernel where it
+  // takes the group, else one call each
+  const bool streaming = lmode == SZO_MODE_AUTO && act == SZO_BF16;
+  auto lin_group = [&](int layer, int j0, int n, const void* x, void* const* outs) -> szo_status {
+    const int t0 = layer * m->n_lin + j0;
+    const szo_linear* plans[3];
+    const float* sv[3];
+    for (int i = 0; i < n; ++i) {
+      plans[i] = m->plans[t0 + i];
+      sv[i] = Sv + m->offsets[t0 + i];
+    }
+    if (streaming && skinny_group_applies(plans, n, M)) return linear_fwd_skinny_group(plans, n, x, nullptr, M, sv, outs, act, st);
+    for (int i = 0; i < n; ++i) SZO_TRY(lin(layer, j0 + i, x, outs[i]));
+    return SZO_OK;
+  };
   embed_kernel<<<static_cast<unsigned>(M), 128, 0, st>>>(tokens, static_cast<const __nv_bfloat16*>(m->top.embed),
                                                         static_cast<const __nv_bfloat16*>(m->top.pos), Tn, d, c.vocab, m->h, 0, pos_dev);
   count_launch();
@@ -1167,32 +1291,49 @@ szo_status run_decode_t(szo_model* m, const int32_t* tokens, int B, int Tn, cons
     add_norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, pending, L.attn_norm_g, L.attn_norm_b, d, c.norm_eps,
                                                                 opt, 1, 0, a);
     count_launch();
-    SZO_TRY(lin(l, 0, a, q));
-    SZO_TRY(lin(l, 1, a, k));
-    SZO_TRY(lin(l, 2, a, v));
-    if (!opt) {
-      const int64_t n_vec = M * (H + Hkv) * ((hd / 2) / Vec16<T>::kN);
-      rope_kernel<T><<<blocks_for(n_vec, 256), 256, 0, st>>>(q, k, m->rope_tab, M, Tn, H, Hkv, hd, 0, pos_dev);
-      count_launch();
+    {
+      void* const qkv[3] = {q, k, v};
+      SZO_TRY(lin_group(l, 0, 3, a, qkv));
     }
     T* kc = static_cast<T*>(m->kcache) + l * layer_cache;
     T* vc = static_cast<T*>(m->vcache) + l * layer_cache;
-    const int64_t n_vec = M * dkv / Vec16<T>::kN;
-    kv_append_kernel<T><<<blocks_for(2 * n_vec, 256), 256, 0, st>>>(k, v, kc, vc, Tn, pos_dev, Smax, dkv, n_vec);
     dim3 grid(static_cast<unsigned>(Tn), H, B);
     const float scale = 1.0f / sqrtf(static_cast<float>(hd));
-    if (hd == 64) attn_decode_kernel<T, 64><<<grid, 128, 0, st>>>(q, kc, vc, o, Tn, pos_dev, Smax, H, Hkv, scale);
-    else attn_decode_kernel<T, 128><<<grid, 128, 0, st>>>(q, kc, vc, o, Tn, pos_dev, Smax, H, Hkv, scale);
-    count_launch(2);
+    if (Tn <= 16) {
+      // rotation, cache append and attention in one launch
+      const float2* tab = opt ? nullptr : m->rope_tab;
+      if (hd == 64) attn_decode_fused_kernel<T, 64><<<grid, 128, 0, st>>>(q, k, v, kc, vc, o, tab, Tn, pos_dev, Smax, H, Hkv, scale);
+      else attn_decode_fused_kernel<T, 128><<<grid, 128, 0, st>>>(q, k, v, kc, vc, o, tab, Tn, pos_dev, Smax, H, Hkv, scale);
+      count_launch();
+    } else {
+      if (!opt) {
+        const int64_t n_rot = M * (H + Hkv) * ((hd / 2) / Vec16<T>::kN);
+        rope_kernel<T><<<blocks_for(n_rot, 256), 256, 0, st>>>(q, k, m->rope_tab, M, Tn, H, Hkv, hd, 0, pos_dev);
+        count_launch();
+      }
+      const int64_t n_vec = M * dkv / Vec16<T>::kN;
+      kv_append_kernel<T><<<blocks_for(2 * n_vec, 256), 256, 0, st>>>(k, v, kc, vc, Tn, pos_dev, Smax, dkv, n_vec);
+      if (hd == 64) attn_decode_kernel<T, 64><<<grid, 128, 0, st>>>(q, kc, vc, o, Tn, pos_dev, Smax, H, Hkv, scale);
+      else attn_decode_kernel<T, 128><<<grid, 128, 0, st>>>(q, kc, vc, o, Tn, pos_dev, Smax, H, Hkv, scale);
+      count_launch(2);
+    }
     SZO_TRY(lin(l, 3, o, y));
     add_norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, y, L.mlp_norm_g, L.mlp_norm_b, d, c.norm_eps, opt, 1, 0, a);
     count_launch();
     if (!opt) {
-      SZO_TRY(lin(l, 4, a, gate));
-      SZO_TRY(lin(l, 5, a, up));
-      silu_mul_kernel<T><<<blocks_for(M * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, up, M * ff, gate);
-      count_launch();
-      SZO_TRY(lin(l, 6, gate, y));
+      void* const gu[2] = {gate, up};
+      SZO_TRY(lin_group(l, 4, 2, a, gu));
+      const szo_linear* down = m->plans[l * m->n_lin + 6];
+      if (streaming && skinny_group_applies(&down, 1, M)) {
+        // silu(gate) * up is formed while the down projection stages its activations
+        const float* sv = Sv + m->offsets[l * m->n_lin + 6];
+        void* const out[1] = {y};
+        SZO_TRY(linear_fwd_skinny_group(&down, 1, gate, up, M, &sv, out, act, st));
+      } else {
+        silu_mul_kernel<T><<<blocks_for(M * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, up, M * ff, gate);
+        count_launch();
+        SZO_TRY(lin(l, 6, gate, y));
+      }
     } else {
       SZO_TRY(lin(l, 4, a, gate));
       relu_kernel<T><<<blocks_for(M * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, M * ff);

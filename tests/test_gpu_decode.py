@@ -26,7 +26,7 @@ def test_decode_steps_match_the_oracle(B, name, act):
     fx = DecoderFixture(name, seed=6, mask="random", B=3, S=32)
     om = fx.oracle_model()
     S_np = om.S + np.float32(1e-3)                              # any values: the sparse term must be live
-    toks = fx.batch(0)[:, :12]
+    toks = fx.batch(0)[:, :24]
     lin_W = om.lin_W(S_np)
     cache = mo.KVCache(om.cfg.n_layers)
     a, md = (B.SZO_F32, B.MODE_FP32_VALIDATE) if act == "f32" else (B.SZO_BF16, B.MODE_SPARSE_ADD)
@@ -49,6 +49,16 @@ def test_decode_steps_match_the_oracle(B, name, act):
     ref = mo.decode_step(om.cfg, om.params, lin_W, toks[:, 4:8], cache2).numpy()
     got = m.decode_step(torch.from_numpy(np.ascontiguousarray(toks[:, 4:8])).cuda(), 0).cpu().numpy()
     assert np.max(np.abs(got - ref)) <= tol * np.max(np.abs(ref))
+    # a prompt of more than 16 tokens (rotation, cache append and attention as separate launches), then
+    # one token on top of it (the fused launch reading that cache)
+    cache3 = mo.KVCache(om.cfg.n_layers)
+    at = 0
+    for T in (20, 1):
+        ref = mo.decode_step(om.cfg, om.params, lin_W, toks[:, at:at + T], cache3).numpy()
+        got = m.decode_step(torch.from_numpy(np.ascontiguousarray(toks[:, at:at + T])).cuda(), at).cpu().numpy()
+        at += T
+        assert np.max(np.abs(got - ref)) <= tol * np.max(np.abs(ref)), (name, act, "long prompt", T)
+    assert B.device_status() == 0
     m.close()
 
 
