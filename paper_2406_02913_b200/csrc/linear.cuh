@@ -43,6 +43,11 @@ szo_status linear_spmm(const szo_linear* p, const void* x, int64_t M, const floa
 // Weight-streaming kernel for at most 16 tokens (gemm_skinny.cu): int4 plans, K a multiple of 128;
 // the sparse term is added in fp32 from the CSR rows (SparseAddMM).  Needs no workspace.
 bool skinny_applies(const szo_linear* p, int64_t M);
+// One to four tokens (gemm_gemv.cu): a CTA per 16 weight rows, no K-split between CTAs; same
+// arguments as linear_fwd_skinny_group, which hands such calls over.
+bool gemv_applies(const szo_linear* const* plans, int n, int64_t M);
+szo_status linear_fwd_gemv(const szo_linear* const* plans, int n, const void* x, const void* x_mul, int64_t M,
+                           const float* const* S_pert, void* const* y, int y_dtype, cudaStream_t st);
 // Up to three matrices that read the same activations in one launch (same K, G and table type);
 // x_mul != NULL: the activations are silu(x) * x_mul rounded to bf16, formed while they are staged.
 bool skinny_group_applies(const szo_linear* const* plans, int n, int64_t M);

@@ -372,6 +372,35 @@ def test_one_full_width_layer_against_the_oracle(B):
             m.close()
 
 
+def test_token_steps_of_one_full_width_layer_against_the_oracle(B):
+    """Token generation on one decoder layer at the Llama-2-7B width (the few-token kernels at the
+    widths they are built for: q/k/v and gate/up in one launch each, SiLU gating formed inside the
+    down projection, rotation + cache append + attention in one kernel): a prompt of 3 tokens, then
+    single tokens, for 2 sequences and for 1, against the oracle's incremental decode."""
+    from oracle import model_oracle as mo
+    from tests.fixtures import DecoderFixture
+    fx = DecoderFixture("llama2_7b", seed=9, mask="random", B=2, S=16, n_layers=1)
+    om = fx.oracle_model()
+    S_np = om.S + np.float32(1e-3)
+    lin_W = om.lin_W(S_np)
+    toks = fx.batch(0)[:, :8]
+    t = fx.gpu_tensors(torch, None)
+    S = torch.from_numpy(S_np.copy()).cuda()
+    m = B.Model(fx.shape, fx.names, t, S, act_dtype=B.SZO_BF16, linear_mode=B.MODE_SPARSE_ADD, max_batch=fx.B, max_seq=fx.S)
+    m.enable_decode()
+    for nseq in (2, 1):
+        cache = mo.KVCache(om.cfg.n_layers)
+        at = 0
+        for T in (3, 1, 1, 2):
+            tk = np.ascontiguousarray(toks[:nseq, at:at + T])
+            ref = mo.decode_step(om.cfg, om.params, lin_W, tk, cache).numpy()
+            got = m.decode_step(torch.from_numpy(tk).cuda(), at).cpu().numpy()
+            at += T
+            assert np.max(np.abs(got - ref)) <= 2e-2 * np.max(np.abs(ref)), (nseq, at)
+    assert B.device_status() == 0
+    m.close()
+
+
 def test_two_full_width_layers_paired_form_in_the_bench_configuration(B):
     """The step bench.py times (paired form, 16 x 256 tokens, 2-candidate loss) on two full-width layers:
     the fp64 oracle cannot run this size, so the projected gradient of the bf16 tensor-core path is held

@@ -113,6 +113,12 @@ SKINNY_CASES = [
     (128, 128, 128, "bf16", 3, 5e-2, True),         # one K step: seven CTAs of the cluster idle; dense mask
     (512, 1024, 256, "f16", 7, 1e-3, False),        # a quantization group spans two steps
     (640, 2048, 64, "bf16", 16, 3e-2, True),        # small groups; more sparse entries per 16 rows than one chunk
+    # at most four tokens, groups of a multiple of 128, at least eight K steps: the kernel with one CTA per 16 rows
+    (200, 1024, 128, "bf16", 1, 5e-3, True),        # N not a multiple of 16; one step per warp
+    (512, 4096, 128, "bf16", 1, 1e-3, False),       # four steps per warp: the ring exactly full
+    (304, 11008, 128, "f16", 4, 2e-3, True),        # 86 steps: 10 or 11 per warp, slots refilled; four tokens
+    (256, 2048, 256, "f16", 3, 3e-2, False),        # a group spans two steps; 61 entries per row: several rounds of the sparse warp
+    (1024, 4096, 128, "bf16", 2, 1e-3, True),
 ]
 
 
