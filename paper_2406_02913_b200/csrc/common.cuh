@@ -53,6 +53,34 @@ inline size_t round_up(size_t a, size_t b) { return (a + b - 1) / b * b; }
     if (s__ != SZO_OK) return s__;       \
   } while (0)
 
+// Chained launches (programmatic dependent launch).  A token step is a chain of short kernels, each
+// reading what the one before wrote; launched `chained`, a kernel may be placed on the SMs while its
+// predecessor drains and do there whatever does not depend on it (the weight-streaming kernels start
+// reading their weights).  Rules for a kernel that may be launched this way: chain_release() first
+// (lets ITS successor be placed early), chain_wait() before the first access to anything an earlier
+// kernel of the stream wrote or still reads.  chain_wait returns only when the predecessor grid has
+// completed and its writes are visible, so the kernels of a chain still run their dependent parts in
+// order.  Both are no-ops in a kernel launched the ordinary way.
+#ifdef __CUDACC__
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_maybe_chained(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                        bool chained, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = chained ? attr : nullptr;
+  cfg.numAttrs = chained ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // Launch counter used by the model to report how many kernels one step enqueued.
 extern thread_local int64_t g_launch_count;
 inline void count_launch(int n = 1) { g_launch_count += n; }

@@ -68,6 +68,14 @@ struct GemvArgs {
 // lanes' chunks of a turn are side by side.
 __device__ __forceinline__ int gv_chunk_pos(int c) { return (c & ~15) | ((c & 3) << 2) | ((c >> 2) & 3); }
 
+// D = A B
+__device__ __forceinline__ void gv_mma_new(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
+}
+// D = A B + D
 __device__ __forceinline__ void gv_mma_acc(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -133,6 +141,7 @@ __global__ void __launch_bounds__(kGvThreads, 2) szo_linear_gemv_kernel(const __
     return a.sub[(a.n > 1 && grp >= a.sub[1].cta_begin) + (a.n > 2 && grp >= a.sub[2].cta_begin)];
   };
 
+  chain_release();
   // ---------------------------------------------------------------- weight warps: start the stream
   const int s_begin = warp < kGvWarps ? warp * n_steps / kGvWarps : 0;
   const int n_my = warp < kGvWarps ? (warp + 1) * n_steps / kGvWarps - s_begin : 0;
@@ -207,6 +216,7 @@ __global__ void __launch_bounds__(kGvThreads, 2) szo_linear_gemv_kernel(const __
     }
   };
   // ---------------------------------------------------------------- everybody: stage the activations, once
+  chain_wait();          // the weights above are nobody's output; the activations are the predecessor's
   {
     // (all loads of a batch first: a chunk is one round trip to L2, and there are one to five batches)
     const int chunks = static_cast<int>(K / 8), total_chunks = chunks * M;
@@ -258,7 +268,8 @@ __global__ void __launch_bounds__(kGvThreads, 2) szo_linear_gemv_kernel(const __
     // q % kGvDepth (the loop is unrolled over the slots, a row group may end in any of them).
     int it = 0, cj = 0, grp = static_cast<int>(blockIdx.x);
     float tot[4] = {0.f, 0.f, 0.f, 0.f};
-    const __nv_bfloat16* xs0 = sx + static_cast<size_t>(g) * ld + s_begin * kGvStepK + t * 8;   // token g (if there is one)
+    // token g of the MMA's eight; where there is none, token 0 again: those columns of the result are never read
+    const __nv_bfloat16* xs0 = sx + static_cast<size_t>(g < M ? g : 0) * ld + s_begin * kGvStepK + t * 8;
     const float* xsum0 = xsum + s_begin * 8 + 2 * t;                                              // tokens 2t, 2t+1
     while (grp < total) {
 #pragma unroll
@@ -268,7 +279,7 @@ __global__ void __launch_bounds__(kGvThreads, 2) szo_linear_gemv_kernel(const __
           const float2 pa = rpa[d], pb = rpb[d];
           const uint32_t qa[4] = {wa.x, wa.y, wa.z, wa.w}, qb[4] = {wb.x, wb.y, wb.z, wb.w};
           const __nv_bfloat16* xs = xs0 + cj * kGvStepK;
-          float accq[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};   // even and odd words: two shorter chains
+          float accq[2][4];                                 // even and odd words: two shorter chains
 #pragma unroll
           for (int wd = 0; wd < 4; ++wd) {                  // one 32-bit word = 8 columns = two k16 MMAs
             uint32_t a0[4], a1[4];
@@ -280,9 +291,9 @@ __global__ void __launch_bounds__(kGvThreads, 2) szo_linear_gemv_kernel(const __
             a1[1] = ((qb[wd] >> 8) & 0x000F000Fu) | 0x43004300u;
             a1[2] = ((qa[wd] >> 12) & 0x000F000Fu) | 0x43004300u;
             a1[3] = ((qb[wd] >> 12) & 0x000F000Fu) | 0x43004300u;
-            uint4 xv = make_uint4(0u, 0u, 0u, 0u);
-            if (g < M) xv = *reinterpret_cast<const uint4*>(xs + wd * 32);
-            gv_mma_acc(accq[wd & 1], a0, xv.x, xv.y);
+            const uint4 xv = *reinterpret_cast<const uint4*>(xs + wd * 32);
+            if (wd < 2) gv_mma_new(accq[wd & 1], a0, xv.x, xv.y);
+            else gv_mma_acc(accq[wd & 1], a0, xv.x, xv.y);
             gv_mma_acc(accq[wd & 1], a1, xv.z, xv.w);
           }
           const float2 fa = gv_sz_f32<kBf16Tables>(pa), fb = gv_sz_f32<kBf16Tables>(pb);
@@ -375,7 +386,7 @@ constexpr size_t kGvMaxDynSmem = 200 * 1024;
 
 template <bool kBf16Tables, typename TY>
 szo_status launch_gemv(const szo_linear* const* plans, int n, const void* x, const void* x_mul, int64_t M,
-                       const float* const* S, void* const* y, cudaStream_t st) {
+                       const float* const* S, void* const* y, cudaStream_t st, bool chained) {
   auto kern = szo_linear_gemv_kernel<kBf16Tables, TY>;
   static bool configured[64] = {false};
   static std::mutex mu;
@@ -410,7 +421,7 @@ szo_status launch_gemv(const szo_linear* const* plans, int n, const void* x, con
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int per_sm = (2 * (smem + 9 * 1024) <= 227 * 1024) ? 2 : 1;
   const int grid = ctas < per_sm * sms ? ctas : per_sm * sms;
-  kern<<<static_cast<unsigned>(grid), kGvThreads, smem, st>>>(a, ctas);
+  SZO_CHECK_CUDA(launch_maybe_chained(kern, dim3(static_cast<unsigned>(grid)), dim3(kGvThreads), smem, st, chained, a, ctas));
   count_launch();
   SZO_CHECK_LAUNCH("szo_linear_gemv_kernel");
   return SZO_OK;
@@ -437,15 +448,15 @@ bool gemv_applies(const szo_linear* const* plans, int n, int64_t M) {
 }
 
 szo_status linear_fwd_gemv(const szo_linear* const* plans, int n, const void* x, const void* x_mul, int64_t M,
-                           const float* const* S_pert, void* const* y, int y_dtype, cudaStream_t st) {
+                           const float* const* S_pert, void* const* y, int y_dtype, cudaStream_t st, bool chained) {
   SZO_REQUIRE(gemv_applies(plans, n, M), SZO_ERR_UNSUPPORTED, "shapes not covered by the few-token kernel");
   const bool bf = plans[0]->sz_dtype == SZO_BF16;
   if (y_dtype == SZO_F32) {
-    if (bf) return launch_gemv<true, float>(plans, n, x, x_mul, M, S_pert, y, st);
-    return launch_gemv<false, float>(plans, n, x, x_mul, M, S_pert, y, st);
+    if (bf) return launch_gemv<true, float>(plans, n, x, x_mul, M, S_pert, y, st, chained);
+    return launch_gemv<false, float>(plans, n, x, x_mul, M, S_pert, y, st, chained);
   }
-  if (bf) return launch_gemv<true, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st);
-  return launch_gemv<false, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st);
+  if (bf) return launch_gemv<true, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st, chained);
+  return launch_gemv<false, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st, chained);
 }
 
 }  // namespace szo

@@ -46,13 +46,16 @@ bool skinny_applies(const szo_linear* p, int64_t M);
 // One to four tokens (gemm_gemv.cu): a CTA per 16 weight rows, no K-split between CTAs; same
 // arguments as linear_fwd_skinny_group, which hands such calls over.
 bool gemv_applies(const szo_linear* const* plans, int n, int64_t M);
+// chained: launched as part of a chain of dependent kernels (common.cuh); x, x_mul must then be the only
+// arguments that an earlier kernel of the stream writes.
 szo_status linear_fwd_gemv(const szo_linear* const* plans, int n, const void* x, const void* x_mul, int64_t M,
-                           const float* const* S_pert, void* const* y, int y_dtype, cudaStream_t st);
+                           const float* const* S_pert, void* const* y, int y_dtype, cudaStream_t st, bool chained = false);
 // Up to three matrices that read the same activations in one launch (same K, G and table type);
 // x_mul != NULL: the activations are silu(x) * x_mul rounded to bf16, formed while they are staged.
 bool skinny_group_applies(const szo_linear* const* plans, int n, int64_t M);
 szo_status linear_fwd_skinny_group(const szo_linear* const* plans, int n, const void* x, const void* x_mul, int64_t M,
-                                   const float* const* S_pert, void* const* y, int y_dtype, cudaStream_t st);
+                                   const float* const* S_pert, void* const* y, int y_dtype, cudaStream_t st,
+                                   bool chained = false);
 szo_status linear_fwd_skinny(const szo_linear* p, const void* x, int64_t M, const float* S_pert, void* y, int y_dtype,
                              cudaStream_t st);
 

@@ -58,6 +58,8 @@ add_norm_kernel(float* __restrict__ h, const T* __restrict__ y, const float* __r
                 int64_t row_offset, TO* __restrict__ out) {
   constexpr int kMaxV = 8;                       // float4 per thread: d <= 256 * 4 * 8
   __shared__ float scratch[32];
+  chain_release();
+  chain_wait();
   const int64_t m = static_cast<int64_t>(blockIdx.x) * row_stride + row_offset;
   float* x = h + m * d;
   TO* o = out + static_cast<int64_t>(blockIdx.x) * d;
@@ -455,6 +457,8 @@ attn_decode_fused_kernel(const T* __restrict__ q, const T* __restrict__ k_new, c
   constexpr int E = HD / 32, half = HD / 2;
   __shared__ float part_acc[4][HD];
   __shared__ float part_m[4], part_l[4];
+  chain_release();
+  chain_wait();
   const int pos0 = *pos_dev;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int t = blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
@@ -1269,6 +1273,13 @@ szo_status run_decode_t(szo_model* m, const int32_t* tokens, int B, int Tn, cons
   // n matrices that read the same activations: one launch of the weight-streaming kernel where it
   // takes the group, else one call each
   const bool streaming = lmode == SZO_MODE_AUTO && act == SZO_BF16;
+  // The layer kernels of a few-token step are launched as a chain (common.cuh): each may be placed while
+  // the one before drains.  SZO_DECODE_CHAIN=0 launches them the ordinary way (A/B measurement).
+  static const bool chain_on = [] {
+    const char* e = getenv("SZO_DECODE_CHAIN");
+    return e == nullptr || e[0] != '0';
+  }();
+  const bool chained = streaming && chain_on && M <= 16;
   auto lin_group = [&](int layer, int j0, int n, const void* x, void* const* outs) -> szo_status {
     const int t0 = layer * m->n_lin + j0;
     const szo_linear* plans[3];
@@ -1277,7 +1288,8 @@ szo_status run_decode_t(szo_model* m, const int32_t* tokens, int B, int Tn, cons
       plans[i] = m->plans[t0 + i];
       sv[i] = Sv + m->offsets[t0 + i];
     }
-    if (streaming && skinny_group_applies(plans, n, M)) return linear_fwd_skinny_group(plans, n, x, nullptr, M, sv, outs, act, st);
+    if (streaming && skinny_group_applies(plans, n, M))
+      return linear_fwd_skinny_group(plans, n, x, nullptr, M, sv, outs, act, st, chained);
     for (int i = 0; i < n; ++i) SZO_TRY(lin(layer, j0 + i, x, outs[i]));
     return SZO_OK;
   };
@@ -1288,8 +1300,8 @@ szo_status run_decode_t(szo_model* m, const int32_t* tokens, int B, int Tn, cons
   const int64_t layer_cache = static_cast<int64_t>(c.max_batch) * Smax * dkv;
   for (int l = 0; l < c.n_layers; ++l) {
     const szo_layer_weights& L = m->layers[l];
-    add_norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, pending, L.attn_norm_g, L.attn_norm_b, d, c.norm_eps,
-                                                                opt, 1, 0, a);
+    SZO_CHECK_CUDA(launch_maybe_chained(add_norm_kernel<T, T>, dim3(static_cast<unsigned>(M)), dim3(256), 0, st, chained, m->h,
+                                        pending, L.attn_norm_g, L.attn_norm_b, d, c.norm_eps, opt, int64_t(1), int64_t(0), a));
     count_launch();
     {
       void* const qkv[3] = {q, k, v};
@@ -1302,8 +1314,9 @@ szo_status run_decode_t(szo_model* m, const int32_t* tokens, int B, int Tn, cons
     if (Tn <= 16) {
       // rotation, cache append and attention in one launch
       const float2* tab = opt ? nullptr : m->rope_tab;
-      if (hd == 64) attn_decode_fused_kernel<T, 64><<<grid, 128, 0, st>>>(q, k, v, kc, vc, o, tab, Tn, pos_dev, Smax, H, Hkv, scale);
-      else attn_decode_fused_kernel<T, 128><<<grid, 128, 0, st>>>(q, k, v, kc, vc, o, tab, Tn, pos_dev, Smax, H, Hkv, scale);
+      auto attn = hd == 64 ? attn_decode_fused_kernel<T, 64> : attn_decode_fused_kernel<T, 128>;
+      SZO_CHECK_CUDA(launch_maybe_chained(attn, grid, dim3(128), 0, st, chained, q, k, v, kc, vc, o, tab, Tn, pos_dev, Smax, H, Hkv,
+                                          scale));
       count_launch();
     } else {
       if (!opt) {
@@ -1317,8 +1330,13 @@ szo_status run_decode_t(szo_model* m, const int32_t* tokens, int B, int Tn, cons
       else attn_decode_kernel<T, 128><<<grid, 128, 0, st>>>(q, kc, vc, o, Tn, pos_dev, Smax, H, Hkv, scale);
       count_launch(2);
     }
-    SZO_TRY(lin(l, 3, o, y));
-    add_norm_kernel<T><<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, y, L.mlp_norm_g, L.mlp_norm_b, d, c.norm_eps, opt, 1, 0, a);
+    {
+      void* const out[1] = {y};
+      SZO_TRY(lin_group(l, 3, 1, o, out));
+    }
+    SZO_CHECK_CUDA(launch_maybe_chained(add_norm_kernel<T, T>, dim3(static_cast<unsigned>(M)), dim3(256), 0, st, chained, m->h,
+                                        static_cast<const T*>(y), L.mlp_norm_g, L.mlp_norm_b, d, c.norm_eps, opt, int64_t(1),
+                                        int64_t(0), a));
     count_launch();
     if (!opt) {
       void* const gu[2] = {gate, up};
@@ -1328,7 +1346,7 @@ szo_status run_decode_t(szo_model* m, const int32_t* tokens, int B, int Tn, cons
         // silu(gate) * up is formed while the down projection stages its activations
         const float* sv = Sv + m->offsets[l * m->n_lin + 6];
         void* const out[1] = {y};
-        SZO_TRY(linear_fwd_skinny_group(&down, 1, gate, up, M, &sv, out, act, st));
+        SZO_TRY(linear_fwd_skinny_group(&down, 1, gate, up, M, &sv, out, act, st, chained));
       } else {
         silu_mul_kernel<T><<<blocks_for(M * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, up, M * ff, gate);
         count_launch();
