@@ -218,6 +218,7 @@ szo_linear_skinny_kernel(const __grid_constant__ SkinnyArgs a) {
   }
   __syncthreads();
   bool failed = false;
+  chain_release();
 
   if (warp == kWarpProducer) {
     // ---------------------------------------------------------------- producer
@@ -286,6 +287,7 @@ szo_linear_skinny_kernel(const __grid_constant__ SkinnyArgs a) {
       load_rp(cid + n_clusters, b1, e1);
     }
     // ---------------------------------------------------------------- workers: stage the activations
+    chain_wait();        // (launched in a chain: the activations are the predecessor's output; weights and entries are nobody's)
     {
       // a thread takes one 16-byte chunk (8 columns) of the 8 tokens of a token tile: 8 loads, the same chunks into the
       // [token][column] tile, and their 8 x 8 transpose into the [column][token] copy
@@ -590,7 +592,7 @@ size_t skinny_dyn_smem(int64_t K, int G, int kT, int n_stages = kStages) {
 
 template <bool kBf16Tables, bool kGroupMma, typename TY, int kNT>
 szo_status launch_skinny(const szo_linear* const* plans, int n, const void* x, const void* x_mul, int64_t M,
-                         const float* const* S, void* const* y, cudaStream_t st) {
+                         const float* const* S, void* const* y, cudaStream_t st, bool chained) {
   auto kern = szo_linear_skinny_kernel<kBf16Tables, kGroupMma, TY, kNT>;
   const szo_linear* p = plans[0];
   // A ring of 8 steps when two CTAs of that size still share an SM (or when 4 would not change that
@@ -651,7 +653,9 @@ szo_status launch_skinny(const szo_linear* const* plans, int n, const void* x, c
   }
   a.n_tiles = n_tiles;
   const int n_clusters = n_tiles < max_clusters ? n_tiles : max_clusters;
-  kern<<<static_cast<unsigned>(kSplit * n_clusters), kThreads, smem, st>>>(a);
+  // (with two token tiles per CTA an early-placed successor costs more than it hides: 4.8 -> 5.4 ms per 16-token step)
+  SZO_CHECK_CUDA(launch_maybe_chained(kern, dim3(static_cast<unsigned>(kSplit * n_clusters)), dim3(kThreads), smem, st,
+                                      chained && kNT == 1, a));
   count_launch();
   SZO_CHECK_LAUNCH("szo_linear_skinny_kernel");
   return SZO_OK;
@@ -659,14 +663,14 @@ szo_status launch_skinny(const szo_linear* const* plans, int n, const void* x, c
 
 template <bool kBf16Tables, typename TY>
 szo_status launch_skinny_nt(const szo_linear* const* plans, int n, const void* x, const void* x_mul, int64_t M,
-                            const float* const* S, void* const* y, cudaStream_t st) {
+                            const float* const* S, void* const* y, cudaStream_t st, bool chained) {
   const bool group = plans[0]->G % kStepK == 0;
   if (M <= kTok) {
-    if (group) return launch_skinny<kBf16Tables, true, TY, 1>(plans, n, x, x_mul, M, S, y, st);
-    return launch_skinny<kBf16Tables, false, TY, 1>(plans, n, x, x_mul, M, S, y, st);
+    if (group) return launch_skinny<kBf16Tables, true, TY, 1>(plans, n, x, x_mul, M, S, y, st, chained);
+    return launch_skinny<kBf16Tables, false, TY, 1>(plans, n, x, x_mul, M, S, y, st, chained);
   }
-  if (group) return launch_skinny<kBf16Tables, true, TY, 2>(plans, n, x, x_mul, M, S, y, st);
-  return launch_skinny<kBf16Tables, false, TY, 2>(plans, n, x, x_mul, M, S, y, st);
+  if (group) return launch_skinny<kBf16Tables, true, TY, 2>(plans, n, x, x_mul, M, S, y, st, chained);
+  return launch_skinny<kBf16Tables, false, TY, 2>(plans, n, x, x_mul, M, S, y, st, chained);
 }
 
 }  // namespace
@@ -695,11 +699,11 @@ szo_status linear_fwd_skinny_group(const szo_linear* const* plans, int n, const 
   if (gemv_applies(plans, n, M)) return linear_fwd_gemv(plans, n, x, x_mul, M, S_pert, y, y_dtype, st, chained);
   const bool bf = plans[0]->sz_dtype == SZO_BF16;
   if (y_dtype == SZO_F32) {
-    if (bf) return launch_skinny_nt<true, float>(plans, n, x, x_mul, M, S_pert, y, st);
-    return launch_skinny_nt<false, float>(plans, n, x, x_mul, M, S_pert, y, st);
+    if (bf) return launch_skinny_nt<true, float>(plans, n, x, x_mul, M, S_pert, y, st, chained);
+    return launch_skinny_nt<false, float>(plans, n, x, x_mul, M, S_pert, y, st, chained);
   }
-  if (bf) return launch_skinny_nt<true, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st);
-  return launch_skinny_nt<false, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st);
+  if (bf) return launch_skinny_nt<true, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st, chained);
+  return launch_skinny_nt<false, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st, chained);
 }
 
 szo_status linear_fwd_skinny(const szo_linear* p, const void* x, int64_t M, const float* S_pert, void* y, int y_dtype,
