@@ -22,7 +22,11 @@
 //     sums are double-buffered, so the weight warps never wait for it.
 // One launch serves up to three matrices that read the same activations (q/k/v, gate/up); the
 // activations may be silu(x) * x_mul formed while they are staged.  Quantization groups must be
-// multiples of 128 columns.  The kernel waits on nothing but its own block barriers.
+// multiples of 128 columns.
+// Codes into a per-row table of 16 values (the non-uniform 4-bit format) take the same kernel: the
+// tables of the 16 rows (512 bytes as bf16) travel with every step in the registers that otherwise
+// carry (scale, zero), are put into the warp's own shared memory when a row group begins, and every
+// code is looked up there (one 2-byte read of shared memory per code instead of half an AND-OR).  The kernel waits on nothing but its own block barriers.
 #include <cstdlib>
 #include <mutex>
 
@@ -40,10 +44,12 @@ constexpr int kGvStepK = 128;        // columns per step
 constexpr int kGvDepth = 4;          // steps in flight per warp (registers)
 constexpr int kGvMaxTok = 2;          // more tokens: the 16-token kernel (staging four rows of x per CTA costs more than its rendezvous)
 constexpr int kGvPad = 32;           // elements added to a token row in shared memory
+constexpr int kGvTabStride = 48;     // bytes per row of a warp's table block in shared memory (32 used)
 
 struct GemvSub {
   const uint8_t* codes_tiled;
   const float2* sz;
+  const __nv_bfloat16* lut; // [Npad][16] (table-coded weights), else NULL
   int64_t Npad;
   const int32_t* row_ptr;   // NULL: no sparse entries
   const int32_t* ent_col;
@@ -123,10 +129,11 @@ __device__ __forceinline__ void gv_bar_arrive(int id) {
 
 // Grid: persistent CTAs; CTA b takes the 16-row groups b, b + gridDim.x, ... of the `total` groups of
 // all matrices (numbered in matrix order).
-template <bool kBf16Tables, typename TY>
+template <bool kLut, bool kBf16Tables, typename TY>
 __global__ void __launch_bounds__(kGvThreads, 2) szo_linear_gemv_kernel(const __grid_constant__ GemvArgs a, int total) {
   extern __shared__ __align__(128) unsigned char smem_gv[];
   __shared__ float part[2][kGvWarps][kGvRows * 8];        // [buffer][warp][row][token]
+  __shared__ __align__(16) unsigned char wtab_s[kLut ? kGvWarps * kGvRows * kGvTabStride : 16];   // per warp: the 16 rows' tables
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
@@ -147,7 +154,7 @@ __global__ void __launch_bounds__(kGvThreads, 2) szo_linear_gemv_kernel(const __
   const int n_my = warp < kGvWarps ? (warp + 1) * n_steps / kGvWarps - s_begin : 0;
   // fetch cursor: step fj of group fg, with running pointers to this lane's 16 bytes of row g in k-block
   // (t >> 1) of that step (row g + 8 is 256 bytes further) and to its (scale, zero) entry (rows g, g + 8)
-  const int steps_per_qgroup = G / kGvStepK;            // steps that share one (scale, zero) entry
+  const int steps_per_qgroup = kLut ? 1 : G / kGvStepK; // steps that share one (scale, zero) entry
   int fg = static_cast<int>(blockIdx.x), fj = 0, fzc = 0;
   const uint8_t* fc = nullptr;
   const float2* fz = nullptr;
@@ -158,19 +165,30 @@ __global__ void __launch_bounds__(kGvThreads, 2) szo_linear_gemv_kernel(const __
     fc = sb.codes_tiled + (static_cast<int64_t>(r16 >> 3) * (K / 64) + 2 * s_begin + (t >> 1)) * 4096 + (r16 & 7) * 512 +
          g * 32 + (t & 1) * 16;
     fNpad = sb.Npad;
-    fz = sb.sz + static_cast<int64_t>(r16) * kGvRows + g + static_cast<int64_t>(s_begin / steps_per_qgroup) * fNpad;
-    fzc = s_begin % steps_per_qgroup;
+    if constexpr (kLut) {
+      // lane l carries half l & 1 of the table of row l >> 1 (16 bytes)
+      fz = reinterpret_cast<const float2*>(sb.lut + (static_cast<int64_t>(r16) * kGvRows + (lane >> 1)) * 16 + (lane & 1) * 8);
+    } else {
+      fz = sb.sz + static_cast<int64_t>(r16) * kGvRows + g + static_cast<int64_t>(s_begin / steps_per_qgroup) * fNpad;
+      fzc = s_begin % steps_per_qgroup;
+    }
   };
   auto fetch = [&](uint4& wa, uint4& wb, float2& pa, float2& pb) {     // the step under the cursor, then advance it
     if (fg < total) {
       wa = gv_ld_stream(fc);
       wb = gv_ld_stream(fc + 8 * 32);
-      pa = __ldg(fz);
-      pb = __ldg(fz + 8);
       fc += 2 * 4096;
-      if (++fzc == steps_per_qgroup) {
-        fzc = 0;
-        fz += fNpad;
+      if constexpr (kLut) {
+        const float4 tb = __ldg(reinterpret_cast<const float4*>(fz));     // (L2 after the group's first step)
+        pa = make_float2(tb.x, tb.y);
+        pb = make_float2(tb.z, tb.w);
+      } else {
+        pa = __ldg(fz);
+        pb = __ldg(fz + 8);
+        if (++fzc == steps_per_qgroup) {
+          fzc = 0;
+          fz += fNpad;
+        }
       }
       if (++fj == n_my) {
         fj = 0;
@@ -280,29 +298,67 @@ __global__ void __launch_bounds__(kGvThreads, 2) szo_linear_gemv_kernel(const __
           const uint32_t qa[4] = {wa.x, wa.y, wa.z, wa.w}, qb[4] = {wb.x, wb.y, wb.z, wb.w};
           const __nv_bfloat16* xs = xs0 + cj * kGvStepK;
           float accq[2][4];                                 // even and odd words: two shorter chains
+          if constexpr (kLut) {
+            unsigned char* wtab = wtab_s + warp * (kGvRows * kGvTabStride);
+            if (cj == 0) {                                  // a new row group: its tables into the warp's block
+              __syncwarp();
+              *reinterpret_cast<float4*>(wtab + (lane >> 1) * kGvTabStride + (lane & 1) * 16) = make_float4(pa.x, pa.y, pb.x, pb.y);
+              __syncwarp();
+            }
+            const unsigned char* ta = wtab + g * kGvTabStride;          // row g; row g + 8 is 8 strides further
+            auto look = [&](const unsigned char* tab, uint32_t q, int lo_shift) -> uint32_t {
+              // bf16 pair (table[nibble at lo_shift], table[nibble at lo_shift + 16]); byte offset = 2 * nibble
+              const uint32_t o0 = lo_shift == 0 ? (q << 1) & 0x1Eu : (q >> (lo_shift - 1)) & 0x1Eu;
+              const uint32_t o1 = (q >> (lo_shift + 15)) & 0x1Eu;
+              const uint32_t v0 = *reinterpret_cast<const unsigned short*>(tab + o0);
+              const uint32_t v1 = *reinterpret_cast<const unsigned short*>(tab + o1);
+              return v0 | (v1 << 16);
+            };
 #pragma unroll
-          for (int wd = 0; wd < 4; ++wd) {                  // one 32-bit word = 8 columns = two k16 MMAs
-            uint32_t a0[4], a1[4];
-            a0[0] = (qa[wd] & 0x000F000Fu) | 0x43004300u;
-            a0[1] = (qb[wd] & 0x000F000Fu) | 0x43004300u;
-            a0[2] = ((qa[wd] >> 4) & 0x000F000Fu) | 0x43004300u;
-            a0[3] = ((qb[wd] >> 4) & 0x000F000Fu) | 0x43004300u;
-            a1[0] = ((qa[wd] >> 8) & 0x000F000Fu) | 0x43004300u;
-            a1[1] = ((qb[wd] >> 8) & 0x000F000Fu) | 0x43004300u;
-            a1[2] = ((qa[wd] >> 12) & 0x000F000Fu) | 0x43004300u;
-            a1[3] = ((qb[wd] >> 12) & 0x000F000Fu) | 0x43004300u;
-            const uint4 xv = *reinterpret_cast<const uint4*>(xs + wd * 32);
-            if (wd < 2) gv_mma_new(accq[wd & 1], a0, xv.x, xv.y);
-            else gv_mma_acc(accq[wd & 1], a0, xv.x, xv.y);
-            gv_mma_acc(accq[wd & 1], a1, xv.z, xv.w);
+            for (int wd = 0; wd < 4; ++wd) {
+              uint32_t a0[4], a1[4];
+              a0[0] = look(ta, qa[wd], 0);
+              a0[1] = look(ta + 8 * kGvTabStride, qb[wd], 0);
+              a0[2] = look(ta, qa[wd], 4);
+              a0[3] = look(ta + 8 * kGvTabStride, qb[wd], 4);
+              a1[0] = look(ta, qa[wd], 8);
+              a1[1] = look(ta + 8 * kGvTabStride, qb[wd], 8);
+              a1[2] = look(ta, qa[wd], 12);
+              a1[3] = look(ta + 8 * kGvTabStride, qb[wd], 12);
+              const uint4 xv = *reinterpret_cast<const uint4*>(xs + wd * 32);
+              if (wd < 2) gv_mma_new(accq[wd & 1], a0, xv.x, xv.y);
+              else gv_mma_acc(accq[wd & 1], a0, xv.x, xv.y);
+              gv_mma_acc(accq[wd & 1], a1, xv.z, xv.w);
+            }
+            tot[0] += accq[0][0] + accq[1][0];
+            tot[1] += accq[0][1] + accq[1][1];
+            tot[2] += accq[0][2] + accq[1][2];
+            tot[3] += accq[0][3] + accq[1][3];
+          } else {
+#pragma unroll
+            for (int wd = 0; wd < 4; ++wd) {                // one 32-bit word = 8 columns = two k16 MMAs
+              uint32_t a0[4], a1[4];
+              a0[0] = (qa[wd] & 0x000F000Fu) | 0x43004300u;
+              a0[1] = (qb[wd] & 0x000F000Fu) | 0x43004300u;
+              a0[2] = ((qa[wd] >> 4) & 0x000F000Fu) | 0x43004300u;
+              a0[3] = ((qb[wd] >> 4) & 0x000F000Fu) | 0x43004300u;
+              a1[0] = ((qa[wd] >> 8) & 0x000F000Fu) | 0x43004300u;
+              a1[1] = ((qb[wd] >> 8) & 0x000F000Fu) | 0x43004300u;
+              a1[2] = ((qa[wd] >> 12) & 0x000F000Fu) | 0x43004300u;
+              a1[3] = ((qb[wd] >> 12) & 0x000F000Fu) | 0x43004300u;
+              const uint4 xv = *reinterpret_cast<const uint4*>(xs + wd * 32);
+              if (wd < 2) gv_mma_new(accq[wd & 1], a0, xv.x, xv.y);
+              else gv_mma_acc(accq[wd & 1], a0, xv.x, xv.y);
+              gv_mma_acc(accq[wd & 1], a1, xv.z, xv.w);
+            }
+            const float2 fa = gv_sz_f32<kBf16Tables>(pa), fb = gv_sz_f32<kBf16Tables>(pb);
+            const float za = fmaf(-128.f, fa.x, fa.y), zb = fmaf(-128.f, fb.x, fb.y);
+            const float2 xs2 = *reinterpret_cast<const float2*>(xsum0 + cj * 8);
+            tot[0] = fmaf(fa.x, accq[0][0] + accq[1][0], fmaf(za, xs2.x, tot[0]));
+            tot[1] = fmaf(fa.x, accq[0][1] + accq[1][1], fmaf(za, xs2.y, tot[1]));
+            tot[2] = fmaf(fb.x, accq[0][2] + accq[1][2], fmaf(zb, xs2.x, tot[2]));
+            tot[3] = fmaf(fb.x, accq[0][3] + accq[1][3], fmaf(zb, xs2.y, tot[3]));
           }
-          const float2 fa = gv_sz_f32<kBf16Tables>(pa), fb = gv_sz_f32<kBf16Tables>(pb);
-          const float za = fmaf(-128.f, fa.x, fa.y), zb = fmaf(-128.f, fb.x, fb.y);
-          const float2 xs2 = *reinterpret_cast<const float2*>(xsum0 + cj * 8);
-          tot[0] = fmaf(fa.x, accq[0][0] + accq[1][0], fmaf(za, xs2.x, tot[0]));
-          tot[1] = fmaf(fa.x, accq[0][1] + accq[1][1], fmaf(za, xs2.y, tot[1]));
-          tot[2] = fmaf(fb.x, accq[0][2] + accq[1][2], fmaf(zb, xs2.x, tot[2]));
-          tot[3] = fmaf(fb.x, accq[0][3] + accq[1][3], fmaf(zb, xs2.y, tot[3]));
           fetch(rwa[d], rwb[d], rpa[d], rpb[d]);            // (after the slot's last use: no copies of its registers)
           if (++cj == n_my) {                               // the row group is complete
             const int buf = it & 1;
@@ -384,10 +440,10 @@ size_t gemv_dyn_smem(int64_t K, int64_t M) {
 }
 constexpr size_t kGvMaxDynSmem = 200 * 1024;
 
-template <bool kBf16Tables, typename TY>
+template <bool kLut, bool kBf16Tables, typename TY>
 szo_status launch_gemv(const szo_linear* const* plans, int n, const void* x, const void* x_mul, int64_t M,
                        const float* const* S, void* const* y, cudaStream_t st, bool chained) {
-  auto kern = szo_linear_gemv_kernel<kBf16Tables, TY>;
+  auto kern = szo_linear_gemv_kernel<kLut, kBf16Tables, TY>;
   static bool configured[64] = {false};
   static std::mutex mu;
   int dev = 0;
@@ -411,8 +467,8 @@ szo_status launch_gemv(const szo_linear* const* plans, int n, const void* x, con
   int ctas = 0;
   for (int i = 0; i < n; ++i) {
     const szo_linear* q = plans[i];
-    a.sub[i] = GemvSub{q->codes_tiled, q->sz, q->Npad, q->nnz > 0 ? q->row_ptr : nullptr, q->ent_col, S[i], q->bias, y[i],
-                       q->N, ctas};
+    a.sub[i] = GemvSub{q->codes_tiled, q->sz, q->lut_bf16, q->Npad, q->nnz > 0 ? q->row_ptr : nullptr, q->ent_col, S[i],
+                       q->bias, y[i], q->N, ctas};
     ctas += static_cast<int>(ceil_div(q->N, kGvRows));
   }
   // persistent CTAs: as many as are resident at once (two per SM while the activations leave room)
@@ -429,8 +485,8 @@ szo_status launch_gemv(const szo_linear* const* plans, int n, const void* x, con
 
 }  // namespace
 
-// int4 plans with groups of a multiple of 128 columns, at most four tokens, up to three matrices with
-// the same K, group size and table type.  SZO_GEMV=0 switches the kernel off (A/B measurement).
+// int4 plans with groups of a multiple of 128 columns or with per-row tables, at most two tokens, up to
+// three matrices with the same K, group size and table type.  SZO_GEMV=0 switches the kernel off (A/B measurement).
 bool gemv_applies(const szo_linear* const* plans, int n, int64_t M) {
   static const bool off = [] {
     const char* e = getenv("SZO_GEMV");
@@ -438,11 +494,13 @@ bool gemv_applies(const szo_linear* const* plans, int n, int64_t M) {
   }();
   if (off || n < 1 || n > 3 || M < 1 || M > kGvMaxTok) return false;
   const szo_linear* p = plans[0];
-  if (p->G <= 0 || p->G % kGvStepK != 0 || p->K % kGvStepK != 0 || p->K / kGvStepK < kGvWarps ||
+  const bool lut = p->G == -1 && p->lut_bf16 != nullptr;
+  if (!(lut || (p->G > 0 && p->G % kGvStepK == 0)) || p->K % kGvStepK != 0 || p->K / kGvStepK < kGvWarps ||
       gemv_dyn_smem(p->K, M) > kGvMaxDynSmem)
     return false;
   for (int i = 0; i < n; ++i)
-    if (plans[i]->K != p->K || plans[i]->G != p->G || plans[i]->sz_dtype != p->sz_dtype || plans[i]->codes_tiled == nullptr)
+    if (plans[i]->K != p->K || plans[i]->G != p->G || plans[i]->sz_dtype != p->sz_dtype || plans[i]->codes_tiled == nullptr ||
+        (lut && plans[i]->lut_bf16 == nullptr))
       return false;
   return true;
 }
@@ -451,12 +509,16 @@ szo_status linear_fwd_gemv(const szo_linear* const* plans, int n, const void* x,
                            const float* const* S_pert, void* const* y, int y_dtype, cudaStream_t st, bool chained) {
   SZO_REQUIRE(gemv_applies(plans, n, M), SZO_ERR_UNSUPPORTED, "shapes not covered by the few-token kernel");
   const bool bf = plans[0]->sz_dtype == SZO_BF16;
-  if (y_dtype == SZO_F32) {
-    if (bf) return launch_gemv<true, float>(plans, n, x, x_mul, M, S_pert, y, st, chained);
-    return launch_gemv<false, float>(plans, n, x, x_mul, M, S_pert, y, st, chained);
+  if (plans[0]->G == -1) {                    // (the plan's bf16 copy of the tables is read: the tables' own type does not matter)
+    if (y_dtype == SZO_F32) return launch_gemv<true, false, float>(plans, n, x, x_mul, M, S_pert, y, st, chained);
+    return launch_gemv<true, false, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st, chained);
   }
-  if (bf) return launch_gemv<true, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st, chained);
-  return launch_gemv<false, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st, chained);
+  if (y_dtype == SZO_F32) {
+    if (bf) return launch_gemv<false, true, float>(plans, n, x, x_mul, M, S_pert, y, st, chained);
+    return launch_gemv<false, false, float>(plans, n, x, x_mul, M, S_pert, y, st, chained);
+  }
+  if (bf) return launch_gemv<false, true, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st, chained);
+  return launch_gemv<false, false, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st, chained);
 }
 
 }  // namespace szo

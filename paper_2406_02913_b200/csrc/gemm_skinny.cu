@@ -693,10 +693,14 @@ bool skinny_group_applies(const szo_linear* const* plans, int n, int64_t M) {
   return true;
 }
 
+bool few_token_applies(const szo_linear* const* plans, int n, int64_t M) {
+  return gemv_applies(plans, n, M) || skinny_group_applies(plans, n, M);
+}
+
 szo_status linear_fwd_skinny_group(const szo_linear* const* plans, int n, const void* x, const void* x_mul, int64_t M,
                                    const float* const* S_pert, void* const* y, int y_dtype, cudaStream_t st, bool chained) {
-  SZO_REQUIRE(skinny_group_applies(plans, n, M), SZO_ERR_UNSUPPORTED, "shapes not covered by the weight-streaming kernel");
   if (gemv_applies(plans, n, M)) return linear_fwd_gemv(plans, n, x, x_mul, M, S_pert, y, y_dtype, st, chained);
+  SZO_REQUIRE(skinny_group_applies(plans, n, M), SZO_ERR_UNSUPPORTED, "shapes not covered by the weight-streaming kernel");
   const bool bf = plans[0]->sz_dtype == SZO_BF16;
   if (y_dtype == SZO_F32) {
     if (bf) return launch_skinny_nt<true, float>(plans, n, x, x_mul, M, S_pert, y, st, chained);

@@ -378,7 +378,7 @@ szo_status linear_fwd_impl(const szo_linear* p, const void* x, int x_dtype, int6
     SZO_TRY(linear_fwd_tc(p, x, M, nullptr, y, y_dtype, workspace, workspace_bytes, st));
     return linear_spmm(p, x, M, S_pert, y, y_dtype, st);
   }
-  if (mode == SZO_MODE_AUTO && skinny_applies(p, M)) return linear_fwd_skinny(p, x, M, S_pert, y, y_dtype, st);
+  if (mode == SZO_MODE_AUTO && few_token_applies(&p, 1, M)) return linear_fwd_skinny(p, x, M, S_pert, y, y_dtype, st);
   if (tc_use_materialised(p, M))
     return linear_fwd_tc_materialised(&p, 1, x, M, &S_pert, &y, y_dtype, workspace, workspace_bytes, st);
   unsigned char* ws = static_cast<unsigned char*>(workspace);
@@ -541,7 +541,8 @@ szo_status szo_linear_create_lut(szo_linear_t** out, int64_t N, int64_t K, const
 size_t szo_linear_workspace_bytes(const szo_linear_t* p, int64_t M, int32_t mode) {
   if (!p) return 0;
   if (mode == SZO_MODE_FP32_VALIDATE) return linear_ws_fp32(p, M);
-  if (mode == SZO_MODE_AUTO && skinny_applies(p, M)) return 0;
+  const szo_linear* self = p;
+  if (mode == SZO_MODE_AUTO && few_token_applies(&self, 1, M)) return 0;
   const szo_linear* pp = p;
   const size_t tail = tc_tail_ws_bytes(&pp, 1, M);                     // K-split tiles of the last round
   if (mode == SZO_MODE_SPMM) return tail;

@@ -53,6 +53,7 @@ szo_status linear_fwd_gemv(const szo_linear* const* plans, int n, const void* x,
 // Up to three matrices that read the same activations in one launch (same K, G and table type);
 // x_mul != NULL: the activations are silu(x) * x_mul rounded to bf16, formed while they are staged.
 bool skinny_group_applies(const szo_linear* const* plans, int n, int64_t M);
+bool few_token_applies(const szo_linear* const* plans, int n, int64_t M);     // either few-token kernel takes the group
 szo_status linear_fwd_skinny_group(const szo_linear* const* plans, int n, const void* x, const void* x_mul, int64_t M,
                                    const float* const* S_pert, void* const* y, int y_dtype, cudaStream_t st,
                                    bool chained = false);

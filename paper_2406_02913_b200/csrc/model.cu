@@ -1288,7 +1288,7 @@ szo_status run_decode_t(szo_model* m, const int32_t* tokens, int B, int Tn, cons
       plans[i] = m->plans[t0 + i];
       sv[i] = Sv + m->offsets[t0 + i];
     }
-    if (streaming && skinny_group_applies(plans, n, M))
+    if (streaming && few_token_applies(plans, n, M))
       return linear_fwd_skinny_group(plans, n, x, nullptr, M, sv, outs, act, st, chained);
     for (int i = 0; i < n; ++i) SZO_TRY(lin(layer, j0 + i, x, outs[i]));
     return SZO_OK;
@@ -1342,7 +1342,7 @@ szo_status run_decode_t(szo_model* m, const int32_t* tokens, int B, int Tn, cons
       void* const gu[2] = {gate, up};
       SZO_TRY(lin_group(l, 4, 2, a, gu));
       const szo_linear* down = m->plans[l * m->n_lin + 6];
-      if (streaming && skinny_group_applies(&down, 1, M)) {
+      if (streaming && few_token_applies(&down, 1, M)) {
         // silu(gate) * up is formed while the down projection stages its activations
         const float* sv = Sv + m->offsets[l * m->n_lin + 6];
         void* const out[1] = {y};

@@ -117,10 +117,16 @@ def steady_case(M, N, K, G, mode, rho, reps, total_bytes=400e6):
     idx = B.szo_select_mask(g * g, nnz)
     S = W.view(-1)[idx].contiguous()
     W.view(-1)[idx] = 0.0
-    codes, sc, ze = B.szo_quantize(W, G, "bf16")
     n_plans = max(2, int(total_bytes / (N * K / 2)) + 1)
-    keep = [(codes.clone(), sc.clone(), ze.clone(), idx.clone(), S.clone()) for _ in range(n_plans)]
-    plans = [B.Linear(N, K, G, c, s_, z_, "bf16", i_) for (c, s_, z_, i_, _) in keep]
+    if G > 0:
+        codes, sc, ze = B.szo_quantize(W, G, "bf16")
+        keep = [(codes.clone(), sc.clone(), ze.clone(), idx.clone(), S.clone()) for _ in range(n_plans)]
+        plans = [B.Linear(N, K, G, c, s_, z_, "bf16", i_) for (c, s_, z_, i_, _) in keep]
+    else:          # non-uniform 4-bit format: random codes into per-row tables of 16 fp16 values
+        codes = torch.from_numpy(wl.random_codes(N, K, seed=0, i=4)).cuda()
+        lut = torch.from_numpy(wl.random_lut(N, seed=0, i=5)).cuda().to(torch.float16)
+        keep = [(codes.clone(), lut.clone(), None, idx.clone(), S.clone()) for _ in range(n_plans)]
+        plans = [B.Linear(N, K, G, c, None, None, "bf16", i_, lut=l_) for (c, l_, _, i_, _) in keep]
     x = torch.from_numpy(wl.activation(M, K, seed=0, i=3)).cuda().to(torch.bfloat16)
     ys = [torch.empty((M, N), dtype=torch.bfloat16, device="cuda") for _ in range(n_plans)]
     rounds = 4
@@ -151,7 +157,7 @@ def steady_case(M, N, K, G, mode, rho, reps, total_bytes=400e6):
             ts.append(e0.elapsed_time(e1) / (rounds * n_plans))
     med = statistics.median(ts)
     hbm, _, src = peaks()
-    byts = N * K / 2 + 4 * N * K / G + 2 * M * K + 2 * M * N + 8 * nnz
+    byts = N * K / 2 + (4 * N * K / G if G > 0 else 32 * N) + 2 * M * K + 2 * M * N + 8 * nnz
     line = {"case": "linear_steady", "M": M, "N": N, "K": K, "G": G, "mode": mode, "nnz": nnz, "plans": n_plans,
             "us_per_call_median": med * 1e3, "us_per_call_min": min(ts) * 1e3, "gbs": byts / (med * 1e-3) / 1e9,
             "frac_of_hbm": byts / (med * 1e-3) / 1e9 / hbm, "peaks": src, "status": B.device_status()}

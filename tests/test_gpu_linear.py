@@ -236,6 +236,10 @@ LUT_CASES = [
     (200, 320, "f16", 65, 5e-3, False),             # N not a multiple of the tile: padded table rows
     (512, 4096, "f16", 16, 1e-3, True),             # long K, few tokens: K-split tiles
     (128, 64, "bf16", 1, 0.0, False),               # one token, one k-block, no sparse entries
+    # one or two tokens, at least eight 128-column steps: SZO_MODE_AUTO looks the codes up inside the few-token kernel
+    (200, 1024, "f16", 1, 5e-3, True),              # N not a multiple of 16; one step per warp
+    (512, 4096, "bf16", 2, 1e-3, False),
+    (304, 11008, "f16", 1, 2e-3, True),             # 86 steps: several row groups per CTA, tables change with them
 ]
 
 
