@@ -64,6 +64,7 @@ struct GemvArgs {
   int n;
   const __nv_bfloat16* x;
   const __nv_bfloat16* x_mul;   // not NULL: the activations are silu(x) * x_mul
+  FusedNorm norm;               // h_in not NULL: the activations are the normalised residual stream (linear.cuh)
   int M;
   int64_t K;
   int G;
@@ -110,6 +111,20 @@ __device__ __forceinline__ uint4 gv_silu_mul(uint4 g, uint4 u) {
     o[i] = *reinterpret_cast<const uint32_t*>(&r);
   }
   return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// Block-wide sum of 256 threads with the fixed tree of the model's norm kernel: shuffles inside a warp,
+// then the eight warps' values in warp order
+__device__ __forceinline__ float gv_block_sum(float v, float* scratch) {
+#pragma unroll
+  for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float t = 0.f;
+#pragma unroll
+  for (int i = 0; i < kGvThreads / 32; ++i) t += scratch[i];
+  return t;
 }
 
 // streaming 128-bit load: the weights are read once
@@ -235,7 +250,56 @@ __global__ void __launch_bounds__(kGvThreads, 2) szo_linear_gemv_kernel(const __
   };
   // ---------------------------------------------------------------- everybody: stage the activations, once
   chain_wait();          // the weights above are nobody's output; the activations are the predecessor's
-  {
+  if (a.norm.h_in != nullptr) {
+    // residual add and norm (add_norm_kernel's arithmetic and reduction tree, 256 threads): v goes
+    // through shared memory as fp32, since the thread that normalises a 16-byte chunk is not the
+    // one that summed it
+    float* vs = xsum + n_steps * 8;                       // [M][K]
+    float* scratch = &part[0][0][0];
+    const int nv = static_cast<int>(K / 4);
+    for (int m = 0; m < M; ++m) {
+      const float4* hp = reinterpret_cast<const float4*>(a.norm.h_in + static_cast<int64_t>(m) * K);
+      float sum = 0.f;
+      for (int c = threadIdx.x; c < nv; c += kGvThreads) {
+        float4 v = hp[c];
+        if (a.norm.y_add != nullptr) {
+          const uint2 raw = *reinterpret_cast<const uint2*>(a.norm.y_add + static_cast<int64_t>(m) * K + c * 4);
+          v.x += __uint_as_float(raw.x << 16);
+          v.y += __uint_as_float(raw.x & 0xFFFF0000u);
+          v.z += __uint_as_float(raw.y << 16);
+          v.w += __uint_as_float(raw.y & 0xFFFF0000u);
+        }
+        reinterpret_cast<float4*>(vs + static_cast<size_t>(m) * K)[c] = v;
+        if (blockIdx.x == 0) reinterpret_cast<float4*>(a.norm.h_out + static_cast<int64_t>(m) * K)[c] = v;
+        sum += (v.x + v.y) + (v.z + v.w);
+      }
+      const float mu = a.norm.layer_norm ? gv_block_sum(sum, scratch) / static_cast<float>(K) : 0.f;
+      float q = 0.f;
+      for (int c = threadIdx.x; c < nv; c += kGvThreads) {
+        const float4 v = reinterpret_cast<const float4*>(vs + static_cast<size_t>(m) * K)[c];
+        const float a0 = v.x - mu, a1 = v.y - mu, a2 = v.z - mu, a3 = v.w - mu;
+        q += (a0 * a0 + a1 * a1) + (a2 * a2 + a3 * a3);
+      }
+      const float var = gv_block_sum(q, scratch) / static_cast<float>(K);
+      const float r = 1.0f / sqrtf(var + a.norm.eps);
+      for (int c8 = threadIdx.x; c8 < nv / 2; c8 += kGvThreads) {        // one 16-byte chunk of bf16
+        uint32_t o[4];
+#pragma unroll
+        for (int hx = 0; hx < 2; ++hx) {
+          const int c = c8 * 2 + hx;
+          const float4 v = reinterpret_cast<const float4*>(vs + static_cast<size_t>(m) * K)[c];
+          const float4 gm = reinterpret_cast<const float4*>(a.norm.gamma)[c];
+          float4 bt = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (a.norm.beta != nullptr) bt = reinterpret_cast<const float4*>(a.norm.beta)[c];
+          const __nv_bfloat162 lo = __floats2bfloat162_rn((v.x - mu) * r * gm.x + bt.x, (v.y - mu) * r * gm.y + bt.y);
+          const __nv_bfloat162 hi = __floats2bfloat162_rn((v.z - mu) * r * gm.z + bt.z, (v.w - mu) * r * gm.w + bt.w);
+          o[2 * hx] = *reinterpret_cast<const uint32_t*>(&lo);
+          o[2 * hx + 1] = *reinterpret_cast<const uint32_t*>(&hi);
+        }
+        *reinterpret_cast<uint4*>(sx + static_cast<size_t>(m) * ld + gv_chunk_pos(c8) * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+      }
+    }
+  } else {
     // (all loads of a batch first: a chunk is one round trip to L2, and there are one to five batches)
     const int chunks = static_cast<int>(K / 8), total_chunks = chunks * M;
     constexpr int kBatch = 4;
@@ -259,6 +323,8 @@ __global__ void __launch_bounds__(kGvThreads, 2) szo_linear_gemv_kernel(const __
         }
       }
     }
+  }
+  {
     for (int i = threadIdx.x; i < n_steps * 8; i += kGvThreads)
       if ((i & 7) >= M) xsum[i] = 0.f;
     gv_bar_sync(1);
@@ -434,15 +500,15 @@ __global__ void __launch_bounds__(kGvThreads, 2) szo_linear_gemv_kernel(const __
   }
 }
 
-size_t gemv_dyn_smem(int64_t K, int64_t M) {
-  return static_cast<size_t>(M) * (K + kGvPad) * 2 +
-         static_cast<size_t>(K / kGvStepK) * 8 * sizeof(float);
+size_t gemv_dyn_smem(int64_t K, int64_t M, bool norm = false) {
+  return static_cast<size_t>(M) * (K + kGvPad) * 2 + static_cast<size_t>(K / kGvStepK) * 8 * sizeof(float) +
+         (norm ? static_cast<size_t>(M) * K * sizeof(float) : 0);
 }
 constexpr size_t kGvMaxDynSmem = 200 * 1024;
 
 template <bool kLut, bool kBf16Tables, typename TY>
 szo_status launch_gemv(const szo_linear* const* plans, int n, const void* x, const void* x_mul, int64_t M,
-                       const float* const* S, void* const* y, cudaStream_t st, bool chained) {
+                       const float* const* S, void* const* y, cudaStream_t st, bool chained, const FusedNorm* norm) {
   auto kern = szo_linear_gemv_kernel<kLut, kBf16Tables, TY>;
   static bool configured[64] = {false};
   static std::mutex mu;
@@ -461,6 +527,12 @@ szo_status launch_gemv(const szo_linear* const* plans, int n, const void* x, con
   a.n = n;
   a.x = static_cast<const __nv_bfloat16*>(x);
   a.x_mul = static_cast<const __nv_bfloat16*>(x_mul);
+  if (norm != nullptr) {
+    SZO_REQUIRE(norm->h_in != nullptr && norm->h_out != nullptr && norm->h_in != norm->h_out && norm->gamma != nullptr &&
+                    x_mul == nullptr && plans[0]->K <= 8192,
+                SZO_ERR_INVALID_ARG, "fused norm: h_in, h_out (different buffers) and gamma are needed, K at most 8192");
+    a.norm = *norm;
+  }
   a.M = static_cast<int>(M);
   a.K = p->K;
   a.G = p->G;
@@ -472,7 +544,7 @@ szo_status launch_gemv(const szo_linear* const* plans, int n, const void* x, con
     ctas += static_cast<int>(ceil_div(q->N, kGvRows));
   }
   // persistent CTAs: as many as are resident at once (two per SM while the activations leave room)
-  const size_t smem = gemv_dyn_smem(p->K, M);
+  const size_t smem = gemv_dyn_smem(p->K, M, norm != nullptr);
   int sms = 148;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int per_sm = (2 * (smem + 9 * 1024) <= 227 * 1024) ? 2 : 1;
@@ -506,19 +578,20 @@ bool gemv_applies(const szo_linear* const* plans, int n, int64_t M) {
 }
 
 szo_status linear_fwd_gemv(const szo_linear* const* plans, int n, const void* x, const void* x_mul, int64_t M,
-                           const float* const* S_pert, void* const* y, int y_dtype, cudaStream_t st, bool chained) {
+                           const float* const* S_pert, void* const* y, int y_dtype, cudaStream_t st, bool chained,
+                           const FusedNorm* norm) {
   SZO_REQUIRE(gemv_applies(plans, n, M), SZO_ERR_UNSUPPORTED, "shapes not covered by the few-token kernel");
   const bool bf = plans[0]->sz_dtype == SZO_BF16;
   if (plans[0]->G == -1) {                    // (the plan's bf16 copy of the tables is read: the tables' own type does not matter)
-    if (y_dtype == SZO_F32) return launch_gemv<true, false, float>(plans, n, x, x_mul, M, S_pert, y, st, chained);
-    return launch_gemv<true, false, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st, chained);
+    if (y_dtype == SZO_F32) return launch_gemv<true, false, float>(plans, n, x, x_mul, M, S_pert, y, st, chained, norm);
+    return launch_gemv<true, false, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st, chained, norm);
   }
   if (y_dtype == SZO_F32) {
-    if (bf) return launch_gemv<false, true, float>(plans, n, x, x_mul, M, S_pert, y, st, chained);
-    return launch_gemv<false, false, float>(plans, n, x, x_mul, M, S_pert, y, st, chained);
+    if (bf) return launch_gemv<false, true, float>(plans, n, x, x_mul, M, S_pert, y, st, chained, norm);
+    return launch_gemv<false, false, float>(plans, n, x, x_mul, M, S_pert, y, st, chained, norm);
   }
-  if (bf) return launch_gemv<false, true, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st, chained);
-  return launch_gemv<false, false, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st, chained);
+  if (bf) return launch_gemv<false, true, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st, chained, norm);
+  return launch_gemv<false, false, __nv_bfloat16>(plans, n, x, x_mul, M, S_pert, y, st, chained, norm);
 }
 
 }  // namespace szo

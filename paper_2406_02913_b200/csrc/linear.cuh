@@ -46,10 +46,24 @@ bool skinny_applies(const szo_linear* p, int64_t M);
 // One to four tokens (gemm_gemv.cu): a CTA per 16 weight rows, no K-split between CTAs; same
 // arguments as linear_fwd_skinny_group, which hands such calls over.
 bool gemv_applies(const szo_linear* const* plans, int n, int64_t M);
-// chained: launched as part of a chain of dependent kernels (common.cuh); x, x_mul must then be the only
-// arguments that an earlier kernel of the stream writes.
+// chained: launched as part of a chain of dependent kernels (common.cuh); x, x_mul and the norm's inputs must
+// then be the only arguments that an earlier kernel of the stream writes.
+// norm != NULL (x is then unused): the activations are the normalised residual stream, formed while they are
+// staged, row m: v = h_in[m] + y_add[m] (y_add may be NULL), x[m] = RMSNorm or LayerNorm of v times gamma
+// (plus beta) rounded to bf16, the arithmetic of the model's add_norm_kernel; the first CTA also writes v to
+// h_out[m] (h_out must not be h_in: the other CTAs still read it).  K at most 8192.
+struct FusedNorm {
+  const float* h_in;
+  const __nv_bfloat16* y_add;
+  float* h_out;
+  const float* gamma;
+  const float* beta;
+  float eps;
+  bool layer_norm;
+};
 szo_status linear_fwd_gemv(const szo_linear* const* plans, int n, const void* x, const void* x_mul, int64_t M,
-                           const float* const* S_pert, void* const* y, int y_dtype, cudaStream_t st, bool chained = false);
+                           const float* const* S_pert, void* const* y, int y_dtype, cudaStream_t st, bool chained = false,
+                           const FusedNorm* norm = nullptr);
 // Up to three matrices that read the same activations in one launch (same K, G and table type);
 // x_mul != NULL: the activations are silu(x) * x_mul rounded to bf16, formed while they are staged.
 bool skinny_group_applies(const szo_linear* const* plans, int n, int64_t M);

@@ -905,6 +905,7 @@ struct szo_model {
   double* d_scalars = nullptr;
   int64_t last_launches = 0;
   void *kcache = nullptr, *vcache = nullptr;     // [n_layers][max_batch][max_seq][n_kv_heads * head_dim], act dtype
+  float* h2 = nullptr;                           // [2][d_model]: second copy of the residual stream of a one- or two-row token step
   szo_linear_t* decode_head = nullptr;           // LM head plan of the decode path when the loss path has none
   int32_t* d_pos = nullptr;                      // cached positions before the current decode call
   int32_t* dec_tokens = nullptr;                 // the call's tokens, at an address that a captured graph can keep
@@ -1293,6 +1294,30 @@ szo_status run_decode_t(szo_model* m, const int32_t* tokens, int B, int Tn, cons
     for (int i = 0; i < n; ++i) SZO_TRY(lin(layer, j0 + i, x, outs[i]));
     return SZO_OK;
   };
+  // One or two rows: residual add and norm are formed inside the projection that reads them (the
+  // residual stream alternates between m->h and m->h2: a layer reads h, writes h2 in its q/k/v launch,
+  // and h again in its gate/up launch).  SZO_DECODE_FUSED_NORM=0 keeps the separate kernel (A/B).
+  static const bool fuse_norm_on = [] {
+    const char* e = getenv("SZO_DECODE_FUSED_NORM");
+    return e == nullptr || e[0] != '0';
+  }();
+  bool fused_norms = false;                          // decided once: the shapes are those of every layer
+  if constexpr (sizeof(T) == 2) {
+    const szo_linear* const* p0 = m->plans.data();
+    fused_norms = streaming && fuse_norm_on && d <= 8192 && gemv_applies(p0, 3, M) && gemv_applies(p0 + 4, opt ? 1 : 2, M);
+  }
+  auto norm_lin_group = [&](int layer, int j0, int n, const float* h_in, const T* y_add, float* h_out, const float* gamma,
+                            const float* beta, void* const* outs) -> szo_status {
+    const int t0 = layer * m->n_lin + j0;
+    const szo_linear* plans[3];
+    const float* sv[3];
+    for (int i = 0; i < n; ++i) {
+      plans[i] = m->plans[t0 + i];
+      sv[i] = Sv + m->offsets[t0 + i];
+    }
+    const FusedNorm fn{h_in, reinterpret_cast<const __nv_bfloat16*>(y_add), h_out, gamma, beta, c.norm_eps, opt};
+    return linear_fwd_gemv(plans, n, nullptr, nullptr, M, sv, outs, act, st, chained, &fn);
+  };
   embed_kernel<<<static_cast<unsigned>(M), 128, 0, st>>>(tokens, static_cast<const __nv_bfloat16*>(m->top.embed),
                                                         static_cast<const __nv_bfloat16*>(m->top.pos), Tn, d, c.vocab, m->h, 0, pos_dev);
   count_launch();
@@ -1300,12 +1325,16 @@ szo_status run_decode_t(szo_model* m, const int32_t* tokens, int B, int Tn, cons
   const int64_t layer_cache = static_cast<int64_t>(c.max_batch) * Smax * dkv;
   for (int l = 0; l < c.n_layers; ++l) {
     const szo_layer_weights& L = m->layers[l];
-    SZO_CHECK_CUDA(launch_maybe_chained(add_norm_kernel<T, T>, dim3(static_cast<unsigned>(M)), dim3(256), 0, st, chained, m->h,
-                                        pending, L.attn_norm_g, L.attn_norm_b, d, c.norm_eps, opt, int64_t(1), int64_t(0), a));
-    count_launch();
     {
       void* const qkv[3] = {q, k, v};
-      SZO_TRY(lin_group(l, 0, 3, a, qkv));
+      if (fused_norms) {
+        SZO_TRY(norm_lin_group(l, 0, 3, m->h, pending, m->h2, L.attn_norm_g, L.attn_norm_b, qkv));
+      } else {
+        SZO_CHECK_CUDA(launch_maybe_chained(add_norm_kernel<T, T>, dim3(static_cast<unsigned>(M)), dim3(256), 0, st, chained, m->h,
+                                            pending, L.attn_norm_g, L.attn_norm_b, d, c.norm_eps, opt, int64_t(1), int64_t(0), a));
+        count_launch();
+        SZO_TRY(lin_group(l, 0, 3, a, qkv));
+      }
     }
     T* kc = static_cast<T*>(m->kcache) + l * layer_cache;
     T* vc = static_cast<T*>(m->vcache) + l * layer_cache;
@@ -1334,13 +1363,20 @@ szo_status run_decode_t(szo_model* m, const int32_t* tokens, int B, int Tn, cons
       void* const out[1] = {y};
       SZO_TRY(lin_group(l, 3, 1, o, out));
     }
-    SZO_CHECK_CUDA(launch_maybe_chained(add_norm_kernel<T, T>, dim3(static_cast<unsigned>(M)), dim3(256), 0, st, chained, m->h,
-                                        static_cast<const T*>(y), L.mlp_norm_g, L.mlp_norm_b, d, c.norm_eps, opt, int64_t(1),
-                                        int64_t(0), a));
-    count_launch();
-    if (!opt) {
+    {
       void* const gu[2] = {gate, up};
-      SZO_TRY(lin_group(l, 4, 2, a, gu));
+      if (fused_norms) {
+        SZO_TRY(norm_lin_group(l, 4, opt ? 1 : 2, m->h2, y, m->h, L.mlp_norm_g, L.mlp_norm_b, gu));
+      } else {
+        SZO_CHECK_CUDA(launch_maybe_chained(add_norm_kernel<T, T>, dim3(static_cast<unsigned>(M)), dim3(256), 0, st, chained, m->h,
+                                            static_cast<const T*>(y), L.mlp_norm_g, L.mlp_norm_b, d, c.norm_eps, opt, int64_t(1),
+                                            int64_t(0), a));
+        count_launch();
+        if (opt) SZO_TRY(lin(l, 4, a, gate));
+        else SZO_TRY(lin_group(l, 4, 2, a, gu));
+      }
+    }
+    if (!opt) {
       const szo_linear* down = m->plans[l * m->n_lin + 6];
       if (streaming && few_token_applies(&down, 1, M)) {
         // silu(gate) * up is formed while the down projection stages its activations
@@ -1353,7 +1389,6 @@ szo_status run_decode_t(szo_model* m, const int32_t* tokens, int B, int Tn, cons
         SZO_TRY(lin(l, 6, gate, y));
       }
     } else {
-      SZO_TRY(lin(l, 4, a, gate));
       relu_kernel<T><<<blocks_for(M * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, M * ff);
       count_launch();
       SZO_TRY(lin(l, 5, gate, y));
@@ -1782,6 +1817,7 @@ szo_status szo_model_enable_decode(szo_model_t* m, void* stream) {
   SZO_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->kcache), bytes));
   SZO_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->vcache), bytes));
   SZO_TRY(dev_alloc(m, &m->d_pos, sizeof(int32_t)));
+  SZO_TRY(dev_alloc(m, &m->h2, 2 * static_cast<size_t>(c.d_model) * sizeof(float)));
   SZO_TRY(dev_alloc(m, &m->dec_tokens, static_cast<size_t>(m->Mmax) * sizeof(int32_t)));
   SZO_TRY(dev_alloc(m, &m->dec_logits, static_cast<size_t>(c.max_batch) * c.vocab * sizeof(float)));
   SZO_REQUIRE(device_status_word() != nullptr, SZO_ERR_CUDA, "no device status word");    // allocated outside any capture

@@ -372,14 +372,16 @@ def test_one_full_width_layer_against_the_oracle(B):
             m.close()
 
 
-def test_token_steps_of_one_full_width_layer_against_the_oracle(B):
-    """Token generation on one decoder layer at the Llama-2-7B width (the few-token kernels at the
-    widths they are built for: q/k/v and gate/up in one launch each, SiLU gating formed inside the
-    down projection, rotation + cache append + attention in one kernel): a prompt of 3 tokens, then
-    single tokens, for 2 sequences and for 1, against the oracle's incremental decode."""
+@pytest.mark.parametrize("name", ["llama2_7b", "opt_13b"])
+def test_token_steps_of_one_full_width_layer_against_the_oracle(B, name):
+    """Token generation on one decoder layer at the Llama-2-7B and OPT-13B widths (the few-token kernels
+    at the widths they are built for: q/k/v and gate/up in one launch each, residual add and RMSNorm /
+    LayerNorm formed inside those launches, SiLU gating inside the down projection, rotation + cache
+    append + attention in one kernel): a prompt of 3 tokens, then single tokens, for 2 sequences and
+    for 1, against the oracle's incremental decode."""
     from oracle import model_oracle as mo
     from tests.fixtures import DecoderFixture
-    fx = DecoderFixture("llama2_7b", seed=9, mask="random", B=2, S=16, n_layers=1)
+    fx = DecoderFixture(name, seed=9, mask="random", B=2, S=16, n_layers=1)
     om = fx.oracle_model()
     S_np = om.S + np.float32(1e-3)
     lin_W = om.lin_W(S_np)
