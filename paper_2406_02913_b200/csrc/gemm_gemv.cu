@@ -98,8 +98,9 @@ __device__ __forceinline__ float2 gv_sz_f32(float2 p) {
     return p;
 }
 
-// silu(g) * u of eight bf16 pairs, each product rounded to bf16 (the arithmetic of the model's own
-// SiLU-gating kernel, so that either route gives the same bits)
+// silu(g) * u of eight bf16 pairs, each product rounded to bf16.  Every CTA forms all K products, so
+// the fast exponential and division are used (relative error near 2^-21, far below the bf16 rounding
+// of the result; the model's own SiLU-gating kernel uses the exact ones)
 __device__ __forceinline__ uint4 gv_silu_mul(uint4 g, uint4 u) {
   const uint32_t gw[4] = {g.x, g.y, g.z, g.w}, uw[4] = {u.x, u.y, u.z, u.w};
   uint32_t o[4];
@@ -107,7 +108,7 @@ __device__ __forceinline__ uint4 gv_silu_mul(uint4 g, uint4 u) {
   for (int i = 0; i < 4; ++i) {
     const float g0 = __uint_as_float(gw[i] << 16), g1 = __uint_as_float(gw[i] & 0xFFFF0000u);
     const float u0 = __uint_as_float(uw[i] << 16), u1 = __uint_as_float(uw[i] & 0xFFFF0000u);
-    const __nv_bfloat162 r = __floats2bfloat162_rn(g0 / (1.0f + expf(-g0)) * u0, g1 / (1.0f + expf(-g1)) * u1);
+    const __nv_bfloat162 r = __floats2bfloat162_rn(__fdividef(g0, 1.0f + __expf(-g0)) * u0, __fdividef(g1, 1.0f + __expf(-g1)) * u1);
     o[i] = *reinterpret_cast<const uint32_t*>(&r);
   }
   return make_uint4(o[0], o[1], o[2], o[3]);
