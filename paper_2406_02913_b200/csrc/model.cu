@@ -447,91 +447,142 @@ attn_decode_kernel(const T* __restrict__ q, const T* __restrict__ kc, const T* _
 // tokens 0 .. t from k_new / v_new (rotating each key at its position) and the older ones from the
 // cache; the first query head of every key/value head also stores the rotated key and the value of
 // token t in the cache.  No block reads a cache row that this launch writes.  Rotated values are
-// rounded to T exactly where rope_kernel and the cache would round them: same bits as the three
-// separate kernels.
+// rounded to T exactly where rope_kernel and the cache would round them.
+// Sixteen key streams per block: a quarter warp (8 lanes) takes the keys n = s, s + 16, ... of stream
+// s; a lane holds HD / 8 contiguous elements (16- or 32-byte loads), so a key costs three shuffles
+// for the dot product, and four keys are in flight per warp.  Every stream keeps its own online
+// softmax state; the streams are merged at the end in a fixed order (quarters of a warp by two
+// shuffle steps, then the four warps through shared memory).
 template <typename T, int HD>
 __global__ void __launch_bounds__(128)
 attn_decode_fused_kernel(const T* __restrict__ q, const T* __restrict__ k_new, const T* __restrict__ v_new,
                          T* __restrict__ kc, T* __restrict__ vc, T* __restrict__ o, const float2* __restrict__ rope_tab,
                          int Tn, const int32_t* __restrict__ pos_dev, int64_t Smax, int H, int Hkv, float scale) {
-  constexpr int E = HD / 32, half = HD / 2;
+  constexpr int E = HD / 8, half = HD / 2;            // elements per lane; a lane's rotation partner is lane ^ 4
   __shared__ float part_acc[4][HD];
   __shared__ float part_m[4], part_l[4];
   chain_release();
   chain_wait();
   const int pos0 = *pos_dev;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int ql = lane & 7, stream = w * 4 + (lane >> 3);
   const int t = blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
   const int hk = hq / (H / Hkv);
   const int64_t dq = static_cast<int64_t>(H) * HD, dk = static_cast<int64_t>(Hkv) * HD;
-  // element lane + 32 j pairs with lane + 32 (j + E/2): both in this lane
-  auto rotate = [&](float (&x)[E], int pos) {
-    if (rope_tab == nullptr) return;
+  const int e0 = ql * E;                              // first element of this lane
+  auto load = [&](const T* p, float (&x)[E]) {        // E contiguous elements from p + e0
+    constexpr int kN = 16 / static_cast<int>(sizeof(T));
 #pragma unroll
-    for (int j = 0; j < E / 2; ++j) {
-      const float2 cs = rope_tab[static_cast<int64_t>(pos) * half + lane + 32 * j];
-      const float a0 = x[j], b0 = x[j + E / 2];
-      x[j] = to_f32<T>(from_f32<T>(a0 * cs.x - b0 * cs.y));
-      x[j + E / 2] = to_f32<T>(from_f32<T>(b0 * cs.x + a0 * cs.y));
+    for (int i = 0; i < E; i += kN) {
+      const Vec16<T> v = load16(p + e0 + i);
+#pragma unroll
+      for (int j = 0; j < kN; ++j) x[i + j] = to_f32<T>(v.v[j]);
     }
   };
-  const T* qp = q + (static_cast<int64_t>(b) * Tn + t) * dq + hq * HD;
-  float qr[E], acc[E];
+  auto store = [&](T* p, const float (&x)[E]) {
+    constexpr int kN = 16 / static_cast<int>(sizeof(T));
 #pragma unroll
-  for (int j = 0; j < E; ++j) qr[j] = to_f32<T>(qp[lane + 32 * j]);
+    for (int i = 0; i < E; i += kN) {
+      Vec16<T> v;
+#pragma unroll
+      for (int j = 0; j < kN; ++j) v.v[j] = from_f32<T>(x[i + j]);
+      store16(p + e0 + i, v);
+    }
+  };
+  // element e < half pairs with e + half, held by lane ^ 4 at the same index
+  auto rotate = [&](float (&x)[E], int pos) {
+    if (rope_tab == nullptr) return;
+    const bool low = ql < 4;
+    const float2* cs = rope_tab + static_cast<int64_t>(pos) * half + (low ? e0 : e0 - half);
+#pragma unroll
+    for (int i = 0; i < E; ++i) {
+      const float other = __shfl_xor_sync(0xffffffffu, x[i], 4);
+      const float2 c = cs[i];
+      // low half: a cos - b sin with (a, b) = (x, other); high half: b cos + a sin with (a, b) = (other, x)
+      x[i] = to_f32<T>(from_f32<T>(low ? x[i] * c.x - other * c.y : x[i] * c.x + other * c.y));
+    }
+  };
+  float qr[E], acc[E];
+  load(q + (static_cast<int64_t>(b) * Tn + t) * dq + hq * HD, qr);
   rotate(qr, pos0 + t);
 #pragma unroll
-  for (int j = 0; j < E; ++j) {
-    qr[j] *= scale;
-    acc[j] = 0.f;
+  for (int i = 0; i < E; ++i) {
+    qr[i] *= scale;
+    acc[i] = 0.f;
   }
   const T* knb = k_new + static_cast<int64_t>(b) * Tn * dk + hk * HD;
   const T* vnb = v_new + static_cast<int64_t>(b) * Tn * dk + hk * HD;
   T* kb = kc + static_cast<int64_t>(b) * Smax * dk + hk * HD;
   T* vb = vc + static_cast<int64_t>(b) * Smax * dk + hk * HD;
-  if (w == 3 && hq % (H / Hkv) == 0) {          // (the warp with the fewest keys when few are cached)
-    float kv[E];
-#pragma unroll
-    for (int j = 0; j < E; ++j) kv[j] = to_f32<T>(knb[t * dk + lane + 32 * j]);
+  if (w == 3 && hq % (H / Hkv) == 0) {                // (the warp with the fewest keys when few are cached)
+    float kv[E], vv[E];
+    load(knb + t * dk, kv);
+    load(vnb + t * dk, vv);
     rotate(kv, pos0 + t);
-#pragma unroll
-    for (int j = 0; j < E; ++j) {
-      kb[(pos0 + t) * dk + lane + 32 * j] = from_f32<T>(kv[j]);
-      vb[(pos0 + t) * dk + lane + 32 * j] = vnb[t * dk + lane + 32 * j];
+    if (lane < 8) {
+      store(kb + (pos0 + t) * dk, kv);
+      store(vb + (pos0 + t) * dk, vv);
     }
   }
   float mx = -INFINITY, l = 0.f;
-  for (int n = w; n <= pos0 + t; n += 4) {
-    const bool fresh = n >= pos0;
-    const T* kp = fresh ? knb + (n - pos0) * dk : kb + n * dk;
-    const T* vp = fresh ? vnb + (n - pos0) * dk : vb + n * dk;
+  const int last = pos0 + t;
+  for (int n0 = 0; n0 <= last; n0 += 16) {            // (uniform trip count: the rotation shuffles need whole warps)
+    const int n = n0 + stream;
+    const bool live = n <= last;
+    const int nn = live ? n : last;
+    const bool fresh = nn >= pos0;
     float kv[E], vv[E];
+    load(fresh ? knb + (nn - pos0) * dk : kb + nn * dk, kv);
+    load(fresh ? vnb + (nn - pos0) * dk : vb + nn * dk, vv);
+    if (__any_sync(0xffffffffu, fresh)) {
+      float kr[E];
 #pragma unroll
-    for (int j = 0; j < E; ++j) {
-      kv[j] = to_f32<T>(kp[lane + 32 * j]);
-      vv[j] = to_f32<T>(vp[lane + 32 * j]);
+      for (int i = 0; i < E; ++i) kr[i] = kv[i];
+      rotate(kr, nn);
+      if (fresh) {
+#pragma unroll
+        for (int i = 0; i < E; ++i) kv[i] = kr[i];
+      }
     }
-    if (fresh) rotate(kv, n);
     float dot = 0.f;
 #pragma unroll
-    for (int j = 0; j < E; ++j) dot = fmaf(qr[j], kv[j], dot);
+    for (int i = 0; i < E; ++i) dot = fmaf(qr[i], kv[i], dot);
 #pragma unroll
-    for (int off = 16; off; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
-    const float mn = fmaxf(mx, dot);
-    const float corr = expf(mx - mn), p = expf(dot - mn);
-    l = l * corr + p;
+    for (int off = 4; off; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+    if (live) {
+      const float mn = fmaxf(mx, dot);
+      const float corr = expf(mx - mn), p = expf(dot - mn);
+      l = l * corr + p;
 #pragma unroll
-    for (int j = 0; j < E; ++j) acc[j] = fmaf(p, vv[j], acc[j] * corr);
-    mx = mn;
+      for (int i = 0; i < E; ++i) acc[i] = fmaf(p, vv[i], acc[i] * corr);
+      mx = mn;
+    }
   }
+  // merge the four streams of a warp (quarters 0+1 and 2+3, then the two halves), lower stream first
 #pragma unroll
-  for (int j = 0; j < E; ++j) part_acc[w][lane + 32 * j] = acc[j];
-  if (lane == 0) {
-    part_m[w] = mx;
-    part_l[w] = l;
+  for (int off = 8; off <= 16; off <<= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, mx, off), ol = __shfl_xor_sync(0xffffffffu, l, off);
+    const float M2 = fmaxf(mx, om);
+    const float fs = mx == -INFINITY ? 0.f : expf(mx - M2), fo = om == -INFINITY ? 0.f : expf(om - M2);
+    const bool first = (lane & off) == 0;             // this lane's state is the lower stream's
+#pragma unroll
+    for (int i = 0; i < E; ++i) {
+      const float oa = __shfl_xor_sync(0xffffffffu, acc[i], off);
+      acc[i] = first ? fmaf(oa, fo, acc[i] * fs) : fmaf(acc[i], fs, oa * fo);
+    }
+    l = first ? fmaf(ol, fo, l * fs) : fmaf(l, fs, ol * fo);
+    mx = M2;
+  }
+  if (lane < 8) {
+#pragma unroll
+    for (int i = 0; i < E; ++i) part_acc[w][e0 + i] = acc[i];
+    if (lane == 0) {
+      part_m[w] = mx;
+      part_l[w] = l;
+    }
   }
   __syncthreads();
-  if (w == 0) {
+  if (w == 0 && lane < 8) {
     float M = -INFINITY;
 #pragma unroll
     for (int i = 0; i < 4; ++i) M = fmaxf(M, part_m[i]);
@@ -540,15 +591,15 @@ attn_decode_fused_kernel(const T* __restrict__ q, const T* __restrict__ k_new, c
     for (int j = 0; j < E; ++j) out[j] = 0.f;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const float f = part_m[i] == -INFINITY ? 0.f : expf(part_m[i] - M);
+      const float f = part_m[i] == -INFINITY ? 0.f : expf(part_m[i] - M);     // a warp without keys contributes nothing
       L += part_l[i] * f;
 #pragma unroll
-      for (int j = 0; j < E; ++j) out[j] = fmaf(part_acc[i][lane + 32 * j], f, out[j]);
+      for (int j = 0; j < E; ++j) out[j] = fmaf(part_acc[i][e0 + j], f, out[j]);
     }
-    T* op = o + (static_cast<int64_t>(b) * Tn + t) * dq + hq * HD;
     const float inv = 1.0f / L;
 #pragma unroll
-    for (int j = 0; j < E; ++j) op[lane + 32 * j] = from_f32<T>(out[j] * inv);
+    for (int j = 0; j < E; ++j) out[j] *= inv;
+    store(o + (static_cast<int64_t>(b) * Tn + t) * dq + hq * HD, out);
   }
 }
 
