@@ -333,6 +333,19 @@ def replay(S0, gidx, seed: int, log, eps, lr) -> np.ndarray:
     return S
 
 
+def zo_sgd_step_16(loss, S_bits, fmt: str, gidx, seed: int, step: int, eps, lr):
+    """The same step with the sparse values STORED as 16-bit floats (Section 3.5 keeps w_sparse in 16
+    bits; fmt 'bf16' or 'f16').  The paper does not say where the arithmetic of a step happens for
+    such storage; the reading taken: the stored values are widened to fp32 (exact), the step runs in
+    fp32 as zo_sgd_step (perturbations never rounded to 16 bits), and the updated values are rounded
+    to the storage format once, to nearest even.  An update smaller than half a unit in the last
+    place of a stored value therefore leaves it unchanged.  Returns (bits_new, f+, f-, g)."""
+    S = bits16_to_f32(S_bits, fmt)
+    S, f_plus, f_minus, g = zo_sgd_step(loss, S, gidx, seed, step, eps, lr)
+    bits, _ = round_to_16(S, fmt)
+    return bits, f_plus, f_minus, g
+
+
 def zo_sgd_step(loss, S, gidx, seed: int, step: int, eps, lr):
     """One sensitive-sparse ZO-SGD step on the k trainable values S for a loss callable
     loss(S) -> float, in the in-place order of the seed trick (Section 2.1):

@@ -495,3 +495,41 @@ def test_update_scale_and_projected_gradient():
     assert np.isclose(g, 0.25 / (2 * float(eps)), rtol=1e-15)
     sc = so.zo_update_scale(2.5, 2.25, eps, 1e-5)
     assert sc == np.float32(-(float(np.float32(1e-5)) * g)) and sc < 0
+
+
+@pytest.mark.parametrize("fmt", ["f16", "bf16"])
+def test_step_with_16_bit_sparse_storage(fmt):
+    """Section 3.5 (w_sparse kept in 16 bits), reading: fp32 step on the widened values, one rounding to
+    the storage format.  Pinned by what does not involve the oracle's own rounding code: the result
+    of the fp32 step cast by a library (numpy's float16, torch's bfloat16), representability, the
+    half-ulp bound, and the two regimes an update can fall in (lost below half an ulp, visible above)."""
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(5)
+    k = 4096
+    gidx = np.sort(rng.choice(10 ** 6, k, replace=False)).astype(np.int64)
+    a = rng.normal(0, 1, k)
+    loss = lambda S: float(np.dot(a, S.astype(np.float64)))          # linear: g = z.a up to rounding
+    S0 = rng.normal(0, 0.02, k).astype(np.float32)
+    bits0, S0r = so.round_to_16(S0, fmt)
+    for lr in (1e-9, 1e-3):
+        bits1, fp, fm, g = so.zo_sgd_step_16(loss, bits0, fmt, gidx, 77, 3, 1e-3, lr)
+        S32, fp2, fm2, g2 = so.zo_sgd_step(loss, S0r, gidx, 77, 3, 1e-3, lr)
+        assert (fp, fm, g) == (fp2, fm2, g2)                         # the losses see fp32 perturbations of the widened values
+        # a library's cast of the fp32 result
+        if fmt == "f16":
+            lib_bits = S32.astype(np.float16).view(np.uint16)
+        else:
+            lib_bits = torch.from_numpy(S32).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+        assert np.array_equal(bits1, lib_bits)
+        S1 = so.bits16_to_f32(bits1, fmt)
+        assert np.array_equal(so.round_to_16(S1, fmt)[0], bits1)     # representable
+        ulp = np.abs(so.bits16_to_f32(bits1 + np.uint16(1), fmt) - S1)
+        assert np.all(np.abs(S1.astype(np.float64) - S32.astype(np.float64)) <= 0.5 * ulp.astype(np.float64) * (1 + 1e-12))
+        z = so.gaussian(77, 3, gidx)
+        upd = np.abs(np.float64(lr) * g * z)
+        if lr == 1e-9:
+            small = upd < 0.25 * ulp                                  # (all but stored values next to zero)
+            assert small.mean() > 0.99 and np.array_equal(bits1[small], bits0[small])   # such an update is lost
+        else:
+            moved = bits1 != bits0
+            assert moved.mean() > 0.9 and np.all(moved[upd > ulp])                # an update above one ulp always shows
