@@ -156,6 +156,16 @@ szo_status szo_update(float* S, const int64_t* idx, int64_t k, int64_t idx_base,
                       uint64_t step, float lr, const double* f_plus_dev, const double* f_minus_dev,
                       float eps, void* stream);
 
+/* ---- Sparse values stored in 16 bits (Section 3.5: w_sparse is kept in 16 bits).  The paper does not say
+ * where a step's arithmetic happens for such storage; this library widens the stored values to fp32
+ * (exact), runs the step in fp32 (perturbations are never rounded to 16 bits) and rounds the updated
+ * values to the storage format once, to nearest even.
+ * szo_round_sparse16: S[j] = widen(RN_dt(S[j])) in place for j in [0, k), and S16_out[j] = RN_dt(S[j]) when
+ * S16_out != NULL (device, k 16-bit values, caller-owned).  dt: SZO_BF16 or SZO_F16.  Call it after
+ * szo_update to keep S representable in the storage format; values beyond the format's range become
+ * infinities as IEEE rounding says.  Errors: NULL S with k > 0, dt == SZO_F32 -> SZO_ERR_INVALID_ARG. */
+szo_status szo_round_sparse16(float* S, int64_t k, szo_dtype dt, void* S16_out, void* stream);
+
 /* ---- Replay of a run from its log (Section 2.1, the seed trick: z_t is a function of (seed, step_t), so
  * the scalars g_t are a complete record of what a run did to the sparse values:
  * S_T = S_0 - sum_t lr g_t z_t; a checkpoint is S at some step plus the (step, g) pairs since).
@@ -336,6 +346,12 @@ szo_status szo_model_zo_losses(szo_model_t* m, const int32_t* tokens, const int3
                                void* stream);
 szo_status szo_model_zo_apply(szo_model_t* m, float eps, float lr, const double* sums_dev, double* f_plus_dev,
                               double* f_minus_dev, double* g_dev, void* stream);
+/* Storage format of the model's sparse values (see szo_round_sparse16): with dt = SZO_BF16 or SZO_F16 every
+ * update of szo_model_zo_step, szo_model_zo_step_n, szo_model_zo_apply and szo_model_zo_step_host is followed
+ * by one rounding of S to that format (S stays an fp32 array holding representable values; S16_out, when not
+ * NULL, is a caller-owned device array of k_total 16-bit values that receives the stored form after every
+ * update).  The call itself rounds the current S once.  dt = SZO_F32 (the default) switches it off. */
+szo_status szo_model_set_sparse_storage(szo_model_t* m, szo_dtype dt, void* S16_out, void* stream);
 /* Same step through HOST buffers: copies tokens (and labels, cand) to the device, runs the step
  * and copies (f+, f-, g) back into out3_host[3]; synchronises the stream. */
 szo_status szo_model_zo_step_host(szo_model_t* m, const int32_t* tokens_host,

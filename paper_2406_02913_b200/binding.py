@@ -78,6 +78,8 @@ _SIGS = {
     "szo_projected_gradient": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p]),
     "szo_update": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_uint64, C.c_uint64,
                                C.c_float, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]),
+    "szo_round_sparse16": (C.c_int32, [C.c_void_p, C.c_int64, C.c_int, C.c_void_p, C.c_void_p]),
+    "szo_model_set_sparse_storage": (C.c_int32, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]),
     "szo_replay": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_uint64, C.POINTER(C.c_uint64),
                                C.POINTER(C.c_double), C.c_int64, C.c_float, C.c_float, C.c_void_p]),
     "szo_linear_create": (C.c_int32, [C.POINTER(C.c_void_p), C.c_int64, C.c_int64, C.c_int32,
@@ -244,6 +246,12 @@ def szo_replay(S, idx, idx_base: int, seed: int, log, eps: float, lr: float):
     _check(lib().szo_replay(_ptr(S), _ptr(idx), idx.numel(), idx_base, seed, steps, gs, n, eps, lr, _stream()))
 
 
+def szo_round_sparse16(S, fmt: str, out=None):
+    """Rounds S (fp32 CUDA tensor) in place to values representable in 'bf16' or 'f16'; `out` (16-bit tensor of
+    the same length) receives the stored form (szo_round_sparse16)."""
+    _check(lib().szo_round_sparse16(_ptr(S), S.numel(), SZO_BF16 if fmt == "bf16" else SZO_F16, _ptr(out), _stream()))
+
+
 # ------------------------------------------------------------------------------ linear layer
 class Linear:
     """Plan for one decomposed linear (szo_linear_create / szo_linear_fwd)."""
@@ -396,6 +404,13 @@ class Model:
                                        eps, lr, sc[0:1].data_ptr(), sc[1:2].data_ptr(),
                                        sc[2:3].data_ptr(), _stream()))
         return sc[:3]
+
+    def set_sparse_storage(self, fmt, out=None):
+        """Sparse values stored in 'bf16' or 'f16' (None or 'f32': off): every update is followed by one rounding to
+        the format; `out` (16-bit tensor [k_total]) mirrors the stored form (szo_model_set_sparse_storage)."""
+        dt = {None: SZO_F32, "f32": SZO_F32, "bf16": SZO_BF16, "f16": SZO_F16}[fmt]
+        self._keep_s16 = out
+        _check(lib().szo_model_set_sparse_storage(self.h, dt, _ptr(out), _stream()))
 
     def zo_step_n(self, tokens, seed, step, n, eps, lr, labels=None, cand=None) -> torch.Tensor:
         """n-sample SPSA step; returns the device tensor [3, n] of (f+_i, f-_i, g_i) (fp64)."""

@@ -957,6 +957,8 @@ struct szo_model {
   int64_t last_launches = 0;
   void *kcache = nullptr, *vcache = nullptr;     // [n_layers][max_batch][max_seq][n_kv_heads * head_dim], act dtype
   float* h2 = nullptr;                           // [2][d_model]: second copy of the residual stream of a one- or two-row token step
+  int sparse_dt = SZO_F32;                       // storage format of the sparse values (szo_model_set_sparse_storage)
+  void* S16_out = nullptr;                       // caller-owned mirror of the stored form, or NULL
   szo_linear_t* decode_head = nullptr;           // LM head plan of the decode path when the loss path has none
   int32_t* d_pos = nullptr;                      // cached positions before the current decode call
   int32_t* dec_tokens = nullptr;                 // the call's tokens, at an address that a captured graph can keep
@@ -1759,11 +1761,18 @@ static szo_status zo_losses_impl(szo_model* m, const int32_t* tokens, const int3
 }
 
 // Second half: g from the two losses, then S -= lr g z with the kept z.
+// Sparse values kept in 16 bits (Section 3.5): one rounding to the storage format after a step's update
+static szo_status store_sparse(szo_model* m, cudaStream_t st) {
+  if (m->sparse_dt == SZO_F32) return SZO_OK;
+  return szo_round_sparse16(m->S_all, m->k_total, static_cast<szo_dtype>(m->sparse_dt), m->S16_out, st);
+}
+
 static szo_status zo_apply_impl(szo_model* m, float eps, float lr, const double* f_plus_dev, const double* f_minus_dev,
                                 double* g_dev, cudaStream_t st) {
   SZO_TRY(szo_projected_gradient(f_plus_dev, f_minus_dev, eps, g_dev, st));
   ScaleArg su{0.f, lr, eps, f_plus_dev, f_minus_dev};
-  return launch_sparse_axpy_kept(m->S_all, m->S_all, m->zkept, m->k_total, su, st);
+  SZO_TRY(launch_sparse_axpy_kept(m->S_all, m->S_all, m->zkept, m->k_total, su, st));
+  return store_sparse(m, st);
 }
 
 szo_status szo_model_zo_step(szo_model_t* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand,
@@ -1802,9 +1811,18 @@ szo_status szo_model_zo_step_n(szo_model_t* m, const int32_t* tokens, const int3
     ScaleArg su{0.f, lr_n, eps, f_plus_dev + i, f_minus_dev + i};
     SZO_TRY(launch_sparse_axpy(m->S_all, m->S_all, m->gidx, m->k_total, 0, seed, c, su, st));
   }
+  SZO_TRY(store_sparse(m, st));
   m->z_valid = false;
   m->last_launches = g_launch_count - before;
   return SZO_OK;
+}
+
+szo_status szo_model_set_sparse_storage(szo_model_t* m, szo_dtype dt, void* S16_out, void* stream) {
+  SZO_REQUIRE(m != nullptr, SZO_ERR_INVALID_ARG, "model is NULL");
+  SZO_REQUIRE(dt == SZO_F32 || dt == SZO_BF16 || dt == SZO_F16, SZO_ERR_INVALID_ARG, "unknown storage format");
+  m->sparse_dt = dt;
+  m->S16_out = dt == SZO_F32 ? nullptr : S16_out;
+  return store_sparse(m, static_cast<cudaStream_t>(stream));
 }
 
 szo_status szo_model_zo_losses(szo_model_t* m, const int32_t* tokens, const int32_t* labels, const int32_t* cand,

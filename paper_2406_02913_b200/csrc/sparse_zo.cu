@@ -4,6 +4,8 @@
 // Section 3.4 decomposition makes them a contiguous fp32 vector S.  z is regenerated from a
 // counter-based generator (Section 2.1 seed trick) keyed by (seed, step, global parameter index):
 // Philox4x32-10 (Salmon et al., SC'11) followed by the Box-Muller cosine branch.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace szo {
@@ -230,6 +232,21 @@ szo_status launch_sparse_axpy(const float* S_in, float* S_out, const int64_t* id
 
 }  // namespace szo
 
+namespace szo {
+// Sparse values stored in 16 bits (Section 3.5): S[j] = widen(RN_T16(S[j])), optionally the stored form too
+template <typename T16>
+__global__ void round_sparse16_kernel(float* __restrict__ S, int64_t k, T16* __restrict__ out) {
+  const int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (j >= k) return;
+  T16 h;
+  if constexpr (sizeof(T16) == sizeof(__half) && !std::is_same<T16, __nv_bfloat16>::value) h = __float2half_rn(S[j]);
+  else h = __float2bfloat16_rn(S[j]);
+  if (out != nullptr) out[j] = h;
+  if constexpr (std::is_same<T16, __nv_bfloat16>::value) S[j] = __bfloat162float(h);
+  else S[j] = __half2float(h);
+}
+}  // namespace szo
+
 extern "C" {
 
 szo_status szo_perturb(const float* S_in, float* S_out, const int64_t* idx, int64_t k,
@@ -315,6 +332,19 @@ szo_status szo_replay(float* S, const int64_t* idx, int64_t k, int64_t idx_base,
     szo::ScaleArg su{-static_cast<float>(static_cast<double>(lr) * g_host[t]), 0.f, 0.f, nullptr, nullptr};
     SZO_TRY(szo::launch_sparse_axpy(S, S, idx, k, idx_base, seed, steps_host[t], su, st));
   }
+  return SZO_OK;
+}
+
+szo_status szo_round_sparse16(float* S, int64_t k, szo_dtype dt, void* S16_out, void* stream) {
+  SZO_REQUIRE(k >= 0 && (k == 0 || S != nullptr), SZO_ERR_INVALID_ARG, "NULL S or k < 0");
+  SZO_REQUIRE(dt == SZO_BF16 || dt == SZO_F16, SZO_ERR_INVALID_ARG, "the storage format must be SZO_BF16 or SZO_F16");
+  if (k == 0) return SZO_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const unsigned blocks = static_cast<unsigned>(szo::ceil_div(k, 256));
+  if (dt == SZO_BF16) szo::round_sparse16_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(S, k, static_cast<__nv_bfloat16*>(S16_out));
+  else szo::round_sparse16_kernel<__half><<<blocks, 256, 0, st>>>(S, k, static_cast<__half*>(S16_out));
+  szo::count_launch();
+  SZO_CHECK_LAUNCH("round_sparse16_kernel");
   return SZO_OK;
 }
 

@@ -328,3 +328,49 @@ def test_n_sample_spsa_step_matches_the_oracle(B, tiny):
     assert tuple(a) == tuple(b) and torch.equal(S1, S2)
     for mm in (m, m1, m2):
         mm.close()
+
+
+@pytest.mark.parametrize("fmt", ["f16", "bf16"])
+def test_sparse_values_stored_in_16_bits(B, tiny, fmt):
+    """Section 3.5 (w_sparse in 16 bits): szo_round_sparse16 against the oracle's rounding bit for bit, and three
+    steps of a model whose sparse values are stored in the format: after every step S holds representable values,
+    the mirror holds their bits, and S agrees with the oracle's zo_sgd_step_16 to the difference of the two fp32
+    updates (lr |z| times the tolerance on g) plus the one unit in the last place by which values on different
+    sides of a rounding boundary part."""
+    fx = tiny
+    x = torch.from_numpy(wl.rng(3, wl.PURPOSE_WEIGHTS, 1).normal(0, 0.05, 100003).astype(np.float32)).cuda()
+    x[:4] = torch.tensor([0.0, -0.0, 65519.9, 1e-9], device="cuda")
+    ref_bits, ref_vals = so.round_to_16(x.cpu().numpy(), fmt)
+    dt16 = torch.float16 if fmt == "f16" else torch.bfloat16
+    mirror = torch.zeros(x.numel(), dtype=dt16, device="cuda")
+    B.szo_round_sparse16(x, fmt, mirror)
+    assert np.array_equal(x.cpu().numpy().view(np.uint32), ref_vals.view(np.uint32))
+    assert np.array_equal(mirror.cpu().view(torch.int16).numpy().view(np.uint16), ref_bits)
+
+    toks = fx.batch(0)
+    eps, lr = 1e-3, 3e-3
+    om = fx.oracle_model()
+    m, S, _ = build_gpu(B, fx, B.SZO_F32, B.MODE_FP32_VALIDATE)
+    S16 = torch.zeros(S.numel(), dtype=dt16, device="cuda")
+    m.set_sparse_storage(fmt, S16)
+    bits = so.round_to_16(om.S, fmt)[0]
+    assert np.array_equal(S16.cpu().view(torch.int16).numpy().view(np.uint16), bits)       # the call rounds the current S
+    bits0 = bits.copy()
+    for step in range(3):
+        bits, fp, fm, g = so.zo_sgd_step_16(lambda S_: om.loss(S_, toks), bits, fmt, om.gidx, 1234, step, eps, lr)
+        out = m.zo_step(torch.from_numpy(toks).cuda(), 1234, step, eps, lr).cpu().numpy()
+        assert abs(out[0] - fp) <= 2e-6 * abs(fp) and abs(out[2] - g) <= g_tol(g, fp, eps)
+        got = S.cpu().numpy()
+        got_bits = S16.cpu().view(torch.int16).numpy().view(np.uint16)
+        assert np.array_equal(so.round_to_16(got, fmt)[1].view(np.uint32), got.view(np.uint32))     # representable
+        assert np.array_equal(so.round_to_16(got, fmt)[0], got_bits)                                 # the mirror
+        ref = so.bits16_to_f32(bits, fmt)
+        ulp = np.abs(so.bits16_to_f32(bits + np.uint16(1), fmt) - ref)
+        slack = lr * 6.0 * g_tol(g, fp, eps) + 2e-7              # |z| < 6; the in-place order's own ulps of fp32
+        excess = np.abs(got.astype(np.float64) - ref) - ulp - slack
+        assert excess.max() <= 0, (step, excess.max(), int(np.argmax(excess)))
+        assert np.mean(got_bits == bits) > 0.9, (step, np.mean(got_bits == bits))
+        bits = got_bits.copy()                                   # the next step starts from the library's values
+    assert np.mean(bits != bits0) > 0.3                          # the updates are large enough to show in 16 bits
+    m.set_sparse_storage(None)
+    m.close()
