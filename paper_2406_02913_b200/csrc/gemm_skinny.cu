@@ -32,6 +32,9 @@
 //     adds the eight partials of rows 16c .. 16c+15 in CTA order (deterministic), then the sparse
 //     term and the bias, and stores y.  Partials and sparse terms are double-buffered and everyone
 //     waits only for the barrier of the tile before, so nobody stands still for the sum.
+// Codes into a per-row table of 16 values (the non-uniform 4-bit format) take the kernel too: the
+// tile's tables (128 rows x 32 bytes as bf16) travel with every step where the (scale, zero) entries
+// otherwise are, and every code is looked up there.
 // One launch may serve up to three matrices that read the same activations (q/k/v, gate/up of a decoder
 // layer): their 128-row tiles are numbered one after the other, and a tile's number names its matrix.
 // The activations may be formed while they are staged: silu(x) * x_mul, rounded to bf16 (the
@@ -131,6 +134,7 @@ __device__ __forceinline__ void workers_sync() { asm volatile("bar.sync 1, %0;" 
 struct SkinnySub {
   const uint8_t* codes_tiled;
   const float2* sz;
+  const __nv_bfloat16* lut; // [Npad][16] (table-coded weights), else NULL
   int64_t Npad;
   const int32_t* row_ptr;   // NULL: no sparse entries
   const int32_t* ent_col;
@@ -168,13 +172,16 @@ __device__ __forceinline__ int sub_of_tile(const SkinnyArgs& a, int tile) {
   return (a.n > 1 && tile >= a.sub[1].tile_begin) + (a.n > 2 && tile >= a.sub[2].tile_begin);
 }
 
-// kNT: token tiles per CTA (1: up to 8 tokens, 2: up to 16).  kGroupMma: G is a multiple of 128.
+// kNT: token tiles per CTA (1: up to 8 tokens, 2: up to 16).  kDeq: how a code becomes a weight: kDeqGroup: G is a
+// multiple of 128 (scale and zero applied to the sums of a step); kDeqSmall: groups of 32 or 64 (packed bf16
+// conversion per code); kDeqLut: per-row tables.
+constexpr int kDeqSmall = 0, kDeqGroup = 1, kDeqLut = 2;
 // Grid: kSplit * n_clusters CTAs, clusters of kSplit along x; cluster c takes tiles c, c + n_clusters, ...
 // Cluster barriers, the same sequence for every thread (no early exit): number 0 says that every
 // CTA has staged its activations, number it + 1 that part and sparse term of the cluster's tile it
 // are written, the last one that nobody reads a peer any more.  A thread arrives at number k + 1
 // only after it is done with what number k - 1 published (the buffers alternate).
-template <bool kBf16Tables, bool kGroupMma, typename TY, int kNT>
+template <bool kBf16Tables, int kDeq, typename TY, int kNT>
 __global__ void __cluster_dims__(kSplit, 1, 1) __launch_bounds__(kThreads, 2)
 szo_linear_skinny_kernel(const __grid_constant__ SkinnyArgs a) {
   constexpr int kT = kTok * kNT;                       // tokens per CTA
@@ -198,7 +205,7 @@ szo_linear_skinny_kernel(const __grid_constant__ SkinnyArgs a) {
   const int s_begin = rank * n_steps / kSplit, my_steps = (rank + 1) * n_steps / kSplit - s_begin;
   const int ld = ((n_steps + kSplit - 1) / kSplit) * kStepK + kPad;    // the same in every CTA: peers index each other's rows
   const int64_t nkb = K / 64;
-  const int ngs = (G >= kStepK) ? 1 : kStepK / G;       // (scale, zero) groups per step
+  const int ngs = kDeq == kDeqLut ? 4 : ((G >= kStepK) ? 1 : kStepK / G);   // KB per step beside the codes: (scale, zero) groups, or the tables
   const uint32_t stage_bytes = (static_cast<uint32_t>(kSzOff + ngs * 1024) + 127u) & ~127u;
   unsigned char* ring = smem_sk;
   __nv_bfloat16* sx = reinterpret_cast<__nv_bfloat16*>(smem_sk + n_stages * stage_bytes);   // [kT][ld]: the CTA's columns of x
@@ -225,7 +232,7 @@ szo_linear_skinny_kernel(const __grid_constant__ SkinnyArgs a) {
     tc::RingPos p{0, 0};
     int it = 0;
     const uint32_t tx_bytes = 8192u + static_cast<uint32_t>(ngs) * 1024u;
-    const uint32_t steps_per_group = (G >= kStepK) ? static_cast<uint32_t>(G / kStepK) : 0u;   // 0: several groups per step
+    const uint32_t steps_per_group = (kDeq != kDeqLut && G >= kStepK) ? static_cast<uint32_t>(G / kStepK) : 0u;   // 0: several groups per step
     cluster_arrive_relaxed();                           // number 0 (it stages nothing)
     // It takes its turn at barrier number it only after tile it + 1 is issued (as far as the ring lets
     // it), so that the stream does not stop while the cluster meets.
@@ -245,10 +252,14 @@ szo_linear_skinny_kernel(const __grid_constant__ SkinnyArgs a) {
             tc::mbar_expect_tx(bar, tx_bytes);
             tc::bulk_load_1d(dst, src, 4096, bar);
             tc::bulk_load_1d(dst + kBlk1, src + 4096, 4096, bar);
-            const uint32_t grp0 = (steps_per_group > 0) ? static_cast<uint32_t>(s_begin + i) / steps_per_group
-                                                        : static_cast<uint32_t>(s_begin + i) * static_cast<uint32_t>(ngs);
-            const float2* z = zsrc + static_cast<int64_t>(grp0) * Npad;
-            for (int q = 0; q < ngs; ++q, z += Npad) tc::bulk_load_1d(dst + kSzOff + q * 1024, z, 1024, bar);
+            if constexpr (kDeq == kDeqLut) {
+              tc::bulk_load_1d(dst + kSzOff, sb.lut + static_cast<int64_t>(ltile) * kRowsCta * 16, 4096, bar);
+            } else {
+              const uint32_t grp0 = (steps_per_group > 0) ? static_cast<uint32_t>(s_begin + i) / steps_per_group
+                                                          : static_cast<uint32_t>(s_begin + i) * static_cast<uint32_t>(ngs);
+              const float2* z = zsrc + static_cast<int64_t>(grp0) * Npad;
+              for (int q = 0; q < ngs; ++q, z += Npad) tc::bulk_load_1d(dst + kSzOff + q * 1024, z, 1024, bar);
+            }
           }
           src += 8192;
           p.advance(n_stages);
@@ -484,7 +495,8 @@ szo_linear_skinny_kernel(const __grid_constant__ SkinnyArgs a) {
       // -------------------------------------------------------------- weight warps
       tc::RingPos c{0, 0};
       const uint32_t w_off = static_cast<uint32_t>((t >> 1) * kBlk1 + (warp * kRowsWarp + g) * 32 + (t & 1) * 16);
-      const uint32_t z_off = static_cast<uint32_t>(kSzOff + ((G >= kStepK) ? 0 : (t * 32 / G)) * 1024 + (warp * kRowsWarp + g) * 8);
+      const uint32_t z_off = kDeq == kDeqLut ? static_cast<uint32_t>(kSzOff + (warp * kRowsWarp + g) * 32)     // the row's table
+                                             : static_cast<uint32_t>(kSzOff + ((G >= kStepK) ? 0 : (t * 32 / G)) * 1024 + (warp * kRowsWarp + g) * 8);
       int it = 0;
       for (int tile = cid; tile < n_tiles; tile += n_clusters, ++it) {
         float tot[kNT][4];
@@ -494,11 +506,35 @@ szo_linear_skinny_kernel(const __grid_constant__ SkinnyArgs a) {
         auto step_body = [&](int i, const unsigned char* stg) {
           const uint4 wa = *reinterpret_cast<const uint4*>(stg + w_off);
           const uint4 wb = *reinterpret_cast<const uint4*>(stg + w_off + 8 * 32);
-          const float2 pa = *reinterpret_cast<const float2*>(stg + z_off);
-          const float2 pb = *reinterpret_cast<const float2*>(stg + z_off + 8 * 8);
+          float2 pa = make_float2(0.f, 0.f), pb = pa;
+          if constexpr (kDeq != kDeqLut) {
+            pa = *reinterpret_cast<const float2*>(stg + z_off);
+            pb = *reinterpret_cast<const float2*>(stg + z_off + 8 * 8);
+          }
           const uint32_t qa[4] = {wa.x, wa.y, wa.z, wa.w}, qb[4] = {wb.x, wb.y, wb.z, wb.w};
           const __nv_bfloat16* xs = sx + g * ld + i * kStepK + t * 8;      // token g; word wd of this lane: + wd * 32
-          if constexpr (kGroupMma) {
+          if constexpr (kDeq == kDeqLut) {
+            const unsigned char* ta = stg + z_off;                         // table of row g; row g + 8: 8 * 32 bytes further
+            auto look = [&](const unsigned char* tab, uint32_t q, int lo_shift) -> uint32_t {
+              // bf16 pair (table[nibble at lo_shift], table[nibble at lo_shift + 16]); byte offset = 2 * nibble
+              const uint32_t o0 = lo_shift == 0 ? (q << 1) & 0x1Eu : (q >> (lo_shift - 1)) & 0x1Eu;
+              const uint32_t o1 = (q >> (lo_shift + 15)) & 0x1Eu;
+              const uint32_t v0 = *reinterpret_cast<const unsigned short*>(tab + o0);
+              const uint32_t v1 = *reinterpret_cast<const unsigned short*>(tab + o1);
+              return v0 | (v1 << 16);
+            };
+#pragma unroll
+            for (int wd = 0; wd < 4; ++wd) {
+              const uint32_t a0[4] = {look(ta, qa[wd], 0), look(ta + 8 * 32, qb[wd], 0), look(ta, qa[wd], 4), look(ta + 8 * 32, qb[wd], 4)};
+              const uint32_t a1[4] = {look(ta, qa[wd], 8), look(ta + 8 * 32, qb[wd], 8), look(ta, qa[wd], 12), look(ta + 8 * 32, qb[wd], 12)};
+#pragma unroll
+              for (int j = 0; j < kNT; ++j) {
+                const uint4 xv = *reinterpret_cast<const uint4*>(xs + j * kTok * ld + wd * 32);
+                mma_acc(tot[j], a0, xv.x, xv.y);
+                mma_acc(tot[j], a1, xv.z, xv.w);
+              }
+            }
+          } else if constexpr (kDeq == kDeqGroup) {
             float accq[kNT][2][4];                                         // even and odd words: two shorter chains
 #pragma unroll
             for (int wd = 0; wd < 4; ++wd) {                                // one 32-bit word = 8 columns = two k16 MMAs
@@ -584,16 +620,16 @@ szo_linear_skinny_kernel(const __grid_constant__ SkinnyArgs a) {
 
 size_t skinny_dyn_smem(int64_t K, int G, int kT, int n_stages = kStages) {
   const int64_t n_steps = K / kStepK, max_steps = ceil_div(n_steps, kSplit);
-  const size_t ngs = (G >= kStepK) ? 1 : kStepK / G;
+  const size_t ngs = G < 0 ? 4 : ((G >= kStepK) ? 1 : kStepK / G);     // G < 0: per-row tables, 4 KB per step
   const size_t stage = (static_cast<size_t>(kSzOff) + ngs * 1024 + 127) & ~static_cast<size_t>(127);
   return n_stages * stage + static_cast<size_t>(kT) * (max_steps * kStepK + kPad) * 2 + static_cast<size_t>(max_steps) * kT * 4 +
          static_cast<size_t>(max_steps) * kStepK * kT * 2;     // ring, x [token][column], step sums, x [column][token]
 }
 
-template <bool kBf16Tables, bool kGroupMma, typename TY, int kNT>
+template <bool kBf16Tables, int kDeq, typename TY, int kNT>
 szo_status launch_skinny(const szo_linear* const* plans, int n, const void* x, const void* x_mul, int64_t M,
                          const float* const* S, void* const* y, cudaStream_t st, bool chained) {
-  auto kern = szo_linear_skinny_kernel<kBf16Tables, kGroupMma, TY, kNT>;
+  auto kern = szo_linear_skinny_kernel<kBf16Tables, kDeq, TY, kNT>;
   const szo_linear* p = plans[0];
   // A ring of 8 steps when two CTAs of that size still share an SM (or when 4 would not change that
   // either), else 4: two CTAs with 4 steps in flight each hide more than one with 8.
@@ -647,8 +683,8 @@ szo_status launch_skinny(const szo_linear* const* plans, int n, const void* x, c
   int n_tiles = 0;
   for (int i = 0; i < n; ++i) {
     const szo_linear* q = plans[i];
-    a.sub[i] = SkinnySub{q->codes_tiled, q->sz, q->Npad, q->nnz > 0 ? q->row_ptr : nullptr, q->ent_col, S[i], q->bias, y[i],
-                         q->N, n_tiles};
+    a.sub[i] = SkinnySub{q->codes_tiled, q->sz, q->lut_bf16, q->Npad, q->nnz > 0 ? q->row_ptr : nullptr, q->ent_col, S[i],
+                         q->bias, y[i], q->N, n_tiles};
     n_tiles += static_cast<int>(ceil_div(q->N, kRowsCta));
   }
   a.n_tiles = n_tiles;
@@ -664,23 +700,32 @@ szo_status launch_skinny(const szo_linear* const* plans, int n, const void* x, c
 template <bool kBf16Tables, typename TY>
 szo_status launch_skinny_nt(const szo_linear* const* plans, int n, const void* x, const void* x_mul, int64_t M,
                             const float* const* S, void* const* y, cudaStream_t st, bool chained) {
+  if (plans[0]->G < 0) {                       // per-row tables (the plan's bf16 copy: the tables' own type does not matter)
+    if constexpr (!kBf16Tables) {
+      if (M <= kTok) return launch_skinny<false, kDeqLut, TY, 1>(plans, n, x, x_mul, M, S, y, st, chained);
+      return launch_skinny<false, kDeqLut, TY, 2>(plans, n, x, x_mul, M, S, y, st, chained);
+    } else {
+      return fail(SZO_ERR_UNSUPPORTED, "table-coded plans take the f16-table instantiation");
+    }
+  }
   const bool group = plans[0]->G % kStepK == 0;
   if (M <= kTok) {
-    if (group) return launch_skinny<kBf16Tables, true, TY, 1>(plans, n, x, x_mul, M, S, y, st, chained);
-    return launch_skinny<kBf16Tables, false, TY, 1>(plans, n, x, x_mul, M, S, y, st, chained);
+    if (group) return launch_skinny<kBf16Tables, kDeqGroup, TY, 1>(plans, n, x, x_mul, M, S, y, st, chained);
+    return launch_skinny<kBf16Tables, kDeqSmall, TY, 1>(plans, n, x, x_mul, M, S, y, st, chained);
   }
-  if (group) return launch_skinny<kBf16Tables, true, TY, 2>(plans, n, x, x_mul, M, S, y, st, chained);
-  return launch_skinny<kBf16Tables, false, TY, 2>(plans, n, x, x_mul, M, S, y, st, chained);
+  if (group) return launch_skinny<kBf16Tables, kDeqGroup, TY, 2>(plans, n, x, x_mul, M, S, y, st, chained);
+  return launch_skinny<kBf16Tables, kDeqSmall, TY, 2>(plans, n, x, x_mul, M, S, y, st, chained);
 }
 
 }  // namespace
 
 // The shapes the weight-streaming kernel takes: int4 plans with groups of 32, 64 or a multiple of
-// 128 columns, at most 16 tokens, K a multiple of 128 whose per-CTA slice of the tokens fits shared
+// 128 columns or with per-row tables, at most 16 tokens, K a multiple of 128 whose per-CTA slice of the tokens fits shared
 // memory (K up to about 25 000 for 8 tokens, 14 000 for 16).
 bool skinny_applies(const szo_linear* p, int64_t M) {
-  return p->G > 0 && (p->G == 32 || p->G == 64 || p->G % kStepK == 0) && M >= 1 && M <= 2 * kTok &&
-         p->K % kStepK == 0 && skinny_dyn_smem(p->K, p->G, M <= kTok ? kTok : 2 * kTok) <= kMaxDynSmem;
+  const bool lut = p->G == -1 && p->lut_bf16 != nullptr;
+  return (lut || (p->G > 0 && (p->G == 32 || p->G == 64 || p->G % kStepK == 0))) && p->codes_tiled != nullptr && M >= 1 &&
+         M <= 2 * kTok && p->K % kStepK == 0 && skinny_dyn_smem(p->K, p->G, M <= kTok ? kTok : 2 * kTok) <= kMaxDynSmem;
 }
 
 // Up to three matrices with the same K, group size and table type in one launch
@@ -701,7 +746,7 @@ szo_status linear_fwd_skinny_group(const szo_linear* const* plans, int n, const 
                                    const float* const* S_pert, void* const* y, int y_dtype, cudaStream_t st, bool chained) {
   if (gemv_applies(plans, n, M)) return linear_fwd_gemv(plans, n, x, x_mul, M, S_pert, y, y_dtype, st, chained);
   SZO_REQUIRE(skinny_group_applies(plans, n, M), SZO_ERR_UNSUPPORTED, "shapes not covered by the weight-streaming kernel");
-  const bool bf = plans[0]->sz_dtype == SZO_BF16;
+  const bool bf = plans[0]->sz_dtype == SZO_BF16 && plans[0]->G > 0;
   if (y_dtype == SZO_F32) {
     if (bf) return launch_skinny_nt<true, float>(plans, n, x, x_mul, M, S_pert, y, st, chained);
     return launch_skinny_nt<false, float>(plans, n, x, x_mul, M, S_pert, y, st, chained);

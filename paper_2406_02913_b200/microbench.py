@@ -337,7 +337,8 @@ def decode_case(name, Bn, prompt, gen):
     weight_bytes = 0
     for nm in wl.linear_names(shape):
         N, K = wl.linear_shape(shape, nm)
-        weight_bytes += (N * K // 2 + 4 * N * K // shape["group"]) if shape["group"] > 0 else 2 * N * K
+        G = shape["group"]
+        weight_bytes += (N * K // 2 + 4 * N * K // G) if G > 0 else ((N * K // 2 + 32 * N) if G < 0 else 2 * N * K)
     weight_bytes = weight_bytes * shape["n_layers"] + 2 * shape["vocab"] * shape["d_model"]
     hbm = peaks()[0]
     per_step_ms = ms_gen / gen

@@ -240,6 +240,10 @@ LUT_CASES = [
     (200, 1024, "f16", 1, 5e-3, True),              # N not a multiple of 16; one step per warp
     (512, 4096, "bf16", 2, 1e-3, False),
     (304, 11008, "f16", 1, 2e-3, True),             # 86 steps: several row groups per CTA, tables change with them
+    # 3 to 16 tokens, K a multiple of 128: looked up inside the cluster kernel
+    (200, 640, "bf16", 5, 5e-3, True),              # 5 K steps for 8 CTAs, N not a multiple of 128
+    (300, 4224, "f16", 13, 2e-3, True),             # two token tiles, the second ragged
+    (1024, 11008, "f16", 8, 1e-3, False),
 ]
 
 
