@@ -75,6 +75,13 @@ struct GemvArgs {
 // lanes' chunks of a turn are side by side.
 __device__ __forceinline__ int gv_chunk_pos(int c) { return (c & ~15) | ((c & 3) << 2) | ((c >> 2) & 3); }
 
+// (a & b) | c in one instruction (written out: the compiler makes three of the C++ expression)
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+
 // D = A B
 __device__ __forceinline__ void gv_mma_new(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile(
@@ -405,14 +412,14 @@ __global__ void __launch_bounds__(kGvThreads, 2) szo_linear_gemv_kernel(const __
 #pragma unroll
             for (int wd = 0; wd < 4; ++wd) {                // one 32-bit word = 8 columns = two k16 MMAs
               uint32_t a0[4], a1[4];
-              a0[0] = (qa[wd] & 0x000F000Fu) | 0x43004300u;
-              a0[1] = (qb[wd] & 0x000F000Fu) | 0x43004300u;
-              a0[2] = ((qa[wd] >> 4) & 0x000F000Fu) | 0x43004300u;
-              a0[3] = ((qb[wd] >> 4) & 0x000F000Fu) | 0x43004300u;
-              a1[0] = ((qa[wd] >> 8) & 0x000F000Fu) | 0x43004300u;
-              a1[1] = ((qb[wd] >> 8) & 0x000F000Fu) | 0x43004300u;
-              a1[2] = ((qa[wd] >> 12) & 0x000F000Fu) | 0x43004300u;
-              a1[3] = ((qb[wd] >> 12) & 0x000F000Fu) | 0x43004300u;
+              a0[0] = and_or(qa[wd], 0x000F000Fu, 0x43004300u);
+              a0[1] = and_or(qb[wd], 0x000F000Fu, 0x43004300u);
+              a0[2] = and_or(qa[wd] >> 4, 0x000F000Fu, 0x43004300u);
+              a0[3] = and_or(qb[wd] >> 4, 0x000F000Fu, 0x43004300u);
+              a1[0] = and_or(qa[wd] >> 8, 0x000F000Fu, 0x43004300u);
+              a1[1] = and_or(qb[wd] >> 8, 0x000F000Fu, 0x43004300u);
+              a1[2] = and_or(qa[wd] >> 12, 0x000F000Fu, 0x43004300u);
+              a1[3] = and_or(qb[wd] >> 12, 0x000F000Fu, 0x43004300u);
               const uint4 xv = *reinterpret_cast<const uint4*>(xs + wd * 32);
               if (wd < 2) gv_mma_new(accq[wd & 1], a0, xv.x, xv.y);
               else gv_mma_acc(accq[wd & 1], a0, xv.x, xv.y);

@@ -236,7 +236,8 @@ __device__ __forceinline__ uint4 dequant_word(uint32_t w, float2 p) {
     const __nv_bfloat162 m2 = *reinterpret_cast<const __nv_bfloat162*>(&magic);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const uint32_t t = ((w >> (4 * i)) & 0x000F000Fu) | magic;     // one shift and one three-input logic op
+      uint32_t t;                                                    // ((w >> 4 i) & 0x000F000F) | magic: one shift and ONE logic op
+      asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(t) : "r"(w >> (4 * i)), "r"(0x000F000Fu), "r"(magic));   // (written out: the compiler makes two of it)
       const __nv_bfloat162 q2 = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&t), m2);
       const __nv_bfloat162 r = __hfma2(q2, s2, z2);
       o[i] = *reinterpret_cast<const uint32_t*>(&r);
