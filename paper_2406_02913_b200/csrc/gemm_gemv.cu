@@ -1,4 +1,4 @@
-// Weight-streaming form of the decomposed linear for one to four tokens (a token-generation step):
+// Weight-streaming form of the decomposed linear for one or two tokens (a token-generation step):
 //   y[m, n] = sum_k x[m,k] * Dequantize(Q)[n,k] + sum_{(n,c) in mask} x[m,c] * S[n,c] + bias[n]
 // (appendix "Implementation of Sparse Operations in Linear Layers": the SparseAddMM order, which the
 // paper finds the faster one for token generation).  With so few tokens all activations of a row of
@@ -10,9 +10,9 @@
 //   * every lane reads its own 16 bytes of codes per weight row and step straight from global memory
 //     in the fragment layout (the 16 rows of a k-block are 512 contiguous bytes of the tiled codes: one
 //     coalesced 128-bit load per warp), four steps ahead in registers, across row groups (the stream
-//     never drains) and from the first instruction on, before the activations are even staged.  (Bulk copies of 512 bytes into a ring in shared
-//     memory were tried first: the copy engine took about 36 ns per copy whatever its size, 16 us for
-//     the 66 000 copies of an 11008 x 4096 matrix.)
+//     never drains) and from the first instruction on, before the activations are even staged.
+//     (Bulk copies of 512 bytes into a ring in shared memory were tried first: the copy engine took
+//     about 36 ns per copy whatever its size, 16 us for the 66 000 copies of an 11008 x 4096 matrix.)
 //   * the product is the group form of the 16-token kernel: m16n8k16 MMAs of (128 + code) as bf16
 //     against the tokens, scale and zero applied once per 128-column step to the fp32 sums,
 //     sum_k x_k (q_k s + z) = s sum_k x_k (128 + q_k) + (z - 128 s) sum_k x_k;
@@ -20,13 +20,15 @@
 //     ahead, entries and values one ahead, activations from shared memory), then adds the weight
 //     warps' partial sums in warp order, the sparse term and the bias, and stores y; the partial
 //     sums are double-buffered, so the weight warps never wait for it.
-// One launch serves up to three matrices that read the same activations (q/k/v, gate/up); the
-// activations may be silu(x) * x_mul formed while they are staged.  Quantization groups must be
-// multiples of 128 columns.
+// One launch serves up to three matrices that read the same activations (q/k/v, gate/up).  The
+// activations may be formed while they are staged: silu(x) * x_mul (the gated MLP's product), or the
+// normalised residual stream (FusedNorm in linear.cuh: residual add, RMSNorm or LayerNorm).
+// Quantization groups must be multiples of 128 columns.
 // Codes into a per-row table of 16 values (the non-uniform 4-bit format) take the same kernel: the
 // tables of the 16 rows (512 bytes as bf16) travel with every step in the registers that otherwise
 // carry (scale, zero), are put into the warp's own shared memory when a row group begins, and every
-// code is looked up there (one 2-byte read of shared memory per code instead of half an AND-OR).  The kernel waits on nothing but its own block barriers.
+// code is looked up there (one 2-byte read of shared memory per code instead of half an AND-OR).
+// The kernel waits on nothing but its own block barriers.
 #include <cstdlib>
 #include <mutex>
 
@@ -42,7 +44,7 @@ constexpr int kGvWarps = 7;          // weight warps; the eighth forms the spars
 constexpr int kGvThreads = (kGvWarps + 1) * 32;
 constexpr int kGvStepK = 128;        // columns per step
 constexpr int kGvDepth = 4;          // steps in flight per warp (registers)
-constexpr int kGvMaxTok = 2;          // more tokens: the 16-token kernel (staging four rows of x per CTA costs more than its rendezvous)
+constexpr int kGvMaxTok = 2;         // more tokens: the 16-token kernel (staging four rows of x per CTA costs more than its rendezvous)
 constexpr int kGvPad = 32;           // elements added to a token row in shared memory
 constexpr int kGvTabStride = 48;     // bytes per row of a warp's table block in shared memory (32 used)
 
