@@ -142,6 +142,15 @@ szo_status szo_perturb_keep_z(const float* S_in, float* S_out, const int64_t* id
                               void* stream);
 szo_status szo_perturb_kept_z(const float* S_in, float* S_out, const float* z, int64_t k, float scale,
                               void* stream);
+/* The +eps, -2 eps, +eps passes of the seed trick for one (seed, step) in ONE launch (a step that evaluates both
+ * losses from copies of S, or inside the linears, makes the three passes back to back; the pass is bound by
+ * drawing z, so the other two cost their two fused multiply-adds):
+ *   sp = fma(eps, z_j, S_in[j]), sm = fma(-2 eps, z_j, sp), S_out[j] = fma(eps, z_j, sm), z_out[j] = z_j,
+ *   and S_plus[j] = sp, S_minus[j] = sm where those pointers are not NULL (fp32[k], 16-byte aligned).
+ * The same bits as szo_perturb_keep_z(eps), szo_perturb_kept_z(-2 eps), szo_perturb_kept_z(eps) in turn. */
+szo_status szo_perturb3_keep_z(const float* S_in, float* S_out, const int64_t* idx, int64_t k, int64_t idx_base,
+                               uint64_t seed, uint64_t step, float eps, float* z_out, float* S_plus, float* S_minus,
+                               void* stream);
 szo_status szo_update_kept_z(float* S, const float* z, int64_t k, float lr, const double* f_plus_dev,
                              const double* f_minus_dev, float eps, void* stream);
 

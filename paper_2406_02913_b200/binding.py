@@ -72,6 +72,8 @@ _SIGS = {
                                 C.c_uint64, C.c_uint64, C.c_float, C.c_void_p]),
     "szo_perturb_keep_z": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
                                        C.c_uint64, C.c_uint64, C.c_float, C.c_void_p, C.c_void_p]),
+    "szo_perturb3_keep_z": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_uint64, C.c_uint64,
+                                        C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "szo_perturb_kept_z": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_float, C.c_void_p]),
     "szo_update_kept_z": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int64, C.c_float, C.c_void_p, C.c_void_p,
                                       C.c_float, C.c_void_p]),
@@ -219,6 +221,12 @@ def szo_perturb(S_in, S_out, idx, idx_base: int, seed: int, step: int, scale: fl
 def szo_perturb_keep_z(S_in, S_out, idx, idx_base: int, seed: int, step: int, scale: float, z_out):
     _check(lib().szo_perturb_keep_z(_ptr(S_in), _ptr(S_out), _ptr(idx), idx.numel(), idx_base, seed, step,
                                     scale, _ptr(z_out), _stream()))
+
+
+def szo_perturb3_keep_z(S_in, S_out, idx, idx_base: int, seed: int, step: int, eps: float, z_out, S_plus=None, S_minus=None):
+    """The +eps, -2 eps, +eps passes in one launch (szo_perturb3_keep_z)."""
+    _check(lib().szo_perturb3_keep_z(_ptr(S_in), _ptr(S_out), _ptr(idx), idx.numel(), idx_base, seed, step, eps,
+                                     _ptr(z_out), _ptr(S_plus), _ptr(S_minus), _stream()))
 
 
 def szo_perturb_kept_z(S_in, S_out, z, scale: float):

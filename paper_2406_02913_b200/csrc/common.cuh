@@ -97,6 +97,11 @@ struct ScaleArg {
 szo_status launch_sparse_axpy(const float* S_in, float* S_out, const int64_t* idx, int64_t k,
                               int64_t idx_base, uint64_t seed, uint64_t step, ScaleArg sa,
                               cudaStream_t st, float* z_out = nullptr);
+// The +eps, -2 eps, +eps passes of one (seed, step) in one launch, z kept in z_out: S_out takes the value the
+// three passes leave (same roundings); S_plus / S_minus, where not NULL, the values after the first / second
+szo_status launch_sparse_axpy_three(const float* S_in, float* S_out, const int64_t* idx, int64_t k, int64_t idx_base,
+                                    uint64_t seed, uint64_t step, float eps, cudaStream_t st, float* z_out,
+                                    float* S_plus, float* S_minus);
 // S_out[j] = fma(scale, z[j], S_in[j]) with kept z
 szo_status launch_sparse_axpy_kept(const float* S_in, float* S_out, const float* z, int64_t k, ScaleArg sa,
                                    cudaStream_t st);

@@ -1733,21 +1733,15 @@ static szo_status zo_losses_impl(szo_model* m, const int32_t* tokens, const int3
     // S goes through the seed trick's +eps, -2 eps, +eps sequence (so that it ends where the
     // in-place order leaves it) while z is kept; the two forwards then run in the paired form on the
     // restored S, with +-eps z applied inside the linears in fp32
-    SZO_TRY(launch_sparse_axpy(Sv, Sv, m->gidx, k, 0, seed, step, sa, st, m->zkept));
-    sa.scale = -2.0f * eps;
-    SZO_TRY(launch_sparse_axpy_kept(Sv, Sv, m->zkept, k, sa, st));
-    sa.scale = eps;
-    SZO_TRY(launch_sparse_axpy_kept(Sv, Sv, m->zkept, k, sa, st));
+    // (one launch: the pass is bound by drawing z, the other two are its fused multiply-adds)
+    SZO_TRY(launch_sparse_axpy_three(Sv, Sv, m->gidx, k, 0, seed, step, eps, st, m->zkept, nullptr, nullptr));
     return run_loss_paired(m, tokens, labels, cand, B, S, Sv, m->zkept, eps, f_plus_dev, f_minus_dev, st);
   }
   if (dual_forward_applies(m, static_cast<int64_t>(B) * S)) {
     // both forwards side by side: the same arithmetic on S as the in-place sequence below
     // (+eps, -2 eps, +eps), written to two copies, so that every linear makes one weight pass
-    SZO_TRY(launch_sparse_axpy(Sv, m->Splus, m->gidx, k, 0, seed, step, sa, st, m->zkept));   // S+ = S + eps z
-    sa.scale = -2.0f * eps;
-    SZO_TRY(launch_sparse_axpy_kept(m->Splus, m->Sminus, m->zkept, k, sa, st));               // S- = S+ - 2 eps z
-    sa.scale = eps;
-    SZO_TRY(launch_sparse_axpy_kept(m->Sminus, Sv, m->zkept, k, sa, st));                     // S = S- + eps z
+    // S+ = S + eps z, S- = S+ - 2 eps z, S = S- + eps z in one launch
+    SZO_TRY(launch_sparse_axpy_three(Sv, Sv, m->gidx, k, 0, seed, step, eps, st, m->zkept, m->Splus, m->Sminus));
     return run_loss_t<__nv_bfloat16>(m, tokens, labels, cand, B, S, m->Splus, f_plus_dev, st, m->Sminus, f_minus_dev);
   }
   // z is generated once per step (first pass) and kept: the other passes stream it

@@ -100,12 +100,27 @@ __device__ __forceinline__ float resolve_scale(const ScaleArg& a) {
 constexpr int kAxpyPer = 8;
 
 // kKeepZ: also store z_j to z_out[j], for the later passes of the same (seed, step).
-template <bool kKeepZ>
+// kThree: the +eps, -2 eps, +eps passes of the seed trick in one (scale = eps): with sp = fma(eps, z, S),
+// sm = fma(-2 eps, z, sp), s0 = fma(eps, z, sm) (the roundings of the three separate passes), S_out = s0
+// and, where given, S_plus = sp and S_minus = sm.  The pass is bound by drawing z, so the two extra fused
+// multiply-adds and stores cost nothing measurable.
+template <bool kKeepZ, bool kThree>
 __global__ void __launch_bounds__(256)
 sparse_axpy_kernel(const float* S_in, float* S_out,      // may alias (in-place passes): no __restrict__
                    const int64_t* __restrict__ idx, int64_t k, int64_t idx_base, const PhiloxKeys K,
-                   uint32_t step_lo, uint32_t step_hi, ScaleArg sa, float* __restrict__ z_out) {
+                   uint32_t step_lo, uint32_t step_hi, ScaleArg sa, float* __restrict__ z_out,
+                   float* __restrict__ S_plus, float* __restrict__ S_minus) {
   const float scale = resolve_scale(sa);
+  auto apply = [&](float z, float s, float& sp, float& sm) -> float {
+    if constexpr (kThree) {
+      sp = fmaf(scale, z, s);
+      sm = fmaf(-2.0f * scale, z, sp);
+      return fmaf(scale, z, sm);
+    } else {
+      sp = sm = 0.f;
+      return fmaf(scale, z, s);
+    }
+  };
   const int64_t octs = k / kAxpyPer;
   const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
   for (int64_t p = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; p < octs; p += stride) {
@@ -123,12 +138,16 @@ sparse_axpy_kernel(const float* S_in, float* S_out,      // may alias (in-place 
     }
 #pragma unroll
     for (int j = 0; j < 2; ++j) {
-      float4 o;
-      o.x = fmaf(scale, z[4 * j], s[j].x);
-      o.y = fmaf(scale, z[4 * j + 1], s[j].y);
-      o.z = fmaf(scale, z[4 * j + 2], s[j].z);
-      o.w = fmaf(scale, z[4 * j + 3], s[j].w);
+      float4 o, op, om;
+      o.x = apply(z[4 * j], s[j].x, op.x, om.x);
+      o.y = apply(z[4 * j + 1], s[j].y, op.y, om.y);
+      o.z = apply(z[4 * j + 2], s[j].z, op.z, om.z);
+      o.w = apply(z[4 * j + 3], s[j].w, op.w, om.w);
       reinterpret_cast<float4*>(S_out)[2 * p + j] = o;
+      if constexpr (kThree) {
+        if (S_plus != nullptr) reinterpret_cast<float4*>(S_plus)[2 * p + j] = op;
+        if (S_minus != nullptr) reinterpret_cast<float4*>(S_minus)[2 * p + j] = om;
+      }
       if constexpr (kKeepZ)
         reinterpret_cast<float4*>(z_out)[2 * p + j] = make_float4(z[4 * j], z[4 * j + 1], z[4 * j + 2], z[4 * j + 3]);
     }
@@ -137,7 +156,12 @@ sparse_axpy_kernel(const float* S_in, float* S_out,      // may alias (in-place 
   const int64_t j = octs * kAxpyPer + threadIdx.x;
   if (blockIdx.x == 0 && threadIdx.x < kAxpyPer && j < k) {
     const float z = z_of(static_cast<uint64_t>(idx_base + idx[j]), step_lo, step_hi, K);
-    S_out[j] = fmaf(scale, z, S_in[j]);
+    float sp, sm;
+    S_out[j] = apply(z, S_in[j], sp, sm);
+    if constexpr (kThree) {
+      if (S_plus != nullptr) S_plus[j] = sp;
+      if (S_minus != nullptr) S_minus[j] = sm;
+    }
     if constexpr (kKeepZ) z_out[j] = z;
   }
 }
@@ -198,9 +222,9 @@ szo_status launch_sparse_axpy_kept(const float* S_in, float* S_out, const float*
   return SZO_OK;
 }
 
-szo_status launch_sparse_axpy(const float* S_in, float* S_out, const int64_t* idx, int64_t k,
-                              int64_t idx_base, uint64_t seed, uint64_t step, ScaleArg sa,
-                              cudaStream_t st, float* z_out) {
+static szo_status launch_sparse_axpy_any(const float* S_in, float* S_out, const int64_t* idx, int64_t k,
+                                         int64_t idx_base, uint64_t seed, uint64_t step, ScaleArg sa,
+                                         cudaStream_t st, float* z_out, bool three, float* S_plus, float* S_minus) {
   if (k == 0) return SZO_OK;
   PhiloxKeys K;
   uint32_t k0 = static_cast<uint32_t>(seed), k1 = static_cast<uint32_t>(seed >> 32);
@@ -219,15 +243,31 @@ szo_status launch_sparse_axpy(const float* S_in, float* S_out, const int64_t* id
     blocks = ceil_div(ceil_div(quads, sweeps), 256);        // just enough threads for that many sweeps
     if (blocks > wave) blocks = wave;
   }
-  if (z_out != nullptr)
-    sparse_axpy_kernel<true><<<static_cast<unsigned>(blocks), 256, 0, st>>>(
-        S_in, S_out, idx, k, idx_base, K, static_cast<uint32_t>(step), static_cast<uint32_t>(step >> 32), sa, z_out);
+  const uint32_t lo = static_cast<uint32_t>(step), hi = static_cast<uint32_t>(step >> 32);
+  const unsigned nb = static_cast<unsigned>(blocks);
+  if (three)
+    sparse_axpy_kernel<true, true><<<nb, 256, 0, st>>>(S_in, S_out, idx, k, idx_base, K, lo, hi, sa, z_out, S_plus, S_minus);
+  else if (z_out != nullptr)
+    sparse_axpy_kernel<true, false><<<nb, 256, 0, st>>>(S_in, S_out, idx, k, idx_base, K, lo, hi, sa, z_out, nullptr, nullptr);
   else
-    sparse_axpy_kernel<false><<<static_cast<unsigned>(blocks), 256, 0, st>>>(
-        S_in, S_out, idx, k, idx_base, K, static_cast<uint32_t>(step), static_cast<uint32_t>(step >> 32), sa, nullptr);
+    sparse_axpy_kernel<false, false><<<nb, 256, 0, st>>>(S_in, S_out, idx, k, idx_base, K, lo, hi, sa, nullptr, nullptr, nullptr);
   count_launch();
   SZO_CHECK_LAUNCH("sparse_axpy_kernel");
   return SZO_OK;
+}
+
+szo_status launch_sparse_axpy(const float* S_in, float* S_out, const int64_t* idx, int64_t k,
+                              int64_t idx_base, uint64_t seed, uint64_t step, ScaleArg sa,
+                              cudaStream_t st, float* z_out) {
+  return launch_sparse_axpy_any(S_in, S_out, idx, k, idx_base, seed, step, sa, st, z_out, false, nullptr, nullptr);
+}
+
+szo_status launch_sparse_axpy_three(const float* S_in, float* S_out, const int64_t* idx, int64_t k, int64_t idx_base,
+                                    uint64_t seed, uint64_t step, float eps, cudaStream_t st, float* z_out,
+                                    float* S_plus, float* S_minus) {
+  if (z_out == nullptr) return fail(SZO_ERR_INVALID_ARG, "the three-pass form keeps z");
+  ScaleArg sa{eps, 0.f, 0.f, nullptr, nullptr};
+  return launch_sparse_axpy_any(S_in, S_out, idx, k, idx_base, seed, step, sa, st, z_out, true, S_plus, S_minus);
 }
 
 }  // namespace szo
@@ -273,6 +313,20 @@ szo_status szo_perturb_keep_z(const float* S_in, float* S_out, const int64_t* id
   szo::ScaleArg sa{scale, 0.f, 0.f, nullptr, nullptr};
   return szo::launch_sparse_axpy(S_in, S_out, idx, k, idx_base, seed, step, sa, static_cast<cudaStream_t>(stream),
                                  z_out);
+}
+
+szo_status szo_perturb3_keep_z(const float* S_in, float* S_out, const int64_t* idx, int64_t k, int64_t idx_base,
+                               uint64_t seed, uint64_t step, float eps, float* z_out, float* S_plus, float* S_minus,
+                               void* stream) {
+  SZO_REQUIRE(k >= 0, SZO_ERR_INVALID_ARG, "k < 0");
+  if (k == 0) return SZO_OK;
+  SZO_REQUIRE(S_in && S_out && idx && z_out, SZO_ERR_INVALID_ARG, "NULL pointer");
+  SZO_REQUIRE(idx_base >= 0, SZO_ERR_INVALID_ARG, "idx_base < 0");
+  SZO_REQUIRE(szo::aligned16(S_in) && szo::aligned16(S_out) && szo::aligned16(idx) && szo::aligned16(z_out) &&
+                  szo::aligned16(S_plus) && szo::aligned16(S_minus),
+              SZO_ERR_ALIGNMENT, "S_in, S_out, idx, z_out, S_plus and S_minus must be 16-byte aligned");
+  return szo::launch_sparse_axpy_three(S_in, S_out, idx, k, idx_base, seed, step, eps, static_cast<cudaStream_t>(stream),
+                                       z_out, S_plus, S_minus);
 }
 
 szo_status szo_perturb_kept_z(const float* S_in, float* S_out, const float* z, int64_t k, float scale, void* stream) {

@@ -121,6 +121,34 @@ def test_kept_z_passes_equal_the_regenerating_ones(B, k):
                           so.fmaf32(np.float32(0.5), z.cpu().numpy(), b.cpu().numpy()).view(np.uint32))
 
 
+@pytest.mark.parametrize("k", [1, 7, 8, 4099, 250_001])
+def test_three_passes_in_one_launch_equal_the_three_launches(B, k):
+    """szo_perturb3_keep_z: the +eps, -2 eps, +eps passes of one (seed, step) in one launch leave the bits of
+    the three separate launches in S, in S_plus / S_minus (where asked for) and in z; in place and out of place."""
+    n = 6_476_005_376
+    idx = torch.from_numpy(wl.sorted_random_indices(n, k, seed=31, i=k)).cuda()
+    S0 = torch.from_numpy(wl.rng(32, wl.PURPOSE_WEIGHTS, k).normal(0, 0.02, k).astype(np.float32)).cuda()
+    seed, step, eps = 99, 11, 1e-3
+    a = S0.clone()
+    z = torch.empty(k, device="cuda")
+    B.szo_perturb_keep_z(a, a, idx, 5, seed, step, eps, z)
+    plus = a.clone()
+    B.szo_perturb_kept_z(a, a, z, -2.0 * eps)
+    minus = a.clone()
+    B.szo_perturb_kept_z(a, a, z, eps)
+    b, z3 = S0.clone(), torch.full((k,), 7.0, device="cuda")
+    B.szo_perturb3_keep_z(b, b, idx, 5, seed, step, eps, z3)                    # in place, no copies asked for
+    assert torch.equal(a, b) and torch.equal(z, z3)
+    out, p3, m3 = torch.empty_like(S0), torch.empty_like(S0), torch.empty_like(S0)
+    B.szo_perturb3_keep_z(S0, out, idx, 5, seed, step, eps, z3, p3, m3)           # out of place, both copies
+    assert torch.equal(out, a) and torch.equal(p3, plus) and torch.equal(m3, minus)
+    ref = so.perturb(so.perturb(so.perturb(S0.cpu().numpy(), idx.cpu().numpy() + 5, seed, step, np.float32(eps)),
+                                idx.cpu().numpy() + 5, seed, step, np.float32(-2.0) * np.float32(eps)),
+                     idx.cpu().numpy() + 5, seed, step, np.float32(eps))
+    assert np.allclose(out.cpu().numpy(), ref, rtol=0, atol=1e-8)               # (z agrees to 5e-7, eps = 1e-3: an ulp of S or two)
+    assert B.device_status() == 0
+
+
 def test_perturb_empty_and_bad_arguments(B):
     e = torch.empty(0, device="cuda")
     B.szo_perturb(e, e, torch.empty(0, dtype=torch.int64, device="cuda"), 0, 1, 1, 1.0)
