@@ -243,7 +243,7 @@ __device__ __forceinline__ float sinh_small(float a) {
   const float a2 = a * a;
   if (a2 < 0.25f) return a * (1.0f + a2 * (1.0f / 6.0f + a2 * (1.0f / 120.0f + a2 * (1.0f / 5040.0f + a2 * (1.0f / 362880.0f)))));
   const float u = __expf(a);
-  return 0.5f * (u - 1.0f / u);
+  return 0.5f * (u - __fdividef(1.0f, u));
 }
 
 template <int HD>
@@ -395,7 +395,7 @@ flash_attn_pair_bf16_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bflo
         const float e = exp2f(sc[i][j] * scale_log2e - msc[j >> 1]);
         const float a = sd[i][j] * scale;
         const float u = exp2f(sd[i][j] * scale_log2e);
-        pc4[j] = e * 0.5f * (u + 1.0f / u);
+        pc4[j] = e * 0.5f * (u + __fdividef(1.0f, u));          // (fast reciprocal: the result is rounded to bf16)
         pd4[j] = e * sinh_small(a);
       }
       lc[0] += pc4[0] + pc4[1];
