@@ -391,22 +391,34 @@ __global__ void __launch_bounds__(TM == 16 ? 1024 : 512) pair_cross_kernel(const
   const V* xs = reinterpret_cast<const V*>(cross_smem);          // [K][kVecs]
   const int64_t m0 = static_cast<int64_t>(blockIdx.x) * TM;
   {
-    // lane = (column group cg, token t): one 16-byte load of 8 columns of token t, then 8 two-byte
-    // stores xs[c][t]; group cg starts its 8 stores at element cg so that groups use different banks
-    unsigned short* xs16 = reinterpret_cast<unsigned short*>(cross_smem);
+    // lane = (column group, token t): one 16-byte load of 8 columns of token t.  The lanes of tokens 2p and
+    // 2p + 1 then swap halves (the even one sends columns 2, 3, 6, 7 and gets the odd one's 0, 1, 4, 5), so
+    // that each holds both tokens of four columns and stores four 4-byte words xs[c][2p .. 2p + 1]: a
+    // quarter of the instructions of eight 2-byte stores with their selects.
+    uint32_t* xs32 = reinterpret_cast<uint32_t*>(cross_smem);
     constexpr int kLaneTok = TM < 32 ? TM : 32;
-    const int t = threadIdx.x % kLaneTok, cg = (threadIdx.x / kLaneTok) & 7;
+    static_assert(kLaneTok % 2 == 0, "token pairs");
+    const int t = threadIdx.x % kLaneTok;
+    const bool odd = (t & 1) != 0;
     const int64_t per_pass = static_cast<int64_t>(blockDim.x / kLaneTok) * 8;       // columns per pass of the block
     const bool valid = m0 + t < a.M;
     const __nv_bfloat16* row = a.x + (m0 + t) * a.K;
-    for (int64_t c8 = static_cast<int64_t>(threadIdx.x / kLaneTok) * 8; c8 < a.K; c8 += per_pass) {
+    const int64_t c_first = static_cast<int64_t>(threadIdx.x / kLaneTok) * 8;
+    for (int64_t base = 0; base < a.K; base += per_pass) {             // (uniform trip count: the swap needs both lanes)
+      const int64_t c8 = base + c_first;
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (valid) v = *reinterpret_cast<const uint4*>(row + c8);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int el = (i + cg) & 7;
-        const uint32_t w = el < 4 ? (el < 2 ? v.x : v.y) : (el < 6 ? v.z : v.w);      // selects, not an indexed array
-        xs16[(c8 + el) * TM + t] = static_cast<unsigned short>((el & 1) ? w >> 16 : w & 0xFFFFu);
+      if (valid && c8 < a.K) v = *reinterpret_cast<const uint4*>(row + c8);
+      const uint32_t r0 = __shfl_xor_sync(0xffffffffu, odd ? v.x : v.y, 1);
+      const uint32_t r1 = __shfl_xor_sync(0xffffffffu, odd ? v.z : v.w, 1);
+      const uint32_t k0 = odd ? v.y : v.x, k1 = odd ? v.w : v.z;       // columns (2, 3), (6, 7) or (0, 1), (4, 5) of this token
+      const uint32_t lo0 = odd ? r0 : k0, hi0 = odd ? k0 : r0;         // the even token goes to the low half of a word
+      const uint32_t lo1 = odd ? r1 : k1, hi1 = odd ? k1 : r1;
+      if (c8 < a.K) {
+        uint32_t* dst = xs32 + (c8 + (odd ? 2 : 0)) * (TM / 2) + (t >> 1);
+        dst[0] = prmt(lo0, hi0, 0x5410u);
+        dst[TM / 2] = prmt(lo0, hi0, 0x7632u);
+        dst[4 * (TM / 2)] = prmt(lo1, hi1, 0x5410u);
+        dst[5 * (TM / 2)] = prmt(lo1, hi1, 0x7632u);
       }
     }
   }
