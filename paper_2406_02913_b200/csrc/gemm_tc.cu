@@ -544,6 +544,40 @@ uint32_t cross_col_mask(int64_t K) {
   return (1u << bits) - 1u;
 }
 
+// All entries of a model in one launch: colk[e] = the column of entry e in the low 24 bits and the width of
+// its matrix's column field above them (pack_cross_colk)
+__global__ void pack_cross_records_all_kernel(const uint32_t* __restrict__ colk, const float* __restrict__ z, float eps,
+                                              int64_t n, uint32_t* __restrict__ rec) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const uint32_t ck = colk[i];
+  const uint32_t bits = ck >> 24, col_mask = (1u << bits) - 1u;
+  uint32_t b = __float_as_uint(eps * z[i]);
+  b += (col_mask >> 1) + ((b >> bits) & 1u);                          // to nearest, ties to even, at bit `bits`
+  rec[i] = (b & ~col_mask) | (ck & 0x00FFFFFFu);
+}
+__global__ void pack_cross_colk_kernel(const int32_t* __restrict__ col, int64_t n, uint32_t bits, uint32_t* __restrict__ colk) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i < n) colk[i] = static_cast<uint32_t>(col[i]) | (bits << 24);
+}
+
+szo_status pack_cross_colk(const szo_linear* p, uint32_t* colk, cudaStream_t st) {
+  if (p->nnz == 0) return SZO_OK;
+  SZO_REQUIRE(p->K <= (int64_t(1) << 18), SZO_ERR_UNSUPPORTED, "K = %lld too large for the paired form", (long long)p->K);
+  const uint32_t bits = 32u - static_cast<uint32_t>(__builtin_clz(cross_col_mask(p->K)));
+  pack_cross_colk_kernel<<<static_cast<unsigned>(ceil_div(p->nnz, 256)), 256, 0, st>>>(p->ent_col, p->nnz, bits, colk);
+  SZO_CHECK_LAUNCH("pack_cross_colk_kernel");
+  return SZO_OK;
+}
+
+szo_status pack_cross_records_all(const uint32_t* colk, const float* z, float eps, int64_t n, uint32_t* rec, cudaStream_t st) {
+  if (n == 0) return SZO_OK;
+  pack_cross_records_all_kernel<<<static_cast<unsigned>(ceil_div(n, 256)), 256, 0, st>>>(colk, z, eps, n, rec);
+  count_launch();
+  SZO_CHECK_LAUNCH("pack_cross_records_all_kernel");
+  return SZO_OK;
+}
+
 szo_status pack_cross_records(const int32_t* col, const float* z, float eps, int64_t n, int64_t K, uint32_t* rec,
                               cudaStream_t st) {
   if (n == 0) return SZO_OK;

@@ -113,6 +113,10 @@ bool tc_paired_dense_cross(const szo_linear* const* plans, int n);
 szo_status pack_cross_records(const int32_t* col, const float* z, float eps, int64_t n, int64_t K, uint32_t* rec,
                               cudaStream_t st);
 uint32_t cross_col_mask(int64_t K);
+// The records of many matrices in one launch: pack_cross_colk writes, once, (column | field width << 24) of a
+// plan's entries into its part of a model-wide array; pack_cross_records_all then packs all n entries.
+szo_status pack_cross_colk(const szo_linear* p, uint32_t* colk, cudaStream_t st);
+szo_status pack_cross_records_all(const uint32_t* colk, const float* z, float eps, int64_t n, uint32_t* rec, cudaStream_t st);
 size_t tc_paired_rec_bytes(const szo_linear* const* plans, int n);
 szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, const void* x, int64_t M,
                                       const float* const* S_pert, void* const* y, int y_dtype, void* ws,
