@@ -103,3 +103,43 @@ def test_graph_replay_of_token_steps_equals_the_launch_by_launch_form(B):
         m.close()
     assert torch.equal(outs[0], outs[1])
     assert torch.equal(outs[0][:7], outs[0][7:])             # the second pass over the same prompt repeats the first
+
+
+_SWITCH_SCRIPT = r"""
+import sys, numpy as np, torch
+from paper_2406_02913_b200 import binding as B, workloads as wl
+shape = dict(wl.MODEL_SHAPES["llama2_7b"], n_layers=2)
+tensors, S_all = wl.device_decoder_tensors(shape, seed=3)
+m = B.Model(shape, wl.linear_names(shape), tensors, S_all, act_dtype=B.SZO_BF16, linear_mode=B.MODE_SPARSE_ADD,
+            loss_kind=B.LOSS_LM, max_batch=2, max_seq=16)
+m.enable_decode()
+g = torch.Generator(device="cuda"); g.manual_seed(5)
+toks = torch.randint(0, shape["vocab"], (2, 8), generator=g, device="cuda", dtype=torch.int32)
+outs = [m.decode_step(toks[:, :3].contiguous(), 0).clone()]
+for i in range(3, 8):
+    outs.append(m.decode_step(toks[:, i:i + 1].contiguous(), i).clone())
+assert B.device_status() == 0
+np.save(sys.argv[1], torch.stack(outs).cpu().numpy())
+"""
+
+
+def test_switches_of_the_token_step_leave_the_bits_alone(tmp_path):
+    """The token step at the Llama-2-7B width (two layers, two sequences: the 16-row-group kernel with the norms
+    inside the projections, launched as a chain) against the same step with the norms in a kernel of their own
+    and with ordinary launches: the fused norm repeats the separate kernel's arithmetic and reduction tree, and a
+    chained launch changes when a kernel starts, not what it computes, so the logits must be the same bits.  The
+    switches are read once per process: one child process per setting."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = {}
+    for name, extra in (("default", {}), ("separate_norm", {"SZO_DECODE_FUSED_NORM": "0"}), ("no_chain", {"SZO_DECODE_CHAIN": "0"})):
+        out = str(tmp_path / (name + ".npy"))
+        r = subprocess.run([sys.executable, "-c", _SWITCH_SCRIPT, out], cwd=root, env=dict(os.environ, **extra),
+                           capture_output=True, text=True, timeout=600)
+        assert r.returncode == 0, name + ": " + r.stdout[-2000:] + r.stderr[-2000:]
+        res[name] = np.load(out)
+    assert np.isfinite(res["default"]).all()
+    assert np.array_equal(res["default"], res["separate_norm"])
+    assert np.array_equal(res["default"], res["no_chain"])
