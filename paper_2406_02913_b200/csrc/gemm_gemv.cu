@@ -198,22 +198,22 @@ __global__ void __launch_bounds__(kGvThreads, 2) szo_linear_gemv_kernel(const __
       fzc = s_begin % steps_per_qgroup;
     }
   };
+  const bool one_step_groups = steps_per_qgroup == 1;     // G = 128: a new (scale, zero) entry every step
   auto fetch = [&](uint4& wa, uint4& wb, float2& pa, float2& pb) {     // the step under the cursor, then advance it
     if (fg < total) {
-      wa = gv_ld_stream(fc);
-      wb = gv_ld_stream(fc + 8 * 32);
-      fc += 2 * 4096;
+      // (addresses from the step counter: a wide multiply-add each on the FMA pipe, where running pointers and
+      // their counters are four or five instructions on the ALU pipe, the busy one)
+      const uint8_t* src = fc + static_cast<int64_t>(fj) * (2 * 4096);
+      wa = gv_ld_stream(src);
+      wb = gv_ld_stream(src + 8 * 32);
       if constexpr (kLut) {
         const float4 tb = __ldg(reinterpret_cast<const float4*>(fz));     // (L2 after the group's first step)
         pa = make_float2(tb.x, tb.y);
         pb = make_float2(tb.z, tb.w);
       } else {
-        pa = __ldg(fz);
-        pb = __ldg(fz + 8);
-        if (++fzc == steps_per_qgroup) {
-          fzc = 0;
-          fz += fNpad;
-        }
+        const float2* z = fz + static_cast<int64_t>(one_step_groups ? fj : (fzc + fj) / steps_per_qgroup) * fNpad;
+        pa = __ldg(z);
+        pb = __ldg(z + 8);
       }
       if (++fj == n_my) {
         fj = 0;
