@@ -290,6 +290,42 @@ def sparse_pass_roofline(B, torch, k, peaks, launches=100):
     return out
 
 
+# ------------------------------------------------------------------------------------ token generation
+def token_generation(B, torch, model, shape, peaks, prompt=16, gen=128):
+    """Outside the timed steps, on the same model: a prompt of `prompt` tokens, then `gen` single-token steps of one
+    sequence with a KV cache (szo_model_decode_step, replayed as a CUDA graph), timed with CUDA events; every step
+    streams all weights once, so the roofline is the weight bytes over the HBM bandwidth."""
+    from paper_2406_02913_b200 import workloads as wl
+    model.enable_decode()
+    g = torch.Generator(device="cuda")
+    g.manual_seed(11)
+    toks = torch.randint(0, shape["vocab"], (1, prompt), generator=g, device="cuda", dtype=torch.int32)
+    logits = torch.empty((1, shape["vocab"]), dtype=torch.float32, device="cuda")
+    nxt = torch.empty((1, 1), dtype=torch.int32, device="cuda")
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        times = []
+        for rep_i in range(2):                                              # the first pass captures the graphs
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            model.decode_step(toks, 0, logits)
+            e0.record(stream)
+            for i in range(gen):
+                nxt.copy_(torch.argmax(logits, dim=1, keepdim=True))
+                model.decode_step(nxt, prompt + i, logits)
+            e1.record(stream)
+            stream.synchronize()
+            times.append(e0.elapsed_time(e1) / gen)
+    weight_bytes = 0
+    for nm in wl.linear_names(shape):
+        N, K = wl.linear_shape(shape, nm)
+        weight_bytes += N * K // 2 + 4 * N * K // shape["group"]
+    weight_bytes = weight_bytes * shape["n_layers"] + 2 * shape["vocab"] * shape["d_model"]
+    ms = times[-1]
+    return {"batch": 1, "prompt": prompt, "generated": gen, "ms_per_token_step": ms, "tokens_per_s": 1e3 / ms,
+            "weight_bytes_per_step": weight_bytes, "roofline_ms_per_step": weight_bytes / peaks["hbm_gbs"] / 1e6,
+            "frac_of_hbm": weight_bytes / peaks["hbm_gbs"] / 1e6 / ms, "device_status": B.device_status()}
+
+
 # ------------------------------------------------------------------------------------ GPU leg
 def run_ours(args):
     import torch
@@ -390,6 +426,7 @@ def run_ours(args):
     traffic, traffic_of = profiled_traffic()
     k_total = int(model.k_total)
     sparse = sparse_pass_roofline(B, torch, k_total, peaks)
+    decode = token_generation(B, torch, model, shape, peaks)
     cb, _ = oracle_sample(shape)
     cb["other_configs"] = oracle_small_configs()
     per_group = {"paired": "weight pass (int4 -> bf16), SparseAdd scatter of S, ONE szo_linear_tc2_kernel launch over "
@@ -412,6 +449,7 @@ def run_ours(args):
                      "linear_ms_per_step": lin_ms / args.steps,
                      "algorithmic_flops_per_step": 2 * flops_fwd},
         "roofline_sparse": sparse,
+        "token_generation": decode,
         "cpu_baseline": cb,
         "clocks": clk.summary(),
         "last_step": {"f_plus": float(last[0]), "f_minus": float(last[1]), "g": float(last[2])},
