@@ -44,6 +44,12 @@ MODEL_SHAPES = {
                      vocab=1024, max_pos=128, group=128, sz_fmt="bf16", rho=1e-3),
     "tiny_lut": dict(arch="llama", n_layers=2, d_model=256, n_heads=4, n_kv_heads=4, d_ff=1024,
                      vocab=1024, max_pos=0, group=-1, sz_fmt="f16", rho=1e-3),
+    # test shapes wide enough for the kernels of one or two tokens (K >= 896), with grouped-query attention, so
+    # that the q/k/v launch holds matrices of different heights
+    "small_gqa": dict(arch="llama", n_layers=2, d_model=1024, n_heads=16, n_kv_heads=4, d_ff=2816,
+                      vocab=1024, max_pos=0, group=128, sz_fmt="bf16", rho=2e-3),
+    "small_gqa_lut": dict(arch="llama", n_layers=2, d_model=1024, n_heads=16, n_kv_heads=4, d_ff=2816,
+                          vocab=1024, max_pos=0, group=-1, sz_fmt="f16", rho=2e-3),
     "llama2_7b_lut": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, n_kv_heads=32,
                           d_ff=11008, vocab=32000, max_pos=0, group=-1, sz_fmt="f16", rho=1e-3),
     "llama2_7b": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, n_kv_heads=32,

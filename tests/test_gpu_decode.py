@@ -62,6 +62,34 @@ def test_decode_steps_match_the_oracle(B, name, act):
     m.close()
 
 
+@pytest.mark.parametrize("name", ["small_gqa", "small_gqa_lut"])
+def test_token_steps_of_a_wider_grouped_query_decoder(B, name):
+    """Two layers of width 1024 with 16 query and 4 key/value heads (the q/k/v launch of the 16-row-group kernel
+    holds a 1024-row and two 256-row matrices; K = 1024 and 2816: 8 and 22 column steps for seven warps), uniform
+    int4 and table-coded weights: a prompt of 3, single tokens and a pair of tokens, for two sequences (cluster
+    kernel at 6 rows, the other kernel at 2) and for one, against the oracle's incremental decode."""
+    fx = DecoderFixture(name, seed=12, mask="random", B=2, S=16)
+    om = fx.oracle_model()
+    S_np = om.S + np.float32(1e-3)
+    lin_W = om.lin_W(S_np)
+    toks = fx.batch(0)[:, :8]
+    t = fx.gpu_tensors(torch, None)
+    S = torch.from_numpy(S_np.copy()).cuda()
+    m = B.Model(fx.shape, fx.names, t, S, act_dtype=B.SZO_BF16, linear_mode=B.MODE_SPARSE_ADD, max_batch=fx.B, max_seq=fx.S)
+    m.enable_decode()
+    for nseq in (2, 1):
+        cache = mo.KVCache(om.cfg.n_layers)
+        at = 0
+        for T in (3, 1, 1, 2):
+            tk = np.ascontiguousarray(toks[:nseq, at:at + T])
+            ref = mo.decode_step(om.cfg, om.params, lin_W, tk, cache).numpy()
+            got = m.decode_step(torch.from_numpy(tk).cuda(), at).cpu().numpy()
+            at += T
+            assert np.max(np.abs(got - ref)) <= 2e-2 * np.max(np.abs(ref)), (name, nseq, at)
+    assert B.device_status() == 0
+    m.close()
+
+
 def test_decode_argument_errors(B):
     fx = DecoderFixture("tiny", seed=6, mask="random", B=2, S=16, n_layers=1)
     t = fx.gpu_tensors(torch, None)
