@@ -387,15 +387,20 @@ template <int TM, int R, typename TY>
 __global__ void __launch_bounds__(TM == 16 ? 1024 : 512) pair_cross_kernel(const CrossArgs a) {
   using V = typename SlabVec<TM>::type;
   constexpr int kVecs = TM * 2 / static_cast<int>(sizeof(V));    // vectors per column
+  // The slab is kept in kVecs planes, plane q holding tokens q * kTokPlane .. of every column ([plane][K][kTokPlane]):
+  // a lane's 16-byte read of column c then falls into bank group c mod 8 (eight classes for the eight lanes of
+  // a quarter warp; with the two vectors of a column side by side there were four).  Plane 1 starts 64 bytes
+  // further, so that the staging stores of the two planes use different banks.
+  constexpr int kTokPlane = TM / kVecs;
   extern __shared__ __align__(16) unsigned char cross_smem[];
-  const V* xs = reinterpret_cast<const V*>(cross_smem);          // [K][kVecs]
+  const size_t plane_bytes = static_cast<size_t>(a.K) * kTokPlane * sizeof(__nv_bfloat16) + 64;
+  const unsigned char* xs = cross_smem;
   const int64_t m0 = static_cast<int64_t>(blockIdx.x) * TM;
   {
     // lane = (column group, token t): one 16-byte load of 8 columns of token t.  The lanes of tokens 2p and
     // 2p + 1 then swap halves (the even one sends columns 2, 3, 6, 7 and gets the odd one's 0, 1, 4, 5), so
     // that each holds both tokens of four columns and stores four 4-byte words xs[c][2p .. 2p + 1]: a
     // quarter of the instructions of eight 2-byte stores with their selects.
-    uint32_t* xs32 = reinterpret_cast<uint32_t*>(cross_smem);
     constexpr int kLaneTok = TM < 32 ? TM : 32;
     static_assert(kLaneTok % 2 == 0, "token pairs");
     const int t = threadIdx.x % kLaneTok;
@@ -414,11 +419,13 @@ __global__ void __launch_bounds__(TM == 16 ? 1024 : 512) pair_cross_kernel(const
       const uint32_t lo0 = odd ? r0 : k0, hi0 = odd ? k0 : r0;         // the even token goes to the low half of a word
       const uint32_t lo1 = odd ? r1 : k1, hi1 = odd ? k1 : r1;
       if (c8 < a.K) {
-        uint32_t* dst = xs32 + (c8 + (odd ? 2 : 0)) * (TM / 2) + (t >> 1);
+        constexpr int kWp = kTokPlane / 2;                             // words per column and plane
+        uint32_t* dst = reinterpret_cast<uint32_t*>(cross_smem + (t / kTokPlane) * plane_bytes) + (c8 + (odd ? 2 : 0)) * kWp +
+                        ((t % kTokPlane) >> 1);
         dst[0] = prmt(lo0, hi0, 0x5410u);
-        dst[TM / 2] = prmt(lo0, hi0, 0x7632u);
-        dst[4 * (TM / 2)] = prmt(lo1, hi1, 0x5410u);
-        dst[5 * (TM / 2)] = prmt(lo1, hi1, 0x7632u);
+        dst[kWp] = prmt(lo0, hi0, 0x7632u);
+        dst[4 * kWp] = prmt(lo1, hi1, 0x5410u);
+        dst[5 * kWp] = prmt(lo1, hi1, 0x7632u);
       }
     }
   }
@@ -448,7 +455,7 @@ __global__ void __launch_bounds__(TM == 16 ? 1024 : 512) pair_cross_kernel(const
           const uint32_t col = rc & a.col_mask;
 #pragma unroll
           for (int q = 0; q < kVecs; ++q) {
-            const V v = xs[col * kVecs + q];
+            const V v = *reinterpret_cast<const V*>(xs + q * plane_bytes + col * sizeof(V));
             const uint32_t* w = reinterpret_cast<const uint32_t*>(&v);
             constexpr int kW = static_cast<int>(sizeof(V)) / 4;
 #pragma unroll
@@ -506,7 +513,7 @@ __global__ void pack_cross_records_kernel(const int32_t* __restrict__ col, const
 
 template <int TM, int R, typename TY>
 szo_status launch_pair_cross(const CrossArgs& ca, int64_t max_N, cudaStream_t st) {
-  const size_t smem = static_cast<size_t>(ca.K) * TM * sizeof(__nv_bfloat16);
+  const size_t smem = static_cast<size_t>(ca.K) * TM * sizeof(__nv_bfloat16) + 128;       // (+ 64 per plane: see the kernel)
   SZO_CHECK_CUDA(cudaFuncSetAttribute(pair_cross_kernel<TM, R, TY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       static_cast<int>(smem)));
   // few token groups: the rows of a group go to several blocks (each stages the slab again), so that
