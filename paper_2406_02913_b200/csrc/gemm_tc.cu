@@ -5,6 +5,7 @@
 // schedule of the pair-tile kernel (gemm_tc2.cu) and its launch for one layer or for several layers
 // that read the same activations.
 #include <cstdlib>
+#include <vector>
 
 #include "tc_common.cuh"
 
@@ -51,6 +52,12 @@ struct TcPlan {
   int sms;
   int32_t* tickets;     // device, [sms / 2][2][4], zero between launches (K-split tiles of the pair kernel)
   uint64_t clean_epoch; // abort_epoch() when the tickets were last known to be zero
+  // Order in which pair_cross_kernel walks the entries of a weight row: record slot s (a position inside
+  // the row's CSR range) holds entry cross_perm[s] of the same row.  Chosen at plan creation so that the
+  // eight lanes of a quarter warp (eight rows two apart) read columns of different bank groups (column mod 8)
+  // in the same trip wherever the rows' entries allow it.  NULL: entry order (dense masks, which do not take
+  // that kernel, and plans without entries).
+  int32_t* cross_perm;
 };
 
 // Work schedule of the pair-tile kernel over `tiles` pair tiles (see TcParams).  The last, partial
@@ -117,8 +124,60 @@ static szo_status refresh_tickets(const TcPlan* tc, cudaStream_t st) {
   return SZO_OK;
 }
 
+// Host side (plan creation has synchronised; not on a step's path).  The kernel gives lane l of a warp the rows
+// 2 l and 2 l + 1 of a 64-row span and walks the even rows first, then the odd ones: the lanes of a quarter
+// warp thus read, in trip i, entry slot i of eight rows two apart.  For each such set of eight rows and each
+// trip, every row in turn takes one of its remaining entries whose bank group (column mod 8) no earlier row of
+// the trip has taken, or, failing that, its first remaining one.
+static szo_status build_cross_perm(const szo_linear* p, TcPlan* t) {
+  if (p->nnz == 0 || static_cast<double>(p->nnz) >= 0.002 * static_cast<double>(p->N) * static_cast<double>(p->K))
+    return SZO_OK;
+  const int64_t N = p->N;
+  std::vector<int32_t> rp(static_cast<size_t>(N) + 1), col(static_cast<size_t>(p->nnz)), perm(static_cast<size_t>(p->nnz));
+  SZO_CHECK_CUDA(cudaMemcpy(rp.data(), p->row_ptr, rp.size() * sizeof(int32_t), cudaMemcpyDeviceToHost));
+  SZO_CHECK_CUDA(cudaMemcpy(col.data(), p->ent_col, col.size() * sizeof(int32_t), cudaMemcpyDeviceToHost));
+  std::vector<char> taken;
+  for (int64_t n0 = 0; n0 < N; n0 += 16) {
+    for (int parity = 0; parity < 2; ++parity) {
+      int32_t maxlen = 0;
+      for (int l = 0; l < 8; ++l) {
+        const int64_t n = n0 + 2 * l + parity;
+        if (n < N && rp[n + 1] - rp[n] > maxlen) maxlen = rp[n + 1] - rp[n];
+      }
+      taken.assign(static_cast<size_t>(maxlen) * 8, 0);              // [lane][entry of the row]
+      for (int32_t i = 0; i < maxlen; ++i) {
+        unsigned used = 0;
+        for (int l = 0; l < 8; ++l) {
+          const int64_t n = n0 + 2 * l + parity;
+          if (n >= N) continue;
+          const int32_t b = rp[n], len = rp[n + 1] - b;
+          if (i >= len) continue;
+          int32_t pick = -1, first = -1;
+          for (int32_t j = 0; j < len; ++j) {
+            if (taken[static_cast<size_t>(l) * maxlen + j]) continue;
+            if (first < 0) first = j;
+            if (!(used >> (col[b + j] & 7) & 1u)) {
+              pick = j;
+              break;
+            }
+          }
+          if (pick < 0) pick = first;
+          taken[static_cast<size_t>(l) * maxlen + pick] = 1;
+          used |= 1u << (col[b + pick] & 7);
+          perm[b + i] = b + pick;
+        }
+      }
+    }
+  }
+  if (cudaMalloc(&t->cross_perm, perm.size() * sizeof(int32_t)) != cudaSuccess ||
+      cudaMemcpy(t->cross_perm, perm.data(), perm.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess)
+    return fail(SZO_ERR_CUDA, "cannot store the entry order of the sparse product");
+  return SZO_OK;
+}
+
 szo_status tc_plan_create(szo_linear* p, cudaStream_t) {
   TcPlan* t = new TcPlan();
+  t->cross_perm = nullptr;
   int dev = 0;
   t->sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&t->sms, cudaDevAttrMultiProcessorCount, dev);
@@ -138,12 +197,20 @@ szo_status tc_plan_create(szo_linear* p, cudaStream_t) {
   }
   t->clean_epoch = abort_epoch();
   p->tc = t;
+  const szo_status bs = build_cross_perm(p, t);
+  if (bs != SZO_OK) {
+    tc_plan_destroy(p);
+    return bs;
+  }
   return SZO_OK;
 }
 
 void tc_plan_destroy(szo_linear* p) {
   TcPlan* t = static_cast<TcPlan*>(p->tc);
-  if (t) cudaFree(t->tickets);
+  if (t) {
+    cudaFree(t->tickets);
+    cudaFree(t->cross_perm);
+  }
   delete t;
   p->tc = nullptr;
 }
@@ -502,13 +569,16 @@ __global__ void __launch_bounds__(TM == 16 ? 1024 : 512) pair_cross_kernel(const
 // rec[e] = the column of entry e in the low col_bits bits and, above them, fp32(eps * z[e]) rounded to
 // the nearest value with 32 - col_bits bits (sign, exponent and at least 9 bits of mantissa for K up
 // to 16384: 2^-10 relative, a quarter of a bf16 rounding, on a term that ends in a bf16 value)
-__global__ void pack_cross_records_kernel(const int32_t* __restrict__ col, const float* __restrict__ z, float eps,
-                                          int64_t n, uint32_t col_mask, uint32_t* __restrict__ rec) {
+// (perm: the plan's walking order of its entries, TcPlan::cross_perm, or NULL for entry order)
+__global__ void pack_cross_records_kernel(const int32_t* __restrict__ col, const int32_t* __restrict__ perm,
+                                          const float* __restrict__ z, float eps, int64_t n, uint32_t col_mask,
+                                          uint32_t* __restrict__ rec) {
   const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i >= n) return;
-  uint32_t b = __float_as_uint(eps * z[i]);
+  const int64_t e = perm != nullptr ? perm[i] : i;
+  uint32_t b = __float_as_uint(eps * z[e]);
   b += (col_mask >> 1) + ((b >> (32 - __clz(col_mask))) & 1u);       // to nearest, ties to even, at bit col_bits
-  rec[i] = (b & ~col_mask) | static_cast<uint32_t>(col[i]);
+  rec[i] = (b & ~col_mask) | static_cast<uint32_t>(col[e]);
 }
 
 template <int TM, int R, typename TY>
@@ -551,45 +621,54 @@ uint32_t cross_col_mask(int64_t K) {
   return (1u << bits) - 1u;
 }
 
-// All entries of a model in one launch: colk[e] = the column of entry e in the low 24 bits and the width of
-// its matrix's column field above them (pack_cross_colk)
-__global__ void pack_cross_records_all_kernel(const uint32_t* __restrict__ colk, const float* __restrict__ z, float eps,
-                                              int64_t n, uint32_t* __restrict__ rec) {
+// All entries of a model in one launch: colk[s] = the column of record slot s in the low 24 bits and the width of
+// its matrix's column field above them, src[s] = the entry (index into z) the slot holds (pack_cross_colk)
+__global__ void pack_cross_records_all_kernel(const uint32_t* __restrict__ colk, const int32_t* __restrict__ src,
+                                              const float* __restrict__ z, float eps, int64_t n, uint32_t* __restrict__ rec) {
   const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i >= n) return;
   const uint32_t ck = colk[i];
   const uint32_t bits = ck >> 24, col_mask = (1u << bits) - 1u;
-  uint32_t b = __float_as_uint(eps * z[i]);
+  uint32_t b = __float_as_uint(eps * z[src[i]]);
   b += (col_mask >> 1) + ((b >> bits) & 1u);                          // to nearest, ties to even, at bit `bits`
   rec[i] = (b & ~col_mask) | (ck & 0x00FFFFFFu);
 }
-__global__ void pack_cross_colk_kernel(const int32_t* __restrict__ col, int64_t n, uint32_t bits, uint32_t* __restrict__ colk) {
+__global__ void pack_cross_colk_kernel(const int32_t* __restrict__ col, const int32_t* __restrict__ perm, int64_t n,
+                                       uint32_t bits, int32_t base, uint32_t* __restrict__ colk, int32_t* __restrict__ src) {
   const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (i < n) colk[i] = static_cast<uint32_t>(col[i]) | (bits << 24);
+  if (i >= n) return;
+  const int32_t e = perm != nullptr ? perm[i] : static_cast<int32_t>(i);
+  colk[i] = static_cast<uint32_t>(col[e]) | (bits << 24);
+  src[i] = base + e;
 }
 
-szo_status pack_cross_colk(const szo_linear* p, uint32_t* colk, cudaStream_t st) {
+// colk, src: this plan's part of the model-wide arrays; base: where its entries start in the model's z
+szo_status pack_cross_colk(const szo_linear* p, int32_t base, uint32_t* colk, int32_t* src, cudaStream_t st) {
   if (p->nnz == 0) return SZO_OK;
   SZO_REQUIRE(p->K <= (int64_t(1) << 18), SZO_ERR_UNSUPPORTED, "K = %lld too large for the paired form", (long long)p->K);
   const uint32_t bits = 32u - static_cast<uint32_t>(__builtin_clz(cross_col_mask(p->K)));
-  pack_cross_colk_kernel<<<static_cast<unsigned>(ceil_div(p->nnz, 256)), 256, 0, st>>>(p->ent_col, p->nnz, bits, colk);
+  const TcPlan* t = static_cast<const TcPlan*>(p->tc);
+  pack_cross_colk_kernel<<<static_cast<unsigned>(ceil_div(p->nnz, 256)), 256, 0, st>>>(
+      p->ent_col, t != nullptr ? t->cross_perm : nullptr, p->nnz, bits, base, colk, src);
   SZO_CHECK_LAUNCH("pack_cross_colk_kernel");
   return SZO_OK;
 }
 
-szo_status pack_cross_records_all(const uint32_t* colk, const float* z, float eps, int64_t n, uint32_t* rec, cudaStream_t st) {
+szo_status pack_cross_records_all(const uint32_t* colk, const int32_t* src, const float* z, float eps, int64_t n, uint32_t* rec,
+                                  cudaStream_t st) {
   if (n == 0) return SZO_OK;
-  pack_cross_records_all_kernel<<<static_cast<unsigned>(ceil_div(n, 256)), 256, 0, st>>>(colk, z, eps, n, rec);
+  pack_cross_records_all_kernel<<<static_cast<unsigned>(ceil_div(n, 256)), 256, 0, st>>>(colk, src, z, eps, n, rec);
   count_launch();
   SZO_CHECK_LAUNCH("pack_cross_records_all_kernel");
   return SZO_OK;
 }
 
-szo_status pack_cross_records(const int32_t* col, const float* z, float eps, int64_t n, int64_t K, uint32_t* rec,
-                              cudaStream_t st) {
-  if (n == 0) return SZO_OK;
-  SZO_REQUIRE(K <= (int64_t(1) << 18), SZO_ERR_UNSUPPORTED, "K = %lld too large for the paired form", (long long)K);
-  pack_cross_records_kernel<<<static_cast<unsigned>(ceil_div(n, 256)), 256, 0, st>>>(col, z, eps, n, cross_col_mask(K), rec);
+szo_status pack_cross_records(const szo_linear* p, const float* z, float eps, uint32_t* rec, cudaStream_t st) {
+  if (p->nnz == 0) return SZO_OK;
+  SZO_REQUIRE(p->K <= (int64_t(1) << 18), SZO_ERR_UNSUPPORTED, "K = %lld too large for the paired form", (long long)p->K);
+  const TcPlan* t = static_cast<const TcPlan*>(p->tc);
+  pack_cross_records_kernel<<<static_cast<unsigned>(ceil_div(p->nnz, 256)), 256, 0, st>>>(
+      p->ent_col, t != nullptr ? t->cross_perm : nullptr, z, eps, p->nnz, cross_col_mask(p->K), rec);
   count_launch();
   SZO_CHECK_LAUNCH("pack_cross_records_kernel");
   return SZO_OK;

@@ -597,7 +597,7 @@ szo_status szo_linear_fwd_paired(const szo_linear_t* p, const void* x, int64_t M
   const size_t rec_bytes = tc_paired_rec_bytes(&pp, 1);
   uint32_t* rec = reinterpret_cast<uint32_t*>(static_cast<unsigned char*>(workspace) + (need - rec_bytes));
   const bool dense = tc_paired_dense_cross(&pp, 1);
-  SZO_TRY(pack_cross_records(p->ent_col, z, eps, p->nnz, p->K, rec, st));
+  SZO_TRY(pack_cross_records(p, z, eps, rec, st));
   const uint32_t* recs[1] = {rec};
   const PairedArgs pa{recs, &z, eps, dense};
   return linear_fwd_tc_materialised(&pp, 1, x, M, &S, &y, y_dtype, workspace, need - rec_bytes,

@@ -98,9 +98,8 @@ bool tc_use_materialised(const szo_linear* p, int64_t M, bool two_sets = false);
 size_t tc_materialised_ws_bytes(const szo_linear* const* plans, int n, int64_t M, bool ext = false);   // ext: rows 2 K wide
 // Paired form of a ZO step's two forwards (see tc::TcParams): x and every y[i] hold the M centre rows
 // first and the M half-difference rows from row round_up(M, 256) on; S_pert are the unperturbed sparse
-// values; rec[i][e] = column of entry e of plans[i] and eps * z_e in one word (pack_cross_records; the
-// split depends on K only, so one call may pack the entries of matrices with different K one after another
-// only if called per K).
+// values; rec[i][s] = column and eps * z of the entry that record slot s of plans[i] holds, in one word
+// (pack_cross_records: the slots of a weight row are its entries in the plan's walking order).
 // dense: the product runs on the tensor cores instead (eps * z written as a bf16 matrix beside W; z, eps
 // are used, rec is not).
 struct PairedArgs {
@@ -110,13 +109,13 @@ struct PairedArgs {
   bool dense;
 };
 bool tc_paired_dense_cross(const szo_linear* const* plans, int n);
-szo_status pack_cross_records(const int32_t* col, const float* z, float eps, int64_t n, int64_t K, uint32_t* rec,
-                              cudaStream_t st);
+szo_status pack_cross_records(const szo_linear* p, const float* z, float eps, uint32_t* rec, cudaStream_t st);
 uint32_t cross_col_mask(int64_t K);
 // The records of many matrices in one launch: pack_cross_colk writes, once, (column | field width << 24) of a
 // plan's entries into its part of a model-wide array; pack_cross_records_all then packs all n entries.
-szo_status pack_cross_colk(const szo_linear* p, uint32_t* colk, cudaStream_t st);
-szo_status pack_cross_records_all(const uint32_t* colk, const float* z, float eps, int64_t n, uint32_t* rec, cudaStream_t st);
+szo_status pack_cross_colk(const szo_linear* p, int32_t base, uint32_t* colk, int32_t* src, cudaStream_t st);
+szo_status pack_cross_records_all(const uint32_t* colk, const int32_t* src, const float* z, float eps, int64_t n, uint32_t* rec,
+                                  cudaStream_t st);
 size_t tc_paired_rec_bytes(const szo_linear* const* plans, int n);
 szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, const void* x, int64_t M,
                                       const float* const* S_pert, void* const* y, int y_dtype, void* ws,
