@@ -52,12 +52,6 @@ struct TcPlan {
   int sms;
   int32_t* tickets;     // device, [sms / 2][2][4], zero between launches (K-split tiles of the pair kernel)
   uint64_t clean_epoch; // abort_epoch() when the tickets were last known to be zero
-  // Order in which pair_cross_kernel walks the entries of a weight row: record slot s (a position inside
-  // the row's CSR range) holds entry cross_perm[s] of the same row.  Chosen at plan creation so that the
-  // eight lanes of a quarter warp (eight rows two apart) read columns of different bank groups (column mod 8)
-  // in the same trip wherever the rows' entries allow it.  NULL: entry order (dense masks, which do not take
-  // that kernel, and plans without entries).
-  int32_t* cross_perm;
 };
 
 // Work schedule of the pair-tile kernel over `tiles` pair tiles (see TcParams).  The last, partial
@@ -124,60 +118,8 @@ static szo_status refresh_tickets(const TcPlan* tc, cudaStream_t st) {
   return SZO_OK;
 }
 
-// Host side (plan creation has synchronised; not on a step's path).  The kernel gives lane l of a warp the rows
-// 2 l and 2 l + 1 of a 64-row span and walks the even rows first, then the odd ones: the lanes of a quarter
-// warp thus read, in trip i, entry slot i of eight rows two apart.  For each such set of eight rows and each
-// trip, every row in turn takes one of its remaining entries whose bank group (column mod 8) no earlier row of
-// the trip has taken, or, failing that, its first remaining one.
-static szo_status build_cross_perm(const szo_linear* p, TcPlan* t) {
-  if (p->nnz == 0 || static_cast<double>(p->nnz) >= 0.002 * static_cast<double>(p->N) * static_cast<double>(p->K))
-    return SZO_OK;
-  const int64_t N = p->N;
-  std::vector<int32_t> rp(static_cast<size_t>(N) + 1), col(static_cast<size_t>(p->nnz)), perm(static_cast<size_t>(p->nnz));
-  SZO_CHECK_CUDA(cudaMemcpy(rp.data(), p->row_ptr, rp.size() * sizeof(int32_t), cudaMemcpyDeviceToHost));
-  SZO_CHECK_CUDA(cudaMemcpy(col.data(), p->ent_col, col.size() * sizeof(int32_t), cudaMemcpyDeviceToHost));
-  std::vector<char> taken;
-  for (int64_t n0 = 0; n0 < N; n0 += 16) {
-    for (int parity = 0; parity < 2; ++parity) {
-      int32_t maxlen = 0;
-      for (int l = 0; l < 8; ++l) {
-        const int64_t n = n0 + 2 * l + parity;
-        if (n < N && rp[n + 1] - rp[n] > maxlen) maxlen = rp[n + 1] - rp[n];
-      }
-      taken.assign(static_cast<size_t>(maxlen) * 8, 0);              // [lane][entry of the row]
-      for (int32_t i = 0; i < maxlen; ++i) {
-        unsigned used = 0;
-        for (int l = 0; l < 8; ++l) {
-          const int64_t n = n0 + 2 * l + parity;
-          if (n >= N) continue;
-          const int32_t b = rp[n], len = rp[n + 1] - b;
-          if (i >= len) continue;
-          int32_t pick = -1, first = -1;
-          for (int32_t j = 0; j < len; ++j) {
-            if (taken[static_cast<size_t>(l) * maxlen + j]) continue;
-            if (first < 0) first = j;
-            if (!(used >> (col[b + j] & 7) & 1u)) {
-              pick = j;
-              break;
-            }
-          }
-          if (pick < 0) pick = first;
-          taken[static_cast<size_t>(l) * maxlen + pick] = 1;
-          used |= 1u << (col[b + pick] & 7);
-          perm[b + i] = b + pick;
-        }
-      }
-    }
-  }
-  if (cudaMalloc(&t->cross_perm, perm.size() * sizeof(int32_t)) != cudaSuccess ||
-      cudaMemcpy(t->cross_perm, perm.data(), perm.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess)
-    return fail(SZO_ERR_CUDA, "cannot store the entry order of the sparse product");
-  return SZO_OK;
-}
-
 szo_status tc_plan_create(szo_linear* p, cudaStream_t) {
   TcPlan* t = new TcPlan();
-  t->cross_perm = nullptr;
   int dev = 0;
   t->sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&t->sms, cudaDevAttrMultiProcessorCount, dev);
@@ -197,7 +139,7 @@ szo_status tc_plan_create(szo_linear* p, cudaStream_t) {
   }
   t->clean_epoch = abort_epoch();
   p->tc = t;
-  const szo_status bs = build_cross_perm(p, t);
+  const szo_status bs = cross_plan_create(p);
   if (bs != SZO_OK) {
     tc_plan_destroy(p);
     return bs;
@@ -207,11 +149,9 @@ szo_status tc_plan_create(szo_linear* p, cudaStream_t) {
 
 void tc_plan_destroy(szo_linear* p) {
   TcPlan* t = static_cast<TcPlan*>(p->tc);
-  if (t) {
-    cudaFree(t->tickets);
-    cudaFree(t->cross_perm);
-  }
+  if (t) cudaFree(t->tickets);
   delete t;
+  cross_plan_destroy(p);
   p->tc = nullptr;
 }
 
@@ -404,275 +344,7 @@ __global__ void scatter_add_bf16_kernel(const MatArgs a) {
   *el = __float2bfloat16_rn(__bfloat162float(base) + S[e]);
 }
 
-// Sparse product of the paired form: yd[t][n] += eps * sum_e z_e * xc[t][col_e] over the sensitive entries e
-// of weight row n (Zbar of Definition 4 times the centre activations), for the M half-difference
-// rows of up to three matrices that share x; runs after the tensor-core launch that wrote xd W^T into
-// those rows.  The sum is formed in fp32 and added to the stored value, one rounding (the
-// half-difference has its own exponent, so a second bf16 rounding costs 2^-9 of ITS size, not of
-// the centre's).
-// A block owns TM tokens and a share of the weight rows: it stages xc[those tokens][all K columns] in
-// shared memory transposed, xs[c][TM] (16-byte reads along the token rows, 2-byte stores rotated so
-// that the four column groups of a warp hit different banks), then each thread walks weight rows:
-// every entry is one 16-byte (TM = 8) read of shared memory and TM fused multiply-adds; y is read and
-// written 64 contiguous bytes per token and warp.  Tried first: columns of a transposed copy of xc
-// read from L2 per entry (8 KB per entry, 2.6 TB/s: 20 ms of a Llama-2-7B-shaped step), and the slab
-// copied from that transposed copy (16 bytes every 8 KB: the strided reads camp on a few L2 slices,
-// 25 ms).  The epilogue of the tensor-core kernel is on that kernel's critical path
-// (adding this sum there, from xT or from a buffer, made the decoder-block linears 45 % slower), which
-// is why it is a pass of its own.
-struct CrossSub {
-  const int32_t* row_ptr;
-  const uint32_t* rec;   // per entry: column in the low col_bits bits, the leading bits of fp32(eps * z) above them
-  void* yd;              // first half-difference row of this matrix's y
-  int64_t N;
-};
-struct CrossArgs {
-  CrossSub sub[3];
-  int n;
-  const __nv_bfloat16* x;   // centre rows [M][K]
-  int64_t M, K;
-  uint32_t col_mask;        // (1 << col_bits) - 1, col_bits = bits needed for K - 1
-};
-template <int TM> struct SlabVec;
-template <> struct SlabVec<16> { using type = uint4; };   // two per column
-template <> struct SlabVec<8> { using type = uint4; };
-template <> struct SlabVec<4> { using type = uint2; };
-template <> struct SlabVec<2> { using type = uint32_t; };
-
-// R weight rows per thread (2 when N is even: y is then read and written four bytes per lane).  The rows of
-// a lane are walked one after the other, and a warp runs each walk as long as its longest row: at 4
-// entries per row that is about twice the mean.  Giving lane l the l-th longest and the l-th shortest
-// row of a 64-row group instead (so that lanes finish together) measured 16 % slower: the walks are
-// still separate loops, and the two rows of a lane are then no longer adjacent (two-byte accesses to y).
-// A sorted-slice layout (rows of a 256-row window ordered by entry count, 32 equally long rows per warp,
-// records of a trip side by side, sums passed through a shared-memory tile and added to y eight bytes at
-// a time by four independent thread groups per block) removed the idle lanes (119 M instructions
-// against 140 M) but tripled the shared-memory wavefronts (37 M, 22 M of them bank conflicts: all
-// 32 lanes now read random columns, and the tile is written at random rows): 265 us against 211 at
-// K = 4096, 3 % ahead at K = 11008; not kept.
-template <int TM, int R, typename TY>
-__global__ void __launch_bounds__(TM == 16 ? 1024 : 512) pair_cross_kernel(const CrossArgs a) {
-  using V = typename SlabVec<TM>::type;
-  constexpr int kVecs = TM * 2 / static_cast<int>(sizeof(V));    // vectors per column
-  // The slab is kept in kVecs planes, plane q holding tokens q * kTokPlane .. of every column ([plane][K][kTokPlane]):
-  // a lane's 16-byte read of column c then falls into bank group c mod 8 (eight classes for the eight lanes of
-  // a quarter warp; with the two vectors of a column side by side there were four).  Plane 1 starts 64 bytes
-  // further, so that the staging stores of the two planes use different banks.
-  constexpr int kTokPlane = TM / kVecs;
-  extern __shared__ __align__(16) unsigned char cross_smem[];
-  const size_t plane_bytes = static_cast<size_t>(a.K) * kTokPlane * sizeof(__nv_bfloat16) + 64;
-  const unsigned char* xs = cross_smem;
-  const int64_t m0 = static_cast<int64_t>(blockIdx.x) * TM;
-  {
-    // lane = (column group, token t): one 16-byte load of 8 columns of token t.  The lanes of tokens 2p and
-    // 2p + 1 then swap halves (the even one sends columns 2, 3, 6, 7 and gets the odd one's 0, 1, 4, 5), so
-    // that each holds both tokens of four columns and stores four 4-byte words xs[c][2p .. 2p + 1]: a
-    // quarter of the instructions of eight 2-byte stores with their selects.
-    constexpr int kLaneTok = TM < 32 ? TM : 32;
-    static_assert(kLaneTok % 2 == 0, "token pairs");
-    const int t = threadIdx.x % kLaneTok;
-    const bool odd = (t & 1) != 0;
-    const int64_t per_pass = static_cast<int64_t>(blockDim.x / kLaneTok) * 8;       // columns per pass of the block
-    const bool valid = m0 + t < a.M;
-    const __nv_bfloat16* row = a.x + (m0 + t) * a.K;
-    const int64_t c_first = static_cast<int64_t>(threadIdx.x / kLaneTok) * 8;
-    for (int64_t base = 0; base < a.K; base += per_pass) {             // (uniform trip count: the swap needs both lanes)
-      const int64_t c8 = base + c_first;
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (valid && c8 < a.K) v = *reinterpret_cast<const uint4*>(row + c8);
-      const uint32_t r0 = __shfl_xor_sync(0xffffffffu, odd ? v.x : v.y, 1);
-      const uint32_t r1 = __shfl_xor_sync(0xffffffffu, odd ? v.z : v.w, 1);
-      const uint32_t k0 = odd ? v.y : v.x, k1 = odd ? v.w : v.z;       // columns (2, 3), (6, 7) or (0, 1), (4, 5) of this token
-      const uint32_t lo0 = odd ? r0 : k0, hi0 = odd ? k0 : r0;         // the even token goes to the low half of a word
-      const uint32_t lo1 = odd ? r1 : k1, hi1 = odd ? k1 : r1;
-      if (c8 < a.K) {
-        constexpr int kWp = kTokPlane / 2;                             // words per column and plane
-        uint32_t* dst = reinterpret_cast<uint32_t*>(cross_smem + (t / kTokPlane) * plane_bytes) + (c8 + (odd ? 2 : 0)) * kWp +
-                        ((t % kTokPlane) >> 1);
-        dst[0] = prmt(lo0, hi0, 0x5410u);
-        dst[kWp] = prmt(lo0, hi0, 0x7632u);
-        dst[4 * kWp] = prmt(lo1, hi1, 0x5410u);
-        dst[5 * kWp] = prmt(lo1, hi1, 0x7632u);
-      }
-    }
-  }
-  __syncthreads();
-  const int cnt = static_cast<int>(a.M - m0 < TM ? a.M - m0 : TM);
-  for (int s = 0; s < a.n; ++s) {
-    const int32_t* row_ptr = s == 0 ? a.sub[0].row_ptr : (s == 1 ? a.sub[1].row_ptr : a.sub[2].row_ptr);
-    if (row_ptr == nullptr) continue;
-    const uint32_t* rec = s == 0 ? a.sub[0].rec : (s == 1 ? a.sub[1].rec : a.sub[2].rec);
-    TY* yd = static_cast<TY*>(s == 0 ? a.sub[0].yd : (s == 1 ? a.sub[1].yd : a.sub[2].yd));
-    const int64_t N = s == 0 ? a.sub[0].N : (s == 1 ? a.sub[1].N : a.sub[2].N);
-    // the row shares of the gridDim.y blocks of a token group interleave in units of the block size
-    for (int64_t n = (static_cast<int64_t>(blockIdx.y) * blockDim.x + threadIdx.x) * R; n < N;
-         n += static_cast<int64_t>(gridDim.y) * blockDim.x * R) {
-      int32_t eb[R + 1];
-#pragma unroll
-      for (int r = 0; r <= R; ++r) eb[r] = __ldg(row_ptr + (n + r <= N ? n + r : N));
-      if (eb[0] == eb[R]) continue;
-      float acc[R][TM];
-#pragma unroll
-      for (int r = 0; r < R; ++r) {
-#pragma unroll
-        for (int j = 0; j < TM; ++j) acc[r][j] = 0.f;
-        for (int32_t e = eb[r]; e < eb[r + 1]; ++e) {
-          const uint32_t rc = __ldg(rec + e);
-          const float zz = __uint_as_float(rc & ~a.col_mask);
-          const uint32_t col = rc & a.col_mask;
-#pragma unroll
-          for (int q = 0; q < kVecs; ++q) {
-            const V v = *reinterpret_cast<const V*>(xs + q * plane_bytes + col * sizeof(V));
-            const uint32_t* w = reinterpret_cast<const uint32_t*>(&v);
-            constexpr int kW = static_cast<int>(sizeof(V)) / 4;
-#pragma unroll
-            for (int h = 0; h < kW; ++h) {
-              acc[r][q * kW * 2 + 2 * h] = fmaf(zz, __uint_as_float(w[h] << 16), acc[r][q * kW * 2 + 2 * h]);
-              acc[r][q * kW * 2 + 2 * h + 1] = fmaf(zz, __uint_as_float(w[h] & 0xFFFF0000u), acc[r][q * kW * 2 + 2 * h + 1]);
-            }
-          }
-        }
-      }
-      TY* yp = yd + m0 * N + n;
-      if constexpr (R == 2 && sizeof(TY) == 2) {
-        uint32_t old[TM];
-#pragma unroll
-        for (int j = 0; j < TM; ++j) old[j] = (j < cnt) ? *reinterpret_cast<const uint32_t*>(yp + j * N) : 0u;
-#pragma unroll
-        for (int j = 0; j < TM; ++j) {
-          if (j < cnt) {
-            const __nv_bfloat162 o = __floats2bfloat162_rn(__uint_as_float(old[j] << 16) + acc[0][j],
-                                                            __uint_as_float(old[j] & 0xFFFF0000u) + acc[1][j]);
-            *reinterpret_cast<__nv_bfloat162*>(yp + j * N) = o;
-          }
-        }
-      } else {
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-          if (n + r >= N) continue;
-          float old[TM];
-#pragma unroll
-          for (int j = 0; j < TM; ++j) old[j] = (j < cnt) ? static_cast<float>(yp[j * N + r]) : 0.f;
-#pragma unroll
-          for (int j = 0; j < TM; ++j) {
-            if (j < cnt) {
-              if constexpr (sizeof(TY) == 2) yp[j * N + r] = __float2bfloat16_rn(old[j] + acc[r][j]);
-              else yp[j * N + r] = old[j] + acc[r][j];
-            }
-          }
-        }
-      }
-    }
-  }
-}
-
-// rec[e] = the column of entry e in the low col_bits bits and, above them, fp32(eps * z[e]) rounded to
-// the nearest value with 32 - col_bits bits (sign, exponent and at least 9 bits of mantissa for K up
-// to 16384: 2^-10 relative, a quarter of a bf16 rounding, on a term that ends in a bf16 value)
-// (perm: the plan's walking order of its entries, TcPlan::cross_perm, or NULL for entry order)
-__global__ void pack_cross_records_kernel(const int32_t* __restrict__ col, const int32_t* __restrict__ perm,
-                                          const float* __restrict__ z, float eps, int64_t n, uint32_t col_mask,
-                                          uint32_t* __restrict__ rec) {
-  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  const int64_t e = perm != nullptr ? perm[i] : i;
-  uint32_t b = __float_as_uint(eps * z[e]);
-  b += (col_mask >> 1) + ((b >> (32 - __clz(col_mask))) & 1u);       // to nearest, ties to even, at bit col_bits
-  rec[i] = (b & ~col_mask) | static_cast<uint32_t>(col[e]);
-}
-
-template <int TM, int R, typename TY>
-szo_status launch_pair_cross(const CrossArgs& ca, int64_t max_N, cudaStream_t st) {
-  const size_t smem = static_cast<size_t>(ca.K) * TM * sizeof(__nv_bfloat16) + 128;       // (+ 64 per plane: see the kernel)
-  SZO_CHECK_CUDA(cudaFuncSetAttribute(pair_cross_kernel<TM, R, TY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      static_cast<int>(smem)));
-  // few token groups: the rows of a group go to several blocks (each stages the slab again), so that
-  // the grid covers the SMs
-  const int64_t groups = ceil_div(ca.M, TM);
-  int row_split = static_cast<int>(ceil_div(296, groups));
-  constexpr int kThreads = TM == 16 ? 1024 : 512;
-  const int64_t max_split = ceil_div(max_N, kThreads * R);
-  if (row_split > max_split) row_split = static_cast<int>(max_split);
-  if (row_split < 1) row_split = 1;
-  dim3 grid(static_cast<unsigned>(groups), static_cast<unsigned>(row_split));
-  pair_cross_kernel<TM, R, TY><<<grid, kThreads, smem, st>>>(ca);
-  count_launch();
-  SZO_CHECK_LAUNCH("pair_cross_kernel");
-  return SZO_OK;
-}
-template <int TM>
-szo_status launch_pair_cross_tm(const CrossArgs& ca, int64_t max_N, bool even, bool f32, cudaStream_t st) {
-  if (f32) return launch_pair_cross<TM, 1, float>(ca, max_N, st);
-  if (even) return launch_pair_cross<TM, 2, __nv_bfloat16>(ca, max_N, st);
-  return launch_pair_cross<TM, 1, __nv_bfloat16>(ca, max_N, st);
-}
-
 }  // namespace
-
-size_t tc_paired_rec_bytes(const szo_linear* const* plans, int n) {
-  size_t nnz = 0;
-  for (int i = 0; i < n; ++i) nnz += static_cast<size_t>(plans[i]->nnz);
-  return round_up(nnz * sizeof(uint32_t), 256);
-}
-
-uint32_t cross_col_mask(int64_t K) {
-  uint32_t bits = 1;
-  while ((int64_t(1) << bits) < K) ++bits;
-  return (1u << bits) - 1u;
-}
-
-// All entries of a model in one launch: colk[s] = the column of record slot s in the low 24 bits and the width of
-// its matrix's column field above them, src[s] = the entry (index into z) the slot holds (pack_cross_colk)
-__global__ void pack_cross_records_all_kernel(const uint32_t* __restrict__ colk, const int32_t* __restrict__ src,
-                                              const float* __restrict__ z, float eps, int64_t n, uint32_t* __restrict__ rec) {
-  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  const uint32_t ck = colk[i];
-  const uint32_t bits = ck >> 24, col_mask = (1u << bits) - 1u;
-  uint32_t b = __float_as_uint(eps * z[src[i]]);
-  b += (col_mask >> 1) + ((b >> bits) & 1u);                          // to nearest, ties to even, at bit `bits`
-  rec[i] = (b & ~col_mask) | (ck & 0x00FFFFFFu);
-}
-__global__ void pack_cross_colk_kernel(const int32_t* __restrict__ col, const int32_t* __restrict__ perm, int64_t n,
-                                       uint32_t bits, int32_t base, uint32_t* __restrict__ colk, int32_t* __restrict__ src) {
-  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  const int32_t e = perm != nullptr ? perm[i] : static_cast<int32_t>(i);
-  colk[i] = static_cast<uint32_t>(col[e]) | (bits << 24);
-  src[i] = base + e;
-}
-
-// colk, src: this plan's part of the model-wide arrays; base: where its entries start in the model's z
-szo_status pack_cross_colk(const szo_linear* p, int32_t base, uint32_t* colk, int32_t* src, cudaStream_t st) {
-  if (p->nnz == 0) return SZO_OK;
-  SZO_REQUIRE(p->K <= (int64_t(1) << 18), SZO_ERR_UNSUPPORTED, "K = %lld too large for the paired form", (long long)p->K);
-  const uint32_t bits = 32u - static_cast<uint32_t>(__builtin_clz(cross_col_mask(p->K)));
-  const TcPlan* t = static_cast<const TcPlan*>(p->tc);
-  pack_cross_colk_kernel<<<static_cast<unsigned>(ceil_div(p->nnz, 256)), 256, 0, st>>>(
-      p->ent_col, t != nullptr ? t->cross_perm : nullptr, p->nnz, bits, base, colk, src);
-  SZO_CHECK_LAUNCH("pack_cross_colk_kernel");
-  return SZO_OK;
-}
-
-szo_status pack_cross_records_all(const uint32_t* colk, const int32_t* src, const float* z, float eps, int64_t n, uint32_t* rec,
-                                  cudaStream_t st) {
-  if (n == 0) return SZO_OK;
-  pack_cross_records_all_kernel<<<static_cast<unsigned>(ceil_div(n, 256)), 256, 0, st>>>(colk, src, z, eps, n, rec);
-  count_launch();
-  SZO_CHECK_LAUNCH("pack_cross_records_all_kernel");
-  return SZO_OK;
-}
-
-szo_status pack_cross_records(const szo_linear* p, const float* z, float eps, uint32_t* rec, cudaStream_t st) {
-  if (p->nnz == 0) return SZO_OK;
-  SZO_REQUIRE(p->K <= (int64_t(1) << 18), SZO_ERR_UNSUPPORTED, "K = %lld too large for the paired form", (long long)p->K);
-  const TcPlan* t = static_cast<const TcPlan*>(p->tc);
-  pack_cross_records_kernel<<<static_cast<unsigned>(ceil_div(p->nnz, 256)), 256, 0, st>>>(
-      p->ent_col, t != nullptr ? t->cross_perm : nullptr, z, eps, p->nnz, cross_col_mask(p->K), rec);
-  count_launch();
-  SZO_CHECK_LAUNCH("pack_cross_records_kernel");
-  return SZO_OK;
-}
 
 namespace {
 
@@ -959,33 +631,9 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
     SZO_TRY(launch_pair_kernel(false, false, mx, mw, P, sc.n_pairs, st));
   }
   if (paired != nullptr && nnz_all > 0 && !ext) {
-    CrossArgs ca{};
-    ca.n = n; ca.x = static_cast<const __nv_bfloat16*>(x); ca.M = M; ca.K = p0->K;
-    ca.col_mask = cross_col_mask(p0->K);
-    const size_t y_el = (y_dtype == SZO_F32) ? 4 : 2;
-    int64_t max_N = 0;
-    bool even = true;
-    for (int i = 0; i < n; ++i) {
-      const szo_linear* p = plans[i];
-      if (p->N > max_N) max_N = p->N;
-      if (p->N & 1) even = false;
-      ca.sub[i] = CrossSub{p->nnz > 0 ? p->row_ptr : nullptr, paired->rec[i],
-                           static_cast<unsigned char*>(y[i]) + static_cast<size_t>(Mp) * p->N * y_el, p->N};
-    }
-    const size_t per_token = static_cast<size_t>(p0->K) * sizeof(__nv_bfloat16);
-    const bool f32 = y_dtype == SZO_F32;
-    static const int tm_env = [] {
-      const char* e = getenv("SZO_CROSS_TM");
-      return e == nullptr ? 0 : atoi(e);
-    }();
-    if (tm_env == 8 && 8 * per_token <= 200 * 1024) SZO_TRY(launch_pair_cross_tm<8>(ca, max_N, even, f32, st));
-    else if (16 * per_token <= 200 * 1024 && M >= 2048) SZO_TRY(launch_pair_cross_tm<16>(ca, max_N, even, f32, st));
-    else if (8 * per_token <= 200 * 1024) SZO_TRY(launch_pair_cross_tm<8>(ca, max_N, even, f32, st));
-    else if (4 * per_token <= 200 * 1024) SZO_TRY(launch_pair_cross_tm<4>(ca, max_N, even, f32, st));
-    else {
-      SZO_REQUIRE(2 * per_token <= 200 * 1024, SZO_ERR_UNSUPPORTED, "K = %lld too large for the paired form", (long long)p0->K);
-      SZO_TRY(launch_pair_cross_tm<2>(ca, max_N, even, f32, st));
-    }
+    void* yd[3];
+    for (int i = 0; i < n; ++i) yd[i] = static_cast<unsigned char*>(y[i]) + static_cast<size_t>(Mp) * plans[i]->N * y_elt;
+    SZO_TRY(launch_paired_cross(plans, n, x, M, paired->rec, yd, y_dtype, st));
   }
   return SZO_OK;
 }

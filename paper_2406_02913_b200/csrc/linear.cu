@@ -572,7 +572,7 @@ szo_status szo_linear_fwd(const szo_linear_t* p, const void* x, szo_dtype x_dtyp
 size_t szo_linear_paired_workspace_bytes(const szo_linear_t* p, int64_t M) {
   if (!p || M <= 0 || p->tc == nullptr) return 0;
   const szo_linear* pp = p;
-  return tc_materialised_ws_bytes(&pp, 1, M, tc_paired_dense_cross(&pp, 1)) + tc_paired_rec_bytes(&pp, 1);
+  return tc_materialised_ws_bytes(&pp, 1, M, tc_paired_dense_cross(&pp, 1)) + cross_rec_bytes(&pp, 1);
 }
 
 szo_status szo_linear_fwd_paired(const szo_linear_t* p, const void* x, int64_t M, const float* S, const float* z,
@@ -594,7 +594,7 @@ szo_status szo_linear_fwd_paired(const szo_linear_t* p, const void* x, int64_t M
               "the paired form needs a workspace of %zu bytes", need);
   const szo_linear* pp = p;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const size_t rec_bytes = tc_paired_rec_bytes(&pp, 1);
+  const size_t rec_bytes = cross_rec_bytes(&pp, 1);
   uint32_t* rec = reinterpret_cast<uint32_t*>(static_cast<unsigned char*>(workspace) + (need - rec_bytes));
   const bool dense = tc_paired_dense_cross(&pp, 1);
   SZO_TRY(pack_cross_records(p, z, eps, rec, st));

@@ -25,6 +25,7 @@ struct szo_linear {
   uint16_t* bucket_pos;  // [nnz] byte offset of the element inside its swizzled [128 x 64] bf16 tile, bucket order
   int64_t n_rowgroups, n_kblocks;
   void* tc;              // tensor-core side data (tensor maps), owned; see gemm_tc.cu
+  void* cross;           // record layout of the paired form's sparse product, owned; see cross.cu (NULL: no entries)
   const void* lut;           // caller-owned table [N][16] (G == -1), 16-bit floats of type sz_dtype
   __nv_bfloat16* lut_bf16;   // owned: [Npad][16], RN_bf16 of the table, padding rows zero
 };
@@ -98,8 +99,7 @@ bool tc_use_materialised(const szo_linear* p, int64_t M, bool two_sets = false);
 size_t tc_materialised_ws_bytes(const szo_linear* const* plans, int n, int64_t M, bool ext = false);   // ext: rows 2 K wide
 // Paired form of a ZO step's two forwards (see tc::TcParams): x and every y[i] hold the M centre rows
 // first and the M half-difference rows from row round_up(M, 256) on; S_pert are the unperturbed sparse
-// values; rec[i][s] = column and eps * z of the entry that record slot s of plans[i] holds, in one word
-// (pack_cross_records: the slots of a weight row are its entries in the plan's walking order).
+// values; rec[i] = the packed records of plans[i] (cross.cu).
 // dense: the product runs on the tensor cores instead (eps * z written as a bf16 matrix beside W; z, eps
 // are used, rec is not).
 struct PairedArgs {
@@ -109,14 +109,22 @@ struct PairedArgs {
   bool dense;
 };
 bool tc_paired_dense_cross(const szo_linear* const* plans, int n);
+// Sparse product of the paired form (cross.cu).  A plan has one record slot per entry (the entries of a weight
+// row in the order the kernel walks them); a record is one word, column and eps * z.
+szo_status cross_plan_create(szo_linear* p);     // called by tc_plan_create; needs row_ptr and ent_col
+void cross_plan_destroy(szo_linear* p);
+size_t cross_rec_bytes(const szo_linear* const* plans, int n);
+// rec[s] for the slots of one plan; z: the plan's entries
 szo_status pack_cross_records(const szo_linear* p, const float* z, float eps, uint32_t* rec, cudaStream_t st);
-uint32_t cross_col_mask(int64_t K);
-// The records of many matrices in one launch: pack_cross_colk writes, once, (column | field width << 24) of a
-// plan's entries into its part of a model-wide array; pack_cross_records_all then packs all n entries.
-szo_status pack_cross_colk(const szo_linear* p, int32_t base, uint32_t* colk, int32_t* src, cudaStream_t st);
+// The records of many matrices in one launch: cross_copy_slots writes, once, a plan's slot descriptions into
+// its part of model-wide arrays (src offset by base, where the plan's entries start in the model's z);
+// pack_cross_records_all then packs all n slots.
+szo_status cross_copy_slots(const szo_linear* p, int32_t base, uint32_t* colk, int32_t* src, cudaStream_t st);
 szo_status pack_cross_records_all(const uint32_t* colk, const int32_t* src, const float* z, float eps, int64_t n, uint32_t* rec,
                                   cudaStream_t st);
-size_t tc_paired_rec_bytes(const szo_linear* const* plans, int n);
+// yd[i]: first half-difference row of plans[i]'s y; x: the centre rows
+szo_status launch_paired_cross(const szo_linear* const* plans, int n, const void* x, int64_t M, const uint32_t* const* rec,
+                               void* const* yd, int y_dtype, cudaStream_t st);
 szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, const void* x, int64_t M,
                                       const float* const* S_pert, void* const* y, int y_dtype, void* ws,
                                       size_t ws_bytes, cudaStream_t st, const float* const* S_second = nullptr,

@@ -935,11 +935,13 @@ struct szo_model {
   float* S_all = nullptr;
   int64_t k_total = 0;
   int64_t* gidx = nullptr;
-  uint32_t* colk = nullptr;              // [k_total] per record slot: column | width of the column field << 24 (paired form)
-  int32_t* csrc = nullptr;               // [k_total] per record slot: the entry (index into S_all / z) it holds
+  // paired form, sparse product: linear t's record slots are [offsets[t], offsets[t + 1]) of these arrays
+  uint32_t* colk = nullptr;              // per slot: column | width of the column field << 24
+  int32_t* csrc = nullptr;               // per slot: the entry (index into S_all / z) it holds
+  uint32_t* crecs = nullptr;             // per slot: the record of the current step
   int32_t* geid = nullptr;      // [k_total] entry id in S_all of each bucket-ordered record
   uint16_t* gpos = nullptr;     // [k_total] in-tile position of each bucket-ordered record
-  uint2* recs = nullptr;        // [k_total] (position, value) records of the current forward; paired form: (column, eps z)
+  uint2* recs = nullptr;        // [k_total] (position, value) records of the current forward
   float* zkept = nullptr;       // [k_total] z of the current step, kept by the first perturb pass
   float *Splus = nullptr, *Sminus = nullptr;   // [k_total] the two perturbed copies of S (two forwards side by side)
   bool dual_rows = false;       // the activation buffers hold 2 * Mmax rows
@@ -1214,7 +1216,7 @@ szo_status run_loss_paired(szo_model* m, const int32_t* tokens, const int32_t* l
     for (int i = 0; i < n; ++i) {
       plans[i] = m->plans[t0 + i];
       sv[i] = Sv + m->offsets[t0 + i];
-      crec[i] = reinterpret_cast<const uint32_t*>(m->recs) + m->offsets[t0 + i];
+      crec[i] = m->crecs + m->offsets[t0 + i];
       zz[i] = z + m->offsets[t0 + i];
     }
     if (m->timing) {
@@ -1240,9 +1242,9 @@ szo_status run_loss_paired(szo_model* m, const int32_t* tokens, const int32_t* l
     void* const outs[1] = {out};
     return lin_group(layer, j, 1, x, outs);
   };
-  // (column, eps * z) of every sensitive entry, once for all linears of the step, in one launch (the
+  // (column, eps * z) of every record slot, once for all linears of the step, in one launch (the
   // record layout depends on K: the width of the column field travels with the column)
-  SZO_TRY(pack_cross_records_all(m->colk, m->csrc, z, eps, m->k_total, reinterpret_cast<uint32_t*>(m->recs), st));
+  SZO_TRY(pack_cross_records_all(m->colk, m->csrc, z, eps, m->k_total, m->crecs, st));
   embed_kernel<<<static_cast<unsigned>(M), 128, 0, st>>>(tokens, static_cast<const __nv_bfloat16*>(m->top.embed),
                                                         static_cast<const __nv_bfloat16*>(m->top.pos), S, d, c.vocab, m->h);
   SZO_CHECK_CUDA(cudaMemsetAsync(m->h + Mp * d, 0, static_cast<size_t>(M) * d * sizeof(float), st));   // both forwards embed alike
@@ -1668,15 +1670,14 @@ szo_status szo_model_create(szo_model_t** out, const szo_model_config* cfg, cons
   SZO_M_TRY(dev_alloc(m, &m->zkept, m->k_total * sizeof(float)));
   SZO_M_TRY(dev_alloc(m, &m->colk, m->k_total * sizeof(uint32_t)));
   SZO_M_TRY(dev_alloc(m, &m->csrc, m->k_total * sizeof(int32_t)));
+  SZO_M_TRY(dev_alloc(m, &m->crecs, m->k_total * sizeof(uint32_t)));
   if (m->k_total >= (int64_t(1) << 31)) return bail(fail(SZO_ERR_SHAPE, "more than 2^31 sparse entries"));
   for (size_t t = 0; t < m->plans.size(); ++t) {
     const szo_linear* p = m->plans[t];
     if (p->nnz) {
-      if (p->tc != nullptr && p->K <= (int64_t(1) << 18)) {
-        const szo_status cs = pack_cross_colk(p, static_cast<int32_t>(m->offsets[t]), m->colk + m->offsets[t],
-                                              m->csrc + m->offsets[t], st);
-        if (cs != SZO_OK) return bail(cs);
-      }
+      const szo_status cs = cross_copy_slots(p, static_cast<int32_t>(m->offsets[t]), m->colk + m->offsets[t],
+                                             m->csrc + m->offsets[t], st);
+      if (cs != SZO_OK) return bail(cs);
       offset_eid_kernel<<<blocks_for(p->nnz, 256), 256, 0, st>>>(p->bucket_eid, p->nnz, static_cast<int32_t>(m->offsets[t]),
                                                                m->geid + m->offsets[t]);
       cudaMemcpyAsync(m->gpos + m->offsets[t], p->bucket_pos, p->nnz * sizeof(uint16_t), cudaMemcpyDeviceToDevice, st);

@@ -45,6 +45,9 @@ PAIRED_LINEAR_CASES = [
     (300, 4160, 64, "f16", 257, 2e-3, True),
     (256, 256, 64, "bf16", 200, 5e-2, False),       # 13 entries per weight row
     (1280, 1024, 128, "bf16", 2600, 2e-3, False),   # more tiles than clusters: full rounds and a tail
+    (2080, 512, 128, "bf16", 2100, 1e-3, False),    # sparse product: slabs of 16 tokens, the last one ragged
+    (72, 16384, 128, "bf16", 24, 1e-3, False),      # ... of four tokens: K too wide for eight
+    (251, 512, 128, "bf16", 50, 1e-3, False),       # odd N: one weight row per thread in that product
 ]
 
 
