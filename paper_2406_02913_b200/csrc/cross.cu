@@ -294,6 +294,10 @@ __device__ __forceinline__ void stage_slab(const CrossArgs& a, int64_t m0, unsig
 // against 140 M) but tripled the shared-memory wavefronts (37 M, 22 M of them bank conflicts: all
 // 32 lanes now read random columns, and the tile is written at random rows): 265 us against 211 at
 // K = 4096, 3 % ahead at K = 11008; not kept.
+// The grid is 3.46 waves of equal blocks at M = 4096 (15 % of the SM cycles idle in the last one).  One
+// persistent block per SM with an equal, contiguous share of all (token group, row pair) items ran 151 us
+// against 161 us alone, but 14 us slower behind the tensor-core launch, whose SMs free up one by one; a last
+// quarter of the token groups in blocks a quarter the size was slower as well.  Not kept.
 template <int TM, int R, typename TY>
 __global__ void __launch_bounds__(TM == 16 ? 1024 : 512) pair_cross_kernel(const CrossArgs a) {
   using V = typename SlabVec<TM>::type;
