@@ -227,6 +227,25 @@ def attention_case(Bn, S, H, Hkv, hd, reps):
                       "tflops_causal": flops / (med * 1e-3) / 1e12}), flush=True)
 
 
+def attention_paired_case(Bn, S, H, Hkv, hd, reps):
+    """Causal attention of both forwards of a step as centre and half-difference rows (szo_attention_paired)."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(1)
+    M = Bn * S
+    row0 = B.paired_row0(M)
+
+    def rows(width):
+        t = torch.randn(row0 + M, width, generator=g, device="cuda")
+        t[row0:] *= 1e-3
+        return t.to(torch.bfloat16)
+
+    q, k, v = rows(H * hd), rows(Hkv * hd), rows(Hkv * hd)
+    med, best = time_call(lambda: B.szo_attention_paired(q, k, v, row0, Bn, S, H, Hkv, hd), reps)
+    flops = 4 * 4.0 * Bn * H * S * S * hd / 2          # causal; four products per term
+    print(json.dumps({"case": "attention_paired", "B": Bn, "S": S, "H": H, "Hkv": Hkv, "hd": hd, "ms_median": med,
+                      "ms_min": best, "tflops_causal": flops / (med * 1e-3) / 1e12}), flush=True)
+
+
 def paired_case(M, N, K, G, rho, reps):
     """One linear in the paired form (szo_linear_fwd_paired): M centre rows and M half-difference rows
     in one call: weight pass, SparseAdd scatter, one tensor-core launch over both kinds of rows, the
@@ -391,6 +410,8 @@ def main():
     elif a.what == "attention":
         attention_case(16, 256, 32, 32, 128, a.reps)
         attention_case(8, 512, 32, 8, 128, a.reps)
+        attention_paired_case(16, 256, 32, 32, 128, a.reps)
+        attention_paired_case(8, 512, 32, 8, 128, a.reps)
     else:
         for M in (16, 256, 8192):
             for mode in ("sparse_add", "spmm"):
