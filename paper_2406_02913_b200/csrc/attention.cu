@@ -239,11 +239,26 @@ flash_attn_bf16_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16*
 // tiles (twice the accumulators); the query tiles stay in shared memory.
 constexpr int kKT2 = 32;
 
-__device__ __forceinline__ float sinh_small(float a) {
+// 2^x by the hardware approximation alone (two units in the last place; exp2f adds a rescaling for results
+// below 2^-126, which a probability that is rounded to bf16 does not need)
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// cosh(a) and sinh(a).  The half-difference of a score is small against one (it is of the order of eps
+// times the score), so both come from their series, good to 1e-7 below |a| = 0.5; beyond that from e^a.
+__device__ __forceinline__ void cosh_sinh(float a, float* ch, float* sh) {
   const float a2 = a * a;
-  if (a2 < 0.25f) return a * (1.0f + a2 * (1.0f / 6.0f + a2 * (1.0f / 120.0f + a2 * (1.0f / 5040.0f + a2 * (1.0f / 362880.0f)))));
-  const float u = __expf(a);
-  return 0.5f * (u - __fdividef(1.0f, u));
+  if (a2 < 0.25f) {
+    *ch = 1.0f + a2 * (0.5f + a2 * (1.0f / 24.0f + a2 * (1.0f / 720.0f + a2 * (1.0f / 40320.0f))));
+    *sh = a * (1.0f + a2 * (1.0f / 6.0f + a2 * (1.0f / 120.0f + a2 * (1.0f / 5040.0f + a2 * (1.0f / 362880.0f)))));
+  } else {
+    const float u = __expf(a), r = __fdividef(1.0f, u);
+    *ch = 0.5f * (u + r);
+    *sh = 0.5f * (u - r);
+  }
 }
 
 template <int HD>
@@ -392,11 +407,11 @@ flash_attn_pair_bf16_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bflo
       float pc4[4], pd4[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const float e = exp2f(sc[i][j] * scale_log2e - msc[j >> 1]);
-        const float a = sd[i][j] * scale;
-        const float u = exp2f(sd[i][j] * scale_log2e);
-        pc4[j] = e * 0.5f * (u + __fdividef(1.0f, u));          // (fast reciprocal: the result is rounded to bf16)
-        pd4[j] = e * sinh_small(a);
+        const float e = ex2_approx(sc[i][j] * scale_log2e - msc[j >> 1]);
+        float ch, sh;
+        cosh_sinh(sd[i][j] * scale, &ch, &sh);
+        pc4[j] = e * ch;
+        pd4[j] = e * sh;
       }
       lc[0] += pc4[0] + pc4[1];
       lc[1] += pc4[2] + pc4[3];

@@ -299,7 +299,7 @@ __device__ __forceinline__ void stage_slab(const CrossArgs& a, int64_t m0, unsig
 // against 161 us alone, but 14 us slower behind the tensor-core launch, whose SMs free up one by one; a last
 // quarter of the token groups in blocks a quarter the size was slower as well.  Not kept.
 template <int TM, int R, typename TY>
-__global__ void __launch_bounds__(TM == 16 ? 1024 : 512) pair_cross_kernel(const CrossArgs a) {
+__global__ void __launch_bounds__(TM >= 8 ? 1024 : 512) pair_cross_kernel(const CrossArgs a) {
   using V = typename SlabVec<TM>::type;
   constexpr int kVecs = TM * 2 / static_cast<int>(sizeof(V));    // vectors per column
   constexpr int kTokPlane = TM / kVecs;
@@ -390,7 +390,7 @@ szo_status launch_cross(Kern kern, const char* name, const CrossArgs& ca, int TM
 
 template <int TM>
 szo_status launch_cross_tm(const CrossArgs& ca, int64_t max_N, bool even, bool f32, cudaStream_t st) {
-  constexpr int kThreads = TM == 16 ? 1024 : 512;
+  constexpr int kThreads = TM >= 8 ? 1024 : 512;
   const size_t smem = static_cast<size_t>(ca.K) * TM * sizeof(__nv_bfloat16) + 128;       // (+ 64 per plane)
   if (f32) return launch_cross(pair_cross_kernel<TM, 1, float>, "pair_cross_kernel", ca, TM, kThreads, smem, kThreads, max_N, st);
   if (even)
