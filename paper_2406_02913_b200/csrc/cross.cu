@@ -18,6 +18,10 @@
 // 26.0 M (an 8 x 16-byte ldmatrix phase meets the same bank conflicts as a quarter warp of 16-byte loads, and
 // the records pass through shared memory once more): 157 us against 163 us, and at K = 11008, where only eight
 // tokens fit and half of every mma is empty, 169 us against 146 us.  Not kept: 3 % for eps z rounded to bf16.
+// Nor was fma.rn.f32.bf16 (fp32 += bf16 * bf16 in one instruction, no unpacking of x, eps z as bf16): 78 M
+// instructions against 98 M and 151 us against 161 us alone (ncu), but 12 us SLOWER behind the tensor-core
+// launch at K = 4096 (6 us faster at K = 11008): the kernel waits on its record loads (long scoreboard
+// 6.1 cycles per issue), not on issue slots.
 #include <algorithm>
 #include <cstdlib>
 #include <vector>
