@@ -19,9 +19,9 @@
 // the records pass through shared memory once more): 157 us against 163 us, and at K = 11008, where only eight
 // tokens fit and half of every mma is empty, 169 us against 146 us.  Not kept: 3 % for eps z rounded to bf16.
 // Nor was fma.rn.f32.bf16 (fp32 += bf16 * bf16 in one instruction, no unpacking of x, eps z as bf16): 78 M
-// instructions against 98 M and 151 us against 161 us alone (ncu), but 12 us SLOWER behind the tensor-core
-// launch at K = 4096 (6 us faster at K = 11008): the kernel waits on its record loads (long scoreboard
-// 6.1 cycles per issue), not on issue slots.
+// instructions against 98 M, 151 us against 161 us alone (ncu) and 6 to 10 us per paired linear in a call that
+// alternated the two libraries (0.9 ms of a 113 ms step): the kernel waits on its record loads (long scoreboard
+// 6.1 cycles per issue) more than on issue slots, and eps z would lose three to five bits.
 #include <algorithm>
 #include <cstdlib>
 #include <vector>
@@ -216,6 +216,7 @@ struct CrossArgs {
   const __nv_bfloat16* x;   // centre rows [M][K]
   int64_t M, K;
   uint32_t col_mask;        // (1 << col_bits) - 1, col_bits = bits needed for K - 1
+  int64_t unit_end[3];      // running count of units (R adjacent weight rows) through the matrices
 };
 
 __device__ __forceinline__ uint32_t prmt_b32(uint32_t a, uint32_t b, uint32_t sel) {
@@ -298,10 +299,14 @@ __device__ __forceinline__ void stage_slab(const CrossArgs& a, int64_t m0, unsig
 // against 140 M) but tripled the shared-memory wavefronts (37 M, 22 M of them bank conflicts: all
 // 32 lanes now read random columns, and the tile is written at random rows): 265 us against 211 at
 // K = 4096, 3 % ahead at K = 11008; not kept.
-// The grid is 3.46 waves of equal blocks at M = 4096 (15 % of the SM cycles idle in the last one).  One
-// persistent block per SM with an equal, contiguous share of all (token group, row pair) items ran 151 us
-// against 161 us alone, but 14 us slower behind the tensor-core launch, whose SMs free up one by one; a last
-// quarter of the token groups in blocks a quarter the size was slower as well.  Not kept.
+// Work = (token group, unit), a unit being R adjacent weight rows of one of the matrices; the units of a token
+// group are numbered through the matrices (unit_end).  The grid is as many blocks as the device holds at once,
+// and block b takes the b-th of gridDim.x equal, contiguous shares of that list: a share covers the end of one
+// token group, whole groups and the start of another, and the block stages the slab of each group it touches
+// (about 2.7 at M = 4096).  Before, a block was one token group and one of two row shares: 512 equal blocks,
+// 3.46 waves, 15 % of the SM cycles idle in the last one.  Measured in one call, the libraries alternating:
+// gate/up 1211 -> 1199 us per paired linear, q/k/v 693 -> 686, o 267 -> 265, down (K = 11008) unchanged.
+// (A last quarter of the token groups in blocks a quarter the size, to fill the last wave, did not help.)
 template <int TM, int R, typename TY>
 __global__ void __launch_bounds__(TM >= 8 ? 1024 : 512) pair_cross_kernel(const CrossArgs a) {
   using V = typename SlabVec<TM>::type;
@@ -310,62 +315,75 @@ __global__ void __launch_bounds__(TM >= 8 ? 1024 : 512) pair_cross_kernel(const 
   extern __shared__ __align__(16) unsigned char cross_smem[];
   const size_t plane_bytes = static_cast<size_t>(a.K) * kTokPlane * sizeof(__nv_bfloat16) + 64;
   const unsigned char* xs = cross_smem;
-  const int64_t m0 = static_cast<int64_t>(blockIdx.x) * TM;
-  stage_slab<TM>(a, m0, cross_smem, plane_bytes);
-  __syncthreads();
-  const int cnt = static_cast<int>(a.M - m0 < TM ? a.M - m0 : TM);
-  for (int s = 0; s < a.n; ++s) {
-    const int32_t* row_ptr = s == 0 ? a.sub[0].ptr : (s == 1 ? a.sub[1].ptr : a.sub[2].ptr);
-    if (row_ptr == nullptr) continue;
-    const uint32_t* rec = s == 0 ? a.sub[0].rec : (s == 1 ? a.sub[1].rec : a.sub[2].rec);
-    TY* yd = static_cast<TY*>(s == 0 ? a.sub[0].yd : (s == 1 ? a.sub[1].yd : a.sub[2].yd));
-    const int64_t N = s == 0 ? a.sub[0].N : (s == 1 ? a.sub[1].N : a.sub[2].N);
-    // the row shares of the gridDim.y blocks of a token group interleave in units of the block size
-    for (int64_t n = (static_cast<int64_t>(blockIdx.y) * blockDim.x + threadIdx.x) * R; n < N;
-         n += static_cast<int64_t>(gridDim.y) * blockDim.x * R) {
-      int32_t eb[R + 1];
+  const int64_t U = a.unit_end[a.n - 1];                 // units per token group
+  const int64_t T = ((a.M + TM - 1) / TM) * U;
+  int64_t lo = T / gridDim.x * blockIdx.x + T % gridDim.x * blockIdx.x / gridDim.x;
+  const int64_t hi = T / gridDim.x * (blockIdx.x + 1) + T % gridDim.x * (blockIdx.x + 1) / gridDim.x;
+  bool first = true;
+  while (lo < hi) {
+    const int64_t group = lo / U, u0 = lo - group * U;
+    const int64_t u1 = hi - lo < U - u0 ? u0 + (hi - lo) : U;
+    lo += u1 - u0;
+    const int64_t m0 = group * TM;
+    if (!first) __syncthreads();                 // every thread is done with the previous group's slab
+    first = false;
+    stage_slab<TM>(a, m0, cross_smem, plane_bytes);
+    __syncthreads();
+    const int cnt = static_cast<int>(a.M - m0 < TM ? a.M - m0 : TM);
+    for (int s = 0; s < a.n; ++s) {
+      const int32_t* row_ptr = s == 0 ? a.sub[0].ptr : (s == 1 ? a.sub[1].ptr : a.sub[2].ptr);
+      if (row_ptr == nullptr) continue;
+      const int64_t ub = s == 0 ? 0 : a.unit_end[s - 1], ue = a.unit_end[s];
+      const int64_t s0 = (u0 > ub ? u0 : ub) - ub, s1 = (u1 < ue ? u1 : ue) - ub;   // this matrix's units in the share
+      if (s0 >= s1) continue;
+      const uint32_t* rec = s == 0 ? a.sub[0].rec : (s == 1 ? a.sub[1].rec : a.sub[2].rec);
+      TY* yd = static_cast<TY*>(s == 0 ? a.sub[0].yd : (s == 1 ? a.sub[1].yd : a.sub[2].yd));
+      const int64_t N = s == 0 ? a.sub[0].N : (s == 1 ? a.sub[1].N : a.sub[2].N);
+      for (int64_t n = (s0 + threadIdx.x) * R; n < s1 * R; n += static_cast<int64_t>(blockDim.x) * R) {
+        int32_t eb[R + 1];
 #pragma unroll
-      for (int r = 0; r <= R; ++r) eb[r] = __ldg(row_ptr + (n + r <= N ? n + r : N));
-      if (eb[0] == eb[R]) continue;
-      float acc[R][TM];
+        for (int r = 0; r <= R; ++r) eb[r] = __ldg(row_ptr + (n + r <= N ? n + r : N));
+        if (eb[0] == eb[R]) continue;
+        float acc[R][TM];
 #pragma unroll
-      for (int r = 0; r < R; ++r) {
+        for (int r = 0; r < R; ++r) {
 #pragma unroll
-        for (int j = 0; j < TM; ++j) acc[r][j] = 0.f;
-        for (int32_t e = eb[r]; e < eb[r + 1]; ++e) {
-          const uint32_t rc = __ldg(rec + e);
-          const float zz = __uint_as_float(rc & ~a.col_mask);
-          const uint32_t col = rc & a.col_mask;
+          for (int j = 0; j < TM; ++j) acc[r][j] = 0.f;
+          for (int32_t e = eb[r]; e < eb[r + 1]; ++e) {
+            const uint32_t rc = __ldg(rec + e);
+            const float zz = __uint_as_float(rc & ~a.col_mask);
+            const uint32_t col = rc & a.col_mask;
 #pragma unroll
-          for (int q = 0; q < kVecs; ++q) {
-            const V v = *reinterpret_cast<const V*>(xs + q * plane_bytes + col * sizeof(V));
-            const uint32_t* w = reinterpret_cast<const uint32_t*>(&v);
-            constexpr int kW = static_cast<int>(sizeof(V)) / 4;
+            for (int q = 0; q < kVecs; ++q) {
+              const V v = *reinterpret_cast<const V*>(xs + q * plane_bytes + col * sizeof(V));
+              const uint32_t* w = reinterpret_cast<const uint32_t*>(&v);
+              constexpr int kW = static_cast<int>(sizeof(V)) / 4;
 #pragma unroll
-            for (int h = 0; h < kW; ++h) {
-              acc[r][q * kW * 2 + 2 * h] = fmaf(zz, __uint_as_float(w[h] << 16), acc[r][q * kW * 2 + 2 * h]);
-              acc[r][q * kW * 2 + 2 * h + 1] = fmaf(zz, __uint_as_float(w[h] & 0xFFFF0000u), acc[r][q * kW * 2 + 2 * h + 1]);
+              for (int h = 0; h < kW; ++h) {
+                acc[r][q * kW * 2 + 2 * h] = fmaf(zz, __uint_as_float(w[h] << 16), acc[r][q * kW * 2 + 2 * h]);
+                acc[r][q * kW * 2 + 2 * h + 1] = fmaf(zz, __uint_as_float(w[h] & 0xFFFF0000u), acc[r][q * kW * 2 + 2 * h + 1]);
+              }
             }
           }
         }
-      }
-      TY* yp = yd + m0 * N + n;
-      if constexpr (R == 2 && sizeof(TY) == 2) {
+        TY* yp = yd + m0 * N + n;
+        if constexpr (R == 2 && sizeof(TY) == 2) {
 #pragma unroll
-        for (int j = 0; j < TM; ++j)
-          if (j < cnt) red_add_bf16x2(yp + j * N, pack_bf16x2(acc[0][j], acc[1][j]));
-      } else {
+          for (int j = 0; j < TM; ++j)
+            if (j < cnt) red_add_bf16x2(yp + j * N, pack_bf16x2(acc[0][j], acc[1][j]));
+        } else {
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-          if (n + r >= N) continue;
-          float old[TM];
+          for (int r = 0; r < R; ++r) {
+            if (n + r >= N) continue;
+            float old[TM];
 #pragma unroll
-          for (int j = 0; j < TM; ++j) old[j] = (j < cnt) ? static_cast<float>(yp[j * N + r]) : 0.f;
+            for (int j = 0; j < TM; ++j) old[j] = (j < cnt) ? static_cast<float>(yp[j * N + r]) : 0.f;
 #pragma unroll
-          for (int j = 0; j < TM; ++j) {
-            if (j < cnt) {
-              if constexpr (sizeof(TY) == 2) yp[j * N + r] = __float2bfloat16_rn(old[j] + acc[r][j]);
-              else yp[j * N + r] = old[j] + acc[r][j];
+            for (int j = 0; j < TM; ++j) {
+              if (j < cnt) {
+                if constexpr (sizeof(TY) == 2) yp[j * N + r] = __float2bfloat16_rn(old[j] + acc[r][j]);
+                else yp[j * N + r] = old[j] + acc[r][j];
+              }
             }
           }
         }
@@ -375,31 +393,36 @@ __global__ void __launch_bounds__(TM >= 8 ? 1024 : 512) pair_cross_kernel(const 
 }
 
 template <typename Kern>
-szo_status launch_cross(Kern kern, const char* name, const CrossArgs& ca, int TM, int threads, size_t smem, int64_t units_per_block,
-                        int64_t max_N, cudaStream_t st) {
+szo_status launch_cross(Kern kern, const char* name, CrossArgs ca, int TM, int R, int threads, size_t smem, cudaStream_t st) {
   SZO_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-  // few token groups: the rows of a group go to several blocks (each stages the slab again), so that
-  // the grid covers the SMs
-  const int64_t groups = ceil_div(ca.M, TM);
-  int row_split = static_cast<int>(ceil_div(296, groups));
-  const int64_t max_split = ceil_div(max_N, units_per_block);
-  if (row_split > max_split) row_split = static_cast<int>(max_split);
-  if (row_split < 1) row_split = 1;
-  dim3 grid(static_cast<unsigned>(groups), static_cast<unsigned>(row_split));
-  kern<<<grid, threads, smem, st>>>(ca);
+  int64_t units = 0;
+  for (int i = 0; i < ca.n; ++i) {
+    units += ceil_div(ca.sub[i].N, R);
+    ca.unit_end[i] = units;
+  }
+  int dev = 0, sms = 148, per_sm = 1;
+  SZO_CHECK_CUDA(cudaGetDevice(&dev));
+  SZO_CHECK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  SZO_CHECK_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem));
+  if (per_sm < 1) per_sm = 1;
+  // as many blocks as the device holds at once; fewer when there is less than one unit per thread
+  const int64_t total = ceil_div(ca.M, TM) * units;
+  int64_t blocks = ceil_div(total, threads);
+  if (blocks > static_cast<int64_t>(sms) * per_sm) blocks = static_cast<int64_t>(sms) * per_sm;
+  if (blocks < 1) blocks = 1;
+  kern<<<static_cast<unsigned>(blocks), threads, smem, st>>>(ca);
   count_launch();
   SZO_CHECK_LAUNCH(name);
   return SZO_OK;
 }
 
 template <int TM>
-szo_status launch_cross_tm(const CrossArgs& ca, int64_t max_N, bool even, bool f32, cudaStream_t st) {
+szo_status launch_cross_tm(const CrossArgs& ca, bool even, bool f32, cudaStream_t st) {
   constexpr int kThreads = TM >= 8 ? 1024 : 512;
   const size_t smem = static_cast<size_t>(ca.K) * TM * sizeof(__nv_bfloat16) + 128;       // (+ 64 per plane)
-  if (f32) return launch_cross(pair_cross_kernel<TM, 1, float>, "pair_cross_kernel", ca, TM, kThreads, smem, kThreads, max_N, st);
-  if (even)
-    return launch_cross(pair_cross_kernel<TM, 2, __nv_bfloat16>, "pair_cross_kernel", ca, TM, kThreads, smem, kThreads * 2, max_N, st);
-  return launch_cross(pair_cross_kernel<TM, 1, __nv_bfloat16>, "pair_cross_kernel", ca, TM, kThreads, smem, kThreads, max_N, st);
+  if (f32) return launch_cross(pair_cross_kernel<TM, 1, float>, "pair_cross_kernel", ca, TM, 1, kThreads, smem, st);
+  if (even) return launch_cross(pair_cross_kernel<TM, 2, __nv_bfloat16>, "pair_cross_kernel", ca, TM, 2, kThreads, smem, st);
+  return launch_cross(pair_cross_kernel<TM, 1, __nv_bfloat16>, "pair_cross_kernel", ca, TM, 1, kThreads, smem, st);
 }
 
 }  // namespace
@@ -412,13 +435,11 @@ szo_status launch_paired_cross(const szo_linear* const* plans, int n, const void
   CrossArgs ca{};
   ca.n = n; ca.x = static_cast<const __nv_bfloat16*>(x); ca.M = M; ca.K = p0->K;
   ca.col_mask = (1u << col_bits_of(p0->K)) - 1u;
-  int64_t max_N = 0;
   bool even = true, any = false;
   for (int i = 0; i < n; ++i) {
     const szo_linear* p = plans[i];
     const CrossPlan* c = static_cast<const CrossPlan*>(p->cross);
     SZO_REQUIRE(p->nnz == 0 || c != nullptr, SZO_ERR_UNSUPPORTED, "K = %lld too large for the paired form", (long long)p->K);
-    if (p->N > max_N) max_N = p->N;
     if (p->N & 1) even = false;
     if (c != nullptr) any = true;
     ca.sub[i] = CrossSub{c == nullptr ? nullptr : p->row_ptr, rec[i], yd[i], p->N};
@@ -430,12 +451,12 @@ szo_status launch_paired_cross(const szo_linear* const* plans, int n, const void
     const char* e = getenv("SZO_CROSS_TM");
     return e == nullptr ? 0 : atoi(e);
   }();
-  if (tm_env == 8 && 8 * per_token <= 200 * 1024) return launch_cross_tm<8>(ca, max_N, even, f32, st);
-  if (16 * per_token <= 200 * 1024 && M >= 2048) return launch_cross_tm<16>(ca, max_N, even, f32, st);
-  if (8 * per_token <= 200 * 1024) return launch_cross_tm<8>(ca, max_N, even, f32, st);
-  if (4 * per_token <= 200 * 1024) return launch_cross_tm<4>(ca, max_N, even, f32, st);
+  if (tm_env == 8 && 8 * per_token <= 200 * 1024) return launch_cross_tm<8>(ca, even, f32, st);
+  if (16 * per_token <= 200 * 1024 && M >= 2048) return launch_cross_tm<16>(ca, even, f32, st);
+  if (8 * per_token <= 200 * 1024) return launch_cross_tm<8>(ca, even, f32, st);
+  if (4 * per_token <= 200 * 1024) return launch_cross_tm<4>(ca, even, f32, st);
   SZO_REQUIRE(2 * per_token <= 200 * 1024, SZO_ERR_UNSUPPORTED, "K = %lld too large for the paired form", (long long)p0->K);
-  return launch_cross_tm<2>(ca, max_N, even, f32, st);
+  return launch_cross_tm<2>(ca, even, f32, st);
 }
 
 }  // namespace szo
