@@ -307,6 +307,10 @@ __device__ __forceinline__ void stage_slab(const CrossArgs& a, int64_t m0, unsig
 // 3.46 waves, 15 % of the SM cycles idle in the last one.  Measured in one call, the libraries alternating:
 // gate/up 1211 -> 1199 us per paired linear, q/k/v 693 -> 686, o 267 -> 265, down (K = 11008) unchanged.
 // (A last quarter of the token groups in blocks a quarter the size, to fill the last wave, did not help.)
+// Wide K (a slab of 16 tokens does not fit beyond K = 6400, of 8 beyond 12800): staging the columns in ranges,
+// 16 tokens each, was 6 % faster for a whole paired linear at K = 20480 and 1.5 % at K = 11008, but then an
+// element of y receives one addend per range from blocks that run at the same time: the sum of roundings
+// depends on their order.  Not done: every element gets exactly one addend per launch.
 template <int TM, int R, typename TY>
 __global__ void __launch_bounds__(TM >= 8 ? 1024 : 512) pair_cross_kernel(const CrossArgs a) {
   using V = typename SlabVec<TM>::type;
