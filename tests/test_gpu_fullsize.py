@@ -93,6 +93,65 @@ def test_full_size_linear_sampled_outputs(B, N, K, G, rho, bias, mode):
 
 
 @pytest.mark.parametrize("N,K,bias", [
+    (11008, 4096, False), (4096, 11008, False),      # Llama-2-7B MLP shapes: slabs of 16 and of 8 tokens in the sparse product
+    (5120, 20480, True),                             # OPT-13B fc2: slabs of 4 tokens, bias on the centre rows only
+])
+def test_full_size_paired_linear_sampled_outputs(B, N, K, bias):
+    """szo_linear_fwd_paired at the bench's token count (4096 centre rows and 4096 half-difference rows), int4 G=128,
+    0.1 % mask: sampled outputs of both kinds of rows against the fp64 definition
+    yc = xc W^T + b, yd = xd W^T + eps xc Zbar^T with W = Dequantize(Q) + S (Definition 4 on the decomposition)."""
+    M, G, eps = 4096, 128, 1e-3
+    g = torch.Generator(device="cuda")
+    g.manual_seed(N * 3 + K)
+    codes = torch.randint(0, 256, (N, K // 2), generator=g, device="cuda", dtype=torch.uint8)
+    sc = (0.004 + 0.002 * torch.rand(N, K // G, generator=g, device="cuda")).to(torch.bfloat16)
+    ze = (-7.5 * sc.float()).to(torch.bfloat16)
+    nnz = int(1e-3 * N * K)
+    idx_np = wl.sorted_random_indices(N * K, nnz, seed=N + K + 1)
+    idx = torch.from_numpy(idx_np).cuda()
+    S = (torch.randn(nnz, generator=g, device="cuda") * 0.02).contiguous()
+    z = torch.from_numpy(so.gaussian(99, 7, idx_np)).cuda()
+    b = (torch.randn(N, generator=g, device="cuda") * 0.02) if bias else None
+    row0 = B.paired_row0(M)
+    x = torch.zeros(row0 + M, K, device="cuda", dtype=torch.bfloat16)
+    x[:M] = torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16)
+    x[row0:] = (2e-3 * torch.randn(M, K, generator=g, device="cuda")).to(torch.bfloat16)
+    plan = B.Linear(N, K, G, codes, sc, ze, "bf16", idx, b)
+    y = plan.fwd_paired(x, M, S, z, eps, torch.bfloat16)
+    torch.cuda.synchronize()
+    assert B.device_status() == 0
+
+    r = wl.rng(6, wl.PURPOSE_INDICES, N + K)
+    rows = np.unique(np.concatenate([r.integers(0, N, 24), [0, 1, 2047, 2048, N - 2, N - 1]]))
+    toks = np.unique(np.concatenate([r.integers(0, M, 24), [0, 15, 16, M - 17, M - 1]]))
+    deq = so.dequantize(codes[rows].cpu().numpy(), _bf16_bits(sc[rows]), _bf16_bits(ze[rows]), G, "bf16")     # [rows, K] fp64
+    zbar = np.zeros_like(deq)
+    S_h, z_h = S.cpu().numpy().astype(np.float64), z.cpu().numpy().astype(np.float64)
+    for i, n in enumerate(rows):
+        lo, hi = np.searchsorted(idx_np, [n * K, (n + 1) * K])
+        np.add.at(deq[i], idx_np[lo:hi] - n * K, S_h[lo:hi])
+        np.add.at(zbar[i], idx_np[lo:hi] - n * K, z_h[lo:hi])
+    xc = x[:M][toks].float().cpu().numpy().astype(np.float64)
+    xd = x[row0:][toks].float().cpu().numpy().astype(np.float64)
+    ref_c = xc @ deq.T + (b[rows].cpu().numpy().astype(np.float64)[None, :] if bias else 0.0)
+    ref_d = xd @ deq.T + eps * (xc @ zbar.T)
+    got_c = y[:M][toks][:, rows].float().cpu().numpy().astype(np.float64)
+    got_d = y[row0:][toks][:, rows].float().cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(got_c - ref_c)) <= 2e-2 * np.max(np.abs(ref_c))
+    assert np.max(np.abs(got_d - ref_d)) <= 2e-2 * np.max(np.abs(ref_d))        # each kind of row against its own size
+    # the sparse product alone: with xd = 0 the half-difference rows are eps xc Zbar^T
+    x[row0:] = 0
+    y0 = plan.fwd_paired(x, M, S, z, eps, torch.bfloat16)
+    ref0 = eps * (xc @ zbar.T)
+    got0 = y0[row0:][toks][:, rows].float().cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(got0 - ref0)) <= 2.0 ** -7 * np.max(np.abs(ref0))      # two bf16 roundings: addend, stored sum
+    assert torch.isfinite(y).all()
+    y1 = plan.fwd_paired(x, M, S, z, eps, torch.bfloat16)
+    assert torch.equal(y0, y1)                                                 # bitwise repeatable
+    plan.close()
+
+
+@pytest.mark.parametrize("N,K,bias", [
     (4096, 4096, False), (11008, 4096, False), (4096, 11008, False),      # Llama-2-7B shapes
     (20480, 5120, True), (5120, 20480, True),                             # OPT-13B MLP shapes, biases
 ])
