@@ -456,7 +456,9 @@ szo_status launch_paired_cross(const szo_linear* const* plans, int n, const void
     return e == nullptr ? 0 : atoi(e);
   }();
   if (tm_env == 8 && 8 * per_token <= 200 * 1024) return launch_cross_tm<8>(ca, even, f32, st);
-  if (16 * per_token <= 200 * 1024 && M >= 2048) return launch_cross_tm<16>(ca, even, f32, st);
+  // (16 tokens per slab pay from about 1300 tokens on: 0.493 -> 0.485 ms per paired gate/up linear at M = 1536, equal at
+  // 1024, 0.223 -> 0.227 ms at 512)
+  if (16 * per_token <= 200 * 1024 && ((M >= 1280 && tm_env != 8) || tm_env == 16)) return launch_cross_tm<16>(ca, even, f32, st);
   if (8 * per_token <= 200 * 1024) return launch_cross_tm<8>(ca, even, f32, st);
   if (4 * per_token <= 200 * 1024) return launch_cross_tm<4>(ca, even, f32, st);
   SZO_REQUIRE(2 * per_token <= 200 * 1024, SZO_ERR_UNSUPPORTED, "K = %lld too large for the paired form", (long long)p0->K);
