@@ -1261,9 +1261,14 @@ szo_status run_loss_paired(szo_model* m, const int32_t* tokens, const int32_t* l
     }
     if (!opt) {        // the rotation is linear: the same kernel on both parts
       const int64_t n_vec = M * (H + Hkv) * ((hd / 2) / Vec16<T>::kN);
-      rope_kernel<T><<<blocks_for(n_vec, 256), 256, 0, st>>>(q, k, m->rope_tab, M, S, H, Hkv, hd);
-      rope_kernel<T><<<blocks_for(n_vec, 256), 256, 0, st>>>(q + Mp * d, k + Mp * dkv, m->rope_tab, M, S, H, Hkv, hd);
-      count_launch(2);
+      if (Mp == M) {   // no gap between the two kinds of rows: one launch (a row's position is its index modulo S)
+        rope_kernel<T><<<blocks_for(2 * n_vec, 256), 256, 0, st>>>(q, k, m->rope_tab, 2 * M, S, H, Hkv, hd);
+        count_launch();
+      } else {
+        rope_kernel<T><<<blocks_for(n_vec, 256), 256, 0, st>>>(q, k, m->rope_tab, M, S, H, Hkv, hd);
+        rope_kernel<T><<<blocks_for(n_vec, 256), 256, 0, st>>>(q + Mp * d, k + Mp * dkv, m->rope_tab, M, S, H, Hkv, hd);
+        count_launch(2);
+      }
     }
     SZO_TRY(launch_flash_attention_pair_bf16(q, k, v, o, Mp, B, S, H, Hkv, hd, st));
     SZO_TRY(lin(l, 3, o, y));
