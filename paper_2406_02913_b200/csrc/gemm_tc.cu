@@ -580,13 +580,18 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
     n_tiles += sb.n_tiles;
   }
   P.n_tiles = n_tiles;
-  // bands of token tiles that fit L2 with room to spare (about 32 MB of tokens per band)
+  // bands of token tiles that fit L2 with room to spare: at most 48 MB of tokens per band, and bands of equal
+  // height (32 token tiles: two bands of 16 at K = 4096, four of 8 at K = 11008; measured per paired linear,
+  // 8192 rows: K = 4096, N = 22016: 8 / 12 / 16 / 24 tiles per band 1.265 / 1.240 / 1.226 / 1.251 ms, no bands
+  // 1.31 ms; K = 11008, N = 4096: 4 / 5 / 8 / 16 tiles 0.665 / 0.669 / 0.653 / 0.655 ms, no bands 0.689 ms)
   {
     static const int band_env = [] {
       const char* e = getenv("SZO_TILE_BAND");
       return e == nullptr ? -1 : atoi(e);
     }();
-    int band = static_cast<int>((32ll << 20) / (256 * p0->K * 2));
+    const int64_t band_max = (48ll << 20) / (256 * p0->K * 2);
+    int band = 0;
+    if (band_max >= 1 && P.m_tiles > band_max) band = static_cast<int>(ceil_div(P.m_tiles, ceil_div(P.m_tiles, band_max)));
     if (band_env >= 0) band = band_env;
     P.m_band = (band > 0 && P.m_tiles > band) ? band : 0;
   }

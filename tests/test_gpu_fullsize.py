@@ -384,7 +384,11 @@ def test_two_opt_width_layers_relu_in_the_epilogue(B):
     # fp32 sums run in another order: the losses agree to ~1e-9, not bit for bit
     for i in (0, 1):
         assert abs(float(out_dual[i]) - float(out_seq[i])) <= 1e-7 * abs(float(out_seq[i]))
-    assert float((S_dual - S_seq).abs().max()) <= 4e-9            # at most an fp32 ulp of values ~0.02
+    # the update is lr * g * z: the two g differ as the losses do (divided by 2 eps), |z| stays below 6, and the
+    # result is rounded to fp32 once more
+    dg = abs(float(out_dual[2]) - float(out_seq[2]))
+    assert dg <= 2e-7 * abs(float(out_seq[0])) / 2e-3
+    assert bool(((S_dual - S_seq).abs() <= 1e-6 * 6.0 * dg + 1.2e-7 * S_seq.abs() + 1e-12).all())
     fp, fm = float(out_dual[0]), float(out_dual[1])
     assert abs(0.5 * (fp + fm) - f_seq) <= 1e-3 * abs(f_seq)
     for m in (m_dual, m_seq, m_ref):
