@@ -285,6 +285,8 @@ flash_attn_pair_bf16_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bflo
                             int H, int Hkv, float scale, float scale_log2e) {
   constexpr int LDS = HD + 8;
   extern __shared__ __align__(16) unsigned char smem_attn[];
+  chain_release();
+  chain_wait();
   __nv_bfloat16* sQc = reinterpret_cast<__nv_bfloat16*>(smem_attn);
   __nv_bfloat16* sQd = sQc + kQT * LDS;
   __nv_bfloat16* sKV = sQd + kQT * LDS;          // two stages of (Kc, Kd, Vc, Vd), kKT2 rows each
@@ -527,11 +529,13 @@ szo_status launch_flash_attention_pair_bf16(const void* q, const void* k, const 
   if (hd == 64) {
     SZO_CHECK_CUDA(cudaFuncSetAttribute(flash_attn_pair_bf16_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(smem)));
-    flash_attn_pair_bf16_kernel<64><<<grid, 128, smem, st>>>(qb, kb, vb, ob, row0, S, H, Hkv, scale, scale_log2e);
+    SZO_CHECK_CUDA(launch_maybe_chained(flash_attn_pair_bf16_kernel<64>, grid, dim3(128), smem, st, step_chained(), qb, kb, vb, ob, row0,
+                                        S, H, Hkv, scale, scale_log2e));
   } else {
     SZO_CHECK_CUDA(cudaFuncSetAttribute(flash_attn_pair_bf16_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(smem)));
-    flash_attn_pair_bf16_kernel<128><<<grid, 128, smem, st>>>(qb, kb, vb, ob, row0, S, H, Hkv, scale, scale_log2e);
+    SZO_CHECK_CUDA(launch_maybe_chained(flash_attn_pair_bf16_kernel<128>, grid, dim3(128), smem, st, step_chained(), qb, kb, vb, ob, row0,
+                                        S, H, Hkv, scale, scale_log2e));
   }
   count_launch();
   SZO_CHECK_LAUNCH("flash_attn_pair_bf16_kernel");

@@ -1,6 +1,7 @@
 // Shared host-side helpers of the szo library: error reporting, argument checks, and the
 // declarations of the internal launchers that the model driver calls directly.
 #pragma once
+#include <cstdlib>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -79,6 +80,17 @@ inline cudaError_t launch_maybe_chained(void (*kern)(KArgs...), dim3 grid, dim3 
   cfg.attrs = chained ? attr : nullptr;
   cfg.numAttrs = chained ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
+// The kernels of a training step that follow one another on a stream are launched as a chain too (each starts
+// with chain_release(); chain_wait();, so only its placement on the SMs overlaps the predecessor's last
+// blocks).  SZO_STEP_CHAIN=0: ordinary launches (A/B measurement).
+inline bool step_chained() {
+  static const bool v = [] {
+    const char* e = getenv("SZO_STEP_CHAIN");
+    return !(e != nullptr && e[0] == '0');
+  }();
+  return v;
 }
 
 // Launch counter used by the model to report how many kernels one step enqueued.

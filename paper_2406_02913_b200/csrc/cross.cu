@@ -317,6 +317,8 @@ __global__ void __launch_bounds__(TM >= 8 ? 1024 : 512) pair_cross_kernel(const 
   constexpr int kVecs = TM * 2 / static_cast<int>(sizeof(V));    // vectors per column
   constexpr int kTokPlane = TM / kVecs;
   extern __shared__ __align__(16) unsigned char cross_smem[];
+  chain_release();
+  chain_wait();
   const size_t plane_bytes = static_cast<size_t>(a.K) * kTokPlane * sizeof(__nv_bfloat16) + 64;
   const unsigned char* xs = cross_smem;
   const int64_t U = a.unit_end[a.n - 1];                 // units per token group
@@ -414,7 +416,7 @@ szo_status launch_cross(Kern kern, const char* name, CrossArgs ca, int TM, int R
   int64_t blocks = ceil_div(total, threads);
   if (blocks > static_cast<int64_t>(sms) * per_sm) blocks = static_cast<int64_t>(sms) * per_sm;
   if (blocks < 1) blocks = 1;
-  kern<<<static_cast<unsigned>(blocks), threads, smem, st>>>(ca);
+  SZO_CHECK_CUDA(launch_maybe_chained(kern, dim3(static_cast<unsigned>(blocks)), dim3(threads), smem, st, step_chained(), ca));
   count_launch();
   SZO_CHECK_LAUNCH(name);
   return SZO_OK;

@@ -269,6 +269,8 @@ struct MatArgs {
 // load, so the 32 look-ups of an instruction hit one 32-byte line).
 template <int kKind>
 __global__ void materialise_kernel(const MatArgs a) {
+  chain_release();
+  chain_wait();          // (the scratch it overwrites is what the previous tensor-core launch read)
   int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i >= a.sub[a.n - 1].words_end) return;
   int s = 0;
@@ -323,6 +325,8 @@ __global__ void materialise_kernel(const MatArgs a) {
 // With two sets of sparse values for one weight pass (the two perturbed forwards of a ZO step) the
 // dense values at the masked positions are kept aside by the first scatter and reused by the second.
 __global__ void scatter_add_bf16_kernel(const MatArgs a) {
+  chain_release();
+  chain_wait();
   int64_t e = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (e >= a.sub[a.n - 1].nnz_end) return;
   int s = 0;
@@ -544,9 +548,8 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
     }
   } else if (!resident) {
     const unsigned blocks = static_cast<unsigned>(ceil_div(words, 256));
-    if (p0->G < 0) materialise_kernel<2><<<blocks, 256, 0, st>>>(a);
-    else if (p0->sz_dtype == SZO_BF16) materialise_kernel<1><<<blocks, 256, 0, st>>>(a);
-    else materialise_kernel<0><<<blocks, 256, 0, st>>>(a);
+    auto mk = p0->G < 0 ? materialise_kernel<2> : (p0->sz_dtype == SZO_BF16 ? materialise_kernel<1> : materialise_kernel<0>);
+    SZO_CHECK_CUDA(launch_maybe_chained(mk, dim3(blocks), dim3(256), 0, st, step_chained(), a));
     count_launch();
     SZO_CHECK_LAUNCH("materialise_kernel");
   }
@@ -626,7 +629,8 @@ szo_status linear_fwd_tc_materialised(const szo_linear* const* plans, int n, con
       a.scatter_mode = resident ? 2 : (n_sets == 1 ? 0 : set + 1);
       if (set == 1)
         for (int i = 0; i < n; ++i) a.sub[i].S = S_second[i];
-      scatter_add_bf16_kernel<<<static_cast<unsigned>(ceil_div(nnz, 256)), 256, 0, st>>>(a);
+      SZO_CHECK_CUDA(launch_maybe_chained(scatter_add_bf16_kernel, dim3(static_cast<unsigned>(ceil_div(nnz, 256))), dim3(256), 0, st,
+                                          step_chained(), a));
       count_launch();
     }
     CUtensorMap mx;

@@ -140,6 +140,8 @@ __global__ void rope_table_kernel(int max_seq, int half, double base, float2* __
 template <typename T>
 __global__ void rope_kernel(T* __restrict__ q, T* __restrict__ k, const float2* __restrict__ tab, int64_t M, int S,
                             int H, int Hkv, int hd, int pos0 = 0, const int32_t* __restrict__ pos_dev = nullptr) {
+  chain_release();
+  chain_wait();
   if (pos_dev != nullptr) pos0 = *pos_dev;
   constexpr int kN = 16 / sizeof(T);
   const int half = hd >> 1, vec_per_head = half / kN;
@@ -654,6 +656,8 @@ add_norm_pair_kernel(float* __restrict__ h, const T* __restrict__ y, int64_t row
                      const float* __restrict__ beta, int d, float eps, bool layer_norm, int64_t row_stride,
                      int64_t row_offset, TO* __restrict__ out, int64_t out_row0) {
   __shared__ float2 scratch[32];
+  chain_release();
+  chain_wait();
   const int64_t m = static_cast<int64_t>(blockIdx.x) * row_stride + row_offset;
   float* xc = h + m * d;
   float* xd = h + (row0 + m) * d;
@@ -749,6 +753,8 @@ add_norm_pair_kernel(float* __restrict__ h, const T* __restrict__ y, int64_t row
 // silu: tc = gc sc + gd sd, td = gc sd + gd sc;  out_c = tc uc + td ud,  out_d = tc ud + td uc.
 template <typename T>
 __global__ void silu_mul_pair_kernel(T* __restrict__ gate, const T* __restrict__ up, int64_t n, int64_t off_d) {
+  chain_release();
+  chain_wait();
   constexpr int kN = Vec16<T>::kN;
   const int64_t i = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) * kN;
   if (i >= n) return;
@@ -1252,8 +1258,8 @@ szo_status run_loss_paired(szo_model* m, const int32_t* tokens, const int32_t* l
   const T* pending = nullptr;
   for (int l = 0; l < c.n_layers; ++l) {
     const szo_layer_weights& L = m->layers[l];
-    add_norm_pair<<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, pending, Mp, L.attn_norm_g, L.attn_norm_b, d,
-                                                                     c.norm_eps, opt, 1, 0, a, Mp);
+    SZO_CHECK_CUDA(launch_maybe_chained(add_norm_pair, dim3(static_cast<unsigned>(M)), dim3(256), 0, st, step_chained(), m->h, pending,
+                                        Mp, L.attn_norm_g, L.attn_norm_b, d, c.norm_eps, opt, 1, 0, a, Mp));
     count_launch();
     {
       void* const qkv[3] = {q, k, v};
@@ -1262,7 +1268,8 @@ szo_status run_loss_paired(szo_model* m, const int32_t* tokens, const int32_t* l
     if (!opt) {        // the rotation is linear: the same kernel on both parts
       const int64_t n_vec = M * (H + Hkv) * ((hd / 2) / Vec16<T>::kN);
       if (Mp == M) {   // no gap between the two kinds of rows: one launch (a row's position is its index modulo S)
-        rope_kernel<T><<<blocks_for(2 * n_vec, 256), 256, 0, st>>>(q, k, m->rope_tab, 2 * M, S, H, Hkv, hd);
+        SZO_CHECK_CUDA(launch_maybe_chained(rope_kernel<T>, dim3(blocks_for(2 * n_vec, 256)), dim3(256), 0, st, step_chained(), q, k,
+                                            m->rope_tab, 2 * M, S, H, Hkv, hd, 0, nullptr));
         count_launch();
       } else {
         rope_kernel<T><<<blocks_for(n_vec, 256), 256, 0, st>>>(q, k, m->rope_tab, M, S, H, Hkv, hd);
@@ -1272,13 +1279,14 @@ szo_status run_loss_paired(szo_model* m, const int32_t* tokens, const int32_t* l
     }
     SZO_TRY(launch_flash_attention_pair_bf16(q, k, v, o, Mp, B, S, H, Hkv, hd, st));
     SZO_TRY(lin(l, 3, o, y));
-    add_norm_pair<<<static_cast<unsigned>(M), 256, 0, st>>>(m->h, y, Mp, L.mlp_norm_g, L.mlp_norm_b, d, c.norm_eps,
-                                                                     opt, 1, 0, a, Mp);
+    SZO_CHECK_CUDA(launch_maybe_chained(add_norm_pair, dim3(static_cast<unsigned>(M)), dim3(256), 0, st, step_chained(), m->h, y, Mp,
+                                        L.mlp_norm_g, L.mlp_norm_b, d, c.norm_eps, opt, 1, 0, a, Mp));
     count_launch();
     if (!opt) {
       void* const gu[2] = {gate, up};
       SZO_TRY(lin_group(l, 4, 2, a, gu));
-      silu_mul_pair_kernel<T><<<blocks_for(M * ff / Vec16<T>::kN, 256), 256, 0, st>>>(gate, up, M * ff, Mp * ff);
+      SZO_CHECK_CUDA(launch_maybe_chained(silu_mul_pair_kernel<T>, dim3(blocks_for(M * ff / Vec16<T>::kN, 256)), dim3(256), 0, st,
+                                          step_chained(), gate, up, M * ff, Mp * ff));
       count_launch();
       SZO_TRY(lin(l, 6, gate, y));
     } else {
