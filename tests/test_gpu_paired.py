@@ -221,3 +221,42 @@ def test_paired_step_moves_S_like_the_oracle(B):
     assert np.linalg.norm(err) <= 2 * G_RMS_TOL["llama"] * np.linalg.norm(moved)
     assert B.device_status() == 0
     m.close()
+
+
+_STEP_SWITCH_SCRIPT = r"""
+import sys, numpy as np, torch
+from paper_2406_02913_b200 import binding as B, workloads as wl
+shape = dict(wl.MODEL_SHAPES["llama2_7b"], n_layers=2)
+tensors, S_all = wl.device_decoder_tensors(shape, seed=4)
+Bn, S = 5, 256                                   # 1280 tokens: slabs of 16 tokens in the sparse product
+m = B.Model(shape, wl.linear_names(shape), tensors, S_all, act_dtype=B.SZO_BF16, linear_mode=B.MODE_PAIRED,
+            loss_kind=B.LOSS_CLS2, max_batch=Bn, max_seq=S)
+toks = torch.from_numpy(wl.token_batch(shape["vocab"], Bn, S, 4, wl.PURPOSE_TRAIN_BATCH, 0)).cuda()
+labs = torch.from_numpy(wl.binary_labels(Bn, 4, 0)).cuda()
+cand = torch.tensor([9906, 13], dtype=torch.int32, device="cuda")
+rows = [m.zo_step(toks, 77, step, 1e-3, 1e-4, labs, cand).double().cpu().numpy().copy() for step in range(3)]
+assert B.device_status() == 0
+np.savez(sys.argv[1], out=np.array(rows), S=S_all.cpu().numpy())
+"""
+
+
+def test_switches_of_the_training_step_leave_the_bits_alone(tmp_path):
+    """Three paired steps at the Llama-2-7B width (two layers) with the step's kernels launched as a chain
+    (the default), with ordinary launches, and with the other slab height of the sparse product: a chained
+    launch changes when a kernel starts, not what it computes, and a thread of the sparse product walks the same
+    entries in the same order whatever the number of tokens per slab, so losses, g and the updated sparse
+    values must be the same bits.  The switches are read once per process: one child process per setting."""
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = {}
+    for name, extra in (("default", {}), ("no_chain", {"SZO_STEP_CHAIN": "0"}), ("slab8", {"SZO_CROSS_TM": "8"})):
+        out = str(tmp_path / (name + ".npz"))
+        r = subprocess.run([sys.executable, "-c", _STEP_SWITCH_SCRIPT, out], cwd=root, env=dict(os.environ, **extra),
+                           capture_output=True, text=True, timeout=900)
+        assert r.returncode == 0, name + ": " + r.stdout[-2000:] + r.stderr[-2000:]
+        res[name] = np.load(out)
+    assert np.isfinite(res["default"]["out"]).all()
+    for other in ("no_chain", "slab8"):
+        assert np.array_equal(res["default"]["out"], res[other]["out"]), other
+        assert np.array_equal(res["default"]["S"], res[other]["S"]), other
