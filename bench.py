@@ -40,7 +40,7 @@ EPS, LR, SEED = 1e-3, 1e-6, 1234
 # ncu summary that holds the DRAM traffic of one launch of the dominant kernel, and the sources it was taken from
 TRAFFIC_PROFILE = os.path.join(ROOT, "profiles", "szo_linear_tc2_kernel_paired_gate_up_M8192.md")
 KERNEL_SOURCES = [os.path.join(ROOT, "paper_2406_02913_b200", "csrc", f) for f in ("gemm_tc2.cu", "tc_common.cuh")]
-ORACLE_TOKENS_SAMPLE, ORACLE_K_SAMPLE = 16, 200_000
+ORACLE_TOKENS_SAMPLE, ORACLE_K_SAMPLE = 4096, 6_476_005
 
 
 def measured_peaks():
